@@ -1,0 +1,152 @@
+"""ctypes front end of the CPU oracle (`sq_oracle.cpp`).  TEST INFRASTRUCTURE ONLY.
+
+Only the test suite, the smoke check and the benchmark's CPU-baseline leg may
+import this package; the CUDA library and its Python binding never do.  All
+arrays are numpy; bf16 tensors travel as uint16 bit patterns.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+from dataclasses import dataclass
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "sq_oracle.cpp")
+_LIB = os.path.join(_HERE, "libsq_oracle.so")
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with g++ (-O2, no fast-math, OpenMP over rows)."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        tmp = _LIB + f".tmp{os.getpid()}"
+        subprocess.check_call(["g++", "-O2", "-fopenmp", "-ffp-contract=off", "-shared", "-fPIC",
+                               "-o", tmp, _SRC])
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        _lib = ctypes.CDLL(build())
+        _lib.sqo_equivalent_bits.restype = ctypes.c_double
+        _lib.sqo_equivalent_bits.argtypes = [ctypes.c_double, ctypes.c_double, ctypes.c_double, ctypes.c_int]
+        _lib.sqo_num_threads.restype = ctypes.c_int
+        _lib.sqo_gemm.restype = ctypes.c_int
+    return _lib
+
+
+def _p(a):
+    if a is None:
+        return ctypes.c_void_p(0)
+    assert a.flags["C_CONTIGUOUS"]
+    return ctypes.c_void_p(a.ctypes.data)
+
+
+def _l(v):
+    return ctypes.c_long(int(v))
+
+
+def num_threads() -> int:
+    return int(_load().sqo_num_threads())
+
+
+def equivalent_bits(h_high: float, h_low: float, s: float, on_weights: bool) -> float:
+    return float(_load().sqo_equivalent_bits(h_high, h_low, s, int(on_weights)))
+
+
+@dataclass
+class Encoded:
+    dq4: np.ndarray      # uint8 [M, K/2]
+    vals: np.ndarray     # int8  [M, G, k]
+    idx: np.ndarray | None  # uint8 [M, G, k]; None for static positions
+    s_hi: np.ndarray     # float32 [M]
+    s_lo: np.ndarray     # float32 [M]
+    shift: np.ndarray    # uint8 [M]
+
+
+@dataclass
+class Weights:
+    wq4: np.ndarray      # uint8 [N, K/2]
+    s_w: np.ndarray      # float32 [N]
+    colsum: np.ndarray   # int32 [N]
+    w_sparse: np.ndarray | None  # int8 [N, G*k]; None for dynamic positions
+    wq: np.ndarray       # int8 [N, K] unpacked codes (convenience for tests)
+
+
+def calib_positions(b: int, k: int, calib_bits: np.ndarray, W_bits: np.ndarray | None = None,
+                    return_importance: bool = False):
+    T, K = calib_bits.shape
+    assert K % b == 0 and calib_bits.dtype == np.uint16
+    N = 0 if W_bits is None else W_bits.shape[0]
+    pos = np.zeros((K // b, k), dtype=np.uint8)
+    imp = np.zeros(K, dtype=np.float64) if return_importance else None
+    _load().sqo_calib_positions(ctypes.c_int(b), ctypes.c_int(k), _p(calib_bits), _l(T), _l(K),
+                                _p(W_bits), _l(N), _p(pos), _p(imp))
+    return (pos, imp) if return_importance else pos
+
+
+def pack_weights(b: int, k: int, W_bits: np.ndarray, positions: np.ndarray | None = None) -> Weights:
+    N, K = W_bits.shape
+    assert K % b == 0 and K % 2 == 0 and W_bits.dtype == np.uint16
+    G = K // b
+    wq4 = np.zeros((N, K // 2), dtype=np.uint8)
+    s_w = np.zeros(N, dtype=np.float32)
+    colsum = np.zeros(N, dtype=np.int32)
+    w_sparse = np.zeros((N, G * k), dtype=np.int8) if positions is not None else None
+    wq = np.zeros((N, K), dtype=np.int8)
+    _load().sqo_pack_weights(ctypes.c_int(b), ctypes.c_int(k), _p(W_bits), _l(N), _l(K), _p(positions),
+                             _p(wq4), _p(s_w), _p(colsum), _p(w_sparse), _p(wq))
+    return Weights(wq4, s_w, colsum, w_sparse, wq)
+
+
+def encode(b: int, k: int, X_bits: np.ndarray, positions: np.ndarray | None = None) -> Encoded:
+    M, K = X_bits.shape
+    assert K % b == 0 and K % 2 == 0 and X_bits.dtype == np.uint16
+    G = K // b
+    dq4 = np.zeros((M, K // 2), dtype=np.uint8)
+    vals = np.zeros((M, G, k), dtype=np.int8)
+    idx = np.zeros((M, G, k), dtype=np.uint8) if positions is None else None
+    s_hi = np.zeros(M, dtype=np.float32)
+    s_lo = np.zeros(M, dtype=np.float32)
+    shift = np.zeros(M, dtype=np.uint8)
+    _load().sqo_encode(ctypes.c_int(b), ctypes.c_int(k), _p(X_bits), _l(M), _l(K), _p(positions),
+                       _p(dq4), _p(vals), _p(idx), _p(s_hi), _p(s_lo), _p(shift))
+    return Encoded(dq4, vals, idx, s_hi, s_lo, shift)
+
+
+def gemm(b: int, k: int, A: Encoded, W: Weights, positions: np.ndarray | None = None,
+         rows=None, cols=None):
+    """Returns (acc int32, ref32 float32, out bf16-bits uint16), each [n_rows, n_cols]."""
+    M, Kh = A.dq4.shape
+    K = Kh * 2
+    N = W.wq4.shape[0]
+    rows_a = None if rows is None else np.ascontiguousarray(rows, dtype=np.int64)
+    cols_a = None if cols is None else np.ascontiguousarray(cols, dtype=np.int64)
+    R = M if rows_a is None else len(rows_a)
+    C = N if cols_a is None else len(cols_a)
+    acc = np.zeros((R, C), dtype=np.int32)
+    ref = np.zeros((R, C), dtype=np.float32)
+    out = np.zeros((R, C), dtype=np.uint16)
+    ov = _load().sqo_gemm(ctypes.c_int(b), ctypes.c_int(k), _p(A.dq4), _p(A.vals), _p(A.idx),
+                          _p(positions), _p(A.s_hi), _p(A.shift), _p(W.wq4), _p(W.s_w),
+                          _l(M), _l(N), _l(K), _p(rows_a), _l(R), _p(cols_a), _l(C),
+                          _p(acc), _p(ref), _p(out))
+    if ov:
+        raise OverflowError("an accumulator does not fit in int32")
+    return acc, ref, out
+
+
+def decode(b: int, k: int, A: Encoded, positions: np.ndarray | None = None):
+    """Returns (x_hat float32 [M,K], x_hat bf16-bits uint16 [M,K])."""
+    M, Kh = A.dq4.shape
+    K = Kh * 2
+    xf = np.zeros((M, K), dtype=np.float32)
+    xb = np.zeros((M, K), dtype=np.uint16)
+    _load().sqo_decode(ctypes.c_int(b), ctypes.c_int(k), _p(A.dq4), _p(A.vals), _p(A.idx), _p(positions),
+                       _p(A.s_hi), _p(A.s_lo), _l(M), _l(K), _p(xf), _p(xb))
+    return xf, xb
