@@ -1,0 +1,188 @@
+/*
+ * sq.h -- C ABI of the B200 (sm_100a) SQ-format library.
+ *
+ * SQ-format (arXiv 2512.05409, Section 3.1, Eq. 1) stores one GEMM operand as
+ * banks of b consecutive elements in which a fixed number k = (1-s)*b of entries
+ * is kept in a high precision h_high and the rest in a low precision h_low, plus
+ * scales and a mask.  This library implements the setting the paper runs on GPUs
+ * (Section 4.1: h_high = INT8, h_low = INT4) for ACTIVATIONS in SQ-format times
+ * INT4 per-output-channel weights:
+ *
+ *     sq_calib_positions   static mask from a calibration batch  (Algorithm 2)
+ *     sq_pack_weights      INT4 weights (+ the Alg. 2 row reorder for static masks)
+ *     sq_encode            bf16 activations -> SQ-format         (Sections 3.2.2, 3.3)
+ *     sq_gemm              dense INT4 + sparse INT8 products, one int32 accumulator,
+ *                          one dequantising epilogue             (Section 3.3, Fig. 2b)
+ *     sq_decode            SQ-format -> bf16                     (inverse of Eq. 1)
+ *
+ * Conventions shared by every call
+ *   - Tensors are dense and row-major.  Activations X are [M, K] and weights W are
+ *     [N, K], both with K contiguous.  Banks run along K: bank g of a row covers
+ *     elements g*b .. g*b+b-1, G = K/b banks per row.
+ *   - Every tensor pointer is a DEVICE pointer owned by the caller, 16-byte aligned,
+ *     sized with sq_encoded_sizes / sq_weights_sizes.  The library allocates nothing
+ *     and frees nothing.  The sq_format, sq_encoded and sq_weights structs themselves
+ *     live in HOST memory and are read during the call only.
+ *   - `cuda_stream` is a cudaStream_t passed as void* (NULL = the default stream).
+ *     Calls validate their arguments on the host, enqueue their kernels on that
+ *     stream and return without synchronising.  An argument error is reported
+ *     synchronously and launches nothing.
+ *   - Shape rules: b in {32, 64, 128}; 1 <= k <= b/2; K % 128 == 0 (hence K % b == 0);
+ *     K <= SQ_MAX_K; N % 8 == 0; M, N >= 0.  A zero-sized problem (M == 0, or N == 0 for
+ *     the weight and GEMM calls) returns SQ_OK right after the shape checks, launches
+ *     nothing and does not look at the tensor pointers.
+ *   - Inputs are assumed finite.  Rows whose largest magnitude is 0, or lies in
+ *     [2^-100, 2^100], are handled exactly; anything else is unspecified.
+ *   - Kernels never trap and never spin without bound: a device-side wait that runs
+ *     out records SQ_ERR_TIMEOUT in a per-device status word (see sq_device_status)
+ *     and the kernel returns after releasing its tensor memory.
+ *   - No exceptions, no aborts, no printing.  The library needs an sm_100 device.
+ *
+ * Number formats (layout version 1)
+ *   - INT4 codes are symmetric in [-7, 7] and INT8 codes in [-127, 127]: the most
+ *     negative code is never produced (Section 3.2.1).  Two INT4 codes share a byte,
+ *     element 2i in the low nibble and 2i+1 in the high nibble, two's complement.
+ *   - RNE(p) below is round-half-to-even of the EXACT real product p.
+ */
+#ifndef SQ_B200_H_
+#define SQ_B200_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define SQ_LAYOUT_VERSION 1
+#define SQ_MAX_K 65536
+
+typedef enum {
+  SQ_OK = 0,
+  SQ_ERR_INVALID_ARG = 1,  /* a size or format field violates the shape rules      */
+  SQ_ERR_UNSUPPORTED = 2,  /* valid in principle but outside what is built (K > SQ_MAX_K) */
+  SQ_ERR_NULL_POINTER = 3, /* a required pointer is NULL                            */
+  SQ_ERR_ALIGNMENT = 4,    /* a tensor pointer is not 16-byte aligned               */
+  SQ_ERR_ARCH = 5,         /* the current device is not sm_100                      */
+  SQ_ERR_CUDA = 6,         /* a CUDA runtime call failed (launch, attribute, copy)  */
+  SQ_ERR_TIMEOUT = 7       /* a bounded device-side wait expired (sq_device_status) */
+} sq_status;
+
+typedef enum { SQ_POS_DYNAMIC = 0, SQ_POS_STATIC = 1 } sq_pos_mode;
+
+/* The part of the Eq. 1 tuple that is a parameter (h_high = INT8, h_low = INT4 fixed). */
+typedef struct {
+  int32_t bank;     /* b: bank size along K, one of 32, 64, 128                   */
+  int32_t k;        /* INT8 entries per bank, k = (1-s)*b, 1 <= k <= b/2          */
+  int32_t pos_mode; /* sq_pos_mode: how the k positions of a bank are chosen      */
+  int32_t version;  /* SQ_LAYOUT_VERSION                                          */
+} sq_format;
+
+/* An activation tensor in SQ-format (device pointers).  G = K/b.
+ *   dq4   uint8 [M, K/2]   dense INT4 component, 0 at the bank's k selected positions
+ *   vals  int8  [M, G, k]  sparse INT8 component, in ascending bank-local position
+ *   idx   uint8 [M, G, k]  bank-local positions (0..b-1) of vals, ascending;
+ *                          NULL / unused when pos_mode == SQ_POS_STATIC
+ *   s_hi  float [M]        scale of the INT8 component: amax / 127
+ *   s_lo  float [M]        scale of the INT4 component: s_hi * 2^shift
+ *   shift uint8 [M]        e in 0..4
+ * Element j of row m decodes to s_hi*vals at a selected position and s_lo*dq4 elsewhere. */
+typedef struct {
+  uint8_t* dq4;
+  int8_t* vals;
+  uint8_t* idx;
+  float* s_hi;
+  float* s_lo;
+  uint8_t* shift;
+} sq_encoded;
+
+/* Packed weights (device pointers).
+ *   wq4      uint8 [N, K/2]  INT4 codes, per-output-channel symmetric
+ *   s_w      float [N]       per-channel scale: wmax / 7
+ *   colsum   int32 [N]       sum over K of the channel's INT4 codes
+ *   w_sparse int8  [N, G*k]  static masks only: the codes of the selected input
+ *                            channels gathered bank by bank (Algorithm 2's reorder),
+ *                            w_sparse[n, g*k+i] = code[n, g*b + positions[g][i]];
+ *                            NULL / unused when pos_mode == SQ_POS_DYNAMIC */
+typedef struct {
+  uint8_t* wq4;
+  float* s_w;
+  int32_t* colsum;
+  int8_t* w_sparse;
+} sq_weights;
+
+/* Text for a status code (static storage, never NULL). */
+const char* sq_status_string(sq_status status);
+
+/* Bytes each member of sq_encoded needs for an [M, K] tensor, in member order
+ * (dq4, vals, idx, s_hi, s_lo, shift).  idx is 0 for static positions. */
+sq_status sq_encoded_sizes(const sq_format* fmt, int64_t M, int64_t K, size_t bytes_out[6]);
+
+/* Bytes each member of sq_weights needs for [N, K] weights, in member order
+ * (wq4, s_w, colsum, w_sparse).  w_sparse is 0 for dynamic positions. */
+sq_status sq_weights_sizes(const sq_format* fmt, int64_t N, int64_t K, size_t bytes_out[4]);
+
+/* Static positions (Algorithm 2; Section 3.2.2).  Setup call, not on the timed path.
+ *   Abar_j = (sum_t |calib[t,j]|) / T     per-channel mean magnitude, fp64, t ascending
+ *   r_j    = sum_n W[n,j]                 signed sum over output channels, fp64, n ascending
+ *            (r_j = 1 when W_bf16 is NULL, which ranks by activations alone)
+ *   I_j    = |Abar_j * r_j|
+ *   positions[g, 0..k) = the k bank-local indices of bank g with the largest I_j
+ *                        (equal I_j: smaller j first), stored ascending.
+ * calib_bf16: device bf16 [T, K], T >= 1.  W_bf16: device bf16 [N, K] or NULL.
+ * positions: device uint8 [K/b, k], written.  fmt->pos_mode must be SQ_POS_STATIC. */
+sq_status sq_calib_positions(const sq_format* fmt, const void* calib_bf16, int64_t T, int64_t K,
+                             const void* W_bf16, int64_t N, uint8_t* positions, void* cuda_stream);
+
+/* Per-output-channel symmetric INT4 weights (the uniformly quantised operand of
+ * Section 3.1 / "classic quantization" of Section 3.2; Algorithm 2's Quant and reorder).
+ *   wmax = max_j |W[n,j]|;  code = clamp(RNE(W[n,j] * (7.0f / wmax)), -7, 7);
+ *   s_w[n] = wmax / 7.0f (both IEEE fp32 divisions); an all-zero channel gets codes 0, s_w 0.
+ * W_bf16: device bf16 [N, K].  positions: device uint8 [K/b, k] for static formats
+ * (as written by sq_calib_positions; trusted: distinct, ascending, < b), NULL for
+ * dynamic ones.  out: all members written (w_sparse only for static formats). */
+sq_status sq_pack_weights(const sq_format* fmt, const void* W_bf16, int64_t N, int64_t K,
+                          const uint8_t* positions, sq_weights* out, void* cuda_stream);
+
+/* Activation encode (Sections 3.2.2 and 3.3), per token row m with a_j = X[m,j]:
+ *   amax = max_j |a_j|
+ *   S    = per bank, the k positions: dynamic -> the k largest |a_j| of the bank
+ *          (equal magnitude: smaller j first); static -> positions[g]
+ *   rmax = max over j not in S of |a_j|
+ *   amax == 0: every code 0, shift 0, s_hi = s_lo = 0.  Otherwise
+ *   inv  = 127.0f / amax,  s_hi = amax / 127.0f            (IEEE fp32 divisions)
+ *   e    = min{ e in 0..4 : RNE(rmax * inv * 2^-e) <= 7 }, or 4;  s_lo = s_hi * 2^e
+ *   j in S:     vals = clamp(RNE(a_j * inv), -127, 127), dense nibble 0
+ *   j not in S: dq4  = clamp(RNE(a_j * inv * 2^-e), -7, 7)
+ * X_bf16: device bf16 [M, K].  positions: as for sq_pack_weights.  out: every member
+ * written (idx only for dynamic formats). */
+sq_status sq_encode(const sq_format* fmt, const void* X_bf16, int64_t M, int64_t K,
+                    const uint8_t* positions, sq_encoded* out, void* cuda_stream);
+
+/* Hybrid GEMM (Section 3.3): the dense INT4 product and the sparse INT8 product go
+ * into ONE int32 accumulator, followed by one dequantising epilogue:
+ *   acc[m,n] = sum_j ( (dq4[m,j] << shift[m]) + [j in S_m] vals[m,j] ) * code[n,j]
+ *   out[m,n] = bf16_rne( ((float)acc[m,n] * s_hi[m]) * s_w[n] )
+ * A: an encoding of an [M, K] tensor.  W: packed [N, K] weights of the same format.
+ * positions: static formats only (the mask the two were built with), else NULL.
+ * out_bf16: device bf16 [M, N], written.  acc_out: device int32 [M, N] or NULL; when
+ * given, the raw accumulators are written as well (used by parity tests). */
+sq_status sq_gemm(const sq_format* fmt, const sq_encoded* A, const sq_weights* W,
+                  const uint8_t* positions, int64_t M, int64_t N, int64_t K, void* out_bf16,
+                  int32_t* acc_out, void* cuda_stream);
+
+/* Decode (inverse of Eq. 1): out[m,j] = bf16_rne(s_hi[m]*vals) at selected positions,
+ * bf16_rne(s_lo[m]*dq4) elsewhere.  out_bf16: device bf16 [M, K], written. */
+sq_status sq_decode(const sq_format* fmt, const sq_encoded* A, const uint8_t* positions,
+                    int64_t M, int64_t K, void* out_bf16, void* cuda_stream);
+
+/* Reads and clears the current device's status word.  Synchronises `cuda_stream`
+ * first, so every kernel enqueued on it before the call has finished.  Returns
+ * SQ_OK, SQ_ERR_TIMEOUT if a kernel gave up on a bounded wait since the last call
+ * (its outputs are then undefined), or SQ_ERR_CUDA if the stream reports an error. */
+sq_status sq_device_status(void* cuda_stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SQ_B200_H_ */

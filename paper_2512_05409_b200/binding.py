@@ -1,0 +1,250 @@
+"""Thin ctypes binding of the C-ABI library (argument marshalling only).
+
+Every function has the name and the argument order of its C counterpart in
+`include/sq.h`; tensors are torch CUDA tensors whose `data_ptr()` is handed over,
+and the stream is torch's current stream unless one is given.  Nothing is computed
+here: every step of the path runs in the library's kernels.  There is no CPU
+fallback -- if the library cannot be loaded the import fails.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from dataclasses import dataclass
+
+import torch
+
+from . import build as _build
+
+SQ_OK = 0
+SQ_ERR_INVALID_ARG = 1
+SQ_ERR_UNSUPPORTED = 2
+SQ_ERR_NULL_POINTER = 3
+SQ_ERR_ALIGNMENT = 4
+SQ_ERR_ARCH = 5
+SQ_ERR_CUDA = 6
+SQ_ERR_TIMEOUT = 7
+
+SQ_POS_DYNAMIC = 0
+SQ_POS_STATIC = 1
+SQ_LAYOUT_VERSION = 1
+SQ_MAX_K = 65536
+
+
+class sq_format(ctypes.Structure):
+    _fields_ = [("bank", ctypes.c_int32), ("k", ctypes.c_int32),
+                ("pos_mode", ctypes.c_int32), ("version", ctypes.c_int32)]
+
+
+class sq_encoded(ctypes.Structure):
+    _fields_ = [("dq4", ctypes.c_void_p), ("vals", ctypes.c_void_p), ("idx", ctypes.c_void_p),
+                ("s_hi", ctypes.c_void_p), ("s_lo", ctypes.c_void_p), ("shift", ctypes.c_void_p)]
+
+
+class sq_weights(ctypes.Structure):
+    _fields_ = [("wq4", ctypes.c_void_p), ("s_w", ctypes.c_void_p), ("colsum", ctypes.c_void_p),
+                ("w_sparse", ctypes.c_void_p)]
+
+
+class SqError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {sq_status_string(status)} (status {status})")
+
+
+def _load() -> ctypes.CDLL:
+    path = _build.LIB
+    if _build.needs_build():
+        path = _build.build()          # raises if nvcc is missing or the build fails
+    lib = ctypes.CDLL(path)
+    P, I64, VP = ctypes.POINTER, ctypes.c_int64, ctypes.c_void_p
+    lib.sq_status_string.restype = ctypes.c_char_p
+    lib.sq_status_string.argtypes = [ctypes.c_int]
+    lib.sq_encoded_sizes.argtypes = [P(sq_format), I64, I64, P(ctypes.c_size_t)]
+    lib.sq_weights_sizes.argtypes = [P(sq_format), I64, I64, P(ctypes.c_size_t)]
+    lib.sq_calib_positions.argtypes = [P(sq_format), VP, I64, I64, VP, I64, VP, VP]
+    lib.sq_pack_weights.argtypes = [P(sq_format), VP, I64, I64, VP, P(sq_weights), VP]
+    lib.sq_encode.argtypes = [P(sq_format), VP, I64, I64, VP, P(sq_encoded), VP]
+    lib.sq_gemm.argtypes = [P(sq_format), P(sq_encoded), P(sq_weights), VP, I64, I64, I64, VP, VP, VP]
+    lib.sq_decode.argtypes = [P(sq_format), P(sq_encoded), VP, I64, I64, VP, VP]
+    lib.sq_device_status.argtypes = [VP]
+    for name in ("sq_encoded_sizes", "sq_weights_sizes", "sq_calib_positions", "sq_pack_weights",
+                 "sq_encode", "sq_gemm", "sq_decode", "sq_device_status"):
+        getattr(lib, name).restype = ctypes.c_int
+    return lib
+
+
+_lib = _load()
+LIBRARY_PATH = _build.LIB
+
+
+def _ptr(t):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream(stream):
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return ctypes.c_void_p(stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream))
+
+
+def _check(status: int, where: str):
+    if status != SQ_OK:
+        raise SqError(status, where)
+
+
+def make_format(bank: int, k: int, static: bool) -> sq_format:
+    return sq_format(bank, k, SQ_POS_STATIC if static else SQ_POS_DYNAMIC, SQ_LAYOUT_VERSION)
+
+
+@dataclass
+class Encoded:
+    """Torch-owned buffers of one sq_encoded (idx is None for static positions)."""
+    dq4: torch.Tensor
+    vals: torch.Tensor
+    idx: torch.Tensor | None
+    s_hi: torch.Tensor
+    s_lo: torch.Tensor
+    shift: torch.Tensor
+
+    def c_struct(self) -> sq_encoded:
+        return sq_encoded(self.dq4.data_ptr(), self.vals.data_ptr(),
+                          self.idx.data_ptr() if self.idx is not None else None,
+                          self.s_hi.data_ptr(), self.s_lo.data_ptr(), self.shift.data_ptr())
+
+
+@dataclass
+class Weights:
+    """Torch-owned buffers of one sq_weights (w_sparse is None for dynamic positions)."""
+    wq4: torch.Tensor
+    s_w: torch.Tensor
+    colsum: torch.Tensor
+    w_sparse: torch.Tensor | None
+
+    def c_struct(self) -> sq_weights:
+        return sq_weights(self.wq4.data_ptr(), self.s_w.data_ptr(), self.colsum.data_ptr(),
+                          self.w_sparse.data_ptr() if self.w_sparse is not None else None)
+
+
+def sq_status_string(status: int) -> str:
+    return _lib.sq_status_string(int(status)).decode()
+
+
+def sq_encoded_sizes(fmt: sq_format, M: int, K: int) -> list[int]:
+    out = (ctypes.c_size_t * 6)()
+    _check(_lib.sq_encoded_sizes(ctypes.byref(fmt), M, K, out), "sq_encoded_sizes")
+    return list(out)
+
+
+def sq_weights_sizes(fmt: sq_format, N: int, K: int) -> list[int]:
+    out = (ctypes.c_size_t * 4)()
+    _check(_lib.sq_weights_sizes(ctypes.byref(fmt), N, K, out), "sq_weights_sizes")
+    return list(out)
+
+
+def _buf(nbytes: int, dtype, device):
+    # at least 16 bytes so that an empty tensor still has a valid, aligned pointer
+    n = max(nbytes, 16) // torch.empty((), dtype=dtype).element_size()
+    return torch.empty(n, dtype=dtype, device=device)
+
+
+def alloc_encoded(fmt: sq_format, M: int, K: int, device="cuda") -> Encoded:
+    sz = sq_encoded_sizes(fmt, M, K)
+    gk = (K // fmt.bank) * fmt.k
+    dq4 = _buf(sz[0], torch.uint8, device)[: sz[0]].view(M, K // 2)
+    vals = _buf(sz[1], torch.int8, device)[: sz[1]].view(M, K // fmt.bank, fmt.k)
+    idx = None
+    if fmt.pos_mode == SQ_POS_DYNAMIC:
+        idx = _buf(sz[2], torch.uint8, device)[: sz[2]].view(M, K // fmt.bank, fmt.k)
+    s_hi = _buf(sz[3], torch.float32, device)[:M]
+    s_lo = _buf(sz[4], torch.float32, device)[:M]
+    shift = _buf(sz[5], torch.uint8, device)[:M]
+    assert gk * M == sz[1]
+    return Encoded(dq4, vals, idx, s_hi, s_lo, shift)
+
+
+def alloc_weights(fmt: sq_format, N: int, K: int, device="cuda") -> Weights:
+    sz = sq_weights_sizes(fmt, N, K)
+    wq4 = _buf(sz[0], torch.uint8, device)[: sz[0]].view(N, K // 2)
+    s_w = _buf(sz[1], torch.float32, device)[:N]
+    colsum = _buf(sz[2], torch.int32, device)[:N]
+    w_sparse = None
+    if fmt.pos_mode == SQ_POS_STATIC:
+        w_sparse = _buf(sz[3], torch.int8, device)[: sz[3]].view(N, (K // fmt.bank) * fmt.k)
+    return Weights(wq4, s_w, colsum, w_sparse)
+
+
+def _bf16_2d(t: torch.Tensor, name: str):
+    if t.dtype != torch.bfloat16 or t.dim() != 2 or not t.is_contiguous() or not t.is_cuda:
+        raise ValueError(f"{name} must be a contiguous 2-D CUDA bf16 tensor")
+    return t.shape
+
+
+def sq_calib_positions(fmt: sq_format, calib: torch.Tensor, W: torch.Tensor | None = None,
+                       positions: torch.Tensor | None = None, stream=None) -> torch.Tensor:
+    T, K = _bf16_2d(calib, "calib")
+    N = 0
+    if W is not None:
+        N, K2 = _bf16_2d(W, "W")
+        if K2 != K:
+            raise ValueError("calib and W disagree on K")
+    if positions is None:
+        positions = _buf(max(K // fmt.bank, 1) * fmt.k, torch.uint8, calib.device)[: (K // fmt.bank) * fmt.k]
+        positions = positions.view(K // fmt.bank, fmt.k)
+    _check(_lib.sq_calib_positions(ctypes.byref(fmt), _ptr(calib), T, K, _ptr(W), N, _ptr(positions),
+                                   _stream(stream)), "sq_calib_positions")
+    return positions
+
+
+def sq_pack_weights(fmt: sq_format, W: torch.Tensor, positions: torch.Tensor | None = None,
+                    out: Weights | None = None, stream=None) -> Weights:
+    N, K = _bf16_2d(W, "W")
+    if out is None:
+        out = alloc_weights(fmt, N, K, W.device)
+    cs = out.c_struct()
+    _check(_lib.sq_pack_weights(ctypes.byref(fmt), _ptr(W), N, K, _ptr(positions), ctypes.byref(cs),
+                                _stream(stream)), "sq_pack_weights")
+    return out
+
+
+def sq_encode(fmt: sq_format, X: torch.Tensor, positions: torch.Tensor | None = None,
+              out: Encoded | None = None, stream=None) -> Encoded:
+    M, K = _bf16_2d(X, "X")
+    if out is None:
+        out = alloc_encoded(fmt, M, K, X.device)
+    cs = out.c_struct()
+    _check(_lib.sq_encode(ctypes.byref(fmt), _ptr(X), M, K, _ptr(positions), ctypes.byref(cs),
+                          _stream(stream)), "sq_encode")
+    return out
+
+
+def sq_gemm(fmt: sq_format, A: Encoded, W: Weights, positions: torch.Tensor | None = None,
+            out: torch.Tensor | None = None, acc_out: torch.Tensor | None = None, stream=None) -> torch.Tensor:
+    M, K = A.dq4.shape[0], A.dq4.shape[1] * 2
+    N = W.wq4.shape[0]
+    if out is None:
+        out = _buf(M * N * 2, torch.bfloat16, A.dq4.device)[: M * N].view(M, N)
+    ca, cw = A.c_struct(), W.c_struct()
+    _check(_lib.sq_gemm(ctypes.byref(fmt), ctypes.byref(ca), ctypes.byref(cw), _ptr(positions), M, N, K,
+                        _ptr(out), _ptr(acc_out), _stream(stream)), "sq_gemm")
+    return out
+
+
+def sq_decode(fmt: sq_format, A: Encoded, positions: torch.Tensor | None = None,
+              out: torch.Tensor | None = None, stream=None) -> torch.Tensor:
+    M, K = A.dq4.shape[0], A.dq4.shape[1] * 2
+    if out is None:
+        out = _buf(M * K * 2, torch.bfloat16, A.dq4.device)[: M * K].view(M, K)
+    ca = A.c_struct()
+    _check(_lib.sq_decode(ctypes.byref(fmt), ctypes.byref(ca), _ptr(positions), M, K, _ptr(out),
+                          _stream(stream)), "sq_decode")
+    return out
+
+
+def sq_device_status(stream=None) -> int:
+    return int(_lib.sq_device_status(_stream(stream)))
+
+
+def raw():
+    """The ctypes CDLL itself (for tests that pass hand-made pointers)."""
+    return _lib

@@ -1,0 +1,227 @@
+// C ABI entry points: argument validation, then one launcher per call.
+#include "sq_host.h"
+
+namespace sq {
+
+// Per-device status word.  A kernel that gives up on a bounded wait stores an
+// sq_status here; sq_device_status() reads and clears it.
+__device__ int g_status_word;
+
+int* status_word() {
+  int* ptr = nullptr;
+  if (cudaGetSymbolAddress(reinterpret_cast<void**>(&ptr), g_status_word) != cudaSuccess) return nullptr;
+  return ptr;
+}
+
+namespace {
+
+bool aligned16(const void* ptr) { return (reinterpret_cast<uintptr_t>(ptr) & 15u) == 0; }
+
+sq_status check_format(const sq_format* fmt) {
+  if (fmt == nullptr) return SQ_ERR_NULL_POINTER;
+  if (fmt->version != SQ_LAYOUT_VERSION) return SQ_ERR_INVALID_ARG;
+  if (fmt->bank != 32 && fmt->bank != 64 && fmt->bank != 128) return SQ_ERR_INVALID_ARG;
+  if (fmt->k < 1 || fmt->k > fmt->bank / 2) return SQ_ERR_INVALID_ARG;
+  if (fmt->pos_mode != SQ_POS_DYNAMIC && fmt->pos_mode != SQ_POS_STATIC) return SQ_ERR_INVALID_ARG;
+  return SQ_OK;
+}
+
+sq_status check_k(int64_t K) {
+  if (K <= 0 || K % 128 != 0) return SQ_ERR_INVALID_ARG;
+  if (K > SQ_MAX_K) return SQ_ERR_UNSUPPORTED;
+  return SQ_OK;
+}
+
+// The kernels are built for sm_100a only; refuse anything else before launching.
+sq_status check_device() {
+  int dev = 0, major = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return SQ_ERR_CUDA;
+  if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return SQ_ERR_CUDA;
+  return major == 10 ? SQ_OK : SQ_ERR_ARCH;
+}
+
+#define SQ_TRY(expr)                 \
+  do {                               \
+    const sq_status st_ = (expr);    \
+    if (st_ != SQ_OK) return st_;    \
+  } while (0)
+
+sq_status check_encoded(const sq_format* fmt, const sq_encoded* A) {
+  if (A == nullptr) return SQ_ERR_NULL_POINTER;
+  if (!A->dq4 || !A->vals || !A->s_hi || !A->s_lo || !A->shift) return SQ_ERR_NULL_POINTER;
+  if (fmt->pos_mode == SQ_POS_DYNAMIC && !A->idx) return SQ_ERR_NULL_POINTER;
+  if (!aligned16(A->dq4) || !aligned16(A->vals) || !aligned16(A->s_hi) || !aligned16(A->s_lo) ||
+      !aligned16(A->shift))
+    return SQ_ERR_ALIGNMENT;
+  if (fmt->pos_mode == SQ_POS_DYNAMIC && !aligned16(A->idx)) return SQ_ERR_ALIGNMENT;
+  return SQ_OK;
+}
+
+sq_status check_weights(const sq_format* fmt, const sq_weights* W) {
+  if (W == nullptr) return SQ_ERR_NULL_POINTER;
+  if (!W->wq4 || !W->s_w || !W->colsum) return SQ_ERR_NULL_POINTER;
+  if (fmt->pos_mode == SQ_POS_STATIC && !W->w_sparse) return SQ_ERR_NULL_POINTER;
+  if (!aligned16(W->wq4) || !aligned16(W->s_w) || !aligned16(W->colsum)) return SQ_ERR_ALIGNMENT;
+  if (fmt->pos_mode == SQ_POS_STATIC && !aligned16(W->w_sparse)) return SQ_ERR_ALIGNMENT;
+  return SQ_OK;
+}
+
+sq_status check_positions(const sq_format* fmt, const uint8_t* positions) {
+  if (fmt->pos_mode == SQ_POS_STATIC) {
+    if (positions == nullptr) return SQ_ERR_NULL_POINTER;
+    if (!aligned16(positions)) return SQ_ERR_ALIGNMENT;
+  } else if (positions != nullptr) {
+    return SQ_ERR_INVALID_ARG;
+  }
+  return SQ_OK;
+}
+
+sq_status from_cuda(cudaError_t err) { return err == cudaSuccess ? SQ_OK : SQ_ERR_CUDA; }
+
+}  // namespace
+}  // namespace sq
+
+using namespace sq;
+
+extern "C" {
+
+const char* sq_status_string(sq_status status) {
+  switch (status) {
+    case SQ_OK: return "ok";
+    case SQ_ERR_INVALID_ARG: return "invalid argument";
+    case SQ_ERR_UNSUPPORTED: return "unsupported size";
+    case SQ_ERR_NULL_POINTER: return "null pointer";
+    case SQ_ERR_ALIGNMENT: return "pointer not 16-byte aligned";
+    case SQ_ERR_ARCH: return "device is not sm_100";
+    case SQ_ERR_CUDA: return "CUDA runtime error";
+    case SQ_ERR_TIMEOUT: return "device-side wait timed out";
+  }
+  return "unknown status";
+}
+
+sq_status sq_encoded_sizes(const sq_format* fmt, int64_t M, int64_t K, size_t bytes_out[6]) {
+  SQ_TRY(check_format(fmt));
+  if (bytes_out == nullptr) return SQ_ERR_NULL_POINTER;
+  if (M < 0) return SQ_ERR_INVALID_ARG;
+  SQ_TRY(check_k(K));
+  const size_t m = (size_t)M, gk = (size_t)(K / fmt->bank) * (size_t)fmt->k;
+  bytes_out[0] = m * (size_t)(K / 2);
+  bytes_out[1] = m * gk;
+  bytes_out[2] = fmt->pos_mode == SQ_POS_DYNAMIC ? m * gk : 0;
+  bytes_out[3] = m * sizeof(float);
+  bytes_out[4] = m * sizeof(float);
+  bytes_out[5] = m;
+  return SQ_OK;
+}
+
+sq_status sq_weights_sizes(const sq_format* fmt, int64_t N, int64_t K, size_t bytes_out[4]) {
+  SQ_TRY(check_format(fmt));
+  if (bytes_out == nullptr) return SQ_ERR_NULL_POINTER;
+  if (N < 0 || N % 8 != 0) return SQ_ERR_INVALID_ARG;
+  SQ_TRY(check_k(K));
+  const size_t n = (size_t)N, gk = (size_t)(K / fmt->bank) * (size_t)fmt->k;
+  bytes_out[0] = n * (size_t)(K / 2);
+  bytes_out[1] = n * sizeof(float);
+  bytes_out[2] = n * sizeof(int32_t);
+  bytes_out[3] = fmt->pos_mode == SQ_POS_STATIC ? n * gk : 0;
+  return SQ_OK;
+}
+
+sq_status sq_calib_positions(const sq_format* fmt, const void* calib_bf16, int64_t T, int64_t K,
+                             const void* W_bf16, int64_t N, uint8_t* positions, void* cuda_stream) {
+  SQ_TRY(check_format(fmt));
+  if (fmt->pos_mode != SQ_POS_STATIC) return SQ_ERR_INVALID_ARG;
+  SQ_TRY(check_k(K));
+  if (T < 1 || (W_bf16 != nullptr && N < 1)) return SQ_ERR_INVALID_ARG;
+  if (calib_bf16 == nullptr || positions == nullptr) return SQ_ERR_NULL_POINTER;
+  if (!aligned16(calib_bf16) || !aligned16(positions) || !aligned16(W_bf16)) return SQ_ERR_ALIGNMENT;
+  SQ_TRY(check_device());
+  return from_cuda(launch_calib_positions(fmt->bank, fmt->k, static_cast<const uint16_t*>(calib_bf16), T, K,
+                                          static_cast<const uint16_t*>(W_bf16), N, positions,
+                                          static_cast<cudaStream_t>(cuda_stream)));
+}
+
+sq_status sq_pack_weights(const sq_format* fmt, const void* W_bf16, int64_t N, int64_t K,
+                          const uint8_t* positions, sq_weights* out, void* cuda_stream) {
+  SQ_TRY(check_format(fmt));
+  SQ_TRY(check_k(K));
+  if (N < 0 || N % 8 != 0) return SQ_ERR_INVALID_ARG;
+  if (N == 0) return SQ_OK;
+  if (W_bf16 == nullptr) return SQ_ERR_NULL_POINTER;
+  if (!aligned16(W_bf16)) return SQ_ERR_ALIGNMENT;
+  SQ_TRY(check_positions(fmt, positions));
+  SQ_TRY(check_weights(fmt, out));
+  SQ_TRY(check_device());
+  sq_weights o = *out;
+  if (fmt->pos_mode != SQ_POS_STATIC) o.w_sparse = nullptr;
+  return from_cuda(launch_pack_weights(fmt->bank, fmt->k, static_cast<const uint16_t*>(W_bf16), N, K, positions, o,
+                                       static_cast<cudaStream_t>(cuda_stream)));
+}
+
+sq_status sq_encode(const sq_format* fmt, const void* X_bf16, int64_t M, int64_t K,
+                    const uint8_t* positions, sq_encoded* out, void* cuda_stream) {
+  SQ_TRY(check_format(fmt));
+  SQ_TRY(check_k(K));
+  if (M < 0) return SQ_ERR_INVALID_ARG;
+  if (M == 0) return SQ_OK;  // nothing to do: pointers of an empty tensor may be NULL
+  if (X_bf16 == nullptr) return SQ_ERR_NULL_POINTER;
+  if (!aligned16(X_bf16)) return SQ_ERR_ALIGNMENT;
+  SQ_TRY(check_positions(fmt, positions));
+  SQ_TRY(check_encoded(fmt, out));
+  SQ_TRY(check_device());
+  return from_cuda(launch_encode(fmt->bank, fmt->k, fmt->pos_mode == SQ_POS_STATIC,
+                                 static_cast<const uint16_t*>(X_bf16), M, K, positions, *out,
+                                 static_cast<cudaStream_t>(cuda_stream)));
+}
+
+sq_status sq_gemm(const sq_format* fmt, const sq_encoded* A, const sq_weights* W,
+                  const uint8_t* positions, int64_t M, int64_t N, int64_t K, void* out_bf16,
+                  int32_t* acc_out, void* cuda_stream) {
+  SQ_TRY(check_format(fmt));
+  SQ_TRY(check_k(K));
+  if (M < 0 || N < 0 || N % 8 != 0 || M > INT32_MAX || N > INT32_MAX) return SQ_ERR_INVALID_ARG;
+  if (M == 0 || N == 0) return SQ_OK;
+  SQ_TRY(check_positions(fmt, positions));
+  SQ_TRY(check_encoded(fmt, A));
+  SQ_TRY(check_weights(fmt, W));
+  if (out_bf16 == nullptr) return SQ_ERR_NULL_POINTER;
+  if (!aligned16(out_bf16) || !aligned16(acc_out)) return SQ_ERR_ALIGNMENT;
+  if ((M + 127) / 128 > 65535) return SQ_ERR_UNSUPPORTED;
+  SQ_TRY(check_device());
+  int* status = status_word();
+  if (status == nullptr) return SQ_ERR_CUDA;
+  return from_cuda(launch_gemm(fmt->bank, fmt->k, *A, *W, positions, M, N, K, static_cast<uint16_t*>(out_bf16),
+                               acc_out, status, static_cast<cudaStream_t>(cuda_stream)));
+}
+
+sq_status sq_decode(const sq_format* fmt, const sq_encoded* A, const uint8_t* positions,
+                    int64_t M, int64_t K, void* out_bf16, void* cuda_stream) {
+  SQ_TRY(check_format(fmt));
+  SQ_TRY(check_k(K));
+  if (M < 0) return SQ_ERR_INVALID_ARG;
+  if (M == 0) return SQ_OK;
+  SQ_TRY(check_positions(fmt, positions));
+  SQ_TRY(check_encoded(fmt, A));
+  if (out_bf16 == nullptr) return SQ_ERR_NULL_POINTER;
+  if (!aligned16(out_bf16)) return SQ_ERR_ALIGNMENT;
+  SQ_TRY(check_device());
+  sq_encoded a = *A;
+  if (fmt->pos_mode == SQ_POS_STATIC) a.idx = nullptr;
+  return from_cuda(launch_decode(fmt->bank, fmt->k, a, positions, M, K, static_cast<uint16_t*>(out_bf16),
+                                 static_cast<cudaStream_t>(cuda_stream)));
+}
+
+sq_status sq_device_status(void* cuda_stream) {
+  SQ_TRY(check_device());
+  if (cudaStreamSynchronize(static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess) return SQ_ERR_CUDA;
+  int word = 0;
+  if (cudaMemcpyFromSymbol(&word, g_status_word, sizeof(int)) != cudaSuccess) return SQ_ERR_CUDA;
+  if (word != 0) {
+    const int zero = 0;
+    if (cudaMemcpyToSymbol(g_status_word, &zero, sizeof(int)) != cudaSuccess) return SQ_ERR_CUDA;
+    return static_cast<sq_status>(word);
+  }
+  return SQ_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,31 @@
+// Host-side launcher prototypes shared by the translation units of the library.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/sq.h"
+
+namespace sq {
+
+// Device address of the per-device status word (0 = fine, else an sq_status).
+int* status_word();
+
+cudaError_t launch_calib_positions(int b, int k, const uint16_t* calib, int64_t T, int64_t K,
+                                   const uint16_t* W, int64_t N, uint8_t* positions,
+                                   cudaStream_t st);
+
+cudaError_t launch_pack_weights(int b, int k, const uint16_t* W, int64_t N, int64_t K,
+                                const uint8_t* positions, const sq_weights& out, cudaStream_t st);
+
+cudaError_t launch_encode(int b, int k, bool is_static, const uint16_t* X, int64_t M, int64_t K,
+                          const uint8_t* positions, const sq_encoded& out, cudaStream_t st);
+
+cudaError_t launch_decode(int b, int k, const sq_encoded& A, const uint8_t* positions, int64_t M,
+                          int64_t K, uint16_t* out, cudaStream_t st);
+
+cudaError_t launch_gemm(int b, int k, const sq_encoded& A, const sq_weights& W,
+                        const uint8_t* positions, int64_t M, int64_t N, int64_t K, uint16_t* out,
+                        int32_t* acc_out, int* status, cudaStream_t st);
+
+}  // namespace sq

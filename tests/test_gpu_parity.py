@@ -1,0 +1,207 @@
+"""Parity of the CUDA path (through the C ABI) with the CPU oracle on the same seeded inputs.
+
+Integers (packed nibbles, INT8 values, indices, shifts, positions, accumulators) must be
+bit-exact; scales are produced by the same IEEE operations and must be bit-exact too; bf16
+outputs must be within a relative error of 1e-2 of the oracle's fp32 result (they are in
+fact equal unless a rounding mode differs).
+"""
+import numpy as np
+import pytest
+import torch
+
+import gen
+import oracle
+import paper_2512_05409_b200 as sq
+from helpers import bits_to_f32
+
+pytestmark = pytest.mark.gpu
+
+REL_TOL = 1e-2   # max |gpu - ref32| / |ref32| for bf16 outputs (exact zero where ref32 == 0)
+
+
+def _np(t):
+    return t.detach().cpu().numpy()
+
+
+def _bits(t):
+    return gen.bf16_bits(t)
+
+
+def assert_bf16_close(gpu_bf16: torch.Tensor, ref32: np.ndarray):
+    got = gpu_bf16.float().cpu().numpy().astype(np.float64)
+    ref = ref32.astype(np.float64)
+    zero = ref == 0
+    assert np.all(got[zero] == 0)
+    rel = np.abs(got[~zero] - ref[~zero]) / np.abs(ref[~zero])
+    assert rel.size == 0 or rel.max() <= REL_TOL, rel.max()
+
+
+def check_status():
+    assert sq.sq_device_status() == sq.SQ_OK
+
+
+def compare_encoded(enc_gpu: sq.Encoded, enc_ref: oracle.Encoded, rows=None):
+    sl = slice(None) if rows is None else rows
+    assert np.array_equal(_np(enc_gpu.dq4)[sl], enc_ref.dq4)
+    assert np.array_equal(_np(enc_gpu.vals)[sl], enc_ref.vals)
+    if enc_ref.idx is not None:
+        assert np.array_equal(_np(enc_gpu.idx)[sl], enc_ref.idx)
+    assert np.array_equal(_np(enc_gpu.shift)[sl], enc_ref.shift)
+    assert np.array_equal(_np(enc_gpu.s_hi)[sl].view(np.uint32), enc_ref.s_hi.view(np.uint32))
+    assert np.array_equal(_np(enc_gpu.s_lo)[sl].view(np.uint32), enc_ref.s_lo.view(np.uint32))
+
+
+def compare_weights(w_gpu: sq.Weights, w_ref: oracle.Weights, rows=None):
+    sl = slice(None) if rows is None else rows
+    assert np.array_equal(_np(w_gpu.wq4)[sl], w_ref.wq4)
+    assert np.array_equal(_np(w_gpu.colsum)[sl], w_ref.colsum)
+    assert np.array_equal(_np(w_gpu.s_w)[sl].view(np.uint32), w_ref.s_w.view(np.uint32))
+    if w_ref.w_sparse is not None:
+        assert np.array_equal(_np(w_gpu.w_sparse)[sl], w_ref.w_sparse)
+
+
+def run_pipeline(M, N, K, b, k, static, seed=0, dist="student_t3", frac=0.01, scale=20.0, T=64,
+                 X=None, full_gemm=True):
+    """Whole path on the GPU vs the oracle; returns nothing, asserts everything."""
+    dev = "cuda"
+    fmt = sq.make_format(b, k, static)
+    if X is None:
+        X = gen.activations(M, K, seed=seed, dist=dist, outlier_fraction=frac, outlier_scale=scale, device=dev)
+    W = gen.weights(N, K, seed=seed, device=dev)
+    Xb, Wb = _bits(X), _bits(W)
+
+    pos = pos_ref = None
+    if static:
+        calib = gen.calibration_batch(T, K, seed=seed, dist=dist, outlier_fraction=frac, outlier_scale=scale,
+                                      device=dev)
+        pos = sq.sq_calib_positions(fmt, calib, W)
+        pos_ref = oracle.calib_positions(b, k, _bits(calib), Wb)
+        assert np.array_equal(_np(pos), pos_ref)
+
+    w_gpu = sq.sq_pack_weights(fmt, W, pos)
+    w_ref = oracle.pack_weights(b, k, Wb, pos_ref)
+    compare_weights(w_gpu, w_ref)
+
+    enc_gpu = sq.sq_encode(fmt, X, pos)
+    enc_ref = oracle.encode(b, k, Xb, pos_ref)
+    compare_encoded(enc_gpu, enc_ref)
+
+    dec_gpu = sq.sq_decode(fmt, enc_gpu, pos)
+    _, dec_ref_bits = oracle.decode(b, k, enc_ref, pos_ref)
+    assert np.array_equal(_bits(dec_gpu), dec_ref_bits)
+
+    acc_gpu = torch.full((M, N), 12345, dtype=torch.int32, device=dev)
+    out_gpu = sq.sq_gemm(fmt, enc_gpu, w_gpu, pos, acc_out=acc_gpu)
+    check_status()
+    if full_gemm:
+        acc_ref, ref32, out_ref = oracle.gemm(b, k, enc_ref, w_ref, pos_ref)
+        assert np.array_equal(_np(acc_gpu), acc_ref)
+        assert_bf16_close(out_gpu, ref32)
+        assert np.array_equal(_bits(out_gpu), out_ref)   # same IEEE ops, same order: equal in practice
+    else:
+        rng = np.random.default_rng(seed)
+        rows = np.unique(np.concatenate([[0, M - 1], rng.integers(0, M, 24)]))
+        cols = np.unique(np.concatenate([[0, N - 1], rng.integers(0, N, 96)]))
+        acc_ref, ref32, out_ref = oracle.gemm(b, k, enc_ref, w_ref, pos_ref, rows=rows, cols=cols)
+        assert np.array_equal(_np(acc_gpu)[np.ix_(rows, cols)], acc_ref)
+        assert_bf16_close(out_gpu[rows][:, cols], ref32)
+    # without the accumulator dump the bf16 output is the same
+    out2 = sq.sq_gemm(fmt, enc_gpu, w_gpu, pos)
+    assert torch.equal(out2, out_gpu)
+    check_status()
+
+
+# ----------------------------------------------------------------------------- small, ragged, multi-tile
+
+@pytest.mark.parametrize("b,k,static", [
+    (64, 8, False), (64, 8, True), (32, 2, False), (32, 8, True), (128, 16, True), (128, 8, False),
+    (64, 16, False), (64, 4, True), (128, 32, False), (32, 1, False), (64, 32, True),
+])
+def test_small_ragged_shapes(b, k, static):
+    # 2 M-tiles with a ragged tail, 2 N-tiles with a ragged tail, 3 K steps
+    run_pipeline(M=200, N=328, K=384, b=b, k=k, static=static, seed=b + k)
+
+
+@pytest.mark.parametrize("M", [1, 16, 127, 128, 129])
+def test_row_counts_around_a_tile(M):
+    run_pipeline(M=M, N=264, K=256, b=64, k=8, static=False, seed=M)
+
+
+def test_deep_k_exceeds_the_pipeline_depth():
+    # 12 K steps (> 2x the number of shared-memory stages), one tile
+    run_pipeline(M=96, N=128, K=1536, b=64, k=8, static=False, seed=7)
+    run_pipeline(M=96, N=128, K=1536, b=128, k=16, static=True, seed=8)
+
+
+def test_config1_single_gemm():
+    """M=64, K=N=4096, N(0,1) activations with 1% channels x20, b=64, k=8 dynamic."""
+    run_pipeline(M=64, N=4096, K=4096, b=64, k=8, static=False, seed=0, dist="normal", frac=0.01, scale=20.0)
+
+
+def test_degenerate_rows():
+    """Zero rows, constant rows (every element ties), one-hot rows, and a row that clamps."""
+    K, b, k = 256, 64, 8
+    X = gen.activations(8, K, seed=3, device="cpu").float()
+    X[0] = 0
+    X[1] = -3.0
+    X[2] = 0
+    X[2, 77] = 2.5
+    X[3, :] = 1.0
+    X[3, 5] = 1.0078125          # barely above the ties
+    X[4] = X[4].abs().clamp_min(0.5)   # all close to each other -> shift 4 and clamping
+    X = X.to(torch.bfloat16).cuda()
+    run_pipeline(M=8, N=64, K=K, b=b, k=k, static=False, X=X)
+    run_pipeline(M=8, N=64, K=K, b=b, k=k, static=True, X=X)
+
+
+def test_empty_problem_is_a_no_op():
+    fmt = sq.make_format(64, 8, False)
+    X = torch.empty(0, 256, dtype=torch.bfloat16, device="cuda")
+    enc = sq.sq_encode(fmt, X)
+    W = gen.weights(16, 256, device="cuda")
+    w = sq.sq_pack_weights(fmt, W)
+    out = sq.sq_gemm(fmt, enc, w)
+    assert out.shape == (0, 16)
+    assert sq.sq_decode(fmt, enc).shape == (0, 256)
+    check_status()
+
+
+def test_maximum_k():
+    """K = SQ_MAX_K: the largest row the encoder stages and the largest accumulation depth."""
+    K = sq.SQ_MAX_K
+    b, k = 128, 16
+    fmt = sq.make_format(b, k, False)
+    X = gen.activations(4, K, seed=1, device="cuda")
+    W = gen.weights(8, K, seed=1, device="cuda")
+    enc = sq.sq_encode(fmt, X)
+    w = sq.sq_pack_weights(fmt, W)
+    acc = torch.zeros(4, 8, dtype=torch.int32, device="cuda")
+    out = sq.sq_gemm(fmt, enc, w, acc_out=acc)
+    check_status()
+    enc_ref = oracle.encode(b, k, _bits(X))
+    w_ref = oracle.pack_weights(b, k, _bits(W))
+    compare_encoded(enc, enc_ref)
+    acc_ref, ref32, _ = oracle.gemm(b, k, enc_ref, w_ref)
+    assert np.array_equal(_np(acc), acc_ref)
+    assert_bf16_close(out, ref32)
+
+
+def test_worst_case_accumulator_magnitude():
+    """All-maximal codes of one sign: the internal offset form must not overflow int32."""
+    K, b, k = 8192, 64, 8
+    fmt = sq.make_format(b, k, False)
+    X = torch.full((2, K), 3.0, dtype=torch.bfloat16, device="cuda")
+    X[1] = -3.0
+    W = torch.full((8, K), 0.5, dtype=torch.bfloat16, device="cuda")
+    W[1] = -0.5
+    enc = sq.sq_encode(fmt, X)
+    w = sq.sq_pack_weights(fmt, W)
+    acc = torch.zeros(2, 8, dtype=torch.int32, device="cuda")
+    sq.sq_gemm(fmt, enc, w, acc_out=acc)
+    check_status()
+    enc_ref = oracle.encode(b, k, _bits(X))
+    w_ref = oracle.pack_weights(b, k, _bits(W))
+    acc_ref, _, _ = oracle.gemm(b, k, enc_ref, w_ref)
+    assert np.array_equal(_np(acc), acc_ref)
+    # (K/b)*k entries at 127 and the rest at 7 << 4 = 112, times 7
+    assert abs(int(acc_ref[0, 0])) == ((K // b) * k * 127 + (K - (K // b) * k) * 112) * 7
