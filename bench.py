@@ -1,0 +1,391 @@
+#!/usr/bin/env python
+"""Benchmark of the SQ-format hot path on B200.
+
+One "step" is one pass of the whole path over one batch of synthetic activations of the
+70B-decoder-shaped prefill linears (M = 4096 tokens through the fused-QKV, O, fused gate-up
+and down projections; b = 128, k = 16 static positions): for each linear, sq_encode of its
+bf16 input followed by sq_gemm against its packed INT4 weights.  `value` is the effective
+throughput 2*M*N*K summed over the four linears divided by the step time (encode included),
+with inputs resident in HBM; `e2e` is the same metric with the inputs in pinned host memory
+and the outputs copied back inside the timed region.  The roofline object covers the GEMM
+kernel (tensor bound); `encode` reports the bandwidth-bound encode kernel on the 8192 x 8192
+bandwidth test.  `--impl reference` times the CPU oracle on a bounded sample instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import gen  # noqa: E402
+
+METRIC = "sq_gemm effective TOPS (% of INT8 tensor peak); sq_encode GB/s (% of HBM)"
+UNIT = "TOPS"
+WORKLOAD = "70B-decoder-shaped prefill linears: M=4096 x (K,N) in {(8192,10240),(8192,8192),(8192,57344),(28672,8192)}; b=128,k=16 static"
+SHAPES_70B = [(8192, 10240), (8192, 8192), (8192, 57344), (28672, 8192)]
+M_70B, BANK_70B, K_70B = 4096, 128, 16
+INT8_OVER_BF16 = 2.0        # nominal dense INT8 : bf16 tensor rate on B200 (4.5 : 2.25 PFLOP/s)
+FALLBACK_HBM_GBS, FALLBACK_BF16_TFLOPS = 6650.0, 1590.0
+# DRAM bytes per GEMM launch measured by ncu (see profiles/); None until a capture exists.
+GEMM_TRAFFIC_BYTES_PER_LAUNCH = None
+ENCODE_TRAFFIC_BYTES_PER_LAUNCH = None
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {"hbm_gbs": float(p["hbm_gbs"]), "bf16_tflops": float(p["bf16_tflops"]),
+                "bf16_tflops_sustained": float(p.get("bf16_tflops_sustained", p["bf16_tflops"])),
+                "source": "measured"}
+    return {"hbm_gbs": FALLBACK_HBM_GBS, "bf16_tflops": FALLBACK_BF16_TFLOPS,
+            "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons of one GPU while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.lines, self.proc = index, [], None
+
+    def __enter__(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}",
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+        return self
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def __exit__(self, *exc):
+        if self.proc is not None:
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=5)
+            except subprocess.TimeoutExpired:
+                self.proc.kill()
+
+    def summary(self):
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.lines:
+            parts = [x.strip() for x in line.split(",")]
+            if len(parts) < 6:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for name, flag in zip(names, parts[2:6]):
+                if flag.lower().startswith("active"):
+                    reasons.add(name)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        return {"sm_mhz": statistics.median(sm), "sm_max_mhz": max(mx), "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+def physical_gpu_index(local: int) -> int:
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+    if vis:
+        try:
+            return int(vis.split(",")[local])
+        except (ValueError, IndexError):
+            return local
+    return local
+
+
+# ----------------------------------------------------------------------------- the CUDA arm
+
+class Linear:
+    """One linear layer of the workload: packed weights, static positions, I/O buffers."""
+
+    def __init__(self, sq, M, K, N, bank, k, static, seed, dev, dist="student_t3"):
+        self.M, self.K, self.N = M, K, N
+        self.fmt = sq.make_format(bank, k, static)
+        W = gen.weights(N, K, seed=seed, device=dev)
+        self.pos = None
+        if static:
+            calib = gen.calibration_batch(512, K, seed=seed, dist=dist, outlier_fraction=0.01,
+                                          outlier_scale=20.0, device=dev)
+            self.pos = sq.sq_calib_positions(self.fmt, calib, W)
+            del calib
+        self.w = sq.sq_pack_weights(self.fmt, W, self.pos)
+        del W
+        self.X = gen.activations(M, K, seed=seed, dist=dist, outlier_fraction=0.01, outlier_scale=20.0, device=dev)
+        self.enc = sq.alloc_encoded(self.fmt, M, K, dev)
+        self.out = torch.empty(M, N, dtype=torch.bfloat16, device=dev)
+        self.ops = 2.0 * M * N * K
+        # algorithmic bytes: packed activations + packed weights + bf16 output
+        payload = 0.5 + (1.0 if static else 2.0) * k / bank
+        self.gemm_bytes = M * K * payload + N * K / 2 + 2.0 * M * N
+        self.encode_bytes = M * K * (2.0 + payload) + 9.0 * M
+
+    def step(self, sq, events=None):
+        if events is not None:
+            events[0].record()
+        sq.sq_encode(self.fmt, self.X, self.pos, out=self.enc)
+        if events is not None:
+            events[1].record()
+        sq.sq_gemm(self.fmt, self.enc, self.w, self.pos, out=self.out)
+        if events is not None:
+            events[2].record()
+
+
+def bench_encode_only(sq, dev, peaks, iters=20):
+    """The bandwidth test: 8192 x 8192 bf16, Student-t with 0.5% channels x50, b=64, k in {4,8,16}."""
+    M = K = 8192
+    res = []
+    # three input buffers in rotation (384 MB > L2) so no launch finds its input in L2
+    Xs = [gen.activations(M, K, seed=s, outlier_fraction=0.005, outlier_scale=50.0, device=dev) for s in range(3)]
+    calib = gen.calibration_batch(512, K, seed=0, outlier_fraction=0.005, outlier_scale=50.0, device=dev)
+    for static in (False, True):
+        for k in (4, 8, 16):
+            fmt = sq.make_format(64, k, static)
+            pos = sq.sq_calib_positions(fmt, calib) if static else None
+            enc = sq.alloc_encoded(fmt, M, K, dev)
+            for i in range(3):
+                sq.sq_encode(fmt, Xs[i % 3], pos, out=enc)
+            torch.cuda.synchronize()
+            evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(iters)]
+            for i in range(iters):
+                evs[i][0].record()
+                sq.sq_encode(fmt, Xs[i % 3], pos, out=enc)
+                evs[i][1].record()
+            torch.cuda.synchronize()
+            ms = statistics.median(a.elapsed_time(b) for a, b in evs)
+            nbytes = M * K * (2.0 + 0.5 + (1.0 if static else 2.0) * k / 64) + 9.0 * M
+            gbs = nbytes / (ms * 1e-3) / 1e9
+            res.append({"mode": "static" if static else "dynamic", "k": k, "ms": round(ms, 4),
+                        "GBps": round(gbs, 1), "frac_of_measured_hbm": round(gbs / peaks["hbm_gbs"], 4),
+                        "frac_of_8TBps": round(gbs / 8000.0, 4)})
+    return res
+
+
+def oracle_sample(K, N, bank, k, seed, rows=32, cols=512):
+    """Times the CPU oracle (encode + GEMM) on a bounded sample of one linear of the workload."""
+    import oracle
+    Xb = gen.bf16_bits(gen.activations(rows, K, seed=seed, outlier_fraction=0.01, outlier_scale=20.0))
+    Wb = gen.bf16_bits(gen.weights(cols, K, seed=seed))
+    calib = gen.bf16_bits(gen.calibration_batch(64, K, seed=seed, outlier_fraction=0.01, outlier_scale=20.0))
+    pos = oracle.calib_positions(bank, k, calib, Wb)
+    pw = oracle.pack_weights(bank, k, Wb, pos)
+    t0 = time.perf_counter()
+    enc = oracle.encode(bank, k, Xb, pos)
+    oracle.gemm(bank, k, enc, pw, pos)
+    dt = time.perf_counter() - t0
+    return 2.0 * rows * cols * K, dt, oracle.num_threads()
+
+
+def run_reference(args):
+    """CPU oracle arm: same metric and config, each step a bounded sample of the workload."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    K, N = SHAPES_70B[1]
+    sample = {"rows": 256, "cols": 2048}
+    for _ in range(args.warmup):
+        oracle_sample(K, N, BANK_70B, K_70B, 0, **sample)
+    ops = dt = 0.0
+    cores = 1
+    for _ in range(args.steps):
+        o, d, cores = oracle_sample(K, N, BANK_70B, K_70B, 0, **sample)
+        ops += o
+        dt += d
+    tops = ops / dt / 1e12
+    desc = f"encode + GEMM of {sample['rows']} token rows x {sample['cols']} output channels of the (K,N)=({K},{N}) linear per step"
+    line = {"impl": "reference", "metric": METRIC, "value": tops, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int8",
+            "data": "synthetic", "config": {"workload": WORKLOAD, "sample": desc},
+            "cpu_baseline": {"value": tops, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc},
+            "e2e": {"value": tops, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+def run_cuda(args):
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+
+    import paper_2512_05409_b200 as sq
+    peaks = load_peaks()
+
+    # weak scaling: every rank owns its own batch of M tokens (tokens are independent units)
+    M = args.m
+    layers = [Linear(sq, M, K, N, BANK_70B, K_70B, True, seed=rank * 16 + i, dev=dev) for i, (K, N) in enumerate(SHAPES_70B)]
+    total_ops = sum(l.ops for l in layers)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 3)):
+        for l in layers:
+            l.step(sq)
+    barrier()
+    assert sq.sq_device_status() == sq.SQ_OK
+
+    # ---- device-resident timing (inputs larger than L2: ~0.9 GB of packed weights + activations per step)
+    evs = [[[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in layers] for _ in range(args.steps)]
+    with ClockSampler(physical_gpu_index(local)) as clocks:
+        barrier()
+        t_first = torch.cuda.Event(enable_timing=True)
+        t_last = torch.cuda.Event(enable_timing=True)
+        t_first.record()
+        for s in range(args.steps):
+            for li, l in enumerate(layers):
+                l.step(sq, evs[s][li])
+        t_last.record()
+        barrier()
+        total_ms = t_first.elapsed_time(t_last)
+        if total_ms < 1500:      # keep the sampler alive long enough to see the loaded clocks
+            t_end = time.time() + 1.0
+            while time.time() < t_end:
+                for l in layers:
+                    l.step(sq)
+                torch.cuda.synchronize()
+    clk = clocks.summary()
+    assert sq.sq_device_status() == sq.SQ_OK
+
+    t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
+    if dist is not None:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    total_ms_max = float(t.item())
+    ms_per_step = total_ms_max / args.steps
+    value = world * total_ops / (ms_per_step * 1e-3) / 1e12
+
+    gemm_ms = sum(e[1].elapsed_time(e[2]) for st in evs for e in st)
+    enc_ms = sum(e[0].elapsed_time(e[1]) for st in evs for e in st)
+    n_gemm = args.steps * len(layers)
+    gemm_tops = total_ops * args.steps / (gemm_ms * 1e-3) / 1e12
+    int8_peak = peaks["bf16_tflops"] * INT8_OVER_BF16
+    enc_bytes = sum(l.encode_bytes for l in layers) * args.steps
+    enc_gbs = enc_bytes / (enc_ms * 1e-3) / 1e9
+
+    # ---- end to end: pinned host inputs, device->host outputs, all inside the timed region
+    host_X = [torch.empty(l.X.shape, dtype=torch.bfloat16).pin_memory() for l in layers]
+    host_out = [torch.empty(l.out.shape, dtype=torch.bfloat16).pin_memory() for l in layers]
+    for hx, l in zip(host_X, layers):
+        hx.copy_(l.X)
+    h2d = sum(hx.numel() * 2 for hx in host_X)
+    d2h = sum(ho.numel() * 2 for ho in host_out)
+    e2e_steps = max(1, min(args.steps, 3))
+
+    def e2e_step():
+        for hx, ho, l in zip(host_X, host_out, layers):
+            l.X.copy_(hx, non_blocking=True)
+            l.step(sq)
+            ho.copy_(l.out, non_blocking=True)
+
+    e2e_step()
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(e2e_steps):
+        e2e_step()
+    e1.record()
+    barrier()
+    t = torch.tensor([e0.elapsed_time(e1)], dtype=torch.float64, device=dev)
+    if dist is not None:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    e2e_value = world * total_ops / (float(t.item()) / e2e_steps * 1e-3) / 1e12
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "int8", "data": "synthetic",
+        "config": {"workload": WORKLOAD, "M_per_gpu": M, "bank": BANK_70B, "k": K_70B, "positions": "static",
+                   "step": "sq_encode + sq_gemm for each of the four linears",
+                   "l2": "inputs larger than L2 (packed weights + activations + outputs of a step ~2.5 GB)",
+                   "sharding": "tokens (M) per rank, weights replicated, no data-path collective"},
+        "clocks": clk,
+        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "steps": e2e_steps},
+        "gpu_launches": 2 * len(layers) * args.steps,
+        "roofline": {"kernel": "sq_gemm", "bound": "tensor", "achieved": gemm_tops, "peak": int8_peak,
+                     "unit": "TOPS", "frac": gemm_tops / int8_peak,
+                     "peak_source": f"2 x {peaks['source']} bf16 burst ({peaks['bf16_tflops']} TFLOP/s); INT8:bf16 nominal ratio 2",
+                     "frac_of_sustained": gemm_tops / (peaks["bf16_tflops_sustained"] * INT8_OVER_BF16),
+                     "frac_of_nominal_4500": gemm_tops / 4500.0,
+                     "avg_launch_ms": gemm_ms / n_gemm, "launches": n_gemm,
+                     "traffic": GEMM_TRAFFIC_BYTES_PER_LAUNCH},
+        "roofline_encode_in_step": {"kernel": "sq_encode", "bound": "hbm", "achieved": enc_gbs,
+                                    "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": enc_gbs / peaks["hbm_gbs"],
+                                    "peak_source": peaks["source"], "traffic": ENCODE_TRAFFIC_BYTES_PER_LAUNCH},
+    }
+    if rank == 0:
+        if not args.no_encode_bench:
+            del host_X, host_out
+            line["encode"] = {"workload": "sq_encode alone: bf16 8192 x 8192, Student-t nu=3, 0.5% channels x50, b=64; 3 inputs in rotation (> L2)",
+                              "results": bench_encode_only(sq, dev, peaks)}
+        if not args.no_cpu_baseline and world == 1:
+            K, N = SHAPES_70B[1]
+            ops = dt = 0.0
+            cores = 1
+            t_end = time.time() + 12.0
+            n = 0
+            while time.time() < t_end or n == 0:
+                o, d, cores = oracle_sample(K, N, BANK_70B, K_70B, 0, rows=128, cols=1024)
+                ops, dt, n = ops + o, dt + d, n + 1
+            line["cpu_baseline"] = {"value": ops / dt / 1e12, "unit": UNIT, "cores": cores, "kind": "oracle",
+                                    "sample": f"{n} x (encode + GEMM of 128 token rows x 1024 output channels of the (K,N)=({K},{N}) linear)"}
+        print(json.dumps(line))
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", choices=["cuda", "reference"], default="cuda")
+    ap.add_argument("--m", type=int, default=M_70B, help="tokens per GPU (default: the workload's 4096)")
+    ap.add_argument("--no-encode-bench", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_cuda(args)
+
+
+if __name__ == "__main__":
+    main()
