@@ -246,7 +246,9 @@ def run_cuda(args):
 
     # weak scaling: every rank owns its own batch of M tokens (tokens are independent units)
     M = args.m
-    layers = [Linear(sq, M, K, N, BANK_70B, K_70B, True, seed=rank * 16 + i, dev=dev) for i, (K, N) in enumerate(SHAPES_70B)]
+    chosen = [int(x) for x in args.linears.split(",")] if args.linears else list(range(len(SHAPES_70B)))
+    layers = [Linear(sq, M, SHAPES_70B[i][0], SHAPES_70B[i][1], BANK_70B, K_70B, True, seed=rank * 16 + i, dev=dev)
+              for i in chosen]
     total_ops = sum(l.ops for l in layers)
 
     def barrier():
@@ -330,7 +332,7 @@ def run_cuda(args):
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "int8", "data": "synthetic",
-        "config": {"workload": WORKLOAD, "M_per_gpu": M, "bank": BANK_70B, "k": K_70B, "positions": "static",
+        "config": {"workload": WORKLOAD if not args.linears else WORKLOAD + f" [subset {args.linears}]", "M_per_gpu": M, "bank": BANK_70B, "k": K_70B, "positions": "static",
                    "step": "sq_encode + sq_gemm for each of the four linears",
                    "l2": "inputs larger than L2 (packed weights + activations + outputs of a step ~2.5 GB)",
                    "sharding": "tokens (M) per rank, weights replicated, no data-path collective"},
@@ -378,6 +380,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", choices=["cuda", "reference"], default="cuda")
     ap.add_argument("--m", type=int, default=M_70B, help="tokens per GPU (default: the workload's 4096)")
+    ap.add_argument("--linears", type=str, default="",
+                    help="comma-separated indices into the four linears (default: all four; a subset is for profiling)")
     ap.add_argument("--no-encode-bench", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()

@@ -5,10 +5,10 @@
 //
 // sm_100 has no INT4 MMA, so both operands are widened to 8 bits on chip.  The two
 // components of the activation live on one integer grid (the dense one coarsened by
-// 2^e), so they can be MERGED into a single 8-bit operand before the tensor core
-// sees them: the dense nibbles are widened and shifted, then the k sparse INT8
-// entries of every bank overwrite the (zero) places they belong to.  One MMA stream,
-// one int32 accumulator in tensor memory, one epilogue.
+// 2^e), so they are MERGED into a single 8-bit operand before the tensor core sees
+// them: the dense nibbles are widened and shifted, then the k sparse INT8 entries of
+// every bank overwrite the (zero) places they belong to.  One MMA stream, one int32
+// accumulator in tensor memory, one epilogue.
 //
 // Operand encodings inside the kernel (chosen so the widening is a few logic ops on
 // eight nibbles at a time, never a per-byte sign extension):
@@ -28,6 +28,15 @@
 // Shared-memory operand layout: K-major, 128-byte rows (one K step = 128 elements),
 // 128-byte swizzle (the 16-byte chunk index is XORed with row % 8), 8-row groups 1024
 // bytes apart: the canonical layout a tcgen05 shared-memory descriptor describes.
+//
+// Kernel organisation: persistent, one CTA per SM, warp-specialised.
+//   warps 0-7   producers: global loads (register-prefetched two K steps ahead), widening,
+//               sparse merge, stores into a ring of NS shared-memory stages
+//   warp  8     one thread issues the MMAs and commits stage / accumulator barriers
+//   warps 9-12  epilogue: tcgen05.ld of one of two accumulator buffers, dequantise, store;
+//               overlaps the main loop of the next tile
+// Every wait is bounded; a wait that runs out raises an abort flag that releases all
+// other waits, the kernel records SQ_ERR_TIMEOUT and frees its tensor memory.
 #include "sq_device.cuh"
 #include "sq_host.h"
 
@@ -35,9 +44,14 @@ namespace sq {
 
 namespace {
 
-constexpr int BM = 128;       // rows of A per CTA = TMEM lanes
-constexpr int BK = 128;       // K elements per pipeline step = bytes per operand row
-constexpr int kThreads = 256;
+constexpr int BM = 128;  // rows of A per tile = TMEM lanes
+constexpr int BK = 128;  // K elements per pipeline step = bytes per operand row
+constexpr int kProdWarps = 8;
+constexpr int kProdThreads = kProdWarps * 32;
+constexpr int kMmaWarp = kProdWarps;
+constexpr int kEpiWarp0 = kProdWarps + 1;
+constexpr int kEpiWarps = 4;
+constexpr int kThreads = (kProdWarps + 1 + kEpiWarps) * 32;
 
 struct GemmParams {
   const uint8_t* dq4;
@@ -53,6 +67,7 @@ struct GemmParams {
   int32_t* acc_out;
   int* status;
   int M, N, K, b, k;
+  int log2k;      // log2(k) when the word path is usable, else -1
 };
 
 // Shared-memory matrix descriptor: K-major, SWIZZLE_128B, 8-row groups 1024 B apart.
@@ -69,61 +84,67 @@ __device__ __forceinline__ uint64_t make_desc(uint32_t saddr) {
 // Instruction descriptor: D = s32, A = u8, B = s8, both K-major, M = 128, N = BN.
 template <int BN>
 __device__ __forceinline__ constexpr uint32_t make_idesc() {
-  return (2u << 4)                      // D format: S32
-         | (0u << 7)                    // A format: unsigned 8-bit
-         | (1u << 10)                   // B format: signed 8-bit
-         | ((uint32_t)(BN >> 3) << 17)  // N
-         | ((uint32_t)(BM >> 4) << 24); // M
-}
-
-// Byte offset inside a [rows][128 B] swizzled tile of K-position p (0..127) of `row`.
-__device__ __forceinline__ uint32_t swz(uint32_t row, uint32_t p) {
-  return row * 128u + ((((p >> 4) ^ row) & 7u) << 4) + (p & 15u);
-}
-
-// K-position (within the 128 of a step) where element jj is stored: blocks of 32,
-// even elements first.
-__device__ __forceinline__ uint32_t kpos(uint32_t jj) {
-  return (jj & ~31u) | ((jj & 1u) << 4) | ((jj & 31u) >> 1);
+  return (2u << 4)                       // D format: S32
+         | (0u << 7)                     // A format: unsigned 8-bit
+         | (1u << 10)                    // B format: signed 8-bit
+         | ((uint32_t)(BN >> 3) << 17)   // N
+         | ((uint32_t)(BM >> 4) << 24);  // M
 }
 
 template <int BN, int NS>
 struct Smem {
-  static constexpr int kA = BM * BK;   // 16 KB
+  static constexpr int kA = BM * BK;  // 16 KB
   static constexpr int kB = BN * BK;
   static constexpr int kBytes = NS * (kA + kB) + 1024 /*alignment slack*/ + 256 /*barriers*/;
 };
 
+// Four bank-local indices in one word -> their K positions inside the bank's 32-blocks
+// (even elements first, then odd ones), bytewise.
+__device__ __forceinline__ uint32_t kpos4(uint32_t w) {
+  return (w & 0x60606060u) | ((w & 0x01010101u) << 4) | ((w >> 1) & 0x0F0F0F0Fu);
+}
+__device__ __forceinline__ uint32_t kpos1(uint32_t jj) {
+  return (jj & 0x60u) | ((jj & 1u) << 4) | ((jj & 31u) >> 1);
+}
+
 }  // namespace
 
-template <int BN, int NS>
+template <int BN, int NS, int MAXT>
 __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const GemmParams p) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* smem = smem_raw + (base - smem_u32(smem_raw));
-  uint8_t* sA = smem;                                  // NS x [128][128]
-  uint8_t* sB = smem + NS * Smem<BN, NS>::kA;          // NS x [BN][128]
+  uint8_t* sA = smem;                          // NS x [128][128]
+  uint8_t* sB = smem + NS * Smem<BN, NS>::kA;  // NS x [BN][128]
   uint8_t* sCtl = sB + NS * Smem<BN, NS>::kB;
-  const uint32_t bar_empty = smem_u32(sCtl);           // NS x 8 B
-  const uint32_t bar_done = bar_empty + 8 * NS;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(sCtl + 8 * NS + 8);
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(sCtl + 8 * NS + 16);
+  const uint32_t bar_full = smem_u32(sCtl);    // NS x 8 B
+  const uint32_t bar_empty = bar_full + 8 * NS;
+  const uint32_t bar_tfull = bar_empty + 8 * NS;  // 2 x 8 B
+  const uint32_t bar_tempty = bar_tfull + 16;     // 2 x 8 B
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(sCtl + 16 * NS + 32);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(sCtl + 16 * NS + 40);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int tile_n = blockIdx.x * BN;
-  const int tile_m = blockIdx.y * BM;
   const int KS = p.K / BK;
   const int Kh = p.K / 2;
-  const int G = p.K / p.b;
+  const int tiles_m = (p.M + BM - 1) / BM;
+  const int tiles_n = (p.N + BN - 1) / BN;
+  const int ntiles = tiles_m * tiles_n;
 
   if (tid == 0) {
-    for (int s = 0; s < NS; ++s) mbar_init(bar_empty + 8 * s, 1);
-    mbar_init(bar_done, 1);
+    for (int s = 0; s < NS; ++s) {
+      mbar_init(bar_full + 8 * s, kProdThreads);
+      mbar_init(bar_empty + 8 * s, 1);
+    }
+    for (int bq = 0; bq < 2; ++bq) {
+      mbar_init(bar_tfull + 8 * bq, 1);
+      mbar_init(bar_tempty + 8 * bq, kEpiWarps * 32);
+    }
     *abort_flag = 0;
     fence_mbar_init();
   }
-  if (warp == 0) {
-    tmem_alloc(smem_u32(tmem_slot), BN);
+  if (warp == kMmaWarp) {
+    tmem_alloc(smem_u32(tmem_slot), 2 * BN);
     tmem_relinquish();
   }
   tc_fence_before();
@@ -131,139 +152,247 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const GemmParams p) {
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
 
-  constexpr uint32_t idesc = make_idesc<BN>();
-  const int banks_per_step = BK / p.b;
-  const int nb = banks_per_step * p.k;  // sparse entries per row per step
-  bool ok = true;
+  if (warp < kProdWarps) {
+    // =============================================================== producers
+    const int pw = warp;
+    const int r7 = lane >> 2;  // row within an 8-row group (= row % 8)
+    const int c = lane & 3;    // packed 16-byte chunk within the K step
+    const uint32_t sw_even = (uint32_t)(((2 * c) ^ r7) << 4);
+    const uint32_t a_row0 = (uint32_t)(16 * pw + r7) * 128u;         // + i * 1024
+    const uint32_t b_row0 = (uint32_t)((BN / 8) * pw + r7) * 128u;   // + i * 1024
+    constexpr int NB_TASKS = BN / 64;                                // B chunks per thread per step
+    const int GK = (p.K / p.b) * p.k;
+    const int nb = (BK / p.b) * p.k;  // sparse entries per row per K step
+    const bool word_path = p.log2k >= 0;
+    const int nw_log = word_path ? (31 - __clz(nb >> 2)) : 0;  // log2(words per row per step)
+    const int ntask = word_path ? ((16 << nw_log) + 31) >> 5 : 0;
 
-  for (int ks = 0; ks < KS && ok; ++ks) {
-    const int s = ks % NS;
-    uint8_t* a_st = sA + s * Smem<BN, NS>::kA;
-    uint8_t* b_st = sB + s * Smem<BN, NS>::kB;
-    if (ks >= NS) {
-      // the MMAs that read this stage NS steps ago must have finished
-      const bool w = mbar_wait(bar_empty + 8 * s, (uint32_t)((ks / NS - 1) & 1), abort_flag);
-      ok = __syncthreads_and(w);
+    uint32_t it = 0;
+    for (int tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
+      const int tile_m = (tile % tiles_m) * BM;
+      const int tile_n = (tile / tiles_m) * BN;
+      const uint8_t* a_ptr[2];
+      uint32_t a_mul[2], a_off[2];
+#pragma unroll
+      for (int i = 0; i < 2; ++i) {
+        const int m = min(tile_m + 16 * pw + 8 * i + r7, p.M - 1);
+        a_ptr[i] = p.dq4 + (size_t)m * Kh + c * 16;
+        const int e = p.shift[m];
+        a_mul[i] = 1u << e;
+        a_off[i] = 0x01010101u * (uint32_t)(128 - (8 << e));
+      }
+      const uint8_t* b_ptr[NB_TASKS];
+#pragma unroll
+      for (int i = 0; i < NB_TASKS; ++i) {
+        const int n = min(tile_n + (BN / 8) * pw + 8 * i + r7, p.N - 1);
+        b_ptr[i] = p.wq4 + (size_t)n * Kh + c * 16;
+      }
+      // sparse word tasks of this warp's 16 rows: task t = lane + 32*j -> (row, word)
+      size_t sp_off[MAXT];
+      uint32_t sp_bank4[MAXT];
+#pragma unroll
+      for (int j = 0; j < MAXT; ++j) {
+        const int t = lane + 32 * j;
+        const int row_l = t >> nw_log, q = t & ((1 << nw_log) - 1);
+        const int m = min(tile_m + 16 * pw + (row_l & 15), p.M - 1);
+        sp_off[j] = (size_t)m * GK + 4 * q;
+        uint32_t b4 = 0;
+        if (word_path) {
+#pragma unroll
+          for (int u = 0; u < 4; ++u) b4 |= (uint32_t)(((4 * q + u) >> p.log2k) * p.b) << (8 * u);
+        }
+        sp_bank4[j] = b4;
+      }
+
+      uint4 ra[2][2], rb[2][NB_TASKS];  // [prefetch slot][task]
+      auto load_step = [&](int slot, int ks) {
+#pragma unroll
+        for (int i = 0; i < 2; ++i) ra[slot][i] = ldg_nc_v4(a_ptr[i] + (size_t)ks * 64);
+#pragma unroll
+        for (int i = 0; i < NB_TASKS; ++i) rb[slot][i] = ldg_nc_v4(b_ptr[i] + (size_t)ks * 64);
+      };
+      auto process = [&](int slot, int ks) -> bool {
+        const int s = it % NS;
+        if (!mbar_wait(bar_empty + 8 * s, ((it / NS) & 1u) ^ 1u, abort_flag)) return false;
+        uint8_t* a_st = sA + s * Smem<BN, NS>::kA;
+        uint8_t* b_st = sB + s * Smem<BN, NS>::kB;
+        // sparse words first: their latency hides behind the widening below
+        uint32_t sv[MAXT], si[MAXT];
+        if (word_path) {
+#pragma unroll
+          for (int j = 0; j < MAXT; ++j) {
+            if (j < ntask) {
+              const size_t o = sp_off[j] + (size_t)ks * nb;
+              sv[j] = __ldg(reinterpret_cast<const uint32_t*>(p.vals + o));
+              const int q4 = 4 * ((lane + 32 * j) & ((1 << nw_log) - 1));
+              si[j] = p.idx != nullptr ? __ldg(reinterpret_cast<const uint32_t*>(p.idx + o))
+                                       : __ldg(reinterpret_cast<const uint32_t*>(p.pos + (size_t)ks * nb + q4));
+            }
+          }
+        }
+        // ---- widen A: nibble -> u * 2^e + (128 - 8 * 2^e)
+#pragma unroll
+        for (int i = 0; i < 2; ++i) {
+          const uint32_t in[4] = {ra[slot][i].x, ra[slot][i].y, ra[slot][i].z, ra[slot][i].w};
+          uint32_t ev[4], od[4];
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            const uint32_t u = in[q] ^ 0x88888888u;
+            ev[q] = (u & 0x0F0F0F0Fu) * a_mul[i] + a_off[i];
+            od[q] = ((u >> 4) & 0x0F0F0F0Fu) * a_mul[i] + a_off[i];
+          }
+          uint8_t* dst = a_st + a_row0 + i * 1024;
+          *reinterpret_cast<uint4*>(dst + sw_even) = make_uint4(ev[0], ev[1], ev[2], ev[3]);
+          *reinterpret_cast<uint4*>(dst + (sw_even ^ 16u)) = make_uint4(od[0], od[1], od[2], od[3]);
+        }
+        // ---- widen B: nibble -> 16 * code
+#pragma unroll
+        for (int i = 0; i < NB_TASKS; ++i) {
+          const uint32_t in[4] = {rb[slot][i].x, rb[slot][i].y, rb[slot][i].z, rb[slot][i].w};
+          uint32_t ev[4], od[4];
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            ev[q] = (in[q] << 4) & 0xF0F0F0F0u;
+            od[q] = in[q] & 0xF0F0F0F0u;
+          }
+          uint8_t* dst = b_st + b_row0 + i * 1024;
+          *reinterpret_cast<uint4*>(dst + sw_even) = make_uint4(ev[0], ev[1], ev[2], ev[3]);
+          *reinterpret_cast<uint4*>(dst + (sw_even ^ 16u)) = make_uint4(od[0], od[1], od[2], od[3]);
+        }
+        __syncwarp();  // this warp's 16 A rows are complete before any lane overwrites bytes in them
+        // ---- sparse INT8 entries overwrite their places (rows 16*pw .. 16*pw+15 of the tile)
+        if (word_path) {
+#pragma unroll
+          for (int j = 0; j < MAXT; ++j) {
+            if (j < ntask) {
+              const int t = lane + 32 * j;
+              const int row = 16 * pw + ((t >> nw_log) & 15);
+              if ((t >> nw_log) < 16) {
+                const uint32_t r7s = 0x01010101u * (uint32_t)((row & 7) << 4);
+                const uint32_t pos4 = (kpos4(si[j]) + sp_bank4[j]) ^ r7s;
+                const uint32_t vx = sv[j] ^ 0x80808080u;
+                uint8_t* rowp = a_st + row * 128;
+#pragma unroll
+                for (int u = 0; u < 4; ++u) rowp[(pos4 >> (8 * u)) & 0xFFu] = (uint8_t)(vx >> (8 * u));
+              }
+            }
+          }
+        } else {
+          for (int t = lane; t < 16 * nb; t += 32) {
+            const int row_l = t / nb, i = t - row_l * nb;
+            const int row = 16 * pw + row_l;
+            const int m = min(tile_m + row, p.M - 1);
+            const int bank = i / p.k, slot_i = i - bank * p.k;
+            const int g = ks * (BK / p.b) + bank;
+            const size_t entry = (size_t)m * GK + (size_t)g * p.k + slot_i;
+            const uint32_t local = p.idx != nullptr ? p.idx[entry] : p.pos[(size_t)g * p.k + slot_i];
+            const uint32_t kp = (kpos1(local) + (uint32_t)(bank * p.b)) ^ (uint32_t)((row & 7) << 4);
+            a_st[row * 128 + kp] = (uint8_t)((uint8_t)p.vals[entry] ^ 0x80u);
+          }
+        }
+        fence_proxy_async_smem();  // generic-proxy writes -> visible to the tensor core's async reads
+        mbar_arrive(bar_full + 8 * s);
+        ++it;
+        return true;
+      };
+
+      bool ok = true;
+      load_step(0, 0);
+      if (KS > 1) load_step(1, 1);
+      for (int ks = 0; ks < KS && ok; ks += 2) {
+        ok = process(0, ks);
+        if (ok && ks + 2 < KS) load_step(0, ks + 2);
+        if (ok && ks + 1 < KS) {
+          ok = process(1, ks + 1);
+          if (ok && ks + 3 < KS) load_step(1, ks + 3);
+        }
+      }
       if (!ok) break;
     }
-    // ---- widen A: 128 rows x 4 packed chunks of 16 B (32 nibbles) -> two 16 B chunks each
-    for (int t = tid; t < BM * 4; t += kThreads) {
-      const int row = t >> 2, c = t & 3;
-      const int m = tile_m + row;
-      uint4 w = make_uint4(0, 0, 0, 0);
-      int e = 0;
-      if (m < p.M) {
-        w = ldg_nc_v4(p.dq4 + (size_t)m * Kh + (size_t)ks * 64 + c * 16);
-        e = p.shift[m];
-      }
-      const uint32_t off = 0x01010101u * (uint32_t)(128 - (8 << e));
-      const uint32_t in[4] = {w.x, w.y, w.z, w.w};
-      uint32_t ev[4], od[4];
+  } else if (warp == kMmaWarp) {
+    // =============================================================== MMA issuer
+    if (lane == 0) {
+      constexpr uint32_t idesc = make_idesc<BN>();
+      uint32_t it = 0, tc = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < ntiles && ok; tile += gridDim.x, ++tc) {
+        const uint32_t buf = tc & 1u;
+        ok = mbar_wait(bar_tempty + 8 * buf, ((tc >> 1) & 1u) ^ 1u, abort_flag);
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t d = tmem + buf * BN;
+        for (int ks = 0; ks < KS; ++ks, ++it) {
+          const int s = it % NS;
+          ok = mbar_wait(bar_full + 8 * s, (it / NS) & 1u, abort_flag);
+          if (!ok) break;
+          tc_fence_after();
+          const uint64_t da = make_desc(smem_u32(sA + s * Smem<BN, NS>::kA));
+          const uint64_t db = make_desc(smem_u32(sB + s * Smem<BN, NS>::kB));
 #pragma unroll
-      for (int q = 0; q < 4; ++q) {
-        const uint32_t u = in[q] ^ 0x88888888u;  // offset-binary nibbles
-        ev[q] = ((u & 0x0F0F0F0Fu) << e) + off;
-        od[q] = (((u >> 4) & 0x0F0F0F0Fu) << e) + off;
-      }
-      const uint32_t r7 = row & 7;
-      *reinterpret_cast<uint4*>(a_st + row * 128 + (((2 * c) ^ r7) << 4)) = make_uint4(ev[0], ev[1], ev[2], ev[3]);
-      *reinterpret_cast<uint4*>(a_st + row * 128 + (((2 * c + 1) ^ r7) << 4)) = make_uint4(od[0], od[1], od[2], od[3]);
-    }
-    // ---- widen B: BN rows x 4 packed chunks -> 16 * code
-    for (int t = tid; t < BN * 4; t += kThreads) {
-      const int row = t >> 2, c = t & 3;
-      const int n = tile_n + row;
-      uint4 w = make_uint4(0, 0, 0, 0);
-      if (n < p.N) w = ldg_nc_v4(p.wq4 + (size_t)n * Kh + (size_t)ks * 64 + c * 16);
-      const uint32_t in[4] = {w.x, w.y, w.z, w.w};
-      uint32_t ev[4], od[4];
-#pragma unroll
-      for (int q = 0; q < 4; ++q) {
-        ev[q] = (in[q] << 4) & 0xF0F0F0F0u;
-        od[q] = in[q] & 0xF0F0F0F0u;
-      }
-      const uint32_t r7 = row & 7;
-      *reinterpret_cast<uint4*>(b_st + row * 128 + (((2 * c) ^ r7) << 4)) = make_uint4(ev[0], ev[1], ev[2], ev[3]);
-      *reinterpret_cast<uint4*>(b_st + row * 128 + (((2 * c + 1) ^ r7) << 4)) = make_uint4(od[0], od[1], od[2], od[3]);
-    }
-    __syncthreads();
-    // ---- sparse INT8 entries overwrite their places in the widened A tile
-    for (int t = tid; t < BM * nb; t += kThreads) {
-      const int row = t / nb, i = t - row * nb;
-      const int m = tile_m + row;
-      if (m < p.M) {
-        const int bank = i / p.k;
-        const int g = ks * banks_per_step + bank;
-        const size_t entry = ((size_t)m * G + g) * p.k + (i - bank * p.k);
-        const int local = p.idx != nullptr ? p.idx[entry] : p.pos[(size_t)g * p.k + (i - bank * p.k)];
-        const uint32_t jj = (uint32_t)(bank * p.b + local);
-        a_st[swz((uint32_t)row, kpos(jj))] = (uint8_t)((uint8_t)p.vals[entry] ^ 0x80u);
+          for (int kk = 0; kk < BK / 32; ++kk)  // 32 bytes of K per MMA: +2 in 16-byte address units
+            umma_i8(d, da + 2 * kk, db + 2 * kk, idesc, (ks > 0 || kk > 0) ? 1u : 0u);
+          umma_commit(bar_empty + 8 * s);
+        }
+        if (ok) umma_commit(bar_tfull + 8 * buf);
       }
     }
-    fence_proxy_async_smem();  // generic-proxy writes -> visible to the tensor core's async reads
-    __syncthreads();
-    if (tid == 0) {
+    __syncwarp();
+  } else {
+    // =============================================================== epilogue
+    const int q = warp & 3;  // TMEM lane quarter this warp may read
+    uint32_t tc = 0;
+    for (int tile = blockIdx.x; tile < ntiles; tile += gridDim.x, ++tc) {
+      const int tile_m = (tile % tiles_m) * BM;
+      const int tile_n = (tile / tiles_m) * BN;
+      const uint32_t buf = tc & 1u;
+      if (!mbar_wait(bar_tfull + 8 * buf, (tc >> 1) & 1u, abort_flag)) break;
       tc_fence_after();
-      const uint64_t da = make_desc(smem_u32(a_st));
-      const uint64_t db = make_desc(smem_u32(b_st));
+      const int m = tile_m + 32 * q + lane;
+      const float sh = (m < p.M) ? p.s_hi[m] : 0.f;
+      for (int c0 = 0; c0 < BN; c0 += 32) {
+        uint32_t v[32];
+        tmem_ld32(tmem + ((uint32_t)(32 * q) << 16) + buf * BN + (uint32_t)c0, v);
+        tmem_ld_wait();
+        const int n0 = tile_n + c0;
+        if (m < p.M && n0 < p.N) {
 #pragma unroll
-      for (int kk = 0; kk < BK / 32; ++kk)  // 32 bytes of K per MMA: +2 in 16-byte address units
-        umma_i8(tmem, da + 2 * kk, db + 2 * kk, idesc, (ks > 0 || kk > 0) ? 1u : 0u);
-      umma_commit(bar_empty + 8 * s);
-      if (ks == KS - 1) umma_commit(bar_done);
-    }
-  }
-
-  if (ok) {
-    const bool w = mbar_wait(bar_done, 0, abort_flag);
-    ok = __syncthreads_and(w);
-  }
-  tc_fence_after();
-
-  if (ok) {
-    // ---- epilogue: warp w reads TMEM lanes 32*(w%4).., columns half (w/4)
-    const int q = warp & 3, h = warp >> 2;
-    const int m = tile_m + 32 * q + lane;
-    const float sh = (m < p.M) ? p.s_hi[m] : 0.f;
-    for (int c0 = h * (BN / 2); c0 < (h + 1) * (BN / 2); c0 += 32) {
-      uint32_t v[32];
-      tmem_ld32(tmem + ((uint32_t)(32 * q) << 16) + (uint32_t)c0, v);
-      tmem_ld_wait();
-      const int n0 = tile_n + c0;
-      if (m < p.M && n0 < p.N) {
+          for (int c8 = 0; c8 < 32; c8 += 8) {
+            if (n0 + c8 < p.N) {  // N % 8 == 0: a group of 8 columns is all in or all out
+              int acc[8];
+              uint32_t o[4];
+              const int4 cs0 = __ldg(reinterpret_cast<const int4*>(p.colsum + n0 + c8));
+              const int4 cs1 = __ldg(reinterpret_cast<const int4*>(p.colsum + n0 + c8 + 4));
+              const float4 sw0 = __ldg(reinterpret_cast<const float4*>(p.s_w + n0 + c8));
+              const float4 sw1 = __ldg(reinterpret_cast<const float4*>(p.s_w + n0 + c8 + 4));
+              const int cs[8] = {cs0.x, cs0.y, cs0.z, cs0.w, cs1.x, cs1.y, cs1.z, cs1.w};
+              const float sw[8] = {sw0.x, sw0.y, sw0.z, sw0.w, sw1.x, sw1.y, sw1.z, sw1.w};
 #pragma unroll
-        for (int c8 = 0; c8 < 32; c8 += 8) {
-          if (n0 + c8 < p.N) {  // N % 8 == 0: a group of 8 columns is all in or all out
-            int acc[8];
-            uint32_t o[4];
+              for (int cc = 0; cc < 8; ++cc) acc[cc] = ((int)v[c8 + cc] - 2048 * cs[cc]) >> 4;
 #pragma unroll
-            for (int c = 0; c < 8; ++c) {
-              const int n = n0 + c8 + c;
-              acc[c] = ((int)v[c8 + c] - 2048 * __ldg(p.colsum + n)) >> 4;
-            }
-#pragma unroll
-            for (int c = 0; c < 8; c += 2) {
-              const float f0 = ((float)acc[c] * sh) * __ldg(p.s_w + n0 + c8 + c);
-              const float f1 = ((float)acc[c + 1] * sh) * __ldg(p.s_w + n0 + c8 + c + 1);
-              o[c >> 1] = f32_to_bf16_bits(f0) | (f32_to_bf16_bits(f1) << 16);
-            }
-            *reinterpret_cast<uint4*>(p.out + (size_t)m * p.N + n0 + c8) = make_uint4(o[0], o[1], o[2], o[3]);
-            if (p.acc_out != nullptr) {
-              int4* dst = reinterpret_cast<int4*>(p.acc_out + (size_t)m * p.N + n0 + c8);
-              dst[0] = make_int4(acc[0], acc[1], acc[2], acc[3]);
-              dst[1] = make_int4(acc[4], acc[5], acc[6], acc[7]);
+              for (int cc = 0; cc < 8; cc += 2) {
+                const float f0 = ((float)acc[cc] * sh) * sw[cc];
+                const float f1 = ((float)acc[cc + 1] * sh) * sw[cc + 1];
+                o[cc >> 1] = f32_to_bf16_bits(f0) | (f32_to_bf16_bits(f1) << 16);
+              }
+              *reinterpret_cast<uint4*>(p.out + (size_t)m * p.N + n0 + c8) = make_uint4(o[0], o[1], o[2], o[3]);
+              if (p.acc_out != nullptr) {
+                int4* dst = reinterpret_cast<int4*>(p.acc_out + (size_t)m * p.N + n0 + c8);
+                dst[0] = make_int4(acc[0], acc[1], acc[2], acc[3]);
+                dst[1] = make_int4(acc[4], acc[5], acc[6], acc[7]);
+              }
             }
           }
         }
       }
+      tc_fence_before();
+      mbar_arrive(bar_tempty + 8 * buf);
     }
-  } else if (tid == 0) {
-    atomicExch(p.status, (int)SQ_ERR_TIMEOUT);
   }
 
   tc_fence_before();
   __syncthreads();
-  if (warp == 0) tmem_dealloc(tmem, BN);
+  if (tid == 0 && *abort_flag) atomicExch(p.status, (int)SQ_ERR_TIMEOUT);
+  if (warp == kMmaWarp) tmem_dealloc(tmem, 2 * BN);
 }
 
 cudaError_t launch_gemm(int b, int k, const sq_encoded& A, const sq_weights& W,
@@ -288,11 +417,39 @@ cudaError_t launch_gemm(int b, int k, const sq_encoded& A, const sq_weights& W,
   p.K = (int)K;
   p.b = b;
   p.k = k;
-  const int smem = Smem<BN, NS>::kBytes;
-  cudaError_t err = cudaFuncSetAttribute(gemm_kernel<BN, NS>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  // 32-bit word loads of the sparse entries need k a power of two, at least four entries per
+  // row per K step and 4-byte aligned row starts; anything else takes the byte-wise path.
+  const int nb = (BK / b) * k;
+  const int64_t GK = (K / b) * k;
+  const bool pow2 = (k & (k - 1)) == 0;
+  p.log2k = -1;
+  if (pow2 && nb >= 4 && GK % 4 == 0) {
+    int l = 0;
+    while ((1 << l) < k) ++l;
+    p.log2k = l;
+  }
+
+  static int sm_count[64] = {0};
+  int dev = 0;
+  cudaError_t err = cudaGetDevice(&dev);
   if (err != cudaSuccess) return err;
-  dim3 grid((unsigned)((N + BN - 1) / BN), (unsigned)((M + BM - 1) / BM));
-  gemm_kernel<BN, NS><<<grid, kThreads, smem, st>>>(p);
+  if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+  if (sm_count[dev] == 0) {
+    err = cudaDeviceGetAttribute(&sm_count[dev], cudaDevAttrMultiProcessorCount, dev);
+    if (err != cudaSuccess) return err;
+  }
+  const int64_t ntiles = ((M + BM - 1) / BM) * ((N + BN - 1) / BN);
+  const unsigned grid = (unsigned)(ntiles < sm_count[dev] ? ntiles : sm_count[dev]);
+  const int smem = Smem<BN, NS>::kBytes;
+  if (nb <= 16) {
+    err = cudaFuncSetAttribute(gemm_kernel<BN, NS, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (err != cudaSuccess) return err;
+    gemm_kernel<BN, NS, 2><<<grid, kThreads, smem, st>>>(p);
+  } else {
+    err = cudaFuncSetAttribute(gemm_kernel<BN, NS, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (err != cudaSuccess) return err;
+    gemm_kernel<BN, NS, 8><<<grid, kThreads, smem, st>>>(p);
+  }
   return cudaGetLastError();
 }
 
