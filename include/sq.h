@@ -101,8 +101,9 @@ typedef struct {
  *   s_w      float [N]       per-channel scale: wmax / 7
  *   colsum   int32 [N]       sum over K of the channel's INT4 codes
  *   w_sparse int8  [N, G*k]  static masks only: the codes of the selected input
- *                            channels gathered bank by bank (Algorithm 2's reorder),
- *                            w_sparse[n, g*k+i] = code[n, g*b + positions[g][i]];
+ *                            channels gathered bank by bank (Algorithm 2's reorder) and
+ *                            kept in sixteenths, the unit the GEMM's INT8 weight operand
+ *                            uses: w_sparse[n, g*k+i] = 16 * code[n, g*b + positions[g][i]];
  *                            NULL / unused when pos_mode == SQ_POS_DYNAMIC */
 typedef struct {
   uint8_t* wq4;

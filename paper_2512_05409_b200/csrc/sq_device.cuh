@@ -72,20 +72,44 @@ __device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity) {
   return ok != 0;
 }
 
-// Bounded wait: polls at most kSpinLimit times (with a short sleep once the fast
-// polls are used up, about a quarter of a second in total) and reports failure
-// instead of spinning forever.  `abort_flag` (shared memory) lets one role's
-// failure release every other role's wait.
-constexpr uint32_t kSpinFast = 2048;
-constexpr uint32_t kSpinLimit = 4u << 20;
+// try_wait lets the hardware park the warp until the phase completes or the time hint
+// (nanoseconds) runs out, so a waiting role does not burn issue slots.
+__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity, uint32_t hint_ns) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity), "r"(hint_ns)
+      : "memory");
+  return ok != 0;
+}
+
+// Bounded waits.  Both poll test_wait at most a fixed number of times and then report
+// failure instead of spinning forever; `abort_flag` (shared memory) lets one role's failure
+// release every other role's wait.
+//   mbar_wait       tight polling, for waits that are normally short (pipeline stages);
+//                   gives up after about a quarter of a second
+//   mbar_wait_idle  polls with a sleep in between, for roles that wait out a whole main
+//                   loop and should not take issue slots from the working warps
+constexpr uint32_t kSpinLimit = 1u << 24;
+constexpr uint32_t kIdleLimit = 1u << 21;
 
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
   for (uint32_t it = 0; it < kSpinLimit; ++it) {
     if (mbar_test(bar, parity)) return true;
-    if (it >= kSpinFast) {
-      if (*abort_flag) return false;
-      __nanosleep(64);
-    }
+    if ((it & 1023u) == 1023u && *abort_flag) return false;
+  }
+  *abort_flag = 1;
+  return false;
+}
+
+__device__ __forceinline__ bool mbar_wait_idle(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  for (uint32_t it = 0; it < kIdleLimit; ++it) {
+    if (mbar_test(bar, parity)) return true;
+    if (*abort_flag) return false;
+    __nanosleep(100);
   }
   *abort_flag = 1;
   return false;

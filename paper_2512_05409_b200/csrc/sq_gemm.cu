@@ -29,16 +29,35 @@
 // 128-byte swizzle (the 16-byte chunk index is XORed with row % 8), 8-row groups 1024
 // bytes apart: the canonical layout a tcgen05 shared-memory descriptor describes.
 //
+// Static positions take a second form of the sparse product (Section 3.3, Fig. 2b: the mask
+// only selects and gathers activation tiles because the weight rows were reordered offline):
+// vals [M, G*k] and w_sparse [N, G*k] are plain INT8 matrices, so the sparse product is
+// G*k/128 extra K steps whose tiles TMA writes straight into the same shared-memory stages
+// (swizzled by the TMA unit, no thread touches them) and whose MMAs (A signed this time, the
+// gathered weights already in sixteenths) accumulate into the same tensor-memory tile.
+//
 // Kernel organisation: persistent, one CTA per SM, warp-specialised.
 //   warps 0-7   producers: global loads (register-prefetched two K steps ahead), widening,
-//               sparse merge, stores into a ring of NS shared-memory stages
+//               sparse merge (dynamic positions), stores into a ring of NS shared-memory stages
 //   warp  8     one thread issues the MMAs and commits stage / accumulator barriers
 //   warps 9-12  epilogue: tcgen05.ld of one of two accumulator buffers, dequantise, store;
 //               overlaps the main loop of the next tile
+//   warp  13    one thread issues the TMA loads of the sparse K steps (static positions)
 // Every wait is bounded; a wait that runs out raises an abort flag that releases all
 // other waits, the kernel records SQ_ERR_TIMEOUT and frees its tensor memory.
+#include <cuda.h>
+#include <cudaTypedefs.h>
+#include <string.h>
+
 #include "sq_device.cuh"
 #include "sq_host.h"
+
+#ifndef SQ_SPARSE_PREFETCH
+#define SQ_SPARSE_PREFETCH 1
+#endif
+#ifndef SQ_E_PER_STEP
+#define SQ_E_PER_STEP 0
+#endif
 
 namespace sq {
 
@@ -49,9 +68,9 @@ constexpr int BK = 128;  // K elements per pipeline step = bytes per operand row
 constexpr int kProdWarps = 8;
 constexpr int kProdThreads = kProdWarps * 32;
 constexpr int kMmaWarp = kProdWarps;
-constexpr int kEpiWarp0 = kProdWarps + 1;
 constexpr int kEpiWarps = 4;
-constexpr int kThreads = (kProdWarps + 1 + kEpiWarps) * 32;
+constexpr int kTmaWarp = kProdWarps + 1 + kEpiWarps;
+constexpr int kThreads = (kProdWarps + 1 + kEpiWarps + 1) * 32;
 
 struct GemmParams {
   const uint8_t* dq4;
@@ -68,6 +87,7 @@ struct GemmParams {
   int* status;
   int M, N, K, b, k;
   int log2k;      // log2(k) when the word path is usable, else -1
+  int SS;         // sparse K steps per tile (static positions through TMA), else 0
 };
 
 // Shared-memory matrix descriptor: K-major, SWIZZLE_128B, 8-row groups 1024 B apart.
@@ -81,11 +101,11 @@ __device__ __forceinline__ uint64_t make_desc(uint32_t saddr) {
   return d;
 }
 
-// Instruction descriptor: D = s32, A = u8, B = s8, both K-major, M = 128, N = BN.
+// Instruction descriptor: D = s32, A = u8 or s8, B = s8, both K-major, M = 128, N = BN.
 template <int BN>
-__device__ __forceinline__ constexpr uint32_t make_idesc() {
+__device__ __forceinline__ constexpr uint32_t make_idesc(bool a_signed) {
   return (2u << 4)                       // D format: S32
-         | (0u << 7)                     // A format: unsigned 8-bit
+         | ((a_signed ? 1u : 0u) << 7)   // A format: 0 = unsigned, 1 = signed 8-bit
          | (1u << 10)                    // B format: signed 8-bit
          | ((uint32_t)(BN >> 3) << 17)   // N
          | ((uint32_t)(BM >> 4) << 24);  // M
@@ -109,8 +129,21 @@ __device__ __forceinline__ uint32_t kpos1(uint32_t jj) {
 
 }  // namespace
 
-template <int BN, int NS, int MAXT>
-__global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const GemmParams p) {
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+
+// 2-D tiled TMA load into this CTA's shared memory; x (bytes here) must be a multiple of 16.
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(dst),
+      "l"(map), "r"(x), "r"(y), "r"(bar)
+      : "memory");
+}
+
+template <int BN, int NS, int MAXT, bool STMA>
+__global__ void __launch_bounds__(kThreads, 1)
+    gemm_kernel(const GemmParams p, const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* smem = smem_raw + (base - smem_u32(smem_raw));
@@ -121,8 +154,9 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const GemmParams p) {
   const uint32_t bar_empty = bar_full + 8 * NS;
   const uint32_t bar_tfull = bar_empty + 8 * NS;  // 2 x 8 B
   const uint32_t bar_tempty = bar_tfull + 16;     // 2 x 8 B
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(sCtl + 16 * NS + 32);
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(sCtl + 16 * NS + 40);
+  const uint32_t bar_sfull = bar_tempty + 16;     // NS x 8 B: sparse K steps filled by TMA
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(sCtl + 24 * NS + 32);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(sCtl + 24 * NS + 40);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int KS = p.K / BK;
@@ -130,11 +164,13 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const GemmParams p) {
   const int tiles_m = (p.M + BM - 1) / BM;
   const int tiles_n = (p.N + BN - 1) / BN;
   const int ntiles = tiles_m * tiles_n;
+  const int SS = STMA ? p.SS : 0;  // sparse K steps that follow the KS dense steps of every tile
 
   if (tid == 0) {
     for (int s = 0; s < NS; ++s) {
       mbar_init(bar_full + 8 * s, kProdThreads);
       mbar_init(bar_empty + 8 * s, 1);
+      mbar_init(bar_sfull + 8 * s, 1);
     }
     for (int bq = 0; bq < 2; ++bq) {
       mbar_init(bar_tfull + 8 * bq, 1);
@@ -163,157 +199,227 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const GemmParams p) {
     constexpr int NB_TASKS = BN / 64;                                // B chunks per thread per step
     const int GK = (p.K / p.b) * p.k;
     const int nb = (BK / p.b) * p.k;  // sparse entries per row per K step
-    const bool word_path = p.log2k >= 0;
+    const bool word_path = !STMA && p.log2k >= 0;
     const int nw_log = word_path ? (31 - __clz(nb >> 2)) : 0;  // log2(words per row per step)
     const int ntask = word_path ? ((16 << nw_log) + 31) >> 5 : 0;
 
-    uint32_t it = 0;
-    for (int tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
-      const int tile_m = (tile % tiles_m) * BM;
-      const int tile_n = (tile / tiles_m) * BN;
-      const uint8_t* a_ptr[2];
-      uint32_t a_mul[2], a_off[2];
+    // tile-independent part of this lane's sparse word tasks: task t = lane + 32*j covers
+    // word (t mod words-per-row) of row (t div words-per-row) of the warp's 16 rows
+    uint32_t sp_bank4[MAXT];
+#pragma unroll
+    for (int j = 0; j < MAXT; ++j) {
+      const int q = (lane + 32 * j) & ((1 << nw_log) - 1);
+      uint32_t b4 = 0;
+      if (word_path) {
+#pragma unroll
+        for (int u = 0; u < 4; ++u) b4 |= (uint32_t)(((4 * q + u) >> p.log2k) * p.b) << (8 * u);
+      }
+      sp_bank4[j] = b4;
+    }
+
+    // ---- load side: runs two K steps ahead of the processing side, across tile boundaries
+    int lt = blockIdx.x, lks = 0;
+    const uint8_t* a_ptr[2];
+    const uint8_t* e_ptr[2];
+    const uint8_t* b_ptr[NB_TASKS];
+    size_t sp_off[MAXT];
+    auto set_load_tile = [&]() {
+      const int tile_m = (lt % tiles_m) * BM;
+      const int tile_n = (lt / tiles_m) * BN;
 #pragma unroll
       for (int i = 0; i < 2; ++i) {
-        const int m = min(tile_m + 16 * pw + 8 * i + r7, p.M - 1);
+        const int m = min(tile_m + 16 * pw + 8 * i + r7, p.M - 1);  // rows past M repeat the last row
         a_ptr[i] = p.dq4 + (size_t)m * Kh + c * 16;
-        const int e = p.shift[m];
-        a_mul[i] = 1u << e;
-        a_off[i] = 0x01010101u * (uint32_t)(128 - (8 << e));
+        e_ptr[i] = p.shift + m;
       }
-      const uint8_t* b_ptr[NB_TASKS];
 #pragma unroll
       for (int i = 0; i < NB_TASKS; ++i) {
         const int n = min(tile_n + (BN / 8) * pw + 8 * i + r7, p.N - 1);
         b_ptr[i] = p.wq4 + (size_t)n * Kh + c * 16;
       }
-      // sparse word tasks of this warp's 16 rows: task t = lane + 32*j -> (row, word)
-      size_t sp_off[MAXT];
-      uint32_t sp_bank4[MAXT];
 #pragma unroll
       for (int j = 0; j < MAXT; ++j) {
         const int t = lane + 32 * j;
-        const int row_l = t >> nw_log, q = t & ((1 << nw_log) - 1);
-        const int m = min(tile_m + 16 * pw + (row_l & 15), p.M - 1);
-        sp_off[j] = (size_t)m * GK + 4 * q;
-        uint32_t b4 = 0;
-        if (word_path) {
-#pragma unroll
-          for (int u = 0; u < 4; ++u) b4 |= (uint32_t)(((4 * q + u) >> p.log2k) * p.b) << (8 * u);
-        }
-        sp_bank4[j] = b4;
+        const int m = min(tile_m + 16 * pw + ((t >> nw_log) & 15), p.M - 1);
+        sp_off[j] = (size_t)m * GK + 4 * (t & ((1 << nw_log) - 1));
       }
-
-      uint4 ra[2][2], rb[2][NB_TASKS];  // [prefetch slot][task]
-      auto load_step = [&](int slot, int ks) {
+    };
+    uint4 ra[2][2], rb[2][NB_TASKS];  // [prefetch slot][task]
+    uint32_t re[2][2], sv[2][MAXT], si[2][MAXT];
+    auto load_next = [&](int slot) {
+      if (lt >= ntiles) return;
 #pragma unroll
-        for (int i = 0; i < 2; ++i) ra[slot][i] = ldg_nc_v4(a_ptr[i] + (size_t)ks * 64);
+      for (int i = 0; i < 2; ++i) {
+        ra[slot][i] = ldg_nc_v4(a_ptr[i] + (size_t)lks * 64);
+#if SQ_E_PER_STEP
+        re[slot][i] = __ldg(e_ptr[i]);
+#endif
+      }
 #pragma unroll
-        for (int i = 0; i < NB_TASKS; ++i) rb[slot][i] = ldg_nc_v4(b_ptr[i] + (size_t)ks * 64);
-      };
-      auto process = [&](int slot, int ks) -> bool {
-        const int s = it % NS;
-        if (!mbar_wait(bar_empty + 8 * s, ((it / NS) & 1u) ^ 1u, abort_flag)) return false;
-        uint8_t* a_st = sA + s * Smem<BN, NS>::kA;
-        uint8_t* b_st = sB + s * Smem<BN, NS>::kB;
-        // sparse words first: their latency hides behind the widening below
-        uint32_t sv[MAXT], si[MAXT];
-        if (word_path) {
+      for (int i = 0; i < NB_TASKS; ++i) rb[slot][i] = ldg_nc_v4(b_ptr[i] + (size_t)lks * 64);
+#if SQ_SPARSE_PREFETCH
+      if (word_path) {
 #pragma unroll
-          for (int j = 0; j < MAXT; ++j) {
-            if (j < ntask) {
-              const size_t o = sp_off[j] + (size_t)ks * nb;
-              sv[j] = __ldg(reinterpret_cast<const uint32_t*>(p.vals + o));
-              const int q4 = 4 * ((lane + 32 * j) & ((1 << nw_log) - 1));
-              si[j] = p.idx != nullptr ? __ldg(reinterpret_cast<const uint32_t*>(p.idx + o))
-                                       : __ldg(reinterpret_cast<const uint32_t*>(p.pos + (size_t)ks * nb + q4));
-            }
+        for (int j = 0; j < MAXT; ++j) {
+          if (j < ntask) {
+            const size_t o = sp_off[j] + (size_t)lks * nb;
+            sv[slot][j] = __ldg(reinterpret_cast<const uint32_t*>(p.vals + o));
+            const int q4 = 4 * ((lane + 32 * j) & ((1 << nw_log) - 1));
+            si[slot][j] = p.idx != nullptr
+                              ? __ldg(reinterpret_cast<const uint32_t*>(p.idx + o))
+                              : __ldg(reinterpret_cast<const uint32_t*>(p.pos + (size_t)lks * nb + q4));
           }
         }
-        // ---- widen A: nibble -> u * 2^e + (128 - 8 * 2^e)
+      }
+#endif
+      if (++lks == KS) {
+        lks = 0;
+        lt += gridDim.x;
+        if (lt < ntiles) set_load_tile();
+      }
+    };
+
+    // ---- processing side
+    uint32_t it = 0;
+    uint32_t pmul[2] = {1, 1}, poff[2] = {0, 0};
+    int pt = blockIdx.x, pks = 0;  // tile and K step being processed (the byte-wise path needs them)
+    auto process = [&](int slot) -> bool {
+      const int s = it % NS;
+      if (!mbar_wait(bar_empty + 8 * s, ((it / NS) & 1u) ^ 1u, abort_flag)) return false;
+      uint8_t* a_st = sA + s * Smem<BN, NS>::kA;
+      uint8_t* b_st = sB + s * Smem<BN, NS>::kB;
+#if !SQ_SPARSE_PREFETCH
+      if (word_path) {
+        const int tile_m = (pt % tiles_m) * BM;
+#pragma unroll
+        for (int j = 0; j < MAXT; ++j) {
+          if (j < ntask) {
+            const int t = lane + 32 * j;
+            const int m = min(tile_m + 16 * pw + ((t >> nw_log) & 15), p.M - 1);
+            const int q4 = 4 * (t & ((1 << nw_log) - 1));
+            const size_t o = (size_t)m * GK + q4 + (size_t)pks * nb;
+            sv[slot][j] = __ldg(reinterpret_cast<const uint32_t*>(p.vals + o));
+            si[slot][j] = p.idx != nullptr
+                              ? __ldg(reinterpret_cast<const uint32_t*>(p.idx + o))
+                              : __ldg(reinterpret_cast<const uint32_t*>(p.pos + (size_t)pks * nb + q4));
+          }
+        }
+      }
+#endif
+#if !SQ_E_PER_STEP
+      if (pks == 0) {  // the rows' shifts change with the tile only
+        const int tile_m = (pt % tiles_m) * BM;
 #pragma unroll
         for (int i = 0; i < 2; ++i) {
-          const uint32_t in[4] = {ra[slot][i].x, ra[slot][i].y, ra[slot][i].z, ra[slot][i].w};
-          uint32_t ev[4], od[4];
-#pragma unroll
-          for (int q = 0; q < 4; ++q) {
-            const uint32_t u = in[q] ^ 0x88888888u;
-            ev[q] = (u & 0x0F0F0F0Fu) * a_mul[i] + a_off[i];
-            od[q] = ((u >> 4) & 0x0F0F0F0Fu) * a_mul[i] + a_off[i];
-          }
-          uint8_t* dst = a_st + a_row0 + i * 1024;
-          *reinterpret_cast<uint4*>(dst + sw_even) = make_uint4(ev[0], ev[1], ev[2], ev[3]);
-          *reinterpret_cast<uint4*>(dst + (sw_even ^ 16u)) = make_uint4(od[0], od[1], od[2], od[3]);
-        }
-        // ---- widen B: nibble -> 16 * code
-#pragma unroll
-        for (int i = 0; i < NB_TASKS; ++i) {
-          const uint32_t in[4] = {rb[slot][i].x, rb[slot][i].y, rb[slot][i].z, rb[slot][i].w};
-          uint32_t ev[4], od[4];
-#pragma unroll
-          for (int q = 0; q < 4; ++q) {
-            ev[q] = (in[q] << 4) & 0xF0F0F0F0u;
-            od[q] = in[q] & 0xF0F0F0F0u;
-          }
-          uint8_t* dst = b_st + b_row0 + i * 1024;
-          *reinterpret_cast<uint4*>(dst + sw_even) = make_uint4(ev[0], ev[1], ev[2], ev[3]);
-          *reinterpret_cast<uint4*>(dst + (sw_even ^ 16u)) = make_uint4(od[0], od[1], od[2], od[3]);
-        }
-        __syncwarp();  // this warp's 16 A rows are complete before any lane overwrites bytes in them
-        // ---- sparse INT8 entries overwrite their places (rows 16*pw .. 16*pw+15 of the tile)
-        if (word_path) {
-#pragma unroll
-          for (int j = 0; j < MAXT; ++j) {
-            if (j < ntask) {
-              const int t = lane + 32 * j;
-              const int row = 16 * pw + ((t >> nw_log) & 15);
-              if ((t >> nw_log) < 16) {
-                const uint32_t r7s = 0x01010101u * (uint32_t)((row & 7) << 4);
-                const uint32_t pos4 = (kpos4(si[j]) + sp_bank4[j]) ^ r7s;
-                const uint32_t vx = sv[j] ^ 0x80808080u;
-                uint8_t* rowp = a_st + row * 128;
-#pragma unroll
-                for (int u = 0; u < 4; ++u) rowp[(pos4 >> (8 * u)) & 0xFFu] = (uint8_t)(vx >> (8 * u));
-              }
-            }
-          }
-        } else {
-          for (int t = lane; t < 16 * nb; t += 32) {
-            const int row_l = t / nb, i = t - row_l * nb;
-            const int row = 16 * pw + row_l;
-            const int m = min(tile_m + row, p.M - 1);
-            const int bank = i / p.k, slot_i = i - bank * p.k;
-            const int g = ks * (BK / p.b) + bank;
-            const size_t entry = (size_t)m * GK + (size_t)g * p.k + slot_i;
-            const uint32_t local = p.idx != nullptr ? p.idx[entry] : p.pos[(size_t)g * p.k + slot_i];
-            const uint32_t kp = (kpos1(local) + (uint32_t)(bank * p.b)) ^ (uint32_t)((row & 7) << 4);
-            a_st[row * 128 + kp] = (uint8_t)((uint8_t)p.vals[entry] ^ 0x80u);
-          }
-        }
-        fence_proxy_async_smem();  // generic-proxy writes -> visible to the tensor core's async reads
-        mbar_arrive(bar_full + 8 * s);
-        ++it;
-        return true;
-      };
-
-      bool ok = true;
-      load_step(0, 0);
-      if (KS > 1) load_step(1, 1);
-      for (int ks = 0; ks < KS && ok; ks += 2) {
-        ok = process(0, ks);
-        if (ok && ks + 2 < KS) load_step(0, ks + 2);
-        if (ok && ks + 1 < KS) {
-          ok = process(1, ks + 1);
-          if (ok && ks + 3 < KS) load_step(1, ks + 3);
+          const uint32_t e = p.shift[min(tile_m + 16 * pw + 8 * i + r7, p.M - 1)];
+          pmul[i] = 1u << e;
+          poff[i] = 0x01010101u * (128u - (8u << e));
         }
       }
-      if (!ok) break;
+#endif
+      // ---- widen A: nibble -> u * 2^e + (128 - 8 * 2^e)
+#pragma unroll
+      for (int i = 0; i < 2; ++i) {
+        const uint32_t in[4] = {ra[slot][i].x, ra[slot][i].y, ra[slot][i].z, ra[slot][i].w};
+#if SQ_E_PER_STEP
+        const uint32_t a_mul = 1u << re[slot][i];
+        const uint32_t a_off = 0x01010101u * (128u - (8u << re[slot][i]));
+#else
+        const uint32_t a_mul = pmul[i], a_off = poff[i];
+#endif
+        uint32_t ev[4], od[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          const uint32_t u = in[q] ^ 0x88888888u;
+          ev[q] = (u & 0x0F0F0F0Fu) * a_mul + a_off;
+          od[q] = ((u >> 4) & 0x0F0F0F0Fu) * a_mul + a_off;
+        }
+        uint8_t* dst = a_st + a_row0 + i * 1024;
+        *reinterpret_cast<uint4*>(dst + sw_even) = make_uint4(ev[0], ev[1], ev[2], ev[3]);
+        *reinterpret_cast<uint4*>(dst + (sw_even ^ 16u)) = make_uint4(od[0], od[1], od[2], od[3]);
+      }
+      // ---- widen B: nibble -> 16 * code
+#pragma unroll
+      for (int i = 0; i < NB_TASKS; ++i) {
+        const uint32_t in[4] = {rb[slot][i].x, rb[slot][i].y, rb[slot][i].z, rb[slot][i].w};
+        uint32_t ev[4], od[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          ev[q] = (in[q] << 4) & 0xF0F0F0F0u;
+          od[q] = in[q] & 0xF0F0F0F0u;
+        }
+        uint8_t* dst = b_st + b_row0 + i * 1024;
+        *reinterpret_cast<uint4*>(dst + sw_even) = make_uint4(ev[0], ev[1], ev[2], ev[3]);
+        *reinterpret_cast<uint4*>(dst + (sw_even ^ 16u)) = make_uint4(od[0], od[1], od[2], od[3]);
+      }
+      __syncwarp();  // this warp's 16 A rows are complete before any lane overwrites bytes in them
+      // ---- sparse INT8 entries overwrite their places (rows 16*pw .. 16*pw+15 of the tile)
+      if (word_path) {
+#pragma unroll
+        for (int j = 0; j < MAXT; ++j) {
+          if (j < ntask) {
+            const int t = lane + 32 * j;
+            if ((t >> nw_log) < 16) {
+              const int row = 16 * pw + (t >> nw_log);
+              const uint32_t r7s = 0x01010101u * (uint32_t)((row & 7) << 4);
+              const uint32_t pos4 = (kpos4(si[slot][j]) + sp_bank4[j]) ^ r7s;
+              const uint32_t vx = sv[slot][j] ^ 0x80808080u;
+              uint8_t* rowp = a_st + row * 128;
+#pragma unroll
+              for (int u = 0; u < 4; ++u) rowp[(pos4 >> (8 * u)) & 0xFFu] = (uint8_t)(vx >> (8 * u));
+            }
+          }
+        }
+      } else if (!STMA) {
+        const int tile_m = (pt % tiles_m) * BM;
+        for (int t = lane; t < 16 * nb; t += 32) {
+          const int row_l = t / nb, i = t - row_l * nb;
+          const int row = 16 * pw + row_l;
+          const int m = min(tile_m + row, p.M - 1);
+          const int bank = i / p.k, slot_i = i - bank * p.k;
+          const int g = pks * (BK / p.b) + bank;
+          const size_t entry = (size_t)m * GK + (size_t)g * p.k + slot_i;
+          const uint32_t local = p.idx != nullptr ? p.idx[entry] : p.pos[(size_t)g * p.k + slot_i];
+          const uint32_t kp = (kpos1(local) + (uint32_t)(bank * p.b)) ^ (uint32_t)((row & 7) << 4);
+          a_st[row * 128 + kp] = (uint8_t)((uint8_t)p.vals[entry] ^ 0x80u);
+        }
+      }
+      fence_proxy_async_smem();  // generic-proxy writes -> visible to the tensor core's async reads
+      mbar_arrive(bar_full + 8 * s);
+      ++it;
+      if (++pks == KS) {
+        pks = 0;
+        pt += gridDim.x;
+        // The sparse K steps of the tile use the next SS ring slots (TMA fills them).  They are
+        // waited for one by one, not skipped: a parity wait only tells the current phase from
+        // the previous one, so no role may fall more than one use behind on any stage.
+        for (int ss = 0; ss < SS; ++ss, ++it) {
+          if (!mbar_wait(bar_empty + 8 * (it % NS), ((it / NS) & 1u) ^ 1u, abort_flag)) return false;
+        }
+      }
+      return true;
+    };
+
+    const int my_tiles = (ntiles - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
+    const int total = my_tiles * KS;
+    set_load_tile();
+    load_next(0);
+    load_next(1);
+    for (int g = 0; g < total; g += 2) {
+      if (!process(0)) break;
+      load_next(0);
+      if (g + 1 < total) {
+        if (!process(1)) break;
+        load_next(1);
+      }
     }
   } else if (warp == kMmaWarp) {
     // =============================================================== MMA issuer
     if (lane == 0) {
-      constexpr uint32_t idesc = make_idesc<BN>();
+      constexpr uint32_t idesc = make_idesc<BN>(false);
+      constexpr uint32_t idesc_sparse = make_idesc<BN>(true);
       uint32_t it = 0, tc = 0;
+      uint32_t ph_dense = 0, ph_sparse = 0;  // per-stage phase bits of the two kinds of "full" barrier
       bool ok = true;
       for (int tile = blockIdx.x; tile < ntiles && ok; tile += gridDim.x, ++tc) {
         const uint32_t buf = tc & 1u;
@@ -321,19 +427,49 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const GemmParams p) {
         if (!ok) break;
         tc_fence_after();
         const uint32_t d = tmem + buf * BN;
-        for (int ks = 0; ks < KS; ++ks, ++it) {
+        for (int ks = 0; ks < KS + SS; ++ks, ++it) {
           const int s = it % NS;
-          ok = mbar_wait(bar_full + 8 * s, (it / NS) & 1u, abort_flag);
+          const bool sparse_step = ks >= KS;
+          if (!sparse_step) {
+            ok = mbar_wait(bar_full + 8 * s, (ph_dense >> s) & 1u, abort_flag);
+            ph_dense ^= 1u << s;
+          } else {
+            ok = mbar_wait(bar_sfull + 8 * s, (ph_sparse >> s) & 1u, abort_flag);
+            ph_sparse ^= 1u << s;
+          }
           if (!ok) break;
           tc_fence_after();
           const uint64_t da = make_desc(smem_u32(sA + s * Smem<BN, NS>::kA));
           const uint64_t db = make_desc(smem_u32(sB + s * Smem<BN, NS>::kB));
+          const uint32_t id = sparse_step ? idesc_sparse : idesc;
 #pragma unroll
           for (int kk = 0; kk < BK / 32; ++kk)  // 32 bytes of K per MMA: +2 in 16-byte address units
-            umma_i8(d, da + 2 * kk, db + 2 * kk, idesc, (ks > 0 || kk > 0) ? 1u : 0u);
+            umma_i8(d, da + 2 * kk, db + 2 * kk, id, (ks > 0 || kk > 0) ? 1u : 0u);
           umma_commit(bar_empty + 8 * s);
         }
         if (ok) umma_commit(bar_tfull + 8 * buf);
+      }
+    }
+    __syncwarp();
+  } else if (warp == kTmaWarp) {
+    // =============================================================== TMA (sparse K steps)
+    if (STMA && lane == 0) {
+      uint32_t tc = 0, it = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < ntiles && ok; tile += gridDim.x, ++tc) {
+        const int tile_m = (tile % tiles_m) * BM;
+        const int tile_n = (tile / tiles_m) * BN;
+        // every ring slot is waited for in order (see the producers); only the sparse ones are filled
+        for (int step = 0; step < KS + SS && ok; ++step, ++it) {
+          const int s = it % NS;
+          ok = mbar_wait(bar_empty + 8 * s, ((it / NS) & 1u) ^ 1u, abort_flag);
+          if (!ok || step < KS) continue;
+          const int ss = step - KS;
+          // rows past M / N and columns past G*k are filled with zeros by the TMA unit
+          mbar_expect_tx(bar_sfull + 8 * s, (uint32_t)(Smem<BN, NS>::kA + Smem<BN, NS>::kB));
+          tma_load_2d(smem_u32(sA + s * Smem<BN, NS>::kA), &map_a, ss * BK, tile_m, bar_sfull + 8 * s);
+          tma_load_2d(smem_u32(sB + s * Smem<BN, NS>::kB), &map_b, ss * BK, tile_n, bar_sfull + 8 * s);
+        }
       }
     }
     __syncwarp();
@@ -345,7 +481,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const GemmParams p) {
       const int tile_m = (tile % tiles_m) * BM;
       const int tile_n = (tile / tiles_m) * BN;
       const uint32_t buf = tc & 1u;
-      if (!mbar_wait(bar_tfull + 8 * buf, (tc >> 1) & 1u, abort_flag)) break;
+      if (!mbar_wait_idle(bar_tfull + 8 * buf, (tc >> 1) & 1u, abort_flag)) break;
       tc_fence_after();
       const int m = tile_m + 32 * q + lane;
       const float sh = (m < p.M) ? p.s_hi[m] : 0.f;
@@ -441,15 +577,53 @@ cudaError_t launch_gemm(int b, int k, const sq_encoded& A, const sq_weights& W,
   const int64_t ntiles = ((M + BM - 1) / BM) * ((N + BN - 1) / BN);
   const unsigned grid = (unsigned)(ntiles < sm_count[dev] ? ntiles : sm_count[dev]);
   const int smem = Smem<BN, NS>::kBytes;
-  if (nb <= 16) {
-    err = cudaFuncSetAttribute(gemm_kernel<BN, NS, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-    if (err != cudaSuccess) return err;
-    gemm_kernel<BN, NS, 2><<<grid, kThreads, smem, st>>>(p);
-  } else {
-    err = cudaFuncSetAttribute(gemm_kernel<BN, NS, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-    if (err != cudaSuccess) return err;
-    gemm_kernel<BN, NS, 8><<<grid, kThreads, smem, st>>>(p);
+
+  // Static positions: the sparse product runs as extra K steps over vals [M, G*k] and
+  // w_sparse [N, G*k], fetched by TMA.  A TMA row pitch must be a multiple of 16 bytes; any
+  // other G*k falls back to merging the entries into the dense tile like dynamic positions.
+  CUtensorMap map_a, map_b;
+  memset(&map_a, 0, sizeof(map_a));
+  memset(&map_b, 0, sizeof(map_b));
+  p.SS = 0;
+  const bool stma = positions != nullptr && GK % 16 == 0;
+  if (stma) {
+    static PFN_cuTensorMapEncodeTiled encode = nullptr;
+    if (encode == nullptr) {
+      void* fn = nullptr;
+      cudaDriverEntryPointQueryResult qres;
+      err = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
+      if (err != cudaSuccess) return err;
+      if (fn == nullptr || qres != cudaDriverEntryPointSuccess) return cudaErrorNotSupported;
+      encode = reinterpret_cast<PFN_cuTensorMapEncodeTiled>(fn);
+    }
+    const cuuint32_t estr[2] = {1, 1};
+    const cuuint64_t pitch[1] = {(cuuint64_t)GK};
+    const cuuint64_t dim_a[2] = {(cuuint64_t)GK, (cuuint64_t)M};
+    const cuuint64_t dim_b[2] = {(cuuint64_t)GK, (cuuint64_t)N};
+    const cuuint32_t box_a[2] = {BK, BM};
+    const cuuint32_t box_b[2] = {BK, BN};
+    if (encode(&map_a, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<int8_t*>(A.vals), dim_a, pitch, box_a, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+      return cudaErrorInvalidValue;
+    if (encode(&map_b, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, W.w_sparse, dim_b, pitch, box_b, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+      return cudaErrorInvalidValue;
+    p.SS = (int)((GK + BK - 1) / BK);
   }
+
+#define SQ_LAUNCH_GEMM(MAXT_, STMA_)                                                                  \
+  do {                                                                                                \
+    err = cudaFuncSetAttribute(gemm_kernel<BN, NS, MAXT_, STMA_>,                                     \
+                               cudaFuncAttributeMaxDynamicSharedMemorySize, smem);                    \
+    if (err != cudaSuccess) return err;                                                               \
+    gemm_kernel<BN, NS, MAXT_, STMA_><<<grid, kThreads, smem, st>>>(p, map_a, map_b);                 \
+  } while (0)
+  if (stma) SQ_LAUNCH_GEMM(1, true);
+  else if (nb <= 16) SQ_LAUNCH_GEMM(2, false);
+  else SQ_LAUNCH_GEMM(8, false);
+#undef SQ_LAUNCH_GEMM
   return cudaGetLastError();
 }
 

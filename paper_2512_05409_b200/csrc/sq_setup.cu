@@ -117,7 +117,7 @@ __global__ void __launch_bounds__(256) pack_weights_kernel(int b, int k, const u
       const int64_t g = t / k;
       const int64_t j = g * b + positions[t];
       const int q = min(7, max(-7, rne_prod(bf16_bits_to_f32(row[j]), c)));
-      w_sparse[n * GK + t] = (int8_t)q;
+      w_sparse[n * GK + t] = (int8_t)(16 * q);  // sixteenths: the GEMM's weight operand unit
     }
   }
 }
