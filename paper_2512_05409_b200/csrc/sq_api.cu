@@ -169,8 +169,10 @@ sq_status sq_encode(const sq_format* fmt, const void* X_bf16, int64_t M, int64_t
   SQ_TRY(check_positions(fmt, positions));
   SQ_TRY(check_encoded(fmt, out));
   SQ_TRY(check_device());
+  int* status = status_word();
+  if (status == nullptr) return SQ_ERR_CUDA;
   return from_cuda(launch_encode(fmt->bank, fmt->k, fmt->pos_mode == SQ_POS_STATIC,
-                                 static_cast<const uint16_t*>(X_bf16), M, K, positions, *out,
+                                 static_cast<const uint16_t*>(X_bf16), M, K, positions, *out, status,
                                  static_cast<cudaStream_t>(cuda_stream)));
 }
 

@@ -105,6 +105,20 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
   return false;
 }
 
+// mbar_wait_park: the hardware parks the warp (try_wait with a time hint) instead of polling;
+// for waits on data in flight from HBM, where a microsecond of wake-up slack costs nothing but
+// polling would take issue slots from the warps that have work.  Bounded like the others.
+constexpr uint32_t kParkTries = 1u << 17;
+__device__ __forceinline__ bool mbar_wait_park(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  if (mbar_test(bar, parity)) return true;
+  for (uint32_t it = 0; it < kParkTries; ++it) {
+    if (mbar_try(bar, parity, 2000u)) return true;
+    if (*abort_flag) return false;
+  }
+  *abort_flag = 1;
+  return false;
+}
+
 __device__ __forceinline__ bool mbar_wait_idle(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
   for (uint32_t it = 0; it < kIdleLimit; ++it) {
     if (mbar_test(bar, parity)) return true;

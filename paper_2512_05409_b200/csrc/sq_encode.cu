@@ -1,4 +1,27 @@
 // Activation encode (bf16 -> SQ-format) and decode (SQ-format -> bf16).
+//
+// Encode is one pass over HBM: 2 B read and 0.5 + 2k/b B (dynamic) or 0.5 + k/b B (static)
+// written per element.  The scale of a row is its maximum, so a row must be seen in full
+// before anything can be quantised: a GROUP of 1-16 warps owns one token row at a time,
+// staged in shared memory by one bulk asynchronous copy (double-buffered when two rows
+// fit); the host picks the group size so that a block of 16 warps (8 for b = 128) keeps as
+// many rows in flight as shared memory allows.  Groups synchronise on their own named
+// barrier, never block-wide.
+//
+//   phase 1  (dynamic) each lane owns whole banks.  The k-th largest magnitude of a bank is
+//            found with a sorting network on packed bf16x2 magnitudes (two columns at once;
+//            sorted runs of k merged with truncation), then one compare pass builds the
+//            selection mask and the largest unselected magnitude; equal magnitudes at the
+//            threshold are resolved towards the lower index.
+//            (static) the given positions are copied out and zeroed in the staged row.
+//   reduce   row maximum and largest unselected magnitude over the group -> inv, s_hi,
+//            shift e, s_lo
+//   phase 2  selected values -> INT8 in ascending position (and their indices), zeroed in
+//            the staged row; then the whole row -> INT4, eight codes per 32-bit word, in a
+//            coalesced sweep (the zeroed places give the zero nibbles the format asks for).
+//
+// Formats outside the fast kernels' set (k not a power of two, k/b other than 1/2 .. 1/16 for
+// dynamic positions) take a plain one-block-per-row kernel that ranks every element.
 #include "sq_device.cuh"
 #include "sq_host.h"
 
@@ -18,10 +41,507 @@ __device__ __forceinline__ uint32_t block_max_u32(uint32_t v, uint32_t* scratch)
   return r;
 }
 
+__device__ __forceinline__ uint32_t warp_max_u32(uint32_t v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = max(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+
+// packed bf16x2 helpers on raw 32-bit registers (magnitudes: non-negative, finite)
+__device__ __forceinline__ uint32_t max2(uint32_t a, uint32_t b) {
+  uint32_t d;
+  asm("max.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+  return d;
+}
+__device__ __forceinline__ uint32_t min2(uint32_t a, uint32_t b) {
+  uint32_t d;
+  asm("min.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+  return d;
+}
+__device__ __forceinline__ uint32_t ge2_mask(uint32_t a, uint32_t b) {  // 0xFFFF per half where a >= b
+  uint32_t d;
+  asm("set.ge.u32.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+  return d;
+}
+__device__ __forceinline__ uint32_t swap_halves(uint32_t a) { return __byte_perm(a, a, 0x1032); }
+
+// compare-exchange, larger first
+__device__ __forceinline__ void ce(uint32_t& a, uint32_t& b) {
+  const uint32_t hi = max2(a, b), lo = min2(a, b);
+  a = hi;
+  b = lo;
+}
+
+// Batcher's odd-even merge sort of r[0..N), descending, both bf16 columns at once.
+template <int N>
+__device__ __forceinline__ void sort_desc(uint32_t* r) {
+#pragma unroll
+  for (int p = 1; p < N; p <<= 1) {
+#pragma unroll
+    for (int k = p; k >= 1; k >>= 1) {
+#pragma unroll
+      for (int j = k % p; j <= N - 1 - k; j += 2 * k) {
+#pragma unroll
+        for (int i = 0; i < k; ++i) {
+          if (i + j + k < N && (i + j) / (2 * p) == (i + j + k) / (2 * p)) ce(r[i + j], r[i + j + k]);
+        }
+      }
+    }
+  }
+}
+
+// r[0..N) bitonic -> sorted descending.
+template <int N>
+__device__ __forceinline__ void bitonic_merge_desc(uint32_t* r) {
+#pragma unroll
+  for (int s = N / 2; s >= 1; s >>= 1) {
+#pragma unroll
+    for (int i = 0; i < N; ++i) {
+      if ((i & s) == 0) ce(r[i], r[i + s]);
+    }
+  }
+}
+
+// bits 0..15 of x -> even bit positions, bits 16..31 -> odd bit positions.
+__device__ __forceinline__ uint32_t spread16(uint32_t x) {
+  x &= 0xFFFFu;
+  x = (x | (x << 8)) & 0x00FF00FFu;
+  x = (x | (x << 4)) & 0x0F0F0F0Fu;
+  x = (x | (x << 2)) & 0x33333333u;
+  x = (x | (x << 1)) & 0x55555555u;
+  return x;
+}
+__device__ __forceinline__ uint32_t interleave_halves(uint32_t x) { return spread16(x) | (spread16(x >> 16) << 1); }
+
+// Eight fp32 values holding integers in their low mantissa bits (magic-number rounding)
+// -> eight two's-complement nibbles, element i in nibble i.
+__device__ __forceinline__ uint32_t pack_nibbles(const float (&r)[8]) {
+  const uint32_t u0 = __float_as_uint(r[0]), u1 = __float_as_uint(r[1]), u2 = __float_as_uint(r[2]),
+                 u3 = __float_as_uint(r[3]), u4 = __float_as_uint(r[4]), u5 = __float_as_uint(r[5]),
+                 u6 = __float_as_uint(r[6]), u7 = __float_as_uint(r[7]);
+  const uint32_t ev = __byte_perm(__byte_perm(u0, u2, 0x0040), __byte_perm(u4, u6, 0x0040), 0x5410);
+  const uint32_t od = __byte_perm(__byte_perm(u1, u3, 0x0040), __byte_perm(u5, u7, 0x0040), 0x5410);
+  return (ev & 0x0F0F0F0Fu) | ((od << 4) & 0xF0F0F0F0u);
+}
+
+// Row scales from the two maxima (bf16 magnitude bit patterns).
+struct RowScale {
+  float inv, inv_lo, s_hi, s_lo;
+  int e;
+  bool clamp;  // some dense code may exceed 7 before clamping (only possible when e == 4)
+};
+__device__ __forceinline__ RowScale row_scale(uint32_t amax_bits, uint32_t rmax_bits) {
+  RowScale rs;
+  const float amax = bf16_bits_to_f32(amax_bits), rmax = bf16_bits_to_f32(rmax_bits);
+  rs.inv = amax > 0.f ? __fdiv_rn(127.0f, amax) : 0.f;
+  rs.s_hi = amax > 0.f ? __fdiv_rn(amax, 127.0f) : 0.f;
+  int e = 0;
+  if (amax > 0.f) {
+    e = 4;
+#pragma unroll
+    for (int t = 4; t >= 0; --t) {
+      if (rne_prod(rmax, rs.inv * (1.0f / (float)(1 << t))) <= 7) e = t;  // ends on the smallest fitting t
+    }
+  }
+  rs.e = e;
+  rs.inv_lo = rs.inv * (1.0f / (float)(1 << e));
+  rs.s_lo = rs.s_hi * (float)(1 << e);
+  rs.clamp = rne_prod(rmax, rs.inv_lo) > 7;
+  return rs;
+}
+
+__device__ __forceinline__ void bulk_copy_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+  asm volatile(
+      "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
+      "l"(src), "r"(bytes), "r"(bar)
+      : "memory");
+}
+
+// Eight bf16 (four packed words) times c, rounded half-even to integers held in the low
+// mantissa bits (magic-number rounding); two FMAs per instruction on the packed fp32 pipe,
+// each half rounding like fmaf.
+__device__ __forceinline__ void quant8(const uint4& v, float c, float (&r)[8]) {
+  const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+  const float2 cc = make_float2(c, c), mm = make_float2(kMagic, kMagic);
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    const float2 a = make_float2(__uint_as_float(w[q] << 16), __uint_as_float(w[q] & 0xFFFF0000u));
+    const float2 d = __ffma2_rn(a, cc, mm);
+    r[2 * q] = d.x;
+    r[2 * q + 1] = d.y;
+  }
+}
+
+// The coalesced INT4 sweep over a staged row (selected places already zeroed): lane l of the
+// group takes 16-byte chunks l, l + gsize, ... and writes one 32-bit word per chunk.
+__device__ __forceinline__ void dense_sweep(const uint16_t* row, int K, const RowScale& rs, uint8_t* dq4_row, int lane,
+                                            int gsize) {
+  const float c = rs.inv_lo;
+  const uint4* src = reinterpret_cast<const uint4*>(row) + lane;
+  uint32_t* dst = reinterpret_cast<uint32_t*>(dq4_row) + lane;
+  const int iters = (K / 8 - lane + gsize - 1) / gsize;
+  if (!rs.clamp) {
+#pragma unroll 2
+    for (int i = 0; i < iters; ++i, src += gsize, dst += gsize) {
+      float r[8];
+      quant8(*src, c, r);
+      *dst = pack_nibbles(r);
+    }
+  } else {
+    for (int i = 0; i < iters; ++i, src += gsize, dst += gsize) {
+      float r[8];
+      quant8(*src, c, r);
+#pragma unroll
+      for (int q = 0; q < 8; ++q) r[q] = fminf(fmaxf(r[q], kMagic - 7.0f), kMagic + 7.0f);
+      *dst = pack_nibbles(r);
+    }
+  }
+}
+
+struct EncodeParams {
+  const uint16_t* X;
+  const uint8_t* positions;
+  uint8_t* dq4;
+  int8_t* vals;
+  uint8_t* idx;
+  float* s_hi;
+  float* s_lo;
+  uint8_t* shift;
+  int* status;
+  int64_t M;
+  int K, k;
+  int nbuf;           // row buffers per group (1 or 2)
+  int rw;             // warps per row group
+  int group_stride;   // bytes of shared memory per group
+};
+
+__device__ __forceinline__ void group_sync(int rw, int grp) {
+  if (rw == 1) __syncwarp();
+  else asm volatile("bar.sync %0, %1;" ::"r"(1 + grp), "r"(rw * 32) : "memory");
+}
+
 }  // namespace
 
-// One block per token row; the row is staged in shared memory because the scale
-// (row maximum) must be known before anything is quantised.
+// ------------------------------------------------------------------------------------------------
+// Row-group kernel.  B = bank size; KK = k for dynamic positions (a power of two), 0 for static.
+template <int B, int KK>
+__global__ void __launch_bounds__(B == 128 ? 256 : 512) encode_rows_kernel(const EncodeParams p) {
+  extern __shared__ __align__(128) uint8_t smem_enc[];
+  constexpr bool kStatic = (KK == 0);
+  constexpr int NP = B / 2;          // packed registers per bank
+  constexpr int NCH = B / 8;         // 16-byte chunks per bank
+  constexpr int NM = (B + 63) / 64;  // 64-bit mask words per bank
+  const int warp = threadIdx.x >> 5;
+  const int rw = p.rw, grp = warp / rw;
+  const int lane = (warp % rw) * 32 + (threadIdx.x & 31);  // lane within the row group
+  const int gsize = rw * 32;
+  const int ngroups = (blockDim.x >> 5) / rw;
+  const int K = p.K, G = K / B, k = kStatic ? p.k : KK;
+  const int GK = G * k;
+  const int nbuf = p.nbuf;
+
+  // shared memory: [static only: table of selected element offsets, uint16 [GK]] then per group
+  // [nbuf rows][stash of selected raw values, uint16 [GK]][4 mbarriers][2 x 16 exchange words]
+  const size_t table_bytes = kStatic ? (((size_t)GK * 2 + 127) & ~(size_t)127) : 0;
+  uint16_t* jt = reinterpret_cast<uint16_t*>(smem_enc);
+  uint8_t* wbase = smem_enc + table_bytes + (size_t)grp * p.group_stride;
+  uint16_t* stash = reinterpret_cast<uint16_t*>(wbase + (size_t)nbuf * K * 2);
+  const size_t stash_bytes = ((size_t)GK * 2 + 15) & ~(size_t)15;
+  const uint32_t bar0 = smem_u32(reinterpret_cast<uint8_t*>(stash) + stash_bytes);
+  uint32_t* exch = reinterpret_cast<uint32_t*>(reinterpret_cast<uint8_t*>(stash) + stash_bytes + 32);
+  __shared__ int abort_flag_s;
+  volatile int* abort_flag = &abort_flag_s;
+
+  if (threadIdx.x == 0) abort_flag_s = 0;
+  if (lane == 0) {
+    for (int i = 0; i < 4; ++i) mbar_init(bar0 + 8 * i, 1);
+    fence_mbar_init();
+  }
+  if constexpr (kStatic) {
+    // element offset inside a row of every selected position, in the order vals are stored
+    for (int t = threadIdx.x; t < GK; t += blockDim.x) jt[t] = (uint16_t)((t / k) * B + p.positions[t]);
+  }
+  __syncthreads();
+
+  const int64_t gw = (int64_t)blockIdx.x * ngroups + grp;
+  const int64_t wstride = (int64_t)gridDim.x * ngroups;
+  const uint32_t row_bytes = (uint32_t)K * 2;
+
+  // Ring of nbuf row buffers: the row processed in iteration `it` sits in buffer it % nbuf and
+  // rows up to nbuf - 1 iterations ahead are already on their way (with one buffer the next
+  // row is requested only after the current one is done).
+  const int ahead = nbuf > 1 ? nbuf - 1 : 1;
+  if (lane == 0) {
+    for (int i = 0; i < ahead; ++i) {
+      const int64_t mi = gw + (int64_t)i * wstride;
+      if (mi < p.M && (nbuf > 1 || i == 0))
+        bulk_copy_g2s(smem_u32(wbase + (size_t)i * row_bytes), p.X + mi * K, row_bytes, bar0 + 8 * i);
+    }
+  }
+
+  uint32_t cur = 0, parity = 0;
+  for (int64_t m = gw; m < p.M; m += wstride) {
+    uint16_t* row = reinterpret_cast<uint16_t*>(wbase + (size_t)cur * row_bytes);
+    if (nbuf > 1 && lane == 0) {
+      // the buffer released at the end of the previous iteration takes the row `ahead` steps on
+      const int64_t mn = m + (int64_t)ahead * wstride;
+      const uint32_t nb = cur == 0 ? (uint32_t)nbuf - 1 : cur - 1;
+      if (mn < p.M) bulk_copy_g2s(smem_u32(wbase + (size_t)nb * row_bytes), p.X + mn * K, row_bytes, bar0 + 8 * nb);
+    }
+    if (!mbar_wait_park(bar0 + 8 * cur, parity, abort_flag)) break;
+
+    uint32_t lane_amax = 0, lane_rmax = 0;
+    if constexpr (!kStatic) {
+      // ------------------------------------------------------------ phase 1: selection
+      // conflict-free chunk rotation: consecutive lanes start on different 16-byte bank groups
+      const int rot = (B == 32) ? ((lane >> 1) & (NCH - 1)) : (lane & (NCH - 1));
+      for (int g = lane; g < G; g += gsize) {
+        uint16_t* bank = row + g * B;
+        uint32_t x[NP];
+#pragma unroll
+        for (int c = 0; c < NCH; ++c) {
+          const uint4 v = *reinterpret_cast<const uint4*>(bank + ((c + rot) & (NCH - 1)) * 8);
+          x[4 * c] = v.x & 0x7FFF7FFFu;
+          x[4 * c + 1] = v.y & 0x7FFF7FFFu;
+          x[4 * c + 2] = v.z & 0x7FFF7FFFu;
+          x[4 * c + 3] = v.w & 0x7FFF7FFFu;
+        }
+        // k-th largest magnitude: sorted runs of KK per column, merged with truncation
+        uint32_t s[NP];
+#pragma unroll
+        for (int i = 0; i < NP; ++i) s[i] = x[i];
+#pragma unroll
+        for (int grp2 = 0; grp2 < NP / KK; ++grp2) sort_desc<KK>(s + grp2 * KK);
+#pragma unroll
+        for (int span = KK; span < NP; span *= 2) {
+#pragma unroll
+          for (int a = 0; a + span < NP; a += 2 * span) {
+#pragma unroll
+            for (int i = 0; i < KK; ++i) s[a + i] = max2(s[a + i], s[a + span + KK - 1 - i]);
+            bitonic_merge_desc<KK>(s + a);
+          }
+        }
+        // s[0..KK): per column the KK largest, descending.  Across the two columns:
+        uint32_t d[KK];
+#pragma unroll
+        for (int i = 0; i < KK; ++i) d[i] = max2(s[i], swap_halves(s[KK - 1 - i]));
+#pragma unroll
+        for (int w = KK / 2; w >= 1; w /= 2) {
+#pragma unroll
+          for (int i = 0; i < w; ++i) d[i] = min2(d[i], d[i + w]);
+        }
+        const uint32_t T = d[0] & 0xFFFFu;  // k-th largest magnitude of the bank (with multiplicity)
+        const uint32_t bank_max = max(s[0] & 0xFFFFu, s[0] >> 16);
+        lane_amax = max(lane_amax, bank_max);
+
+        // compare pass: selection mask (slot order) and the largest magnitude below T
+        const uint32_t T2 = T * 0x10001u;
+        uint32_t acc[NP / 16];
+        uint32_t below = 0;
+#pragma unroll
+        for (int w = 0; w < NP / 16; ++w) acc[w] = 0;
+#pragma unroll
+        for (int q = 0; q < NP; ++q) {
+          const uint32_t ge = ge2_mask(x[q], T2);
+          acc[q / 16] |= ge & (0x00010001u << (q % 16));
+          below = max2(below, x[q] & ~ge);
+        }
+        uint64_t sel[NM];
+#pragma unroll
+        for (int w = 0; w < NM; ++w) sel[w] = 0;
+#pragma unroll
+        for (int w = 0; w < NP / 16; ++w) sel[w / 2] |= (uint64_t)interleave_halves(acc[w]) << (32 * (w & 1));
+        // slot order -> element order: slot c holds chunk (c + rot) mod NCH
+        if (B == 128) {
+          const int sh = 8 * rot;  // 0..120
+          uint64_t lo = sel[0], hi = sel[NM - 1];
+          if (sh >= 64) {
+            const uint64_t t = lo;
+            lo = hi;
+            hi = t;
+          }
+          const int r = sh & 63;
+          if (r) {
+            const uint64_t nlo = (lo << r) | (hi >> (64 - r)), nhi = (hi << r) | (lo >> (64 - r));
+            lo = nlo;
+            hi = nhi;
+          }
+          sel[0] = lo;
+          sel[NM - 1] = hi;
+        } else if (B == 64) {
+          const int r = 8 * rot;
+          if (r) sel[0] = (sel[0] << r) | (sel[0] >> (64 - r));
+        } else {
+          const uint32_t v = (uint32_t)sel[0];
+          sel[0] = (uint64_t)__funnelshift_l(v, v, 8 * rot);
+        }
+        int cnt = 0;
+#pragma unroll
+        for (int w = 0; w < NM; ++w) cnt += __popcll(sel[w]);
+        uint32_t rest = max(below & 0xFFFFu, below >> 16);
+        if (cnt > KK) {
+          // more than k elements reach T: drop the equal ones with the largest indices
+          rest = T;
+          int excess = cnt - KK;
+#pragma unroll
+          for (int w = NM - 1; w >= 0; --w) {
+            uint64_t scan = sel[w];
+            while (excess > 0 && scan != 0) {
+              const int pos = 63 - __clzll((long long)scan);
+              scan &= ~(1ull << pos);
+              if ((uint32_t)(bank[64 * w + pos] & 0x7FFFu) == T) {
+                sel[w] &= ~(1ull << pos);
+                --excess;
+              }
+            }
+          }
+        }
+        lane_rmax = max(lane_rmax, rest);
+
+        // the k selected elements in ascending position: raw values to the stash, zero in the
+        // staged row, positions to global memory (they do not depend on the scale)
+        uint32_t iout[(KK + 3) / 4];
+#pragma unroll
+        for (int w = 0; w < (KK + 3) / 4; ++w) iout[w] = 0;
+        uint32_t m0 = (uint32_t)sel[0], m1 = (uint32_t)(sel[0] >> 32), m2 = 0, m3 = 0;
+        if (NM == 2) {
+          m2 = (uint32_t)sel[NM - 1];
+          m3 = (uint32_t)(sel[NM - 1] >> 32);
+        }
+        uint16_t* sg = stash + g * KK;
+#pragma unroll
+        for (int i = 0; i < KK; ++i) {
+          // lowest set bit of the (up to 128-bit) mask, then clear it
+          uint32_t word = m0, base = 0;
+          if (B >= 64 && word == 0) {
+            word = m1;
+            base = 32;
+          }
+          if (B == 128 && word == 0) {
+            word = m2;
+            base = 64;
+            if (word == 0) {
+              word = m3;
+              base = 96;
+            }
+          }
+          const uint32_t bit = word & (0u - word);
+          const uint32_t pos = base + (31u - (uint32_t)__clz((int)bit));
+          if (base == 0) m0 ^= bit;
+          else if (base == 32) m1 ^= bit;
+          else if (base == 64) m2 ^= bit;
+          else m3 ^= bit;
+          sg[i] = bank[pos];
+          bank[pos] = 0;
+          iout[i / 4] = __byte_perm(iout[i / 4], pos, 0x3210 ^ (0x4 << (4 * (i % 4))) ^ ((i % 4) << (4 * (i % 4))));
+        }
+        uint8_t* idst = p.idx + ((size_t)m * G + g) * KK;
+        if (KK >= 16) {
+#pragma unroll
+          for (int w = 0; w < KK / 16; ++w)
+            reinterpret_cast<uint4*>(idst)[w] = make_uint4(iout[4 * w], iout[4 * w + 1], iout[4 * w + 2], iout[4 * w + 3]);
+        } else if (KK == 8) {
+          *reinterpret_cast<uint2*>(idst) = make_uint2(iout[0], iout[1]);
+        } else if (KK == 4) {
+          *reinterpret_cast<uint32_t*>(idst) = iout[0];
+        } else if (KK == 2) {
+          *reinterpret_cast<uint16_t*>(idst) = (uint16_t)iout[0];
+        } else {
+          *idst = (uint8_t)iout[0];
+        }
+      }
+    } else {
+      // ------------------------------------------------------------ phase 1 (static): stash and zero
+#pragma unroll 4
+      for (int t = lane; t < GK; t += gsize) {
+        const int j = jt[t];
+        const uint16_t v = row[j];
+        stash[t] = v;
+        row[j] = 0;
+        lane_amax = max(lane_amax, (uint32_t)(v & 0x7FFFu));
+      }
+      group_sync(rw, grp);
+      const uint4* src = reinterpret_cast<const uint4*>(row) + lane;
+      const int iters = (K / 8 - lane + gsize - 1) / gsize;
+#pragma unroll 4
+      for (int i = 0; i < iters; ++i, src += gsize) {
+        const uint4 v = *src;
+        const uint32_t mx = max2(max2(v.x & 0x7FFF7FFFu, v.y & 0x7FFF7FFFu), max2(v.z & 0x7FFF7FFFu, v.w & 0x7FFF7FFFu));
+        lane_rmax = max(lane_rmax, max(mx & 0xFFFFu, mx >> 16));
+      }
+      lane_amax = max(lane_amax, lane_rmax);
+    }
+
+    uint32_t amax_bits = __reduce_max_sync(0xffffffffu, lane_amax);
+    uint32_t rmax_bits = __reduce_max_sync(0xffffffffu, lane_rmax);
+    if (rw > 1) {
+      if ((threadIdx.x & 31) == 0) {
+        exch[warp % rw] = amax_bits;
+        exch[16 + warp % rw] = rmax_bits;
+      }
+      group_sync(rw, grp);  // also: every stash entry of the row is written
+      amax_bits = rmax_bits = 0;
+      for (int w = 0; w < rw; ++w) {
+        amax_bits = max(amax_bits, exch[w]);
+        rmax_bits = max(rmax_bits, exch[16 + w]);
+      }
+    } else {
+      __syncwarp();
+    }
+    RowScale rs;
+    if ((threadIdx.x & 31) == 0) rs = row_scale(amax_bits, rmax_bits);  // one lane computes, the warp shares
+    rs.inv = __shfl_sync(0xffffffffu, rs.inv, 0);
+    rs.inv_lo = __shfl_sync(0xffffffffu, rs.inv_lo, 0);
+    rs.clamp = __shfl_sync(0xffffffffu, (int)rs.clamp, 0) != 0;
+    if (lane == 0) {
+      p.s_hi[m] = rs.s_hi;
+      p.s_lo[m] = rs.s_lo;
+      p.shift[m] = (uint8_t)rs.e;
+    }
+
+    // -------------------------------------------------------------- phase 2a: sparse component
+    {
+      int8_t* vdst = p.vals + (size_t)m * GK;
+      if ((GK & 3) == 0) {
+        for (int t4 = lane * 4; t4 < GK; t4 += gsize * 4) {
+          const uint2 sv = *reinterpret_cast<const uint2*>(stash + t4);
+          const uint32_t w[2] = {sv.x, sv.y};
+          uint32_t o = 0;
+#pragma unroll
+          for (int q = 0; q < 2; ++q) {  // |a * inv| <= 127 by construction: no clamp
+            const uint32_t q0 = __float_as_uint(__fmaf_rn(__uint_as_float(w[q] << 16), rs.inv, kMagic)) & 0xFFu;
+            const uint32_t q1 = __float_as_uint(__fmaf_rn(__uint_as_float(w[q] & 0xFFFF0000u), rs.inv, kMagic)) & 0xFFu;
+            o |= (q0 << (16 * q)) | (q1 << (16 * q + 8));
+          }
+          *reinterpret_cast<uint32_t*>(vdst + t4) = o;
+        }
+      } else {
+        for (int t = lane; t < GK; t += gsize)
+          vdst[t] = (int8_t)(__float_as_uint(__fmaf_rn(bf16_bits_to_f32(stash[t]), rs.inv, kMagic)) & 0xFFu);
+      }
+    }
+
+    // -------------------------------------------------------------- phase 2b: dense component
+    // (the group barrier above also ordered the zeroing of the selected places before this sweep)
+    dense_sweep(row, K, rs, p.dq4 + (size_t)m * (K / 2), lane, gsize);
+
+    // the row buffer is about to be refilled by the async proxy: order this group's generic
+    // accesses before it
+    fence_proxy_async_smem();
+    group_sync(rw, grp);
+    if (nbuf == 1 && m + wstride < p.M && lane == 0)
+      bulk_copy_g2s(smem_u32(wbase), p.X + (m + wstride) * K, row_bytes, bar0);
+    if (++cur == (uint32_t)nbuf) {
+      cur = 0;
+      parity ^= 1u;
+    }
+  }
+  if (*abort_flag && lane == 0) atomicExch(p.status, (int)SQ_ERR_TIMEOUT);
+}
+
+// ------------------------------------------------------------------------------------------------
+// Plain kernel for any (b, k): one block per token row, the row staged in shared memory.
 //   phase 1  load the row, row maximum -> inv = 127/amax, s_hi = amax/127
 //   phase 2  positions: dynamic = rank every element of a bank by (magnitude, then lower
 //            index) and keep ranks < k; static = the given positions.  Selected elements
@@ -30,14 +550,13 @@ __device__ __forceinline__ uint32_t block_max_u32(uint32_t v, uint32_t* scratch)
 //   phase 3  maximum of what is left -> shift e, s_lo
 //   phase 4  INT4 codes of the staged row (zeros at the selected places), 8 per 32-bit word
 template <int B>
-__global__ void __launch_bounds__(256) encode_kernel(int k, bool is_static, const uint16_t* __restrict__ X, int64_t K,
-                                                     const uint8_t* __restrict__ positions,
-                                                     uint8_t* __restrict__ dq4, int8_t* __restrict__ vals,
-                                                     uint8_t* __restrict__ idx, float* __restrict__ s_hi,
-                                                     float* __restrict__ s_lo, uint8_t* __restrict__ shift) {
+__global__ void __launch_bounds__(256) encode_generic_kernel(int k, bool is_static, const uint16_t* __restrict__ X, int64_t K,
+                                                             const uint8_t* __restrict__ positions,
+                                                             uint8_t* __restrict__ dq4, int8_t* __restrict__ vals,
+                                                             uint8_t* __restrict__ idx, float* __restrict__ s_hi,
+                                                             float* __restrict__ s_lo, uint8_t* __restrict__ shift) {
   extern __shared__ __align__(16) uint16_t srow[];
   __shared__ uint32_t scratch[8];
-  __shared__ int sE;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int64_t m = blockIdx.x;
   const int64_t G = K / B;
@@ -54,9 +573,9 @@ __global__ void __launch_bounds__(256) encode_kernel(int k, bool is_static, cons
       mx = max(mx, (w[q] >> 16) & 0x7FFFu);
     }
   }
-  const float amax = bf16_bits_to_f32(block_max_u32(mx, scratch));  // barrier inside: row staged
+  const uint32_t amax_bits = block_max_u32(mx, scratch);  // barrier inside: row staged
+  const float amax = bf16_bits_to_f32(amax_bits);
   const float inv = amax > 0.f ? __fdiv_rn(127.0f, amax) : 0.f;
-  const float sh = amax > 0.f ? __fdiv_rn(amax, 127.0f) : 0.f;
 
   if (is_static) {
     const int64_t GK = G * k;
@@ -118,34 +637,21 @@ __global__ void __launch_bounds__(256) encode_kernel(int k, bool is_static, cons
       rm = max(rm, (w[q] >> 16) & 0x7FFFu);
     }
   }
-  const float rmax = bf16_bits_to_f32(block_max_u32(rm, scratch));
+  const uint32_t rmax_bits = block_max_u32(rm, scratch);
+  const RowScale rs = row_scale(amax_bits, rmax_bits);
   if (tid == 0) {
-    int e = 0;
-    if (amax > 0.f) {
-      e = 4;
-      for (int t = 0; t <= 4; ++t) {
-        if (rne_prod(rmax, inv * (1.0f / (float)(1 << t))) <= 7) {
-          e = t;
-          break;
-        }
-      }
-    }
-    sE = e;
-    s_hi[m] = sh;
-    s_lo[m] = sh * (float)(1 << e);
-    shift[m] = (uint8_t)e;
+    s_hi[m] = rs.s_hi;
+    s_lo[m] = rs.s_lo;
+    shift[m] = (uint8_t)rs.e;
   }
-  __syncthreads();
-  const float inv_lo = inv * (1.0f / (float)(1 << sE));
-
   for (int64_t i = (int64_t)tid * 8; i < K; i += 256 * 8) {
     const uint4 v = *reinterpret_cast<const uint4*>(srow + i);
     const uint32_t w[4] = {v.x, v.y, v.z, v.w};
     uint32_t word = 0;
 #pragma unroll
     for (int q = 0; q < 4; ++q) {
-      int q0 = rne_prod(bf16_bits_to_f32(w[q] & 0xFFFFu), inv_lo);
-      int q1 = rne_prod(bf16_bits_to_f32(w[q] >> 16), inv_lo);
+      int q0 = rne_prod(bf16_bits_to_f32(w[q] & 0xFFFFu), rs.inv_lo);
+      int q1 = rne_prod(bf16_bits_to_f32(w[q] >> 16), rs.inv_lo);
       q0 = min(7, max(-7, q0));
       q1 = min(7, max(-7, q1));
       word |= (uint32_t)(q0 & 0xF) << (8 * q);
@@ -187,24 +693,103 @@ __global__ void __launch_bounds__(256) decode_kernel(int b, int k, const uint8_t
   }
 }
 
-cudaError_t launch_encode(int b, int k, bool is_static, const uint16_t* X, int64_t M, int64_t K,
-                          const uint8_t* positions, const sq_encoded& out, cudaStream_t st) {
-  const size_t smem = (size_t)K * 2;
-  cudaError_t err = cudaSuccess;
-#define SQ_LAUNCH_ENCODE(BB)                                                                         \
-  do {                                                                                               \
-    err = cudaFuncSetAttribute(encode_kernel<BB>, cudaFuncAttributeMaxDynamicSharedMemorySize,       \
-                               (int)smem);                                                           \
-    if (err != cudaSuccess) return err;                                                              \
-    encode_kernel<BB><<<(unsigned)M, 256, smem, st>>>(k, is_static, X, K, positions, out.dq4,        \
-                                                      out.vals, out.idx, out.s_hi, out.s_lo,         \
-                                                      out.shift);                                    \
-  } while (0)
-  if (b == 32) SQ_LAUNCH_ENCODE(32);
-  else if (b == 64) SQ_LAUNCH_ENCODE(64);
-  else SQ_LAUNCH_ENCODE(128);
-#undef SQ_LAUNCH_ENCODE
+namespace {
+
+template <int B, int KK>
+cudaError_t launch_rows(const EncodeParams& base, cudaStream_t st) {
+  EncodeParams p = base;
+  const int K = p.K, G = K / B, k = (KK == 0) ? p.k : KK;
+  constexpr int NM = (B + 63) / 64;
+  constexpr int kMaxWarps = (B == 128) ? 8 : 16;
+  const size_t side = (((size_t)G * k * 2) + 15) & ~(size_t)15;            // stash of selected raw values
+  const size_t table = (KK == 0) ? ((((size_t)G * k * 2) + 127) & ~(size_t)127) : 0;  // static offset table
+  const size_t budget = 208 * 1024 - table;
+  const size_t row = (size_t)K * 2;
+  const size_t extra = side + 32 + 128 + 128;  // side buffer, four mbarriers, exchange words, rounding
+  // Pick the group size that keeps the most rows in flight per SM (groups x rows requested
+  // ahead), preferring more groups on a tie; one single-buffered group if two rows never fit.
+  int rw = kMaxWarps, nbuf = 1, best = 0;
+  for (int cand = 1; cand <= kMaxWarps; cand *= 2) {
+    const int groups = kMaxWarps / cand;
+    if (cand == 1 && groups > 15) continue;  // one warp per row needs no named barrier, but keep ids in range
+    const size_t per = budget / groups;
+    if (per < extra + 2 * row) continue;
+    int nb = (int)((per - extra) / row);
+    if (nb > 4) nb = 4;
+    const int score = groups * (nb - 1);
+    if (score > best) {
+      best = score;
+      rw = cand;
+      nbuf = nb;
+    }
+  }
+  const size_t per_group = (((size_t)nbuf * row + extra) + 127) & ~(size_t)127;
+  if (per_group > 224 * 1024) return cudaErrorInvalidValue;
+  const int ngroups = kMaxWarps / rw;
+  p.nbuf = nbuf;
+  p.rw = rw;
+  p.group_stride = (int)per_group;
+  const size_t smem = table + per_group * ngroups;
+
+  int dev = 0, sms = 0;
+  cudaError_t err = cudaGetDevice(&dev);
+  if (err != cudaSuccess) return err;
+  err = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  if (err != cudaSuccess) return err;
+  err = cudaFuncSetAttribute(encode_rows_kernel<B, KK>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (err != cudaSuccess) return err;
+  int64_t blocks = (p.M + ngroups - 1) / ngroups;
+  if (blocks > sms) blocks = sms;
+  encode_rows_kernel<B, KK><<<(unsigned)blocks, kMaxWarps * 32, smem, st>>>(p);
   return cudaGetLastError();
+}
+
+template <int B>
+cudaError_t launch_generic(int k, bool is_static, const uint16_t* X, int64_t M, int64_t K, const uint8_t* positions,
+                           const sq_encoded& out, cudaStream_t st) {
+  const size_t smem = (size_t)K * 2;
+  cudaError_t err = cudaFuncSetAttribute(encode_generic_kernel<B>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (err != cudaSuccess) return err;
+  encode_generic_kernel<B><<<(unsigned)M, 256, smem, st>>>(k, is_static, X, K, positions, out.dq4, out.vals, out.idx,
+                                                          out.s_hi, out.s_lo, out.shift);
+  return cudaGetLastError();
+}
+
+}  // namespace
+
+cudaError_t launch_encode(int b, int k, bool is_static, const uint16_t* X, int64_t M, int64_t K,
+                          const uint8_t* positions, const sq_encoded& out, int* status, cudaStream_t st) {
+  EncodeParams p;
+  p.X = X;
+  p.positions = positions;
+  p.dq4 = out.dq4;
+  p.vals = out.vals;
+  p.idx = out.idx;
+  p.s_hi = out.s_hi;
+  p.s_lo = out.s_lo;
+  p.shift = out.shift;
+  p.status = status;
+  p.M = M;
+  p.K = (int)K;
+  p.k = k;
+  p.nbuf = 1;
+  p.rw = 1;
+  p.group_stride = 0;
+  if (is_static) {
+    if (b == 32) return launch_rows<32, 0>(p, st);
+    if (b == 64) return launch_rows<64, 0>(p, st);
+    return launch_rows<128, 0>(p, st);
+  }
+  // dynamic fast kernels: k/b in {1/16, 1/8, 1/4, 1/2}
+#define SQ_DYN(BB, KK_) \
+  if (b == BB && k == KK_) return launch_rows<BB, KK_>(p, st);
+  SQ_DYN(32, 2) SQ_DYN(32, 4) SQ_DYN(32, 8) SQ_DYN(32, 16)
+  SQ_DYN(64, 4) SQ_DYN(64, 8) SQ_DYN(64, 16) SQ_DYN(64, 32)
+  SQ_DYN(128, 8) SQ_DYN(128, 16) SQ_DYN(128, 32) SQ_DYN(128, 64)
+#undef SQ_DYN
+  if (b == 32) return launch_generic<32>(k, false, X, M, K, positions, out, st);
+  if (b == 64) return launch_generic<64>(k, false, X, M, K, positions, out, st);
+  return launch_generic<128>(k, false, X, M, K, positions, out, st);
 }
 
 cudaError_t launch_decode(int b, int k, const sq_encoded& A, const uint8_t* positions, int64_t M,

@@ -19,7 +19,7 @@ cudaError_t launch_pack_weights(int b, int k, const uint16_t* W, int64_t N, int6
                                 const uint8_t* positions, const sq_weights& out, cudaStream_t st);
 
 cudaError_t launch_encode(int b, int k, bool is_static, const uint16_t* X, int64_t M, int64_t K,
-                          const uint8_t* positions, const sq_encoded& out, cudaStream_t st);
+                          const uint8_t* positions, const sq_encoded& out, int* status, cudaStream_t st);
 
 cudaError_t launch_decode(int b, int k, const sq_encoded& A, const uint8_t* positions, int64_t M,
                           int64_t K, uint16_t* out, cudaStream_t st);
