@@ -166,10 +166,15 @@ __device__ __forceinline__ void quant8(const uint4& v, float c, float (&r)[8]) {
   const float2 cc = make_float2(c, c), mm = make_float2(kMagic, kMagic);
 #pragma unroll
   for (int q = 0; q < 4; ++q) {
+#ifdef SQ_X_SCALAR_FMA
+    r[2 * q] = __fmaf_rn(__uint_as_float(w[q] << 16), c, kMagic);
+    r[2 * q + 1] = __fmaf_rn(__uint_as_float(w[q] & 0xFFFF0000u), c, kMagic);
+#else
     const float2 a = make_float2(__uint_as_float(w[q] << 16), __uint_as_float(w[q] & 0xFFFF0000u));
     const float2 d = __ffma2_rn(a, cc, mm);
     r[2 * q] = d.x;
     r[2 * q + 1] = d.y;
+#endif
   }
 }
 
@@ -706,26 +711,34 @@ cudaError_t launch_rows(const EncodeParams& base, cudaStream_t st) {
   const size_t budget = 208 * 1024 - table;
   const size_t row = (size_t)K * 2;
   const size_t extra = side + 32 + 128 + 128;  // side buffer, four mbarriers, exchange words, rounding
-  // Pick the group size that keeps the most rows in flight per SM (groups x rows requested
-  // ahead), preferring more groups on a tie; one single-buffered group if two rows never fit.
+  // Rows are single-buffered: with 16 resident warps the rows other groups have in flight
+  // hide the copy latency, and a second buffer would only cost warps.  Pick the group size
+  // that keeps the most warps resident, preferring smaller groups (less per-row overhead per
+  // element) on a tie.
   int rw = kMaxWarps, nbuf = 1, best = 0;
   for (int cand = 1; cand <= kMaxWarps; cand *= 2) {
-    const int groups = kMaxWarps / cand;
-    if (cand == 1 && groups > 15) continue;  // one warp per row needs no named barrier, but keep ids in range
-    const size_t per = budget / groups;
-    if (per < extra + 2 * row) continue;
-    int nb = (int)((per - extra) / row);
-    if (nb > 4) nb = 4;
-    const int score = groups * (nb - 1);
-    if (score > best) {
-      best = score;
+    const size_t per = ((row + extra) + 127) & ~(size_t)127;
+    if (per > budget) break;
+    int groups = (int)(budget / per);
+    if (groups > kMaxWarps / cand) groups = kMaxWarps / cand;
+    if (groups > 15) groups = 15;  // named barrier ids 1..15
+    if (groups * cand > best) {
+      best = groups * cand;
       rw = cand;
-      nbuf = nb;
     }
   }
+#ifdef SQ_X_RW
+  rw = SQ_X_RW;
+  nbuf = SQ_X_NBUF;
+#endif
   const size_t per_group = (((size_t)nbuf * row + extra) + 127) & ~(size_t)127;
   if (per_group > 224 * 1024) return cudaErrorInvalidValue;
-  const int ngroups = kMaxWarps / rw;
+  int ngroups = kMaxWarps / rw;
+  {
+    const size_t fit = (208 * 1024 - table) / ((((size_t)nbuf * row + extra) + 127) & ~(size_t)127);
+    if ((size_t)ngroups > fit) ngroups = (int)fit;
+    if (ngroups < 1) ngroups = 1;
+  }
   p.nbuf = nbuf;
   p.rw = rw;
   p.group_stride = (int)per_group;
@@ -740,7 +753,7 @@ cudaError_t launch_rows(const EncodeParams& base, cudaStream_t st) {
   if (err != cudaSuccess) return err;
   int64_t blocks = (p.M + ngroups - 1) / ngroups;
   if (blocks > sms) blocks = sms;
-  encode_rows_kernel<B, KK><<<(unsigned)blocks, kMaxWarps * 32, smem, st>>>(p);
+  encode_rows_kernel<B, KK><<<(unsigned)blocks, ngroups * rw * 32, smem, st>>>(p);
   return cudaGetLastError();
 }
 

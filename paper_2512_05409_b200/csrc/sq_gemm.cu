@@ -168,7 +168,11 @@ __global__ void __launch_bounds__(kThreads, 1)
 
   if (tid == 0) {
     for (int s = 0; s < NS; ++s) {
+#ifndef SQ_X_NOARRIVE_ALL
       mbar_init(bar_full + 8 * s, kProdThreads);
+#else
+      mbar_init(bar_full + 8 * s, kProdWarps);
+#endif
       mbar_init(bar_empty + 8 * s, 1);
       mbar_init(bar_sfull + 8 * s, 1);
     }
@@ -248,6 +252,14 @@ __global__ void __launch_bounds__(kThreads, 1)
     uint32_t re[2][2], sv[2][MAXT], si[2][MAXT];
     auto load_next = [&](int slot) {
       if (lt >= ntiles) return;
+#ifdef SQ_X_NOLOAD
+      if (lt >= 0) {
+        for (int i = 0; i < 2; ++i) ra[slot][i] = make_uint4(lks, lt, 3, 4);
+        for (int i = 0; i < NB_TASKS; ++i) rb[slot][i] = make_uint4(lks, lt, 5, 6);
+        if (++lks == KS) { lks = 0; lt += gridDim.x; }
+        return;
+      }
+#endif
 #pragma unroll
       for (int i = 0; i < 2; ++i) {
         ra[slot][i] = ldg_nc_v4(a_ptr[i] + (size_t)lks * 64);
@@ -317,6 +329,10 @@ __global__ void __launch_bounds__(kThreads, 1)
         }
       }
 #endif
+#ifdef SQ_X_NOWORK
+      if (ra[slot][0].x == 0x12345u) a_st[0] = (uint8_t)rb[slot][0].x;  // keep the loads alive
+      if (false)
+#endif
       // ---- widen A: nibble -> u * 2^e + (128 - 8 * 2^e)
 #pragma unroll
       for (int i = 0; i < 2; ++i) {
@@ -339,6 +355,9 @@ __global__ void __launch_bounds__(kThreads, 1)
         *reinterpret_cast<uint4*>(dst + (sw_even ^ 16u)) = make_uint4(od[0], od[1], od[2], od[3]);
       }
       // ---- widen B: nibble -> 16 * code
+#ifdef SQ_X_NOWORK
+      if (false)
+#endif
 #pragma unroll
       for (int i = 0; i < NB_TASKS; ++i) {
         const uint32_t in[4] = {rb[slot][i].x, rb[slot][i].y, rb[slot][i].z, rb[slot][i].w};
@@ -384,8 +403,15 @@ __global__ void __launch_bounds__(kThreads, 1)
           a_st[row * 128 + kp] = (uint8_t)((uint8_t)p.vals[entry] ^ 0x80u);
         }
       }
+#ifndef SQ_X_NOFENCE
       fence_proxy_async_smem();  // generic-proxy writes -> visible to the tensor core's async reads
+#endif
+#ifndef SQ_X_NOARRIVE_ALL
       mbar_arrive(bar_full + 8 * s);
+#else
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar_full + 8 * s);
+#endif
       ++it;
       if (++pks == KS) {
         pks = 0;
