@@ -5,18 +5,23 @@
 //
 // sm_100 has no INT4 MMA, so both operands are widened to 8 bits on chip.  The two
 // components of the activation live on one integer grid (the dense one coarsened by
-// 2^e), so they are MERGED into a single 8-bit operand before the tensor core sees
-// them: the dense nibbles are widened and shifted, then the k sparse INT8 entries of
-// every bank overwrite the (zero) places they belong to.  One MMA stream, one int32
-// accumulator in tensor memory, one epilogue.
+// 2^e), so they go into ONE int32 accumulator in tensor memory:
+//   dynamic positions: the k sparse INT8 entries of every bank overwrite the (zero) places
+//     they belong to in the widened dense tile before the tensor core sees it;
+//   static positions (Section 3.3, Fig. 2b: the mask only selects and gathers activation
+//     tiles because the weight rows were reordered offline): vals [M, G*k] and w_sparse
+//     [N, G*k] are plain INT8 matrices, so the sparse product is G*k/128 extra K steps whose
+//     tiles TMA writes straight into the same shared-memory stages (swizzled by the TMA
+//     unit, no thread touches them) and whose MMAs accumulate into the same tile.
 //
 // Operand encodings inside the kernel (chosen so the widening is a few logic ops on
 // eight nibbles at a time, never a per-byte sign extension):
 //   A is fed UNSIGNED with an offset of 128:  a_u = a + 128, a in [-127, 127].
 //     dense:  nibble q in two's complement -> u = q ^ 8 = q + 8 in [1, 15];
 //             a_u = u * 2^e + (128 - 8 * 2^e)      (no carries between bytes)
-//     sparse: a_u = vals ^ 0x80
-//   B is fed SIGNED as 16 * code: a nibble moved to the top of its byte.
+//     sparse (merged): a_u = vals ^ 0x80;  sparse (extra K steps): A signed, vals as stored
+//   B is fed SIGNED as 16 * code: a nibble moved to the top of its byte (w_sparse is stored
+//   that way already).
 //   Hence acc_internal = 16 * acc + 2048 * colsum[n]; the epilogue undoes both exactly.
 //   |acc_internal| <= K * 255 * 112 < 2^31 for K <= 65536.
 //
@@ -29,19 +34,16 @@
 // 128-byte swizzle (the 16-byte chunk index is XORed with row % 8), 8-row groups 1024
 // bytes apart: the canonical layout a tcgen05 shared-memory descriptor describes.
 //
-// Static positions take a second form of the sparse product (Section 3.3, Fig. 2b: the mask
-// only selects and gathers activation tiles because the weight rows were reordered offline):
-// vals [M, G*k] and w_sparse [N, G*k] are plain INT8 matrices, so the sparse product is
-// G*k/128 extra K steps whose tiles TMA writes straight into the same shared-memory stages
-// (swizzled by the TMA unit, no thread touches them) and whose MMAs (A signed this time, the
-// gathered weights already in sixteenths) accumulate into the same tensor-memory tile.
+// Tiling: a CTA computes 256 x 256 outputs as two 128-row sub-tiles that share every
+// widened weight stage (one third less widening work and L2 traffic per MMA than 128 x 256)
+// and fill all 512 tensor-memory columns.  The last, partial wave of a launch is cut into
+// 128 x 256 tiles so that it spreads over twice as many SMs.
 //
 // Kernel organisation: persistent, one CTA per SM, warp-specialised.
-//   warps 0-7   producers: global loads (register-prefetched two K steps ahead), widening,
-//               sparse merge (dynamic positions), stores into a ring of NS shared-memory stages
+//   warps 0-7   producers: global loads (register-prefetched), widening, sparse merge
+//               (dynamic positions), stores into a ring of NS shared-memory stages
 //   warp  8     one thread issues the MMAs and commits stage / accumulator barriers
-//   warps 9-12  epilogue: tcgen05.ld of one of two accumulator buffers, dequantise, store;
-//               overlaps the main loop of the next tile
+//   warps 9-12  epilogue: tcgen05.ld, dequantise, store
 //   warp  13    one thread issues the TMA loads of the sparse K steps (static positions)
 // Every wait is bounded; a wait that runs out raises an abort flag that releases all
 // other waits, the kernel records SQ_ERR_TIMEOUT and frees its tensor memory.
@@ -52,25 +54,27 @@
 #include "sq_device.cuh"
 #include "sq_host.h"
 
-#ifndef SQ_SPARSE_PREFETCH
-#define SQ_SPARSE_PREFETCH 1
-#endif
-#ifndef SQ_E_PER_STEP
-#define SQ_E_PER_STEP 0
-#endif
-
 namespace sq {
 
 namespace {
 
-constexpr int BM = 128;  // rows of A per tile = TMEM lanes
-constexpr int BK = 128;  // K elements per pipeline step = bytes per operand row
+constexpr int BM = 128;   // rows of one sub-tile = TMEM lanes
+constexpr int BN = 256;   // output channels per tile = TMEM columns of one accumulator
+constexpr int BK = 128;   // K elements per pipeline step = bytes per operand row
+constexpr int NS = 3;     // shared-memory stages
 constexpr int kProdWarps = 8;
 constexpr int kProdThreads = kProdWarps * 32;
 constexpr int kMmaWarp = kProdWarps;
 constexpr int kEpiWarps = 4;
 constexpr int kTmaWarp = kProdWarps + 1 + kEpiWarps;
 constexpr int kThreads = (kProdWarps + 1 + kEpiWarps + 1) * 32;
+constexpr int kStageA = 2 * BM * BK;  // 32 KB: two sub-tiles of A
+constexpr int kStageB = BN * BK;      // 32 KB
+constexpr int kCtlBytes = 256;            // barriers, tensor-memory slot, abort flag
+constexpr int kEpiConstBytes = 2 * BN * 4;  // per tile: 2048 * colsum[n] and s_w[n] of its columns
+constexpr int kSmemBytes = NS * (kStageA + kStageB) + 1024 /*alignment slack*/ + kCtlBytes + kEpiConstBytes;
+constexpr int kATasks = 4;  // 16-byte packed chunks of A per producer thread per step
+constexpr int kBTasks = 4;
 
 struct GemmParams {
   const uint8_t* dq4;
@@ -86,9 +90,38 @@ struct GemmParams {
   int32_t* acc_out;
   int* status;
   int M, N, K, b, k;
-  int log2k;      // log2(k) when the word path is usable, else -1
-  int SS;         // sparse K steps per tile (static positions through TMA), else 0
+  int log2k;       // log2(k) when the word path is usable, else -1
+  int SS;          // sparse K steps per tile (static positions through TMA), else 0
+  // work list: `n_pairs` tiles of two sub-tiles (256 rows) followed by `n_singles` tiles of one
+  int n_pairs, n_singles, n_split;  // n_split: singles that come from cutting pair tiles in two
+  int mp, mu, tiles_n;              // row pairs, row units (128 rows), column tiles
 };
+
+struct Tile {
+  int m0, n0, nsub;
+};
+
+// Entry j of the work list (identical in every role of every CTA).
+__device__ __forceinline__ Tile tile_of(const GemmParams& p, int j) {
+  Tile t;
+  if (j < p.n_pairs) {
+    t.m0 = (j % p.mp) * (2 * BM);
+    t.n0 = (j / p.mp) * BN;
+    t.nsub = 2;
+  } else {
+    const int s = j - p.n_pairs;
+    t.nsub = 1;
+    if (s < p.n_split) {
+      const int pj = p.n_pairs + s / 2;
+      t.m0 = (pj % p.mp) * (2 * BM) + (s & 1) * BM;
+      t.n0 = (pj / p.mp) * BN;
+    } else {  // the odd last row unit
+      t.m0 = (p.mu - 1) * BM;
+      t.n0 = (s - p.n_split) * BN;
+    }
+  }
+  return t;
+}
 
 // Shared-memory matrix descriptor: K-major, SWIZZLE_128B, 8-row groups 1024 B apart.
 __device__ __forceinline__ uint64_t make_desc(uint32_t saddr) {
@@ -102,7 +135,6 @@ __device__ __forceinline__ uint64_t make_desc(uint32_t saddr) {
 }
 
 // Instruction descriptor: D = s32, A = u8 or s8, B = s8, both K-major, M = 128, N = BN.
-template <int BN>
 __device__ __forceinline__ constexpr uint32_t make_idesc(bool a_signed) {
   return (2u << 4)                       // D format: S32
          | ((a_signed ? 1u : 0u) << 7)   // A format: 0 = unsigned, 1 = signed 8-bit
@@ -110,13 +142,6 @@ __device__ __forceinline__ constexpr uint32_t make_idesc(bool a_signed) {
          | ((uint32_t)(BN >> 3) << 17)   // N
          | ((uint32_t)(BM >> 4) << 24);  // M
 }
-
-template <int BN, int NS>
-struct Smem {
-  static constexpr int kA = BM * BK;  // 16 KB
-  static constexpr int kB = BN * BK;
-  static constexpr int kBytes = NS * (kA + kB) + 1024 /*alignment slack*/ + 256 /*barriers*/;
-};
 
 // Four bank-local indices in one word -> their K positions inside the bank's 32-blocks
 // (even elements first, then odd ones), bytewise.
@@ -126,8 +151,6 @@ __device__ __forceinline__ uint32_t kpos4(uint32_t w) {
 __device__ __forceinline__ uint32_t kpos1(uint32_t jj) {
   return (jj & 0x60u) | ((jj & 1u) << 4) | ((jj & 31u) >> 1);
 }
-
-}  // namespace
 
 __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
@@ -141,45 +164,41 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
       : "memory");
 }
 
-template <int BN, int NS, int MAXT, bool STMA>
+}  // namespace
+
+// MAXT: sparse word tasks per producer lane per K step that are prefetched in registers.
+// STMA: static positions through TMA-fed extra K steps.
+template <int MAXT, bool STMA>
 __global__ void __launch_bounds__(kThreads, 1)
     gemm_kernel(const GemmParams p, const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* smem = smem_raw + (base - smem_u32(smem_raw));
-  uint8_t* sA = smem;                          // NS x [128][128]
-  uint8_t* sB = smem + NS * Smem<BN, NS>::kA;  // NS x [BN][128]
-  uint8_t* sCtl = sB + NS * Smem<BN, NS>::kB;
-  const uint32_t bar_full = smem_u32(sCtl);    // NS x 8 B
-  const uint32_t bar_empty = bar_full + 8 * NS;
-  const uint32_t bar_tfull = bar_empty + 8 * NS;  // 2 x 8 B
-  const uint32_t bar_tempty = bar_tfull + 16;     // 2 x 8 B
-  const uint32_t bar_sfull = bar_tempty + 16;     // NS x 8 B: sparse K steps filled by TMA
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(sCtl + 24 * NS + 32);
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(sCtl + 24 * NS + 40);
+  uint8_t* sA = smem;                 // NS x [256][128]
+  uint8_t* sB = smem + NS * kStageA;  // NS x [256][128]
+  uint8_t* sCtl = sB + NS * kStageB;
+  const uint32_t bar_full = smem_u32(sCtl);       // NS x 8 B: dense K steps filled by the producers
+  const uint32_t bar_empty = bar_full + 8 * NS;   // NS x 8 B: stage consumed by the MMAs
+  const uint32_t bar_sfull = bar_empty + 8 * NS;  // NS x 8 B: sparse K steps filled by TMA
+  const uint32_t bar_tfull = bar_sfull + 8 * NS;  // accumulators complete
+  const uint32_t bar_tempty = bar_tfull + 8;      // accumulators read out
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(sCtl + 24 * NS + 16);  // control block: kCtlBytes
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(sCtl + 24 * NS + 24);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int KS = p.K / BK;
   const int Kh = p.K / 2;
-  const int tiles_m = (p.M + BM - 1) / BM;
-  const int tiles_n = (p.N + BN - 1) / BN;
-  const int ntiles = tiles_m * tiles_n;
+  const int nwork = p.n_pairs + p.n_singles;
   const int SS = STMA ? p.SS : 0;  // sparse K steps that follow the KS dense steps of every tile
 
   if (tid == 0) {
     for (int s = 0; s < NS; ++s) {
-#ifndef SQ_X_NOARRIVE_ALL
       mbar_init(bar_full + 8 * s, kProdThreads);
-#else
-      mbar_init(bar_full + 8 * s, kProdWarps);
-#endif
       mbar_init(bar_empty + 8 * s, 1);
       mbar_init(bar_sfull + 8 * s, 1);
     }
-    for (int bq = 0; bq < 2; ++bq) {
-      mbar_init(bar_tfull + 8 * bq, 1);
-      mbar_init(bar_tempty + 8 * bq, kEpiWarps * 32);
-    }
+    mbar_init(bar_tfull, 1);
+    mbar_init(bar_tempty, kEpiWarps * 32);
     *abort_flag = 0;
     fence_mbar_init();
   }
@@ -194,21 +213,22 @@ __global__ void __launch_bounds__(kThreads, 1)
 
   if (warp < kProdWarps) {
     // =============================================================== producers
+    // Warp pw widens A rows 32*pw .. 32*pw+31 (of the 256 of a stage) and B rows 32*pw .. +31;
+    // lane -> (row % 8, packed 16-byte chunk), so one load instruction covers 8 rows x 64 B.
     const int pw = warp;
-    const int r7 = lane >> 2;  // row within an 8-row group (= row % 8)
-    const int c = lane & 3;    // packed 16-byte chunk within the K step
+    const int r7 = lane >> 2;
+    const int c = lane & 3;
     const uint32_t sw_even = (uint32_t)(((2 * c) ^ r7) << 4);
-    const uint32_t a_row0 = (uint32_t)(16 * pw + r7) * 128u;         // + i * 1024
-    const uint32_t b_row0 = (uint32_t)((BN / 8) * pw + r7) * 128u;   // + i * 1024
-    constexpr int NB_TASKS = BN / 64;                                // B chunks per thread per step
+    const uint32_t row0 = (uint32_t)(32 * pw + r7) * 128u;  // + i * 1024 for task i
     const int GK = (p.K / p.b) * p.k;
     const int nb = (BK / p.b) * p.k;  // sparse entries per row per K step
     const bool word_path = !STMA && p.log2k >= 0;
     const int nw_log = word_path ? (31 - __clz(nb >> 2)) : 0;  // log2(words per row per step)
-    const int ntask = word_path ? ((16 << nw_log) + 31) >> 5 : 0;
+    const int ntask = word_path ? ((32 << nw_log) + 31) >> 5 : 0;  // word tasks per lane (32 rows per warp)
+    const bool sp_prefetch = ntask <= MAXT;
 
     // tile-independent part of this lane's sparse word tasks: task t = lane + 32*j covers
-    // word (t mod words-per-row) of row (t div words-per-row) of the warp's 16 rows
+    // word (t mod words-per-row) of row (t div words-per-row) of the warp's 32 rows
     uint32_t sp_bank4[MAXT];
 #pragma unroll
     for (int j = 0; j < MAXT; ++j) {
@@ -221,145 +241,122 @@ __global__ void __launch_bounds__(kThreads, 1)
       sp_bank4[j] = b4;
     }
 
-    // ---- load side: runs two K steps ahead of the processing side, across tile boundaries
-    int lt = blockIdx.x, lks = 0;
-    const uint8_t* a_ptr[2];
-    const uint8_t* e_ptr[2];
-    const uint8_t* b_ptr[NB_TASKS];
-    size_t sp_off[MAXT];
+    // ---- load side: runs ahead of the processing side, across tile boundaries
+    int lj = blockIdx.x, lks = 0;  // work-list entry and K step of the next load
+    int l_nsub = 0;
+    uint32_t a_off[kATasks], b_off[kBTasks];  // byte offsets into dq4 / wq4 (tensors < 4 GB)
+    uint32_t sp_off[MAXT];
     auto set_load_tile = [&]() {
-      const int tile_m = (lt % tiles_m) * BM;
-      const int tile_n = (lt / tiles_m) * BN;
+      const Tile t = tile_of(p, lj);
+      l_nsub = t.nsub;
 #pragma unroll
-      for (int i = 0; i < 2; ++i) {
-        const int m = min(tile_m + 16 * pw + 8 * i + r7, p.M - 1);  // rows past M repeat the last row
-        a_ptr[i] = p.dq4 + (size_t)m * Kh + c * 16;
-        e_ptr[i] = p.shift + m;
+      for (int i = 0; i < kATasks; ++i) {
+        const int m = min(t.m0 + 32 * pw + 8 * i + r7, p.M - 1);  // rows past M repeat the last row
+        a_off[i] = (uint32_t)m * (uint32_t)Kh + c * 16;
       }
 #pragma unroll
-      for (int i = 0; i < NB_TASKS; ++i) {
-        const int n = min(tile_n + (BN / 8) * pw + 8 * i + r7, p.N - 1);
-        b_ptr[i] = p.wq4 + (size_t)n * Kh + c * 16;
+      for (int i = 0; i < kBTasks; ++i) {
+        const int n = min(t.n0 + 32 * pw + 8 * i + r7, p.N - 1);
+        b_off[i] = (uint32_t)n * (uint32_t)Kh + c * 16;
       }
 #pragma unroll
       for (int j = 0; j < MAXT; ++j) {
-        const int t = lane + 32 * j;
-        const int m = min(tile_m + 16 * pw + ((t >> nw_log) & 15), p.M - 1);
-        sp_off[j] = (size_t)m * GK + 4 * (t & ((1 << nw_log) - 1));
+        const int tt = lane + 32 * j;
+        const int m = min(t.m0 + 32 * pw + ((tt >> nw_log) & 31), p.M - 1);
+        sp_off[j] = (uint32_t)m * (uint32_t)GK + 4 * (tt & ((1 << nw_log) - 1));
       }
     };
-    uint4 ra[2][2], rb[2][NB_TASKS];  // [prefetch slot][task]
-    uint32_t re[2][2], sv[2][MAXT], si[2][MAXT];
+    uint4 ra[2][kATasks], rb[2][kBTasks];  // [prefetch slot][task]
+    uint32_t sv[2][MAXT], si[2][MAXT];
     auto load_next = [&](int slot) {
-      if (lt >= ntiles) return;
+      if (lj >= nwork) return;
+      const uint32_t koff = (uint32_t)lks * 64u;
 #ifdef SQ_X_NOLOAD
-      if (lt >= 0) {
-        for (int i = 0; i < 2; ++i) ra[slot][i] = make_uint4(lks, lt, 3, 4);
-        for (int i = 0; i < NB_TASKS; ++i) rb[slot][i] = make_uint4(lks, lt, 5, 6);
-        if (++lks == KS) { lks = 0; lt += gridDim.x; }
+      if (lj >= 0) {
+        for (int i = 0; i < kATasks; ++i) ra[slot][i] = make_uint4(lks, lj, 3, 4);
+        for (int i = 0; i < kBTasks; ++i) rb[slot][i] = make_uint4(lks, lj, 5, 6);
+        if (++lks == KS) { lks = 0; lj += gridDim.x; if (lj < nwork) set_load_tile(); }
         return;
       }
 #endif
+      // a single-sub-tile entry only has A rows 0..127: warps 4-7 have none
+      const bool has_a = l_nsub == 2 || pw < 4;
+      if (has_a) {
 #pragma unroll
-      for (int i = 0; i < 2; ++i) {
-        ra[slot][i] = ldg_nc_v4(a_ptr[i] + (size_t)lks * 64);
-#if SQ_E_PER_STEP
-        re[slot][i] = __ldg(e_ptr[i]);
-#endif
+        for (int i = 0; i < kATasks; ++i) ra[slot][i] = ldg_nc_v4(p.dq4 + a_off[i] + koff);
       }
 #pragma unroll
-      for (int i = 0; i < NB_TASKS; ++i) rb[slot][i] = ldg_nc_v4(b_ptr[i] + (size_t)lks * 64);
-#if SQ_SPARSE_PREFETCH
-      if (word_path) {
+      for (int i = 0; i < kBTasks; ++i) rb[slot][i] = ldg_nc_v4(p.wq4 + b_off[i] + koff);
+      if (word_path && sp_prefetch && has_a) {
 #pragma unroll
         for (int j = 0; j < MAXT; ++j) {
           if (j < ntask) {
-            const size_t o = sp_off[j] + (size_t)lks * nb;
+            const uint32_t o = sp_off[j] + (uint32_t)lks * (uint32_t)nb;
             sv[slot][j] = __ldg(reinterpret_cast<const uint32_t*>(p.vals + o));
             const int q4 = 4 * ((lane + 32 * j) & ((1 << nw_log) - 1));
-            si[slot][j] = p.idx != nullptr
-                              ? __ldg(reinterpret_cast<const uint32_t*>(p.idx + o))
-                              : __ldg(reinterpret_cast<const uint32_t*>(p.pos + (size_t)lks * nb + q4));
+            si[slot][j] = p.idx != nullptr ? __ldg(reinterpret_cast<const uint32_t*>(p.idx + o))
+                                           : __ldg(reinterpret_cast<const uint32_t*>(p.pos + lks * nb + q4));
           }
         }
       }
-#endif
       if (++lks == KS) {
         lks = 0;
-        lt += gridDim.x;
-        if (lt < ntiles) set_load_tile();
+        lj += gridDim.x;
+        if (lj < nwork) set_load_tile();
       }
     };
 
     // ---- processing side
     uint32_t it = 0;
-    uint32_t pmul[2] = {1, 1}, poff[2] = {0, 0};
-    int pt = blockIdx.x, pks = 0;  // tile and K step being processed (the byte-wise path needs them)
+    uint32_t pmul[kATasks], poff[kATasks];
+#pragma unroll
+    for (int i = 0; i < kATasks; ++i) {
+      pmul[i] = 1;
+      poff[i] = 0;
+    }
+    int pj = blockIdx.x, pks = 0;  // work-list entry and K step being processed
+    Tile pt = tile_of(p, pj);
     auto process = [&](int slot) -> bool {
       const int s = it % NS;
       if (!mbar_wait(bar_empty + 8 * s, ((it / NS) & 1u) ^ 1u, abort_flag)) return false;
-      uint8_t* a_st = sA + s * Smem<BN, NS>::kA;
-      uint8_t* b_st = sB + s * Smem<BN, NS>::kB;
-#if !SQ_SPARSE_PREFETCH
-      if (word_path) {
-        const int tile_m = (pt % tiles_m) * BM;
+      uint8_t* a_st = sA + s * kStageA;
+      uint8_t* b_st = sB + s * kStageB;
+      const bool has_a = pt.nsub == 2 || pw < 4;
+      if (pks == 0 && has_a) {  // the rows' shifts change with the tile only
 #pragma unroll
-        for (int j = 0; j < MAXT; ++j) {
-          if (j < ntask) {
-            const int t = lane + 32 * j;
-            const int m = min(tile_m + 16 * pw + ((t >> nw_log) & 15), p.M - 1);
-            const int q4 = 4 * (t & ((1 << nw_log) - 1));
-            const size_t o = (size_t)m * GK + q4 + (size_t)pks * nb;
-            sv[slot][j] = __ldg(reinterpret_cast<const uint32_t*>(p.vals + o));
-            si[slot][j] = p.idx != nullptr
-                              ? __ldg(reinterpret_cast<const uint32_t*>(p.idx + o))
-                              : __ldg(reinterpret_cast<const uint32_t*>(p.pos + (size_t)pks * nb + q4));
-          }
-        }
-      }
-#endif
-#if !SQ_E_PER_STEP
-      if (pks == 0) {  // the rows' shifts change with the tile only
-        const int tile_m = (pt % tiles_m) * BM;
-#pragma unroll
-        for (int i = 0; i < 2; ++i) {
-          const uint32_t e = p.shift[min(tile_m + 16 * pw + 8 * i + r7, p.M - 1)];
+        for (int i = 0; i < kATasks; ++i) {
+          const uint32_t e = p.shift[min(pt.m0 + 32 * pw + 8 * i + r7, p.M - 1)];
           pmul[i] = 1u << e;
           poff[i] = 0x01010101u * (128u - (8u << e));
         }
       }
-#endif
 #ifdef SQ_X_NOWORK
       if (ra[slot][0].x == 0x12345u) a_st[0] = (uint8_t)rb[slot][0].x;  // keep the loads alive
       if (false)
 #endif
       // ---- widen A: nibble -> u * 2^e + (128 - 8 * 2^e)
+      if (has_a) {
 #pragma unroll
-      for (int i = 0; i < 2; ++i) {
-        const uint32_t in[4] = {ra[slot][i].x, ra[slot][i].y, ra[slot][i].z, ra[slot][i].w};
-#if SQ_E_PER_STEP
-        const uint32_t a_mul = 1u << re[slot][i];
-        const uint32_t a_off = 0x01010101u * (128u - (8u << re[slot][i]));
-#else
-        const uint32_t a_mul = pmul[i], a_off = poff[i];
-#endif
-        uint32_t ev[4], od[4];
+        for (int i = 0; i < kATasks; ++i) {
+          const uint32_t in[4] = {ra[slot][i].x, ra[slot][i].y, ra[slot][i].z, ra[slot][i].w};
+          uint32_t ev[4], od[4];
 #pragma unroll
-        for (int q = 0; q < 4; ++q) {
-          const uint32_t u = in[q] ^ 0x88888888u;
-          ev[q] = (u & 0x0F0F0F0Fu) * a_mul + a_off;
-          od[q] = ((u >> 4) & 0x0F0F0F0Fu) * a_mul + a_off;
+          for (int q = 0; q < 4; ++q) {
+            const uint32_t u = in[q] ^ 0x88888888u;
+            ev[q] = (u & 0x0F0F0F0Fu) * pmul[i] + poff[i];
+            od[q] = ((u >> 4) & 0x0F0F0F0Fu) * pmul[i] + poff[i];
+          }
+          uint8_t* dst = a_st + row0 + i * 1024;
+          *reinterpret_cast<uint4*>(dst + sw_even) = make_uint4(ev[0], ev[1], ev[2], ev[3]);
+          *reinterpret_cast<uint4*>(dst + (sw_even ^ 16u)) = make_uint4(od[0], od[1], od[2], od[3]);
         }
-        uint8_t* dst = a_st + a_row0 + i * 1024;
-        *reinterpret_cast<uint4*>(dst + sw_even) = make_uint4(ev[0], ev[1], ev[2], ev[3]);
-        *reinterpret_cast<uint4*>(dst + (sw_even ^ 16u)) = make_uint4(od[0], od[1], od[2], od[3]);
       }
       // ---- widen B: nibble -> 16 * code
 #ifdef SQ_X_NOWORK
       if (false)
 #endif
 #pragma unroll
-      for (int i = 0; i < NB_TASKS; ++i) {
+      for (int i = 0; i < kBTasks; ++i) {
         const uint32_t in[4] = {rb[slot][i].x, rb[slot][i].y, rb[slot][i].z, rb[slot][i].w};
         uint32_t ev[4], od[4];
 #pragma unroll
@@ -367,19 +364,19 @@ __global__ void __launch_bounds__(kThreads, 1)
           ev[q] = (in[q] << 4) & 0xF0F0F0F0u;
           od[q] = in[q] & 0xF0F0F0F0u;
         }
-        uint8_t* dst = b_st + b_row0 + i * 1024;
+        uint8_t* dst = b_st + row0 + i * 1024;
         *reinterpret_cast<uint4*>(dst + sw_even) = make_uint4(ev[0], ev[1], ev[2], ev[3]);
         *reinterpret_cast<uint4*>(dst + (sw_even ^ 16u)) = make_uint4(od[0], od[1], od[2], od[3]);
       }
-      __syncwarp();  // this warp's 16 A rows are complete before any lane overwrites bytes in them
-      // ---- sparse INT8 entries overwrite their places (rows 16*pw .. 16*pw+15 of the tile)
-      if (word_path) {
+      // ---- sparse INT8 entries overwrite their places (rows 32*pw .. 32*pw+31 of the stage)
+      if (!STMA && has_a) {
+        __syncwarp();  // this warp's A rows are complete before any lane overwrites bytes in them
+        if (word_path) {
 #pragma unroll
-        for (int j = 0; j < MAXT; ++j) {
-          if (j < ntask) {
-            const int t = lane + 32 * j;
-            if ((t >> nw_log) < 16) {
-              const int row = 16 * pw + (t >> nw_log);
+          for (int j = 0; j < MAXT; ++j) {
+            if (j < ntask && sp_prefetch) {
+              const int tt = lane + 32 * j;
+              const int row = 32 * pw + (tt >> nw_log);
               const uint32_t r7s = 0x01010101u * (uint32_t)((row & 7) << 4);
               const uint32_t pos4 = (kpos4(si[slot][j]) + sp_bank4[j]) ^ r7s;
               const uint32_t vx = sv[slot][j] ^ 0x80808080u;
@@ -388,34 +385,46 @@ __global__ void __launch_bounds__(kThreads, 1)
               for (int u = 0; u < 4; ++u) rowp[(pos4 >> (8 * u)) & 0xFFu] = (uint8_t)(vx >> (8 * u));
             }
           }
-        }
-      } else if (!STMA) {
-        const int tile_m = (pt % tiles_m) * BM;
-        for (int t = lane; t < 16 * nb; t += 32) {
-          const int row_l = t / nb, i = t - row_l * nb;
-          const int row = 16 * pw + row_l;
-          const int m = min(tile_m + row, p.M - 1);
-          const int bank = i / p.k, slot_i = i - bank * p.k;
-          const int g = pks * (BK / p.b) + bank;
-          const size_t entry = (size_t)m * GK + (size_t)g * p.k + slot_i;
-          const uint32_t local = p.idx != nullptr ? p.idx[entry] : p.pos[(size_t)g * p.k + slot_i];
-          const uint32_t kp = (kpos1(local) + (uint32_t)(bank * p.b)) ^ (uint32_t)((row & 7) << 4);
-          a_st[row * 128 + kp] = (uint8_t)((uint8_t)p.vals[entry] ^ 0x80u);
+          if (!sp_prefetch) {  // many entries per step: word loads without register prefetch
+            for (int tt = lane; tt < (32 << nw_log); tt += 32) {
+              const int row_l = tt >> nw_log, q = tt & ((1 << nw_log) - 1);
+              const int row = 32 * pw + row_l;
+              const int m = min(pt.m0 + row, p.M - 1);
+              const uint32_t o = (uint32_t)m * (uint32_t)GK + (uint32_t)pks * (uint32_t)nb + 4 * q;
+              const uint32_t vw = __ldg(reinterpret_cast<const uint32_t*>(p.vals + o));
+              const uint32_t iw = p.idx != nullptr ? __ldg(reinterpret_cast<const uint32_t*>(p.idx + o))
+                                                   : __ldg(reinterpret_cast<const uint32_t*>(p.pos + pks * nb + 4 * q));
+              uint32_t b4 = 0;
+#pragma unroll
+              for (int u = 0; u < 4; ++u) b4 |= (uint32_t)(((4 * q + u) >> p.log2k) * p.b) << (8 * u);
+              const uint32_t pos4 = (kpos4(iw) + b4) ^ (0x01010101u * (uint32_t)((row & 7) << 4));
+              const uint32_t vx = vw ^ 0x80808080u;
+              uint8_t* rowp = a_st + row * 128;
+#pragma unroll
+              for (int u = 0; u < 4; ++u) rowp[(pos4 >> (8 * u)) & 0xFFu] = (uint8_t)(vx >> (8 * u));
+            }
+          }
+        } else {
+          for (int tt = lane; tt < 32 * nb; tt += 32) {
+            const int row_l = tt / nb, i = tt - row_l * nb;
+            const int row = 32 * pw + row_l;
+            const int m = min(pt.m0 + row, p.M - 1);
+            const int bank = i / p.k, slot_i = i - bank * p.k;
+            const int g = pks * (BK / p.b) + bank;
+            const size_t entry = (size_t)m * GK + (size_t)g * p.k + slot_i;
+            const uint32_t local = p.idx != nullptr ? p.idx[entry] : p.pos[(size_t)g * p.k + slot_i];
+            const uint32_t kp = (kpos1(local) + (uint32_t)(bank * p.b)) ^ (uint32_t)((row & 7) << 4);
+            a_st[row * 128 + kp] = (uint8_t)((uint8_t)p.vals[entry] ^ 0x80u);
+          }
         }
       }
-#ifndef SQ_X_NOFENCE
       fence_proxy_async_smem();  // generic-proxy writes -> visible to the tensor core's async reads
-#endif
-#ifndef SQ_X_NOARRIVE_ALL
       mbar_arrive(bar_full + 8 * s);
-#else
-      __syncwarp();
-      if (lane == 0) mbar_arrive(bar_full + 8 * s);
-#endif
       ++it;
       if (++pks == KS) {
         pks = 0;
-        pt += gridDim.x;
+        pj += gridDim.x;
+        if (pj < nwork) pt = tile_of(p, pj);
         // The sparse K steps of the tile use the next SS ring slots (TMA fills them).  They are
         // waited for one by one, not skipped: a parity wait only tells the current phase from
         // the previous one, so no role may fall more than one use behind on any stage.
@@ -426,7 +435,7 @@ __global__ void __launch_bounds__(kThreads, 1)
       return true;
     };
 
-    const int my_tiles = (ntiles - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
+    const int my_tiles = (nwork - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
     const int total = my_tiles * KS;
     set_load_tile();
     load_next(0);
@@ -442,17 +451,16 @@ __global__ void __launch_bounds__(kThreads, 1)
   } else if (warp == kMmaWarp) {
     // =============================================================== MMA issuer
     if (lane == 0) {
-      constexpr uint32_t idesc = make_idesc<BN>(false);
-      constexpr uint32_t idesc_sparse = make_idesc<BN>(true);
+      constexpr uint32_t idesc = make_idesc(false);
+      constexpr uint32_t idesc_sparse = make_idesc(true);
       uint32_t it = 0, tc = 0;
       uint32_t ph_dense = 0, ph_sparse = 0;  // per-stage phase bits of the two kinds of "full" barrier
       bool ok = true;
-      for (int tile = blockIdx.x; tile < ntiles && ok; tile += gridDim.x, ++tc) {
-        const uint32_t buf = tc & 1u;
-        ok = mbar_wait(bar_tempty + 8 * buf, ((tc >> 1) & 1u) ^ 1u, abort_flag);
+      for (int j = blockIdx.x; j < nwork && ok; j += gridDim.x, ++tc) {
+        const int nsub = tile_of(p, j).nsub;
+        ok = mbar_wait(bar_tempty, (tc & 1u) ^ 1u, abort_flag);  // previous tile's accumulators read out
         if (!ok) break;
         tc_fence_after();
-        const uint32_t d = tmem + buf * BN;
         for (int ks = 0; ks < KS + SS; ++ks, ++it) {
           const int s = it % NS;
           const bool sparse_step = ks >= KS;
@@ -465,26 +473,27 @@ __global__ void __launch_bounds__(kThreads, 1)
           }
           if (!ok) break;
           tc_fence_after();
-          const uint64_t da = make_desc(smem_u32(sA + s * Smem<BN, NS>::kA));
-          const uint64_t db = make_desc(smem_u32(sB + s * Smem<BN, NS>::kB));
+          const uint64_t db = make_desc(smem_u32(sB + s * kStageB));
           const uint32_t id = sparse_step ? idesc_sparse : idesc;
+          for (int sub = 0; sub < nsub; ++sub) {
+            const uint64_t da = make_desc(smem_u32(sA + s * kStageA + sub * (BM * BK)));
 #pragma unroll
-          for (int kk = 0; kk < BK / 32; ++kk)  // 32 bytes of K per MMA: +2 in 16-byte address units
-            umma_i8(d, da + 2 * kk, db + 2 * kk, id, (ks > 0 || kk > 0) ? 1u : 0u);
+            for (int kk = 0; kk < BK / 32; ++kk)  // 32 bytes of K per MMA: +2 in 16-byte address units
+              umma_i8(tmem + sub * BN, da + 2 * kk, db + 2 * kk, id, (ks > 0 || kk > 0) ? 1u : 0u);
+          }
           umma_commit(bar_empty + 8 * s);
         }
-        if (ok) umma_commit(bar_tfull + 8 * buf);
+        if (ok) umma_commit(bar_tfull);
       }
     }
     __syncwarp();
   } else if (warp == kTmaWarp) {
     // =============================================================== TMA (sparse K steps)
     if (STMA && lane == 0) {
-      uint32_t tc = 0, it = 0;
+      uint32_t it = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; tile < ntiles && ok; tile += gridDim.x, ++tc) {
-        const int tile_m = (tile % tiles_m) * BM;
-        const int tile_n = (tile / tiles_m) * BN;
+      for (int j = blockIdx.x; j < nwork && ok; j += gridDim.x) {
+        const Tile t = tile_of(p, j);
         // every ring slot is waited for in order (see the producers); only the sparse ones are filled
         for (int step = 0; step < KS + SS && ok; ++step, ++it) {
           const int s = it % NS;
@@ -492,9 +501,9 @@ __global__ void __launch_bounds__(kThreads, 1)
           if (!ok || step < KS) continue;
           const int ss = step - KS;
           // rows past M / N and columns past G*k are filled with zeros by the TMA unit
-          mbar_expect_tx(bar_sfull + 8 * s, (uint32_t)(Smem<BN, NS>::kA + Smem<BN, NS>::kB));
-          tma_load_2d(smem_u32(sA + s * Smem<BN, NS>::kA), &map_a, ss * BK, tile_m, bar_sfull + 8 * s);
-          tma_load_2d(smem_u32(sB + s * Smem<BN, NS>::kB), &map_b, ss * BK, tile_n, bar_sfull + 8 * s);
+          mbar_expect_tx(bar_sfull + 8 * s, (uint32_t)(kStageA + kStageB));
+          tma_load_2d(smem_u32(sA + s * kStageA), &map_a, ss * BK, t.m0, bar_sfull + 8 * s);
+          tma_load_2d(smem_u32(sB + s * kStageB), &map_b, ss * BK, t.n0, bar_sfull + 8 * s);
         }
       }
     }
@@ -502,52 +511,67 @@ __global__ void __launch_bounds__(kThreads, 1)
   } else {
     // =============================================================== epilogue
     const int q = warp & 3;  // TMEM lane quarter this warp may read
+    const int et = tid - (kMmaWarp + 1) * 32;  // 0..127 among the epilogue threads
+    int32_t* s_cs = reinterpret_cast<int32_t*>(sCtl + kCtlBytes);  // 2048 * colsum of the tile's columns
+    float* s_sw = reinterpret_cast<float*>(sCtl + kCtlBytes + BN * 4);
     uint32_t tc = 0;
-    for (int tile = blockIdx.x; tile < ntiles; tile += gridDim.x, ++tc) {
-      const int tile_m = (tile % tiles_m) * BM;
-      const int tile_n = (tile / tiles_m) * BN;
-      const uint32_t buf = tc & 1u;
-      if (!mbar_wait_idle(bar_tfull + 8 * buf, (tc >> 1) & 1u, abort_flag)) break;
+    for (int j = blockIdx.x; j < nwork; j += gridDim.x, ++tc) {
+      const Tile t = tile_of(p, j);
+      // the tile's column constants are fetched while the main loop is still running
+      for (int cc = et; cc < BN; cc += kEpiWarps * 32) {
+        const int n = min(t.n0 + cc, p.N - 1);
+        s_cs[cc] = 2048 * __ldg(p.colsum + n);
+        s_sw[cc] = __ldg(p.s_w + n);
+      }
+      asm volatile("bar.sync 1, %0;" ::"n"(kEpiWarps * 32) : "memory");
+      if (!mbar_wait_idle(bar_tfull, tc & 1u, abort_flag)) break;
       tc_fence_after();
-      const int m = tile_m + 32 * q + lane;
-      const float sh = (m < p.M) ? p.s_hi[m] : 0.f;
-      for (int c0 = 0; c0 < BN; c0 += 32) {
-        uint32_t v[32];
-        tmem_ld32(tmem + ((uint32_t)(32 * q) << 16) + buf * BN + (uint32_t)c0, v);
-        tmem_ld_wait();
-        const int n0 = tile_n + c0;
-        if (m < p.M && n0 < p.N) {
+#ifdef SQ_X_NOEPI
+      for (int sub = 0; sub < 0; ++sub) {
+#else
+      for (int sub = 0; sub < t.nsub; ++sub) {
+#endif
+        const int m = t.m0 + sub * BM + 32 * q + lane;
+        const float sh = (m < p.M) ? p.s_hi[m] : 0.f;
+        for (int c0 = 0; c0 < BN; c0 += 32) {
+          uint32_t v[32];
+          tmem_ld32(tmem + ((uint32_t)(32 * q) << 16) + (uint32_t)(sub * BN + c0), v);
+          tmem_ld_wait();
+          const int n0 = t.n0 + c0;
+          if (m < p.M && n0 < p.N) {
 #pragma unroll
-          for (int c8 = 0; c8 < 32; c8 += 8) {
-            if (n0 + c8 < p.N) {  // N % 8 == 0: a group of 8 columns is all in or all out
-              int acc[8];
-              uint32_t o[4];
-              const int4 cs0 = __ldg(reinterpret_cast<const int4*>(p.colsum + n0 + c8));
-              const int4 cs1 = __ldg(reinterpret_cast<const int4*>(p.colsum + n0 + c8 + 4));
-              const float4 sw0 = __ldg(reinterpret_cast<const float4*>(p.s_w + n0 + c8));
-              const float4 sw1 = __ldg(reinterpret_cast<const float4*>(p.s_w + n0 + c8 + 4));
-              const int cs[8] = {cs0.x, cs0.y, cs0.z, cs0.w, cs1.x, cs1.y, cs1.z, cs1.w};
-              const float sw[8] = {sw0.x, sw0.y, sw0.z, sw0.w, sw1.x, sw1.y, sw1.z, sw1.w};
+            for (int c8 = 0; c8 < 32; c8 += 8) {
+              if (n0 + c8 < p.N) {  // N % 8 == 0: a group of 8 columns is all in or all out
+                int acc[8];
+                uint32_t o[4];
+                const int4 cs0 = *reinterpret_cast<const int4*>(s_cs + c0 + c8);
+                const int4 cs1 = *reinterpret_cast<const int4*>(s_cs + c0 + c8 + 4);
+                const float4 sw0 = *reinterpret_cast<const float4*>(s_sw + c0 + c8);
+                const float4 sw1 = *reinterpret_cast<const float4*>(s_sw + c0 + c8 + 4);
+                const int cs[8] = {cs0.x, cs0.y, cs0.z, cs0.w, cs1.x, cs1.y, cs1.z, cs1.w};
+                const float sw[8] = {sw0.x, sw0.y, sw0.z, sw0.w, sw1.x, sw1.y, sw1.z, sw1.w};
 #pragma unroll
-              for (int cc = 0; cc < 8; ++cc) acc[cc] = ((int)v[c8 + cc] - 2048 * cs[cc]) >> 4;
+                for (int cc = 0; cc < 8; ++cc) acc[cc] = ((int)v[c8 + cc] - cs[cc]) >> 4;
 #pragma unroll
-              for (int cc = 0; cc < 8; cc += 2) {
-                const float f0 = ((float)acc[cc] * sh) * sw[cc];
-                const float f1 = ((float)acc[cc + 1] * sh) * sw[cc + 1];
-                o[cc >> 1] = f32_to_bf16_bits(f0) | (f32_to_bf16_bits(f1) << 16);
-              }
-              *reinterpret_cast<uint4*>(p.out + (size_t)m * p.N + n0 + c8) = make_uint4(o[0], o[1], o[2], o[3]);
-              if (p.acc_out != nullptr) {
-                int4* dst = reinterpret_cast<int4*>(p.acc_out + (size_t)m * p.N + n0 + c8);
-                dst[0] = make_int4(acc[0], acc[1], acc[2], acc[3]);
-                dst[1] = make_int4(acc[4], acc[5], acc[6], acc[7]);
+                for (int cc = 0; cc < 8; cc += 2) {
+                  const float f0 = ((float)acc[cc] * sh) * sw[cc];
+                  const float f1 = ((float)acc[cc + 1] * sh) * sw[cc + 1];
+                  o[cc >> 1] = f32_to_bf16_bits(f0) | (f32_to_bf16_bits(f1) << 16);
+                }
+                *reinterpret_cast<uint4*>(p.out + (size_t)m * p.N + n0 + c8) = make_uint4(o[0], o[1], o[2], o[3]);
+                if (p.acc_out != nullptr) {
+                  int4* dst = reinterpret_cast<int4*>(p.acc_out + (size_t)m * p.N + n0 + c8);
+                  dst[0] = make_int4(acc[0], acc[1], acc[2], acc[3]);
+                  dst[1] = make_int4(acc[4], acc[5], acc[6], acc[7]);
+                }
               }
             }
           }
         }
       }
       tc_fence_before();
-      mbar_arrive(bar_tempty + 8 * buf);
+      mbar_arrive(bar_tempty);
+      asm volatile("bar.sync 1, %0;" ::"n"(kEpiWarps * 32) : "memory");  // all four warps are done with the constants
     }
   }
 
@@ -560,7 +584,6 @@ __global__ void __launch_bounds__(kThreads, 1)
 cudaError_t launch_gemm(int b, int k, const sq_encoded& A, const sq_weights& W,
                         const uint8_t* positions, int64_t M, int64_t N, int64_t K, uint16_t* out,
                         int32_t* acc_out, int* status, cudaStream_t st) {
-  constexpr int BN = 256, NS = 4;
   GemmParams p;
   p.dq4 = A.dq4;
   p.vals = A.vals;
@@ -579,10 +602,12 @@ cudaError_t launch_gemm(int b, int k, const sq_encoded& A, const sq_weights& W,
   p.K = (int)K;
   p.b = b;
   p.k = k;
+  // the kernel addresses the packed tensors with 32-bit byte offsets
+  const int64_t GK = (K / b) * k;
+  if (M * (K / 2) >= (1ll << 32) || N * (K / 2) >= (1ll << 32) || M * GK >= (1ll << 32)) return cudaErrorInvalidValue;
   // 32-bit word loads of the sparse entries need k a power of two, at least four entries per
   // row per K step and 4-byte aligned row starts; anything else takes the byte-wise path.
   const int nb = (BK / b) * k;
-  const int64_t GK = (K / b) * k;
   const bool pow2 = (k & (k - 1)) == 0;
   p.log2k = -1;
   if (pow2 && nb >= 4 && GK % 4 == 0) {
@@ -600,9 +625,20 @@ cudaError_t launch_gemm(int b, int k, const sq_encoded& A, const sq_weights& W,
     err = cudaDeviceGetAttribute(&sm_count[dev], cudaDevAttrMultiProcessorCount, dev);
     if (err != cudaSuccess) return err;
   }
-  const int64_t ntiles = ((M + BM - 1) / BM) * ((N + BN - 1) / BN);
-  const unsigned grid = (unsigned)(ntiles < sm_count[dev] ? ntiles : sm_count[dev]);
-  const int smem = Smem<BN, NS>::kBytes;
+  const int sms = sm_count[dev];
+
+  // Work list: 256-row tiles while they fill whole waves of the SMs; the remainder of the
+  // row pairs is cut into 128-row tiles so the last wave spreads over twice as many SMs.
+  p.mu = (int)((M + BM - 1) / BM);
+  p.mp = p.mu / 2;
+  p.tiles_n = (int)((N + BN - 1) / BN);
+  const int64_t pair_tiles = (int64_t)p.mp * p.tiles_n;
+  const int64_t as_pairs = (pair_tiles / sms) * sms;
+  p.n_pairs = (int)as_pairs;
+  p.n_split = (int)(2 * (pair_tiles - as_pairs));
+  p.n_singles = p.n_split + (p.mu & 1) * p.tiles_n;
+  const int64_t nwork = (int64_t)p.n_pairs + p.n_singles;
+  const unsigned grid = (unsigned)(nwork < sms ? nwork : sms);
 
   // Static positions: the sparse product runs as extra K steps over vals [M, G*k] and
   // w_sparse [N, G*k], fetched by TMA.  A TMA row pitch must be a multiple of 16 bytes; any
@@ -626,7 +662,7 @@ cudaError_t launch_gemm(int b, int k, const sq_encoded& A, const sq_weights& W,
     const cuuint64_t pitch[1] = {(cuuint64_t)GK};
     const cuuint64_t dim_a[2] = {(cuuint64_t)GK, (cuuint64_t)M};
     const cuuint64_t dim_b[2] = {(cuuint64_t)GK, (cuuint64_t)N};
-    const cuuint32_t box_a[2] = {BK, BM};
+    const cuuint32_t box_a[2] = {BK, 2 * BM};
     const cuuint32_t box_b[2] = {BK, BN};
     if (encode(&map_a, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<int8_t*>(A.vals), dim_a, pitch, box_a, estr,
                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
@@ -639,16 +675,15 @@ cudaError_t launch_gemm(int b, int k, const sq_encoded& A, const sq_weights& W,
     p.SS = (int)((GK + BK - 1) / BK);
   }
 
-#define SQ_LAUNCH_GEMM(MAXT_, STMA_)                                                                  \
-  do {                                                                                                \
-    err = cudaFuncSetAttribute(gemm_kernel<BN, NS, MAXT_, STMA_>,                                     \
-                               cudaFuncAttributeMaxDynamicSharedMemorySize, smem);                    \
-    if (err != cudaSuccess) return err;                                                               \
-    gemm_kernel<BN, NS, MAXT_, STMA_><<<grid, kThreads, smem, st>>>(p, map_a, map_b);                 \
+#define SQ_LAUNCH_GEMM(MAXT_, STMA_)                                                                        \
+  do {                                                                                                      \
+    err = cudaFuncSetAttribute(gemm_kernel<MAXT_, STMA_>, cudaFuncAttributeMaxDynamicSharedMemorySize,      \
+                               kSmemBytes);                                                                 \
+    if (err != cudaSuccess) return err;                                                                     \
+    gemm_kernel<MAXT_, STMA_><<<grid, kThreads, kSmemBytes, st>>>(p, map_a, map_b);                         \
   } while (0)
   if (stma) SQ_LAUNCH_GEMM(1, true);
-  else if (nb <= 16) SQ_LAUNCH_GEMM(2, false);
-  else SQ_LAUNCH_GEMM(8, false);
+  else SQ_LAUNCH_GEMM(4, false);
 #undef SQ_LAUNCH_GEMM
   return cudaGetLastError();
 }
