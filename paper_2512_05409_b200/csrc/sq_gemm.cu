@@ -61,18 +61,23 @@ namespace {
 constexpr int BM = 128;   // rows of one sub-tile = TMEM lanes
 constexpr int BN = 256;   // output channels per tile = TMEM columns of one accumulator
 constexpr int BK = 128;   // K elements per pipeline step = bytes per operand row
-constexpr int NS = 3;     // shared-memory stages
+constexpr int NS = 2;     // stages of widened (8-bit) operands
+constexpr int NP = 2;     // stages of packed (4-bit) operands as TMA delivers them
 constexpr int kProdWarps = 8;
 constexpr int kProdThreads = kProdWarps * 32;
 constexpr int kMmaWarp = kProdWarps;
 constexpr int kEpiWarps = 4;
-constexpr int kTmaWarp = kProdWarps + 1 + kEpiWarps;
-constexpr int kThreads = (kProdWarps + 1 + kEpiWarps + 1) * 32;
+constexpr int kTmaWarp = kProdWarps + 1 + kEpiWarps;  // packed dense tiles
+constexpr int kTmaSparseWarp = kTmaWarp + 1;          // INT8 tiles of the sparse K steps
+constexpr int kThreads = (kProdWarps + 1 + kEpiWarps + 2) * 32;
 constexpr int kStageA = 2 * BM * BK;  // 32 KB: two sub-tiles of A
 constexpr int kStageB = BN * BK;      // 32 KB
 constexpr int kCtlBytes = 256;            // barriers, tensor-memory slot, abort flag
 constexpr int kEpiConstBytes = 2 * BN * 4;  // per tile: 2048 * colsum[n] and s_w[n] of its columns
-constexpr int kSmemBytes = NS * (kStageA + kStageB) + 1024 /*alignment slack*/ + kCtlBytes + kEpiConstBytes;
+constexpr int kPackA = 2 * BM * (BK / 2);  // 16 KB: 256 rows x 64 packed bytes
+constexpr int kPackB = BN * (BK / 2);      // 16 KB
+constexpr int kSmemBytes =
+    NS * (kStageA + kStageB) + NP * (kPackA + kPackB) + 1024 /*alignment slack*/ + kCtlBytes + kEpiConstBytes;
 constexpr int kATasks = 4;  // 16-byte packed chunks of A per producer thread per step
 constexpr int kBTasks = 4;
 
@@ -170,24 +175,28 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
 // STMA: static positions through TMA-fed extra K steps.
 template <int MAXT, bool STMA>
 __global__ void __launch_bounds__(kThreads, 1)
-    gemm_kernel(const GemmParams p, const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b) {
+    gemm_kernel(const GemmParams p, const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+                const __grid_constant__ CUtensorMap map_a4, const __grid_constant__ CUtensorMap map_b4) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* smem = smem_raw + (base - smem_u32(smem_raw));
-  uint8_t* sA = smem;                 // NS x [256][128]
-  uint8_t* sB = smem + NS * kStageA;  // NS x [256][128]
-  uint8_t* sCtl = sB + NS * kStageB;
-  const uint32_t bar_full = smem_u32(sCtl);       // NS x 8 B: dense K steps filled by the producers
-  const uint32_t bar_empty = bar_full + 8 * NS;   // NS x 8 B: stage consumed by the MMAs
-  const uint32_t bar_sfull = bar_empty + 8 * NS;  // NS x 8 B: sparse K steps filled by TMA
-  const uint32_t bar_tfull = bar_sfull + 8 * NS;  // accumulators complete
-  const uint32_t bar_tempty = bar_tfull + 8;      // accumulators read out
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(sCtl + 24 * NS + 16);  // control block: kCtlBytes
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(sCtl + 24 * NS + 24);
+  uint8_t* sA = smem;                      // NS x [256][128] widened A
+  uint8_t* sB = sA + NS * kStageA;         // NS x [256][128] widened B
+  uint8_t* sPA = sB + NS * kStageB;        // NP x [256][64]  packed A as loaded
+  uint8_t* sPB = sPA + NP * kPackA;        // NP x [256][64]  packed B as loaded
+  uint8_t* sCtl = sPB + NP * kPackB;
+  const uint32_t bar_full = smem_u32(sCtl);         // NS: dense K step widened by the producers
+  const uint32_t bar_empty = bar_full + 8 * NS;     // NS: widened stage consumed by the MMAs
+  const uint32_t bar_sfull = bar_empty + 8 * NS;    // NS: sparse K step filled by TMA
+  const uint32_t bar_pfull = bar_sfull + 8 * NS;    // NP: packed stage landed
+  const uint32_t bar_pempty = bar_pfull + 8 * NP;   // NP: packed stage read into registers
+  const uint32_t bar_tfull = bar_pempty + 8 * NP;   // accumulators complete
+  const uint32_t bar_tempty = bar_tfull + 8;        // accumulators read out
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(sCtl + 24 * NS + 16 * NP + 16);  // control block: kCtlBytes
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(sCtl + 24 * NS + 16 * NP + 24);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int KS = p.K / BK;
-  const int Kh = p.K / 2;
   const int nwork = p.n_pairs + p.n_singles;
   const int SS = STMA ? p.SS : 0;  // sparse K steps that follow the KS dense steps of every tile
 
@@ -196,6 +205,10 @@ __global__ void __launch_bounds__(kThreads, 1)
       mbar_init(bar_full + 8 * s, kProdThreads);
       mbar_init(bar_empty + 8 * s, 1);
       mbar_init(bar_sfull + 8 * s, 1);
+    }
+    for (int s = 0; s < NP; ++s) {
+      mbar_init(bar_pfull + 8 * s, 1);
+      mbar_init(bar_pempty + 8 * s, kProdThreads);
     }
     mbar_init(bar_tfull, 1);
     mbar_init(bar_tempty, kEpiWarps * 32);
@@ -214,12 +227,14 @@ __global__ void __launch_bounds__(kThreads, 1)
   if (warp < kProdWarps) {
     // =============================================================== producers
     // Warp pw widens A rows 32*pw .. 32*pw+31 (of the 256 of a stage) and B rows 32*pw .. +31;
-    // lane -> (row % 8, packed 16-byte chunk), so one load instruction covers 8 rows x 64 B.
+    // lane -> (row % 8, packed 16-byte chunk): a quarter warp reads 128 contiguous packed bytes
+    // and its two stores land on eight different 16-byte chunks of the swizzled rows.
     const int pw = warp;
     const int r7 = lane >> 2;
     const int c = lane & 3;
     const uint32_t sw_even = (uint32_t)(((2 * c) ^ r7) << 4);
-    const uint32_t row0 = (uint32_t)(32 * pw + r7) * 128u;  // + i * 1024 for task i
+    const uint32_t row0 = (uint32_t)(32 * pw + r7) * 128u;          // widened: + i * 1024 for task i
+    const uint32_t prow0 = (uint32_t)(32 * pw + r7) * 64u + c * 16;  // packed:  + i * 512
     const int GK = (p.K / p.b) * p.k;
     const int nb = (BK / p.b) * p.k;  // sparse entries per row per K step
     const bool word_path = !STMA && p.log2k >= 0;
@@ -241,53 +256,24 @@ __global__ void __launch_bounds__(kThreads, 1)
       sp_bank4[j] = b4;
     }
 
-    // ---- load side: runs ahead of the processing side, across tile boundaries
-    int lj = blockIdx.x, lks = 0;  // work-list entry and K step of the next load
+    // ---- sparse words (dynamic positions) are prefetched in registers two steps ahead
+    int lj = blockIdx.x, lks = 0;  // work-list entry and K step of the next sparse-word load
     int l_nsub = 0;
-    uint32_t a_off[kATasks], b_off[kBTasks];  // byte offsets into dq4 / wq4 (tensors < 4 GB)
     uint32_t sp_off[MAXT];
     auto set_load_tile = [&]() {
       const Tile t = tile_of(p, lj);
       l_nsub = t.nsub;
 #pragma unroll
-      for (int i = 0; i < kATasks; ++i) {
-        const int m = min(t.m0 + 32 * pw + 8 * i + r7, p.M - 1);  // rows past M repeat the last row
-        a_off[i] = (uint32_t)m * (uint32_t)Kh + c * 16;
-      }
-#pragma unroll
-      for (int i = 0; i < kBTasks; ++i) {
-        const int n = min(t.n0 + 32 * pw + 8 * i + r7, p.N - 1);
-        b_off[i] = (uint32_t)n * (uint32_t)Kh + c * 16;
-      }
-#pragma unroll
       for (int j = 0; j < MAXT; ++j) {
         const int tt = lane + 32 * j;
-        const int m = min(t.m0 + 32 * pw + ((tt >> nw_log) & 31), p.M - 1);
+        const int m = min(t.m0 + 32 * pw + ((tt >> nw_log) & 31), p.M - 1);  // rows past M repeat the last row
         sp_off[j] = (uint32_t)m * (uint32_t)GK + 4 * (tt & ((1 << nw_log) - 1));
       }
     };
-    uint4 ra[2][kATasks], rb[2][kBTasks];  // [prefetch slot][task]
     uint32_t sv[2][MAXT], si[2][MAXT];
     auto load_next = [&](int slot) {
       if (lj >= nwork) return;
-      const uint32_t koff = (uint32_t)lks * 64u;
-#ifdef SQ_X_NOLOAD
-      if (lj >= 0) {
-        for (int i = 0; i < kATasks; ++i) ra[slot][i] = make_uint4(lks, lj, 3, 4);
-        for (int i = 0; i < kBTasks; ++i) rb[slot][i] = make_uint4(lks, lj, 5, 6);
-        if (++lks == KS) { lks = 0; lj += gridDim.x; if (lj < nwork) set_load_tile(); }
-        return;
-      }
-#endif
-      // a single-sub-tile entry only has A rows 0..127: warps 4-7 have none
-      const bool has_a = l_nsub == 2 || pw < 4;
-      if (has_a) {
-#pragma unroll
-        for (int i = 0; i < kATasks; ++i) ra[slot][i] = ldg_nc_v4(p.dq4 + a_off[i] + koff);
-      }
-#pragma unroll
-      for (int i = 0; i < kBTasks; ++i) rb[slot][i] = ldg_nc_v4(p.wq4 + b_off[i] + koff);
-      if (word_path && sp_prefetch && has_a) {
+      if (word_path && sp_prefetch && (l_nsub == 2 || pw < 4)) {
 #pragma unroll
         for (int j = 0; j < MAXT; ++j) {
           if (j < ntask) {
@@ -307,7 +293,8 @@ __global__ void __launch_bounds__(kThreads, 1)
     };
 
     // ---- processing side
-    uint32_t it = 0;
+    uint32_t it = 0;   // position in the ring of widened stages (dense and sparse steps)
+    uint32_t pit = 0;  // position in the ring of packed stages (dense steps only)
     uint32_t pmul[kATasks], poff[kATasks];
 #pragma unroll
     for (int i = 0; i < kATasks; ++i) {
@@ -317,11 +304,25 @@ __global__ void __launch_bounds__(kThreads, 1)
     int pj = blockIdx.x, pks = 0;  // work-list entry and K step being processed
     Tile pt = tile_of(p, pj);
     auto process = [&](int slot) -> bool {
+      const bool has_a = pt.nsub == 2 || pw < 4;  // a single-sub-tile entry only has A rows 0..127
+      // ---- packed operands: wait for the TMA tiles, pull this thread's chunks into registers,
+      //      hand the packed stage back
+      const int ps = pit % NP;
+      if (!mbar_wait(bar_pfull + 8 * ps, (pit / NP) & 1u, abort_flag)) return false;
+      uint4 ra[kATasks], rb[kBTasks];
+      const uint8_t* pa = sPA + ps * kPackA + prow0;
+      const uint8_t* pb = sPB + ps * kPackB + prow0;
+#pragma unroll
+      for (int i = 0; i < kATasks; ++i) ra[i] = *reinterpret_cast<const uint4*>(pa + i * 512);
+#pragma unroll
+      for (int i = 0; i < kBTasks; ++i) rb[i] = *reinterpret_cast<const uint4*>(pb + i * 512);
+      mbar_arrive(bar_pempty + 8 * ps);
+      ++pit;
+
       const int s = it % NS;
       if (!mbar_wait(bar_empty + 8 * s, ((it / NS) & 1u) ^ 1u, abort_flag)) return false;
       uint8_t* a_st = sA + s * kStageA;
       uint8_t* b_st = sB + s * kStageB;
-      const bool has_a = pt.nsub == 2 || pw < 4;
       if (pks == 0 && has_a) {  // the rows' shifts change with the tile only
 #pragma unroll
         for (int i = 0; i < kATasks; ++i) {
@@ -330,15 +331,11 @@ __global__ void __launch_bounds__(kThreads, 1)
           poff[i] = 0x01010101u * (128u - (8u << e));
         }
       }
-#ifdef SQ_X_NOWORK
-      if (ra[slot][0].x == 0x12345u) a_st[0] = (uint8_t)rb[slot][0].x;  // keep the loads alive
-      if (false)
-#endif
       // ---- widen A: nibble -> u * 2^e + (128 - 8 * 2^e)
       if (has_a) {
 #pragma unroll
         for (int i = 0; i < kATasks; ++i) {
-          const uint32_t in[4] = {ra[slot][i].x, ra[slot][i].y, ra[slot][i].z, ra[slot][i].w};
+          const uint32_t in[4] = {ra[i].x, ra[i].y, ra[i].z, ra[i].w};
           uint32_t ev[4], od[4];
 #pragma unroll
           for (int q = 0; q < 4; ++q) {
@@ -352,12 +349,9 @@ __global__ void __launch_bounds__(kThreads, 1)
         }
       }
       // ---- widen B: nibble -> 16 * code
-#ifdef SQ_X_NOWORK
-      if (false)
-#endif
 #pragma unroll
       for (int i = 0; i < kBTasks; ++i) {
-        const uint32_t in[4] = {rb[slot][i].x, rb[slot][i].y, rb[slot][i].z, rb[slot][i].w};
+        const uint32_t in[4] = {rb[i].x, rb[i].y, rb[i].z, rb[i].w};
         uint32_t ev[4], od[4];
 #pragma unroll
         for (int q = 0; q < 4; ++q) {
@@ -488,7 +482,26 @@ __global__ void __launch_bounds__(kThreads, 1)
     }
     __syncwarp();
   } else if (warp == kTmaWarp) {
-    // =============================================================== TMA (sparse K steps)
+    // =============================================================== TMA: packed dense tiles
+    if (lane == 0) {
+      uint32_t pit = 0;
+      bool ok = true;
+      for (int j = blockIdx.x; j < nwork && ok; j += gridDim.x) {
+        const Tile t = tile_of(p, j);
+        for (int ks = 0; ks < KS && ok; ++ks, ++pit) {
+          const int ps = pit % NP;
+          ok = mbar_wait(bar_pempty + 8 * ps, ((pit / NP) & 1u) ^ 1u, abort_flag);
+          if (!ok) break;
+          // rows past M / N come back as zeros (code 0)
+          mbar_expect_tx(bar_pfull + 8 * ps, (uint32_t)(kPackA + kPackB));
+          tma_load_2d(smem_u32(sPA + ps * kPackA), &map_a4, ks * (BK / 2), t.m0, bar_pfull + 8 * ps);
+          tma_load_2d(smem_u32(sPB + ps * kPackB), &map_b4, ks * (BK / 2), t.n0, bar_pfull + 8 * ps);
+        }
+      }
+    }
+    __syncwarp();
+  } else if (warp == kTmaSparseWarp) {
+    // =============================================================== TMA: sparse K steps
     if (STMA && lane == 0) {
       uint32_t it = 0;
       bool ok = true;
@@ -643,22 +656,37 @@ cudaError_t launch_gemm(int b, int k, const sq_encoded& A, const sq_weights& W,
   // Static positions: the sparse product runs as extra K steps over vals [M, G*k] and
   // w_sparse [N, G*k], fetched by TMA.  A TMA row pitch must be a multiple of 16 bytes; any
   // other G*k falls back to merging the entries into the dense tile like dynamic positions.
-  CUtensorMap map_a, map_b;
+  CUtensorMap map_a, map_b, map_a4, map_b4;
   memset(&map_a, 0, sizeof(map_a));
   memset(&map_b, 0, sizeof(map_b));
+  static PFN_cuTensorMapEncodeTiled encode = nullptr;
+  if (encode == nullptr) {
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    err = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
+    if (err != cudaSuccess) return err;
+    if (fn == nullptr || qres != cudaDriverEntryPointSuccess) return cudaErrorNotSupported;
+    encode = reinterpret_cast<PFN_cuTensorMapEncodeTiled>(fn);
+  }
+  const cuuint32_t estr[2] = {1, 1};
+  {
+    // packed operands: [rows, K/2] bytes, boxes of 256 rows x 64 bytes, stored unswizzled
+    const cuuint64_t pitch4[1] = {(cuuint64_t)(K / 2)};
+    const cuuint64_t dim_a4[2] = {(cuuint64_t)(K / 2), (cuuint64_t)M};
+    const cuuint64_t dim_b4[2] = {(cuuint64_t)(K / 2), (cuuint64_t)N};
+    const cuuint32_t box4[2] = {BK / 2, 2 * BM};
+    if (encode(&map_a4, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, A.dq4, dim_a4, pitch4, box4, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+      return cudaErrorInvalidValue;
+    if (encode(&map_b4, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, W.wq4, dim_b4, pitch4, box4, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+      return cudaErrorInvalidValue;
+  }
   p.SS = 0;
   const bool stma = positions != nullptr && GK % 16 == 0;
   if (stma) {
-    static PFN_cuTensorMapEncodeTiled encode = nullptr;
-    if (encode == nullptr) {
-      void* fn = nullptr;
-      cudaDriverEntryPointQueryResult qres;
-      err = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
-      if (err != cudaSuccess) return err;
-      if (fn == nullptr || qres != cudaDriverEntryPointSuccess) return cudaErrorNotSupported;
-      encode = reinterpret_cast<PFN_cuTensorMapEncodeTiled>(fn);
-    }
-    const cuuint32_t estr[2] = {1, 1};
     const cuuint64_t pitch[1] = {(cuuint64_t)GK};
     const cuuint64_t dim_a[2] = {(cuuint64_t)GK, (cuuint64_t)M};
     const cuuint64_t dim_b[2] = {(cuuint64_t)GK, (cuuint64_t)N};
@@ -680,7 +708,7 @@ cudaError_t launch_gemm(int b, int k, const sq_encoded& A, const sq_weights& W,
     err = cudaFuncSetAttribute(gemm_kernel<MAXT_, STMA_>, cudaFuncAttributeMaxDynamicSharedMemorySize,      \
                                kSmemBytes);                                                                 \
     if (err != cudaSuccess) return err;                                                                     \
-    gemm_kernel<MAXT_, STMA_><<<grid, kThreads, kSmemBytes, st>>>(p, map_a, map_b);                         \
+    gemm_kernel<MAXT_, STMA_><<<grid, kThreads, kSmemBytes, st>>>(p, map_a, map_b, map_a4, map_b4);         \
   } while (0)
   if (stma) SQ_LAUNCH_GEMM(1, true);
   else SQ_LAUNCH_GEMM(4, false);
