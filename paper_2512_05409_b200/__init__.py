@@ -11,3 +11,4 @@ from .binding import (  # noqa: F401
     sq_weights_sizes, sq_calib_positions, sq_pack_weights, sq_encode, sq_gemm, sq_decode,
     sq_device_status, raw,
 )
+from .sharding import row_shard  # noqa: F401,E402
