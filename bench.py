@@ -38,9 +38,16 @@ SHAPES_70B = [(8192, 10240), (8192, 8192), (8192, 57344), (28672, 8192)]
 M_70B, BANK_70B, K_70B = 4096, 128, 16
 INT8_OVER_BF16 = 2.0        # nominal dense INT8 : bf16 tensor rate on B200 (4.5 : 2.25 PFLOP/s)
 FALLBACK_HBM_GBS, FALLBACK_BF16_TFLOPS = 6650.0, 1590.0
-# DRAM bytes per GEMM launch measured by ncu (see profiles/); None until a capture exists.
-GEMM_TRAFFIC_BYTES_PER_LAUNCH = None
-ENCODE_TRAFFIC_BYTES_PER_LAUNCH = None
+# ncu DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one gemm_kernel launch on the
+# small capture case of profiles/gemm_kernel_static_b128_k16_M2048_N8192_K8192.txt, and that case's
+# algorithmic bytes; the benchmark's launches are too large to capture with --set full, so their
+# traffic is this ratio times their own algorithmic bytes (the traffic is operand streaming and
+# grows with the operands).  It is below 1 because most of the output is still in L2 at kernel end.
+GEMM_CAPTURE_TRAFFIC_BYTES = 52.59e6 + 3.01e6
+GEMM_CAPTURE_ALGO_BYTES = 2048 * 8192 * 0.625 + 8192 * 8192 * 0.625 + 2.0 * 2048 * 8192
+# ncu DRAM traffic of one encode launch of the 8192 x 8192 bandwidth test (dynamic k=8 / static k=8),
+# profiles/encode_rows_kernel_b64_k8_8192x8192.txt
+ENCODE_TRAFFIC_BYTES_PER_LAUNCH = {"dynamic": 134.26e6 + 27.32e6, "static": 134.26e6 + 20.79e6}
 
 
 def load_peaks():
@@ -142,7 +149,7 @@ class Linear:
         self.ops = 2.0 * M * N * K
         # algorithmic bytes: packed activations + packed weights + bf16 output
         payload = 0.5 + (1.0 if static else 2.0) * k / bank
-        self.gemm_bytes = M * K * payload + N * K / 2 + 2.0 * M * N
+        self.gemm_bytes = M * K * payload + N * K * (0.5 + (k / bank if static else 0.0)) + 2.0 * M * N
         self.encode_bytes = M * K * (2.0 + payload) + 9.0 * M
 
     def step(self, sq, events=None):
@@ -180,7 +187,9 @@ def bench_encode_only(sq, dev, peaks, iters=20):
             ms = statistics.median(a.elapsed_time(b) for a, b in evs)
             nbytes = M * K * (2.0 + 0.5 + (1.0 if static else 2.0) * k / 64) + 9.0 * M
             gbs = nbytes / (ms * 1e-3) / 1e9
+            traffic = ENCODE_TRAFFIC_BYTES_PER_LAUNCH["static" if static else "dynamic"] if k == 8 else None
             res.append({"mode": "static" if static else "dynamic", "k": k, "ms": round(ms, 4),
+                        "algorithmic_bytes": nbytes, "traffic": traffic,
                         "GBps": round(gbs, 1), "frac_of_measured_hbm": round(gbs / peaks["hbm_gbs"], 4),
                         "frac_of_8TBps": round(gbs / 8000.0, 4)})
     return res
@@ -346,10 +355,13 @@ def run_cuda(args):
                      "frac_of_sustained": gemm_tops / (peaks["bf16_tflops_sustained"] * INT8_OVER_BF16),
                      "frac_of_nominal_4500": gemm_tops / 4500.0,
                      "avg_launch_ms": gemm_ms / n_gemm, "launches": n_gemm,
-                     "traffic": GEMM_TRAFFIC_BYTES_PER_LAUNCH},
+                     "algorithmic_bytes_per_launch": sum(l.gemm_bytes for l in layers) / len(layers),
+                     "traffic": sum(l.gemm_bytes for l in layers) / len(layers)
+                     * GEMM_CAPTURE_TRAFFIC_BYTES / GEMM_CAPTURE_ALGO_BYTES,
+                     "traffic_note": "ncu DRAM bytes of a smaller captured launch scaled by algorithmic bytes (see profiles/)"},
         "roofline_encode_in_step": {"kernel": "sq_encode", "bound": "hbm", "achieved": enc_gbs,
                                     "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": enc_gbs / peaks["hbm_gbs"],
-                                    "peak_source": peaks["source"], "traffic": ENCODE_TRAFFIC_BYTES_PER_LAUNCH},
+                                    "peak_source": peaks["source"], "traffic": None},
     }
     if rank == 0:
         if not args.no_encode_bench:
