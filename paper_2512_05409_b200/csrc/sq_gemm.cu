@@ -62,7 +62,7 @@ constexpr int BM = 128;   // rows of one sub-tile = TMEM lanes
 constexpr int BN = 256;   // output channels per tile = TMEM columns of one accumulator
 constexpr int BK = 128;   // K elements per pipeline step = bytes per operand row
 constexpr int NS = 2;     // stages of widened (8-bit) operands
-constexpr int NP = 2;     // stages of packed (4-bit) operands as TMA delivers them
+constexpr int NP = 3;     // stages of packed (4-bit) operands as TMA delivers them
 constexpr int kProdWarps = 8;
 constexpr int kProdThreads = kProdWarps * 32;
 constexpr int kMmaWarp = kProdWarps;
@@ -76,8 +76,7 @@ constexpr int kCtlBytes = 256;            // barriers, tensor-memory slot, abort
 constexpr int kEpiConstBytes = 2 * BN * 4;  // per tile: 2048 * colsum[n] and s_w[n] of its columns
 constexpr int kPackA = 2 * BM * (BK / 2);  // 16 KB: 256 rows x 64 packed bytes
 constexpr int kPackB = BN * (BK / 2);      // 16 KB
-constexpr int kSmemBytes =
-    NS * (kStageA + kStageB) + NP * (kPackA + kPackB) + 1024 /*alignment slack*/ + kCtlBytes + kEpiConstBytes;
+constexpr int kSmemBytes = NS * (kStageA + kStageB) + NP * (kPackA + kPackB) + kCtlBytes + kEpiConstBytes;
 constexpr int kATasks = 4;  // 16-byte packed chunks of A per producer thread per step
 constexpr int kBTasks = 4;
 
@@ -177,9 +176,14 @@ template <int MAXT, bool STMA>
 __global__ void __launch_bounds__(kThreads, 1)
     gemm_kernel(const GemmParams p, const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                 const __grid_constant__ CUtensorMap map_a4, const __grid_constant__ CUtensorMap map_b4) {
-  extern __shared__ uint8_t smem_raw[];
-  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-  uint8_t* smem = smem_raw + (base - smem_u32(smem_raw));
+  // The kernel has no static shared memory, so the dynamic block starts at the 1024-byte
+  // aligned base the swizzled operand layout needs; checked below, never assumed.
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
+  uint8_t* smem = smem_raw;
+  if ((smem_u32(smem_raw) & 1023u) != 0) {
+    if (threadIdx.x == 0) atomicExch(p.status, (int)SQ_ERR_CUDA);
+    return;
+  }
   uint8_t* sA = smem;                      // NS x [256][128] widened A
   uint8_t* sB = sA + NS * kStageA;         // NS x [256][128] widened B
   uint8_t* sPA = sB + NS * kStageB;        // NP x [256][64]  packed A as loaded
@@ -316,7 +320,6 @@ __global__ void __launch_bounds__(kThreads, 1)
       for (int i = 0; i < kATasks; ++i) ra[i] = *reinterpret_cast<const uint4*>(pa + i * 512);
 #pragma unroll
       for (int i = 0; i < kBTasks; ++i) rb[i] = *reinterpret_cast<const uint4*>(pb + i * 512);
-      mbar_arrive(bar_pempty + 8 * ps);
       ++pit;
 
       const int s = it % NS;
@@ -362,6 +365,10 @@ __global__ void __launch_bounds__(kThreads, 1)
         *reinterpret_cast<uint4*>(dst + sw_even) = make_uint4(ev[0], ev[1], ev[2], ev[3]);
         *reinterpret_cast<uint4*>(dst + (sw_even ^ 16u)) = make_uint4(od[0], od[1], od[2], od[3]);
       }
+      // The packed stage goes back to the TMA thread only now: shared-memory loads are
+      // asynchronous, and an arrive issued right behind them could let the refill overtake
+      // them; after the widening every loaded register has been consumed.
+      mbar_arrive(bar_pempty + 8 * ps);
       // ---- sparse INT8 entries overwrite their places (rows 32*pw .. 32*pw+31 of the stage)
       if (!STMA && has_a) {
         __syncwarp();  // this warp's A rows are complete before any lane overwrites bytes in them

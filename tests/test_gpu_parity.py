@@ -205,3 +205,32 @@ def test_worst_case_accumulator_magnitude():
     assert np.array_equal(_np(acc), acc_ref)
     # (K/b)*k entries at 127 and the rest at 7 << 4 = 112, times 7
     assert abs(int(acc_ref[0, 0])) == ((K // b) * k * 127 + (K - (K // b) * k) * 112) * 7
+
+
+@pytest.mark.parametrize("M,N,K,b,k,static", [
+    (128, 256 * 300, 1024, 64, 8, False),     # 300 single tiles: two or three per SM, 8 K steps each
+    (512, 256 * 160, 512, 128, 16, True),     # 296 pair tiles + 48 single tiles, TMA-fed sparse K steps
+    (640, 256 * 150, 768, 64, 8, False),      # pairs, split pairs and the odd last row unit together
+])
+def test_several_tiles_per_sm(M, N, K, b, k, static):
+    """Persistent-kernel steady state: every SM walks through several tiles, so the pipelines
+    wrap around tile boundaries.  Sampled token rows are checked over EVERY output channel."""
+    fmt = sq.make_format(b, k, static)
+    X = gen.activations(M, K, seed=11, device="cuda")
+    W = gen.weights(N, K, seed=11, device="cuda")
+    pos = pos_ref = None
+    if static:
+        pos = sq.sq_calib_positions(fmt, gen.calibration_batch(64, K, seed=11, device="cuda"))
+        pos_ref = _np(pos)
+    w = sq.sq_pack_weights(fmt, W, pos)
+    enc = sq.sq_encode(fmt, X, pos)
+    rows = np.unique(np.clip(np.concatenate([[0, 127, 128, M - 1], np.arange(5, M, max(M // 12, 1))]), 0, M - 1))
+    enc_ref = oracle.encode(b, k, _bits(X)[rows], pos_ref)
+    w_ref = oracle.pack_weights(b, k, _bits(W), pos_ref)
+    acc_ref, ref32, _ = oracle.gemm(b, k, enc_ref, w_ref, pos_ref)
+    for _ in range(3):                          # a race would not show on every launch
+        acc = torch.empty(M, N, dtype=torch.int32, device="cuda")
+        out = sq.sq_gemm(fmt, enc, w, pos, acc_out=acc)
+        check_status()
+        assert np.array_equal(_np(acc)[rows], acc_ref)
+        assert_bf16_close(out[torch.from_numpy(rows).cuda()], ref32)
