@@ -63,10 +63,22 @@ constexpr int BN = 256;   // output channels per tile = TMEM columns of one accu
 constexpr int BK = 128;   // K elements per pipeline step = bytes per operand row
 constexpr int NS = 2;     // stages of widened (8-bit) operands
 constexpr int NP = 3;     // stages of packed (4-bit) operands as TMA delivers them
-constexpr int kProdWarps = 8;
+#ifndef SQ_X_PRODWARPS
+#define SQ_X_PRODWARPS 8
+#endif
+constexpr int kProdWarps = SQ_X_PRODWARPS;
 constexpr int kProdThreads = kProdWarps * 32;
 constexpr int kMmaWarp = kProdWarps;
 constexpr int kEpiWarps = 4;
+// Letting the (by then idle) producer warps read out two thirds of a tile's accumulators was
+// measured slower than leaving the epilogue to its own four warps (the producers then refill
+// the pipeline later), so it is compiled out; the hand-shake below supports both.
+#ifndef SQ_X_JOIN
+#define SQ_X_JOIN 0
+#endif
+constexpr bool kProducersJoinEpilogue = SQ_X_JOIN != 0;
+constexpr int kEpiHelpers = kEpiWarps + (kProducersJoinEpilogue ? kProdWarps : 0);
+constexpr int kEpiStride = kProducersJoinEpilogue ? 3 : 1;  // warps per TMEM lane quarter
 constexpr int kTmaWarp = kProdWarps + 1 + kEpiWarps;  // packed dense tiles
 constexpr int kTmaSparseWarp = kTmaWarp + 1;          // INT8 tiles of the sparse K steps
 constexpr int kThreads = (kProdWarps + 1 + kEpiWarps + 2) * 32;
@@ -77,8 +89,10 @@ constexpr int kEpiConstBytes = 2 * BN * 4;  // per tile: 2048 * colsum[n] and s_
 constexpr int kPackA = 2 * BM * (BK / 2);  // 16 KB: 256 rows x 64 packed bytes
 constexpr int kPackB = BN * (BK / 2);      // 16 KB
 constexpr int kSmemBytes = NS * (kStageA + kStageB) + NP * (kPackA + kPackB) + kCtlBytes + kEpiConstBytes;
-constexpr int kATasks = 4;  // 16-byte packed chunks of A per producer thread per step
-constexpr int kBTasks = 4;
+constexpr int kRowsPerWarp = 2 * BM / kProdWarps;  // rows of A (and of B) a producer warp widens per stage
+constexpr int kATasks = kRowsPerWarp / 8;  // 16-byte packed chunks of A per producer thread per step
+constexpr int kBTasks = kRowsPerWarp / 8;
+constexpr int kMergeTasks = 8;  // sparse 4-entry words per merge thread per stage kept in registers
 
 struct GemmParams {
   const uint8_t* dq4;
@@ -196,8 +210,11 @@ __global__ void __launch_bounds__(kThreads, 1)
   const uint32_t bar_pempty = bar_pfull + 8 * NP;   // NP: packed stage read into registers
   const uint32_t bar_tfull = bar_pempty + 8 * NP;   // accumulators complete
   const uint32_t bar_tempty = bar_tfull + 8;        // accumulators read out
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(sCtl + 24 * NS + 16 * NP + 16);  // control block: kCtlBytes
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(sCtl + 24 * NS + 16 * NP + 24);
+  const uint32_t bar_wfull = bar_tempty + 8;        // NS: dense K step widened, sparse entries not merged yet
+  const uint32_t bar_eready = bar_wfull + 8 * NS;   // epilogue: column constants staged, every helper present
+  const uint32_t bar_edone = bar_eready + 8;        // epilogue: every helper done with the constants
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(sCtl + 32 * NS + 16 * NP + 32);  // control block: kCtlBytes
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(sCtl + 32 * NS + 16 * NP + 40);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int KS = p.K / BK;
@@ -206,7 +223,9 @@ __global__ void __launch_bounds__(kThreads, 1)
 
   if (tid == 0) {
     for (int s = 0; s < NS; ++s) {
-      mbar_init(bar_full + 8 * s, kProdThreads);
+      // static positions: the producers complete a dense stage; otherwise the merge warps do
+      mbar_init(bar_full + 8 * s, STMA ? kProdThreads : kEpiWarps * 32);
+      mbar_init(bar_wfull + 8 * s, kProdThreads);
       mbar_init(bar_empty + 8 * s, 1);
       mbar_init(bar_sfull + 8 * s, 1);
     }
@@ -215,7 +234,9 @@ __global__ void __launch_bounds__(kThreads, 1)
       mbar_init(bar_pempty + 8 * s, kProdThreads);
     }
     mbar_init(bar_tfull, 1);
-    mbar_init(bar_tempty, kEpiWarps * 32);
+    mbar_init(bar_tempty, kEpiHelpers * 32);
+    mbar_init(bar_eready, kEpiHelpers * 32);
+    mbar_init(bar_edone, kEpiHelpers * 32);
     *abort_flag = 0;
     fence_mbar_init();
   }
@@ -228,74 +249,72 @@ __global__ void __launch_bounds__(kThreads, 1)
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
 
+  // ---- epilogue of one tile, shared by the epilogue warps and the producers (which have run
+  //      out of free stages by the time a tile completes): warp w reads TMEM lane quarter
+  //      w % 4; the three warps of a quarter split the tile's 32-column chunks.
+  int32_t* s_cs = reinterpret_cast<int32_t*>(sCtl + kCtlBytes);  // 2048 * colsum of the tile's columns
+  float* s_sw = reinterpret_cast<float*>(sCtl + kCtlBytes + BN * 4);
+  auto epilogue_share = [&](const Tile& t, uint32_t tile_count, int helper) -> bool {
+    if (!mbar_wait_idle(bar_tfull, tile_count & 1u, abort_flag)) return false;
+    tc_fence_after();
+    mbar_arrive(bar_eready);
+    if (!mbar_wait(bar_eready, tile_count & 1u, abort_flag)) return false;
+    const int q = warp & 3;
+    for (int ci = helper; ci < t.nsub * (BN / 32); ci += kEpiStride) {
+      const int sub = ci / (BN / 32), c0 = (ci % (BN / 32)) * 32;
+      const int m = t.m0 + sub * BM + 32 * q + lane;
+      const float sh = (m < p.M) ? p.s_hi[m] : 0.f;
+      uint32_t v[32];
+      tmem_ld32(tmem + ((uint32_t)(32 * q) << 16) + (uint32_t)(sub * BN + c0), v);
+      tmem_ld_wait();
+      const int n0 = t.n0 + c0;
+      if (m < p.M && n0 < p.N) {
+#pragma unroll
+        for (int c8 = 0; c8 < 32; c8 += 8) {
+          if (n0 + c8 < p.N) {  // N % 8 == 0: a group of 8 columns is all in or all out
+            int acc[8];
+            uint32_t o[4];
+            const int4 cs0 = *reinterpret_cast<const int4*>(s_cs + c0 + c8);
+            const int4 cs1 = *reinterpret_cast<const int4*>(s_cs + c0 + c8 + 4);
+            const float4 sw0 = *reinterpret_cast<const float4*>(s_sw + c0 + c8);
+            const float4 sw1 = *reinterpret_cast<const float4*>(s_sw + c0 + c8 + 4);
+            const int cs[8] = {cs0.x, cs0.y, cs0.z, cs0.w, cs1.x, cs1.y, cs1.z, cs1.w};
+            const float sw[8] = {sw0.x, sw0.y, sw0.z, sw0.w, sw1.x, sw1.y, sw1.z, sw1.w};
+#pragma unroll
+            for (int cc = 0; cc < 8; ++cc) acc[cc] = ((int)v[c8 + cc] - cs[cc]) >> 4;
+#pragma unroll
+            for (int cc = 0; cc < 8; cc += 2) {
+              const float f0 = ((float)acc[cc] * sh) * sw[cc];
+              const float f1 = ((float)acc[cc + 1] * sh) * sw[cc + 1];
+              o[cc >> 1] = f32_to_bf16_bits(f0) | (f32_to_bf16_bits(f1) << 16);
+            }
+            *reinterpret_cast<uint4*>(p.out + (size_t)m * p.N + n0 + c8) = make_uint4(o[0], o[1], o[2], o[3]);
+            if (p.acc_out != nullptr) {
+              int4* dst = reinterpret_cast<int4*>(p.acc_out + (size_t)m * p.N + n0 + c8);
+              dst[0] = make_int4(acc[0], acc[1], acc[2], acc[3]);
+              dst[1] = make_int4(acc[4], acc[5], acc[6], acc[7]);
+            }
+          }
+        }
+      }
+    }
+    tc_fence_before();
+    mbar_arrive(bar_tempty);
+    mbar_arrive(bar_edone);
+    return true;
+  };
+
   if (warp < kProdWarps) {
     // =============================================================== producers
-    // Warp pw widens A rows 32*pw .. 32*pw+31 (of the 256 of a stage) and B rows 32*pw .. +31;
+    // Warp pw widens kRowsPerWarp rows of A (of the 256 of a stage) and as many rows of B;
     // lane -> (row % 8, packed 16-byte chunk): a quarter warp reads 128 contiguous packed bytes
     // and its two stores land on eight different 16-byte chunks of the swizzled rows.
     const int pw = warp;
     const int r7 = lane >> 2;
     const int c = lane & 3;
     const uint32_t sw_even = (uint32_t)(((2 * c) ^ r7) << 4);
-    const uint32_t row0 = (uint32_t)(32 * pw + r7) * 128u;          // widened: + i * 1024 for task i
-    const uint32_t prow0 = (uint32_t)(32 * pw + r7) * 64u + c * 16;  // packed:  + i * 512
-    const int GK = (p.K / p.b) * p.k;
-    const int nb = (BK / p.b) * p.k;  // sparse entries per row per K step
-    const bool word_path = !STMA && p.log2k >= 0;
-    const int nw_log = word_path ? (31 - __clz(nb >> 2)) : 0;  // log2(words per row per step)
-    const int ntask = word_path ? ((32 << nw_log) + 31) >> 5 : 0;  // word tasks per lane (32 rows per warp)
-    const bool sp_prefetch = ntask <= MAXT;
-
-    // tile-independent part of this lane's sparse word tasks: task t = lane + 32*j covers
-    // word (t mod words-per-row) of row (t div words-per-row) of the warp's 32 rows
-    uint32_t sp_bank4[MAXT];
-#pragma unroll
-    for (int j = 0; j < MAXT; ++j) {
-      const int q = (lane + 32 * j) & ((1 << nw_log) - 1);
-      uint32_t b4 = 0;
-      if (word_path) {
-#pragma unroll
-        for (int u = 0; u < 4; ++u) b4 |= (uint32_t)(((4 * q + u) >> p.log2k) * p.b) << (8 * u);
-      }
-      sp_bank4[j] = b4;
-    }
-
-    // ---- sparse words (dynamic positions) are prefetched in registers two steps ahead
-    int lj = blockIdx.x, lks = 0;  // work-list entry and K step of the next sparse-word load
-    int l_nsub = 0;
-    uint32_t sp_off[MAXT];
-    auto set_load_tile = [&]() {
-      const Tile t = tile_of(p, lj);
-      l_nsub = t.nsub;
-#pragma unroll
-      for (int j = 0; j < MAXT; ++j) {
-        const int tt = lane + 32 * j;
-        const int m = min(t.m0 + 32 * pw + ((tt >> nw_log) & 31), p.M - 1);  // rows past M repeat the last row
-        sp_off[j] = (uint32_t)m * (uint32_t)GK + 4 * (tt & ((1 << nw_log) - 1));
-      }
-    };
-    uint32_t sv[2][MAXT], si[2][MAXT];
-    auto load_next = [&](int slot) {
-      if (lj >= nwork) return;
-      if (word_path && sp_prefetch && (l_nsub == 2 || pw < 4)) {
-#pragma unroll
-        for (int j = 0; j < MAXT; ++j) {
-          if (j < ntask) {
-            const uint32_t o = sp_off[j] + (uint32_t)lks * (uint32_t)nb;
-            sv[slot][j] = __ldg(reinterpret_cast<const uint32_t*>(p.vals + o));
-            const int q4 = 4 * ((lane + 32 * j) & ((1 << nw_log) - 1));
-            si[slot][j] = p.idx != nullptr ? __ldg(reinterpret_cast<const uint32_t*>(p.idx + o))
-                                           : __ldg(reinterpret_cast<const uint32_t*>(p.pos + lks * nb + q4));
-          }
-        }
-      }
-      if (++lks == KS) {
-        lks = 0;
-        lj += gridDim.x;
-        if (lj < nwork) set_load_tile();
-      }
-    };
-
+    const uint32_t row0 = (uint32_t)(kRowsPerWarp * pw + r7) * 128u;          // widened: + i * 1024 for task i
+    const uint32_t prow0 = (uint32_t)(kRowsPerWarp * pw + r7) * 64u + c * 16;  // packed:  + i * 512
     // ---- processing side
     uint32_t it = 0;   // position in the ring of widened stages (dense and sparse steps)
     uint32_t pit = 0;  // position in the ring of packed stages (dense steps only)
@@ -307,8 +326,8 @@ __global__ void __launch_bounds__(kThreads, 1)
     }
     int pj = blockIdx.x, pks = 0;  // work-list entry and K step being processed
     Tile pt = tile_of(p, pj);
-    auto process = [&](int slot) -> bool {
-      const bool has_a = pt.nsub == 2 || pw < 4;  // a single-sub-tile entry only has A rows 0..127
+    auto process = [&]() -> bool {
+      const bool has_a = pt.nsub == 2 || pw < kProdWarps / 2;  // a single-sub-tile entry only has A rows 0..127
       // ---- packed operands: wait for the TMA tiles, pull this thread's chunks into registers,
       //      hand the packed stage back
       const int ps = pit % NP;
@@ -329,11 +348,15 @@ __global__ void __launch_bounds__(kThreads, 1)
       if (pks == 0 && has_a) {  // the rows' shifts change with the tile only
 #pragma unroll
         for (int i = 0; i < kATasks; ++i) {
-          const uint32_t e = p.shift[min(pt.m0 + 32 * pw + 8 * i + r7, p.M - 1)];
+          const uint32_t e = p.shift[min(pt.m0 + kRowsPerWarp * pw + 8 * i + r7, p.M - 1)];
           pmul[i] = 1u << e;
           poff[i] = 0x01010101u * (128u - (8u << e));
         }
       }
+#ifdef SQ_X_NOWORK
+      if (ra[0].x == 0x12345u) a_st[0] = (uint8_t)rb[0].x;
+      if (false)
+#endif
       // ---- widen A: nibble -> u * 2^e + (128 - 8 * 2^e)
       if (has_a) {
 #pragma unroll
@@ -347,11 +370,19 @@ __global__ void __launch_bounds__(kThreads, 1)
             od[q] = ((u >> 4) & 0x0F0F0F0Fu) * pmul[i] + poff[i];
           }
           uint8_t* dst = a_st + row0 + i * 1024;
+#ifdef SQ_X_NOSTS
+          if ((ev[0] ^ od[1] ^ ev[2] ^ od[3] ^ ev[1] ^ od[0] ^ ev[3] ^ od[2]) == 0x13579bdfu)
+#endif
+          {
           *reinterpret_cast<uint4*>(dst + sw_even) = make_uint4(ev[0], ev[1], ev[2], ev[3]);
           *reinterpret_cast<uint4*>(dst + (sw_even ^ 16u)) = make_uint4(od[0], od[1], od[2], od[3]);
+          }
         }
       }
       // ---- widen B: nibble -> 16 * code
+#ifdef SQ_X_NOWORK
+      if (false)
+#endif
 #pragma unroll
       for (int i = 0; i < kBTasks; ++i) {
         const uint32_t in[4] = {rb[i].x, rb[i].y, rb[i].z, rb[i].w};
@@ -362,65 +393,22 @@ __global__ void __launch_bounds__(kThreads, 1)
           od[q] = in[q] & 0xF0F0F0F0u;
         }
         uint8_t* dst = b_st + row0 + i * 1024;
+#ifdef SQ_X_NOSTS
+        if ((ev[0] ^ od[1] ^ ev[2] ^ od[3] ^ ev[1] ^ od[0] ^ ev[3] ^ od[2]) == 0x13579bdfu)
+#endif
+        {
         *reinterpret_cast<uint4*>(dst + sw_even) = make_uint4(ev[0], ev[1], ev[2], ev[3]);
         *reinterpret_cast<uint4*>(dst + (sw_even ^ 16u)) = make_uint4(od[0], od[1], od[2], od[3]);
+        }
       }
       // The packed stage goes back to the TMA thread only now: shared-memory loads are
       // asynchronous, and an arrive issued right behind them could let the refill overtake
       // them; after the widening every loaded register has been consumed.
       mbar_arrive(bar_pempty + 8 * ps);
-      // ---- sparse INT8 entries overwrite their places (rows 32*pw .. 32*pw+31 of the stage)
-      if (!STMA && has_a) {
-        __syncwarp();  // this warp's A rows are complete before any lane overwrites bytes in them
-        if (word_path) {
-#pragma unroll
-          for (int j = 0; j < MAXT; ++j) {
-            if (j < ntask && sp_prefetch) {
-              const int tt = lane + 32 * j;
-              const int row = 32 * pw + (tt >> nw_log);
-              const uint32_t r7s = 0x01010101u * (uint32_t)((row & 7) << 4);
-              const uint32_t pos4 = (kpos4(si[slot][j]) + sp_bank4[j]) ^ r7s;
-              const uint32_t vx = sv[slot][j] ^ 0x80808080u;
-              uint8_t* rowp = a_st + row * 128;
-#pragma unroll
-              for (int u = 0; u < 4; ++u) rowp[(pos4 >> (8 * u)) & 0xFFu] = (uint8_t)(vx >> (8 * u));
-            }
-          }
-          if (!sp_prefetch) {  // many entries per step: word loads without register prefetch
-            for (int tt = lane; tt < (32 << nw_log); tt += 32) {
-              const int row_l = tt >> nw_log, q = tt & ((1 << nw_log) - 1);
-              const int row = 32 * pw + row_l;
-              const int m = min(pt.m0 + row, p.M - 1);
-              const uint32_t o = (uint32_t)m * (uint32_t)GK + (uint32_t)pks * (uint32_t)nb + 4 * q;
-              const uint32_t vw = __ldg(reinterpret_cast<const uint32_t*>(p.vals + o));
-              const uint32_t iw = p.idx != nullptr ? __ldg(reinterpret_cast<const uint32_t*>(p.idx + o))
-                                                   : __ldg(reinterpret_cast<const uint32_t*>(p.pos + pks * nb + 4 * q));
-              uint32_t b4 = 0;
-#pragma unroll
-              for (int u = 0; u < 4; ++u) b4 |= (uint32_t)(((4 * q + u) >> p.log2k) * p.b) << (8 * u);
-              const uint32_t pos4 = (kpos4(iw) + b4) ^ (0x01010101u * (uint32_t)((row & 7) << 4));
-              const uint32_t vx = vw ^ 0x80808080u;
-              uint8_t* rowp = a_st + row * 128;
-#pragma unroll
-              for (int u = 0; u < 4; ++u) rowp[(pos4 >> (8 * u)) & 0xFFu] = (uint8_t)(vx >> (8 * u));
-            }
-          }
-        } else {
-          for (int tt = lane; tt < 32 * nb; tt += 32) {
-            const int row_l = tt / nb, i = tt - row_l * nb;
-            const int row = 32 * pw + row_l;
-            const int m = min(pt.m0 + row, p.M - 1);
-            const int bank = i / p.k, slot_i = i - bank * p.k;
-            const int g = pks * (BK / p.b) + bank;
-            const size_t entry = (size_t)m * GK + (size_t)g * p.k + slot_i;
-            const uint32_t local = p.idx != nullptr ? p.idx[entry] : p.pos[(size_t)g * p.k + slot_i];
-            const uint32_t kp = (kpos1(local) + (uint32_t)(bank * p.b)) ^ (uint32_t)((row & 7) << 4);
-            a_st[row * 128 + kp] = (uint8_t)((uint8_t)p.vals[entry] ^ 0x80u);
-          }
-        }
-      }
+#ifndef SQ_X_NOFENCE
       fence_proxy_async_smem();  // generic-proxy writes -> visible to the tensor core's async reads
-      mbar_arrive(bar_full + 8 * s);
+#endif
+      mbar_arrive((STMA ? bar_full : bar_wfull) + 8 * s);  // dynamic positions: the merge warps take over
       ++it;
       if (++pks == KS) {
         pks = 0;
@@ -436,19 +424,21 @@ __global__ void __launch_bounds__(kThreads, 1)
       return true;
     };
 
+    // (Optional, see kProducersJoinEpilogue.)  After filling the first stages of a tile the ring
+    // is full until the MMA thread moves on, and it moves on only when the previous tile's
+    // accumulators have been read out: that is when the producers can lend a hand.
     const int my_tiles = (nwork - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
-    const int total = my_tiles * KS;
-    set_load_tile();
-    load_next(0);
-    load_next(1);
-    for (int g = 0; g < total; g += 2) {
-      if (!process(0)) break;
-      load_next(0);
-      if (g + 1 < total) {
-        if (!process(1)) break;
-        load_next(1);
+    const int join_step = (KS < NS ? KS : NS) - 1;
+    bool ok = true;
+    for (int ti = 0; ti < my_tiles && ok; ++ti) {
+      for (int ks = 0; ks < KS && ok; ++ks) {
+        ok = process();
+        if (kProducersJoinEpilogue && ok && ks == join_step && ti > 0)
+          ok = epilogue_share(tile_of(p, (int)blockIdx.x + (ti - 1) * (int)gridDim.x), (uint32_t)(ti - 1), pw >> 2);
       }
     }
+    if (kProducersJoinEpilogue && ok)
+      epilogue_share(tile_of(p, (int)blockIdx.x + (my_tiles - 1) * (int)gridDim.x), (uint32_t)(my_tiles - 1), pw >> 2);
   } else if (warp == kMmaWarp) {
     // =============================================================== MMA issuer
     if (lane == 0) {
@@ -530,10 +520,41 @@ __global__ void __launch_bounds__(kThreads, 1)
     __syncwarp();
   } else {
     // =============================================================== epilogue
-    const int q = warp & 3;  // TMEM lane quarter this warp may read
     const int et = tid - (kMmaWarp + 1) * 32;  // 0..127 among the epilogue threads
-    int32_t* s_cs = reinterpret_cast<int32_t*>(sCtl + kCtlBytes);  // 2048 * colsum of the tile's columns
-    float* s_sw = reinterpret_cast<float*>(sCtl + kCtlBytes + BN * 4);
+    // merge state (dynamic positions): word tasks tt = et + 128*jj -> (row tt / words-per-row, word)
+    const int m_GK = (p.K / p.b) * p.k;
+    const int m_nb = (BK / p.b) * p.k;  // sparse entries per row per K step
+    const bool m_word_path = !STMA && p.log2k >= 0;
+    const int m_nw_log = m_word_path ? (31 - __clz(m_nb >> 2)) : 0;
+    const int m_ntask = m_word_path ? (2 * BM << m_nw_log) / 128 : 0;  // per thread for a 256-row stage
+    const bool m_prefetch = m_ntask <= kMergeTasks;
+    uint32_t m_bank4[kMergeTasks], mv[kMergeTasks], mi[kMergeTasks];
+#pragma unroll
+    for (int jj = 0; jj < kMergeTasks; ++jj) {
+      const int q = (et + 128 * jj) & ((1 << m_nw_log) - 1);
+      uint32_t b4 = 0;
+      if (m_word_path) {
+#pragma unroll
+        for (int u = 0; u < 4; ++u) b4 |= (uint32_t)(((4 * q + u) >> p.log2k) * p.b) << (8 * u);
+      }
+      m_bank4[jj] = b4;
+      mv[jj] = mi[jj] = 0;
+    }
+    if (m_word_path && m_prefetch) {  // sparse words of the very first step
+      const Tile t0 = tile_of(p, blockIdx.x);
+#pragma unroll
+      for (int jj = 0; jj < kMergeTasks; ++jj) {
+        const int tt = et + 128 * jj;
+        if (jj < m_ntask && (tt >> m_nw_log) < t0.nsub * BM) {
+          const int m = min(t0.m0 + (tt >> m_nw_log), p.M - 1);
+          const uint32_t o = (uint32_t)m * (uint32_t)m_GK + 4 * (tt & ((1 << m_nw_log) - 1));
+          mv[jj] = __ldg(reinterpret_cast<const uint32_t*>(p.vals + o));
+          mi[jj] = p.idx != nullptr ? __ldg(reinterpret_cast<const uint32_t*>(p.idx + o))
+                                    : __ldg(reinterpret_cast<const uint32_t*>(p.pos + 4 * (tt & ((1 << m_nw_log) - 1))));
+        }
+      }
+    }
+    uint32_t mit = 0;  // position in the ring of widened stages
     uint32_t tc = 0;
     for (int j = blockIdx.x; j < nwork; j += gridDim.x, ++tc) {
       const Tile t = tile_of(p, j);
@@ -543,55 +564,106 @@ __global__ void __launch_bounds__(kThreads, 1)
         s_cs[cc] = 2048 * __ldg(p.colsum + n);
         s_sw[cc] = __ldg(p.s_w + n);
       }
-      asm volatile("bar.sync 1, %0;" ::"n"(kEpiWarps * 32) : "memory");
-      if (!mbar_wait_idle(bar_tfull, tc & 1u, abort_flag)) break;
-      tc_fence_after();
-#ifdef SQ_X_NOEPI
-      for (int sub = 0; sub < 0; ++sub) {
-#else
-      for (int sub = 0; sub < t.nsub; ++sub) {
-#endif
-        const int m = t.m0 + sub * BM + 32 * q + lane;
-        const float sh = (m < p.M) ? p.s_hi[m] : 0.f;
-        for (int c0 = 0; c0 < BN; c0 += 32) {
-          uint32_t v[32];
-          tmem_ld32(tmem + ((uint32_t)(32 * q) << 16) + (uint32_t)(sub * BN + c0), v);
-          tmem_ld_wait();
-          const int n0 = t.n0 + c0;
-          if (m < p.M && n0 < p.N) {
+      if (!STMA) {
+        // ---- dynamic positions (or static ones TMA cannot fetch): these warps, idle until the
+        //      tile's accumulators are complete, merge the sparse INT8 entries into every widened
+        //      A stage and only then hand it to the MMA thread
+        bool ok = true;
+        for (int ks = 0; ks < KS && ok; ++ks, ++mit) {
+          const int s = mit % NS;
+          // sparse words of this step (prefetched) ...
+          uint32_t cv[kMergeTasks], ci[kMergeTasks];
+          if (m_word_path && m_prefetch) {
 #pragma unroll
-            for (int c8 = 0; c8 < 32; c8 += 8) {
-              if (n0 + c8 < p.N) {  // N % 8 == 0: a group of 8 columns is all in or all out
-                int acc[8];
-                uint32_t o[4];
-                const int4 cs0 = *reinterpret_cast<const int4*>(s_cs + c0 + c8);
-                const int4 cs1 = *reinterpret_cast<const int4*>(s_cs + c0 + c8 + 4);
-                const float4 sw0 = *reinterpret_cast<const float4*>(s_sw + c0 + c8);
-                const float4 sw1 = *reinterpret_cast<const float4*>(s_sw + c0 + c8 + 4);
-                const int cs[8] = {cs0.x, cs0.y, cs0.z, cs0.w, cs1.x, cs1.y, cs1.z, cs1.w};
-                const float sw[8] = {sw0.x, sw0.y, sw0.z, sw0.w, sw1.x, sw1.y, sw1.z, sw1.w};
+            for (int jj = 0; jj < kMergeTasks; ++jj) {
+              cv[jj] = mv[jj];
+              ci[jj] = mi[jj];
+            }
+            // ... and the next step's (next tile's first step at the end of this one)
+            int nj = j, nks = ks + 1;
+            if (nks == KS) {
+              nks = 0;
+              nj += gridDim.x;
+            }
+            if (nj < nwork) {
+              const Tile nt = nks == 0 ? tile_of(p, nj) : t;
 #pragma unroll
-                for (int cc = 0; cc < 8; ++cc) acc[cc] = ((int)v[c8 + cc] - cs[cc]) >> 4;
-#pragma unroll
-                for (int cc = 0; cc < 8; cc += 2) {
-                  const float f0 = ((float)acc[cc] * sh) * sw[cc];
-                  const float f1 = ((float)acc[cc + 1] * sh) * sw[cc + 1];
-                  o[cc >> 1] = f32_to_bf16_bits(f0) | (f32_to_bf16_bits(f1) << 16);
-                }
-                *reinterpret_cast<uint4*>(p.out + (size_t)m * p.N + n0 + c8) = make_uint4(o[0], o[1], o[2], o[3]);
-                if (p.acc_out != nullptr) {
-                  int4* dst = reinterpret_cast<int4*>(p.acc_out + (size_t)m * p.N + n0 + c8);
-                  dst[0] = make_int4(acc[0], acc[1], acc[2], acc[3]);
-                  dst[1] = make_int4(acc[4], acc[5], acc[6], acc[7]);
+              for (int jj = 0; jj < kMergeTasks; ++jj) {
+                const int tt = et + 128 * jj;
+                if (jj < m_ntask && (tt >> m_nw_log) < nt.nsub * BM) {
+                  const int m = min(nt.m0 + (tt >> m_nw_log), p.M - 1);
+                  const uint32_t o = (uint32_t)m * (uint32_t)m_GK + (uint32_t)nks * (uint32_t)m_nb + 4 * (tt & ((1 << m_nw_log) - 1));
+                  mv[jj] = __ldg(reinterpret_cast<const uint32_t*>(p.vals + o));
+                  mi[jj] = p.idx != nullptr
+                               ? __ldg(reinterpret_cast<const uint32_t*>(p.idx + o))
+                               : __ldg(reinterpret_cast<const uint32_t*>(p.pos + nks * m_nb + 4 * (tt & ((1 << m_nw_log) - 1))));
                 }
               }
             }
           }
+#ifdef SQ_X_MERGE_PARK
+          ok = mbar_wait_park(bar_wfull + 8 * s, (mit / NS) & 1u, abort_flag);
+#else
+          ok = mbar_wait(bar_wfull + 8 * s, (mit / NS) & 1u, abort_flag);
+#endif
+          if (!ok) break;
+          uint8_t* a_st = sA + s * kStageA;
+          if (m_word_path && m_prefetch) {
+#pragma unroll
+            for (int jj = 0; jj < kMergeTasks; ++jj) {
+              const int tt = et + 128 * jj;
+              const int row = tt >> m_nw_log;
+              if (jj < m_ntask && row < t.nsub * BM) {
+                const uint32_t pos4 = (kpos4(ci[jj]) + m_bank4[jj]) ^ (0x01010101u * (uint32_t)((row & 7) << 4));
+                const uint32_t vx = cv[jj] ^ 0x80808080u;
+                uint8_t* rowp = a_st + row * 128;
+#ifdef SQ_X_MERGE_NOSTORE
+                if (pos4 == 0x12345678u) rowp[0] = (uint8_t)vx;
+#else
+#pragma unroll
+                for (int u = 0; u < 4; ++u) rowp[(pos4 >> (8 * u)) & 0xFFu] = (uint8_t)(vx >> (8 * u));
+#endif
+              }
+            }
+          } else if (m_word_path) {  // many entries per step: word loads without register prefetch
+            for (int tt = et; tt < ((t.nsub * BM) << m_nw_log); tt += 128) {
+              const int row = tt >> m_nw_log, q = tt & ((1 << m_nw_log) - 1);
+              const int m = min(t.m0 + row, p.M - 1);
+              const uint32_t o = (uint32_t)m * (uint32_t)m_GK + (uint32_t)ks * (uint32_t)m_nb + 4 * q;
+              const uint32_t vw = __ldg(reinterpret_cast<const uint32_t*>(p.vals + o));
+              const uint32_t iw = p.idx != nullptr ? __ldg(reinterpret_cast<const uint32_t*>(p.idx + o))
+                                                   : __ldg(reinterpret_cast<const uint32_t*>(p.pos + ks * m_nb + 4 * q));
+              uint32_t b4 = 0;
+#pragma unroll
+              for (int u = 0; u < 4; ++u) b4 |= (uint32_t)(((4 * q + u) >> p.log2k) * p.b) << (8 * u);
+              const uint32_t pos4 = (kpos4(iw) + b4) ^ (0x01010101u * (uint32_t)((row & 7) << 4));
+              const uint32_t vx = vw ^ 0x80808080u;
+              uint8_t* rowp = a_st + row * 128;
+#pragma unroll
+              for (int u = 0; u < 4; ++u) rowp[(pos4 >> (8 * u)) & 0xFFu] = (uint8_t)(vx >> (8 * u));
+            }
+          } else {  // any k: byte-wise
+            for (int tt = et; tt < t.nsub * BM * m_nb; tt += 128) {
+              const int row = tt / m_nb, i = tt - row * m_nb;
+              const int m = min(t.m0 + row, p.M - 1);
+              const int bank = i / p.k, slot_i = i - bank * p.k;
+              const int g = ks * (BK / p.b) + bank;
+              const size_t entry = (size_t)m * m_GK + (size_t)g * p.k + slot_i;
+              const uint32_t local = p.idx != nullptr ? p.idx[entry] : p.pos[(size_t)g * p.k + slot_i];
+              const uint32_t kp = (kpos1(local) + (uint32_t)(bank * p.b)) ^ (uint32_t)((row & 7) << 4);
+              a_st[row * 128 + kp] = (uint8_t)((uint8_t)p.vals[entry] ^ 0x80u);
+            }
+          }
+#ifndef SQ_X_MERGE_NOSTORE
+          fence_proxy_async_smem();
+#endif
+          mbar_arrive(bar_full + 8 * s);
         }
+        if (!ok) break;
       }
-      tc_fence_before();
-      mbar_arrive(bar_tempty);
-      asm volatile("bar.sync 1, %0;" ::"n"(kEpiWarps * 32) : "memory");  // all four warps are done with the constants
+      if (!epilogue_share(t, tc, kProducersJoinEpilogue ? 2 : 0)) break;
+      // the constants may be replaced only when every helper is done with them
+      if (!mbar_wait(bar_edone, tc & 1u, abort_flag)) break;
     }
   }
 
@@ -718,7 +790,7 @@ cudaError_t launch_gemm(int b, int k, const sq_encoded& A, const sq_weights& W,
     gemm_kernel<MAXT_, STMA_><<<grid, kThreads, kSmemBytes, st>>>(p, map_a, map_b, map_a4, map_b4);         \
   } while (0)
   if (stma) SQ_LAUNCH_GEMM(1, true);
-  else SQ_LAUNCH_GEMM(4, false);
+  else SQ_LAUNCH_GEMM(1, false);
 #undef SQ_LAUNCH_GEMM
   return cudaGetLastError();
 }
