@@ -72,34 +72,59 @@ __device__ __forceinline__ void ce(uint32_t& a, uint32_t& b) {
   b = lo;
 }
 
-// Batcher's odd-even merge sort of r[0..N), descending, both bf16 columns at once.
-template <int N>
-__device__ __forceinline__ void sort_desc(uint32_t* r) {
-#pragma unroll
-  for (int p = 1; p < N; p <<= 1) {
-#pragma unroll
-    for (int k = p; k >= 1; k >>= 1) {
-#pragma unroll
-      for (int j = k % p; j <= N - 1 - k; j += 2 * k) {
-#pragma unroll
-        for (int i = 0; i < k; ++i) {
-          if (i + j + k < N && (i + j) / (2 * p) == (i + j + k) / (2 * p)) ce(r[i + j], r[i + j + k]);
-        }
-      }
-    }
+// Batcher's odd-even merge sort of r[LO..LO+N), descending, both bf16 columns at once.
+// Written as compile-time recursion so that every index is a constant and the array stays
+// in registers whatever N is.
+template <int I, int END, int STEP, int R>
+__device__ __forceinline__ void ce_run(uint32_t* r) {  // ce(i, i+R) for i = I, I+STEP, ... < END
+  if constexpr (I < END) {
+    ce(r[I], r[I + R]);
+    ce_run<I + STEP, END, STEP, R>(r);
   }
 }
+template <int LO, int HI, int R>  // HI inclusive
+__device__ __forceinline__ void oe_merge(uint32_t* r) {
+  constexpr int STEP = R * 2;
+  if constexpr (STEP < HI - LO) {
+    oe_merge<LO, HI, STEP>(r);
+    oe_merge<LO + R, HI, STEP>(r);
+    ce_run<LO + R, HI - R, STEP, R>(r);
+  } else {
+    ce(r[LO], r[LO + R]);
+  }
+}
+template <int LO, int HI>  // HI inclusive
+__device__ __forceinline__ void oe_sort(uint32_t* r) {
+  if constexpr (HI - LO >= 1) {
+    constexpr int MID = LO + (HI - LO) / 2;
+    oe_sort<LO, MID>(r);
+    oe_sort<MID + 1, HI>(r);
+    oe_merge<LO, HI, 1>(r);
+  }
+}
+template <int N>
+__device__ __forceinline__ void sort_desc(uint32_t* r) {
+  oe_sort<0, N - 1>(r);
+}
 
-// r[0..N) bitonic -> sorted descending.
+// r[0..N) bitonic -> sorted descending (compile-time recursion, see above).
+template <int N, int S, int I>
+__device__ __forceinline__ void bitonic_stage(uint32_t* r) {
+  if constexpr (I < N) {
+    if constexpr ((I & S) == 0) ce(r[I], r[I + S]);
+    bitonic_stage<N, S, I + 1>(r);
+  }
+}
+template <int N, int S>
+__device__ __forceinline__ void bitonic_stages(uint32_t* r) {
+  if constexpr (S >= 1) {
+    bitonic_stage<N, S, 0>(r);
+    bitonic_stages<N, S / 2>(r);
+  }
+}
 template <int N>
 __device__ __forceinline__ void bitonic_merge_desc(uint32_t* r) {
-#pragma unroll
-  for (int s = N / 2; s >= 1; s >>= 1) {
-#pragma unroll
-    for (int i = 0; i < N; ++i) {
-      if ((i & s) == 0) ce(r[i], r[i + s]);
-    }
-  }
+  bitonic_stages<N, N / 2>(r);
 }
 
 // bits 0..15 of x -> even bit positions, bits 16..31 -> odd bit positions.
