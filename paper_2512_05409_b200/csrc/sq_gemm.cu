@@ -286,7 +286,7 @@ __global__ void __launch_bounds__(kThreads, 1)
             for (int cc = 0; cc < 8; cc += 2) {
               const float f0 = ((float)acc[cc] * sh) * sw[cc];
               const float f1 = ((float)acc[cc + 1] * sh) * sw[cc + 1];
-              o[cc >> 1] = f32_to_bf16_bits(f0) | (f32_to_bf16_bits(f1) << 16);
+              o[cc >> 1] = pack_bf16x2(f0, f1);
             }
             *reinterpret_cast<uint4*>(p.out + (size_t)m * p.N + n0 + c8) = make_uint4(o[0], o[1], o[2], o[3]);
             if (p.acc_out != nullptr) {
