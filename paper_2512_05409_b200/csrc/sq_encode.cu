@@ -3,9 +3,9 @@
 // Encode is one pass over HBM: 2 B read and 0.5 + 2k/b B (dynamic) or 0.5 + k/b B (static)
 // written per element.  The scale of a row is its maximum, so a row must be seen in full
 // before anything can be quantised: a GROUP of 1-16 warps owns one token row at a time,
-// staged in shared memory by one bulk asynchronous copy (double-buffered when two rows
-// fit); the host picks the group size so that a block of 16 warps (8 for b = 128) keeps as
-// many rows in flight as shared memory allows.  Groups synchronise on their own named
+// staged in shared memory by one bulk asynchronous copy; the host picks the group size
+// that keeps the most warps resident (16 per block, 8 for b = 128), so that the rows other
+// groups have in flight hide the copy latency.  Groups synchronise on their own named
 // barrier, never block-wide.
 //
 //   phase 1  (dynamic) each lane owns whole banks.  The k-th largest magnitude of a bank is
@@ -39,12 +39,6 @@ __device__ __forceinline__ uint32_t block_max_u32(uint32_t v, uint32_t* scratch)
   uint32_t r = 0;
   for (int q = 0; q < (int)(blockDim.x >> 5); ++q) r = max(r, scratch[q]);
   return r;
-}
-
-__device__ __forceinline__ uint32_t warp_max_u32(uint32_t v) {
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) v = max(v, __shfl_xor_sync(0xffffffffu, v, o));
-  return v;
 }
 
 // packed bf16x2 helpers on raw 32-bit registers (magnitudes: non-negative, finite)
@@ -191,15 +185,10 @@ __device__ __forceinline__ void quant8(const uint4& v, float c, float (&r)[8]) {
   const float2 cc = make_float2(c, c), mm = make_float2(kMagic, kMagic);
 #pragma unroll
   for (int q = 0; q < 4; ++q) {
-#ifdef SQ_X_SCALAR_FMA
-    r[2 * q] = __fmaf_rn(__uint_as_float(w[q] << 16), c, kMagic);
-    r[2 * q + 1] = __fmaf_rn(__uint_as_float(w[q] & 0xFFFF0000u), c, kMagic);
-#else
     const float2 a = make_float2(__uint_as_float(w[q] << 16), __uint_as_float(w[q] & 0xFFFF0000u));
     const float2 d = __ffma2_rn(a, cc, mm);
     r[2 * q] = d.x;
     r[2 * q + 1] = d.y;
-#endif
   }
 }
 
@@ -729,7 +718,6 @@ template <int B, int KK>
 cudaError_t launch_rows(const EncodeParams& base, cudaStream_t st) {
   EncodeParams p = base;
   const int K = p.K, G = K / B, k = (KK == 0) ? p.k : KK;
-  constexpr int NM = (B + 63) / 64;
   constexpr int kMaxWarps = (B == 128) ? 8 : 16;
   const size_t side = (((size_t)G * k * 2) + 15) & ~(size_t)15;            // stash of selected raw values
   const size_t table = (KK == 0) ? ((((size_t)G * k * 2) + 127) & ~(size_t)127) : 0;  // static offset table
@@ -752,10 +740,6 @@ cudaError_t launch_rows(const EncodeParams& base, cudaStream_t st) {
       rw = cand;
     }
   }
-#ifdef SQ_X_RW
-  rw = SQ_X_RW;
-  nbuf = SQ_X_NBUF;
-#endif
   const size_t per_group = (((size_t)nbuf * row + extra) + 127) & ~(size_t)127;
   if (per_group > 224 * 1024) return cudaErrorInvalidValue;
   int ngroups = kMaxWarps / rw;

@@ -39,12 +39,17 @@
 // and fill all 512 tensor-memory columns.  The last, partial wave of a launch is cut into
 // 128 x 256 tiles so that it spreads over twice as many SMs.
 //
-// Kernel organisation: persistent, one CTA per SM, warp-specialised.
-//   warps 0-7   producers: global loads (register-prefetched), widening, sparse merge
-//               (dynamic positions), stores into a ring of NS shared-memory stages
+// Kernel organisation: persistent, one CTA per SM, warp-specialised, two-level pipeline
+// (packed ring -> widened ring -> tensor cores).
+//   warp  13    one thread streams the packed 4-bit tiles (256 rows x 64 B of A and of B per
+//               K step) into a ring of NP packed stages by TMA
+//   warps 0-7   producers: read their chunks of a packed stage, widen them, store the
+//               swizzled 8-bit layout into a ring of NS widened stages
+//   warps 9-12  dynamic positions: merge the sparse INT8 entries into each widened A stage
+//               (byte stores, four positions per SWAR step) before it goes to the MMA thread;
+//               for every tile: epilogue (tcgen05.ld, dequantise, bf16, 16-byte stores)
 //   warp  8     one thread issues the MMAs and commits stage / accumulator barriers
-//   warps 9-12  epilogue: tcgen05.ld, dequantise, store
-//   warp  13    one thread issues the TMA loads of the sparse K steps (static positions)
+//   warp  14    static positions: one thread issues the TMA loads of the sparse K steps
 // Every wait is bounded; a wait that runs out raises an abort flag that releases all
 // other waits, the kernel records SQ_ERR_TIMEOUT and frees its tensor memory.
 #include <cuda.h>
@@ -63,20 +68,14 @@ constexpr int BN = 256;   // output channels per tile = TMEM columns of one accu
 constexpr int BK = 128;   // K elements per pipeline step = bytes per operand row
 constexpr int NS = 2;     // stages of widened (8-bit) operands
 constexpr int NP = 3;     // stages of packed (4-bit) operands as TMA delivers them
-#ifndef SQ_X_PRODWARPS
-#define SQ_X_PRODWARPS 8
-#endif
-constexpr int kProdWarps = SQ_X_PRODWARPS;
+constexpr int kProdWarps = 8;
 constexpr int kProdThreads = kProdWarps * 32;
 constexpr int kMmaWarp = kProdWarps;
 constexpr int kEpiWarps = 4;
 // Letting the (by then idle) producer warps read out two thirds of a tile's accumulators was
 // measured slower than leaving the epilogue to its own four warps (the producers then refill
 // the pipeline later), so it is compiled out; the hand-shake below supports both.
-#ifndef SQ_X_JOIN
-#define SQ_X_JOIN 0
-#endif
-constexpr bool kProducersJoinEpilogue = SQ_X_JOIN != 0;
+constexpr bool kProducersJoinEpilogue = false;
 constexpr int kEpiHelpers = kEpiWarps + (kProducersJoinEpilogue ? kProdWarps : 0);
 constexpr int kEpiStride = kProducersJoinEpilogue ? 3 : 1;  // warps per TMEM lane quarter
 constexpr int kTmaWarp = kProdWarps + 1 + kEpiWarps;  // packed dense tiles
@@ -353,10 +352,6 @@ __global__ void __launch_bounds__(kThreads, 1)
           poff[i] = 0x01010101u * (128u - (8u << e));
         }
       }
-#ifdef SQ_X_NOWORK
-      if (ra[0].x == 0x12345u) a_st[0] = (uint8_t)rb[0].x;
-      if (false)
-#endif
       // ---- widen A: nibble -> u * 2^e + (128 - 8 * 2^e)
       if (has_a) {
 #pragma unroll
@@ -370,9 +365,6 @@ __global__ void __launch_bounds__(kThreads, 1)
             od[q] = ((u >> 4) & 0x0F0F0F0Fu) * pmul[i] + poff[i];
           }
           uint8_t* dst = a_st + row0 + i * 1024;
-#ifdef SQ_X_NOSTS
-          if ((ev[0] ^ od[1] ^ ev[2] ^ od[3] ^ ev[1] ^ od[0] ^ ev[3] ^ od[2]) == 0x13579bdfu)
-#endif
           {
           *reinterpret_cast<uint4*>(dst + sw_even) = make_uint4(ev[0], ev[1], ev[2], ev[3]);
           *reinterpret_cast<uint4*>(dst + (sw_even ^ 16u)) = make_uint4(od[0], od[1], od[2], od[3]);
@@ -380,9 +372,6 @@ __global__ void __launch_bounds__(kThreads, 1)
         }
       }
       // ---- widen B: nibble -> 16 * code
-#ifdef SQ_X_NOWORK
-      if (false)
-#endif
 #pragma unroll
       for (int i = 0; i < kBTasks; ++i) {
         const uint32_t in[4] = {rb[i].x, rb[i].y, rb[i].z, rb[i].w};
@@ -393,9 +382,6 @@ __global__ void __launch_bounds__(kThreads, 1)
           od[q] = in[q] & 0xF0F0F0F0u;
         }
         uint8_t* dst = b_st + row0 + i * 1024;
-#ifdef SQ_X_NOSTS
-        if ((ev[0] ^ od[1] ^ ev[2] ^ od[3] ^ ev[1] ^ od[0] ^ ev[3] ^ od[2]) == 0x13579bdfu)
-#endif
         {
         *reinterpret_cast<uint4*>(dst + sw_even) = make_uint4(ev[0], ev[1], ev[2], ev[3]);
         *reinterpret_cast<uint4*>(dst + (sw_even ^ 16u)) = make_uint4(od[0], od[1], od[2], od[3]);
@@ -405,9 +391,7 @@ __global__ void __launch_bounds__(kThreads, 1)
       // asynchronous, and an arrive issued right behind them could let the refill overtake
       // them; after the widening every loaded register has been consumed.
       mbar_arrive(bar_pempty + 8 * ps);
-#ifndef SQ_X_NOFENCE
       fence_proxy_async_smem();  // generic-proxy writes -> visible to the tensor core's async reads
-#endif
       mbar_arrive((STMA ? bar_full : bar_wfull) + 8 * s);  // dynamic positions: the merge warps take over
       ++it;
       if (++pks == KS) {
@@ -601,11 +585,7 @@ __global__ void __launch_bounds__(kThreads, 1)
               }
             }
           }
-#ifdef SQ_X_MERGE_PARK
-          ok = mbar_wait_park(bar_wfull + 8 * s, (mit / NS) & 1u, abort_flag);
-#else
           ok = mbar_wait(bar_wfull + 8 * s, (mit / NS) & 1u, abort_flag);
-#endif
           if (!ok) break;
           uint8_t* a_st = sA + s * kStageA;
           if (m_word_path && m_prefetch) {
@@ -617,12 +597,8 @@ __global__ void __launch_bounds__(kThreads, 1)
                 const uint32_t pos4 = (kpos4(ci[jj]) + m_bank4[jj]) ^ (0x01010101u * (uint32_t)((row & 7) << 4));
                 const uint32_t vx = cv[jj] ^ 0x80808080u;
                 uint8_t* rowp = a_st + row * 128;
-#ifdef SQ_X_MERGE_NOSTORE
-                if (pos4 == 0x12345678u) rowp[0] = (uint8_t)vx;
-#else
 #pragma unroll
                 for (int u = 0; u < 4; ++u) rowp[(pos4 >> (8 * u)) & 0xFFu] = (uint8_t)(vx >> (8 * u));
-#endif
               }
             }
           } else if (m_word_path) {  // many entries per step: word loads without register prefetch
@@ -654,9 +630,7 @@ __global__ void __launch_bounds__(kThreads, 1)
               a_st[row * 128 + kp] = (uint8_t)((uint8_t)p.vals[entry] ^ 0x80u);
             }
           }
-#ifndef SQ_X_MERGE_NOSTORE
           fence_proxy_async_smem();
-#endif
           mbar_arrive(bar_full + 8 * s);
         }
         if (!ok) break;
