@@ -22,6 +22,7 @@
 //
 // Formats outside the fast kernels' set (k not a power of two, k/b other than 1/2 .. 1/16 for
 // dynamic positions) take a plain one-block-per-row kernel that ranks every element.
+#include <cstdlib>
 #include "sq_device.cuh"
 #include "sq_host.h"
 
@@ -169,6 +170,27 @@ __device__ __forceinline__ RowScale row_scale(uint32_t amax_bits, uint32_t rmax_
   return rs;
 }
 
+// The same scales computed by a whole warp at once (every lane returns all of them): the two
+// divisions run side by side on even and odd lanes, and the five candidate shifts are tried by
+// five lanes and picked with a ballot, instead of one lane walking through all of it.
+__device__ __forceinline__ RowScale row_scale_warp(uint32_t amax_bits, uint32_t rmax_bits, int lane) {
+  RowScale rs;
+  const float amax = bf16_bits_to_f32(amax_bits), rmax = bf16_bits_to_f32(rmax_bits);
+  const bool odd = lane & 1;
+  const float quot = __fdiv_rn(odd ? amax : 127.0f, odd ? 127.0f : amax);
+  const bool nz = amax > 0.f;
+  rs.inv = nz ? __shfl_sync(0xffffffffu, quot, 0) : 0.f;
+  rs.s_hi = nz ? __shfl_sync(0xffffffffu, quot, 1) : 0.f;
+  const int t = lane < 4 ? lane : 4;
+  const bool fits = rne_prod(rmax, rs.inv * __int_as_float((127 - t) << 23)) <= 7;
+  const uint32_t fit_mask = __ballot_sync(0xffffffffu, fits) & 0x1Fu;
+  rs.e = !nz ? 0 : (fit_mask ? __ffs((int)fit_mask) - 1 : 4);
+  rs.inv_lo = rs.inv * __int_as_float((127 - rs.e) << 23);
+  rs.s_lo = rs.s_hi * (float)(1 << rs.e);
+  rs.clamp = rne_prod(rmax, rs.inv_lo) > 7;
+  return rs;
+}
+
 __device__ __forceinline__ void bulk_copy_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
   asm volatile(
@@ -229,7 +251,7 @@ struct EncodeParams {
   uint8_t* shift;
   int* status;
   int64_t M;
-  int K, k;
+  int K, k, b;
   int nbuf;           // row buffers per group (1 or 2)
   int rw;             // warps per row group
   int group_stride;   // bytes of shared memory per group
@@ -508,11 +530,7 @@ __global__ void __launch_bounds__(B == 128 ? 256 : 512) encode_rows_kernel(const
     } else {
       __syncwarp();
     }
-    RowScale rs;
-    if ((threadIdx.x & 31) == 0) rs = row_scale(amax_bits, rmax_bits);  // one lane computes, the warp shares
-    rs.inv = __shfl_sync(0xffffffffu, rs.inv, 0);
-    rs.inv_lo = __shfl_sync(0xffffffffu, rs.inv_lo, 0);
-    rs.clamp = __shfl_sync(0xffffffffu, (int)rs.clamp, 0) != 0;
+    const RowScale rs = row_scale_warp(amax_bits, rmax_bits, threadIdx.x & 31);
     if (lane == 0) {
       p.s_hi[m] = rs.s_hi;
       p.s_lo[m] = rs.s_lo;
@@ -557,6 +575,161 @@ __global__ void __launch_bounds__(B == 128 ? 256 : 512) encode_rows_kernel(const
     }
   }
   if (*abort_flag && lane == 0) atomicExch(p.status, (int)SQ_ERR_TIMEOUT);
+}
+
+// ------------------------------------------------------------------------------------------------
+// Static positions, row held in registers.  A row is split over `rw` warps; each warp keeps its
+// slice of NCL * 256 elements in NCL 16-byte register quads per lane (lane l owns chunks l,
+// l + 32, ...: every load and every INT4 store is one fully coalesced warp access) and nothing
+// of the row is staged in shared memory.  What the positions imply is the same for every row,
+// so it is tabulated once per block: per element a half-word magnitude mask (0x7FFF, or 0 at a
+// selected place) and the element offset of every selected place.  Per row:
+//   load; in the same breath fetch the selected values a second time (asynchronous 4-byte
+//   copies into shared memory) -> maxima of all and of the unselected magnitudes -> scales
+//   -> INT8 codes of the selected values, INT4 codes straight from the registers (selected
+//   places were cleared there while taking the maxima).
+// The kernel is bound by instruction issue, which is why the masks are tables.
+template <int NCL, int NT>
+__global__ void __launch_bounds__(NT, 1) encode_static_regs_kernel(const EncodeParams p) {
+  extern __shared__ __align__(128) uint8_t smem_enc[];
+  const int K = p.K, k = p.k;
+  const int GK = (K / p.b) * k;
+  const int rw = p.rw;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int grp = warp / rw, slice = warp % rw;
+  const int glane = slice * 32 + lane, gsize = rw * 32;
+  const int ngroups = (NT / 32) / rw;
+  constexpr int S8 = NCL * 32;  // 16-byte chunks per warp slice
+
+  // shared memory: [magnitude masks, uint16 [K]] [selected offsets, uint16 [GK]] then per group [gathered words, uint32 [GK]] and, after all
+  // of those, 16 exchange words per group
+  const size_t jt_bytes = ((size_t)GK * 2 + 15) & ~(size_t)15;
+  const size_t stash_bytes = ((size_t)GK * 4 + 15) & ~(size_t)15;
+  uint16_t* hmask = reinterpret_cast<uint16_t*>(smem_enc);
+  uint16_t* jt = hmask + K;
+  uint32_t* stash = reinterpret_cast<uint32_t*>(reinterpret_cast<uint8_t*>(jt) + jt_bytes + stash_bytes * grp);
+  uint32_t* exch = reinterpret_cast<uint32_t*>(reinterpret_cast<uint8_t*>(jt) + jt_bytes + stash_bytes * ngroups) + grp * 16;
+  const uint32_t stash_s = smem_u32(stash);
+
+  for (int i = threadIdx.x; i < K / 2; i += NT) reinterpret_cast<uint32_t*>(hmask)[i] = 0x7FFF7FFFu;
+  __syncthreads();
+  for (int t = threadIdx.x; t < GK; t += NT) {
+    const int j = (t / k) * p.b + p.positions[t];
+    jt[t] = (uint16_t)j;
+    hmask[j] = 0;
+  }
+  __syncthreads();
+
+  const int64_t gw = (int64_t)blockIdx.x * ngroups + grp;
+  const int64_t wstride = (int64_t)gridDim.x * ngroups;
+  for (int64_t m = gw; m < p.M; m += wstride) {
+    const uint16_t* xrow = p.X + m * K;
+    const uint4* src = reinterpret_cast<const uint4*>(xrow) + slice * S8 + lane;
+    uint4 v[NCL];
+#pragma unroll
+    for (int c = 0; c < NCL; ++c) v[c] = __ldg(src + c * 32);
+    // The selected values come a second time, as the aligned 32-bit words that hold them,
+    // by asynchronous copies straight into shared memory: all in flight together with the
+    // row itself, no registers held.
+#pragma unroll 4
+    for (int t = glane; t < GK; t += gsize) {
+      const uint32_t j = jt[t];
+      asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(stash_s + 4u * (uint32_t)t), "l"(xrow + (j & ~1u))
+                   : "memory");
+    }
+
+    const uint4* mk = reinterpret_cast<const uint4*>(hmask) + slice * S8 + lane;
+    uint32_t r2 = 0, a2 = 0;
+#pragma unroll
+    for (int c = 0; c < NCL; ++c) {
+      const uint4 q = mk[c * 32];
+      a2 = max2(a2, max2(max2(v[c].x & 0x7FFF7FFFu, v[c].y & 0x7FFF7FFFu),
+                         max2(v[c].z & 0x7FFF7FFFu, v[c].w & 0x7FFF7FFFu)));
+      r2 = max2(r2, max2(max2(v[c].x & q.x, v[c].y & q.y), max2(v[c].z & q.z, v[c].w & q.w)));
+      // selected places become (signed) zeros: their codes must not reach the packing below
+      v[c].x &= q.x | 0x80008000u;
+      v[c].y &= q.y | 0x80008000u;
+      v[c].z &= q.z | 0x80008000u;
+      v[c].w &= q.w | 0x80008000u;
+    }
+    const uint32_t lane_rmax = max(r2 & 0xFFFFu, r2 >> 16);
+
+    const uint32_t lane_amax = max(a2 & 0xFFFFu, a2 >> 16);  // selected places included
+    asm volatile("cp.async.wait_all;" ::: "memory");
+
+    uint32_t amax_bits = __reduce_max_sync(0xffffffffu, lane_amax);
+    uint32_t rmax_bits = __reduce_max_sync(0xffffffffu, lane_rmax);
+    if (rw > 1) {
+      if (lane == 0) {
+        exch[slice] = amax_bits;
+        exch[8 + slice] = rmax_bits;
+      }
+      group_sync(rw, grp);  // also: every gathered word of the row is in the stash
+      amax_bits = rmax_bits = 0;
+      for (int w = 0; w < rw; ++w) {
+        amax_bits = max(amax_bits, exch[w]);
+        rmax_bits = max(rmax_bits, exch[8 + w]);
+      }
+    } else {
+      __syncwarp();
+    }
+    const RowScale rs = row_scale_warp(amax_bits, rmax_bits, lane);
+    if (glane == 0) {
+      p.s_hi[m] = rs.s_hi;
+      p.s_lo[m] = rs.s_lo;
+      p.shift[m] = (uint8_t)rs.e;
+    }
+
+    // sparse component: INT8 codes of the gathered values (|a * inv| <= 127 by construction)
+    {
+      int8_t* vdst = p.vals + (size_t)m * GK;
+      if ((GK & 3) == 0) {
+        for (int t4 = glane * 4; t4 < GK; t4 += gsize * 4) {
+          const uint4 sw = *reinterpret_cast<const uint4*>(stash + t4);
+          const uint2 jj = *reinterpret_cast<const uint2*>(jt + t4);
+          const uint32_t w[4] = {sw.x, sw.y, sw.z, sw.w};
+          const uint32_t odd[4] = {jj.x & 1u, (jj.x >> 16) & 1u, jj.y & 1u, (jj.y >> 16) & 1u};
+          uint32_t o = 0;
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            const uint32_t a = odd[q] ? (w[q] & 0xFFFF0000u) : (w[q] << 16);
+            o |= (__float_as_uint(__fmaf_rn(__uint_as_float(a), rs.inv, kMagic)) & 0xFFu) << (8 * q);
+          }
+          *reinterpret_cast<uint32_t*>(vdst + t4) = o;
+        }
+      } else {
+        for (int t = glane; t < GK; t += gsize) {
+          const uint32_t a = (jt[t] & 1u) ? (stash[t] & 0xFFFF0000u) : (stash[t] << 16);
+          vdst[t] = (int8_t)(__float_as_uint(__fmaf_rn(__uint_as_float(a), rs.inv, kMagic)) & 0xFFu);
+        }
+      }
+    }
+
+    // dense component: INT4 codes of the registers, one 32-bit word per chunk
+    uint32_t* dst = reinterpret_cast<uint32_t*>(p.dq4 + (size_t)m * (K / 2)) + slice * S8 + lane;
+    const float cq = rs.inv_lo;
+    if (rs.clamp) {
+      // Codes beyond +-7 are possible: limit the inputs instead of the codes, two elements per
+      // instruction.  xl = the bf16 at or just below 7 / cq still rounds to code 7, anything
+      // larger in magnitude would round to 7 or more, anything smaller is untouched.
+      const uint32_t xl = __float_as_uint(__fdiv_rd(7.0f, cq)) >> 16;
+      const uint32_t hi2 = xl | (xl << 16), lo2 = hi2 | 0x80008000u;
+#pragma unroll
+      for (int c = 0; c < NCL; ++c) {
+        v[c].x = max2(min2(v[c].x, hi2), lo2);
+        v[c].y = max2(min2(v[c].y, hi2), lo2);
+        v[c].z = max2(min2(v[c].z, hi2), lo2);
+        v[c].w = max2(min2(v[c].w, hi2), lo2);
+      }
+    }
+#pragma unroll
+    for (int c = 0; c < NCL; ++c) {
+      float r[8];
+      quant8(v[c], cq, r);
+      dst[c * 32] = pack_nibbles(r);
+    }
+    group_sync(rw, grp);  // the stash and the exchange words are reused by the next row
+  }
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -766,6 +939,47 @@ cudaError_t launch_rows(const EncodeParams& base, cudaStream_t st) {
   return cudaGetLastError();
 }
 
+// Register-resident static kernel: usable when a row splits into 1, 2, 4 or 8 warp slices of
+// NCL * 256 elements with NCL one of the instantiated sizes, and its tables fit in shared memory.
+template <int NCL, int NT>
+cudaError_t launch_static_regs_as(EncodeParams p, int rw, cudaStream_t st) {
+  const int GK = (p.K / p.b) * p.k;
+  const int ngroups = (NT / 32) / rw;
+  const size_t jt_bytes = ((size_t)GK * 2 + 15) & ~(size_t)15;
+  const size_t stash_bytes = ((size_t)GK * 4 + 15) & ~(size_t)15;
+  const size_t smem = (size_t)p.K * 2 + jt_bytes + (stash_bytes + 64) * ngroups;
+  if (smem > 200 * 1024) return cudaErrorNotSupported;
+  p.rw = rw;
+  int dev = 0, sms = 0;
+  cudaError_t err = cudaGetDevice(&dev);
+  if (err != cudaSuccess) return err;
+  err = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  if (err != cudaSuccess) return err;
+  err = cudaFuncSetAttribute(encode_static_regs_kernel<NCL, NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (err != cudaSuccess) return err;
+  int64_t blocks = (p.M + ngroups - 1) / ngroups;
+  if (blocks > sms) blocks = sms;
+  encode_static_regs_kernel<NCL, NT><<<(unsigned)blocks, NT, smem, st>>>(p);
+  return cudaGetLastError();
+}
+
+// cudaErrorNotSupported = this shape is left to the shared-memory kernel.  Slices of at most
+// 16 chunks per lane keep 16 warps resident (measured faster than fewer warps holding more).
+cudaError_t launch_static_regs(const EncodeParams& p, cudaStream_t st) {
+  if (p.K % 256 != 0 || p.K > 65535) return cudaErrorNotSupported;
+  for (int rw = 1; rw <= 8; rw *= 2) {
+    if ((p.K / 256) % rw != 0) continue;
+    switch (p.K / 256 / rw) {
+      case 8: return launch_static_regs_as<8, 512>(p, rw, st);
+      case 12: return launch_static_regs_as<12, 512>(p, rw, st);
+      case 14: return launch_static_regs_as<14, 512>(p, rw, st);
+      case 16: return launch_static_regs_as<16, 512>(p, rw, st);
+      default: break;
+    }
+  }
+  return cudaErrorNotSupported;
+}
+
 template <int B>
 cudaError_t launch_generic(int k, bool is_static, const uint16_t* X, int64_t M, int64_t K, const uint8_t* positions,
                            const sq_encoded& out, cudaStream_t st) {
@@ -794,10 +1008,13 @@ cudaError_t launch_encode(int b, int k, bool is_static, const uint16_t* X, int64
   p.M = M;
   p.K = (int)K;
   p.k = k;
+  p.b = b;
   p.nbuf = 1;
   p.rw = 1;
   p.group_stride = 0;
   if (is_static) {
+    const cudaError_t err = launch_static_regs(p, st);
+    if (err != cudaErrorNotSupported) return err;
     if (b == 32) return launch_rows<32, 0>(p, st);
     if (b == 64) return launch_rows<64, 0>(p, st);
     return launch_rows<128, 0>(p, st);

@@ -234,3 +234,31 @@ def test_several_tiles_per_sm(M, N, K, b, k, static):
         check_status()
         assert np.array_equal(_np(acc)[rows], acc_ref)
         assert_bf16_close(out[torch.from_numpy(rows).cuda()], ref32)
+
+
+# ----------------------------------------------------------------------------- encode: rows held in registers
+
+@pytest.mark.parametrize("K,b,k", [
+    (2048, 64, 8), (4096, 32, 4), (4096, 128, 64), (6144, 64, 4), (7168, 128, 16),
+    (12288, 64, 8), (14336, 64, 8), (16384, 32, 8), (24576, 128, 16), (32768, 64, 16),
+])
+def test_static_encode_row_slices_in_registers(K, b, k):
+    """Static positions with rows of 1, 2 or 4 warp slices, a ragged row count, and rows that
+    are all zero, all ties, one-hot, and clamping."""
+    M = 333
+    fmt = sq.make_format(b, k, True)
+    X = gen.activations(M, K, seed=K + k, outlier_fraction=0.01, outlier_scale=30.0, device="cpu").float()
+    X[0] = 0
+    X[1] = -3.0
+    X[2] = 0
+    X[2, K - 3] = 2.5
+    X[3] = X[3].abs().clamp_min(0.5)
+    X[M - 1] = 1.0
+    X = X.to(torch.bfloat16).cuda()
+    calib = gen.calibration_batch(64, K, seed=K, outlier_fraction=0.01, outlier_scale=30.0, device="cuda")
+    pos = sq.sq_calib_positions(fmt, calib)
+    pos_ref = oracle.calib_positions(b, k, _bits(calib))
+    assert np.array_equal(_np(pos), pos_ref)
+    enc = sq.sq_encode(fmt, X, pos)
+    check_status()
+    compare_encoded(enc, oracle.encode(b, k, _bits(X), pos_ref))
