@@ -230,11 +230,20 @@ __device__ __forceinline__ void dense_sweep(const uint16_t* row, int K, const Ro
       *dst = pack_nibbles(r);
     }
   } else {
+    // Codes beyond +-7 are possible: limit the inputs instead of the codes, two elements per
+    // instruction.  xl = the bf16 at or just below 7 / c still rounds to code 7, anything
+    // larger in magnitude would round to 7 or more, anything smaller is untouched.
+    const uint32_t xl = __float_as_uint(__fdiv_rd(7.0f, c)) >> 16;
+    const uint32_t hi2 = xl | (xl << 16), lo2 = hi2 | 0x80008000u;
+#pragma unroll 2
     for (int i = 0; i < iters; ++i, src += gsize, dst += gsize) {
+      uint4 v = *src;
+      v.x = max2(min2(v.x, hi2), lo2);
+      v.y = max2(min2(v.y, hi2), lo2);
+      v.z = max2(min2(v.z, hi2), lo2);
+      v.w = max2(min2(v.w, hi2), lo2);
       float r[8];
-      quant8(*src, c, r);
-#pragma unroll
-      for (int q = 0; q < 8; ++q) r[q] = fminf(fmaxf(r[q], kMagic - 7.0f), kMagic + 7.0f);
+      quant8(v, c, r);
       *dst = pack_nibbles(r);
     }
   }
