@@ -34,15 +34,21 @@
 // 128-byte swizzle (the 16-byte chunk index is XORed with row % 8), 8-row groups 1024
 // bytes apart: the canonical layout a tcgen05 shared-memory descriptor describes.
 //
-// Tiling: a CTA computes 256 x 256 outputs as two 128-row sub-tiles that share every
-// widened weight stage (one third less widening work and L2 traffic per MMA than 128 x 256)
-// and fill all 512 tensor-memory columns.  The last, partial wave of a launch is cut into
-// 128 x 256 tiles so that it spreads over twice as many SMs.
+// Tiling: a CTA accumulates 256 rows x 256 output channels as two 128-row sub-tiles that share
+// every widened weight stage and fill all 512 tensor-memory columns.  Above 128 rows the CTAs
+// work in PAIRS (clusters of two, `tcgen05.mma.cta_group::2`): the pair computes 512 x 256, each
+// CTA owns 256 rows of A and only HALF of the weight tile, which the pair's tensor cores read
+// from both shared memories.  Per MMA a CTA then widens a quarter less and its shared memory
+// serves a third less operand traffic; shared-memory bandwidth (widening stores + tensor-core
+// operand reads) is what bounds the single-CTA form.  The last, partial wave of a launch is cut
+// into tiles of one sub-tile per CTA so that it spreads over twice as many SMs.
 //
 // Kernel organisation: persistent, one CTA per SM, warp-specialised, two-level pipeline
-// (packed ring -> widened ring -> tensor cores).
-//   warp  13    one thread streams the packed 4-bit tiles (256 rows x 64 B of A and of B per
-//               K step) into a ring of NP packed stages by TMA
+// (packed ring -> widened ring -> tensor cores).  In a pair only the leader CTA's MMA thread
+// issues; both CTAs' producers arrive on the leader's "full" barriers (remote mbarrier
+// arrives), and the MMA completions are multicast to both CTAs' "empty" barriers.
+//   warp  13    one thread streams the packed 4-bit tiles (256 rows x 64 B of A, 256 or 128 rows
+//               of B per K step) into a ring of NP packed stages by TMA
 //   warps 0-7   producers: read their chunks of a packed stage, widen them, store the
 //               swizzled 8-bit layout into a ring of NS widened stages
 //   warps 9-12  dynamic positions: merge the sparse INT8 entries into each widened A stage
@@ -67,8 +73,6 @@ namespace {
 constexpr int BM = 128;   // rows of one sub-tile = TMEM lanes
 constexpr int BN = 256;   // output channels per tile = TMEM columns of one accumulator
 constexpr int BK = 128;   // K elements per pipeline step = bytes per operand row
-constexpr int NS = 2;     // stages of widened (8-bit) operands
-constexpr int NP = 3;     // stages of packed (4-bit) operands as TMA delivers them
 constexpr int kProdWarps = 8;
 constexpr int kProdThreads = kProdWarps * 32;
 constexpr int kMmaWarp = kProdWarps;
@@ -83,15 +87,28 @@ constexpr int kTmaWarp = kProdWarps + 1 + kEpiWarps;  // packed dense tiles
 constexpr int kTmaSparseWarp = kTmaWarp + 1;          // INT8 tiles of the sparse K steps
 constexpr int kThreads = (kProdWarps + 1 + kEpiWarps + 2) * 32;
 constexpr int kStageA = 2 * BM * BK;  // 32 KB: two sub-tiles of A
-constexpr int kStageB = BN * BK;      // 32 KB
 constexpr int kCtlBytes = 256;            // barriers, tensor-memory slot, abort flag
 constexpr int kEpiConstBytes = 2 * BN * 4;  // per tile: 2048 * colsum[n] and s_w[n] of its columns
 constexpr int kPackA = 2 * BM * (BK / 2);  // 16 KB: 256 rows x 64 packed bytes
-constexpr int kPackB = BN * (BK / 2);      // 16 KB
-constexpr int kSmemBytes = NS * (kStageA + kStageB) + NP * (kPackA + kPackB) + kCtlBytes + kEpiConstBytes;
-constexpr int kRowsPerWarp = 2 * BM / kProdWarps;  // rows of A (and of B) a producer warp widens per stage
+constexpr int kRowsPerWarp = 2 * BM / kProdWarps;  // rows of A a producer warp widens per stage
 constexpr int kATasks = kRowsPerWarp / 8;  // 16-byte packed chunks of A per producer thread per step
-constexpr int kBTasks = kRowsPerWarp / 8;
+
+// What depends on how many CTAs share a tensor-core tile.  PAIR = 1: one CTA computes 256 x 256
+// alone.  PAIR = 2: the two CTAs of a cluster compute 512 x 256 with `cta_group::2` MMAs; each
+// owns 256 rows of A and HALF of the weight tile (128 output channels), which the pair's tensor
+// cores read from both shared memories, so a CTA widens and holds a quarter less per MMA and
+// its shared memory serves a third less operand traffic -- the pipe this kernel is bound by.
+template <int PAIR>
+struct Geo {
+  static constexpr int NS = PAIR == 2 ? 3 : 2;  // stages of widened (8-bit) operands
+  static constexpr int NP = 3;  // stages of packed (4-bit) operands as TMA delivers them
+  static constexpr int BNL = BN / PAIR;          // weight rows (output channels) held by one CTA
+  static constexpr int kStageB = BNL * BK;       // 32 / 16 KB
+  static constexpr int kPackB = BNL * (BK / 2);  // 16 / 8 KB
+  static constexpr int kRowsPerWarpB = BNL / kProdWarps;
+  static constexpr int kBTasks = kRowsPerWarpB / 8;
+  static constexpr int kSmemBytes = NS * (kStageA + kStageB) + NP * (kPackA + kPackB) + kCtlBytes + kEpiConstBytes;
+};
 constexpr int kMergeTasks = 8;  // sparse 4-entry words per merge thread per stage kept in registers
 
 struct GemmParams {
@@ -110,20 +127,24 @@ struct GemmParams {
   int M, N, K, b, k;
   int log2k;       // log2(k) when the word path is usable, else -1
   int SS;          // sparse K steps per tile (static positions through TMA), else 0
-  // work list: `n_pairs` tiles of two sub-tiles (256 rows) followed by `n_singles` tiles of one
+  // work list: `n_pairs` tiles of two sub-tiles per CTA followed by `n_singles` tiles of one;
+  // a row unit is 128 rows per CTA of the pair (128 or 256 rows)
   int n_pairs, n_singles, n_split;  // n_split: singles that come from cutting pair tiles in two
-  int mp, mu, tiles_n;              // row pairs, row units (128 rows), column tiles
+  int mp, mu, tiles_n;              // row pairs, row units, column tiles
 };
 
 struct Tile {
-  int m0, n0, nsub;
+  int m0, n0, nsub;  // first row of THIS CTA, first output channel of the tile, sub-tiles per CTA
+  int nb0;           // first weight row THIS CTA loads and widens
 };
 
-// Entry j of the work list (identical in every role of every CTA).
-__device__ __forceinline__ Tile tile_of(const GemmParams& p, int j) {
+// Entry j of the work list (identical in every role of both CTAs of a pair, up to the rank).
+template <int PAIR>
+__device__ __forceinline__ Tile tile_of(const GemmParams& p, int j, int rank) {
+  constexpr int U = BM * PAIR;  // rows of a row unit
   Tile t;
   if (j < p.n_pairs) {
-    t.m0 = (j % p.mp) * (2 * BM);
+    t.m0 = (j % p.mp) * (2 * U);
     t.n0 = (j / p.mp) * BN;
     t.nsub = 2;
   } else {
@@ -131,13 +152,15 @@ __device__ __forceinline__ Tile tile_of(const GemmParams& p, int j) {
     t.nsub = 1;
     if (s < p.n_split) {
       const int pj = p.n_pairs + s / 2;
-      t.m0 = (pj % p.mp) * (2 * BM) + (s & 1) * BM;
+      t.m0 = (pj % p.mp) * (2 * U) + (s & 1) * U;
       t.n0 = (pj / p.mp) * BN;
     } else {  // the odd last row unit
-      t.m0 = (p.mu - 1) * BM;
+      t.m0 = (p.mu - 1) * U;
       t.n0 = (s - p.n_split) * BN;
     }
   }
+  t.m0 += rank * t.nsub * BM;
+  t.nb0 = t.n0 + rank * (BN / PAIR);
   return t;
 }
 
@@ -152,13 +175,13 @@ __device__ __forceinline__ uint64_t make_desc(uint32_t saddr) {
   return d;
 }
 
-// Instruction descriptor: D = s32, A = u8 or s8, B = s8, both K-major, M = 128, N = BN.
-__device__ __forceinline__ constexpr uint32_t make_idesc(bool a_signed) {
+// Instruction descriptor: D = s32, A = u8 or s8, B = s8, both K-major, N = BN.
+__device__ __forceinline__ constexpr uint32_t make_idesc(bool a_signed, int m) {
   return (2u << 4)                       // D format: S32
          | ((a_signed ? 1u : 0u) << 7)   // A format: 0 = unsigned, 1 = signed 8-bit
          | (1u << 10)                    // B format: signed 8-bit
          | ((uint32_t)(BN >> 3) << 17)   // N
-         | ((uint32_t)(BM >> 4) << 24);  // M
+         | ((uint32_t)(m >> 4) << 24);   // M (of the whole instruction: 128 per participating CTA)
 }
 
 // Four bank-local indices in one word -> their K positions inside the bank's 32-blocks
@@ -184,68 +207,98 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
 
 }  // namespace
 
-// MAXT: sparse word tasks per producer lane per K step that are prefetched in registers.
-// STMA: static positions through TMA-fed extra K steps.
-template <int MAXT, bool STMA>
+// Arrive on / wait for a barrier that lives in the pair's leader CTA.
+template <int PAIR>
+__device__ __forceinline__ void arrive_leader(uint32_t bar) {
+  if (PAIR == 2) mbar_arrive_cta(bar, 0);
+  else mbar_arrive(bar);
+}
+template <int PAIR>
+__device__ __forceinline__ bool wait_leader(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  return PAIR == 2 ? mbar_wait_cluster(bar, parity, abort_flag) : mbar_wait(bar, parity, abort_flag);
+}
+
+// PAIR: CTAs per tensor-core tile (see Geo).  STMA: static positions through TMA-fed extra K steps.
+template <int PAIR, bool STMA>
 __global__ void __launch_bounds__(kThreads, 1)
     gemm_kernel(const GemmParams p, const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                 const __grid_constant__ CUtensorMap map_a4, const __grid_constant__ CUtensorMap map_b4) {
+  using G = Geo<PAIR>;
+  constexpr int NS = G::NS, NP = G::NP;
+  constexpr int kStageB = G::kStageB, kPackB = G::kPackB, kBTasks = G::kBTasks;
   // The kernel has no static shared memory, so the dynamic block starts at the 1024-byte
   // aligned base the swizzled operand layout needs; checked below, never assumed.
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   uint8_t* smem = smem_raw;
+  // (uniform over the pair: both CTAs see the same offset of the dynamic block)
   if ((smem_u32(smem_raw) & 1023u) != 0) {
     if (threadIdx.x == 0) atomicExch(p.status, (int)SQ_ERR_CUDA);
     return;
   }
   uint8_t* sA = smem;                      // NS x [256][128] widened A
-  uint8_t* sB = sA + NS * kStageA;         // NS x [256][128] widened B
+  uint8_t* sB = sA + NS * kStageA;         // NS x [BNL][128] widened B
   uint8_t* sPA = sB + NS * kStageB;        // NP x [256][64]  packed A as loaded
-  uint8_t* sPB = sPA + NP * kPackA;        // NP x [256][64]  packed B as loaded
+  uint8_t* sPB = sPA + NP * kPackA;        // NP x [BNL][64]  packed B as loaded
   uint8_t* sCtl = sPB + NP * kPackB;
-  const uint32_t bar_full = smem_u32(sCtl);         // NS: dense K step widened by the producers
+  // mbarriers.  "leader" = waited for by the MMA thread of the pair's rank-0 CTA only; both
+  // CTAs arrive there.  Everything else is local to a CTA (signalled in both by multicast
+  // commits where the tensor core is the one that arrives).
+  const uint32_t bar_full = smem_u32(sCtl);         // NS, leader: dense K step widened (and merged)
   const uint32_t bar_empty = bar_full + 8 * NS;     // NS: widened stage consumed by the MMAs
-  const uint32_t bar_sfull = bar_empty + 8 * NS;    // NS: sparse K step filled by TMA
+  const uint32_t bar_sfull = bar_empty + 8 * NS;    // NS: sparse K step filled by this CTA's TMA
   const uint32_t bar_pfull = bar_sfull + 8 * NS;    // NP: packed stage landed
   const uint32_t bar_pempty = bar_pfull + 8 * NP;   // NP: packed stage read into registers
   const uint32_t bar_tfull = bar_pempty + 8 * NP;   // accumulators complete
-  const uint32_t bar_tempty = bar_tfull + 8;        // accumulators read out
+  const uint32_t bar_tempty = bar_tfull + 8;        // leader: accumulators read out
   const uint32_t bar_wfull = bar_tempty + 8;        // NS: dense K step widened, sparse entries not merged yet
   const uint32_t bar_eready = bar_wfull + 8 * NS;   // epilogue: column constants staged, every helper present
   const uint32_t bar_edone = bar_eready + 8;        // epilogue: every helper done with the constants
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(sCtl + 32 * NS + 16 * NP + 32);  // control block: kCtlBytes
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(sCtl + 32 * NS + 16 * NP + 40);
+  const uint32_t bar_sfullp = bar_edone + 8;        // NS, leader: sparse K step filled by the peer's TMA
+  static_assert(8 * (5 * NS + 2 * NP + 4) + 16 <= kCtlBytes, "control block too small");
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(sCtl + 8 * (5 * NS + 2 * NP + 4));
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(sCtl + 8 * (5 * NS + 2 * NP + 4) + 8);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  // Rank in the pair (0 = leader; clusters are (PAIR,1,1), so it is blockIdx.x % PAIR), this
+  // pair's index and the number of pairs.  Spelled out at every use instead of being kept in
+  // variables: derived from blockIdx/gridDim right where they are needed they stay in the
+  // uniform datapath, which the single-thread roles (MMA issue, TMA) depend on.
+#define rank ((int)blockIdx.x % PAIR)
+#define cl ((int)blockIdx.x / PAIR)
+#define ncl ((int)gridDim.x / PAIR)
   const int KS = p.K / BK;
   const int nwork = p.n_pairs + p.n_singles;
   const int SS = STMA ? p.SS : 0;  // sparse K steps that follow the KS dense steps of every tile
 
   if (tid == 0) {
     for (int s = 0; s < NS; ++s) {
-      // static positions: the producers complete a dense stage; otherwise the merge warps do
-      mbar_init(bar_full + 8 * s, STMA ? kProdThreads : kEpiWarps * 32);
-      mbar_init(bar_wfull + 8 * s, kProdThreads);
+      // Every thread arrives for itself right after its own proxy fence (one arrival per warp
+      // behind a __syncwarp was measured slower).  Static positions: the producers complete a
+      // dense stage; otherwise the merge warps do.
+      mbar_init(bar_full + 8 * s, PAIR * (STMA ? kProdWarps : kEpiWarps) * 32);
+      mbar_init(bar_wfull + 8 * s, kProdWarps * 32);
       mbar_init(bar_empty + 8 * s, 1);
       mbar_init(bar_sfull + 8 * s, 1);
+      mbar_init(bar_sfullp + 8 * s, 1);
     }
     for (int s = 0; s < NP; ++s) {
       mbar_init(bar_pfull + 8 * s, 1);
       mbar_init(bar_pempty + 8 * s, kProdThreads);
     }
     mbar_init(bar_tfull, 1);
-    mbar_init(bar_tempty, kEpiHelpers * 32);
+    mbar_init(bar_tempty, PAIR * kEpiHelpers * 32);
     mbar_init(bar_eready, kEpiHelpers * 32);
     mbar_init(bar_edone, kEpiHelpers * 32);
     *abort_flag = 0;
     fence_mbar_init();
   }
   if (warp == kMmaWarp) {
-    tmem_alloc(smem_u32(tmem_slot), 2 * BN);
-    tmem_relinquish();
+    tmem_alloc<PAIR>(smem_u32(tmem_slot), 2 * BN);
+    tmem_relinquish<PAIR>();
   }
   tc_fence_before();
   __syncthreads();
+  if (PAIR == 2) cluster_sync_all();  // the peer's barriers exist before anything arrives on them
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
 
@@ -299,7 +352,7 @@ __global__ void __launch_bounds__(kThreads, 1)
       }
     }
     tc_fence_before();
-    mbar_arrive(bar_tempty);
+    arrive_leader<PAIR>(bar_tempty);
     mbar_arrive(bar_edone);
     return true;
   };
@@ -315,6 +368,8 @@ __global__ void __launch_bounds__(kThreads, 1)
     const uint32_t sw_even = (uint32_t)(((2 * c) ^ r7) << 4);
     const uint32_t row0 = (uint32_t)(kRowsPerWarp * pw + r7) * 128u;          // widened: + i * 1024 for task i
     const uint32_t prow0 = (uint32_t)(kRowsPerWarp * pw + r7) * 64u + c * 16;  // packed:  + i * 512
+    const uint32_t rowb0 = (uint32_t)(G::kRowsPerWarpB * pw + r7) * 128u;      // the same for this CTA's rows of B
+    const uint32_t prowb0 = (uint32_t)(G::kRowsPerWarpB * pw + r7) * 64u + c * 16;
     // ---- processing side
     uint32_t it = 0;   // position in the ring of widened stages (dense and sparse steps)
     uint32_t pit = 0;  // position in the ring of packed stages (dense steps only)
@@ -324,8 +379,8 @@ __global__ void __launch_bounds__(kThreads, 1)
       pmul[i] = 1;
       poff[i] = 0;
     }
-    int pj = blockIdx.x, pks = 0;  // work-list entry and K step being processed
-    Tile pt = tile_of(p, pj);
+    int pj = cl, pks = 0;  // work-list entry and K step being processed
+    Tile pt = tile_of<PAIR>(p, pj, rank);
     auto process = [&]() -> bool {
       const bool has_a = pt.nsub == 2 || pw < kProdWarps / 2;  // a single-sub-tile entry only has A rows 0..127
       // ---- packed operands: wait for the TMA tiles, pull this thread's chunks into registers,
@@ -334,7 +389,7 @@ __global__ void __launch_bounds__(kThreads, 1)
       if (!mbar_wait(bar_pfull + 8 * ps, (pit / NP) & 1u, abort_flag)) return false;
       uint4 ra[kATasks], rb[kBTasks];
       const uint8_t* pa = sPA + ps * kPackA + prow0;
-      const uint8_t* pb = sPB + ps * kPackB + prow0;
+      const uint8_t* pb = sPB + ps * kPackB + prowb0;
 #pragma unroll
       for (int i = 0; i < kATasks; ++i) ra[i] = *reinterpret_cast<const uint4*>(pa + i * 512);
 #pragma unroll
@@ -382,7 +437,7 @@ __global__ void __launch_bounds__(kThreads, 1)
           ev[q] = (in[q] << 4) & 0xF0F0F0F0u;
           od[q] = in[q] & 0xF0F0F0F0u;
         }
-        uint8_t* dst = b_st + row0 + i * 1024;
+        uint8_t* dst = b_st + rowb0 + i * 1024;
         {
         *reinterpret_cast<uint4*>(dst + sw_even) = make_uint4(ev[0], ev[1], ev[2], ev[3]);
         *reinterpret_cast<uint4*>(dst + (sw_even ^ 16u)) = make_uint4(od[0], od[1], od[2], od[3]);
@@ -393,12 +448,13 @@ __global__ void __launch_bounds__(kThreads, 1)
       // them; after the widening every loaded register has been consumed.
       mbar_arrive(bar_pempty + 8 * ps);
       fence_proxy_async_smem();  // generic-proxy writes -> visible to the tensor core's async reads
-      mbar_arrive((STMA ? bar_full : bar_wfull) + 8 * s);  // dynamic positions: the merge warps take over
+      if (STMA) arrive_leader<PAIR>(bar_full + 8 * s);
+      else mbar_arrive(bar_wfull + 8 * s);  // dynamic positions: the merge warps take over
       ++it;
       if (++pks == KS) {
         pks = 0;
-        pj += gridDim.x;
-        if (pj < nwork) pt = tile_of(p, pj);
+        pj += ncl;
+        if (pj < nwork) pt = tile_of<PAIR>(p, pj, rank);
         // The sparse K steps of the tile use the next SS ring slots (TMA fills them).  They are
         // waited for one by one, not skipped: a parity wait only tells the current phase from
         // the previous one, so no role may fall more than one use behind on any stage.
@@ -412,39 +468,41 @@ __global__ void __launch_bounds__(kThreads, 1)
     // (Optional, see kProducersJoinEpilogue.)  After filling the first stages of a tile the ring
     // is full until the MMA thread moves on, and it moves on only when the previous tile's
     // accumulators have been read out: that is when the producers can lend a hand.
-    const int my_tiles = (nwork - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
+    const int my_tiles = (nwork - cl + ncl - 1) / ncl;
     const int join_step = (KS < NS ? KS : NS) - 1;
     bool ok = true;
     for (int ti = 0; ti < my_tiles && ok; ++ti) {
       for (int ks = 0; ks < KS && ok; ++ks) {
         ok = process();
         if (kProducersJoinEpilogue && ok && ks == join_step && ti > 0)
-          ok = epilogue_share(tile_of(p, (int)blockIdx.x + (ti - 1) * (int)gridDim.x), (uint32_t)(ti - 1), pw >> 2);
+          ok = epilogue_share(tile_of<PAIR>(p, cl + (ti - 1) * ncl, rank), (uint32_t)(ti - 1), pw >> 2);
       }
     }
     if (kProducersJoinEpilogue && ok)
-      epilogue_share(tile_of(p, (int)blockIdx.x + (my_tiles - 1) * (int)gridDim.x), (uint32_t)(my_tiles - 1), pw >> 2);
+      epilogue_share(tile_of<PAIR>(p, cl + (my_tiles - 1) * ncl, rank), (uint32_t)(my_tiles - 1), pw >> 2);
   } else if (warp == kMmaWarp) {
     // =============================================================== MMA issuer
-    if (lane == 0) {
-      constexpr uint32_t idesc = make_idesc(false);
-      constexpr uint32_t idesc_sparse = make_idesc(true);
+    // (the leader CTA's; the peer's MMA warp only holds its half of the tensor-memory allocation)
+    if (lane == 0 && rank == 0) {
+      constexpr uint32_t idesc = make_idesc(false, BM * PAIR);
+      constexpr uint32_t idesc_sparse = make_idesc(true, BM * PAIR);
       uint32_t it = 0, tc = 0;
       uint32_t ph_dense = 0, ph_sparse = 0;  // per-stage phase bits of the two kinds of "full" barrier
       bool ok = true;
-      for (int j = blockIdx.x; j < nwork && ok; j += gridDim.x, ++tc) {
-        const int nsub = tile_of(p, j).nsub;
-        ok = mbar_wait(bar_tempty, (tc & 1u) ^ 1u, abort_flag);  // previous tile's accumulators read out
+      for (int j = cl; j < nwork && ok; j += ncl, ++tc) {
+        const int nsub = tile_of<PAIR>(p, j, rank).nsub;
+        ok = wait_leader<PAIR>(bar_tempty, (tc & 1u) ^ 1u, abort_flag);  // previous tile's accumulators read out (both CTAs)
         if (!ok) break;
         tc_fence_after();
         for (int ks = 0; ks < KS + SS; ++ks, ++it) {
           const int s = it % NS;
           const bool sparse_step = ks >= KS;
           if (!sparse_step) {
-            ok = mbar_wait(bar_full + 8 * s, (ph_dense >> s) & 1u, abort_flag);
+            ok = wait_leader<PAIR>(bar_full + 8 * s, (ph_dense >> s) & 1u, abort_flag);
             ph_dense ^= 1u << s;
           } else {
             ok = mbar_wait(bar_sfull + 8 * s, (ph_sparse >> s) & 1u, abort_flag);
+            if (ok && PAIR == 2) ok = wait_leader<PAIR>(bar_sfullp + 8 * s, (ph_sparse >> s) & 1u, abort_flag);
             ph_sparse ^= 1u << s;
           }
           if (!ok) break;
@@ -455,11 +513,11 @@ __global__ void __launch_bounds__(kThreads, 1)
             const uint64_t da = make_desc(smem_u32(sA + s * kStageA + sub * (BM * BK)));
 #pragma unroll
             for (int kk = 0; kk < BK / 32; ++kk)  // 32 bytes of K per MMA: +2 in 16-byte address units
-              umma_i8(tmem + sub * BN, da + 2 * kk, db + 2 * kk, id, (ks > 0 || kk > 0) ? 1u : 0u);
+              umma_i8<PAIR>(tmem + sub * BN, da + 2 * kk, db + 2 * kk, id, (ks > 0 || kk > 0) ? 1u : 0u);
           }
-          umma_commit(bar_empty + 8 * s);
+          umma_commit<PAIR>(bar_empty + 8 * s);
         }
-        if (ok) umma_commit(bar_tfull);
+        if (ok) umma_commit<PAIR>(bar_tfull);
       }
     }
     __syncwarp();
@@ -468,8 +526,8 @@ __global__ void __launch_bounds__(kThreads, 1)
     if (lane == 0) {
       uint32_t pit = 0;
       bool ok = true;
-      for (int j = blockIdx.x; j < nwork && ok; j += gridDim.x) {
-        const Tile t = tile_of(p, j);
+      for (int j = cl; j < nwork && ok; j += ncl) {
+        const Tile t = tile_of<PAIR>(p, j, rank);
         for (int ks = 0; ks < KS && ok; ++ks, ++pit) {
           const int ps = pit % NP;
           ok = mbar_wait(bar_pempty + 8 * ps, ((pit / NP) & 1u) ^ 1u, abort_flag);
@@ -477,7 +535,7 @@ __global__ void __launch_bounds__(kThreads, 1)
           // rows past M / N come back as zeros (code 0)
           mbar_expect_tx(bar_pfull + 8 * ps, (uint32_t)(kPackA + kPackB));
           tma_load_2d(smem_u32(sPA + ps * kPackA), &map_a4, ks * (BK / 2), t.m0, bar_pfull + 8 * ps);
-          tma_load_2d(smem_u32(sPB + ps * kPackB), &map_b4, ks * (BK / 2), t.n0, bar_pfull + 8 * ps);
+          tma_load_2d(smem_u32(sPB + ps * kPackB), &map_b4, ks * (BK / 2), t.nb0, bar_pfull + 8 * ps);
         }
       }
     }
@@ -485,10 +543,10 @@ __global__ void __launch_bounds__(kThreads, 1)
   } else if (warp == kTmaSparseWarp) {
     // =============================================================== TMA: sparse K steps
     if (STMA && lane == 0) {
-      uint32_t it = 0;
+      uint32_t it = 0, ph_fwd = 0;
       bool ok = true;
-      for (int j = blockIdx.x; j < nwork && ok; j += gridDim.x) {
-        const Tile t = tile_of(p, j);
+      for (int j = cl; j < nwork && ok; j += ncl) {
+        const Tile t = tile_of<PAIR>(p, j, rank);
         // every ring slot is waited for in order (see the producers); only the sparse ones are filled
         for (int step = 0; step < KS + SS && ok; ++step, ++it) {
           const int s = it % NS;
@@ -498,7 +556,13 @@ __global__ void __launch_bounds__(kThreads, 1)
           // rows past M / N and columns past G*k are filled with zeros by the TMA unit
           mbar_expect_tx(bar_sfull + 8 * s, (uint32_t)(kStageA + kStageB));
           tma_load_2d(smem_u32(sA + s * kStageA), &map_a, ss * BK, t.m0, bar_sfull + 8 * s);
-          tma_load_2d(smem_u32(sB + s * kStageB), &map_b, ss * BK, t.n0, bar_sfull + 8 * s);
+          tma_load_2d(smem_u32(sB + s * kStageB), &map_b, ss * BK, t.nb0, bar_sfull + 8 * s);
+          if (PAIR == 2 && rank != 0) {
+            // the leader's MMA thread cannot watch this CTA's barrier: tell it when the tiles landed
+            ok = mbar_wait(bar_sfull + 8 * s, (ph_fwd >> s) & 1u, abort_flag);
+            ph_fwd ^= 1u << s;
+            if (ok) mbar_arrive_cta(bar_sfullp + 8 * s, 0);
+          }
         }
       }
     }
@@ -549,7 +613,7 @@ __global__ void __launch_bounds__(kThreads, 1)
         }
       }
     };
-    if (m_row_path) row_fetch(tile_of(p, blockIdx.x), 0);
+    if (m_row_path) row_fetch(tile_of<PAIR>(p, cl, rank), 0);
     uint32_t m_bank4[kMergeTasks], mv[kMergeTasks], mi[kMergeTasks];
 #pragma unroll
     for (int jj = 0; jj < kMergeTasks; ++jj) {
@@ -563,7 +627,7 @@ __global__ void __launch_bounds__(kThreads, 1)
       mv[jj] = mi[jj] = 0;
     }
     if (m_word_path && m_prefetch) {  // sparse words of the very first step
-      const Tile t0 = tile_of(p, blockIdx.x);
+      const Tile t0 = tile_of<PAIR>(p, cl, rank);
 #pragma unroll
       for (int jj = 0; jj < kMergeTasks; ++jj) {
         const int tt = et + 128 * jj;
@@ -578,8 +642,8 @@ __global__ void __launch_bounds__(kThreads, 1)
     }
     uint32_t mit = 0;  // position in the ring of widened stages
     uint32_t tc = 0;
-    for (int j = blockIdx.x; j < nwork; j += gridDim.x, ++tc) {
-      const Tile t = tile_of(p, j);
+    for (int j = cl; j < nwork; j += ncl, ++tc) {
+      const Tile t = tile_of<PAIR>(p, j, rank);
       // the tile's column constants are fetched while the main loop is still running
       for (int cc = et; cc < BN; cc += kEpiWarps * 32) {
         const int n = min(t.n0 + cc, p.N - 1);
@@ -604,9 +668,9 @@ __global__ void __launch_bounds__(kThreads, 1)
             int nj = j, nks = ks + 1;
             if (nks == KS) {
               nks = 0;
-              nj += gridDim.x;
+              nj += ncl;
             }
-            if (nj < nwork) row_fetch(nks == 0 ? tile_of(p, nj) : t, nks);
+            if (nj < nwork) row_fetch(nks == 0 ? tile_of<PAIR>(p, nj, rank) : t, nks);
           }
           if (m_word_path && m_prefetch) {
 #pragma unroll
@@ -618,10 +682,10 @@ __global__ void __launch_bounds__(kThreads, 1)
             int nj = j, nks = ks + 1;
             if (nks == KS) {
               nks = 0;
-              nj += gridDim.x;
+              nj += ncl;
             }
             if (nj < nwork) {
-              const Tile nt = nks == 0 ? tile_of(p, nj) : t;
+              const Tile nt = nks == 0 ? tile_of<PAIR>(p, nj, rank) : t;
 #pragma unroll
               for (int jj = 0; jj < kMergeTasks; ++jj) {
                 const int tt = et + 128 * jj;
@@ -700,7 +764,7 @@ __global__ void __launch_bounds__(kThreads, 1)
             }
           }
           fence_proxy_async_smem();
-          mbar_arrive(bar_full + 8 * s);
+          arrive_leader<PAIR>(bar_full + 8 * s);
         }
         if (!ok) break;
       }
@@ -712,8 +776,14 @@ __global__ void __launch_bounds__(kThreads, 1)
 
   tc_fence_before();
   __syncthreads();
+  // Neither CTA of a pair may leave (or free tensor memory) while the other can still arrive on
+  // its barriers or have MMAs reading its shared memory.
+  if (PAIR == 2) cluster_sync_all();
   if (tid == 0 && *abort_flag) atomicExch(p.status, (int)SQ_ERR_TIMEOUT);
-  if (warp == kMmaWarp) tmem_dealloc(tmem, 2 * BN);
+  if (warp == kMmaWarp) tmem_dealloc<PAIR>(tmem, 2 * BN);
+#undef rank
+#undef cl
+#undef ncl
 }
 
 cudaError_t launch_gemm(int b, int k, const sq_encoded& A, const sq_weights& W,
@@ -752,6 +822,7 @@ cudaError_t launch_gemm(int b, int k, const sq_encoded& A, const sq_weights& W,
   }
 
   static int sm_count[64] = {0};
+  static int pair_slots[64][2] = {{0}};  // CTA pairs that can be resident at once, per kernel variant
   int dev = 0;
   cudaError_t err = cudaGetDevice(&dev);
   if (err != cudaSuccess) return err;
@@ -760,20 +831,53 @@ cudaError_t launch_gemm(int b, int k, const sq_encoded& A, const sq_weights& W,
     err = cudaDeviceGetAttribute(&sm_count[dev], cudaDevAttrMultiProcessorCount, dev);
     if (err != cudaSuccess) return err;
   }
-  const int sms = sm_count[dev];
+  const bool stma = positions != nullptr && GK % 16 == 0;
+  // One CTA per tile for at most 128 rows (a second CTA would have no rows); CTA pairs otherwise.
+  const int pair = M > BM ? 2 : 1;
+  int slots = sm_count[dev];  // tiles in flight at once
+  if (pair == 2) {
+    if (pair_slots[dev][stma] == 0) {
+      cudaLaunchConfig_t qc;
+      memset(&qc, 0, sizeof(qc));
+      cudaLaunchAttribute qa[1];
+      qa[0].id = cudaLaunchAttributeClusterDimension;
+      qa[0].val.clusterDim.x = 2;
+      qa[0].val.clusterDim.y = 1;
+      qa[0].val.clusterDim.z = 1;
+      qc.gridDim = dim3((unsigned)(sm_count[dev] & ~1), 1, 1);
+      qc.blockDim = dim3(kThreads, 1, 1);
+      qc.dynamicSmemBytes = Geo<2>::kSmemBytes;
+      qc.attrs = qa;
+      qc.numAttrs = 1;
+      int n = 0;
+      if (stma) {
+        err = cudaFuncSetAttribute(gemm_kernel<2, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, Geo<2>::kSmemBytes);
+        if (err == cudaSuccess) err = cudaOccupancyMaxActiveClusters(&n, gemm_kernel<2, true>, &qc);
+      } else {
+        err = cudaFuncSetAttribute(gemm_kernel<2, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, Geo<2>::kSmemBytes);
+        if (err == cudaSuccess) err = cudaOccupancyMaxActiveClusters(&n, gemm_kernel<2, false>, &qc);
+      }
+      if (err != cudaSuccess) return err;
+      if (n < 1) return cudaErrorLaunchOutOfResources;
+      pair_slots[dev][stma] = n;
+    }
+    slots = pair_slots[dev][stma];
+  }
 
-  // Work list: 256-row tiles while they fill whole waves of the SMs; the remainder of the
-  // row pairs is cut into 128-row tiles so the last wave spreads over twice as many SMs.
-  p.mu = (int)((M + BM - 1) / BM);
+  // Work list: tiles of two row units per CTA while they fill whole waves of the slots; the
+  // remainder of the row pairs is cut into tiles of one row unit so the last wave spreads over
+  // twice as many slots.  (Row unit: 128 rows per CTA of the tile.)
+  const int U = BM * pair;
+  p.mu = (int)((M + U - 1) / U);
   p.mp = p.mu / 2;
   p.tiles_n = (int)((N + BN - 1) / BN);
   const int64_t pair_tiles = (int64_t)p.mp * p.tiles_n;
-  const int64_t as_pairs = (pair_tiles / sms) * sms;
+  const int64_t as_pairs = (pair_tiles / slots) * slots;
   p.n_pairs = (int)as_pairs;
   p.n_split = (int)(2 * (pair_tiles - as_pairs));
   p.n_singles = p.n_split + (p.mu & 1) * p.tiles_n;
   const int64_t nwork = (int64_t)p.n_pairs + p.n_singles;
-  const unsigned grid = (unsigned)(nwork < sms ? nwork : sms);
+  const unsigned grid = (unsigned)(nwork < slots ? nwork : slots) * (unsigned)pair;
 
   // Static positions: the sparse product runs as extra K steps over vals [M, G*k] and
   // w_sparse [N, G*k], fetched by TMA.  A TMA row pitch must be a multiple of 16 bytes; any
@@ -797,23 +901,23 @@ cudaError_t launch_gemm(int b, int k, const sq_encoded& A, const sq_weights& W,
     const cuuint64_t dim_a4[2] = {(cuuint64_t)(K / 2), (cuuint64_t)M};
     const cuuint64_t dim_b4[2] = {(cuuint64_t)(K / 2), (cuuint64_t)N};
     const cuuint32_t box4[2] = {BK / 2, 2 * BM};
+    const cuuint32_t box4b[2] = {BK / 2, (cuuint32_t)(BN / pair)};
     if (encode(&map_a4, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, A.dq4, dim_a4, pitch4, box4, estr,
                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
       return cudaErrorInvalidValue;
-    if (encode(&map_b4, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, W.wq4, dim_b4, pitch4, box4, estr,
+    if (encode(&map_b4, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, W.wq4, dim_b4, pitch4, box4b, estr,
                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
       return cudaErrorInvalidValue;
   }
   p.SS = 0;
-  const bool stma = positions != nullptr && GK % 16 == 0;
   if (stma) {
     const cuuint64_t pitch[1] = {(cuuint64_t)GK};
     const cuuint64_t dim_a[2] = {(cuuint64_t)GK, (cuuint64_t)M};
     const cuuint64_t dim_b[2] = {(cuuint64_t)GK, (cuuint64_t)N};
     const cuuint32_t box_a[2] = {BK, 2 * BM};
-    const cuuint32_t box_b[2] = {BK, BN};
+    const cuuint32_t box_b[2] = {BK, (cuuint32_t)(BN / pair)};
     if (encode(&map_a, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<int8_t*>(A.vals), dim_a, pitch, box_a, estr,
                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
@@ -825,15 +929,34 @@ cudaError_t launch_gemm(int b, int k, const sq_encoded& A, const sq_weights& W,
     p.SS = (int)((GK + BK - 1) / BK);
   }
 
-#define SQ_LAUNCH_GEMM(MAXT_, STMA_)                                                                        \
+#define SQ_LAUNCH_GEMM(PAIR_, STMA_)                                                                        \
   do {                                                                                                      \
-    err = cudaFuncSetAttribute(gemm_kernel<MAXT_, STMA_>, cudaFuncAttributeMaxDynamicSharedMemorySize,      \
-                               kSmemBytes);                                                                 \
+    err = cudaFuncSetAttribute(gemm_kernel<PAIR_, STMA_>, cudaFuncAttributeMaxDynamicSharedMemorySize,      \
+                               Geo<PAIR_>::kSmemBytes);                                                     \
     if (err != cudaSuccess) return err;                                                                     \
-    gemm_kernel<MAXT_, STMA_><<<grid, kThreads, kSmemBytes, st>>>(p, map_a, map_b, map_a4, map_b4);         \
+    cudaLaunchConfig_t lc;                                                                                  \
+    memset(&lc, 0, sizeof(lc));                                                                             \
+    cudaLaunchAttribute la[1];                                                                              \
+    la[0].id = cudaLaunchAttributeClusterDimension;                                                         \
+    la[0].val.clusterDim.x = PAIR_;                                                                         \
+    la[0].val.clusterDim.y = 1;                                                                             \
+    la[0].val.clusterDim.z = 1;                                                                             \
+    lc.gridDim = dim3(grid, 1, 1);                                                                          \
+    lc.blockDim = dim3(kThreads, 1, 1);                                                                     \
+    lc.dynamicSmemBytes = Geo<PAIR_>::kSmemBytes;                                                           \
+    lc.stream = st;                                                                                         \
+    lc.attrs = la;                                                                                          \
+    lc.numAttrs = (PAIR_ == 2) ? 1 : 0;                                                                     \
+    err = cudaLaunchKernelEx(&lc, gemm_kernel<PAIR_, STMA_>, p, map_a, map_b, map_a4, map_b4);              \
+    if (err != cudaSuccess) return err;                                                                     \
   } while (0)
-  if (stma) SQ_LAUNCH_GEMM(1, true);
-  else SQ_LAUNCH_GEMM(1, false);
+  if (pair == 2) {
+    if (stma) SQ_LAUNCH_GEMM(2, true);
+    else SQ_LAUNCH_GEMM(2, false);
+  } else {
+    if (stma) SQ_LAUNCH_GEMM(1, true);
+    else SQ_LAUNCH_GEMM(1, false);
+  }
 #undef SQ_LAUNCH_GEMM
   return cudaGetLastError();
 }
