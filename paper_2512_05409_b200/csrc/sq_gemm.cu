@@ -872,7 +872,15 @@ cudaError_t launch_gemm(int b, int k, const sq_encoded& A, const sq_weights& W,
   p.mp = p.mu / 2;
   p.tiles_n = (int)((N + BN - 1) / BN);
   const int64_t pair_tiles = (int64_t)p.mp * p.tiles_n;
-  const int64_t as_pairs = (pair_tiles / slots) * slots;
+  int64_t as_pairs = (pair_tiles / slots) * slots;
+  {
+    // Cutting the remainder pays only if it saves waves: a one-sub-tile tile costs about 0.65
+    // of a two-sub-tile one (it widens the same weight stage for half the MMA work).
+    const int64_t rem = pair_tiles - as_pairs;
+    const double cost_whole = (double)((rem + slots - 1) / slots);
+    const double cost_cut = 0.65 * (double)((2 * rem + slots - 1) / slots);
+    if (cost_whole <= cost_cut) as_pairs = pair_tiles;
+  }
   p.n_pairs = (int)as_pairs;
   p.n_split = (int)(2 * (pair_tiles - as_pairs));
   p.n_singles = p.n_split + (p.mu & 1) * p.tiles_n;
