@@ -208,9 +208,13 @@ def test_worst_case_accumulator_magnitude():
 
 
 @pytest.mark.parametrize("M,N,K,b,k,static", [
-    (128, 256 * 300, 1024, 64, 8, False),     # 300 single tiles: two or three per SM, 8 K steps each
-    (512, 256 * 160, 512, 128, 16, True),     # 296 pair tiles + 48 single tiles, TMA-fed sparse K steps
-    (640, 256 * 150, 768, 64, 8, False),      # pairs, split pairs and the odd last row unit together
+    (128, 256 * 300, 1024, 64, 8, False),     # one CTA per tile: 300 tiles, two or three per SM, 8 K steps each
+    (512, 256 * 160, 512, 128, 16, True),     # CTA pairs: whole tiles + a last wave cut in two, TMA-fed sparse K steps
+    (640, 256 * 150, 768, 64, 8, False),      # CTA pairs: whole tiles, cut tiles and the odd last row unit together
+    (512, 256 * 60, 384, 64, 8, True),        # CTA pairs: one wave of whole tiles (cutting would not save a wave)
+    (257, 256 * 80, 256, 64, 8, False),       # CTA pairs: second row unit holds a single row
+    (256, 256 * 90, 256, 32, 4, True),        # CTA pairs: exactly one row unit (only "odd unit" tiles)
+    (1031, 264, 640, 128, 16, False),         # CTA pairs: ragged rows and a ragged, single column tile
 ])
 def test_several_tiles_per_sm(M, N, K, b, k, static):
     """Persistent-kernel steady state: every SM walks through several tiles, so the pipelines
