@@ -218,12 +218,21 @@ __device__ __forceinline__ bool wait_leader(uint32_t bar, uint32_t parity, volat
   return PAIR == 2 ? mbar_wait_cluster(bar, parity, abort_flag) : mbar_wait(bar, parity, abort_flag);
 }
 
-// PAIR: CTAs per tensor-core tile (see Geo).  STMA: static positions through TMA-fed extra K steps.
-template <int PAIR, bool STMA>
+// PAIR: CTAs per tensor-core tile (see Geo).
+// MODE: how the sparse part reaches the tensor core.
+//   kModeMergeEpi   the epilogue warps merge the sparse entries into every widened A stage
+//                   (any bank size and k; also static positions TMA cannot fetch)
+//   kModeTma        static positions: TMA-fed extra K steps
+//   kModeMergeProd  16 sparse entries per row and K step (k/b = 1/8): every producer thread
+//                   merges one row of the 32 its warp has just widened -- no hand-over to
+//                   other warps, eight warps share the work
+constexpr int kModeMergeEpi = 0, kModeTma = 1, kModeMergeProd = 2;
+template <int PAIR, int MODE>
 __global__ void __launch_bounds__(kThreads, 1)
     gemm_kernel(const GemmParams p, const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                 const __grid_constant__ CUtensorMap map_a4, const __grid_constant__ CUtensorMap map_b4) {
   using G = Geo<PAIR>;
+  constexpr bool STMA = MODE == kModeTma, PMERGE = MODE == kModeMergeProd;
   constexpr int NS = G::NS, NP = G::NP;
   constexpr int kStageB = G::kStageB, kPackB = G::kPackB, kBTasks = G::kBTasks;
   // The kernel has no static shared memory, so the dynamic block starts at the 1024-byte
@@ -275,7 +284,7 @@ __global__ void __launch_bounds__(kThreads, 1)
       // Every thread arrives for itself right after its own proxy fence (one arrival per warp
       // behind a __syncwarp was measured slower).  Static positions: the producers complete a
       // dense stage; otherwise the merge warps do.
-      mbar_init(bar_full + 8 * s, PAIR * (STMA ? kProdWarps : kEpiWarps) * 32);
+      mbar_init(bar_full + 8 * s, PAIR * ((STMA || PMERGE) ? kProdWarps : kEpiWarps) * 32);
       mbar_init(bar_wfull + 8 * s, kProdWarps * 32);
       mbar_init(bar_empty + 8 * s, 1);
       mbar_init(bar_sfull + 8 * s, 1);
@@ -381,8 +390,39 @@ __global__ void __launch_bounds__(kThreads, 1)
     }
     int pj = cl, pks = 0;  // work-list entry and K step being processed
     Tile pt = tile_of<PAIR>(p, pj, rank);
+    // producer-side merge (PMERGE): lane l of the warp owns row 32 * pw + l of the stage and
+    // keeps that row's 16 sparse values and positions of the coming K step in registers
+    const int GKp = (p.K / p.b) * p.k;
+    uint4 nrv = make_uint4(0, 0, 0, 0), nri = nrv;
+    uint32_t pm_bank4[4] = {0, 0, 0, 0};
+    if (PMERGE) {
+#pragma unroll
+      for (int w = 0; w < 4; ++w)
+#pragma unroll
+        for (int u = 0; u < 4; ++u) pm_bank4[w] |= (uint32_t)(((4 * w + u) >> p.log2k) * p.b) << (8 * u);
+    }
+    auto sparse_fetch = [&](const Tile& ft, int fks) {
+      const int m = min(ft.m0 + 32 * pw + lane, p.M - 1);
+      const size_t o = (size_t)m * (size_t)GKp + (size_t)fks * 16;
+      const uint8_t* ip = p.idx != nullptr ? p.idx + o : p.pos + (size_t)fks * 16;
+      // (volatile: issued here, a whole K step before their use)
+      asm volatile("ld.global.nc.v4.u32 {%0,%1,%2,%3}, [%4];"
+                   : "=r"(nrv.x), "=r"(nrv.y), "=r"(nrv.z), "=r"(nrv.w)
+                   : "l"(p.vals + o));
+      asm volatile("ld.global.nc.v4.u32 {%0,%1,%2,%3}, [%4];"
+                   : "=r"(nri.x), "=r"(nri.y), "=r"(nri.z), "=r"(nri.w)
+                   : "l"(ip));
+    };
+    if (PMERGE && cl < nwork) sparse_fetch(pt, 0);
     auto process = [&]() -> bool {
       const bool has_a = pt.nsub == 2 || pw < kProdWarps / 2;  // a single-sub-tile entry only has A rows 0..127
+      uint4 crv, cri;
+      if (PMERGE) {
+        crv = nrv;
+        cri = nri;
+        if (pks + 1 < KS) sparse_fetch(pt, pks + 1);
+        else if (pj + ncl < nwork) sparse_fetch(tile_of<PAIR>(p, pj + ncl, rank), 0);
+      }
       // ---- packed operands: wait for the TMA tiles, pull this thread's chunks into registers,
       //      hand the packed stage back
       const int ps = pit % NP;
@@ -443,12 +483,27 @@ __global__ void __launch_bounds__(kThreads, 1)
         *reinterpret_cast<uint4*>(dst + (sw_even ^ 16u)) = make_uint4(od[0], od[1], od[2], od[3]);
         }
       }
+      if (PMERGE && has_a) {
+        __syncwarp();  // the warp's 32 rows are written: each lane now patches one of them
+        const int row = 32 * pw + lane;
+        const uint32_t swz = 0x01010101u * (uint32_t)((row & 7) << 4);
+        uint8_t* rowp = a_st + row * 128;
+        const uint32_t vw[4] = {crv.x, crv.y, crv.z, crv.w};
+        const uint32_t iw[4] = {cri.x, cri.y, cri.z, cri.w};
+#pragma unroll
+        for (int w = 0; w < 4; ++w) {
+          const uint32_t pos4 = (kpos4(iw[w]) + pm_bank4[w]) ^ swz;
+          const uint32_t vx = vw[w] ^ 0x80808080u;
+#pragma unroll
+          for (int u = 0; u < 4; ++u) rowp[(pos4 >> (8 * u)) & 0xFFu] = (uint8_t)(vx >> (8 * u));
+        }
+      }
       // The packed stage goes back to the TMA thread only now: shared-memory loads are
       // asynchronous, and an arrive issued right behind them could let the refill overtake
       // them; after the widening every loaded register has been consumed.
       mbar_arrive(bar_pempty + 8 * ps);
       fence_proxy_async_smem();  // generic-proxy writes -> visible to the tensor core's async reads
-      if (STMA) arrive_leader<PAIR>(bar_full + 8 * s);
+      if (STMA || PMERGE) arrive_leader<PAIR>(bar_full + 8 * s);
       else mbar_arrive(bar_wfull + 8 * s);  // dynamic positions: the merge warps take over
       ++it;
       if (++pks == KS) {
@@ -573,7 +628,7 @@ __global__ void __launch_bounds__(kThreads, 1)
     // merge state (dynamic positions): word tasks tt = et + 128*jj -> (row tt / words-per-row, word)
     const int m_GK = (p.K / p.b) * p.k;
     const int m_nb = (BK / p.b) * p.k;  // sparse entries per row per K step
-    const bool m_word_path = !STMA && p.log2k >= 0;
+    const bool m_word_path = !STMA && !PMERGE && p.log2k >= 0;
     const int m_nw_log = m_word_path ? (31 - __clz(m_nb >> 2)) : 0;
     const int m_ntask = m_word_path ? (2 * BM << m_nw_log) / 128 : 0;  // per thread for a 256-row stage
     // Row path (16 sparse entries per row and K step, the k/b = 1/8 formats): a thread owns rows
@@ -650,7 +705,7 @@ __global__ void __launch_bounds__(kThreads, 1)
         s_cs[cc] = 2048 * __ldg(p.colsum + n);
         s_sw[cc] = __ldg(p.s_w + n);
       }
-      if (!STMA) {
+      if (!STMA && !PMERGE) {
         // ---- dynamic positions (or static ones TMA cannot fetch): these warps, idle until the
         //      tile's accumulators are complete, merge the sparse INT8 entries into every widened
         //      A stage and only then hand it to the MMA thread
@@ -822,7 +877,7 @@ cudaError_t launch_gemm(int b, int k, const sq_encoded& A, const sq_weights& W,
   }
 
   static int sm_count[64] = {0};
-  static int pair_slots[64][2] = {{0}};  // CTA pairs that can be resident at once, per kernel variant
+  static int pair_slots[64][3] = {{0}};  // CTA pairs that can be resident at once, per kernel variant
   int dev = 0;
   cudaError_t err = cudaGetDevice(&dev);
   if (err != cudaSuccess) return err;
@@ -832,11 +887,16 @@ cudaError_t launch_gemm(int b, int k, const sq_encoded& A, const sq_weights& W,
     if (err != cudaSuccess) return err;
   }
   const bool stma = positions != nullptr && GK % 16 == 0;
+  // 16 sparse entries per row and K step, fetched with aligned 16-byte loads: the producers merge
+  const uint8_t* pos_src = positions == nullptr ? A.idx : positions;
+  const bool pmerge = !stma && nb == 16 && p.log2k >= 0 && GK % 16 == 0 &&
+                      ((reinterpret_cast<uintptr_t>(A.vals) | reinterpret_cast<uintptr_t>(pos_src)) & 15) == 0;
+  const int mode = stma ? kModeTma : (pmerge ? kModeMergeProd : kModeMergeEpi);
   // One CTA per tile for at most 128 rows (a second CTA would have no rows); CTA pairs otherwise.
   const int pair = M > BM ? 2 : 1;
   int slots = sm_count[dev];  // tiles in flight at once
   if (pair == 2) {
-    if (pair_slots[dev][stma] == 0) {
+    if (pair_slots[dev][mode] == 0) {
       cudaLaunchConfig_t qc;
       memset(&qc, 0, sizeof(qc));
       cudaLaunchAttribute qa[1];
@@ -850,18 +910,16 @@ cudaError_t launch_gemm(int b, int k, const sq_encoded& A, const sq_weights& W,
       qc.attrs = qa;
       qc.numAttrs = 1;
       int n = 0;
-      if (stma) {
-        err = cudaFuncSetAttribute(gemm_kernel<2, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, Geo<2>::kSmemBytes);
-        if (err == cudaSuccess) err = cudaOccupancyMaxActiveClusters(&n, gemm_kernel<2, true>, &qc);
-      } else {
-        err = cudaFuncSetAttribute(gemm_kernel<2, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, Geo<2>::kSmemBytes);
-        if (err == cudaSuccess) err = cudaOccupancyMaxActiveClusters(&n, gemm_kernel<2, false>, &qc);
-      }
+      const void* fn = mode == kModeTma ? (const void*)gemm_kernel<2, kModeTma>
+                       : mode == kModeMergeProd ? (const void*)gemm_kernel<2, kModeMergeProd>
+                                                : (const void*)gemm_kernel<2, kModeMergeEpi>;
+      err = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, Geo<2>::kSmemBytes);
+      if (err == cudaSuccess) err = cudaOccupancyMaxActiveClusters(&n, fn, &qc);
       if (err != cudaSuccess) return err;
       if (n < 1) return cudaErrorLaunchOutOfResources;
-      pair_slots[dev][stma] = n;
+      pair_slots[dev][mode] = n;
     }
-    slots = pair_slots[dev][stma];
+    slots = pair_slots[dev][mode];
   }
 
   // Work list: tiles of two row units per CTA while they fill whole waves of the slots; the
@@ -937,9 +995,9 @@ cudaError_t launch_gemm(int b, int k, const sq_encoded& A, const sq_weights& W,
     p.SS = (int)((GK + BK - 1) / BK);
   }
 
-#define SQ_LAUNCH_GEMM(PAIR_, STMA_)                                                                        \
+#define SQ_LAUNCH_GEMM(PAIR_, MODE_)                                                                        \
   do {                                                                                                      \
-    err = cudaFuncSetAttribute(gemm_kernel<PAIR_, STMA_>, cudaFuncAttributeMaxDynamicSharedMemorySize,      \
+    err = cudaFuncSetAttribute(gemm_kernel<PAIR_, MODE_>, cudaFuncAttributeMaxDynamicSharedMemorySize,      \
                                Geo<PAIR_>::kSmemBytes);                                                     \
     if (err != cudaSuccess) return err;                                                                     \
     cudaLaunchConfig_t lc;                                                                                  \
@@ -955,15 +1013,17 @@ cudaError_t launch_gemm(int b, int k, const sq_encoded& A, const sq_weights& W,
     lc.stream = st;                                                                                         \
     lc.attrs = la;                                                                                          \
     lc.numAttrs = (PAIR_ == 2) ? 1 : 0;                                                                     \
-    err = cudaLaunchKernelEx(&lc, gemm_kernel<PAIR_, STMA_>, p, map_a, map_b, map_a4, map_b4);              \
+    err = cudaLaunchKernelEx(&lc, gemm_kernel<PAIR_, MODE_>, p, map_a, map_b, map_a4, map_b4);              \
     if (err != cudaSuccess) return err;                                                                     \
   } while (0)
   if (pair == 2) {
-    if (stma) SQ_LAUNCH_GEMM(2, true);
-    else SQ_LAUNCH_GEMM(2, false);
+    if (mode == kModeTma) SQ_LAUNCH_GEMM(2, kModeTma);
+    else if (mode == kModeMergeProd) SQ_LAUNCH_GEMM(2, kModeMergeProd);
+    else SQ_LAUNCH_GEMM(2, kModeMergeEpi);
   } else {
-    if (stma) SQ_LAUNCH_GEMM(1, true);
-    else SQ_LAUNCH_GEMM(1, false);
+    if (mode == kModeTma) SQ_LAUNCH_GEMM(1, kModeTma);
+    else if (mode == kModeMergeProd) SQ_LAUNCH_GEMM(1, kModeMergeProd);
+    else SQ_LAUNCH_GEMM(1, kModeMergeEpi);
   }
 #undef SQ_LAUNCH_GEMM
   return cudaGetLastError();
