@@ -598,27 +598,61 @@ __global__ void __launch_bounds__(kThreads, 1)
   } else if (warp == kTmaSparseWarp) {
     // =============================================================== TMA: sparse K steps
     if (STMA && lane == 0) {
-      uint32_t it = 0, ph_fwd = 0;
+      uint32_t it = 0;
+      // The leader's MMA thread cannot watch the peer's barriers, so the peer's thread tells it
+      // when each of its tiles has landed.  It does so while waiting for the next free slot
+      // (never blocking on a load it has just issued), oldest load first.
+      const bool forwards = PAIR == 2 && rank != 0;
+      uint32_t fq[NS];            // slots of the loads not yet reported, in issue order
+      uint32_t fq_head = 0, fq_n = 0, ph_fwd = 0;
+      auto try_forward = [&]() {
+        while (fq_n > 0) {
+          const uint32_t fs = fq[fq_head % NS];
+          if (!mbar_test(bar_sfull + 8 * fs, (ph_fwd >> fs) & 1u)) break;
+          ph_fwd ^= 1u << fs;
+          mbar_arrive_cta(bar_sfullp + 8 * fs, 0);
+          ++fq_head;
+          --fq_n;
+        }
+      };
       bool ok = true;
       for (int j = cl; j < nwork && ok; j += ncl) {
         const Tile t = tile_of<PAIR>(p, j, rank);
         // every ring slot is waited for in order (see the producers); only the sparse ones are filled
         for (int step = 0; step < KS + SS && ok; ++step, ++it) {
           const int s = it % NS;
-          ok = mbar_wait(bar_empty + 8 * s, ((it / NS) & 1u) ^ 1u, abort_flag);
+          const uint32_t par = ((it / NS) & 1u) ^ 1u;
+          if (!forwards) {
+            ok = mbar_wait(bar_empty + 8 * s, par, abort_flag);
+          } else {
+            ok = false;
+            for (uint32_t n = 0; n < kSpinLimit; ++n) {
+              if (mbar_test(bar_empty + 8 * s, par)) {
+                ok = true;
+                break;
+              }
+              try_forward();
+              if ((n & 1023u) == 1023u && *abort_flag) break;
+            }
+            if (!ok) *abort_flag = 1;
+          }
           if (!ok || step < KS) continue;
           const int ss = step - KS;
           // rows past M / N and columns past G*k are filled with zeros by the TMA unit
           mbar_expect_tx(bar_sfull + 8 * s, (uint32_t)(kStageA + kStageB));
           tma_load_2d(smem_u32(sA + s * kStageA), &map_a, ss * BK, t.m0, bar_sfull + 8 * s);
           tma_load_2d(smem_u32(sB + s * kStageB), &map_b, ss * BK, t.nb0, bar_sfull + 8 * s);
-          if (PAIR == 2 && rank != 0) {
-            // the leader's MMA thread cannot watch this CTA's barrier: tell it when the tiles landed
-            ok = mbar_wait(bar_sfull + 8 * s, (ph_fwd >> s) & 1u, abort_flag);
-            ph_fwd ^= 1u << s;
-            if (ok) mbar_arrive_cta(bar_sfullp + 8 * s, 0);
+          if (forwards) {
+            fq[(fq_head + fq_n) % NS] = (uint32_t)s;
+            ++fq_n;
+            try_forward();
           }
         }
+      }
+      // report what is still in flight
+      for (uint32_t n = 0; forwards && ok && fq_n > 0 && n < kSpinLimit; ++n) {
+        try_forward();
+        if ((n & 1023u) == 1023u && *abort_flag) break;
       }
     }
     __syncwarp();
