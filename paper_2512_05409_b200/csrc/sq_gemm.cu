@@ -665,44 +665,7 @@ __global__ void __launch_bounds__(kThreads, 1)
     const bool m_word_path = !STMA && !PMERGE && p.log2k >= 0;
     const int m_nw_log = m_word_path ? (31 - __clz(m_nb >> 2)) : 0;
     const int m_ntask = m_word_path ? (2 * BM << m_nw_log) / 128 : 0;  // per thread for a 256-row stage
-    // Row path (16 sparse entries per row and K step, the k/b = 1/8 formats): a thread owns rows
-    // et and et + 128 of the stage and fetches each row's 16 values and 16 positions as one
-    // 16-byte load apiece, one K step ahead.
-    const bool m_row_path = m_word_path && m_nb == 16 && (m_GK & 15) == 0 &&
-                            ((reinterpret_cast<uintptr_t>(p.vals) | reinterpret_cast<uintptr_t>(p.idx) |
-                              reinterpret_cast<uintptr_t>(p.pos)) & 15) == 0;
-    const bool m_prefetch = !m_row_path && m_ntask <= kMergeTasks;
-    uint4 rv[2], ri[2];
-    rv[0] = rv[1] = ri[0] = ri[1] = make_uint4(0, 0, 0, 0);
-    uint32_t r_bank4[4];
-#pragma unroll
-    for (int w = 0; w < 4; ++w) {
-      uint32_t b4 = 0;
-      if (m_row_path) {
-#pragma unroll
-        for (int u = 0; u < 4; ++u) b4 |= (uint32_t)(((4 * w + u) >> p.log2k) * p.b) << (8 * u);
-      }
-      r_bank4[w] = b4;
-    }
-    auto row_fetch = [&](const Tile& ft, int fks) {
-#pragma unroll
-      for (int h = 0; h < 2; ++h) {
-        if (h < ft.nsub) {
-          const int m = min(ft.m0 + h * BM + et, p.M - 1);
-          const size_t o = (size_t)m * (size_t)m_GK + (size_t)fks * 16;
-          // (volatile: issued here, a whole K step before their use, not wherever the compiler
-          // would sink them to)
-          const uint8_t* ip = p.idx != nullptr ? p.idx + o : p.pos + (size_t)fks * 16;
-          asm volatile("ld.global.nc.v4.u32 {%0,%1,%2,%3}, [%4];"
-                       : "=r"(rv[h].x), "=r"(rv[h].y), "=r"(rv[h].z), "=r"(rv[h].w)
-                       : "l"(p.vals + o));
-          asm volatile("ld.global.nc.v4.u32 {%0,%1,%2,%3}, [%4];"
-                       : "=r"(ri[h].x), "=r"(ri[h].y), "=r"(ri[h].z), "=r"(ri[h].w)
-                       : "l"(ip));
-        }
-      }
-    };
-    if (m_row_path) row_fetch(tile_of<PAIR>(p, cl, rank), 0);
+    const bool m_prefetch = m_ntask <= kMergeTasks;
     uint32_t m_bank4[kMergeTasks], mv[kMergeTasks], mi[kMergeTasks];
 #pragma unroll
     for (int jj = 0; jj < kMergeTasks; ++jj) {
@@ -748,19 +711,6 @@ __global__ void __launch_bounds__(kThreads, 1)
           const int s = mit % NS;
           // sparse words of this step (prefetched) ...
           uint32_t cv[kMergeTasks], ci[kMergeTasks];
-          uint4 crv[2], cri[2];
-          if (m_row_path) {
-            crv[0] = rv[0];
-            crv[1] = rv[1];
-            cri[0] = ri[0];
-            cri[1] = ri[1];
-            int nj = j, nks = ks + 1;
-            if (nks == KS) {
-              nks = 0;
-              nj += ncl;
-            }
-            if (nj < nwork) row_fetch(nks == 0 ? tile_of<PAIR>(p, nj, rank) : t, nks);
-          }
           if (m_word_path && m_prefetch) {
 #pragma unroll
             for (int jj = 0; jj < kMergeTasks; ++jj) {
@@ -792,25 +742,7 @@ __global__ void __launch_bounds__(kThreads, 1)
           ok = mbar_wait(bar_wfull + 8 * s, (mit / NS) & 1u, abort_flag);
           if (!ok) break;
           uint8_t* a_st = sA + s * kStageA;
-          if (m_row_path) {
-#pragma unroll
-            for (int h = 0; h < 2; ++h) {
-              if (h < t.nsub) {
-                const int row = h * BM + et;
-                const uint32_t swz = 0x01010101u * (uint32_t)((row & 7) << 4);
-                uint8_t* rowp = a_st + row * 128;
-                const uint32_t vw[4] = {crv[h].x, crv[h].y, crv[h].z, crv[h].w};
-                const uint32_t iw[4] = {cri[h].x, cri[h].y, cri[h].z, cri[h].w};
-#pragma unroll
-                for (int w = 0; w < 4; ++w) {
-                  const uint32_t pos4 = (kpos4(iw[w]) + r_bank4[w]) ^ swz;
-                  const uint32_t vx = vw[w] ^ 0x80808080u;
-#pragma unroll
-                  for (int u = 0; u < 4; ++u) rowp[(pos4 >> (8 * u)) & 0xFFu] = (uint8_t)(vx >> (8 * u));
-                }
-              }
-            }
-          } else if (m_word_path && m_prefetch) {
+          if (m_word_path && m_prefetch) {
 #pragma unroll
             for (int jj = 0; jj < kMergeTasks; ++jj) {
               const int tt = et + 128 * jj;
