@@ -172,6 +172,22 @@ sq_status sq_gemm(const sq_format* fmt, const sq_encoded* A, const sq_weights* W
                   const uint8_t* positions, int64_t M, int64_t N, int64_t K, void* out_bf16,
                   int32_t* acc_out, void* cuda_stream);
 
+/* The same product (Section 3.3) with a caller-owned workspace, for the decode-shaped case
+ * of few tokens (M <= 128): a launch then has only N/256 output tiles, each walking all of
+ * K, so most SMs idle.  Given a workspace the call may cut K into up to 8 parts that run
+ * on different SMs, leave their raw int32 partial sums in the workspace ([parts][M][N]) and
+ * add them up in a second kernel on the same stream.  The result is bit-identical to
+ * sq_gemm's (integer partial sums, the same epilogue operations in the same order).
+ * sq_gemm_workspace_bytes: *bytes = the size with which this shape would be split, 0 if it
+ * would not be (M > 128, too many tiles already, or too few K steps).
+ * workspace: device memory, 16-byte aligned, or NULL (= sq_gemm); a smaller workspace than
+ * asked for is used for fewer parts or not at all, never an error.  Its contents are
+ * undefined afterwards; calls that share a workspace must not overlap on the GPU. */
+sq_status sq_gemm_workspace_bytes(const sq_format* fmt, int64_t M, int64_t N, int64_t K, size_t* bytes);
+sq_status sq_gemm_ws(const sq_format* fmt, const sq_encoded* A, const sq_weights* W,
+                     const uint8_t* positions, int64_t M, int64_t N, int64_t K, void* out_bf16,
+                     int32_t* acc_out, void* workspace, size_t workspace_bytes, void* cuda_stream);
+
 /* Decode (inverse of Eq. 1): out[m,j] = bf16_rne(s_hi[m]*vals) at selected positions,
  * bf16_rne(s_lo[m]*dq4) elsewhere.  out_bf16: device bf16 [M, K], written. */
 sq_status sq_decode(const sq_format* fmt, const sq_encoded* A, const uint8_t* positions,

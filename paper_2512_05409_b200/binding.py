@@ -66,10 +66,13 @@ def _load() -> ctypes.CDLL:
     lib.sq_pack_weights.argtypes = [P(sq_format), VP, I64, I64, VP, P(sq_weights), VP]
     lib.sq_encode.argtypes = [P(sq_format), VP, I64, I64, VP, P(sq_encoded), VP]
     lib.sq_gemm.argtypes = [P(sq_format), P(sq_encoded), P(sq_weights), VP, I64, I64, I64, VP, VP, VP]
+    lib.sq_gemm_ws.argtypes = [P(sq_format), P(sq_encoded), P(sq_weights), VP, I64, I64, I64, VP, VP, VP,
+                               ctypes.c_size_t, VP]
+    lib.sq_gemm_workspace_bytes.argtypes = [P(sq_format), I64, I64, I64, P(ctypes.c_size_t)]
     lib.sq_decode.argtypes = [P(sq_format), P(sq_encoded), VP, I64, I64, VP, VP]
     lib.sq_device_status.argtypes = [VP]
     for name in ("sq_encoded_sizes", "sq_weights_sizes", "sq_calib_positions", "sq_pack_weights",
-                 "sq_encode", "sq_gemm", "sq_decode", "sq_device_status"):
+                 "sq_encode", "sq_gemm", "sq_gemm_ws", "sq_gemm_workspace_bytes", "sq_decode", "sq_device_status"):
         getattr(lib, name).restype = ctypes.c_int
     return lib
 
@@ -218,16 +221,49 @@ def sq_encode(fmt: sq_format, X: torch.Tensor, positions: torch.Tensor | None = 
     return out
 
 
-def sq_gemm(fmt: sq_format, A: Encoded, W: Weights, positions: torch.Tensor | None = None,
-            out: torch.Tensor | None = None, acc_out: torch.Tensor | None = None, stream=None) -> torch.Tensor:
+def sq_gemm_workspace_bytes(fmt: sq_format, M: int, N: int, K: int) -> int:
+    need = ctypes.c_size_t(0)
+    _check(_lib.sq_gemm_workspace_bytes(ctypes.byref(fmt), M, N, K, ctypes.byref(need)), "sq_gemm_workspace_bytes")
+    return int(need.value)
+
+
+def sq_gemm_ws(fmt: sq_format, A: Encoded, W: Weights, positions: torch.Tensor | None = None,
+               out: torch.Tensor | None = None, acc_out: torch.Tensor | None = None,
+               workspace: torch.Tensor | None = None, stream=None) -> torch.Tensor:
     M, K = A.dq4.shape[0], A.dq4.shape[1] * 2
     N = W.wq4.shape[0]
     if out is None:
         out = _buf(M * N * 2, torch.bfloat16, A.dq4.device)[: M * N].view(M, N)
     ca, cw = A.c_struct(), W.c_struct()
-    _check(_lib.sq_gemm(ctypes.byref(fmt), ctypes.byref(ca), ctypes.byref(cw), _ptr(positions), M, N, K,
-                        _ptr(out), _ptr(acc_out), _stream(stream)), "sq_gemm")
+    nbytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    _check(_lib.sq_gemm_ws(ctypes.byref(fmt), ctypes.byref(ca), ctypes.byref(cw), _ptr(positions), M, N, K,
+                           _ptr(out), _ptr(acc_out), _ptr(workspace), nbytes, _stream(stream)), "sq_gemm_ws")
     return out
+
+
+def sq_gemm(fmt: sq_format, A: Encoded, W: Weights, positions: torch.Tensor | None = None,
+            out: torch.Tensor | None = None, acc_out: torch.Tensor | None = None, stream=None,
+            use_workspace: bool = True) -> torch.Tensor:
+    """sq_gemm of the C ABI; decode-shaped calls (few rows) go through sq_gemm_ws with a scratch buffer
+    cached per device (so calls on one device must not overlap on the GPU: keep them on one stream,
+    or pass use_workspace=False)."""
+    M, K = A.dq4.shape[0], A.dq4.shape[1] * 2
+    N = W.wq4.shape[0]
+    need = sq_gemm_workspace_bytes(fmt, M, N, K) if use_workspace else 0
+    ws = _workspace(need, A.dq4.device) if need else None
+    return sq_gemm_ws(fmt, A, W, positions, out=out, acc_out=acc_out, workspace=ws, stream=stream)
+
+
+_workspaces: dict = {}
+
+
+def _workspace(nbytes: int, device) -> torch.Tensor:
+    key = str(device)
+    buf = _workspaces.get(key)
+    if buf is None or buf.numel() < nbytes:
+        buf = torch.empty(max(nbytes, 1 << 20), dtype=torch.uint8, device=device)
+        _workspaces[key] = buf
+    return buf
 
 
 def sq_decode(fmt: sq_format, A: Encoded, positions: torch.Tensor | None = None,

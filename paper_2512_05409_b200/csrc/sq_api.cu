@@ -176,9 +176,21 @@ sq_status sq_encode(const sq_format* fmt, const void* X_bf16, int64_t M, int64_t
                                  static_cast<cudaStream_t>(cuda_stream)));
 }
 
-sq_status sq_gemm(const sq_format* fmt, const sq_encoded* A, const sq_weights* W,
-                  const uint8_t* positions, int64_t M, int64_t N, int64_t K, void* out_bf16,
-                  int32_t* acc_out, void* cuda_stream) {
+sq_status sq_gemm_workspace_bytes(const sq_format* fmt, int64_t M, int64_t N, int64_t K, size_t* bytes) {
+  SQ_TRY(check_format(fmt));
+  SQ_TRY(check_k(K));
+  if (bytes == nullptr) return SQ_ERR_NULL_POINTER;
+  if (M < 0 || N < 0 || N % 8 != 0 || M > INT32_MAX || N > INT32_MAX) return SQ_ERR_INVALID_ARG;
+  *bytes = 0;
+  if (M == 0 || N == 0) return SQ_OK;
+  SQ_TRY(check_device());
+  *bytes = gemm_workspace_bytes(M, N, K);
+  return SQ_OK;
+}
+
+sq_status sq_gemm_ws(const sq_format* fmt, const sq_encoded* A, const sq_weights* W,
+                     const uint8_t* positions, int64_t M, int64_t N, int64_t K, void* out_bf16,
+                     int32_t* acc_out, void* workspace, size_t workspace_bytes, void* cuda_stream) {
   SQ_TRY(check_format(fmt));
   SQ_TRY(check_k(K));
   if (M < 0 || N < 0 || N % 8 != 0 || M > INT32_MAX || N > INT32_MAX) return SQ_ERR_INVALID_ARG;
@@ -187,13 +199,20 @@ sq_status sq_gemm(const sq_format* fmt, const sq_encoded* A, const sq_weights* W
   SQ_TRY(check_encoded(fmt, A));
   SQ_TRY(check_weights(fmt, W));
   if (out_bf16 == nullptr) return SQ_ERR_NULL_POINTER;
-  if (!aligned16(out_bf16) || !aligned16(acc_out)) return SQ_ERR_ALIGNMENT;
+  if (!aligned16(out_bf16) || !aligned16(acc_out) || !aligned16(workspace)) return SQ_ERR_ALIGNMENT;
   if ((M + 127) / 128 > 65535) return SQ_ERR_UNSUPPORTED;
   SQ_TRY(check_device());
   int* status = status_word();
   if (status == nullptr) return SQ_ERR_CUDA;
   return from_cuda(launch_gemm(fmt->bank, fmt->k, *A, *W, positions, M, N, K, static_cast<uint16_t*>(out_bf16),
-                               acc_out, status, static_cast<cudaStream_t>(cuda_stream)));
+                               acc_out, status, workspace, workspace == nullptr ? 0 : workspace_bytes,
+                               static_cast<cudaStream_t>(cuda_stream)));
+}
+
+sq_status sq_gemm(const sq_format* fmt, const sq_encoded* A, const sq_weights* W,
+                  const uint8_t* positions, int64_t M, int64_t N, int64_t K, void* out_bf16,
+                  int32_t* acc_out, void* cuda_stream) {
+  return sq_gemm_ws(fmt, A, W, positions, M, N, K, out_bf16, acc_out, nullptr, 0, cuda_stream);
 }
 
 sq_status sq_decode(const sq_format* fmt, const sq_encoded* A, const uint8_t* positions,

@@ -124,9 +124,12 @@ struct GemmParams {
   uint16_t* out;
   int32_t* acc_out;
   int* status;
+  int32_t* ws;     // split-K: raw partial accumulators [splits][M][N], else nullptr
   int M, N, K, b, k;
   int log2k;       // log2(k) when the word path is usable, else -1
   int SS;          // sparse K steps per tile (static positions through TMA), else 0
+  int splits;      // split-K: work items per output tile (each walks KS dense K steps), else 1
+  int KS;          // dense K steps per work item
   // work list: `n_pairs` tiles of two sub-tiles per CTA followed by `n_singles` tiles of one;
   // a row unit is 128 rows per CTA of the pair (128 or 256 rows)
   int n_pairs, n_singles, n_split;  // n_split: singles that come from cutting pair tiles in two
@@ -136,13 +139,16 @@ struct GemmParams {
 struct Tile {
   int m0, n0, nsub;  // first row of THIS CTA, first output channel of the tile, sub-tiles per CTA
   int nb0;           // first weight row THIS CTA loads and widens
+  int split, k0;     // split-K: which part of K this work item covers and its first K step
+  int ss;            // sparse K steps of this work item (the first part of K takes them all)
 };
 
 // Entry j of the work list (identical in every role of both CTAs of a pair, up to the rank).
-template <int PAIR>
+template <int PAIR, bool SPLITK>
 __device__ __forceinline__ Tile tile_of(const GemmParams& p, int j, int rank) {
   constexpr int U = BM * PAIR;  // rows of a row unit
   Tile t;
+  t.split = 0;
   if (j < p.n_pairs) {
     t.m0 = (j % p.mp) * (2 * U);
     t.n0 = (j / p.mp) * BN;
@@ -154,13 +160,21 @@ __device__ __forceinline__ Tile tile_of(const GemmParams& p, int j, int rank) {
       const int pj = p.n_pairs + s / 2;
       t.m0 = (pj % p.mp) * (2 * U) + (s & 1) * U;
       t.n0 = (pj / p.mp) * BN;
-    } else {  // the odd last row unit
+    } else {  // the odd last row unit (with split-K: `splits` work items per column tile)
+      const int q = s - p.n_split;
       t.m0 = (p.mu - 1) * U;
-      t.n0 = (s - p.n_split) * BN;
+      if (SPLITK) {
+        t.n0 = (q % p.tiles_n) * BN;
+        t.split = q / p.tiles_n;
+      } else {
+        t.n0 = q * BN;
+      }
     }
   }
   t.m0 += rank * t.nsub * BM;
   t.nb0 = t.n0 + rank * (BN / PAIR);
+  t.k0 = SPLITK ? t.split * p.KS : 0;
+  t.ss = (!SPLITK || t.split == 0) ? p.SS : 0;
   return t;
 }
 
@@ -227,7 +241,7 @@ __device__ __forceinline__ bool wait_leader(uint32_t bar, uint32_t parity, volat
 //                   merges one row of the 32 its warp has just widened -- no hand-over to
 //                   other warps, eight warps share the work
 constexpr int kModeMergeEpi = 0, kModeTma = 1, kModeMergeProd = 2;
-template <int PAIR, int MODE>
+template <int PAIR, int MODE, bool SPLITK>
 __global__ void __launch_bounds__(kThreads, 1)
     gemm_kernel(const GemmParams p, const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                 const __grid_constant__ CUtensorMap map_a4, const __grid_constant__ CUtensorMap map_b4) {
@@ -275,9 +289,8 @@ __global__ void __launch_bounds__(kThreads, 1)
 #define rank ((int)blockIdx.x % PAIR)
 #define cl ((int)blockIdx.x / PAIR)
 #define ncl ((int)gridDim.x / PAIR)
-  const int KS = p.K / BK;
+  const int KS = SPLITK ? p.KS : p.K / BK;  // dense K steps of a work item (all of K unless split)
   const int nwork = p.n_pairs + p.n_singles;
-  const int SS = STMA ? p.SS : 0;  // sparse K steps that follow the KS dense steps of every tile
 
   if (tid == 0) {
     for (int s = 0; s < NS; ++s) {
@@ -330,7 +343,17 @@ __global__ void __launch_bounds__(kThreads, 1)
       tmem_ld32(tmem + ((uint32_t)(32 * q) << 16) + (uint32_t)(sub * BN + c0), v);
       tmem_ld_wait();
       const int n0 = t.n0 + c0;
-      if (m < p.M && n0 < p.N) {
+      if (SPLITK) {
+        // split-K: this work item's raw partial sums; splitk_finish_kernel adds the parts
+        if (m < p.M) {
+          int32_t* wrow = p.ws + ((size_t)t.split * p.M + m) * p.N + n0;
+          for (int c8 = 0; c8 < 32 && n0 + c8 < p.N; c8 += 8) {
+            int4* dst = reinterpret_cast<int4*>(wrow + c8);
+            dst[0] = make_int4((int)v[c8], (int)v[c8 + 1], (int)v[c8 + 2], (int)v[c8 + 3]);
+            dst[1] = make_int4((int)v[c8 + 4], (int)v[c8 + 5], (int)v[c8 + 6], (int)v[c8 + 7]);
+          }
+        }
+      } else if (m < p.M && n0 < p.N) {
 #pragma unroll
         for (int c8 = 0; c8 < 32; c8 += 8) {
           if (n0 + c8 < p.N) {  // N % 8 == 0: a group of 8 columns is all in or all out
@@ -389,7 +412,7 @@ __global__ void __launch_bounds__(kThreads, 1)
       poff[i] = 0;
     }
     int pj = cl, pks = 0;  // work-list entry and K step being processed
-    Tile pt = tile_of<PAIR>(p, pj, rank);
+    Tile pt = tile_of<PAIR, SPLITK>(p, pj, rank);
     // producer-side merge (PMERGE): lane l of the warp owns row 32 * pw + l of the stage and
     // keeps that row's 16 sparse values and positions of the coming K step in registers
     const int GKp = (p.K / p.b) * p.k;
@@ -413,15 +436,18 @@ __global__ void __launch_bounds__(kThreads, 1)
                    : "=r"(nri.x), "=r"(nri.y), "=r"(nri.z), "=r"(nri.w)
                    : "l"(ip));
     };
-    if (PMERGE && cl < nwork) sparse_fetch(pt, 0);
+    if (PMERGE && cl < nwork) sparse_fetch(pt, pt.k0);
     auto process = [&]() -> bool {
       const bool has_a = pt.nsub == 2 || pw < kProdWarps / 2;  // a single-sub-tile entry only has A rows 0..127
       uint4 crv, cri;
       if (PMERGE) {
         crv = nrv;
         cri = nri;
-        if (pks + 1 < KS) sparse_fetch(pt, pks + 1);
-        else if (pj + ncl < nwork) sparse_fetch(tile_of<PAIR>(p, pj + ncl, rank), 0);
+        if (pks + 1 < KS) sparse_fetch(pt, pt.k0 + pks + 1);
+        else if (pj + ncl < nwork) {
+          const Tile nt = tile_of<PAIR, SPLITK>(p, pj + ncl, rank);
+          sparse_fetch(nt, nt.k0);
+        }
       }
       // ---- packed operands: wait for the TMA tiles, pull this thread's chunks into registers,
       //      hand the packed stage back
@@ -508,8 +534,9 @@ __global__ void __launch_bounds__(kThreads, 1)
       ++it;
       if (++pks == KS) {
         pks = 0;
+        const int SS = STMA ? pt.ss : 0;  // sparse K steps of the work item just finished
         pj += ncl;
-        if (pj < nwork) pt = tile_of<PAIR>(p, pj, rank);
+        if (pj < nwork) pt = tile_of<PAIR, SPLITK>(p, pj, rank);
         // The sparse K steps of the tile use the next SS ring slots (TMA fills them).  They are
         // waited for one by one, not skipped: a parity wait only tells the current phase from
         // the previous one, so no role may fall more than one use behind on any stage.
@@ -530,11 +557,11 @@ __global__ void __launch_bounds__(kThreads, 1)
       for (int ks = 0; ks < KS && ok; ++ks) {
         ok = process();
         if (kProducersJoinEpilogue && ok && ks == join_step && ti > 0)
-          ok = epilogue_share(tile_of<PAIR>(p, cl + (ti - 1) * ncl, rank), (uint32_t)(ti - 1), pw >> 2);
+          ok = epilogue_share(tile_of<PAIR, SPLITK>(p, cl + (ti - 1) * ncl, rank), (uint32_t)(ti - 1), pw >> 2);
       }
     }
     if (kProducersJoinEpilogue && ok)
-      epilogue_share(tile_of<PAIR>(p, cl + (my_tiles - 1) * ncl, rank), (uint32_t)(my_tiles - 1), pw >> 2);
+      epilogue_share(tile_of<PAIR, SPLITK>(p, cl + (my_tiles - 1) * ncl, rank), (uint32_t)(my_tiles - 1), pw >> 2);
   } else if (warp == kMmaWarp) {
     // =============================================================== MMA issuer
     // (the leader CTA's; the peer's MMA warp only holds its half of the tensor-memory allocation)
@@ -545,7 +572,9 @@ __global__ void __launch_bounds__(kThreads, 1)
       uint32_t ph_dense = 0, ph_sparse = 0;  // per-stage phase bits of the two kinds of "full" barrier
       bool ok = true;
       for (int j = cl; j < nwork && ok; j += ncl, ++tc) {
-        const int nsub = tile_of<PAIR>(p, j, rank).nsub;
+        const Tile mt = tile_of<PAIR, SPLITK>(p, j, rank);
+        const int nsub = mt.nsub;
+        const int SS = STMA ? mt.ss : 0;
         ok = wait_leader<PAIR>(bar_tempty, (tc & 1u) ^ 1u, abort_flag);  // previous tile's accumulators read out (both CTAs)
         if (!ok) break;
         tc_fence_after();
@@ -582,15 +611,15 @@ __global__ void __launch_bounds__(kThreads, 1)
       uint32_t pit = 0;
       bool ok = true;
       for (int j = cl; j < nwork && ok; j += ncl) {
-        const Tile t = tile_of<PAIR>(p, j, rank);
+        const Tile t = tile_of<PAIR, SPLITK>(p, j, rank);
         for (int ks = 0; ks < KS && ok; ++ks, ++pit) {
           const int ps = pit % NP;
           ok = mbar_wait(bar_pempty + 8 * ps, ((pit / NP) & 1u) ^ 1u, abort_flag);
           if (!ok) break;
           // rows past M / N come back as zeros (code 0)
           mbar_expect_tx(bar_pfull + 8 * ps, (uint32_t)(kPackA + kPackB));
-          tma_load_2d(smem_u32(sPA + ps * kPackA), &map_a4, ks * (BK / 2), t.m0, bar_pfull + 8 * ps);
-          tma_load_2d(smem_u32(sPB + ps * kPackB), &map_b4, ks * (BK / 2), t.nb0, bar_pfull + 8 * ps);
+          tma_load_2d(smem_u32(sPA + ps * kPackA), &map_a4, (t.k0 + ks) * (BK / 2), t.m0, bar_pfull + 8 * ps);
+          tma_load_2d(smem_u32(sPB + ps * kPackB), &map_b4, (t.k0 + ks) * (BK / 2), t.nb0, bar_pfull + 8 * ps);
         }
       }
     }
@@ -617,7 +646,8 @@ __global__ void __launch_bounds__(kThreads, 1)
       };
       bool ok = true;
       for (int j = cl; j < nwork && ok; j += ncl) {
-        const Tile t = tile_of<PAIR>(p, j, rank);
+        const Tile t = tile_of<PAIR, SPLITK>(p, j, rank);
+        const int SS = t.ss;
         // every ring slot is waited for in order (see the producers); only the sparse ones are filled
         for (int step = 0; step < KS + SS && ok; ++step, ++it) {
           const int s = it % NS;
@@ -679,23 +709,23 @@ __global__ void __launch_bounds__(kThreads, 1)
       mv[jj] = mi[jj] = 0;
     }
     if (m_word_path && m_prefetch) {  // sparse words of the very first step
-      const Tile t0 = tile_of<PAIR>(p, cl, rank);
+      const Tile t0 = tile_of<PAIR, SPLITK>(p, cl, rank);
 #pragma unroll
       for (int jj = 0; jj < kMergeTasks; ++jj) {
         const int tt = et + 128 * jj;
         if (jj < m_ntask && (tt >> m_nw_log) < t0.nsub * BM) {
           const int m = min(t0.m0 + (tt >> m_nw_log), p.M - 1);
-          const uint32_t o = (uint32_t)m * (uint32_t)m_GK + 4 * (tt & ((1 << m_nw_log) - 1));
+          const uint32_t o = (uint32_t)m * (uint32_t)m_GK + (uint32_t)t0.k0 * (uint32_t)m_nb + 4 * (tt & ((1 << m_nw_log) - 1));
           mv[jj] = __ldg(reinterpret_cast<const uint32_t*>(p.vals + o));
           mi[jj] = p.idx != nullptr ? __ldg(reinterpret_cast<const uint32_t*>(p.idx + o))
-                                    : __ldg(reinterpret_cast<const uint32_t*>(p.pos + 4 * (tt & ((1 << m_nw_log) - 1))));
+                                    : __ldg(reinterpret_cast<const uint32_t*>(p.pos + t0.k0 * m_nb + 4 * (tt & ((1 << m_nw_log) - 1))));
         }
       }
     }
     uint32_t mit = 0;  // position in the ring of widened stages
     uint32_t tc = 0;
     for (int j = cl; j < nwork; j += ncl, ++tc) {
-      const Tile t = tile_of<PAIR>(p, j, rank);
+      const Tile t = tile_of<PAIR, SPLITK>(p, j, rank);
       // the tile's column constants are fetched while the main loop is still running
       for (int cc = et; cc < BN; cc += kEpiWarps * 32) {
         const int n = min(t.n0 + cc, p.N - 1);
@@ -724,17 +754,17 @@ __global__ void __launch_bounds__(kThreads, 1)
               nj += ncl;
             }
             if (nj < nwork) {
-              const Tile nt = nks == 0 ? tile_of<PAIR>(p, nj, rank) : t;
+              const Tile nt = nks == 0 ? tile_of<PAIR, SPLITK>(p, nj, rank) : t;
 #pragma unroll
               for (int jj = 0; jj < kMergeTasks; ++jj) {
                 const int tt = et + 128 * jj;
                 if (jj < m_ntask && (tt >> m_nw_log) < nt.nsub * BM) {
                   const int m = min(nt.m0 + (tt >> m_nw_log), p.M - 1);
-                  const uint32_t o = (uint32_t)m * (uint32_t)m_GK + (uint32_t)nks * (uint32_t)m_nb + 4 * (tt & ((1 << m_nw_log) - 1));
+                  const uint32_t o = (uint32_t)m * (uint32_t)m_GK + (uint32_t)(nt.k0 + nks) * (uint32_t)m_nb + 4 * (tt & ((1 << m_nw_log) - 1));
                   mv[jj] = __ldg(reinterpret_cast<const uint32_t*>(p.vals + o));
                   mi[jj] = p.idx != nullptr
                                ? __ldg(reinterpret_cast<const uint32_t*>(p.idx + o))
-                               : __ldg(reinterpret_cast<const uint32_t*>(p.pos + nks * m_nb + 4 * (tt & ((1 << m_nw_log) - 1))));
+                               : __ldg(reinterpret_cast<const uint32_t*>(p.pos + (nt.k0 + nks) * m_nb + 4 * (tt & ((1 << m_nw_log) - 1))));
                 }
               }
             }
@@ -759,10 +789,10 @@ __global__ void __launch_bounds__(kThreads, 1)
             for (int tt = et; tt < ((t.nsub * BM) << m_nw_log); tt += 128) {
               const int row = tt >> m_nw_log, q = tt & ((1 << m_nw_log) - 1);
               const int m = min(t.m0 + row, p.M - 1);
-              const uint32_t o = (uint32_t)m * (uint32_t)m_GK + (uint32_t)ks * (uint32_t)m_nb + 4 * q;
+              const uint32_t o = (uint32_t)m * (uint32_t)m_GK + (uint32_t)(t.k0 + ks) * (uint32_t)m_nb + 4 * q;
               const uint32_t vw = __ldg(reinterpret_cast<const uint32_t*>(p.vals + o));
               const uint32_t iw = p.idx != nullptr ? __ldg(reinterpret_cast<const uint32_t*>(p.idx + o))
-                                                   : __ldg(reinterpret_cast<const uint32_t*>(p.pos + ks * m_nb + 4 * q));
+                                                   : __ldg(reinterpret_cast<const uint32_t*>(p.pos + (t.k0 + ks) * m_nb + 4 * q));
               uint32_t b4 = 0;
 #pragma unroll
               for (int u = 0; u < 4; ++u) b4 |= (uint32_t)(((4 * q + u) >> p.log2k) * p.b) << (8 * u);
@@ -777,7 +807,7 @@ __global__ void __launch_bounds__(kThreads, 1)
               const int row = tt / m_nb, i = tt - row * m_nb;
               const int m = min(t.m0 + row, p.M - 1);
               const int bank = i / p.k, slot_i = i - bank * p.k;
-              const int g = ks * (BK / p.b) + bank;
+              const int g = (t.k0 + ks) * (BK / p.b) + bank;
               const size_t entry = (size_t)m * m_GK + (size_t)g * p.k + slot_i;
               const uint32_t local = p.idx != nullptr ? p.idx[entry] : p.pos[(size_t)g * p.k + slot_i];
               const uint32_t kp = (kpos1(local) + (uint32_t)(bank * p.b)) ^ (uint32_t)((row & 7) << 4);
@@ -807,9 +837,64 @@ __global__ void __launch_bounds__(kThreads, 1)
 #undef ncl
 }
 
+// Split-K, second kernel: out[m, n] from the `splits` raw partial sums of every accumulator
+// (the same integer and fp32 operations, in the same order, as the one-kernel epilogue).
+__global__ void __launch_bounds__(256) splitk_finish_kernel(const int32_t* __restrict__ ws, int splits, int M, int N,
+                                                            const int32_t* __restrict__ colsum,
+                                                            const float* __restrict__ s_hi,
+                                                            const float* __restrict__ s_w, uint16_t* __restrict__ out,
+                                                            int32_t* __restrict__ acc_out) {
+  const int64_t groups = (int64_t)M * (N / 8);
+  for (int64_t gidx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; gidx < groups;
+       gidx += (int64_t)gridDim.x * blockDim.x) {
+    const int m = (int)(gidx / (N / 8)), n = (int)(gidx % (N / 8)) * 8;
+    int v[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+    for (int sp = 0; sp < splits; ++sp) {
+      const int4* src = reinterpret_cast<const int4*>(ws + ((size_t)sp * M + m) * N + n);
+      const int4 a = src[0], b = src[1];
+      v[0] += a.x; v[1] += a.y; v[2] += a.z; v[3] += a.w;
+      v[4] += b.x; v[5] += b.y; v[6] += b.z; v[7] += b.w;
+    }
+    const float sh = s_hi[m];
+    int acc[8];
+    uint32_t o[4];
+#pragma unroll
+    for (int c = 0; c < 8; ++c) acc[c] = (v[c] - 2048 * colsum[n + c]) >> 4;
+#pragma unroll
+    for (int c = 0; c < 8; c += 2)
+      o[c >> 1] = pack_bf16x2(((float)acc[c] * sh) * s_w[n + c], ((float)acc[c + 1] * sh) * s_w[n + c + 1]);
+    *reinterpret_cast<uint4*>(out + (size_t)m * N + n) = make_uint4(o[0], o[1], o[2], o[3]);
+    if (acc_out != nullptr) {
+      int4* dst = reinterpret_cast<int4*>(acc_out + (size_t)m * N + n);
+      dst[0] = make_int4(acc[0], acc[1], acc[2], acc[3]);
+      dst[1] = make_int4(acc[4], acc[5], acc[6], acc[7]);
+    }
+  }
+}
+
+// Split-K (at most 128 rows): how many parts of K per output tile, given the workspace.  With
+// few rows a launch has only N/256 tiles and each walks all of K at about a microsecond per
+// step (cold weight rows), so K is cut into up to 8 parts that run on other SMs at the same time.
+static int choose_splits(int64_t M, int64_t N, int64_t K, int sms, size_t ws_bytes) {
+  if (M > BM) return 1;
+  const int64_t tiles_n = (N + BN - 1) / BN, ks = K / BK;
+  for (int sp = 8; sp >= 2; sp /= 2) {
+    if (tiles_n * sp <= sms && ks % sp == 0 && ks / sp >= 2 && (size_t)sp * M * N * 4 <= ws_bytes) return sp;
+  }
+  return 1;
+}
+
+size_t gemm_workspace_bytes(int64_t M, int64_t N, int64_t K) {
+  int dev = 0, sms = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return 0;
+  if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
+  const int sp = choose_splits(M, N, K, sms, ~(size_t)0);
+  return sp > 1 ? (size_t)sp * M * N * 4 : 0;
+}
+
 cudaError_t launch_gemm(int b, int k, const sq_encoded& A, const sq_weights& W,
                         const uint8_t* positions, int64_t M, int64_t N, int64_t K, uint16_t* out,
-                        int32_t* acc_out, int* status, cudaStream_t st) {
+                        int32_t* acc_out, int* status, void* workspace, size_t workspace_bytes, cudaStream_t st) {
   GemmParams p;
   p.dq4 = A.dq4;
   p.vals = A.vals;
@@ -876,9 +961,9 @@ cudaError_t launch_gemm(int b, int k, const sq_encoded& A, const sq_weights& W,
       qc.attrs = qa;
       qc.numAttrs = 1;
       int n = 0;
-      const void* fn = mode == kModeTma ? (const void*)gemm_kernel<2, kModeTma>
-                       : mode == kModeMergeProd ? (const void*)gemm_kernel<2, kModeMergeProd>
-                                                : (const void*)gemm_kernel<2, kModeMergeEpi>;
+      const void* fn = mode == kModeTma ? (const void*)gemm_kernel<2, kModeTma, false>
+                       : mode == kModeMergeProd ? (const void*)gemm_kernel<2, kModeMergeProd, false>
+                                                : (const void*)gemm_kernel<2, kModeMergeEpi, false>;
       err = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, Geo<2>::kSmemBytes);
       if (err == cudaSuccess) err = cudaOccupancyMaxActiveClusters(&n, fn, &qc);
       if (err != cudaSuccess) return err;
@@ -907,7 +992,19 @@ cudaError_t launch_gemm(int b, int k, const sq_encoded& A, const sq_weights& W,
   }
   p.n_pairs = (int)as_pairs;
   p.n_split = (int)(2 * (pair_tiles - as_pairs));
-  p.n_singles = p.n_split + (p.mu & 1) * p.tiles_n;
+  // split-K (one CTA per tile, at most 128 rows, caller-provided workspace)
+  p.splits = 1;
+  p.ws = nullptr;
+  p.KS = (int)(K / BK);
+  if (pair == 1 && workspace != nullptr) {
+    const int sp = choose_splits(M, N, K, sm_count[dev], workspace_bytes);
+    if (sp > 1) {
+      p.splits = sp;
+      p.ws = static_cast<int32_t*>(workspace);
+      p.KS = (int)(K / BK / sp);
+    }
+  }
+  p.n_singles = p.n_split + (p.mu & 1) * p.tiles_n * p.splits;
   const int64_t nwork = (int64_t)p.n_pairs + p.n_singles;
   const unsigned grid = (unsigned)(nwork < slots ? nwork : slots) * (unsigned)pair;
 
@@ -961,9 +1058,10 @@ cudaError_t launch_gemm(int b, int k, const sq_encoded& A, const sq_weights& W,
     p.SS = (int)((GK + BK - 1) / BK);
   }
 
-#define SQ_LAUNCH_GEMM(PAIR_, MODE_)                                                                        \
+#define SQ_LAUNCH_GEMM(PAIR_, MODE_, SPLIT_)                                                                \
   do {                                                                                                      \
-    err = cudaFuncSetAttribute(gemm_kernel<PAIR_, MODE_>, cudaFuncAttributeMaxDynamicSharedMemorySize,      \
+    err = cudaFuncSetAttribute(gemm_kernel<PAIR_, MODE_, SPLIT_>,                                           \
+                               cudaFuncAttributeMaxDynamicSharedMemorySize,                                 \
                                Geo<PAIR_>::kSmemBytes);                                                     \
     if (err != cudaSuccess) return err;                                                                     \
     cudaLaunchConfig_t lc;                                                                                  \
@@ -979,19 +1077,30 @@ cudaError_t launch_gemm(int b, int k, const sq_encoded& A, const sq_weights& W,
     lc.stream = st;                                                                                         \
     lc.attrs = la;                                                                                          \
     lc.numAttrs = (PAIR_ == 2) ? 1 : 0;                                                                     \
-    err = cudaLaunchKernelEx(&lc, gemm_kernel<PAIR_, MODE_>, p, map_a, map_b, map_a4, map_b4);              \
+    err = cudaLaunchKernelEx(&lc, gemm_kernel<PAIR_, MODE_, SPLIT_>, p, map_a, map_b, map_a4, map_b4);      \
     if (err != cudaSuccess) return err;                                                                     \
   } while (0)
   if (pair == 2) {
-    if (mode == kModeTma) SQ_LAUNCH_GEMM(2, kModeTma);
-    else if (mode == kModeMergeProd) SQ_LAUNCH_GEMM(2, kModeMergeProd);
-    else SQ_LAUNCH_GEMM(2, kModeMergeEpi);
+    if (mode == kModeTma) SQ_LAUNCH_GEMM(2, kModeTma, false);
+    else if (mode == kModeMergeProd) SQ_LAUNCH_GEMM(2, kModeMergeProd, false);
+    else SQ_LAUNCH_GEMM(2, kModeMergeEpi, false);
+  } else if (p.splits > 1) {
+    if (mode == kModeTma) SQ_LAUNCH_GEMM(1, kModeTma, true);
+    else if (mode == kModeMergeProd) SQ_LAUNCH_GEMM(1, kModeMergeProd, true);
+    else SQ_LAUNCH_GEMM(1, kModeMergeEpi, true);
   } else {
-    if (mode == kModeTma) SQ_LAUNCH_GEMM(1, kModeTma);
-    else if (mode == kModeMergeProd) SQ_LAUNCH_GEMM(1, kModeMergeProd);
-    else SQ_LAUNCH_GEMM(1, kModeMergeEpi);
+    if (mode == kModeTma) SQ_LAUNCH_GEMM(1, kModeTma, false);
+    else if (mode == kModeMergeProd) SQ_LAUNCH_GEMM(1, kModeMergeProd, false);
+    else SQ_LAUNCH_GEMM(1, kModeMergeEpi, false);
   }
 #undef SQ_LAUNCH_GEMM
+  if (p.splits > 1) {
+    const int64_t groups = M * (N / 8);
+    int64_t blocks = (groups + 255) / 256;
+    if (blocks > 8 * (int64_t)sm_count[dev]) blocks = 8 * (int64_t)sm_count[dev];
+    splitk_finish_kernel<<<(unsigned)blocks, 256, 0, st>>>(p.ws, p.splits, (int)M, (int)N, W.colsum, A.s_hi, W.s_w, out,
+                                                         acc_out);
+  }
   return cudaGetLastError();
 }
 

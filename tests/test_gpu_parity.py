@@ -266,3 +266,45 @@ def test_static_encode_row_slices_in_registers(K, b, k):
     enc = sq.sq_encode(fmt, X, pos)
     check_status()
     compare_encoded(enc, oracle.encode(b, k, _bits(X), pos_ref))
+
+
+# ----------------------------------------------------------------------------- few rows: split-K through a workspace
+
+@pytest.mark.parametrize("b,k,static", [
+    (64, 8, False),     # producers merge (k/b = 1/8)
+    (64, 16, False),    # epilogue warps merge, word path
+    (32, 1, False),     # epilogue warps merge, byte path
+    (128, 16, True),    # TMA-fed sparse K steps (the first part of K takes them all)
+    (64, 4, True),
+])
+@pytest.mark.parametrize("M,K", [(1, 1024), (64, 2048), (128, 1536), (17, 4096)])
+def test_split_k_with_workspace(b, k, static, M, K):
+    """sq_gemm_ws with a workspace (K cut into parts + finishing kernel) against the oracle and,
+    bit for bit, against the call without a workspace."""
+    N = 520                       # three column tiles, the last one ragged
+    fmt = sq.make_format(b, k, static)
+    X = gen.activations(M, K, seed=M + K, outlier_fraction=0.01, outlier_scale=20.0, device="cuda")
+    W = gen.weights(N, K, seed=K, device="cuda")
+    pos = pos_ref = None
+    if static:
+        pos = sq.sq_calib_positions(fmt, gen.calibration_batch(64, K, seed=K, device="cuda"), W)
+        pos_ref = _np(pos)
+    w = sq.sq_pack_weights(fmt, W, pos)
+    enc = sq.sq_encode(fmt, X, pos)
+    need = sq.sq_gemm_workspace_bytes(fmt, M, N, K)
+    assert need > 0 and need % (M * N * 4) == 0 and need // (M * N * 4) in (2, 4, 8)
+    ws = torch.full((need,), 0xAB, dtype=torch.uint8, device="cuda")     # stale contents must not matter
+    acc = torch.empty(M, N, dtype=torch.int32, device="cuda")
+    out = sq.sq_gemm_ws(fmt, enc, w, pos, acc_out=acc, workspace=ws)
+    out_again = sq.sq_gemm_ws(fmt, enc, w, pos, workspace=ws).clone()
+    acc1 = torch.empty(M, N, dtype=torch.int32, device="cuda")
+    out1 = sq.sq_gemm_ws(fmt, enc, w, pos, acc_out=acc1, workspace=None)
+    small = sq.sq_gemm_ws(fmt, enc, w, pos, workspace=ws[: 2 * M * N * 4]).clone()   # room for two parts only
+    check_status()
+    assert torch.equal(acc, acc1) and torch.equal(out, out1) and torch.equal(out_again, out1) and torch.equal(small, out1)
+    enc_ref = oracle.encode(b, k, _bits(X), pos_ref)
+    w_ref = oracle.pack_weights(b, k, _bits(W), pos_ref)
+    acc_ref, ref32, out_ref = oracle.gemm(b, k, enc_ref, w_ref, pos_ref)
+    assert np.array_equal(_np(acc), acc_ref)
+    assert_bf16_close(out, ref32)
+    assert np.array_equal(_bits(out), out_ref)
