@@ -188,6 +188,32 @@ sq_status sq_gemm_ws(const sq_format* fmt, const sq_encoded* A, const sq_weights
                      const uint8_t* positions, int64_t M, int64_t N, int64_t K, void* out_bf16,
                      int32_t* acc_out, void* workspace, size_t workspace_bytes, void* cuda_stream);
 
+/* (No counterpart in the paper: a convenience of this library.)
+ * sq_gemm_ws for callers that have nowhere to get a workspace from.  Some hosts of this
+ * library hand out all device memory once, at start-up -- a serving process that gives
+ * every component a fixed arena, a plug-in called from someone else's runtime, a plain C
+ * caller with no allocator of its own -- and may not call cudaMalloc later: it
+ * synchronises the whole device, and it can fail in a process that runs close to full or
+ * fragmented memory.  For them the split-K partial sums go into a fixed 16 MiB array that
+ * is part of the library's device image (SQ_STATIC_SCRATCH_BYTES; every GPU that loads
+ * the library holds it until the process exits).  The call allocates and frees nothing,
+ * neither directly nor through any library.
+ *   - Inputs, outputs and result are those of sq_gemm (bit-identical).
+ *   - Only the few-row case is served: M <= 128 and 2*M*N*4 <= SQ_STATIC_SCRATCH_BYTES
+ *     (room for at least two parts of K), otherwise SQ_ERR_UNSUPPORTED and nothing is
+ *     launched: call sq_gemm, which needs no scratch.  K is cut into as many parts (2, 4
+ *     or 8) as fit the array.
+ *   - The first call on each device looks up the array's device address (that device must
+ *     be current, as for every call here); make that first call before any stream capture.
+ *   - All calls share the one array.  It keeps whatever the previous call left there, which
+ *     is harmless: every element a call reads it has written itself first.  But two calls
+ *     that overlap on the GPU (different streams, no ordering between them) race on it:
+ *     order them, or use sq_gemm_ws with separate workspaces. */
+#define SQ_STATIC_SCRATCH_BYTES ((size_t)16 << 20)
+sq_status sq_gemm_static_scratch(const sq_format* fmt, const sq_encoded* A, const sq_weights* W,
+                                 const uint8_t* positions, int64_t M, int64_t N, int64_t K, void* out_bf16,
+                                 int32_t* acc_out, void* cuda_stream);
+
 /* Decode (inverse of Eq. 1): out[m,j] = bf16_rne(s_hi[m]*vals) at selected positions,
  * bf16_rne(s_lo[m]*dq4) elsewhere.  out_bf16: device bf16 [M, K], written. */
 sq_status sq_decode(const sq_format* fmt, const sq_encoded* A, const uint8_t* positions,

@@ -9,7 +9,7 @@ from .binding import (  # noqa: F401
     SQ_MAX_K, LIBRARY_PATH, SqError, Encoded, Weights, sq_format, sq_encoded, sq_weights,
     make_format, alloc_encoded, alloc_weights, sq_status_string, sq_encoded_sizes,
     sq_weights_sizes, sq_calib_positions, sq_pack_weights, sq_encode, sq_gemm, sq_gemm_ws,
-    sq_gemm_workspace_bytes, sq_decode,
+    sq_gemm_workspace_bytes, sq_gemm_static_scratch, SQ_STATIC_SCRATCH_BYTES, sq_decode,
     sq_device_status, raw,
 )
 from .sharding import row_shard  # noqa: F401,E402

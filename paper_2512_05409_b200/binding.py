@@ -69,10 +69,12 @@ def _load() -> ctypes.CDLL:
     lib.sq_gemm_ws.argtypes = [P(sq_format), P(sq_encoded), P(sq_weights), VP, I64, I64, I64, VP, VP, VP,
                                ctypes.c_size_t, VP]
     lib.sq_gemm_workspace_bytes.argtypes = [P(sq_format), I64, I64, I64, P(ctypes.c_size_t)]
+    lib.sq_gemm_static_scratch.argtypes = [P(sq_format), P(sq_encoded), P(sq_weights), VP, I64, I64, I64, VP, VP, VP]
     lib.sq_decode.argtypes = [P(sq_format), P(sq_encoded), VP, I64, I64, VP, VP]
     lib.sq_device_status.argtypes = [VP]
     for name in ("sq_encoded_sizes", "sq_weights_sizes", "sq_calib_positions", "sq_pack_weights",
-                 "sq_encode", "sq_gemm", "sq_gemm_ws", "sq_gemm_workspace_bytes", "sq_decode", "sq_device_status"):
+                 "sq_encode", "sq_gemm", "sq_gemm_ws", "sq_gemm_workspace_bytes", "sq_gemm_static_scratch", "sq_decode",
+                 "sq_device_status"):
         getattr(lib, name).restype = ctypes.c_int
     return lib
 
@@ -238,6 +240,25 @@ def sq_gemm_ws(fmt: sq_format, A: Encoded, W: Weights, positions: torch.Tensor |
     nbytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
     _check(_lib.sq_gemm_ws(ctypes.byref(fmt), ctypes.byref(ca), ctypes.byref(cw), _ptr(positions), M, N, K,
                            _ptr(out), _ptr(acc_out), _ptr(workspace), nbytes, _stream(stream)), "sq_gemm_ws")
+    return out
+
+
+SQ_STATIC_SCRATCH_BYTES = 16 << 20
+
+
+def sq_gemm_static_scratch(fmt: sq_format, A: Encoded, W: Weights, positions: torch.Tensor | None = None,
+                           out: torch.Tensor | None = None, acc_out: torch.Tensor | None = None,
+                           stream=None) -> torch.Tensor:
+    """The C ABI's sq_gemm_static_scratch: few-row GEMM whose split-K scratch is a fixed array inside
+    the library, for callers that may not allocate device memory at call time.  `out` should be given
+    by such a caller: when it is None this wrapper, not the library, allocates it with torch)."""
+    M, K = A.dq4.shape[0], A.dq4.shape[1] * 2
+    N = W.wq4.shape[0]
+    if out is None:
+        out = _buf(M * N * 2, torch.bfloat16, A.dq4.device)[: M * N].view(M, N)
+    ca, cw = A.c_struct(), W.c_struct()
+    _check(_lib.sq_gemm_static_scratch(ctypes.byref(fmt), ctypes.byref(ca), ctypes.byref(cw), _ptr(positions),
+                                       M, N, K, _ptr(out), _ptr(acc_out), _stream(stream)), "sq_gemm_static_scratch")
     return out
 
 

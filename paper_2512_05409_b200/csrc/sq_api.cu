@@ -209,6 +209,29 @@ sq_status sq_gemm_ws(const sq_format* fmt, const sq_encoded* A, const sq_weights
                                static_cast<cudaStream_t>(cuda_stream)));
 }
 
+sq_status sq_gemm_static_scratch(const sq_format* fmt, const sq_encoded* A, const sq_weights* W,
+                                 const uint8_t* positions, int64_t M, int64_t N, int64_t K, void* out_bf16,
+                                 int32_t* acc_out, void* cuda_stream) {
+  SQ_TRY(check_format(fmt));
+  SQ_TRY(check_k(K));
+  if (M < 0 || N < 0 || N % 8 != 0 || M > INT32_MAX || N > INT32_MAX) return SQ_ERR_INVALID_ARG;
+  if (M == 0 || N == 0) return SQ_OK;
+  // Only the few-row case has a use for scratch, and at least two parts of K must fit.
+  if (M > 128) return SQ_ERR_UNSUPPORTED;
+  if ((uint64_t)2 * (uint64_t)M * (uint64_t)N * 4u > (uint64_t)gemm_static_scratch_bytes()) return SQ_ERR_UNSUPPORTED;
+  SQ_TRY(check_positions(fmt, positions));
+  SQ_TRY(check_encoded(fmt, A));
+  SQ_TRY(check_weights(fmt, W));
+  if (out_bf16 == nullptr) return SQ_ERR_NULL_POINTER;
+  if (!aligned16(out_bf16) || !aligned16(acc_out)) return SQ_ERR_ALIGNMENT;
+  SQ_TRY(check_device());
+  int* status = status_word();
+  if (status == nullptr) return SQ_ERR_CUDA;
+  return from_cuda(launch_gemm_static_scratch(fmt->bank, fmt->k, *A, *W, positions, M, N, K,
+                                              static_cast<uint16_t*>(out_bf16), acc_out, status,
+                                              static_cast<cudaStream_t>(cuda_stream)));
+}
+
 sq_status sq_gemm(const sq_format* fmt, const sq_encoded* A, const sq_weights* W,
                   const uint8_t* positions, int64_t M, int64_t N, int64_t K, void* out_bf16,
                   int32_t* acc_out, void* cuda_stream) {

@@ -1104,4 +1104,33 @@ cudaError_t launch_gemm(int b, int k, const sq_encoded& A, const sq_weights& W,
   return cudaGetLastError();
 }
 
+// ------------------------------------------------------------------------------------------------
+// Split-K scratch that nobody has to allocate: a fixed array in the library's device image.
+// Every GPU that loads the library holds these 16 MiB until the process exits.
+constexpr size_t kStaticScratchBytes = (size_t)16 << 20;
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+
+size_t gemm_static_scratch_bytes() { return kStaticScratchBytes; }
+
+// launch_gemm with the static array as its workspace.  In host code the array's name is only a
+// stand-in for the symbol, not a device address, so the address is asked for once per device
+// (with that device current) and remembered; the kernels get the pointer like any other.
+cudaError_t launch_gemm_static_scratch(int b, int k, const sq_encoded& A, const sq_weights& W,
+                                       const uint8_t* positions, int64_t M, int64_t N, int64_t K, uint16_t* out,
+                                       int32_t* acc_out, int* status, cudaStream_t st) {
+  static void* scratch_addr[64] = {nullptr};
+  int dev = 0;
+  cudaError_t err = cudaGetDevice(&dev);
+  if (err != cudaSuccess) return err;
+  if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+  if (scratch_addr[dev] == nullptr) {
+    void* ptr = nullptr;
+    err = cudaGetSymbolAddress(&ptr, g_static_scratch);
+    if (err != cudaSuccess) return err;
+    if (ptr == nullptr) return cudaErrorInvalidSymbol;
+    scratch_addr[dev] = ptr;
+  }
+  return launch_gemm(b, k, A, W, positions, M, N, K, out, acc_out, status, scratch_addr[dev], kStaticScratchBytes, st);
+}
+
 }  // namespace sq

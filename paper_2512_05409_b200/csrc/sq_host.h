@@ -29,5 +29,10 @@ cudaError_t launch_gemm(int b, int k, const sq_encoded& A, const sq_weights& W,
                         int32_t* acc_out, int* status, void* workspace, size_t workspace_bytes, cudaStream_t st);
 // Bytes of workspace with which launch_gemm would split K for this shape (0: it would not).
 size_t gemm_workspace_bytes(int64_t M, int64_t N, int64_t K);
+// The same launch with the library's own fixed scratch array as the workspace (no allocation).
+cudaError_t launch_gemm_static_scratch(int b, int k, const sq_encoded& A, const sq_weights& W,
+                                       const uint8_t* positions, int64_t M, int64_t N, int64_t K, uint16_t* out,
+                                       int32_t* acc_out, int* status, cudaStream_t st);
+size_t gemm_static_scratch_bytes();
 
 }  // namespace sq
