@@ -50,14 +50,20 @@
 //   warp  13    one thread streams the packed 4-bit tiles (256 rows x 64 B of A, 256 or 128 rows
 //               of B per K step) into a ring of NP packed stages by TMA
 //   warps 0-7   producers: read their chunks of a packed stage, widen them, store the
-//               swizzled 8-bit layout into a ring of NS widened stages
-//   warps 9-12  dynamic positions: merge the sparse INT8 entries into each widened A stage
-//               (byte stores, four positions per SWAR step) before it goes to the MMA thread;
-//               for every tile: epilogue (tcgen05.ld, dequantise, bf16, 16-byte stores)
+//               swizzled 8-bit layout into a ring of NS widened stages; dynamic positions with
+//               16 sparse entries per row and K step: each thread then merges the sparse INT8
+//               entries of one of the 32 rows its warp has just written (byte stores, four
+//               positions per SWAR step)
+//   warps 9-12  for every tile: epilogue (tcgen05.ld, dequantise, bf16, 16-byte stores);
+//               dynamic positions in the other formats: they do the merge, between the
+//               producers and the MMA thread
 //   warp  8     one thread issues the MMAs and commits stage / accumulator barriers
 //   warp  14    static positions: one thread issues the TMA loads of the sparse K steps
 // Every wait is bounded; a wait that runs out raises an abort flag that releases all
 // other waits, the kernel records SQ_ERR_TIMEOUT and frees its tensor memory.
+//
+// Few rows (at most 128): a launch has only N/256 tiles, so given a workspace K is cut into
+// parts (work item = column tile x part of K) whose raw partial sums a second kernel adds.
 #include <cuda.h>
 #include <cudaTypedefs.h>
 #include <string.h>
