@@ -91,3 +91,29 @@ def test_zero_sized_problems_are_no_ops():
     assert lib.sq_gemm(ctypes.byref(f), ctypes.byref(enc), ctypes.byref(w), None, 0, 16, 128, 0x8000, None,
                        None) == sq.SQ_OK
     assert lib.sq_decode(ctypes.byref(f), ctypes.byref(enc), None, 0, 128, 0x8000, None) == sq.SQ_OK
+
+
+def test_workspace_entry_points_validate_without_a_device():
+    lib = sq.raw()
+    f = sq.make_format(64, 8, False)
+    enc = sq.sq_encoded(0x1000, 0x2000, 0x3000, 0x4000, 0x5000, 0x6000)
+    w = sq.sq_weights(0x1000, 0x2000, 0x3000, None)
+    need = ctypes.c_size_t(123)
+    assert lib.sq_gemm_workspace_bytes(ctypes.byref(f), 0, 4096, 4096, ctypes.byref(need)) == sq.SQ_OK
+    assert need.value == 0                                                   # nothing to do, nothing needed
+    assert lib.sq_gemm_workspace_bytes(ctypes.byref(f), 16, 4096, 4096, None) == sq.SQ_ERR_NULL_POINTER
+    assert lib.sq_gemm_workspace_bytes(ctypes.byref(f), 16, 12, 4096, ctypes.byref(need)) == sq.SQ_ERR_INVALID_ARG
+    assert lib.sq_gemm_workspace_bytes(ctypes.byref(f), 16, 4096, 100, ctypes.byref(need)) == sq.SQ_ERR_INVALID_ARG
+    # sq_gemm_ws: a misaligned workspace is an argument error, a zero-sized problem is a no-op
+    assert lib.sq_gemm_ws(ctypes.byref(f), ctypes.byref(enc), ctypes.byref(w), None, 4, 16, 128, 0x8000, None,
+                          0x9004, 4096, None) == sq.SQ_ERR_ALIGNMENT
+    assert lib.sq_gemm_ws(ctypes.byref(f), ctypes.byref(enc), ctypes.byref(w), None, 0, 16, 128, 0x8000, None,
+                          0x9000, 4096, None) == sq.SQ_OK
+    # sq_gemm_static_scratch: sizes beyond its fixed array are refused before anything else is looked at
+    assert lib.sq_gemm_static_scratch(ctypes.byref(f), ctypes.byref(enc), ctypes.byref(w), None, 129, 16, 128,
+                                      0x8000, None, None) == sq.SQ_ERR_UNSUPPORTED
+    assert lib.sq_gemm_static_scratch(ctypes.byref(f), ctypes.byref(enc), ctypes.byref(w), None, 128, 16392, 128,
+                                      0x8000, None, None) == sq.SQ_ERR_UNSUPPORTED
+    assert lib.sq_gemm_static_scratch(ctypes.byref(f), ctypes.byref(enc), ctypes.byref(w), None, 0, 16, 128,
+                                      0x8000, None, None) == sq.SQ_OK
+    assert sq.SQ_STATIC_SCRATCH_BYTES == 16 << 20
