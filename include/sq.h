@@ -172,14 +172,16 @@ sq_status sq_gemm(const sq_format* fmt, const sq_encoded* A, const sq_weights* W
                   const uint8_t* positions, int64_t M, int64_t N, int64_t K, void* out_bf16,
                   int32_t* acc_out, void* cuda_stream);
 
-/* The same product (Section 3.3) with a caller-owned workspace, for the decode-shaped case
- * of few tokens (M <= 128): a launch then has only N/256 output tiles, each walking all of
- * K, so most SMs idle.  Given a workspace the call may cut K into up to 8 parts that run
- * on different SMs, leave their raw int32 partial sums in the workspace ([parts][M][N]) and
- * add them up in a second kernel on the same stream.  The result is bit-identical to
- * sq_gemm's (integer partial sums, the same epilogue operations in the same order).
- * sq_gemm_workspace_bytes: *bytes = the size with which this shape would be split, 0 if it
- * would not be (M > 128, too many tiles already, or too few K steps).
+/* The same product (Section 3.3) with a caller-owned workspace.  The result is bit-identical
+ * to sq_gemm's; the workspace only buys speed, in two cases:
+ *   - few tokens (M <= 128, decode-shaped): a launch has only N/256 output tiles, each walking
+ *     all of K, so most SMs idle.  K is cut into up to 8 parts that run on different SMs,
+ *     their raw int32 partial sums go to the workspace ([parts][M][N]) and a second kernel on
+ *     the same stream adds them and runs the epilogue;
+ *   - more tokens with dynamic positions: the activations are expanded once into merged 8-bit
+ *     tensor-core operands ([M][K] bytes in the workspace) instead of being widened and
+ *     merged again for every tile of output channels.
+ * sq_gemm_workspace_bytes: *bytes = the size this shape and format can make use of, 0 if none.
  * workspace: device memory, 16-byte aligned, or NULL (= sq_gemm); a smaller workspace than
  * asked for is used for fewer parts or not at all, never an error.  Its contents are
  * undefined afterwards; calls that share a workspace must not overlap on the GPU. */

@@ -184,7 +184,7 @@ sq_status sq_gemm_workspace_bytes(const sq_format* fmt, int64_t M, int64_t N, in
   *bytes = 0;
   if (M == 0 || N == 0) return SQ_OK;
   SQ_TRY(check_device());
-  *bytes = gemm_workspace_bytes(M, N, K);
+  *bytes = gemm_workspace_bytes(fmt->pos_mode == SQ_POS_STATIC, M, N, K);
   return SQ_OK;
 }
 

@@ -246,13 +246,19 @@ __device__ __forceinline__ bool wait_leader(uint32_t bar, uint32_t parity, volat
 //   kModeMergeProd  16 sparse entries per row and K step (k/b = 1/8): every producer thread
 //                   merges one row of the 32 its warp has just widened -- no hand-over to
 //                   other warps, eight warps share the work
-constexpr int kModeMergeEpi = 0, kModeTma = 1, kModeMergeProd = 2;
+//   kModeA8         the caller gave a workspace of M*K bytes: expand_a8_kernel has written the
+//                   activations there as merged 8-bit operands (dense part widened, sparse
+//                   entries in place, K order of the MMA blocks), once per row instead of once
+//                   per row AND column tile; TMA brings those tiles straight into the widened
+//                   ring and the producers widen only the weights.  No sparse K steps either.
+constexpr int kModeMergeEpi = 0, kModeTma = 1, kModeMergeProd = 2, kModeA8 = 3;
 template <int PAIR, int MODE, bool SPLITK>
 __global__ void __launch_bounds__(kThreads, 1)
     gemm_kernel(const GemmParams p, const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                 const __grid_constant__ CUtensorMap map_a4, const __grid_constant__ CUtensorMap map_b4) {
   using G = Geo<PAIR>;
-  constexpr bool STMA = MODE == kModeTma, PMERGE = MODE == kModeMergeProd;
+  constexpr bool STMA = MODE == kModeTma, PMERGE = MODE == kModeMergeProd, A8 = MODE == kModeA8;
+  constexpr bool ATMA = STMA || A8;  // the second TMA thread fills (some or all) A stages
   constexpr int NS = G::NS, NP = G::NP;
   constexpr int kStageB = G::kStageB, kPackB = G::kPackB, kBTasks = G::kBTasks;
   // The kernel has no static shared memory, so the dynamic block starts at the 1024-byte
@@ -303,7 +309,7 @@ __global__ void __launch_bounds__(kThreads, 1)
       // Every thread arrives for itself right after its own proxy fence (one arrival per warp
       // behind a __syncwarp was measured slower).  Static positions: the producers complete a
       // dense stage; otherwise the merge warps do.
-      mbar_init(bar_full + 8 * s, PAIR * ((STMA || PMERGE) ? kProdWarps : kEpiWarps) * 32);
+      mbar_init(bar_full + 8 * s, PAIR * ((STMA || PMERGE || A8) ? kProdWarps : kEpiWarps) * 32);
       mbar_init(bar_wfull + 8 * s, kProdWarps * 32);
       mbar_init(bar_empty + 8 * s, 1);
       mbar_init(bar_sfull + 8 * s, 1);
@@ -444,7 +450,8 @@ __global__ void __launch_bounds__(kThreads, 1)
     };
     if (PMERGE && cl < nwork) sparse_fetch(pt, pt.k0);
     auto process = [&]() -> bool {
-      const bool has_a = pt.nsub == 2 || pw < kProdWarps / 2;  // a single-sub-tile entry only has A rows 0..127
+      // a single-sub-tile entry only has A rows 0..127; with pre-widened activations there is no A work at all
+      const bool has_a = !A8 && (pt.nsub == 2 || pw < kProdWarps / 2);
       uint4 crv, cri;
       if (PMERGE) {
         crv = nrv;
@@ -535,7 +542,7 @@ __global__ void __launch_bounds__(kThreads, 1)
       // them; after the widening every loaded register has been consumed.
       mbar_arrive(bar_pempty + 8 * ps);
       fence_proxy_async_smem();  // generic-proxy writes -> visible to the tensor core's async reads
-      if (STMA || PMERGE) arrive_leader<PAIR>(bar_full + 8 * s);
+      if (STMA || PMERGE || A8) arrive_leader<PAIR>(bar_full + 8 * s);
       else mbar_arrive(bar_wfull + 8 * s);  // dynamic positions: the merge warps take over
       ++it;
       if (++pks == KS) {
@@ -590,6 +597,11 @@ __global__ void __launch_bounds__(kThreads, 1)
           if (!sparse_step) {
             ok = wait_leader<PAIR>(bar_full + 8 * s, (ph_dense >> s) & 1u, abort_flag);
             ph_dense ^= 1u << s;
+            if (A8) {  // ... and the activation tiles TMA delivers (both CTAs')
+              if (ok) ok = mbar_wait(bar_sfull + 8 * s, (ph_sparse >> s) & 1u, abort_flag);
+              if (ok && PAIR == 2) ok = wait_leader<PAIR>(bar_sfullp + 8 * s, (ph_sparse >> s) & 1u, abort_flag);
+              ph_sparse ^= 1u << s;
+            }
           } else {
             ok = mbar_wait(bar_sfull + 8 * s, (ph_sparse >> s) & 1u, abort_flag);
             if (ok && PAIR == 2) ok = wait_leader<PAIR>(bar_sfullp + 8 * s, (ph_sparse >> s) & 1u, abort_flag);
@@ -623,16 +635,17 @@ __global__ void __launch_bounds__(kThreads, 1)
           ok = mbar_wait(bar_pempty + 8 * ps, ((pit / NP) & 1u) ^ 1u, abort_flag);
           if (!ok) break;
           // rows past M / N come back as zeros (code 0)
-          mbar_expect_tx(bar_pfull + 8 * ps, (uint32_t)(kPackA + kPackB));
-          tma_load_2d(smem_u32(sPA + ps * kPackA), &map_a4, (t.k0 + ks) * (BK / 2), t.m0, bar_pfull + 8 * ps);
+          mbar_expect_tx(bar_pfull + 8 * ps, (uint32_t)((A8 ? 0 : kPackA) + kPackB));
+          if (!A8) tma_load_2d(smem_u32(sPA + ps * kPackA), &map_a4, (t.k0 + ks) * (BK / 2), t.m0, bar_pfull + 8 * ps);
           tma_load_2d(smem_u32(sPB + ps * kPackB), &map_b4, (t.k0 + ks) * (BK / 2), t.nb0, bar_pfull + 8 * ps);
         }
       }
     }
     __syncwarp();
   } else if (warp == kTmaSparseWarp) {
-    // =============================================================== TMA: sparse K steps
-    if (STMA && lane == 0) {
+    // =============================================================== TMA: sparse K steps, or every
+    // step's pre-widened activation tile
+    if (ATMA && lane == 0) {
       uint32_t it = 0;
       // The leader's MMA thread cannot watch the peer's barriers, so the peer's thread tells it
       // when each of its tiles has landed.  It does so while waiting for the next free slot
@@ -653,7 +666,7 @@ __global__ void __launch_bounds__(kThreads, 1)
       bool ok = true;
       for (int j = cl; j < nwork && ok; j += ncl) {
         const Tile t = tile_of<PAIR, SPLITK>(p, j, rank);
-        const int SS = t.ss;
+        const int SS = STMA ? t.ss : 0;
         // every ring slot is waited for in order (see the producers); only the sparse ones are filled
         for (int step = 0; step < KS + SS && ok; ++step, ++it) {
           const int s = it % NS;
@@ -672,12 +685,19 @@ __global__ void __launch_bounds__(kThreads, 1)
             }
             if (!ok) *abort_flag = 1;
           }
-          if (!ok || step < KS) continue;
-          const int ss = step - KS;
-          // rows past M / N and columns past G*k are filled with zeros by the TMA unit
-          mbar_expect_tx(bar_sfull + 8 * s, (uint32_t)(kStageA + kStageB));
-          tma_load_2d(smem_u32(sA + s * kStageA), &map_a, ss * BK, t.m0, bar_sfull + 8 * s);
-          tma_load_2d(smem_u32(sB + s * kStageB), &map_b, ss * BK, t.nb0, bar_sfull + 8 * s);
+          if (!ok) continue;
+          if (A8) {
+            // the merged 8-bit activations of this K step (rows past M come back as zeros)
+            mbar_expect_tx(bar_sfull + 8 * s, (uint32_t)kStageA);
+            tma_load_2d(smem_u32(sA + s * kStageA), &map_a, (t.k0 + step) * BK, t.m0, bar_sfull + 8 * s);
+          } else {
+            if (step < KS) continue;
+            const int ss = step - KS;
+            // rows past M / N and columns past G*k are filled with zeros by the TMA unit
+            mbar_expect_tx(bar_sfull + 8 * s, (uint32_t)(kStageA + kStageB));
+            tma_load_2d(smem_u32(sA + s * kStageA), &map_a, ss * BK, t.m0, bar_sfull + 8 * s);
+            tma_load_2d(smem_u32(sB + s * kStageB), &map_b, ss * BK, t.nb0, bar_sfull + 8 * s);
+          }
           if (forwards) {
             fq[(fq_head + fq_n) % NS] = (uint32_t)s;
             ++fq_n;
@@ -698,7 +718,7 @@ __global__ void __launch_bounds__(kThreads, 1)
     // merge state (dynamic positions): word tasks tt = et + 128*jj -> (row tt / words-per-row, word)
     const int m_GK = (p.K / p.b) * p.k;
     const int m_nb = (BK / p.b) * p.k;  // sparse entries per row per K step
-    const bool m_word_path = !STMA && !PMERGE && p.log2k >= 0;
+    const bool m_word_path = !STMA && !PMERGE && !A8 && p.log2k >= 0;
     const int m_nw_log = m_word_path ? (31 - __clz(m_nb >> 2)) : 0;
     const int m_ntask = m_word_path ? (2 * BM << m_nw_log) / 128 : 0;  // per thread for a 256-row stage
     const bool m_prefetch = m_ntask <= kMergeTasks;
@@ -738,7 +758,7 @@ __global__ void __launch_bounds__(kThreads, 1)
         s_cs[cc] = 2048 * __ldg(p.colsum + n);
         s_sw[cc] = __ldg(p.s_w + n);
       }
-      if (!STMA && !PMERGE) {
+      if (!STMA && !PMERGE && !A8) {
         // ---- dynamic positions (or static ones TMA cannot fetch): these warps, idle until the
         //      tile's accumulators are complete, merge the sparse INT8 entries into every widened
         //      A stage and only then hand it to the MMA thread
@@ -843,6 +863,49 @@ __global__ void __launch_bounds__(kThreads, 1)
 #undef ncl
 }
 
+// Merged 8-bit activations for kModeA8: a8[m][j'] = the operand byte the producers would put into
+// the widened A stage (dense: offset-binary nibble * 2^e + bias; sparse: vals ^ 0x80), j' = the
+// position of element j in the MMA's K order ([16 even | 16 odd] per 32 elements).  One thread
+// per 32-element block: 16 packed bytes in, 32 operand bytes out, then the sparse entries of its
+// bank that fall into the block are patched in.
+__global__ void __launch_bounds__(256) expand_a8_kernel(const uint8_t* __restrict__ dq4, const int8_t* __restrict__ vals,
+                                                        const uint8_t* __restrict__ idx,
+                                                        const uint8_t* __restrict__ pos,
+                                                        const uint8_t* __restrict__ shift, int64_t M, int K, int b,
+                                                        int k, uint8_t* __restrict__ a8) {
+  const int blocks_per_row = K / 32;
+  const int64_t total = M * blocks_per_row;
+  const int GK = (K / b) * k;
+  for (int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; t < total; t += (int64_t)gridDim.x * blockDim.x) {
+    const int64_t m = t / blocks_per_row;
+    const int blk = (int)(t % blocks_per_row);  // elements 32*blk .. 32*blk+31 of the row
+    const uint32_t e = shift[m];
+    const uint32_t pmul = 1u << e, poff = 0x01010101u * (128u - (8u << e));
+    const uint4 in = *reinterpret_cast<const uint4*>(dq4 + m * (K / 2) + blk * 16);
+    const uint32_t w[4] = {in.x, in.y, in.z, in.w};
+    uint32_t o[8];  // bytes 0..15: even elements, 16..31: odd elements
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      const uint32_t u = w[q] ^ 0x88888888u;
+      o[q] = (u & 0x0F0F0F0Fu) * pmul + poff;
+      o[4 + q] = ((u >> 4) & 0x0F0F0F0Fu) * pmul + poff;
+    }
+    uint8_t* orow = a8 + m * K + blk * 32;
+    uint4* dst = reinterpret_cast<uint4*>(orow);
+    dst[0] = make_uint4(o[0], o[1], o[2], o[3]);
+    dst[1] = make_uint4(o[4], o[5], o[6], o[7]);
+    // sparse entries of the bank this block lies in: byte stores over what was just written (the
+    // same thread's later stores to the same bytes win)
+    const int g = (blk * 32) / b, off = (blk * 32) % b;  // bank, and the block's first element inside it
+    const int8_t* v = vals + m * GK + g * k;
+    const uint8_t* ix = idx != nullptr ? idx + m * GK + g * k : pos + g * k;
+    for (int i = 0; i < k; ++i) {
+      const int jj = (int)ix[i] - off;
+      if (jj >= 0 && jj < 32) orow[((jj & 1) << 4) | (jj >> 1)] = (uint8_t)((uint8_t)v[i] ^ 0x80u);
+    }
+  }
+}
+
 // Split-K, second kernel: out[m, n] from the `splits` raw partial sums of every accumulator
 // (the same integer and fp32 operations, in the same order, as the one-kernel epilogue).
 __global__ void __launch_bounds__(256) splitk_finish_kernel(const int32_t* __restrict__ ws, int splits, int M, int N,
@@ -890,10 +953,20 @@ static int choose_splits(int64_t M, int64_t N, int64_t K, int sms, size_t ws_byt
   return 1;
 }
 
-size_t gemm_workspace_bytes(int64_t M, int64_t N, int64_t K) {
+// More than 128 rows, dynamic positions: with M*K bytes of workspace the activations are expanded
+// once into merged 8-bit operands (kModeA8) instead of being widened, and merged, again for every
+// column tile.  Worth it from a few column tiles on.  Not for static positions: their sparse part
+// costs only a few extra K steps, and 8-bit activation tiles double the L2 traffic of the A
+// operand, which then bounds the kernel (measured: 20 % slower than the TMA-fed sparse steps).
+static bool use_a8(bool is_static, int64_t M, int64_t N, int64_t K, size_t ws_bytes) {
+  return !is_static && M > BM && (N + BN - 1) / BN >= 4 && (size_t)M * (size_t)K <= ws_bytes;
+}
+
+size_t gemm_workspace_bytes(bool is_static, int64_t M, int64_t N, int64_t K) {
   int dev = 0, sms = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) return 0;
   if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
+  if (M > BM) return use_a8(is_static, M, N, K, ~(size_t)0) ? (size_t)M * K : 0;
   const int sp = choose_splits(M, N, K, sms, ~(size_t)0);
   return sp > 1 ? (size_t)sp * M * N * 4 : 0;
 }
@@ -934,7 +1007,7 @@ cudaError_t launch_gemm(int b, int k, const sq_encoded& A, const sq_weights& W,
   }
 
   static int sm_count[64] = {0};
-  static int pair_slots[64][3] = {{0}};  // CTA pairs that can be resident at once, per kernel variant
+  static int pair_slots[64][4] = {{0}};  // CTA pairs that can be resident at once, per kernel variant
   int dev = 0;
   cudaError_t err = cudaGetDevice(&dev);
   if (err != cudaSuccess) return err;
@@ -948,7 +1021,8 @@ cudaError_t launch_gemm(int b, int k, const sq_encoded& A, const sq_weights& W,
   const uint8_t* pos_src = positions == nullptr ? A.idx : positions;
   const bool pmerge = !stma && nb == 16 && p.log2k >= 0 && GK % 16 == 0 &&
                       ((reinterpret_cast<uintptr_t>(A.vals) | reinterpret_cast<uintptr_t>(pos_src)) & 15) == 0;
-  const int mode = stma ? kModeTma : (pmerge ? kModeMergeProd : kModeMergeEpi);
+  const bool a8 = workspace != nullptr && use_a8(positions != nullptr, M, N, K, workspace_bytes);
+  const int mode = a8 ? kModeA8 : (stma ? kModeTma : (pmerge ? kModeMergeProd : kModeMergeEpi));
   // One CTA per tile for at most 128 rows (a second CTA would have no rows); CTA pairs otherwise.
   const int pair = M > BM ? 2 : 1;
   int slots = sm_count[dev];  // tiles in flight at once
@@ -969,7 +1043,8 @@ cudaError_t launch_gemm(int b, int k, const sq_encoded& A, const sq_weights& W,
       int n = 0;
       const void* fn = mode == kModeTma ? (const void*)gemm_kernel<2, kModeTma, false>
                        : mode == kModeMergeProd ? (const void*)gemm_kernel<2, kModeMergeProd, false>
-                                                : (const void*)gemm_kernel<2, kModeMergeEpi, false>;
+                       : mode == kModeA8 ? (const void*)gemm_kernel<2, kModeA8, false>
+                                         : (const void*)gemm_kernel<2, kModeMergeEpi, false>;
       err = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, Geo<2>::kSmemBytes);
       if (err == cudaSuccess) err = cudaOccupancyMaxActiveClusters(&n, fn, &qc);
       if (err != cudaSuccess) return err;
@@ -1047,7 +1122,7 @@ cudaError_t launch_gemm(int b, int k, const sq_encoded& A, const sq_weights& W,
       return cudaErrorInvalidValue;
   }
   p.SS = 0;
-  if (stma) {
+  if (stma && !a8) {
     const cuuint64_t pitch[1] = {(cuuint64_t)GK};
     const cuuint64_t dim_a[2] = {(cuuint64_t)GK, (cuuint64_t)M};
     const cuuint64_t dim_b[2] = {(cuuint64_t)GK, (cuuint64_t)N};
@@ -1062,6 +1137,23 @@ cudaError_t launch_gemm(int b, int k, const sq_encoded& A, const sq_weights& W,
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
       return cudaErrorInvalidValue;
     p.SS = (int)((GK + BK - 1) / BK);
+  }
+
+  if (a8) {
+    // the merged 8-bit activations: written once by expand_a8_kernel, read by TMA as [M, K] bytes
+    uint8_t* a8buf = static_cast<uint8_t*>(workspace);
+    const int64_t units = M * (K / 32);
+    int64_t blocks = (units + 255) / 256;
+    if (blocks > 32 * (int64_t)sm_count[dev]) blocks = 32 * (int64_t)sm_count[dev];
+    expand_a8_kernel<<<(unsigned)blocks, 256, 0, st>>>(A.dq4, A.vals, positions == nullptr ? A.idx : nullptr, positions,
+                                                      A.shift, M, (int)K, b, k, a8buf);
+    const cuuint64_t pitch[1] = {(cuuint64_t)K};
+    const cuuint64_t dim_a[2] = {(cuuint64_t)K, (cuuint64_t)M};
+    const cuuint32_t box_a[2] = {BK, 2 * BM};
+    if (encode(&map_a, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, a8buf, dim_a, pitch, box_a, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+      return cudaErrorInvalidValue;
   }
 
 #define SQ_LAUNCH_GEMM(PAIR_, MODE_, SPLIT_)                                                                \
@@ -1087,7 +1179,8 @@ cudaError_t launch_gemm(int b, int k, const sq_encoded& A, const sq_weights& W,
     if (err != cudaSuccess) return err;                                                                     \
   } while (0)
   if (pair == 2) {
-    if (mode == kModeTma) SQ_LAUNCH_GEMM(2, kModeTma, false);
+    if (mode == kModeA8) SQ_LAUNCH_GEMM(2, kModeA8, false);
+    else if (mode == kModeTma) SQ_LAUNCH_GEMM(2, kModeTma, false);
     else if (mode == kModeMergeProd) SQ_LAUNCH_GEMM(2, kModeMergeProd, false);
     else SQ_LAUNCH_GEMM(2, kModeMergeEpi, false);
   } else if (p.splits > 1) {

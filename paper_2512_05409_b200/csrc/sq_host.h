@@ -27,8 +27,8 @@ cudaError_t launch_decode(int b, int k, const sq_encoded& A, const uint8_t* posi
 cudaError_t launch_gemm(int b, int k, const sq_encoded& A, const sq_weights& W,
                         const uint8_t* positions, int64_t M, int64_t N, int64_t K, uint16_t* out,
                         int32_t* acc_out, int* status, void* workspace, size_t workspace_bytes, cudaStream_t st);
-// Bytes of workspace with which launch_gemm would split K for this shape (0: it would not).
-size_t gemm_workspace_bytes(int64_t M, int64_t N, int64_t K);
+// Bytes of workspace launch_gemm can make use of for this shape (0: none).
+size_t gemm_workspace_bytes(bool is_static, int64_t M, int64_t N, int64_t K);
 // The same launch with the library's own fixed scratch array as the workspace (no allocation).
 cudaError_t launch_gemm_static_scratch(int b, int k, const sq_encoded& A, const sq_weights& W,
                                        const uint8_t* positions, int64_t M, int64_t N, int64_t K, uint16_t* out,

@@ -69,7 +69,12 @@ def check_linear(lin: PackedLinear, X: torch.Tensor, seed: int, n_rows=24):
     cols_t = torch.from_numpy(lin.cols).to(DEV)
     assert np.array_equal(_np(acc[rows_t][:, cols_t]), acc_ref)
     assert_bf16_close(out[rows_t][:, cols_t], ref32)
-    del acc, out, enc
+    # the binding's sq_gemm hands the library a workspace (split-K for few rows, pre-widened activations
+    # for dynamic positions); the plain call must give the same bits
+    plain = sq.sq_gemm(lin.fmt, enc, lin.w, lin.pos, use_workspace=False)
+    check_status()
+    assert torch.equal(plain, out)
+    del acc, out, enc, plain
 
 
 # ----------------------------------------------------------------------------- config 2: sq_encode alone
