@@ -95,7 +95,7 @@ constexpr int kThreads = (kProdWarps + 1 + kEpiWarps + 2) * 32;
 constexpr int kStageA = 2 * BM * BK;  // 32 KB: two sub-tiles of A
 constexpr int kCtlBytes = 256;            // barriers, tensor-memory slot, abort flag
 constexpr int kEpiConstBytes = 2 * BN * 4;  // per tile: 2048 * colsum[n] and s_w[n] of its columns
-constexpr int kPackA = 2 * BM * (BK / 2);  // 16 KB: 256 rows x 64 packed bytes
+constexpr int kModeMergeEpi = 0, kModeTma = 1, kModeMergeProd = 2, kModeA8 = 3;  // see gemm_kernel
 constexpr int kRowsPerWarp = 2 * BM / kProdWarps;  // rows of A a producer warp widens per stage
 constexpr int kATasks = kRowsPerWarp / 8;  // 16-byte packed chunks of A per producer thread per step
 
@@ -104,9 +104,13 @@ constexpr int kATasks = kRowsPerWarp / 8;  // 16-byte packed chunks of A per pro
 // owns 256 rows of A and HALF of the weight tile (128 output channels), which the pair's tensor
 // cores read from both shared memories, so a CTA widens and holds a quarter less per MMA and
 // its shared memory serves a third less operand traffic -- the pipe this kernel is bound by.
-template <int PAIR>
+template <int PAIR, int MODE = kModeTma>
 struct Geo {
-  static constexpr int NS = PAIR == 2 ? 3 : 2;  // stages of widened (8-bit) operands
+  // packed A per stage: 256 rows x 64 bytes; none when TMA delivers 8-bit activations
+  static constexpr int kPackA = MODE == kModeA8 ? 0 : 2 * BM * (BK / 2);
+  // stages of widened (8-bit) operands; 8-bit activation tiles land there directly, so that ring
+  // alone hides their latency and gets the room the packed A ring does not need
+  static constexpr int NS = PAIR == 2 ? (MODE == kModeA8 ? 4 : 3) : 2;
   static constexpr int NP = 3;  // stages of packed (4-bit) operands as TMA delivers them
   static constexpr int BNL = BN / PAIR;          // weight rows (output channels) held by one CTA
   static constexpr int kStageB = BNL * BK;       // 32 / 16 KB
@@ -251,16 +255,15 @@ __device__ __forceinline__ bool wait_leader(uint32_t bar, uint32_t parity, volat
 //                   entries in place, K order of the MMA blocks), once per row instead of once
 //                   per row AND column tile; TMA brings those tiles straight into the widened
 //                   ring and the producers widen only the weights.  No sparse K steps either.
-constexpr int kModeMergeEpi = 0, kModeTma = 1, kModeMergeProd = 2, kModeA8 = 3;
 template <int PAIR, int MODE, bool SPLITK>
 __global__ void __launch_bounds__(kThreads, 1)
     gemm_kernel(const GemmParams p, const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                 const __grid_constant__ CUtensorMap map_a4, const __grid_constant__ CUtensorMap map_b4) {
-  using G = Geo<PAIR>;
+  using G = Geo<PAIR, MODE>;
   constexpr bool STMA = MODE == kModeTma, PMERGE = MODE == kModeMergeProd, A8 = MODE == kModeA8;
   constexpr bool ATMA = STMA || A8;  // the second TMA thread fills (some or all) A stages
   constexpr int NS = G::NS, NP = G::NP;
-  constexpr int kStageB = G::kStageB, kPackB = G::kPackB, kBTasks = G::kBTasks;
+  constexpr int kStageB = G::kStageB, kPackB = G::kPackB, kBTasks = G::kBTasks, kPackA = G::kPackA;
   // The kernel has no static shared memory, so the dynamic block starts at the 1024-byte
   // aligned base the swizzled operand layout needs; checked below, never assumed.
   extern __shared__ __align__(1024) uint8_t smem_raw[];
@@ -1037,7 +1040,7 @@ cudaError_t launch_gemm(int b, int k, const sq_encoded& A, const sq_weights& W,
       qa[0].val.clusterDim.z = 1;
       qc.gridDim = dim3((unsigned)(sm_count[dev] & ~1), 1, 1);
       qc.blockDim = dim3(kThreads, 1, 1);
-      qc.dynamicSmemBytes = Geo<2>::kSmemBytes;
+      qc.dynamicSmemBytes = (mode == kModeA8 ? Geo<2, kModeA8>::kSmemBytes : Geo<2>::kSmemBytes);
       qc.attrs = qa;
       qc.numAttrs = 1;
       int n = 0;
@@ -1045,7 +1048,7 @@ cudaError_t launch_gemm(int b, int k, const sq_encoded& A, const sq_weights& W,
                        : mode == kModeMergeProd ? (const void*)gemm_kernel<2, kModeMergeProd, false>
                        : mode == kModeA8 ? (const void*)gemm_kernel<2, kModeA8, false>
                                          : (const void*)gemm_kernel<2, kModeMergeEpi, false>;
-      err = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, Geo<2>::kSmemBytes);
+      err = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (mode == kModeA8 ? Geo<2, kModeA8>::kSmemBytes : Geo<2>::kSmemBytes));
       if (err == cudaSuccess) err = cudaOccupancyMaxActiveClusters(&n, fn, &qc);
       if (err != cudaSuccess) return err;
       if (n < 1) return cudaErrorLaunchOutOfResources;
@@ -1160,7 +1163,7 @@ cudaError_t launch_gemm(int b, int k, const sq_encoded& A, const sq_weights& W,
   do {                                                                                                      \
     err = cudaFuncSetAttribute(gemm_kernel<PAIR_, MODE_, SPLIT_>,                                           \
                                cudaFuncAttributeMaxDynamicSharedMemorySize,                                 \
-                               Geo<PAIR_>::kSmemBytes);                                                     \
+                               Geo<PAIR_, MODE_>::kSmemBytes);                                                     \
     if (err != cudaSuccess) return err;                                                                     \
     cudaLaunchConfig_t lc;                                                                                  \
     memset(&lc, 0, sizeof(lc));                                                                             \
@@ -1171,7 +1174,7 @@ cudaError_t launch_gemm(int b, int k, const sq_encoded& A, const sq_weights& W,
     la[0].val.clusterDim.z = 1;                                                                             \
     lc.gridDim = dim3(grid, 1, 1);                                                                          \
     lc.blockDim = dim3(kThreads, 1, 1);                                                                     \
-    lc.dynamicSmemBytes = Geo<PAIR_>::kSmemBytes;                                                           \
+    lc.dynamicSmemBytes = Geo<PAIR_, MODE_>::kSmemBytes;                                                           \
     lc.stream = st;                                                                                         \
     lc.attrs = la;                                                                                          \
     lc.numAttrs = (PAIR_ == 2) ? 1 : 0;                                                                     \
