@@ -312,7 +312,8 @@ __global__ void __launch_bounds__(kThreads, 1)
       // Every thread arrives for itself right after its own proxy fence (one arrival per warp
       // behind a __syncwarp was measured slower).  Static positions: the producers complete a
       // dense stage; otherwise the merge warps do.
-      mbar_init(bar_full + 8 * s, PAIR * ((STMA || PMERGE || A8) ? kProdWarps : kEpiWarps) * 32);
+      // (TMA-delivered activations: plus, per CTA of the pair, the arrival that announces its tile)
+      mbar_init(bar_full + 8 * s, PAIR * ((STMA || PMERGE || A8) ? kProdWarps : kEpiWarps) * 32 + (A8 ? PAIR : 0));
       mbar_init(bar_wfull + 8 * s, kProdWarps * 32);
       mbar_init(bar_empty + 8 * s, 1);
       mbar_init(bar_sfull + 8 * s, 1);
@@ -594,12 +595,12 @@ __global__ void __launch_bounds__(kThreads, 1)
         ok = wait_leader<PAIR>(bar_tempty, (tc & 1u) ^ 1u, abort_flag);  // previous tile's accumulators read out (both CTAs)
         if (!ok) break;
         tc_fence_after();
-        // What a K step waits for: dense = the producers' (or merge warps') "full"; with
-        // TMA-delivered activations also both CTAs' tile barriers; sparse = only those.  With
-        // TMA-delivered activations the producers run well ahead and three barrier round trips
-        // per step would make this thread the bottleneck, so it polls the NEXT step's barriers
-        // once between the two sub-tiles' MMAs: the answer's latency hides behind the issue of
-        // four MMAs.  (In the other modes the stage is usually not ready yet at that point and
+        // What a K step waits for: dense = the stage's "full" barrier (the producers or merge
+        // warps; with TMA-delivered activations also both CTAs' tiles arrive there); sparse =
+        // both CTAs' tile barriers.  With TMA-delivered activations the producers run well ahead
+        // and this thread's own loop is what paces the tensor pipe, so it polls the NEXT step's
+        // barrier once between the two sub-tiles' MMAs: the answer's latency hides behind the
+        // issue of four MMAs.  (In the other modes the stage is usually not ready yet at that point and
         // the extra poll only delays the second sub-tile: measured 12 % slower.)
         bool seen = false;  // this step's barriers were already found complete
         for (int ks = 0; ks < KS + SS; ++ks, ++it) {
@@ -607,14 +608,14 @@ __global__ void __launch_bounds__(kThreads, 1)
           const bool sparse_step = ks >= KS;
           if (!seen) {
             if (!sparse_step) ok = wait_leader<PAIR>(bar_full + 8 * s, (ph_dense >> s) & 1u, abort_flag);
-            if (ok && (sparse_step || A8)) {
+            if (ok && sparse_step) {
               ok = mbar_wait(bar_sfull + 8 * s, (ph_sparse >> s) & 1u, abort_flag);
               if (ok && PAIR == 2) ok = wait_leader<PAIR>(bar_sfullp + 8 * s, (ph_sparse >> s) & 1u, abort_flag);
             }
           }
           if (!ok) break;
           if (!sparse_step) ph_dense ^= 1u << s;
-          if (sparse_step || A8) ph_sparse ^= 1u << s;
+          if (sparse_step) ph_sparse ^= 1u << s;
           tc_fence_after();
           const uint64_t db = make_desc(smem_u32(sB + s * kStageB));
           const uint32_t id = sparse_step ? idesc_sparse : idesc;
@@ -630,7 +631,7 @@ __global__ void __launch_bounds__(kThreads, 1)
               bool r = true;
               if (!sparse2) r = PAIR == 2 ? mbar_test_cluster(bar_full + 8 * s2, (ph_dense >> s2) & 1u)
                                           : mbar_test(bar_full + 8 * s2, (ph_dense >> s2) & 1u);
-              if (r && (sparse2 || A8)) {
+              if (r && sparse2) {
                 r = mbar_test(bar_sfull + 8 * s2, (ph_sparse >> s2) & 1u);
                 if (r && PAIR == 2) r = mbar_test_cluster(bar_sfullp + 8 * s2, (ph_sparse >> s2) & 1u);
               }
@@ -678,7 +679,7 @@ __global__ void __launch_bounds__(kThreads, 1)
           const uint32_t fs = fq[fq_head % NS];
           if (!mbar_test(bar_sfull + 8 * fs, (ph_fwd >> fs) & 1u)) break;
           ph_fwd ^= 1u << fs;
-          mbar_arrive_cta(bar_sfullp + 8 * fs, 0);
+          mbar_arrive_cta((A8 ? bar_full : bar_sfullp) + 8 * fs, 0);
           ++fq_head;
           --fq_n;
         }
@@ -707,9 +708,13 @@ __global__ void __launch_bounds__(kThreads, 1)
           }
           if (!ok) continue;
           if (A8) {
-            // the merged 8-bit activations of this K step (rows past M come back as zeros)
-            mbar_expect_tx(bar_sfull + 8 * s, (uint32_t)kStageA);
-            tma_load_2d(smem_u32(sA + s * kStageA), &map_a, (t.k0 + step) * BK, t.m0, bar_sfull + 8 * s);
+            // the merged 8-bit activations of this K step (rows past M come back as zeros).  The
+            // leader's tile completes on the stage's "full" barrier itself, the peer's on its own
+            // barrier, from where it is reported to that same "full": the MMA thread then has a
+            // single barrier to look at per step.
+            const uint32_t abar = (forwards ? bar_sfull : bar_full) + 8 * s;
+            mbar_expect_tx(abar, (uint32_t)kStageA);
+            tma_load_2d(smem_u32(sA + s * kStageA), &map_a, (t.k0 + step) * BK, t.m0, abar);
           } else {
             if (step < KS) continue;
             const int ss = step - KS;
