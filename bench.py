@@ -406,7 +406,9 @@ def run_cuda(args):
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "steps": e2e_steps,
                 "note": "pinned host buffers; copies in, kernels and copies out on three streams (PCIe-bound)"},
-        "gpu_launches": 2 * len(layers) * args.steps,
+        # sq_encode + sq_gemm per linear, plus the second kernel a workspace brings with it (activation
+        # expansion above 128 rows, split-K finish at or below)
+        "gpu_launches": sum(2 + (1 if sq.sq_gemm_workspace_bytes(l.fmt, l.M, l.N, l.K) else 0) for l in layers) * args.steps,
         "roofline": {"kernel": "sq_gemm", "bound": "tensor", "achieved": gemm_tops, "peak": int8_peak,
                      "unit": "TOPS", "frac": gemm_tops / int8_peak,
                      "peak_source": f"2 x {peaks['source']} bf16 burst ({peaks['bf16_tflops']} TFLOP/s); INT8:bf16 nominal ratio 2",
