@@ -924,9 +924,22 @@ __global__ void __launch_bounds__(256) expand_a8_kernel(const uint8_t* __restric
     const int g = (blk * 32) / b, off = (blk * 32) % b;  // bank, and the block's first element inside it
     const int8_t* v = vals + m * GK + g * k;
     const uint8_t* ix = idx != nullptr ? idx + m * GK + g * k : pos + g * k;
-    for (int i = 0; i < k; ++i) {
-      const int jj = (int)ix[i] - off;
-      if (jj >= 0 && jj < 32) orow[((jj & 1) << 4) | (jj >> 1)] = (uint8_t)((uint8_t)v[i] ^ 0x80u);
+    if ((k & 7) == 0 && ((reinterpret_cast<uintptr_t>(v) | reinterpret_cast<uintptr_t>(ix)) & 7) == 0) {
+      for (int i8 = 0; i8 < k; i8 += 8) {  // eight entries per pair of 8-byte loads
+        const uint2 iw = *reinterpret_cast<const uint2*>(ix + i8);
+        const uint2 vw = *reinterpret_cast<const uint2*>(v + i8);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          const int jj = (int)(((i < 4 ? iw.x : iw.y) >> (8 * (i & 3))) & 0xFFu) - off;
+          const uint32_t byte = (((i < 4 ? vw.x : vw.y) >> (8 * (i & 3))) & 0xFFu) ^ 0x80u;
+          if (jj >= 0 && jj < 32) orow[((jj & 1) << 4) | (jj >> 1)] = (uint8_t)byte;
+        }
+      }
+    } else {
+      for (int i = 0; i < k; ++i) {
+        const int jj = (int)ix[i] - off;
+        if (jj >= 0 && jj < 32) orow[((jj & 1) << 4) | (jj >> 1)] = (uint8_t)((uint8_t)v[i] ^ 0x80u);
+      }
     }
   }
 }
