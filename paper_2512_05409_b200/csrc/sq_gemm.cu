@@ -898,6 +898,7 @@ __global__ void __launch_bounds__(256) expand_a8_kernel(const uint8_t* __restric
                                                         const uint8_t* __restrict__ pos,
                                                         const uint8_t* __restrict__ shift, int64_t M, int K, int b,
                                                         int k, uint8_t* __restrict__ a8) {
+  __shared__ __align__(16) uint8_t stage[256 * 32];
   const int blocks_per_row = K / 32;
   const int64_t total = M * blocks_per_row;
   const int GK = (K / b) * k;
@@ -915,12 +916,12 @@ __global__ void __launch_bounds__(256) expand_a8_kernel(const uint8_t* __restric
       o[q] = (u & 0x0F0F0F0Fu) * pmul + poff;
       o[4 + q] = ((u >> 4) & 0x0F0F0F0Fu) * pmul + poff;
     }
-    uint8_t* orow = a8 + m * K + blk * 32;
-    uint4* dst = reinterpret_cast<uint4*>(orow);
-    dst[0] = make_uint4(o[0], o[1], o[2], o[3]);
-    dst[1] = make_uint4(o[4], o[5], o[6], o[7]);
-    // sparse entries of the bank this block lies in: byte stores over what was just written (the
-    // same thread's later stores to the same bytes win)
+    // the 32 operand bytes go through shared memory, where the sparse entries of the bank this
+    // block lies in are patched in with byte stores, and leave as two 16-byte stores
+    uint8_t* orow = stage + threadIdx.x * 32;
+    uint4* sdst = reinterpret_cast<uint4*>(orow);
+    sdst[0] = make_uint4(o[0], o[1], o[2], o[3]);
+    sdst[1] = make_uint4(o[4], o[5], o[6], o[7]);
     const int g = (blk * 32) / b, off = (blk * 32) % b;  // bank, and the block's first element inside it
     const int8_t* v = vals + m * GK + g * k;
     const uint8_t* ix = idx != nullptr ? idx + m * GK + g * k : pos + g * k;
@@ -941,6 +942,9 @@ __global__ void __launch_bounds__(256) expand_a8_kernel(const uint8_t* __restric
         if (jj >= 0 && jj < 32) orow[((jj & 1) << 4) | (jj >> 1)] = (uint8_t)((uint8_t)v[i] ^ 0x80u);
       }
     }
+    uint4* dst = reinterpret_cast<uint4*>(a8 + m * K + blk * 32);
+    dst[0] = sdst[0];
+    dst[1] = sdst[1];
   }
 }
 
