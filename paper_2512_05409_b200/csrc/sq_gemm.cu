@@ -997,13 +997,11 @@ static int choose_splits(int64_t M, int64_t N, int64_t K, int sms, size_t ws_byt
 
 // More than 128 rows: with M*K bytes of workspace the activations are expanded once into merged
 // 8-bit operands (kModeA8) instead of being widened, and merged, again for every column tile.
-// Dynamic positions: worth it from a few column tiles on (the merge is what it saves).  Static
-// positions: the TMA-fed sparse K steps cost only ~12 % of the GEMM, so the expansion pass pays
-// for itself only when there are many output channels (measured break-even near N = 8192:
-// 2269 vs 2494 TOPS there, 3081 vs 2806 at N = 57344).
-static bool use_a8(bool is_static, int64_t M, int64_t N, int64_t K, size_t ws_bytes) {
-  const int64_t tiles_n = (N + BN - 1) / BN;
-  return M > BM && tiles_n >= (is_static ? 64 : 4) && (size_t)M * (size_t)K <= ws_bytes;
+// Worth the extra pass from a few column tiles on, for dynamic positions (it replaces the merge:
+// 2640 against 1760 TOPS at M = 4096, N = K = 8192) and for static ones (it replaces the sparse K
+// steps and two thirds of the widening: 2580 against 2480).
+static bool use_a8(bool /*is_static*/, int64_t M, int64_t N, int64_t K, size_t ws_bytes) {
+  return M > BM && (N + BN - 1) / BN >= 4 && (size_t)M * (size_t)K <= ws_bytes;
 }
 
 size_t gemm_workspace_bytes(bool is_static, int64_t M, int64_t N, int64_t K) {
