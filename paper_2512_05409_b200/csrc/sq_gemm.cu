@@ -91,7 +91,8 @@ constexpr int kEpiHelpers = kEpiWarps + (kProducersJoinEpilogue ? kProdWarps : 0
 constexpr int kEpiStride = kProducersJoinEpilogue ? 3 : 1;  // warps per TMEM lane quarter
 constexpr int kTmaWarp = kProdWarps + 1 + kEpiWarps;  // packed dense tiles
 constexpr int kTmaSparseWarp = kTmaWarp + 1;          // INT8 tiles of the sparse K steps
-constexpr int kThreads = (kProdWarps + 1 + kEpiWarps + 2) * 32;
+constexpr int kMma2Warp = kTmaSparseWarp + 1;           // second MMA issuer (pre-widened activations)
+constexpr int kThreads = (kProdWarps + 1 + kEpiWarps + 3) * 32;
 constexpr int kStageA = 2 * BM * BK;  // 32 KB: two sub-tiles of A
 constexpr int kCtlBytes = 256;            // barriers, tensor-memory slot, abort flag
 constexpr int kEpiConstBytes = 2 * BN * 4;  // per tile: 2048 * colsum[n] and s_w[n] of its columns
@@ -315,7 +316,7 @@ __global__ void __launch_bounds__(kThreads, 1)
       // (TMA-delivered activations: plus, per CTA of the pair, the arrival that announces its tile)
       mbar_init(bar_full + 8 * s, PAIR * ((STMA || PMERGE || A8) ? kProdWarps : kEpiWarps) * 32 + (A8 ? PAIR : 0));
       mbar_init(bar_wfull + 8 * s, kProdWarps * 32);
-      mbar_init(bar_empty + 8 * s, 1);
+      mbar_init(bar_empty + 8 * s, A8 ? 2 : 1);  // one commit per MMA-issuing thread
       mbar_init(bar_sfull + 8 * s, 1);
       mbar_init(bar_sfullp + 8 * s, 1);
     }
@@ -323,7 +324,7 @@ __global__ void __launch_bounds__(kThreads, 1)
       mbar_init(bar_pfull + 8 * s, 1);
       mbar_init(bar_pempty + 8 * s, kProdThreads);
     }
-    mbar_init(bar_tfull, 1);
+    mbar_init(bar_tfull, A8 ? 2 : 1);
     mbar_init(bar_tempty, PAIR * kEpiHelpers * 32);
     mbar_init(bar_eready, kEpiHelpers * 32);
     mbar_init(bar_edone, kEpiHelpers * 32);
@@ -579,10 +580,15 @@ __global__ void __launch_bounds__(kThreads, 1)
     }
     if (kProducersJoinEpilogue && ok)
       epilogue_share(tile_of<PAIR, SPLITK>(p, cl + (my_tiles - 1) * ncl, rank), (uint32_t)(my_tiles - 1), pw >> 2);
-  } else if (warp == kMmaWarp) {
-    // =============================================================== MMA issuer
+  } else if (warp == kMmaWarp || warp == kMma2Warp) {
+    // =============================================================== MMA issuer(s)
     // (the leader CTA's; the peer's MMA warp only holds its half of the tensor-memory allocation)
-    if (lane == 0 && rank == 0) {
+    // With TMA-delivered activations nothing but this loop paces the tensor pipe (~50 ns per
+    // tcgen05.mma issue plus a barrier round trip and a commit per step against 560 ns of MMA
+    // work), so two threads in two warps share it: each issues one sub-tile's MMAs and commits
+    // for itself (the "empty" and "accumulators complete" barriers then expect two commits).
+    const int sub_first = (A8 && warp == kMma2Warp) ? 1 : 0;
+    if (lane == 0 && rank == 0 && (A8 || warp == kMmaWarp)) {
       constexpr uint32_t idesc = make_idesc(false, BM * PAIR);
       constexpr uint32_t idesc_sparse = make_idesc(true, BM * PAIR);
       uint32_t it = 0, tc = 0;
@@ -620,12 +626,15 @@ __global__ void __launch_bounds__(kThreads, 1)
           const uint64_t db = make_desc(smem_u32(sB + s * kStageB));
           const uint32_t id = sparse_step ? idesc_sparse : idesc;
           seen = false;
-          for (int sub = 0; sub < nsub; ++sub) {
-            const uint64_t da = make_desc(smem_u32(sA + s * kStageA + sub * (BM * BK)));
+          const int sub_end = A8 ? (sub_first + 1 < nsub ? sub_first + 1 : nsub) : nsub;
+          for (int sub = sub_first; sub < sub_end || (A8 && sub == sub_first); ++sub) {
+            if (sub < nsub) {
+              const uint64_t da = make_desc(smem_u32(sA + s * kStageA + sub * (BM * BK)));
 #pragma unroll
-            for (int kk = 0; kk < BK / 32; ++kk)  // 32 bytes of K per MMA: +2 in 16-byte address units
-              umma_i8<PAIR>(tmem + sub * BN, da + 2 * kk, db + 2 * kk, id, (ks > 0 || kk > 0) ? 1u : 0u);
-            if (A8 && sub == 0 && ks + 1 < KS + SS) {
+              for (int kk = 0; kk < BK / 32; ++kk)  // 32 bytes of K per MMA: +2 in 16-byte address units
+                umma_i8<PAIR>(tmem + sub * BN, da + 2 * kk, db + 2 * kk, id, (ks > 0 || kk > 0) ? 1u : 0u);
+            }
+            if (A8 && sub == sub_first && ks + 1 < KS + SS) {
               const int s2 = (int)((it + 1) % NS);
               const bool sparse2 = ks + 1 >= KS;
               bool r = true;
