@@ -308,3 +308,40 @@ def test_split_k_with_workspace(b, k, static, M, K):
     assert np.array_equal(_np(acc), acc_ref)
     assert_bf16_close(out, ref32)
     assert np.array_equal(_bits(out), out_ref)
+
+
+# ----------------------------------------------------------------------------- many rows: pre-widened activations
+
+@pytest.mark.parametrize("b,k,static", [(64, 8, False), (32, 1, False), (128, 64, False), (128, 16, True), (64, 4, True)])
+@pytest.mark.parametrize("M,K", [(200, 384), (513, 1024)])
+def test_prewidened_activations_with_workspace(b, k, static, M, K):
+    """sq_gemm_ws with M*K bytes of workspace (activations expanded once into 8-bit tensor-core
+    operands) against the oracle and, bit for bit, against the calls without or with too little
+    workspace (which widen, and merge, inside the GEMM kernel)."""
+    N = 1288                      # six column tiles, the last one ragged
+    fmt = sq.make_format(b, k, static)
+    X = gen.activations(M, K, seed=M + K, outlier_fraction=0.01, outlier_scale=20.0, device="cuda")
+    W = gen.weights(N, K, seed=K, device="cuda")
+    pos = pos_ref = None
+    if static:
+        pos = sq.sq_calib_positions(fmt, gen.calibration_batch(64, K, seed=K, device="cuda"), W)
+        pos_ref = _np(pos)
+    w = sq.sq_pack_weights(fmt, W, pos)
+    enc = sq.sq_encode(fmt, X, pos)
+    need = sq.sq_gemm_workspace_bytes(fmt, M, N, K)
+    assert need == M * K
+    ws = torch.full((need,), 0x5A, dtype=torch.uint8, device="cuda")
+    acc = torch.empty(M, N, dtype=torch.int32, device="cuda")
+    out = sq.sq_gemm_ws(fmt, enc, w, pos, acc_out=acc, workspace=ws)
+    again = sq.sq_gemm_ws(fmt, enc, w, pos, workspace=ws).clone()
+    acc0 = torch.empty(M, N, dtype=torch.int32, device="cuda")
+    plain = sq.sq_gemm_ws(fmt, enc, w, pos, acc_out=acc0, workspace=None)
+    short = sq.sq_gemm_ws(fmt, enc, w, pos, workspace=ws[: need - 16]).clone()
+    check_status()
+    assert torch.equal(acc, acc0) and torch.equal(out, plain) and torch.equal(again, plain) and torch.equal(short, plain)
+    enc_ref = oracle.encode(b, k, _bits(X), pos_ref)
+    w_ref = oracle.pack_weights(b, k, _bits(W), pos_ref)
+    acc_ref, ref32, out_ref = oracle.gemm(b, k, enc_ref, w_ref, pos_ref)
+    assert np.array_equal(_np(acc), acc_ref)
+    assert_bf16_close(out, ref32)
+    assert np.array_equal(_bits(out), out_ref)
