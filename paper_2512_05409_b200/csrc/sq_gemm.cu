@@ -72,6 +72,13 @@
 
 #include "sq_host.h"
 
+#define WAIT_PE mbar_wait_park
+#define WAIT_PF mbar_wait_park
+#ifdef PARK_T
+#define WAIT_T mbar_wait_park
+#else
+#define WAIT_T mbar_wait
+#endif
 namespace sq {
 
 namespace {
@@ -96,6 +103,7 @@ constexpr int kThreads = (kProdWarps + 1 + kEpiWarps + 3) * 32;
 constexpr int kStageA = 2 * BM * BK;  // 32 KB: two sub-tiles of A
 constexpr int kCtlBytes = 256;            // barriers, tensor-memory slot, abort flag
 constexpr int kEpiConstBytes = 2 * BN * 4;  // per tile: 2048 * colsum[n] and s_w[n] of its columns
+constexpr int kOutBlock = 32 * 32 * 2;        // one staged output block: 32 rows x 32 bf16
 constexpr int kModeMergeEpi = 0, kModeTma = 1, kModeMergeProd = 2, kModeA8 = 3;  // see gemm_kernel
 constexpr int kRowsPerWarp = 2 * BM / kProdWarps;  // rows of A a producer warp widens per stage
 constexpr int kATasks = kRowsPerWarp / 8;  // 16-byte packed chunks of A per producer thread per step
@@ -112,13 +120,19 @@ struct Geo {
   // stages of widened (8-bit) operands; 8-bit activation tiles land there directly, so that ring
   // alone hides their latency and gets the room the packed A ring does not need
   static constexpr int NS = PAIR == 2 ? (MODE == kModeA8 ? 4 : 3) : 2;
-  static constexpr int NP = 3;  // stages of packed (4-bit) operands as TMA delivers them
+  // stages of packed (4-bit) operands as TMA delivers them (with 8-bit activations only weights
+  // pass through them, and the third stage's room goes to the output staging below)
+  static constexpr int NP = MODE == kModeA8 ? 2 : 3;
   static constexpr int BNL = BN / PAIR;          // weight rows (output channels) held by one CTA
   static constexpr int kStageB = BNL * BK;       // 32 / 16 KB
   static constexpr int kPackB = BNL * (BK / 2);  // 16 / 8 KB
   static constexpr int kRowsPerWarpB = BNL / kProdWarps;
   static constexpr int kBTasks = kRowsPerWarpB / 8;
-  static constexpr int kSmemBytes = NS * (kStageA + kStageB) + NP * (kPackA + kPackB) + kCtlBytes + kEpiConstBytes;
+  // output staging (8-bit activation mode): two 32-row x 32-column bf16 blocks per epilogue warp,
+  // which leave through TMA stores instead of one 16-byte store per thread and row
+  static constexpr int kOutStage = MODE == kModeA8 ? kEpiWarps * 2 * kOutBlock : 0;
+  static constexpr int kSmemBytes =
+      NS * (kStageA + kStageB) + NP * (kPackA + kPackB) + kOutStage + kCtlBytes + kEpiConstBytes;
 };
 constexpr int kMergeTasks = 8;  // sparse 4-entry words per merge thread per stage kept in registers
 
@@ -230,6 +244,23 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
       : "memory");
 }
 
+
+// 2-D tiled TMA store from this CTA's shared memory (rows and columns past the tensor's extent
+// are dropped); x in elements, x * element size a multiple of 16.  One bulk group per store.
+__device__ __forceinline__ void tma_store_2d(uint32_t src, const CUtensorMap* map, int x, int y) {
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];" ::"l"(map), "r"(x), "r"(y),
+               "r"(src)
+               : "memory");
+  asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+}
+// Wait until all but the newest N of this thread's bulk groups have read their shared memory ...
+template <int N>
+__device__ __forceinline__ void bulk_wait_read() {
+  asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
+}
+// ... or have completed altogether.
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+
 }  // namespace
 
 // Arrive on / wait for a barrier that lives in the pair's leader CTA.
@@ -263,6 +294,11 @@ __global__ void __launch_bounds__(kThreads, 1)
   using G = Geo<PAIR, MODE>;
   constexpr bool STMA = MODE == kModeTma, PMERGE = MODE == kModeMergeProd, A8 = MODE == kModeA8;
   constexpr bool ATMA = STMA || A8;  // the second TMA thread fills (some or all) A stages
+  // With 8-bit activations the epilogue is what the tensor pipe waits for between tiles, and its
+  // stores (a thread per row: 32 different 128-byte lines per 16-byte store instruction) were
+  // most of it.  There the bf16 block is staged in shared memory and written by TMA (map_b,
+  // otherwise unused in this mode, describes `out`).
+  constexpr bool TSTORE = A8 && !SPLITK;
   constexpr int NS = G::NS, NP = G::NP;
   constexpr int kStageB = G::kStageB, kPackB = G::kPackB, kBTasks = G::kBTasks, kPackA = G::kPackA;
   // The kernel has no static shared memory, so the dynamic block starts at the 1024-byte
@@ -278,7 +314,8 @@ __global__ void __launch_bounds__(kThreads, 1)
   uint8_t* sB = sA + NS * kStageA;         // NS x [BNL][128] widened B
   uint8_t* sPA = sB + NS * kStageB;        // NP x [256][64]  packed A as loaded
   uint8_t* sPB = sPA + NP * kPackA;        // NP x [BNL][64]  packed B as loaded
-  uint8_t* sCtl = sPB + NP * kPackB;
+  uint8_t* sOut = sPB + NP * kPackB;       // kEpiWarps x 2 x [32][64] staged output blocks (TSTORE)
+  uint8_t* sCtl = sOut + G::kOutStage;
   // mbarriers.  "leader" = waited for by the MMA thread of the pair's rank-0 CTA only; both
   // CTAs arrive there.  Everything else is local to a CTA (signalled in both by multicast
   // commits where the tensor core is the one that arrives).
@@ -346,16 +383,24 @@ __global__ void __launch_bounds__(kThreads, 1)
   //      w % 4; the three warps of a quarter split the tile's 32-column chunks.
   int32_t* s_cs = reinterpret_cast<int32_t*>(sCtl + kCtlBytes);  // 2048 * colsum of the tile's columns
   float* s_sw = reinterpret_cast<float*>(sCtl + kCtlBytes + BN * 4);
+  uint32_t oc = 0;  // TSTORE: blocks this warp has staged so far (their parity picks the buffer)
   auto epilogue_share = [&](const Tile& t, uint32_t tile_count, int helper) -> bool {
+    const int q = warp & 3;
+    // this thread's two rows' scales, requested before the wait so that no chunk waits for them
+    float sh2[2];
+#pragma unroll
+    for (int sub = 0; sub < 2; ++sub) {
+      const int m = t.m0 + sub * BM + 32 * q + lane;
+      sh2[sub] = (sub < t.nsub && m < p.M) ? __ldg(p.s_hi + m) : 0.f;
+    }
     if (!mbar_wait_idle(bar_tfull, tile_count & 1u, abort_flag)) return false;
     tc_fence_after();
     mbar_arrive(bar_eready);
     if (!mbar_wait(bar_eready, tile_count & 1u, abort_flag)) return false;
-    const int q = warp & 3;
     for (int ci = helper; ci < t.nsub * (BN / 32); ci += kEpiStride) {
       const int sub = ci / (BN / 32), c0 = (ci % (BN / 32)) * 32;
       const int m = t.m0 + sub * BM + 32 * q + lane;
-      const float sh = (m < p.M) ? p.s_hi[m] : 0.f;
+      const float sh = sub == 0 ? sh2[0] : sh2[1];
       uint32_t v[32];
       tmem_ld32(tmem + ((uint32_t)(32 * q) << 16) + (uint32_t)(sub * BN + c0), v);
       tmem_ld_wait();
@@ -370,10 +415,19 @@ __global__ void __launch_bounds__(kThreads, 1)
             dst[1] = make_int4((int)v[c8 + 4], (int)v[c8 + 5], (int)v[c8 + 6], (int)v[c8 + 7]);
           }
         }
-      } else if (m < p.M && n0 < p.N) {
+      } else if (TSTORE ? (t.m0 + sub * BM + 32 * q < p.M && n0 < p.N) : (m < p.M && n0 < p.N)) {
+        // TSTORE: the condition is the same for the whole warp; rows and columns of the block
+        // that lie past M or N are computed (from zero rows, clamped constants) and dropped by TMA
+        uint8_t* obuf = sOut + ((q * 2 + (int)(oc & 1u)) * kOutBlock);
+        if (TSTORE) {
+          if (oc >= 2) {  // the store that last used this buffer has read it
+            if (lane == 0) bulk_wait_read<1>();
+            __syncwarp();
+          }
+        }
 #pragma unroll
         for (int c8 = 0; c8 < 32; c8 += 8) {
-          if (n0 + c8 < p.N) {  // N % 8 == 0: a group of 8 columns is all in or all out
+          if (TSTORE || n0 + c8 < p.N) {  // N % 8 == 0: a group of 8 columns is all in or all out
             int acc[8];
             uint32_t o[4];
             const int4 cs0 = *reinterpret_cast<const int4*>(s_cs + c0 + c8);
@@ -390,13 +444,25 @@ __global__ void __launch_bounds__(kThreads, 1)
               const float f1 = ((float)acc[cc + 1] * sh) * sw[cc + 1];
               o[cc >> 1] = pack_bf16x2(f0, f1);
             }
-            *reinterpret_cast<uint4*>(p.out + (size_t)m * p.N + n0 + c8) = make_uint4(o[0], o[1], o[2], o[3]);
-            if (p.acc_out != nullptr) {
+            if (TSTORE) {
+              // row `lane` of the block, 16-byte piece c8 / 8, in the 64-byte swizzle TMA expects
+              *reinterpret_cast<uint4*>(obuf + lane * 64 + ((((c8 >> 3) ^ (lane >> 1)) & 3) << 4)) =
+                  make_uint4(o[0], o[1], o[2], o[3]);
+            } else {
+              *reinterpret_cast<uint4*>(p.out + (size_t)m * p.N + n0 + c8) = make_uint4(o[0], o[1], o[2], o[3]);
+            }
+            if (p.acc_out != nullptr && (!TSTORE || (m < p.M && n0 + c8 < p.N))) {
               int4* dst = reinterpret_cast<int4*>(p.acc_out + (size_t)m * p.N + n0 + c8);
               dst[0] = make_int4(acc[0], acc[1], acc[2], acc[3]);
               dst[1] = make_int4(acc[4], acc[5], acc[6], acc[7]);
             }
           }
+        }
+        if (TSTORE) {
+          fence_proxy_async_smem();
+          __syncwarp();
+          if (lane == 0) tma_store_2d(smem_u32(obuf), &map_b, n0, t.m0 + sub * BM + 32 * q);
+          ++oc;
         }
       }
     }
@@ -470,7 +536,7 @@ __global__ void __launch_bounds__(kThreads, 1)
       // ---- packed operands: wait for the TMA tiles, pull this thread's chunks into registers,
       //      hand the packed stage back
       const int ps = pit % NP;
-      if (!mbar_wait(bar_pfull + 8 * ps, (pit / NP) & 1u, abort_flag)) return false;
+      if (!WAIT_PF(bar_pfull + 8 * ps, (pit / NP) & 1u, abort_flag)) return false;
       uint4 ra[kATasks], rb[kBTasks];
       const uint8_t* pa = sPA + ps * kPackA + prow0;
       const uint8_t* pb = sPB + ps * kPackB + prowb0;
@@ -481,7 +547,7 @@ __global__ void __launch_bounds__(kThreads, 1)
       ++pit;
 
       const int s = it % NS;
-      if (!mbar_wait(bar_empty + 8 * s, ((it / NS) & 1u) ^ 1u, abort_flag)) return false;
+      if (!WAIT_PE(bar_empty + 8 * s, ((it / NS) & 1u) ^ 1u, abort_flag)) return false;
       uint8_t* a_st = sA + s * kStageA;
       uint8_t* b_st = sB + s * kStageB;
       if (pks == 0 && has_a) {  // the rows' shifts change with the tile only
@@ -662,7 +728,7 @@ __global__ void __launch_bounds__(kThreads, 1)
         const Tile t = tile_of<PAIR, SPLITK>(p, j, rank);
         for (int ks = 0; ks < KS && ok; ++ks, ++pit) {
           const int ps = pit % NP;
-          ok = mbar_wait(bar_pempty + 8 * ps, ((pit / NP) & 1u) ^ 1u, abort_flag);
+          ok = WAIT_T(bar_pempty + 8 * ps, ((pit / NP) & 1u) ^ 1u, abort_flag);
           if (!ok) break;
           // rows past M / N come back as zeros (code 0)
           mbar_expect_tx(bar_pfull + 8 * ps, (uint32_t)((A8 ? 0 : kPackA) + kPackB));
@@ -702,7 +768,7 @@ __global__ void __launch_bounds__(kThreads, 1)
           const int s = it % NS;
           const uint32_t par = ((it / NS) & 1u) ^ 1u;
           if (!forwards) {
-            ok = mbar_wait(bar_empty + 8 * s, par, abort_flag);
+            ok = WAIT_T(bar_empty + 8 * s, par, abort_flag);
           } else {
             ok = false;
             for (uint32_t n = 0; n < kSpinLimit; ++n) {
@@ -883,6 +949,7 @@ __global__ void __launch_bounds__(kThreads, 1)
       // the constants may be replaced only when every helper is done with them
       if (!mbar_wait(bar_edone, tc & 1u, abort_flag)) break;
     }
+    if (TSTORE && lane == 0) bulk_wait_all();  // the staged blocks have left before the CTA does
   }
 
   tc_fence_before();
@@ -1203,6 +1270,14 @@ cudaError_t launch_gemm(int b, int k, const sq_encoded& A, const sq_weights& W,
     const cuuint32_t box_a[2] = {BK, 2 * BM};
     if (encode(&map_a, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, a8buf, dim_a, pitch, box_a, estr,
                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+      return cudaErrorInvalidValue;
+    // `out` as [M, N] bf16 for the epilogue's TMA stores: blocks of 32 rows x 32 columns (64 bytes)
+    const cuuint64_t pitch_o[1] = {(cuuint64_t)N * 2};
+    const cuuint64_t dim_o[2] = {(cuuint64_t)N, (cuuint64_t)M};
+    const cuuint32_t box_o[2] = {32, 32};
+    if (encode(&map_b, CU_TENSOR_MAP_DATA_TYPE_UINT16, 2, out, dim_o, pitch_o, box_o, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
       return cudaErrorInvalidValue;
   }
