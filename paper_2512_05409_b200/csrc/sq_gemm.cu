@@ -100,11 +100,17 @@ constexpr int kTmaWarp = kProdWarps + 1 + kEpiWarps;  // packed dense tiles
 constexpr int kTmaSparseWarp = kTmaWarp + 1;          // INT8 tiles of the sparse K steps
 constexpr int kMma2Warp = kTmaSparseWarp + 1;           // second MMA issuer (pre-widened activations)
 constexpr int kThreads = (kProdWarps + 1 + kEpiWarps + 3) * 32;
+// Pre-widened activations: the epilogue is what the tensor pipe waits for between tiles and one
+// warp per scheduler leaves its latencies (tensor-memory load, staging, TMA hand-over) exposed,
+// so four more warps (16..19) join it: two warps per tensor-memory lane quarter.
+constexpr int kEpiWarpsA8 = 8;
+constexpr int kThreadsA8 = kThreads + (kEpiWarpsA8 - kEpiWarps) * 32;
 constexpr int kStageA = 2 * BM * BK;  // 32 KB: two sub-tiles of A
 constexpr int kCtlBytes = 256;            // barriers, tensor-memory slot, abort flag
 constexpr int kEpiConstBytes = 2 * BN * 4;  // per tile: 2048 * colsum[n] and s_w[n] of its columns
 constexpr int kOutBlock = 32 * 32 * 2;        // one staged output block: 32 rows x 32 bf16
 constexpr int kModeMergeEpi = 0, kModeTma = 1, kModeMergeProd = 2, kModeA8 = 3;  // see gemm_kernel
+constexpr int threads_of(int mode) { return mode == kModeA8 ? kThreadsA8 : kThreads; }
 constexpr int kRowsPerWarp = 2 * BM / kProdWarps;  // rows of A a producer warp widens per stage
 constexpr int kATasks = kRowsPerWarp / 8;  // 16-byte packed chunks of A per producer thread per step
 
@@ -128,9 +134,9 @@ struct Geo {
   static constexpr int kPackB = BNL * (BK / 2);  // 16 / 8 KB
   static constexpr int kRowsPerWarpB = BNL / kProdWarps;
   static constexpr int kBTasks = kRowsPerWarpB / 8;
-  // output staging (8-bit activation mode): two 32-row x 32-column bf16 blocks per epilogue warp,
+  // output staging (8-bit activation mode): a 32-row x 32-column bf16 block per epilogue warp,
   // which leave through TMA stores instead of one 16-byte store per thread and row
-  static constexpr int kOutStage = MODE == kModeA8 ? kEpiWarps * 2 * kOutBlock : 0;
+  static constexpr int kOutStage = MODE == kModeA8 ? kEpiWarpsA8 * kOutBlock : 0;
   static constexpr int kSmemBytes =
       NS * (kStageA + kStageB) + NP * (kPackA + kPackB) + kOutStage + kCtlBytes + kEpiConstBytes;
 };
@@ -288,7 +294,7 @@ __device__ __forceinline__ bool wait_leader(uint32_t bar, uint32_t parity, volat
 //                   per row AND column tile; TMA brings those tiles straight into the widened
 //                   ring and the producers widen only the weights.  No sparse K steps either.
 template <int PAIR, int MODE, bool SPLITK>
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(threads_of(MODE), 1)
     gemm_kernel(const GemmParams p, const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                 const __grid_constant__ CUtensorMap map_a4, const __grid_constant__ CUtensorMap map_b4) {
   using G = Geo<PAIR, MODE>;
@@ -299,6 +305,8 @@ __global__ void __launch_bounds__(kThreads, 1)
   // most of it.  There the bf16 block is staged in shared memory and written by TMA (map_b,
   // otherwise unused in this mode, describes `out`).
   constexpr bool TSTORE = A8 && !SPLITK;
+  constexpr int kEpiAll = A8 ? kEpiWarpsA8 : kEpiHelpers;  // warps that read out a tile
+  constexpr int kEpiStep = A8 ? kEpiWarpsA8 / 4 : kEpiStride;  // ... per tensor-memory lane quarter
   constexpr int NS = G::NS, NP = G::NP;
   constexpr int kStageB = G::kStageB, kPackB = G::kPackB, kBTasks = G::kBTasks, kPackA = G::kPackA;
   // The kernel has no static shared memory, so the dynamic block starts at the 1024-byte
@@ -314,7 +322,7 @@ __global__ void __launch_bounds__(kThreads, 1)
   uint8_t* sB = sA + NS * kStageA;         // NS x [BNL][128] widened B
   uint8_t* sPA = sB + NS * kStageB;        // NP x [256][64]  packed A as loaded
   uint8_t* sPB = sPA + NP * kPackA;        // NP x [BNL][64]  packed B as loaded
-  uint8_t* sOut = sPB + NP * kPackB;       // kEpiWarps x 2 x [32][64] staged output blocks (TSTORE)
+  uint8_t* sOut = sPB + NP * kPackB;       // kEpiWarpsA8 x [32][64] staged output blocks (TSTORE)
   uint8_t* sCtl = sOut + G::kOutStage;
   // mbarriers.  "leader" = waited for by the MMA thread of the pair's rank-0 CTA only; both
   // CTAs arrive there.  Everything else is local to a CTA (signalled in both by multicast
@@ -362,9 +370,9 @@ __global__ void __launch_bounds__(kThreads, 1)
       mbar_init(bar_pempty + 8 * s, kProdThreads);
     }
     mbar_init(bar_tfull, A8 ? 2 : 1);
-    mbar_init(bar_tempty, PAIR * kEpiHelpers * 32);
-    mbar_init(bar_eready, kEpiHelpers * 32);
-    mbar_init(bar_edone, kEpiHelpers * 32);
+    mbar_init(bar_tempty, PAIR * kEpiAll * 32);
+    mbar_init(bar_eready, kEpiAll * 32);
+    mbar_init(bar_edone, kEpiAll * 32);
     *abort_flag = 0;
     fence_mbar_init();
   }
@@ -383,7 +391,7 @@ __global__ void __launch_bounds__(kThreads, 1)
   //      w % 4; the three warps of a quarter split the tile's 32-column chunks.
   int32_t* s_cs = reinterpret_cast<int32_t*>(sCtl + kCtlBytes);  // 2048 * colsum of the tile's columns
   float* s_sw = reinterpret_cast<float*>(sCtl + kCtlBytes + BN * 4);
-  uint32_t oc = 0;  // TSTORE: blocks this warp has staged so far (their parity picks the buffer)
+  uint32_t oc = 0;  // TSTORE: blocks this warp has staged so far
   auto epilogue_share = [&](const Tile& t, uint32_t tile_count, int helper) -> bool {
     const int q = warp & 3;
     // this thread's two rows' scales, requested before the wait so that no chunk waits for them
@@ -397,7 +405,7 @@ __global__ void __launch_bounds__(kThreads, 1)
     tc_fence_after();
     mbar_arrive(bar_eready);
     if (!mbar_wait(bar_eready, tile_count & 1u, abort_flag)) return false;
-    for (int ci = helper; ci < t.nsub * (BN / 32); ci += kEpiStride) {
+    for (int ci = helper; ci < t.nsub * (BN / 32); ci += kEpiStep) {
       const int sub = ci / (BN / 32), c0 = (ci % (BN / 32)) * 32;
       const int m = t.m0 + sub * BM + 32 * q + lane;
       const float sh = sub == 0 ? sh2[0] : sh2[1];
@@ -418,10 +426,10 @@ __global__ void __launch_bounds__(kThreads, 1)
       } else if (TSTORE ? (t.m0 + sub * BM + 32 * q < p.M && n0 < p.N) : (m < p.M && n0 < p.N)) {
         // TSTORE: the condition is the same for the whole warp; rows and columns of the block
         // that lie past M or N are computed (from zero rows, clamped constants) and dropped by TMA
-        uint8_t* obuf = sOut + ((q * 2 + (int)(oc & 1u)) * kOutBlock);
+        uint8_t* obuf = sOut + (q + 4 * helper) * kOutBlock;
         if (TSTORE) {
-          if (oc >= 2) {  // the store that last used this buffer has read it
-            if (lane == 0) bulk_wait_read<1>();
+          if (oc > 0) {  // this warp's previous store has read the buffer (the quarter's other warp works meanwhile)
+            if (lane == 0) bulk_wait_read<0>();
             __syncwarp();
           }
         }
@@ -814,7 +822,8 @@ __global__ void __launch_bounds__(kThreads, 1)
     __syncwarp();
   } else {
     // =============================================================== epilogue
-    const int et = tid - (kMmaWarp + 1) * 32;  // 0..127 among the epilogue threads
+    // 0..127 among the epilogue threads (128..255: the four extra warps of the 8-bit activation mode)
+    const int et = warp > kMma2Warp ? 128 + tid - (kMma2Warp + 1) * 32 : tid - (kMmaWarp + 1) * 32;
     // merge state (dynamic positions): word tasks tt = et + 128*jj -> (row tt / words-per-row, word)
     const int m_GK = (p.K / p.b) * p.k;
     const int m_nb = (BK / p.b) * p.k;  // sparse entries per row per K step
@@ -853,7 +862,7 @@ __global__ void __launch_bounds__(kThreads, 1)
     for (int j = cl; j < nwork; j += ncl, ++tc) {
       const Tile t = tile_of<PAIR, SPLITK>(p, j, rank);
       // the tile's column constants are fetched while the main loop is still running
-      for (int cc = et; cc < BN; cc += kEpiWarps * 32) {
+      for (int cc = et; cc < BN; cc += (A8 ? kEpiWarpsA8 : kEpiWarps) * 32) {
         const int n = min(t.n0 + cc, p.N - 1);
         s_cs[cc] = 2048 * __ldg(p.colsum + n);
         s_sw[cc] = __ldg(p.s_w + n);
@@ -945,7 +954,7 @@ __global__ void __launch_bounds__(kThreads, 1)
         }
         if (!ok) break;
       }
-      if (!epilogue_share(t, tc, kProducersJoinEpilogue ? 2 : 0)) break;
+      if (!epilogue_share(t, tc, A8 ? (warp > kMma2Warp ? 1 : 0) : (kProducersJoinEpilogue ? 2 : 0))) break;
       // the constants may be replaced only when every helper is done with them
       if (!mbar_wait(bar_edone, tc & 1u, abort_flag)) break;
     }
@@ -1154,7 +1163,7 @@ cudaError_t launch_gemm(int b, int k, const sq_encoded& A, const sq_weights& W,
       qa[0].val.clusterDim.y = 1;
       qa[0].val.clusterDim.z = 1;
       qc.gridDim = dim3((unsigned)(sm_count[dev] & ~1), 1, 1);
-      qc.blockDim = dim3(kThreads, 1, 1);
+      qc.blockDim = dim3(threads_of(mode), 1, 1);
       qc.dynamicSmemBytes = (mode == kModeA8 ? Geo<2, kModeA8>::kSmemBytes : Geo<2>::kSmemBytes);
       qc.attrs = qa;
       qc.numAttrs = 1;
@@ -1296,7 +1305,7 @@ cudaError_t launch_gemm(int b, int k, const sq_encoded& A, const sq_weights& W,
     la[0].val.clusterDim.y = 1;                                                                             \
     la[0].val.clusterDim.z = 1;                                                                             \
     lc.gridDim = dim3(grid, 1, 1);                                                                          \
-    lc.blockDim = dim3(kThreads, 1, 1);                                                                     \
+    lc.blockDim = dim3(threads_of(MODE_), 1, 1);                                                            \
     lc.dynamicSmemBytes = Geo<PAIR_, MODE_>::kSmemBytes;                                                           \
     lc.stream = st;                                                                                         \
     lc.attrs = la;                                                                                          \
