@@ -44,7 +44,7 @@ FALLBACK_HBM_GBS, FALLBACK_BF16_TFLOPS = 6650.0, 1590.0
 # algorithmic bytes; the benchmark's launches are too large to capture with --set full, so their
 # traffic is this ratio times their own algorithmic bytes (the traffic is operand streaming and
 # grows with the operands).  It is below 1 because most of the output is still in L2 at kernel end.
-GEMM_CAPTURE_TRAFFIC_BYTES = 50.50e6 + 3.62e6
+GEMM_CAPTURE_TRAFFIC_BYTES = 50.58e6 + 4.76e6
 GEMM_CAPTURE_ALGO_BYTES = 2048 * 8192 * 0.625 + 8192 * 8192 * 0.625 + 2.0 * 2048 * 8192
 # ncu DRAM traffic of one encode launch of the 8192 x 8192 bandwidth test (dynamic k=8 / static k=8),
 # profiles/encode_kernels_b64_k8_8192x8192.txt
