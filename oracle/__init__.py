@@ -37,6 +37,7 @@ def _load():
         _lib.sqo_equivalent_bits.argtypes = [ctypes.c_double, ctypes.c_double, ctypes.c_double, ctypes.c_int]
         _lib.sqo_num_threads.restype = ctypes.c_int
         _lib.sqo_gemm.restype = ctypes.c_int
+        _lib.sqo_gemm_indep.restype = ctypes.c_int
     return _lib
 
 
@@ -150,3 +151,39 @@ def decode(b: int, k: int, A: Encoded, positions: np.ndarray | None = None):
     _load().sqo_decode(ctypes.c_int(b), ctypes.c_int(k), _p(A.dq4), _p(A.vals), _p(A.idx), _p(positions),
                        _p(A.s_hi), _p(A.s_lo), _l(M), _l(K), _p(xf), _p(xb))
     return xf, xb
+
+
+def encode_indep(b: int, k: int, X_bits: np.ndarray, positions: np.ndarray) -> Encoded:
+    """Static positions with independent scales of the two parts (s_lo is not tied to s_hi; shift = 0)."""
+    M, K = X_bits.shape
+    assert K % b == 0 and K % 2 == 0 and X_bits.dtype == np.uint16 and positions is not None
+    G = K // b
+    dq4 = np.zeros((M, K // 2), dtype=np.uint8)
+    vals = np.zeros((M, G, k), dtype=np.int8)
+    s_hi = np.zeros(M, dtype=np.float32)
+    s_lo = np.zeros(M, dtype=np.float32)
+    shift = np.zeros(M, dtype=np.uint8)
+    _load().sqo_encode_indep(ctypes.c_int(b), ctypes.c_int(k), _p(X_bits), _l(M), _l(K), _p(positions),
+                             _p(dq4), _p(vals), _p(s_hi), _p(s_lo), _p(shift))
+    return Encoded(dq4, vals, None, s_hi, s_lo, shift)
+
+
+def gemm_indep(b: int, k: int, A: Encoded, W: Weights, positions: np.ndarray, rows=None, cols=None):
+    """Returns (acc_lo int32, acc_hi int32, ref32 float32, out bf16-bits uint16), each [n_rows, n_cols]."""
+    M, Kh = A.dq4.shape
+    K = Kh * 2
+    N = W.wq4.shape[0]
+    rows_a = None if rows is None else np.ascontiguousarray(rows, dtype=np.int64)
+    cols_a = None if cols is None else np.ascontiguousarray(cols, dtype=np.int64)
+    R = M if rows_a is None else len(rows_a)
+    C = N if cols_a is None else len(cols_a)
+    lo = np.zeros((R, C), dtype=np.int32)
+    hi = np.zeros((R, C), dtype=np.int32)
+    ref = np.zeros((R, C), dtype=np.float32)
+    out = np.zeros((R, C), dtype=np.uint16)
+    ov = _load().sqo_gemm_indep(ctypes.c_int(b), ctypes.c_int(k), _p(A.dq4), _p(A.vals), _p(positions),
+                                _p(A.s_hi), _p(A.s_lo), _p(W.wq4), _p(W.s_w), _l(M), _l(N), _l(K),
+                                _p(rows_a), _l(R), _p(cols_a), _l(C), _p(lo), _p(hi), _p(ref), _p(out))
+    if ov:
+        raise OverflowError("an accumulator does not fit in int32")
+    return lo, hi, ref, out

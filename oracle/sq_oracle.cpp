@@ -18,7 +18,9 @@
 //   * static activation split = per bank top (1-s) of I_j = |A_j * sum_i W_ij|:
 //     Section 3.2.2, Algorithm 2;
 //   * hybrid GEMM = dense low-precision product + sparse high-precision
-//     product into one result: Section 1 and Section 3.3 (Fig. 2b).
+//     product into one result: Section 1 and Section 3.3 (Fig. 2b);
+//   * independent-scale variant: separate scales for the high- and the
+//     low-precision part, Algorithm 1 (S_high, S_low).
 // Points on which the paper is silent (scale granularity, tie-breaks, rounding
 // mode, ...) follow the readings listed in the repository's design notes; every
 // one of them is restated next to the code that implements it.
@@ -297,6 +299,100 @@ int sqo_gemm(int b, int k, const uint8_t* dq4, const int8_t* vals, const uint8_t
       const int32_t acc32 = (int32_t)acc;
       const float ref = ((float)acc32 * s_hi[m]) * s_w[n];
       if (acc_out) acc_out[r * C + c] = acc32;
+      if (ref32_out) ref32_out[r * C + c] = ref;
+      if (out_bf16) out_bf16[r * C + c] = f32_to_bf16(ref);
+    }
+  }
+  return overflow;
+}
+
+// ---------------------------------------------------------------------------
+// Independent-scale variant for static positions.  Algorithm 1 quantises the
+// high- and the low-precision part of a bank split with separate scales S_high
+// and S_low; here that rule is applied to the statically split activations of
+// Algorithm 2 (per token row, like the tied-scale encode above):
+//  1. S = positions[g] for every bank g                      (Algorithm 2)
+//  2. smax = max_{j in S} |a_j|,  rmax = max_{j not in S} |a_j|
+//  3. smax > 0: inv_hi = 127.0f/smax, s_hi = smax/127.0f (fp32 divisions); else both 0
+//     rmax > 0: inv_lo = 7.0f/rmax,   s_lo = rmax/7.0f;                     else both 0
+//  4. j in S:     q_hi = clamp(RNE(a_j * inv_hi), -127, 127); dense nibble = 0
+//     j not in S: q_lo = clamp(RNE(a_j * inv_lo), -7, 7)
+//  5. same packing as sqo_encode; no idx (static), no shift (written as 0).
+void sqo_encode_indep(int b, int k, const uint16_t* X, long M, long K, const uint8_t* positions,
+                      uint8_t* dq4, int8_t* vals, float* s_hi, float* s_lo, uint8_t* shift) {
+  const long G = K / b;
+#pragma omp parallel for schedule(static)
+  for (long m = 0; m < M; ++m) {
+    std::vector<float> a(K);
+    std::vector<char> inS(K, 0);
+    for (long j = 0; j < K; ++j) a[j] = bf16_to_f32(X[m * K + j]);
+    for (long g = 0; g < G; ++g)
+      for (int i = 0; i < k; ++i) inS[g * b + positions[g * k + i]] = 1;
+    float smax = 0.f, rmax = 0.f;
+    for (long j = 0; j < K; ++j) {
+      const float mag = std::fabs(a[j]);
+      if (inS[j]) {
+        if (mag > smax) smax = mag;
+      } else {
+        if (mag > rmax) rmax = mag;
+      }
+    }
+    const float inv_hi = smax > 0.f ? 127.0f / smax : 0.f;
+    const float inv_lo = rmax > 0.f ? 7.0f / rmax : 0.f;
+    s_hi[m] = smax > 0.f ? smax / 127.0f : 0.f;
+    s_lo[m] = rmax > 0.f ? rmax / 7.0f : 0.f;
+    shift[m] = 0;
+    std::vector<int> qlo(K, 0);
+    for (long j = 0; j < K; ++j)
+      if (!inS[j]) qlo[j] = (int)clampl(rne_prod(a[j], inv_lo), -7, 7);
+    for (long j = 0; j < K; j += 2)
+      dq4[m * (K / 2) + j / 2] = (uint8_t)((qlo[j] & 0xF) | ((qlo[j + 1] & 0xF) << 4));
+    for (long g = 0; g < G; ++g)
+      for (int i = 0; i < k; ++i) {
+        const long j = g * b + positions[g * k + i];
+        vals[(m * G + g) * k + i] = (int8_t)clampl(rne_prod(a[j], inv_hi), -127, 127);
+      }
+  }
+}
+
+// Hybrid GEMM with independent scales: the two products keep their own int32
+// accumulator and meet in fp32 (Section 3.3's two streams; scales per Algorithm 1).
+//   acc_lo[m,n] = sum_j            q_lo[m,j] * wq[n,j]       (q_lo is 0 at the positions)
+//   acc_hi[m,n] = sum_{j in S}     q_hi[m,j] * wq[n,j]
+//   ref32[m,n]  = fmaf((float)acc_hi, s_hi[m], (float)acc_lo * s_lo[m]) * s_w[n]
+//   out[m,n]    = bf16_rne(ref32)
+// Returns 0, or 1 if an accumulator would not fit in int32.
+int sqo_gemm_indep(int b, int k, const uint8_t* dq4, const int8_t* vals, const uint8_t* positions,
+                   const float* s_hi, const float* s_lo, const uint8_t* wq4, const float* s_w, long M,
+                   long N, long K, const long* rows, long n_rows, const long* cols, long n_cols,
+                   int32_t* acc_lo_out, int32_t* acc_hi_out, float* ref32_out, uint16_t* out_bf16) {
+  const long R = rows ? n_rows : M;
+  const long C = cols ? n_cols : N;
+  const long G = K / b;
+  int overflow = 0;
+#pragma omp parallel for schedule(static) reduction(| : overflow)
+  for (long r = 0; r < R; ++r) {
+    const long m = rows ? rows[r] : r;
+    for (long c = 0; c < C; ++c) {
+      const long n = cols ? cols[c] : c;
+      long long lo = 0, hi = 0;
+      for (long j = 0; j < K; ++j) {
+        unsigned ab = dq4[m * (K / 2) + j / 2], wb = wq4[n * (K / 2) + j / 2];
+        int qa = nibble_to_int((j & 1) ? (ab >> 4) : (ab & 0xF));
+        int qw = nibble_to_int((j & 1) ? (wb >> 4) : (wb & 0xF));
+        lo += (long long)qa * qw;
+      }
+      for (long g = 0; g < G; ++g)
+        for (int i = 0; i < k; ++i) {
+          const long j = g * b + positions[g * k + i];
+          unsigned wb = wq4[n * (K / 2) + j / 2];
+          int qw = nibble_to_int((j & 1) ? (wb >> 4) : (wb & 0xF));
+          hi += (long long)vals[(m * G + g) * k + i] * qw;
+        }
+      if (lo > INT32_MAX || lo < INT32_MIN || hi > INT32_MAX || hi < INT32_MIN) overflow |= 1;
+      const float ref = std::fmaf((float)(int32_t)hi, s_hi[m], (float)(int32_t)lo * s_lo[m]) * s_w[n];
+      if (acc_lo_out) acc_lo_out[r * C + c] = (int32_t)lo;
+      if (acc_hi_out) acc_hi_out[r * C + c] = (int32_t)hi;
       if (ref32_out) ref32_out[r * C + c] = ref;
       if (out_bf16) out_bf16[r * C + c] = f32_to_bf16(ref);
     }

@@ -385,3 +385,120 @@ def test_shift_zero_gemm_equals_plain_w4a8():
     _assert_equal_up_to_double_rounding(q_lo + q_hi, a8, prod32.numpy())
     a8 = np.where(a8 != q_lo + q_hi, q_lo + q_hi, a8)   # take the single-rounding value at the ties
     assert np.array_equal(acc.astype(np.int64), a8 @ pw.wq.astype(np.int64).T)
+
+
+# ----------------------------------------------------------------------------- independent scales (Algorithm 1's S_high / S_low)
+
+def _indep_setup(b, k, M, N, K, seed):
+    x, W = _acts(M, K, seed=seed), _wts(N, K, seed=seed)
+    pos = oracle.calib_positions(b, k, gen.bf16_bits(gen.calibration_batch(32, K, seed=seed)), W)
+    return x, W, pos
+
+
+def test_indep_encode_matches_exact_rational_arithmetic():
+    """Each part is a textbook symmetric quantiser with its own absmax scale: codes, scales and
+    the half-step reconstruction bound, in exact rational arithmetic."""
+    b, k, M, K = 32, 4, 6, 256
+    x, _, pos = _indep_setup(b, k, M, 8, K, seed=41)
+    enc = oracle.encode_indep(b, k, x, pos)
+    assert enc.idx is None and np.all(enc.shift == 0)
+    q_lo, q_hi, sup = sparse_dense_split(enc, b, k, pos)
+    assert np.all(q_lo[sup] == 0) and np.all(q_hi[~sup] == 0)
+    assert np.all(np.abs(q_lo) <= 7) and np.all(np.abs(q_hi) <= 127)
+    a = bits_to_f32(x)
+    for m in range(M):
+        smax = np.float32(np.abs(a[m][sup[m]]).max())
+        rmax = np.float32(np.abs(a[m][~sup[m]]).max())
+        assert enc.s_hi[m] == smax / np.float32(127.0) and enc.s_lo[m] == rmax / np.float32(7.0)
+        inv_hi, inv_lo = np.float32(127.0) / smax, np.float32(7.0) / rmax
+        for j in range(K):
+            inv, lim = (inv_hi, 127) if sup[m, j] else (inv_lo, 7)
+            want = max(-lim, min(lim, rne_fraction(Fraction(float(a[m, j])) * Fraction(float(inv)))))
+            assert (q_hi if sup[m, j] else q_lo)[m, j] == want
+        # the extreme of each part takes the extreme code of its grid
+        assert np.abs(q_hi[m]).max() == 127 and np.abs(q_lo[m]).max() == 7
+    xd, _ = oracle.decode(b, k, enc, pos)
+    step = np.where(sup, enc.s_hi[:, None], enc.s_lo[:, None]).astype(np.float64)
+    assert np.all(np.abs(xd.astype(np.float64) - a) <= 0.5 * step * (1 + 1e-6) + 1e-30)
+
+
+def test_indep_equals_tied_when_the_scales_are_a_power_of_two_apart():
+    """Rows whose largest selected value is 127 * 2^p and whose largest other value is
+    7 * 2^(p+e): both rules give the same inverse scales, so the same codes and, with the dense
+    accumulator shifted by e, the same GEMM accumulator."""
+    b, k, M, N, K = 32, 4, 5, 12, 128
+    x, W, pos = _indep_setup(b, k, M, N, K, seed=43)
+    a = bits_to_f32(x).copy()
+    sup = np.zeros((M, K), dtype=bool)
+    cols = (np.arange(K // b)[:, None] * b + pos.astype(np.int64)).reshape(-1)
+    sup[:, cols] = True
+    for m in range(M):
+        e = m % 5
+        a[m] = np.clip(a[m], -3.0, 3.0)
+        a[m, cols[0]] = 127.0 * 0.125                      # the row maximum, at a selected place
+        other = np.flatnonzero(~sup[m])
+        a[m, other] = np.clip(a[m, other], -7.0 * 0.125 * 2 ** e, 7.0 * 0.125 * 2 ** e)
+        a[m, other[m]] = -7.0 * 0.125 * 2 ** e             # the largest unselected magnitude
+        sel = np.flatnonzero(sup[m])
+        a[m, sel] = np.clip(a[m, sel], -127.0 * 0.125, 127.0 * 0.125)
+    xb = f32_to_bf16_bits(a.astype(np.float32))
+    tied = oracle.encode(b, k, xb, pos)
+    ind = oracle.encode_indep(b, k, xb, pos)
+    assert np.array_equal(tied.shift, np.arange(M) % 5)
+    assert np.array_equal(tied.dq4, ind.dq4) and np.array_equal(tied.vals, ind.vals)
+    assert np.array_equal(tied.s_hi, ind.s_hi) and np.array_equal(tied.s_lo, ind.s_lo)
+    pw = oracle.pack_weights(b, k, W, pos)
+    acc, ref32, out = oracle.gemm(b, k, tied, pw, pos)
+    lo, hi, ref_i, out_i = oracle.gemm_indep(b, k, ind, pw, pos)
+    assert np.array_equal((lo.astype(np.int64) << tied.shift[:, None].astype(np.int64)) + hi, acc.astype(np.int64))
+    # the two epilogues round differently (one product of the merged sum against a fused
+    # multiply-add of the two parts), but only in the last place
+    ulp = np.spacing(np.abs(ref32))
+    assert np.all(np.abs(ref_i - ref32) <= 2 * ulp)
+
+
+def test_indep_gemm_is_two_integer_products_and_matches_fp64():
+    b, k, M, N, K = 32, 8, 9, 11, 128
+    x, W, pos = _indep_setup(b, k, M, N, K, seed=47)
+    enc = oracle.encode_indep(b, k, x, pos)
+    pw = oracle.pack_weights(b, k, W, pos)
+    lo, hi, ref32, out = oracle.gemm_indep(b, k, enc, pw, pos)
+    q_lo, q_hi, sup = sparse_dense_split(enc, b, k, pos)
+    wq = pw.wq.astype(np.int64)
+    assert np.array_equal(lo.astype(np.int64), q_lo @ wq.T)
+    assert np.array_equal(hi.astype(np.int64), q_hi @ wq.T)
+    # the gathered weight rows of Algorithm 2 give the same sparse product
+    cols = (np.arange(K // b)[:, None] * b + pos.astype(np.int64)).reshape(-1)
+    assert np.array_equal(hi.astype(np.int64) * 16, enc.vals.reshape(M, -1).astype(np.int64) @ pw.w_sparse.astype(np.int64).T)
+    assert np.array_equal(pw.w_sparse.astype(np.int64), 16 * wq[:, cols])
+    # fp64 brute force of the dequantised operands
+    xhat = np.where(sup, enc.s_hi.astype(np.float64)[:, None] * q_hi, enc.s_lo.astype(np.float64)[:, None] * q_lo)
+    what = pw.s_w.astype(np.float64)[:, None] * wq.astype(np.float64)
+    brute = np.zeros((M, N))
+    for m in range(M):
+        for n in range(N):
+            brute[m, n] = float(np.dot(xhat[m], what[n]))
+    # fp32 epilogue: the two terms may cancel, so the bound is relative to their magnitudes
+    scale = (np.abs(lo) * enc.s_lo[:, None] + np.abs(hi) * enc.s_hi[:, None]) * np.abs(pw.s_w)[None, :]
+    assert np.all(np.abs(ref32.astype(np.float64) - brute) <= 4 * 2.0 ** -24 * scale + 1e-300)
+    assert np.array_equal(out, f32_to_bf16_bits(ref32))
+    # sampled form returns the same entries
+    rows, cols2 = [3, 8, 0], [5, 10]
+    lo2, hi2, r2, o2 = oracle.gemm_indep(b, k, enc, pw, pos, rows=rows, cols=cols2)
+    assert np.array_equal(lo2, lo[np.ix_(rows, cols2)]) and np.array_equal(hi2, hi[np.ix_(rows, cols2)])
+    assert np.array_equal(r2, ref32[np.ix_(rows, cols2)]) and np.array_equal(o2, out[np.ix_(rows, cols2)])
+
+
+def test_indep_degenerate_rows():
+    b, k, K = 32, 4, 64
+    pos = np.tile(np.arange(k, dtype=np.uint8), (K // b, 1))
+    a = np.zeros((3, K), dtype=np.float32)
+    a[1, 0] = 5.0            # only a selected place is non-zero
+    a[2, 10] = -3.0          # only an unselected place is non-zero
+    enc = oracle.encode_indep(b, k, f32_to_bf16_bits(a), pos)
+    assert np.array_equal(enc.s_hi, np.array([0, 5.0 / 127.0, 0], dtype=np.float32))
+    assert np.array_equal(enc.s_lo, np.array([0, 0, 3.0 / 7.0], dtype=np.float32))
+    q_lo, q_hi, _ = sparse_dense_split(enc, b, k, pos)
+    assert not q_lo[0].any() and not q_hi[0].any()
+    assert q_hi[1, 0] == 127 and not q_lo[1].any()
+    assert q_lo[2, 10] == -7 and not q_hi[2].any()
