@@ -227,7 +227,8 @@ def bench_8b_dynamic(sq, dev, peaks, iters=20):
 
 def bench_format_sweep(sq, dev, peaks, iters=5):
     """The format-parameter sweep at M = 4096, K = N = 8192: bank b in {32, 64, 128} x high-precision
-    fraction k/b in {1/16, 1/8, 1/4}, static and dynamic positions, outlier channels x10 and x50.
+    fraction k/b in {1/16, 1/8, 1/4}, dynamic positions, static positions and static positions with
+    independent scales of the two parts, outlier channels x10 and x50.
     Per point: sq_gemm time (median of CUDA-event pairs, pre-widened mode) and the relative
     Frobenius error of the bf16 output against the fp32 product of the bf16 inputs (a library
     matmul, used only as the yardstick)."""
@@ -246,9 +247,9 @@ def bench_format_sweep(sq, dev, peaks, iters=5):
         for b in (32, 64, 128):
             for frac in (16, 8, 4):
                 k = b // frac
-                for static in (False, True):
-                    fmt = sq.make_format(b, k, static)
-                    pos = sq.sq_calib_positions(fmt, calib, W) if static else None
+                for static, indep in ((False, False), (True, False), (True, True)):
+                    fmt = sq.make_format(b, k, static, independent_scales=indep)
+                    pos = sq.sq_calib_positions(sq.make_format(b, k, True), calib, W) if static else None
                     w = sq.sq_pack_weights(fmt, W, pos)
                     enc = sq.sq_encode(fmt, X, pos)
                     for _ in range(3):
@@ -263,7 +264,8 @@ def bench_format_sweep(sq, dev, peaks, iters=5):
                     ms = statistics.median(a.elapsed_time(c) for a, c in evs)
                     tops = 2.0 * M * N * K / (ms * 1e-3) / 1e12
                     err = float((out.float() - ref).norm()) / ref_norm
-                    res.append({"b": b, "k": k, "positions": "static" if static else "dynamic", "outlier_scale": scale,
+                    res.append({"b": b, "k": k, "positions": ("static, independent scales" if indep else "static") if static else "dynamic",
+                                "outlier_scale": scale,
                                 "gemm_us": round(ms * 1e3, 1), "gemm_TOPS": round(tops, 1),
                                 "frac_of_measured_int8": round(tops / int8_peak, 4),
                                 "frac_of_nominal_4500": round(tops / 4500.0, 4), "rel_err_vs_fp32": round(err, 5)})
@@ -478,7 +480,7 @@ def run_cuda(args):
             line["gemm_8b_dynamic"] = {"workload": "8B-decoder-shaped linears, b=64, k=8, dynamic positions; per-launch CUDA events, median of 20 after 10 warm-ups (small inputs may sit in L2)",
                                        "results": bench_8b_dynamic(sq, dev, peaks)}
             if not args.no_sweep:
-                line["format_sweep"] = {"workload": "M=4096, K=N=8192; b x k/b x static/dynamic x outlier channels x{10,50}; Student-t nu=3 activations, 1% outlier channels; rel_err = ||out - fp32(X W^T)||_F / ||fp32(X W^T)||_F",
+                line["format_sweep"] = {"workload": "M=4096, K=N=8192; b x k/b x {dynamic, static, static with independent scales} x outlier channels x{10,50}; Student-t nu=3 activations, 1% outlier channels; rel_err = ||out - fp32(X W^T)||_F / ||fp32(X W^T)||_F",
                                         "results": bench_format_sweep(sq, dev, peaks)}
             line["encode"] = {"workload": "sq_encode alone: bf16 8192 x 8192, Student-t nu=3, 0.5% channels x50, b=64; 3 inputs in rotation (> L2)",
                               "observed_bound": {"dynamic": "alu: integer/logic pipe 81% busy (ncu), DRAM 30% of peak; exact top-k by sorting network costs ~9 ALU-pipe lane-instructions per element",

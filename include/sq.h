@@ -68,7 +68,17 @@ typedef enum {
   SQ_ERR_TIMEOUT = 7       /* a bounded device-side wait expired (sq_device_status) */
 } sq_status;
 
-typedef enum { SQ_POS_DYNAMIC = 0, SQ_POS_STATIC = 1 } sq_pos_mode;
+/* How the k positions of a bank are chosen and how the two parts are scaled.
+ *   SQ_POS_DYNAMIC       per token, the k largest magnitudes of the bank (Sections 3.2.2, 3.3)
+ *   SQ_POS_STATIC        fixed by calibration (Algorithm 2); scales tied: s_lo = s_hi * 2^shift
+ *   SQ_POS_STATIC_INDEP  the same positions, but the two parts get independent per-token
+ *                        scales as in Algorithm 1 (S_high, S_low): s_hi = (largest selected
+ *                        magnitude)/127, s_lo = (largest other magnitude)/7, shift = 0.  sq_gemm
+ *                        then keeps two int32 accumulators (dense and sparse product) and joins
+ *                        them in fp32: out = bf16(fmaf(acc_hi, s_hi, acc_lo * s_lo) * s_w).
+ *                        Needs (K/b)*k to be a multiple of 16 in sq_gemm; with acc_out != NULL
+ *                        that buffer holds [2, M, N]: acc_lo first, then acc_hi. */
+typedef enum { SQ_POS_DYNAMIC = 0, SQ_POS_STATIC = 1, SQ_POS_STATIC_INDEP = 2 } sq_pos_mode;
 
 /* The part of the Eq. 1 tuple that is a parameter (h_high = INT8, h_low = INT4 fixed). */
 typedef struct {

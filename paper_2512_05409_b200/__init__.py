@@ -5,7 +5,7 @@ The product is the C-ABI shared library built from `csrc/` (declared in
 """
 from .binding import (  # noqa: F401
     SQ_OK, SQ_ERR_INVALID_ARG, SQ_ERR_UNSUPPORTED, SQ_ERR_NULL_POINTER, SQ_ERR_ALIGNMENT,
-    SQ_ERR_ARCH, SQ_ERR_CUDA, SQ_ERR_TIMEOUT, SQ_POS_DYNAMIC, SQ_POS_STATIC, SQ_LAYOUT_VERSION,
+    SQ_ERR_ARCH, SQ_ERR_CUDA, SQ_ERR_TIMEOUT, SQ_POS_DYNAMIC, SQ_POS_STATIC, SQ_POS_STATIC_INDEP, SQ_LAYOUT_VERSION,
     SQ_MAX_K, LIBRARY_PATH, SqError, Encoded, Weights, sq_format, sq_encoded, sq_weights,
     make_format, alloc_encoded, alloc_weights, sq_status_string, sq_encoded_sizes,
     sq_weights_sizes, sq_calib_positions, sq_pack_weights, sq_encode, sq_gemm, sq_gemm_ws,

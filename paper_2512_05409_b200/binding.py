@@ -27,6 +27,7 @@ SQ_ERR_TIMEOUT = 7
 
 SQ_POS_DYNAMIC = 0
 SQ_POS_STATIC = 1
+SQ_POS_STATIC_INDEP = 2
 SQ_LAYOUT_VERSION = 1
 SQ_MAX_K = 65536
 
@@ -98,8 +99,13 @@ def _check(status: int, where: str):
         raise SqError(status, where)
 
 
-def make_format(bank: int, k: int, static: bool) -> sq_format:
-    return sq_format(bank, k, SQ_POS_STATIC if static else SQ_POS_DYNAMIC, SQ_LAYOUT_VERSION)
+def make_format(bank: int, k: int, static: bool, independent_scales: bool = False) -> sq_format:
+    """independent_scales (static positions only): the two parts get their own per-token scales
+    (SQ_POS_STATIC_INDEP) instead of scales tied by a power of two."""
+    if independent_scales and not static:
+        raise ValueError("independent scales are built for static positions")
+    mode = SQ_POS_STATIC_INDEP if independent_scales else (SQ_POS_STATIC if static else SQ_POS_DYNAMIC)
+    return sq_format(bank, k, mode, SQ_LAYOUT_VERSION)
 
 
 @dataclass
@@ -174,7 +180,7 @@ def alloc_weights(fmt: sq_format, N: int, K: int, device="cuda") -> Weights:
     s_w = _buf(sz[1], torch.float32, device)[:N]
     colsum = _buf(sz[2], torch.int32, device)[:N]
     w_sparse = None
-    if fmt.pos_mode == SQ_POS_STATIC:
+    if fmt.pos_mode != SQ_POS_DYNAMIC:
         w_sparse = _buf(sz[3], torch.int8, device)[: sz[3]].view(N, (K // fmt.bank) * fmt.k)
     return Weights(wq4, s_w, colsum, w_sparse)
 

@@ -16,13 +16,17 @@ int* status_word() {
 namespace {
 
 bool aligned16(const void* ptr) { return (reinterpret_cast<uintptr_t>(ptr) & 15u) == 0; }
+// Static positions (tied or independent scales) / the independent-scale variant of them.
+bool is_static(const sq_format* fmt) { return fmt->pos_mode != SQ_POS_DYNAMIC; }
+bool is_indep(const sq_format* fmt) { return fmt->pos_mode == SQ_POS_STATIC_INDEP; }
 
 sq_status check_format(const sq_format* fmt) {
   if (fmt == nullptr) return SQ_ERR_NULL_POINTER;
   if (fmt->version != SQ_LAYOUT_VERSION) return SQ_ERR_INVALID_ARG;
   if (fmt->bank != 32 && fmt->bank != 64 && fmt->bank != 128) return SQ_ERR_INVALID_ARG;
   if (fmt->k < 1 || fmt->k > fmt->bank / 2) return SQ_ERR_INVALID_ARG;
-  if (fmt->pos_mode != SQ_POS_DYNAMIC && fmt->pos_mode != SQ_POS_STATIC) return SQ_ERR_INVALID_ARG;
+  if (fmt->pos_mode != SQ_POS_DYNAMIC && fmt->pos_mode != SQ_POS_STATIC && fmt->pos_mode != SQ_POS_STATIC_INDEP)
+    return SQ_ERR_INVALID_ARG;
   return SQ_OK;
 }
 
@@ -60,14 +64,14 @@ sq_status check_encoded(const sq_format* fmt, const sq_encoded* A) {
 sq_status check_weights(const sq_format* fmt, const sq_weights* W) {
   if (W == nullptr) return SQ_ERR_NULL_POINTER;
   if (!W->wq4 || !W->s_w || !W->colsum) return SQ_ERR_NULL_POINTER;
-  if (fmt->pos_mode == SQ_POS_STATIC && !W->w_sparse) return SQ_ERR_NULL_POINTER;
+  if (is_static(fmt) && !W->w_sparse) return SQ_ERR_NULL_POINTER;
   if (!aligned16(W->wq4) || !aligned16(W->s_w) || !aligned16(W->colsum)) return SQ_ERR_ALIGNMENT;
-  if (fmt->pos_mode == SQ_POS_STATIC && !aligned16(W->w_sparse)) return SQ_ERR_ALIGNMENT;
+  if (is_static(fmt) && !aligned16(W->w_sparse)) return SQ_ERR_ALIGNMENT;
   return SQ_OK;
 }
 
 sq_status check_positions(const sq_format* fmt, const uint8_t* positions) {
-  if (fmt->pos_mode == SQ_POS_STATIC) {
+  if (is_static(fmt)) {
     if (positions == nullptr) return SQ_ERR_NULL_POINTER;
     if (!aligned16(positions)) return SQ_ERR_ALIGNMENT;
   } else if (positions != nullptr) {
@@ -123,14 +127,14 @@ sq_status sq_weights_sizes(const sq_format* fmt, int64_t N, int64_t K, size_t by
   bytes_out[0] = n * (size_t)(K / 2);
   bytes_out[1] = n * sizeof(float);
   bytes_out[2] = n * sizeof(int32_t);
-  bytes_out[3] = fmt->pos_mode == SQ_POS_STATIC ? n * gk : 0;
+  bytes_out[3] = is_static(fmt) ? n * gk : 0;
   return SQ_OK;
 }
 
 sq_status sq_calib_positions(const sq_format* fmt, const void* calib_bf16, int64_t T, int64_t K,
                              const void* W_bf16, int64_t N, uint8_t* positions, void* cuda_stream) {
   SQ_TRY(check_format(fmt));
-  if (fmt->pos_mode != SQ_POS_STATIC) return SQ_ERR_INVALID_ARG;
+  if (!is_static(fmt)) return SQ_ERR_INVALID_ARG;
   SQ_TRY(check_k(K));
   if (T < 1 || (W_bf16 != nullptr && N < 1)) return SQ_ERR_INVALID_ARG;
   if (calib_bf16 == nullptr || positions == nullptr) return SQ_ERR_NULL_POINTER;
@@ -153,7 +157,7 @@ sq_status sq_pack_weights(const sq_format* fmt, const void* W_bf16, int64_t N, i
   SQ_TRY(check_weights(fmt, out));
   SQ_TRY(check_device());
   sq_weights o = *out;
-  if (fmt->pos_mode != SQ_POS_STATIC) o.w_sparse = nullptr;
+  if (!is_static(fmt)) o.w_sparse = nullptr;
   return from_cuda(launch_pack_weights(fmt->bank, fmt->k, static_cast<const uint16_t*>(W_bf16), N, K, positions, o,
                                        static_cast<cudaStream_t>(cuda_stream)));
 }
@@ -171,7 +175,7 @@ sq_status sq_encode(const sq_format* fmt, const void* X_bf16, int64_t M, int64_t
   SQ_TRY(check_device());
   int* status = status_word();
   if (status == nullptr) return SQ_ERR_CUDA;
-  return from_cuda(launch_encode(fmt->bank, fmt->k, fmt->pos_mode == SQ_POS_STATIC,
+  return from_cuda(launch_encode(fmt->bank, fmt->k, is_static(fmt), is_indep(fmt),
                                  static_cast<const uint16_t*>(X_bf16), M, K, positions, *out, status,
                                  static_cast<cudaStream_t>(cuda_stream)));
 }
@@ -184,7 +188,7 @@ sq_status sq_gemm_workspace_bytes(const sq_format* fmt, int64_t M, int64_t N, in
   *bytes = 0;
   if (M == 0 || N == 0) return SQ_OK;
   SQ_TRY(check_device());
-  *bytes = gemm_workspace_bytes(fmt->pos_mode == SQ_POS_STATIC, M, N, K);
+  *bytes = gemm_workspace_bytes(is_static(fmt), is_indep(fmt), M, N, K);
   return SQ_OK;
 }
 
@@ -201,12 +205,15 @@ sq_status sq_gemm_ws(const sq_format* fmt, const sq_encoded* A, const sq_weights
   if (out_bf16 == nullptr) return SQ_ERR_NULL_POINTER;
   if (!aligned16(out_bf16) || !aligned16(acc_out) || !aligned16(workspace)) return SQ_ERR_ALIGNMENT;
   if ((M + 127) / 128 > 65535) return SQ_ERR_UNSUPPORTED;
+  // independent scales: the sparse product runs as TMA-fed K steps of its own, whose row pitch
+  // (G*k bytes) must be a multiple of 16
+  if (is_indep(fmt) && ((K / fmt->bank) * fmt->k) % 16 != 0) return SQ_ERR_UNSUPPORTED;
   SQ_TRY(check_device());
   int* status = status_word();
   if (status == nullptr) return SQ_ERR_CUDA;
-  return from_cuda(launch_gemm(fmt->bank, fmt->k, *A, *W, positions, M, N, K, static_cast<uint16_t*>(out_bf16),
-                               acc_out, status, workspace, workspace == nullptr ? 0 : workspace_bytes,
-                               static_cast<cudaStream_t>(cuda_stream)));
+  return from_cuda(launch_gemm(fmt->bank, fmt->k, is_indep(fmt), *A, *W, positions, M, N, K,
+                               static_cast<uint16_t*>(out_bf16), acc_out, status, workspace,
+                               workspace == nullptr ? 0 : workspace_bytes, static_cast<cudaStream_t>(cuda_stream)));
 }
 
 sq_status sq_gemm_static_scratch(const sq_format* fmt, const sq_encoded* A, const sq_weights* W,
@@ -217,7 +224,7 @@ sq_status sq_gemm_static_scratch(const sq_format* fmt, const sq_encoded* A, cons
   if (M < 0 || N < 0 || N % 8 != 0 || M > INT32_MAX || N > INT32_MAX) return SQ_ERR_INVALID_ARG;
   if (M == 0 || N == 0) return SQ_OK;
   // Only the few-row case has a use for scratch, and at least two parts of K must fit.
-  if (M > 128) return SQ_ERR_UNSUPPORTED;
+  if (M > 128 || is_indep(fmt)) return SQ_ERR_UNSUPPORTED;
   if ((uint64_t)2 * (uint64_t)M * (uint64_t)N * 4u > (uint64_t)gemm_static_scratch_bytes()) return SQ_ERR_UNSUPPORTED;
   SQ_TRY(check_positions(fmt, positions));
   SQ_TRY(check_encoded(fmt, A));
@@ -250,7 +257,7 @@ sq_status sq_decode(const sq_format* fmt, const sq_encoded* A, const uint8_t* po
   if (!aligned16(out_bf16)) return SQ_ERR_ALIGNMENT;
   SQ_TRY(check_device());
   sq_encoded a = *A;
-  if (fmt->pos_mode == SQ_POS_STATIC) a.idx = nullptr;
+  if (is_static(fmt)) a.idx = nullptr;
   return from_cuda(launch_decode(fmt->bank, fmt->k, a, positions, M, K, static_cast<uint16_t*>(out_bf16),
                                  static_cast<cudaStream_t>(cuda_stream)));
 }

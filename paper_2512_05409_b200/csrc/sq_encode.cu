@@ -191,6 +191,20 @@ __device__ __forceinline__ RowScale row_scale_warp(uint32_t amax_bits, uint32_t 
   return rs;
 }
 
+// Independent scales (Algorithm 1's S_high / S_low on a static split): each part is scaled by
+// its own maximum; no shift, and no dense code can pass 7.
+__device__ __forceinline__ RowScale row_scale_indep(uint32_t smax_bits, uint32_t rmax_bits) {
+  RowScale rs;
+  const float smax = bf16_bits_to_f32(smax_bits), rmax = bf16_bits_to_f32(rmax_bits);
+  rs.inv = smax > 0.f ? __fdiv_rn(127.0f, smax) : 0.f;
+  rs.s_hi = smax > 0.f ? __fdiv_rn(smax, 127.0f) : 0.f;
+  rs.inv_lo = rmax > 0.f ? __fdiv_rn(7.0f, rmax) : 0.f;
+  rs.s_lo = rmax > 0.f ? __fdiv_rn(rmax, 7.0f) : 0.f;
+  rs.e = 0;
+  rs.clamp = false;
+  return rs;
+}
+
 __device__ __forceinline__ void bulk_copy_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
   asm volatile(
@@ -598,7 +612,7 @@ __global__ void __launch_bounds__(B == 128 ? 256 : 512) encode_rows_kernel(const
 //   -> INT8 codes of the selected values, INT4 codes straight from the registers (selected
 //   places were cleared there while taking the maxima).
 // The kernel is bound by instruction issue, which is why the masks are tables.
-template <int NCL, int NT>
+template <int NCL, int NT, bool INDEP>
 __global__ void __launch_bounds__(NT, 1) encode_static_regs_kernel(const EncodeParams p) {
   extern __shared__ __align__(128) uint8_t smem_enc[];
   const int K = p.K, k = p.k;
@@ -652,8 +666,13 @@ __global__ void __launch_bounds__(NT, 1) encode_static_regs_kernel(const EncodeP
 #pragma unroll
     for (int c = 0; c < NCL; ++c) {
       const uint4 q = mk[c * 32];
-      a2 = max2(a2, max2(max2(v[c].x & 0x7FFF7FFFu, v[c].y & 0x7FFF7FFFu),
-                         max2(v[c].z & 0x7FFF7FFFu, v[c].w & 0x7FFF7FFFu)));
+      // all magnitudes (tied scales), or only the selected ones (independent scales)
+      if (INDEP)
+        a2 = max2(a2, max2(max2(v[c].x & ~q.x & 0x7FFF7FFFu, v[c].y & ~q.y & 0x7FFF7FFFu),
+                           max2(v[c].z & ~q.z & 0x7FFF7FFFu, v[c].w & ~q.w & 0x7FFF7FFFu)));
+      else
+        a2 = max2(a2, max2(max2(v[c].x & 0x7FFF7FFFu, v[c].y & 0x7FFF7FFFu),
+                           max2(v[c].z & 0x7FFF7FFFu, v[c].w & 0x7FFF7FFFu)));
       r2 = max2(r2, max2(max2(v[c].x & q.x, v[c].y & q.y), max2(v[c].z & q.z, v[c].w & q.w)));
       // selected places become (signed) zeros: their codes must not reach the packing below
       v[c].x &= q.x | 0x80008000u;
@@ -682,7 +701,7 @@ __global__ void __launch_bounds__(NT, 1) encode_static_regs_kernel(const EncodeP
     } else {
       __syncwarp();
     }
-    const RowScale rs = row_scale_warp(amax_bits, rmax_bits, lane);
+    const RowScale rs = INDEP ? row_scale_indep(amax_bits, rmax_bits) : row_scale_warp(amax_bits, rmax_bits, lane);
     if (glane == 0) {
       p.s_hi[m] = rs.s_hi;
       p.s_lo[m] = rs.s_lo;
@@ -751,7 +770,7 @@ __global__ void __launch_bounds__(NT, 1) encode_static_regs_kernel(const EncodeP
 //   phase 3  maximum of what is left -> shift e, s_lo
 //   phase 4  INT4 codes of the staged row (zeros at the selected places), 8 per 32-bit word
 template <int B>
-__global__ void __launch_bounds__(256) encode_generic_kernel(int k, bool is_static, const uint16_t* __restrict__ X, int64_t K,
+__global__ void __launch_bounds__(256) encode_generic_kernel(int k, bool is_static, bool indep, const uint16_t* __restrict__ X, int64_t K,
                                                              const uint8_t* __restrict__ positions,
                                                              uint8_t* __restrict__ dq4, int8_t* __restrict__ vals,
                                                              uint8_t* __restrict__ idx, float* __restrict__ s_hi,
@@ -774,7 +793,13 @@ __global__ void __launch_bounds__(256) encode_generic_kernel(int k, bool is_stat
       mx = max(mx, (w[q] >> 16) & 0x7FFFu);
     }
   }
-  const uint32_t amax_bits = block_max_u32(mx, scratch);  // barrier inside: row staged
+  uint32_t amax_bits = block_max_u32(mx, scratch);  // barrier inside: row staged
+  if (indep) {
+    // independent scales (static positions only): the INT8 grid spans the selected values alone
+    uint32_t sx = 0;
+    for (int64_t t = tid; t < G * k; t += 256) sx = max(sx, (uint32_t)srow[(t / k) * B + positions[t]] & 0x7FFFu);
+    amax_bits = block_max_u32(sx, scratch);
+  }
   const float amax = bf16_bits_to_f32(amax_bits);
   const float inv = amax > 0.f ? __fdiv_rn(127.0f, amax) : 0.f;
 
@@ -839,7 +864,7 @@ __global__ void __launch_bounds__(256) encode_generic_kernel(int k, bool is_stat
     }
   }
   const uint32_t rmax_bits = block_max_u32(rm, scratch);
-  const RowScale rs = row_scale(amax_bits, rmax_bits);
+  const RowScale rs = indep ? row_scale_indep(amax_bits, rmax_bits) : row_scale(amax_bits, rmax_bits);
   if (tid == 0) {
     s_hi[m] = rs.s_hi;
     s_lo[m] = rs.s_lo;
@@ -950,7 +975,7 @@ cudaError_t launch_rows(const EncodeParams& base, cudaStream_t st) {
 
 // Register-resident static kernel: usable when a row splits into 1, 2, 4 or 8 warp slices of
 // NCL * 256 elements with NCL one of the instantiated sizes, and its tables fit in shared memory.
-template <int NCL, int NT>
+template <int NCL, int NT, bool INDEP>
 cudaError_t launch_static_regs_as(EncodeParams p, int rw, cudaStream_t st) {
   const int GK = (p.K / p.b) * p.k;
   const int ngroups = (NT / 32) / rw;
@@ -964,25 +989,26 @@ cudaError_t launch_static_regs_as(EncodeParams p, int rw, cudaStream_t st) {
   if (err != cudaSuccess) return err;
   err = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
   if (err != cudaSuccess) return err;
-  err = cudaFuncSetAttribute(encode_static_regs_kernel<NCL, NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  err = cudaFuncSetAttribute(encode_static_regs_kernel<NCL, NT, INDEP>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (err != cudaSuccess) return err;
   int64_t blocks = (p.M + ngroups - 1) / ngroups;
   if (blocks > sms) blocks = sms;
-  encode_static_regs_kernel<NCL, NT><<<(unsigned)blocks, NT, smem, st>>>(p);
+  encode_static_regs_kernel<NCL, NT, INDEP><<<(unsigned)blocks, NT, smem, st>>>(p);
   return cudaGetLastError();
 }
 
 // cudaErrorNotSupported = this shape is left to the shared-memory kernel.  Slices of at most
 // 16 chunks per lane keep 16 warps resident (measured faster than fewer warps holding more).
+template <bool INDEP>
 cudaError_t launch_static_regs(const EncodeParams& p, cudaStream_t st) {
   if (p.K % 256 != 0 || p.K > 65535) return cudaErrorNotSupported;
   for (int rw = 1; rw <= 8; rw *= 2) {
     if ((p.K / 256) % rw != 0) continue;
     switch (p.K / 256 / rw) {
-      case 8: return launch_static_regs_as<8, 512>(p, rw, st);
-      case 12: return launch_static_regs_as<12, 512>(p, rw, st);
-      case 14: return launch_static_regs_as<14, 512>(p, rw, st);
-      case 16: return launch_static_regs_as<16, 512>(p, rw, st);
+      case 8: return launch_static_regs_as<8, 512, INDEP>(p, rw, st);
+      case 12: return launch_static_regs_as<12, 512, INDEP>(p, rw, st);
+      case 14: return launch_static_regs_as<14, 512, INDEP>(p, rw, st);
+      case 16: return launch_static_regs_as<16, 512, INDEP>(p, rw, st);
       default: break;
     }
   }
@@ -990,19 +1016,19 @@ cudaError_t launch_static_regs(const EncodeParams& p, cudaStream_t st) {
 }
 
 template <int B>
-cudaError_t launch_generic(int k, bool is_static, const uint16_t* X, int64_t M, int64_t K, const uint8_t* positions,
-                           const sq_encoded& out, cudaStream_t st) {
+cudaError_t launch_generic(int k, bool is_static, bool indep, const uint16_t* X, int64_t M, int64_t K,
+                           const uint8_t* positions, const sq_encoded& out, cudaStream_t st) {
   const size_t smem = (size_t)K * 2;
   cudaError_t err = cudaFuncSetAttribute(encode_generic_kernel<B>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (err != cudaSuccess) return err;
-  encode_generic_kernel<B><<<(unsigned)M, 256, smem, st>>>(k, is_static, X, K, positions, out.dq4, out.vals, out.idx,
+  encode_generic_kernel<B><<<(unsigned)M, 256, smem, st>>>(k, is_static, indep, X, K, positions, out.dq4, out.vals, out.idx,
                                                           out.s_hi, out.s_lo, out.shift);
   return cudaGetLastError();
 }
 
 }  // namespace
 
-cudaError_t launch_encode(int b, int k, bool is_static, const uint16_t* X, int64_t M, int64_t K,
+cudaError_t launch_encode(int b, int k, bool is_static, bool indep, const uint16_t* X, int64_t M, int64_t K,
                           const uint8_t* positions, const sq_encoded& out, int* status, cudaStream_t st) {
   EncodeParams p;
   p.X = X;
@@ -1021,8 +1047,16 @@ cudaError_t launch_encode(int b, int k, bool is_static, const uint16_t* X, int64
   p.nbuf = 1;
   p.rw = 1;
   p.group_stride = 0;
+  if (is_static && indep) {
+    // independent scales: the register kernel, or the plain one for row lengths it does not take
+    const cudaError_t err = launch_static_regs<true>(p, st);
+    if (err != cudaErrorNotSupported) return err;
+    if (b == 32) return launch_generic<32>(k, true, true, X, M, K, positions, out, st);
+    if (b == 64) return launch_generic<64>(k, true, true, X, M, K, positions, out, st);
+    return launch_generic<128>(k, true, true, X, M, K, positions, out, st);
+  }
   if (is_static) {
-    const cudaError_t err = launch_static_regs(p, st);
+    const cudaError_t err = launch_static_regs<false>(p, st);
     if (err != cudaErrorNotSupported) return err;
     if (b == 32) return launch_rows<32, 0>(p, st);
     if (b == 64) return launch_rows<64, 0>(p, st);
@@ -1035,9 +1069,9 @@ cudaError_t launch_encode(int b, int k, bool is_static, const uint16_t* X, int64
   SQ_DYN(64, 4) SQ_DYN(64, 8) SQ_DYN(64, 16) SQ_DYN(64, 32)
   SQ_DYN(128, 8) SQ_DYN(128, 16) SQ_DYN(128, 32) SQ_DYN(128, 64)
 #undef SQ_DYN
-  if (b == 32) return launch_generic<32>(k, false, X, M, K, positions, out, st);
-  if (b == 64) return launch_generic<64>(k, false, X, M, K, positions, out, st);
-  return launch_generic<128>(k, false, X, M, K, positions, out, st);
+  if (b == 32) return launch_generic<32>(k, false, false, X, M, K, positions, out, st);
+  if (b == 64) return launch_generic<64>(k, false, false, X, M, K, positions, out, st);
+  return launch_generic<128>(k, false, false, X, M, K, positions, out, st);
 }
 
 cudaError_t launch_decode(int b, int k, const sq_encoded& A, const uint8_t* positions, int64_t M,

@@ -109,7 +109,7 @@ constexpr int kStageA = 2 * BM * BK;  // 32 KB: two sub-tiles of A
 constexpr int kCtlBytes = 256;            // barriers, tensor-memory slot, abort flag
 constexpr int kEpiConstBytes = 2 * BN * 4;  // per tile: 2048 * colsum[n] and s_w[n] of its columns
 constexpr int kOutBlock = 32 * 32 * 2;        // one staged output block: 32 rows x 32 bf16
-constexpr int kModeMergeEpi = 0, kModeTma = 1, kModeMergeProd = 2, kModeA8 = 3;  // see gemm_kernel
+constexpr int kModeMergeEpi = 0, kModeTma = 1, kModeMergeProd = 2, kModeA8 = 3, kModeIndep = 4;  // see gemm_kernel
 constexpr int threads_of(int mode) { return mode == kModeA8 ? kThreadsA8 : kThreads; }
 constexpr int kRowsPerWarp = 2 * BM / kProdWarps;  // rows of A a producer warp widens per stage
 constexpr int kATasks = kRowsPerWarp / 8;  // 16-byte packed chunks of A per producer thread per step
@@ -148,6 +148,7 @@ struct GemmParams {
   const uint8_t* idx;  // dynamic positions [M,G,k] or nullptr
   const uint8_t* pos;  // static positions [G,k] or nullptr
   const float* s_hi;
+  const float* s_lo;  // independent scales only
   const uint8_t* shift;
   const uint8_t* wq4;
   const float* s_w;
@@ -288,6 +289,10 @@ __device__ __forceinline__ bool wait_leader(uint32_t bar, uint32_t parity, volat
 //   kModeMergeProd  16 sparse entries per row and K step (k/b = 1/8): every producer thread
 //                   merges one row of the 32 its warp has just widened -- no hand-over to
 //                   other warps, eight warps share the work
+//   kModeIndep      static positions with independent scales: like kModeTma, but the sparse K
+//                   steps accumulate into a tensor-memory accumulator of their own (the second
+//                   sub-tile's columns: every tile has one sub-tile per CTA) and the epilogue
+//                   joins the two integer sums in fp32 with the row's two scales
 //   kModeA8         the caller gave a workspace of M*K bytes: expand_a8_kernel has written the
 //                   activations there as merged 8-bit operands (dense part widened, sparse
 //                   entries in place, K order of the MMA blocks), once per row instead of once
@@ -298,7 +303,8 @@ __global__ void __launch_bounds__(threads_of(MODE), 1)
     gemm_kernel(const GemmParams p, const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                 const __grid_constant__ CUtensorMap map_a4, const __grid_constant__ CUtensorMap map_b4) {
   using G = Geo<PAIR, MODE>;
-  constexpr bool STMA = MODE == kModeTma, PMERGE = MODE == kModeMergeProd, A8 = MODE == kModeA8;
+  constexpr bool INDEP = MODE == kModeIndep;
+  constexpr bool STMA = MODE == kModeTma || INDEP, PMERGE = MODE == kModeMergeProd, A8 = MODE == kModeA8;
   constexpr bool ATMA = STMA || A8;  // the second TMA thread fills (some or all) A stages
   // With 8-bit activations the epilogue is what the tensor pipe waits for between tiles, and its
   // stores (a thread per row: 32 different 128-byte lines per 16-byte store instruction) were
@@ -401,6 +407,11 @@ __global__ void __launch_bounds__(threads_of(MODE), 1)
       const int m = t.m0 + sub * BM + 32 * q + lane;
       sh2[sub] = (sub < t.nsub && m < p.M) ? __ldg(p.s_hi + m) : 0.f;
     }
+    float sl = 0.f;  // independent scales: the row's dense scale (one sub-tile per CTA)
+    if (INDEP) {
+      const int m = t.m0 + 32 * q + lane;
+      sl = m < p.M ? __ldg(p.s_lo + m) : 0.f;
+    }
     if (!mbar_wait_idle(bar_tfull, tile_count & 1u, abort_flag)) return false;
     tc_fence_after();
     mbar_arrive(bar_eready);
@@ -410,10 +421,44 @@ __global__ void __launch_bounds__(threads_of(MODE), 1)
       const int m = t.m0 + sub * BM + 32 * q + lane;
       const float sh = sub == 0 ? sh2[0] : sh2[1];
       uint32_t v[32];
+      uint32_t vs[INDEP ? 32 : 1];  // independent scales: the sparse product's accumulators
       tmem_ld32(tmem + ((uint32_t)(32 * q) << 16) + (uint32_t)(sub * BN + c0), v);
+      if constexpr (INDEP) tmem_ld32(tmem + ((uint32_t)(32 * q) << 16) + (uint32_t)(BN + c0), vs);
       tmem_ld_wait();
       const int n0 = t.n0 + c0;
-      if (SPLITK) {
+      if constexpr (INDEP) {
+        // out = bf16(fmaf(acc_hi, s_hi, acc_lo * s_lo) * s_w): the dense sum carries the unsigned
+        // operand's offset (2048 * colsum) and both sums the weights' factor 16
+        if (m < p.M && n0 < p.N) {
+#pragma unroll
+          for (int c8 = 0; c8 < 32; c8 += 8) {
+            if (n0 + c8 < p.N) {
+              int lo[8], hi[8];
+              uint32_t o[4];
+#pragma unroll
+              for (int cc = 0; cc < 8; ++cc) {
+                lo[cc] = ((int)v[c8 + cc] - s_cs[c0 + c8 + cc]) >> 4;
+                hi[cc] = (int)vs[c8 + cc] >> 4;
+              }
+#pragma unroll
+              for (int cc = 0; cc < 8; cc += 2) {
+                const float f0 = __fmul_rn(__fmaf_rn((float)hi[cc], sh, __fmul_rn((float)lo[cc], sl)), s_sw[c0 + c8 + cc]);
+                const float f1 = __fmul_rn(__fmaf_rn((float)hi[cc + 1], sh, __fmul_rn((float)lo[cc + 1], sl)), s_sw[c0 + c8 + cc + 1]);
+                o[cc >> 1] = pack_bf16x2(f0, f1);
+              }
+              *reinterpret_cast<uint4*>(p.out + (size_t)m * p.N + n0 + c8) = make_uint4(o[0], o[1], o[2], o[3]);
+              if (p.acc_out != nullptr) {  // [2, M, N]: dense sums, then sparse sums
+                int4* dst = reinterpret_cast<int4*>(p.acc_out + (size_t)m * p.N + n0 + c8);
+                dst[0] = make_int4(lo[0], lo[1], lo[2], lo[3]);
+                dst[1] = make_int4(lo[4], lo[5], lo[6], lo[7]);
+                dst = reinterpret_cast<int4*>(p.acc_out + (size_t)p.M * p.N + (size_t)m * p.N + n0 + c8);
+                dst[0] = make_int4(hi[0], hi[1], hi[2], hi[3]);
+                dst[1] = make_int4(hi[4], hi[5], hi[6], hi[7]);
+              }
+            }
+          }
+        }
+      } else if (SPLITK) {
         // split-K: this work item's raw partial sums; splitk_finish_kernel adds the parts
         if (m < p.M) {
           int32_t* wrow = p.ws + ((size_t)t.split * p.M + m) * p.N + n0;
@@ -706,7 +751,8 @@ __global__ void __launch_bounds__(threads_of(MODE), 1)
               const uint64_t da = make_desc(smem_u32(sA + s * kStageA + sub * (BM * BK)));
 #pragma unroll
               for (int kk = 0; kk < BK / 32; ++kk)  // 32 bytes of K per MMA: +2 in 16-byte address units
-                umma_i8<PAIR>(tmem + sub * BN, da + 2 * kk, db + 2 * kk, id, (ks > 0 || kk > 0) ? 1u : 0u);
+                umma_i8<PAIR>(tmem + ((INDEP && sparse_step) ? BN : sub * BN), da + 2 * kk, db + 2 * kk, id,
+                              ((INDEP && sparse_step) ? (ks > KS || kk > 0) : (ks > 0 || kk > 0)) ? 1u : 0u);
             }
             if (A8 && sub == sub_first && ks + 1 < KS + SS) {
               const int s2 = (int)((it + 1) % NS);
@@ -1089,7 +1135,8 @@ static bool use_a8(bool /*is_static*/, int64_t M, int64_t N, int64_t K, size_t w
   return M > BM && (N + BN - 1) / BN >= 4 && (size_t)M * (size_t)K <= ws_bytes;
 }
 
-size_t gemm_workspace_bytes(bool is_static, int64_t M, int64_t N, int64_t K) {
+size_t gemm_workspace_bytes(bool is_static, bool indep, int64_t M, int64_t N, int64_t K) {
+  if (indep) return 0;  // two accumulators: neither a merged 8-bit operand nor split-K is built for it
   int dev = 0, sms = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) return 0;
   if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
@@ -1098,7 +1145,7 @@ size_t gemm_workspace_bytes(bool is_static, int64_t M, int64_t N, int64_t K) {
   return sp > 1 ? (size_t)sp * M * N * 4 : 0;
 }
 
-cudaError_t launch_gemm(int b, int k, const sq_encoded& A, const sq_weights& W,
+cudaError_t launch_gemm(int b, int k, bool indep, const sq_encoded& A, const sq_weights& W,
                         const uint8_t* positions, int64_t M, int64_t N, int64_t K, uint16_t* out,
                         int32_t* acc_out, int* status, void* workspace, size_t workspace_bytes, cudaStream_t st) {
   GemmParams p;
@@ -1107,6 +1154,7 @@ cudaError_t launch_gemm(int b, int k, const sq_encoded& A, const sq_weights& W,
   p.idx = positions == nullptr ? A.idx : nullptr;
   p.pos = positions;
   p.s_hi = A.s_hi;
+  p.s_lo = A.s_lo;
   p.shift = A.shift;
   p.wq4 = W.wq4;
   p.s_w = W.s_w;
@@ -1134,7 +1182,7 @@ cudaError_t launch_gemm(int b, int k, const sq_encoded& A, const sq_weights& W,
   }
 
   static int sm_count[64] = {0};
-  static int pair_slots[64][4] = {{0}};  // CTA pairs that can be resident at once, per kernel variant
+  static int pair_slots[64][5] = {{0}};  // CTA pairs that can be resident at once, per kernel variant
   int dev = 0;
   cudaError_t err = cudaGetDevice(&dev);
   if (err != cudaSuccess) return err;
@@ -1148,8 +1196,10 @@ cudaError_t launch_gemm(int b, int k, const sq_encoded& A, const sq_weights& W,
   const uint8_t* pos_src = positions == nullptr ? A.idx : positions;
   const bool pmerge = !stma && nb == 16 && p.log2k >= 0 && GK % 16 == 0 &&
                       ((reinterpret_cast<uintptr_t>(A.vals) | reinterpret_cast<uintptr_t>(pos_src)) & 15) == 0;
+  if (indep && !stma) return cudaErrorNotSupported;
+  if (indep) workspace = nullptr;
   const bool a8 = workspace != nullptr && use_a8(positions != nullptr, M, N, K, workspace_bytes);
-  const int mode = a8 ? kModeA8 : (stma ? kModeTma : (pmerge ? kModeMergeProd : kModeMergeEpi));
+  const int mode = indep ? kModeIndep : a8 ? kModeA8 : (stma ? kModeTma : (pmerge ? kModeMergeProd : kModeMergeEpi));
   // One CTA per tile for at most 128 rows (a second CTA would have no rows); CTA pairs otherwise.
   const int pair = M > BM ? 2 : 1;
   int slots = sm_count[dev];  // tiles in flight at once
@@ -1168,7 +1218,8 @@ cudaError_t launch_gemm(int b, int k, const sq_encoded& A, const sq_weights& W,
       qc.attrs = qa;
       qc.numAttrs = 1;
       int n = 0;
-      const void* fn = mode == kModeTma ? (const void*)gemm_kernel<2, kModeTma, false>
+      const void* fn = mode == kModeIndep ? (const void*)gemm_kernel<2, kModeIndep, false>
+                       : mode == kModeTma ? (const void*)gemm_kernel<2, kModeTma, false>
                        : mode == kModeMergeProd ? (const void*)gemm_kernel<2, kModeMergeProd, false>
                        : mode == kModeA8 ? (const void*)gemm_kernel<2, kModeA8, false>
                                          : (const void*)gemm_kernel<2, kModeMergeEpi, false>;
@@ -1198,6 +1249,7 @@ cudaError_t launch_gemm(int b, int k, const sq_encoded& A, const sq_weights& W,
     const double cost_cut = 0.65 * (double)((2 * rem + slots - 1) / slots);
     if (cost_whole <= cost_cut) as_pairs = pair_tiles;
   }
+  if (indep) as_pairs = 0;  // the second accumulator takes the second sub-tile's tensor-memory columns
   p.n_pairs = (int)as_pairs;
   p.n_split = (int)(2 * (pair_tiles - as_pairs));
   // split-K (one CTA per tile, at most 128 rows, caller-provided workspace)
@@ -1313,7 +1365,10 @@ cudaError_t launch_gemm(int b, int k, const sq_encoded& A, const sq_weights& W,
     err = cudaLaunchKernelEx(&lc, gemm_kernel<PAIR_, MODE_, SPLIT_>, p, map_a, map_b, map_a4, map_b4);      \
     if (err != cudaSuccess) return err;                                                                     \
   } while (0)
-  if (pair == 2) {
+  if (mode == kModeIndep) {
+    if (pair == 2) SQ_LAUNCH_GEMM(2, kModeIndep, false);
+    else SQ_LAUNCH_GEMM(1, kModeIndep, false);
+  } else if (pair == 2) {
     if (mode == kModeA8) SQ_LAUNCH_GEMM(2, kModeA8, false);
     else if (mode == kModeTma) SQ_LAUNCH_GEMM(2, kModeTma, false);
     else if (mode == kModeMergeProd) SQ_LAUNCH_GEMM(2, kModeMergeProd, false);
@@ -1364,7 +1419,7 @@ cudaError_t launch_gemm_static_scratch(int b, int k, const sq_encoded& A, const 
     if (ptr == nullptr) return cudaErrorInvalidSymbol;
     scratch_addr[dev] = ptr;
   }
-  return launch_gemm(b, k, A, W, positions, M, N, K, out, acc_out, status, scratch_addr[dev], kStaticScratchBytes, st);
+  return launch_gemm(b, k, false, A, W, positions, M, N, K, out, acc_out, status, scratch_addr[dev], kStaticScratchBytes, st);
 }
 
 }  // namespace sq

@@ -18,17 +18,17 @@ cudaError_t launch_calib_positions(int b, int k, const uint16_t* calib, int64_t 
 cudaError_t launch_pack_weights(int b, int k, const uint16_t* W, int64_t N, int64_t K,
                                 const uint8_t* positions, const sq_weights& out, cudaStream_t st);
 
-cudaError_t launch_encode(int b, int k, bool is_static, const uint16_t* X, int64_t M, int64_t K,
+cudaError_t launch_encode(int b, int k, bool is_static, bool indep, const uint16_t* X, int64_t M, int64_t K,
                           const uint8_t* positions, const sq_encoded& out, int* status, cudaStream_t st);
 
 cudaError_t launch_decode(int b, int k, const sq_encoded& A, const uint8_t* positions, int64_t M,
                           int64_t K, uint16_t* out, cudaStream_t st);
 
-cudaError_t launch_gemm(int b, int k, const sq_encoded& A, const sq_weights& W,
+cudaError_t launch_gemm(int b, int k, bool indep, const sq_encoded& A, const sq_weights& W,
                         const uint8_t* positions, int64_t M, int64_t N, int64_t K, uint16_t* out,
                         int32_t* acc_out, int* status, void* workspace, size_t workspace_bytes, cudaStream_t st);
 // Bytes of workspace launch_gemm can make use of for this shape (0: none).
-size_t gemm_workspace_bytes(bool is_static, int64_t M, int64_t N, int64_t K);
+size_t gemm_workspace_bytes(bool is_static, bool indep, int64_t M, int64_t N, int64_t K);
 // The same launch with the library's own fixed scratch array as the workspace (no allocation).
 cudaError_t launch_gemm_static_scratch(int b, int k, const sq_encoded& A, const sq_weights& W,
                                        const uint8_t* positions, int64_t M, int64_t N, int64_t K, uint16_t* out,

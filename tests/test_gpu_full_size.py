@@ -144,3 +144,30 @@ def test_config5_format_sweep(b, static):
             check_linear(lin, X, seed=k, n_rows=12)
             del lin, X
             torch.cuda.empty_cache()
+
+
+# ----------------------------------------------------------------------------- independent scales at full size
+
+@pytest.mark.parametrize("K,N,b,k", [(8192, 8192, 128, 16), (28672, 8192, 128, 16), (8192, 8192, 64, 8)])
+def test_independent_scales_full_size(K, N, b, k):
+    """SQ_POS_STATIC_INDEP at M = 4096: sampled rows x sampled channels of both accumulators and
+    of the output against the oracle."""
+    M = 4096
+    lin = PackedLinear(N, K, b, k, True, seed=K + N + 1, calib_dist=dict(outlier_fraction=0.01, outlier_scale=20.0))
+    fmt = sq.make_format(b, k, True, independent_scales=True)
+    X = gen.activations(M, K, seed=K + N + 1, outlier_fraction=0.01, outlier_scale=20.0, device=DEV)
+    enc = sq.sq_encode(fmt, X, lin.pos)
+    acc = torch.empty(2, M, N, dtype=torch.int32, device=DEV)
+    out = sq.sq_gemm(fmt, enc, lin.w, lin.pos, acc_out=acc)
+    check_status()
+    rows = _sample(M, 16, 3, always=(0, M - 1, 127, 128, 255, 256))
+    rows_t, cols_t = torch.from_numpy(rows).to(DEV), torch.from_numpy(lin.cols).to(DEV)
+    enc_ref = oracle.encode_indep(b, k, _bits(X[rows_t]), lin.pos_ref)
+    assert np.array_equal(_np(enc.dq4[rows_t]), enc_ref.dq4) and np.array_equal(_np(enc.vals[rows_t]), enc_ref.vals)
+    assert np.array_equal(_np(enc.s_hi[rows_t]).view(np.uint32), enc_ref.s_hi.view(np.uint32))
+    assert np.array_equal(_np(enc.s_lo[rows_t]).view(np.uint32), enc_ref.s_lo.view(np.uint32))
+    assert not _np(enc.shift[rows_t]).any()
+    lo, hi, ref32, out_ref = oracle.gemm_indep(b, k, enc_ref, lin.w_ref, lin.pos_ref)
+    assert np.array_equal(_np(acc[0][rows_t][:, cols_t]), lo) and np.array_equal(_np(acc[1][rows_t][:, cols_t]), hi)
+    assert_bf16_close(out[rows_t][:, cols_t], ref32)
+    assert np.array_equal(_bits(out[rows_t][:, cols_t].contiguous()), out_ref)

@@ -345,3 +345,80 @@ def test_prewidened_activations_with_workspace(b, k, static, M, K):
     assert np.array_equal(_np(acc), acc_ref)
     assert_bf16_close(out, ref32)
     assert np.array_equal(_bits(out), out_ref)
+
+
+# ----------------------------------------------------------------------------- independent scales (static positions)
+
+@pytest.mark.parametrize("b,k", [(64, 8), (128, 16), (32, 8), (128, 64)])
+@pytest.mark.parametrize("M,K", [(37, 2048), (5, 384), (130, 3584)])
+def test_indep_encode_and_decode(b, k, M, K):
+    """SQ_POS_STATIC_INDEP: encode (the register kernel for K = 2048 and 3584, the plain kernel for
+    K = 384) and decode against the oracle, bit for bit."""
+    fmt = sq.make_format(b, k, True, independent_scales=True)
+    X = gen.activations(M, K, seed=M + K + b, outlier_fraction=0.01, outlier_scale=20.0, device="cuda")
+    W = gen.weights(24, K, seed=K, device="cuda")
+    pos = sq.sq_calib_positions(sq.make_format(b, k, True), gen.calibration_batch(64, K, seed=K, device="cuda"), W)
+    enc = sq.sq_encode(fmt, X, pos)
+    check_status()
+    ref = oracle.encode_indep(b, k, _bits(X), _np(pos))
+    compare_encoded(enc, ref)
+    dec = sq.sq_decode(fmt, enc, pos)
+    _, ref_bits = oracle.decode(b, k, ref, _np(pos))
+    assert np.array_equal(_bits(dec), ref_bits)
+
+
+def test_indep_encode_degenerate_rows():
+    b, k, K = 64, 8, 2048
+    fmt = sq.make_format(b, k, True, independent_scales=True)
+    pos = torch.arange(k, dtype=torch.uint8, device="cuda").repeat(K // b, 1).contiguous()
+    X = torch.zeros(4, K, dtype=torch.bfloat16, device="cuda")
+    X[1, 3] = 5.0       # only a selected place
+    X[2, 40] = -3.0     # only an unselected place
+    X[3, 3], X[3, 40] = 1e-30, -1e30
+    enc = sq.sq_encode(fmt, X, pos)
+    check_status()
+    compare_encoded(enc, oracle.encode_indep(b, k, _bits(X), _np(pos)))
+
+
+@pytest.mark.parametrize("b,k", [(64, 8), (128, 16), (32, 4)])
+@pytest.mark.parametrize("M,N,K", [(64, 264, 512), (200, 520, 1024), (513, 1288, 2048), (1, 8, 512)])
+def test_indep_gemm(b, k, M, N, K):
+    """Two accumulators (dense and sparse product) and the fp32 join, against the oracle: both
+    integer sums and the bf16 bits exact; with and without a workspace argument."""
+    fmt = sq.make_format(b, k, True, independent_scales=True)
+    X = gen.activations(M, K, seed=M + N, outlier_fraction=0.01, outlier_scale=20.0, device="cuda")
+    W = gen.weights(N, K, seed=N + K, device="cuda")
+    pos = sq.sq_calib_positions(sq.make_format(b, k, True), gen.calibration_batch(64, K, seed=K, device="cuda"), W)
+    w = sq.sq_pack_weights(fmt, W, pos)
+    enc = sq.sq_encode(fmt, X, pos)
+    assert sq.sq_gemm_workspace_bytes(fmt, M, N, K) == 0
+    acc = torch.empty(2, M, N, dtype=torch.int32, device="cuda")
+    out = sq.sq_gemm(fmt, enc, w, pos, acc_out=acc)
+    ws = torch.empty(M * K, dtype=torch.uint8, device="cuda")
+    out2 = sq.sq_gemm_ws(fmt, enc, w, pos, workspace=ws).clone()
+    check_status()
+    pos_ref = _np(pos)
+    enc_ref = oracle.encode_indep(b, k, _bits(X), pos_ref)
+    w_ref = oracle.pack_weights(b, k, _bits(W), pos_ref)
+    compare_encoded(enc, enc_ref)
+    compare_weights(w, w_ref)
+    lo, hi, ref32, out_ref = oracle.gemm_indep(b, k, enc_ref, w_ref, pos_ref)
+    assert np.array_equal(_np(acc[0]), lo) and np.array_equal(_np(acc[1]), hi)
+    assert_bf16_close(out, ref32)
+    assert np.array_equal(_bits(out), out_ref) and torch.equal(out, out2)
+
+
+def test_indep_gemm_rejects_what_it_cannot_run():
+    fmt = sq.make_format(32, 1, True, independent_scales=True)   # (K/b)*k = 8: not a multiple of 16
+    M, N, K = 16, 64, 256
+    X = gen.activations(M, K, seed=1, device="cuda")
+    W = gen.weights(N, K, seed=1, device="cuda")
+    pos = sq.sq_calib_positions(sq.make_format(32, 1, True), gen.calibration_batch(16, K, seed=1, device="cuda"), W)
+    w = sq.sq_pack_weights(fmt, W, pos)
+    enc = sq.sq_encode(fmt, X, pos)
+    compare_encoded(enc, oracle.encode_indep(32, 1, _bits(X), _np(pos)))
+    with pytest.raises(sq.SqError) as e:
+        sq.sq_gemm(fmt, enc, w, pos)
+    assert e.value.status == sq.SQ_ERR_UNSUPPORTED
+    with pytest.raises(ValueError):
+        sq.make_format(64, 8, False, independent_scales=True)
