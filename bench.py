@@ -132,15 +132,15 @@ def physical_gpu_index(local: int) -> int:
 class Linear:
     """One linear layer of the workload: packed weights, static positions, I/O buffers."""
 
-    def __init__(self, sq, M, K, N, bank, k, static, seed, dev, dist="student_t3"):
+    def __init__(self, sq, M, K, N, bank, k, static, seed, dev, dist="student_t3", independent_scales=False):
         self.M, self.K, self.N = M, K, N
-        self.fmt = sq.make_format(bank, k, static)
+        self.fmt = sq.make_format(bank, k, static, independent_scales=independent_scales)
         W = gen.weights(N, K, seed=seed, device=dev)
         self.pos = None
         if static:
             calib = gen.calibration_batch(512, K, seed=seed, dist=dist, outlier_fraction=0.01,
                                           outlier_scale=20.0, device=dev)
-            self.pos = sq.sq_calib_positions(self.fmt, calib, W)
+            self.pos = sq.sq_calib_positions(sq.make_format(bank, k, True), calib, W)
             del calib
         self.w = sq.sq_pack_weights(self.fmt, W, self.pos)
         del W
@@ -337,7 +337,8 @@ def run_cuda(args):
     # weak scaling: every rank owns its own batch of M tokens (tokens are independent units)
     M = args.m
     chosen = [int(x) for x in args.linears.split(",")] if args.linears else list(range(len(SHAPES_70B)))
-    layers = [Linear(sq, M, SHAPES_70B[i][0], SHAPES_70B[i][1], BANK_70B, K_70B, True, seed=rank * 16 + i, dev=dev)
+    layers = [Linear(sq, M, SHAPES_70B[i][0], SHAPES_70B[i][1], BANK_70B, K_70B, True, seed=rank * 16 + i, dev=dev,
+                     independent_scales=args.independent_scales)
               for i in chosen]
     total_ops = sum(l.ops for l in layers)
 
@@ -449,7 +450,8 @@ def run_cuda(args):
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "int8", "data": "synthetic",
-        "config": {"workload": WORKLOAD if not args.linears else WORKLOAD + f" [subset {args.linears}]", "M_per_gpu": M, "bank": BANK_70B, "k": K_70B, "positions": "static",
+        "config": {"workload": (WORKLOAD if not args.linears else WORKLOAD + f" [subset {args.linears}]")
+                               + (" [variant: independent scales of the two parts]" if args.independent_scales else ""), "M_per_gpu": M, "bank": BANK_70B, "k": K_70B, "positions": "static",
                    "step": "sq_encode + sq_gemm for each of the four linears",
                    "l2": "inputs larger than L2 (packed weights + activations + outputs of a step ~2.5 GB)",
                    "sharding": "tokens (M) per rank, weights replicated, no data-path collective"},
@@ -515,6 +517,8 @@ def main():
     ap.add_argument("--no-encode-bench", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-sweep", action="store_true", help="skip the format-parameter sweep block")
+    ap.add_argument("--independent-scales", action="store_true",
+                    help="run the step with the independent-scale variant of the static format (not the headline)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
