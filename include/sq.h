@@ -165,6 +165,11 @@ sq_status sq_pack_weights(const sq_format* fmt, const void* W_bf16, int64_t N, i
  *   e    = min{ e in 0..4 : RNE(rmax * inv * 2^-e) <= 7 }, or 4;  s_lo = s_hi * 2^e
  *   j in S:     vals = clamp(RNE(a_j * inv), -127, 127), dense nibble 0
  *   j not in S: dq4  = clamp(RNE(a_j * inv * 2^-e), -7, 7)
+ * SQ_POS_STATIC_INDEP (Algorithm 1's separate scales on the static split) instead:
+ *   smax = max over j in S of |a_j|;  smax > 0: inv_hi = 127.0f / smax, s_hi = smax / 127.0f
+ *   rmax > 0: inv_lo = 7.0f / rmax, s_lo = rmax / 7.0f          (a part that is all zero: 0, 0)
+ *   j in S: vals = clamp(RNE(a_j * inv_hi), -127, 127);  else dq4 = clamp(RNE(a_j * inv_lo), -7, 7)
+ *   shift = 0
  * X_bf16: device bf16 [M, K].  positions: as for sq_pack_weights.  out: every member
  * written (idx only for dynamic formats). */
 sq_status sq_encode(const sq_format* fmt, const void* X_bf16, int64_t M, int64_t K,
@@ -174,10 +179,14 @@ sq_status sq_encode(const sq_format* fmt, const void* X_bf16, int64_t M, int64_t
  * into ONE int32 accumulator, followed by one dequantising epilogue:
  *   acc[m,n] = sum_j ( (dq4[m,j] << shift[m]) + [j in S_m] vals[m,j] ) * code[n,j]
  *   out[m,n] = bf16_rne( ((float)acc[m,n] * s_hi[m]) * s_w[n] )
+ * SQ_POS_STATIC_INDEP: two accumulators, acc_lo[m,n] = sum_j dq4[m,j] * code[n,j] and
+ * acc_hi[m,n] = sum_{j in S} vals[m,j] * code[n,j], joined in fp32:
+ *   out[m,n] = bf16_rne( fmaf((float)acc_hi, s_hi[m], (float)acc_lo * s_lo[m]) * s_w[n] )
  * A: an encoding of an [M, K] tensor.  W: packed [N, K] weights of the same format.
  * positions: static formats only (the mask the two were built with), else NULL.
  * out_bf16: device bf16 [M, N], written.  acc_out: device int32 [M, N] or NULL; when
- * given, the raw accumulators are written as well (used by parity tests). */
+ * given, the raw accumulators are written as well (used by parity tests);
+ * SQ_POS_STATIC_INDEP: [2, M, N], acc_lo then acc_hi. */
 sq_status sq_gemm(const sq_format* fmt, const sq_encoded* A, const sq_weights* W,
                   const uint8_t* positions, int64_t M, int64_t N, int64_t K, void* out_bf16,
                   int32_t* acc_out, void* cuda_stream);
@@ -188,9 +197,11 @@ sq_status sq_gemm(const sq_format* fmt, const sq_encoded* A, const sq_weights* W
  *     all of K, so most SMs idle.  K is cut into up to 8 parts that run on different SMs,
  *     their raw int32 partial sums go to the workspace ([parts][M][N]) and a second kernel on
  *     the same stream adds them and runs the epilogue;
- *   - more tokens with dynamic positions: the activations are expanded once into merged 8-bit
- *     tensor-core operands ([M][K] bytes in the workspace) instead of being widened and
- *     merged again for every tile of output channels.
+ *   - more tokens (M > 128, at least four tiles of 256 output channels; dynamic or static
+ *     positions): the activations are expanded once into merged 8-bit tensor-core operands
+ *     ([M][K] bytes in the workspace) instead of being widened and merged again for every
+ *     tile of output channels.
+ * SQ_POS_STATIC_INDEP has no use for a workspace (two scales cannot share one merged operand).
  * sq_gemm_workspace_bytes: *bytes = the size this shape and format can make use of, 0 if none.
  * workspace: device memory, 16-byte aligned, or NULL (= sq_gemm); a smaller workspace than
  * asked for is used for fewer parts or not at all, never an error.  Its contents are
