@@ -216,7 +216,33 @@ def bench_8b_dynamic(sq, dev, peaks, iters=20):
             g_ms = statistics.median(e[1].elapsed_time(e[2]) for e in evs)
             e_ms = statistics.median(e[0].elapsed_time(e[1]) for e in evs)
             tops = l.ops / (g_ms * 1e-3) / 1e12
+            graph_us = None
+            if M <= 128:
+                # decode-sized calls are bound by the host's launch path (Python + two launches); the
+                # same ten calls replayed from a CUDA graph give the GPU's own time per call
+                side = torch.cuda.Stream()
+                side.wait_stream(torch.cuda.current_stream())
+                graph = torch.cuda.CUDAGraph()
+                with torch.cuda.stream(side):
+                    sq.sq_gemm(l.fmt, l.enc, l.w, l.pos, out=l.out)
+                    torch.cuda.synchronize()
+                    with torch.cuda.graph(graph, stream=side):
+                        for _ in range(10):
+                            sq.sq_gemm(l.fmt, l.enc, l.w, l.pos, out=l.out)
+                torch.cuda.synchronize()
+                graph.replay()
+                torch.cuda.synchronize()
+                g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                g0.record()
+                for _ in range(5):
+                    graph.replay()
+                g1.record()
+                torch.cuda.synchronize()
+                graph_us = round(g0.elapsed_time(g1) * 1e3 / 50, 1)
+                del graph
             res.append({"M": M, "K": K, "N": N, "gemm_us": round(g_ms * 1e3, 1), "encode_us": round(e_ms * 1e3, 1),
+                        "gemm_us_graph_replay": graph_us,
+                        "weight_stream_GBps_graph_replay": None if graph_us is None else round(N * K / 2 / (graph_us * 1e-6) / 1e9, 1),
                         "gemm_TOPS": round(tops, 1), "frac_of_measured_int8": round(tops / int8_peak, 4),
                         "frac_of_nominal_4500": round(tops / 4500.0, 4),
                         "weight_stream_GBps": round(N * K / 2 / (g_ms * 1e-3) / 1e9, 1)})

@@ -88,8 +88,16 @@ def _ptr(t):
     return None if t is None else ctypes.c_void_p(t.data_ptr())
 
 
+_raw_stream = getattr(torch._C, "_cuda_getCurrentRawStream", None)
+
+
 def _stream(stream):
+    """The CUDA stream handle to launch on: the given torch stream (or raw handle), else torch's
+    current stream on the current device (the direct lookup is several times cheaper than building
+    a torch.cuda.Stream object, which matters for decode-sized calls)."""
     if stream is None:
+        if _raw_stream is not None:
+            return ctypes.c_void_p(_raw_stream(torch.cuda.current_device()))
         stream = torch.cuda.current_stream()
     return ctypes.c_void_p(stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream))
 
