@@ -8,8 +8,14 @@ namespace sq {
 __device__ int g_status_word;
 
 int* status_word() {
+  // looked up once per device (the call is not free, and decode-sized launches are host-bound)
+  static int* cached[64] = {nullptr};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return nullptr;
+  if (dev >= 0 && dev < 64 && cached[dev] != nullptr) return cached[dev];
   int* ptr = nullptr;
   if (cudaGetSymbolAddress(reinterpret_cast<void**>(&ptr), g_status_word) != cudaSuccess) return nullptr;
+  if (dev >= 0 && dev < 64) cached[dev] = ptr;
   return ptr;
 }
 
@@ -38,9 +44,12 @@ sq_status check_k(int64_t K) {
 
 // The kernels are built for sm_100a only; refuse anything else before launching.
 sq_status check_device() {
+  static int major_of[64] = {0};  // per device, asked once
   int dev = 0, major = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) return SQ_ERR_CUDA;
+  if (dev >= 0 && dev < 64 && major_of[dev] != 0) return major_of[dev] == 10 ? SQ_OK : SQ_ERR_ARCH;
   if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return SQ_ERR_CUDA;
+  if (dev >= 0 && dev < 64) major_of[dev] = major;
   return major == 10 ? SQ_OK : SQ_ERR_ARCH;
 }
 

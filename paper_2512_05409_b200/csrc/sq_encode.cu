@@ -921,6 +921,31 @@ __global__ void __launch_bounds__(256) decode_kernel(int b, int k, const uint8_t
 
 namespace {
 
+// The current device and its SM count (asked once per device: the encode of a few decode tokens
+// is bound by the host's launch path).
+static cudaError_t device_and_sms(int* dev, int* sms) {
+  static int cached[64] = {0};
+  cudaError_t err = cudaGetDevice(dev);
+  if (err != cudaSuccess) return err;
+  if (*dev < 0 || *dev >= 64) return cudaErrorInvalidDevice;
+  if (cached[*dev] == 0) {
+    err = cudaDeviceGetAttribute(&cached[*dev], cudaDevAttrMultiProcessorCount, *dev);
+    if (err != cudaSuccess) return err;
+  }
+  *sms = cached[*dev];
+  return cudaSuccess;
+}
+// Raises a kernel's dynamic shared memory limit when a launch needs more than any before it.
+#define SQ_ENSURE_SMEM(KERNEL_, DEV_, BYTES_)                                                        \
+  do {                                                                                               \
+    static size_t limit_[64] = {0};                                                                  \
+    if ((BYTES_) > limit_[DEV_]) {                                                                   \
+      err = cudaFuncSetAttribute(KERNEL_, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(BYTES_)); \
+      if (err != cudaSuccess) return err;                                                            \
+      limit_[DEV_] = (BYTES_);                                                                       \
+    }                                                                                                \
+  } while (0)
+
 template <int B, int KK>
 cudaError_t launch_rows(const EncodeParams& base, cudaStream_t st) {
   EncodeParams p = base;
@@ -961,12 +986,9 @@ cudaError_t launch_rows(const EncodeParams& base, cudaStream_t st) {
   const size_t smem = table + per_group * ngroups;
 
   int dev = 0, sms = 0;
-  cudaError_t err = cudaGetDevice(&dev);
+  cudaError_t err = device_and_sms(&dev, &sms);
   if (err != cudaSuccess) return err;
-  err = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-  if (err != cudaSuccess) return err;
-  err = cudaFuncSetAttribute(encode_rows_kernel<B, KK>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-  if (err != cudaSuccess) return err;
+  SQ_ENSURE_SMEM((encode_rows_kernel<B, KK>), dev, smem);
   int64_t blocks = (p.M + ngroups - 1) / ngroups;
   if (blocks > sms) blocks = sms;
   encode_rows_kernel<B, KK><<<(unsigned)blocks, ngroups * rw * 32, smem, st>>>(p);
@@ -985,12 +1007,9 @@ cudaError_t launch_static_regs_as(EncodeParams p, int rw, cudaStream_t st) {
   if (smem > 200 * 1024) return cudaErrorNotSupported;
   p.rw = rw;
   int dev = 0, sms = 0;
-  cudaError_t err = cudaGetDevice(&dev);
+  cudaError_t err = device_and_sms(&dev, &sms);
   if (err != cudaSuccess) return err;
-  err = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-  if (err != cudaSuccess) return err;
-  err = cudaFuncSetAttribute(encode_static_regs_kernel<NCL, NT, INDEP>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-  if (err != cudaSuccess) return err;
+  SQ_ENSURE_SMEM((encode_static_regs_kernel<NCL, NT, INDEP>), dev, smem);
   int64_t blocks = (p.M + ngroups - 1) / ngroups;
   if (blocks > sms) blocks = sms;
   encode_static_regs_kernel<NCL, NT, INDEP><<<(unsigned)blocks, NT, smem, st>>>(p);
@@ -1019,8 +1038,10 @@ template <int B>
 cudaError_t launch_generic(int k, bool is_static, bool indep, const uint16_t* X, int64_t M, int64_t K,
                            const uint8_t* positions, const sq_encoded& out, cudaStream_t st) {
   const size_t smem = (size_t)K * 2;
-  cudaError_t err = cudaFuncSetAttribute(encode_generic_kernel<B>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  int dev = 0, sms = 0;
+  cudaError_t err = device_and_sms(&dev, &sms);
   if (err != cudaSuccess) return err;
+  SQ_ENSURE_SMEM((encode_generic_kernel<B>), dev, smem);
   encode_generic_kernel<B><<<(unsigned)M, 256, smem, st>>>(k, is_static, indep, X, K, positions, out.dq4, out.vals, out.idx,
                                                           out.s_hi, out.s_lo, out.shift);
   return cudaGetLastError();

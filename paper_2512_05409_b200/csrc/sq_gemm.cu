@@ -1345,10 +1345,14 @@ cudaError_t launch_gemm(int b, int k, bool indep, const sq_encoded& A, const sq_
 
 #define SQ_LAUNCH_GEMM(PAIR_, MODE_, SPLIT_)                                                                \
   do {                                                                                                      \
-    err = cudaFuncSetAttribute(gemm_kernel<PAIR_, MODE_, SPLIT_>,                                           \
-                               cudaFuncAttributeMaxDynamicSharedMemorySize,                                 \
-                               Geo<PAIR_, MODE_>::kSmemBytes);                                                     \
-    if (err != cudaSuccess) return err;                                                                     \
+    static bool attr_set_[64] = {false}; /* once per kernel variant and device */                          \
+    if (!attr_set_[dev]) {                                                                                  \
+      err = cudaFuncSetAttribute(gemm_kernel<PAIR_, MODE_, SPLIT_>,                                         \
+                                 cudaFuncAttributeMaxDynamicSharedMemorySize,                               \
+                                 Geo<PAIR_, MODE_>::kSmemBytes);                                            \
+      if (err != cudaSuccess) return err;                                                                   \
+      attr_set_[dev] = true;                                                                                \
+    }                                                                                                       \
     cudaLaunchConfig_t lc;                                                                                  \
     memset(&lc, 0, sizeof(lc));                                                                             \
     cudaLaunchAttribute la[1];                                                                              \
