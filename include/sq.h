@@ -186,7 +186,10 @@ sq_status sq_encode(const sq_format* fmt, const void* X_bf16, int64_t M, int64_t
  * positions: static formats only (the mask the two were built with), else NULL.
  * out_bf16: device bf16 [M, N], written.  acc_out: device int32 [M, N] or NULL; when
  * given, the raw accumulators are written as well (used by parity tests);
- * SQ_POS_STATIC_INDEP: [2, M, N], acc_lo then acc_hi. */
+ * SQ_POS_STATIC_INDEP: [2, M, N], acc_lo then acc_hi.
+ * Few rows (M <= 128): K is cut into 2-8 parts that run as one thread-block cluster per tile of
+ * 256 output channels and add their integer partial sums through distributed shared memory
+ * (no scratch memory; the result does not depend on the number of parts). */
 sq_status sq_gemm(const sq_format* fmt, const sq_encoded* A, const sq_weights* W,
                   const uint8_t* positions, int64_t M, int64_t N, int64_t K, void* out_bf16,
                   int32_t* acc_out, void* cuda_stream);

@@ -156,7 +156,8 @@ struct GemmParams {
   uint16_t* out;
   int32_t* acc_out;
   int* status;
-  int32_t* ws;     // split-K: raw partial accumulators [splits][M][N], else nullptr
+  int32_t* ws;     // split-K: raw partial accumulators [splits][M][N]; nullptr: the parts of a tile form a
+                   // thread-block cluster and add their partial sums through distributed shared memory
   int M, N, K, b, k;
   int log2k;       // log2(k) when the word path is usable, else -1
   int SS;          // sparse K steps per tile (static positions through TMA), else 0
@@ -195,9 +196,9 @@ __device__ __forceinline__ Tile tile_of(const GemmParams& p, int j, int rank) {
     } else {  // the odd last row unit (with split-K: `splits` work items per column tile)
       const int q = s - p.n_split;
       t.m0 = (p.mu - 1) * U;
-      if (SPLITK) {
-        t.n0 = (q % p.tiles_n) * BN;
-        t.split = q / p.tiles_n;
+      if (SPLITK) {  // the parts of a tile are neighbours in the work list (= one cluster, if clustered)
+        t.n0 = (q / p.splits) * BN;
+        t.split = q % p.splits;
       } else {
         t.n0 = q * BN;
       }
@@ -457,6 +458,19 @@ __global__ void __launch_bounds__(threads_of(MODE), 1)
               }
             }
           }
+        }
+      } else if (SPLITK && p.ws == nullptr) {
+        // clustered split-K: this CTA's raw partial sums go to its own shared memory (the operand
+        // rings are idle by now: a CTA has a single work item), row-major [128][256] int32 with
+        // the 16-byte chunks of a row XOR-swizzled by the row so that a warp's stores (one row
+        // per lane) spread over the banks; the cluster adds them at the end of the kernel
+        if (m < p.M) {
+          const int r = 32 * q + lane;
+          uint8_t* prow = smem + (size_t)r * (BN * 4);
+#pragma unroll
+          for (int c4 = 0; c4 < 8; ++c4)
+            *reinterpret_cast<int4*>(prow + ((((c0 >> 2) + c4) ^ (r & 7)) << 4)) =
+                make_int4((int)v[4 * c4], (int)v[4 * c4 + 1], (int)v[4 * c4 + 2], (int)v[4 * c4 + 3]);
         }
       } else if (SPLITK) {
         // split-K: this work item's raw partial sums; splitk_finish_kernel adds the parts
@@ -1012,6 +1026,56 @@ __global__ void __launch_bounds__(threads_of(MODE), 1)
   // Neither CTA of a pair may leave (or free tensor memory) while the other can still arrive on
   // its barriers or have MMAs reading its shared memory.
   if (PAIR == 2) cluster_sync_all();
+  if (SPLITK && PAIR == 1 && p.ws == nullptr) {
+    // Clustered split-K: the cluster's CTAs hold the parts of one column tile.  Every thread of
+    // every CTA gets here, whatever happened before (an aborted wait only leaves garbage to
+    // add), so the two cluster barriers cannot be missed by anyone.  CTA r of the cluster then
+    // adds all parts of its share of the columns, read from the peers' shared memory, and runs
+    // the same epilogue arithmetic as the one-kernel path (integer sums: order-free).
+    cluster_sync_all();
+    const int parts = p.splits, r = (int)cluster_ctarank();
+    const int n_tile = ((int)blockIdx.x / parts) * BN;
+    const int m_base = (p.mu - 1) * BM;               // the (only) row unit of a few-row launch
+    const int groups_per_row = (BN / 8) / parts;      // groups of eight columns in this CTA's share
+    const int rows = p.M - m_base;
+    for (int g = tid; g < rows * groups_per_row; g += (int)blockDim.x) {
+      const int row = g / groups_per_row, g8 = r * groups_per_row + g % groups_per_row;
+      const int m = m_base + row, n = n_tile + 8 * g8;
+      if (n >= p.N) continue;
+      int v[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+      const uint32_t base = smem_u32(smem) + (uint32_t)row * (BN * 4);
+      for (int sp = 0; sp < parts; ++sp) {
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          const uint32_t laddr = base + (uint32_t)(((2 * g8 + h) ^ (row & 7)) << 4);
+          int4 a;
+          asm volatile(
+              "{\n\t.reg .b32 ra;\n\t"
+              "mapa.shared::cluster.u32 ra, %4, %5;\n\t"
+              "ld.shared::cluster.v4.s32 {%0, %1, %2, %3}, [ra];\n\t}"
+              : "=r"(a.x), "=r"(a.y), "=r"(a.z), "=r"(a.w)
+              : "r"(laddr), "r"(sp)
+              : "memory");
+          v[4 * h] += a.x; v[4 * h + 1] += a.y; v[4 * h + 2] += a.z; v[4 * h + 3] += a.w;
+        }
+      }
+      const float sh = p.s_hi[m];
+      int acc[8];
+      uint32_t o[4];
+#pragma unroll
+      for (int c = 0; c < 8; ++c) acc[c] = (v[c] - 2048 * p.colsum[n + c]) >> 4;
+#pragma unroll
+      for (int c = 0; c < 8; c += 2)
+        o[c >> 1] = pack_bf16x2(((float)acc[c] * sh) * p.s_w[n + c], ((float)acc[c + 1] * sh) * p.s_w[n + c + 1]);
+      *reinterpret_cast<uint4*>(p.out + (size_t)m * p.N + n) = make_uint4(o[0], o[1], o[2], o[3]);
+      if (p.acc_out != nullptr) {
+        int4* dst = reinterpret_cast<int4*>(p.acc_out + (size_t)m * p.N + n);
+        dst[0] = make_int4(acc[0], acc[1], acc[2], acc[3]);
+        dst[1] = make_int4(acc[4], acc[5], acc[6], acc[7]);
+      }
+    }
+    cluster_sync_all();  // nobody leaves while a peer may still read its partial sums
+  }
   if (tid == 0 && *abort_flag) atomicExch(p.status, (int)SQ_ERR_TIMEOUT);
   if (warp == kMmaWarp) tmem_dealloc<PAIR>(tmem, 2 * BN);
 #undef rank
@@ -1256,12 +1320,53 @@ cudaError_t launch_gemm(int b, int k, bool indep, const sq_encoded& A, const sq_
   p.splits = 1;
   p.ws = nullptr;
   p.KS = (int)(K / BK);
+  int cluster_x = pair;  // CTAs per thread-block cluster
   if (pair == 1 && workspace != nullptr) {
     const int sp = choose_splits(M, N, K, sm_count[dev], workspace_bytes);
     if (sp > 1) {
       p.splits = sp;
       p.ws = static_cast<int32_t*>(workspace);
       p.KS = (int)(K / BK / sp);
+    }
+  } else if (pair == 1 && !indep) {
+    // No workspace: the parts of a column tile run as one thread-block cluster and add their
+    // partial sums through distributed shared memory at the end of the kernel (no second kernel).
+    // The largest cluster size whose clusters can ALL be resident at once (a cluster needs its
+    // SMs inside one GPC, so fewer clusters of 8 fit than SMs / 8; a second wave would cost more
+    // than the longer K walk of a smaller cluster).
+    static int resident[64][3][4] = {{{0}}};  // per device, kernel variant, log2(cluster size): 0 = not asked yet
+    const int variant = mode == kModeTma ? 0 : (mode == kModeMergeProd ? 1 : 2);
+    const int64_t tiles_n = (N + BN - 1) / BN, ks = K / BK;
+    for (int sp = 8, lg = 3; sp >= 2; sp /= 2, --lg) {
+      if (tiles_n * sp > sm_count[dev] || ks % sp != 0 || ks / sp < 2) continue;
+      if (resident[dev][variant][lg] == 0) {
+        cudaLaunchConfig_t qc;
+        memset(&qc, 0, sizeof(qc));
+        cudaLaunchAttribute qa[1];
+        qa[0].id = cudaLaunchAttributeClusterDimension;
+        qa[0].val.clusterDim.x = (unsigned)sp;
+        qa[0].val.clusterDim.y = 1;
+        qa[0].val.clusterDim.z = 1;
+        qc.gridDim = dim3((unsigned)(sm_count[dev] / sp * sp), 1, 1);
+        qc.blockDim = dim3(kThreads, 1, 1);
+        qc.dynamicSmemBytes = Geo<1>::kSmemBytes;
+        qc.attrs = qa;
+        qc.numAttrs = 1;
+        const void* fn = variant == 0 ? (const void*)gemm_kernel<1, kModeTma, true>
+                         : variant == 1 ? (const void*)gemm_kernel<1, kModeMergeProd, true>
+                                        : (const void*)gemm_kernel<1, kModeMergeEpi, true>;
+        int n = 0;
+        err = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, Geo<1>::kSmemBytes);
+        if (err == cudaSuccess) err = cudaOccupancyMaxActiveClusters(&n, fn, &qc);
+        if (err != cudaSuccess) return err;
+        resident[dev][variant][lg] = n > 0 ? n : -1;
+      }
+      if (resident[dev][variant][lg] >= tiles_n) {
+        p.splits = sp;
+        p.KS = (int)(ks / sp);
+        cluster_x = sp;
+        break;
+      }
     }
   }
   p.n_singles = p.n_split + (p.mu & 1) * p.tiles_n * p.splits;
@@ -1357,7 +1462,7 @@ cudaError_t launch_gemm(int b, int k, bool indep, const sq_encoded& A, const sq_
     memset(&lc, 0, sizeof(lc));                                                                             \
     cudaLaunchAttribute la[1];                                                                              \
     la[0].id = cudaLaunchAttributeClusterDimension;                                                         \
-    la[0].val.clusterDim.x = PAIR_;                                                                         \
+    la[0].val.clusterDim.x = (unsigned)cluster_x;                                                           \
     la[0].val.clusterDim.y = 1;                                                                             \
     la[0].val.clusterDim.z = 1;                                                                             \
     lc.gridDim = dim3(grid, 1, 1);                                                                          \
@@ -1365,7 +1470,7 @@ cudaError_t launch_gemm(int b, int k, bool indep, const sq_encoded& A, const sq_
     lc.dynamicSmemBytes = Geo<PAIR_, MODE_>::kSmemBytes;                                                           \
     lc.stream = st;                                                                                         \
     lc.attrs = la;                                                                                          \
-    lc.numAttrs = (PAIR_ == 2) ? 1 : 0;                                                                     \
+    lc.numAttrs = cluster_x > 1 ? 1 : 0;                                                                    \
     err = cudaLaunchKernelEx(&lc, gemm_kernel<PAIR_, MODE_, SPLIT_>, p, map_a, map_b, map_a4, map_b4);      \
     if (err != cudaSuccess) return err;                                                                     \
   } while (0)
@@ -1387,7 +1492,7 @@ cudaError_t launch_gemm(int b, int k, bool indep, const sq_encoded& A, const sq_
     else SQ_LAUNCH_GEMM(1, kModeMergeEpi, false);
   }
 #undef SQ_LAUNCH_GEMM
-  if (p.splits > 1) {
+  if (p.splits > 1 && p.ws != nullptr) {
     const int64_t groups = M * (N / 8);
     int64_t blocks = (groups + 255) / 256;
     if (blocks > 8 * (int64_t)sm_count[dev]) blocks = 8 * (int64_t)sm_count[dev];

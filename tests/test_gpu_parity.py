@@ -280,7 +280,9 @@ def test_static_encode_row_slices_in_registers(K, b, k):
 @pytest.mark.parametrize("M,K", [(1, 1024), (64, 2048), (128, 1536), (17, 4096)])
 def test_split_k_with_workspace(b, k, static, M, K):
     """sq_gemm_ws with a workspace (K cut into parts + finishing kernel) against the oracle and,
-    bit for bit, against the call without a workspace."""
+    bit for bit, against the call without a workspace (K cut into parts that run as one
+    thread-block cluster per column tile and add their partial sums through distributed shared
+    memory)."""
     N = 520                       # three column tiles, the last one ragged
     fmt = sq.make_format(b, k, static)
     X = gen.activations(M, K, seed=M + K, outlier_fraction=0.01, outlier_scale=20.0, device="cuda")
