@@ -575,7 +575,8 @@ __global__ void __launch_bounds__(threads_of(MODE), 1)
         for (int u = 0; u < 4; ++u) pm_bank4[w] |= (uint32_t)(((4 * w + u) >> p.log2k) * p.b) << (8 * u);
     }
     auto sparse_fetch = [&](const Tile& ft, int fks) {
-      const int m = min(ft.m0 + 32 * pw + lane, p.M - 1);
+      if (ft.m0 + 32 * pw + lane >= p.M) return;  // a row past M is not merged
+      const int m = ft.m0 + 32 * pw + lane;
       const size_t o = (size_t)m * (size_t)GKp + (size_t)fks * 16;
       const uint8_t* ip = p.idx != nullptr ? p.idx + o : p.pos + (size_t)fks * 16;
       // (volatile: issued here, a whole K step before their use)
@@ -629,6 +630,9 @@ __global__ void __launch_bounds__(threads_of(MODE), 1)
       if (has_a) {
 #pragma unroll
         for (int i = 0; i < kATasks; ++i) {
+          // eight rows that all lie past M (a launch of a few tokens: most of the tile) keep
+          // whatever the stage holds: their products are never stored
+          if (pt.m0 + kRowsPerWarp * pw + 8 * i >= p.M) continue;
           const uint32_t in[4] = {ra[i].x, ra[i].y, ra[i].z, ra[i].w};
           uint32_t ev[4], od[4];
 #pragma unroll
@@ -663,6 +667,7 @@ __global__ void __launch_bounds__(threads_of(MODE), 1)
       if (PMERGE && has_a) {
         __syncwarp();  // the warp's 32 rows are written: each lane now patches one of them
         const int row = 32 * pw + lane;
+        if (pt.m0 + row < p.M) {
         const uint32_t swz = 0x01010101u * (uint32_t)((row & 7) << 4);
         uint8_t* rowp = a_st + row * 128;
         const uint32_t vw[4] = {crv.x, crv.y, crv.z, crv.w};
@@ -673,6 +678,7 @@ __global__ void __launch_bounds__(threads_of(MODE), 1)
           const uint32_t vx = vw[w] ^ 0x80808080u;
 #pragma unroll
           for (int u = 0; u < 4; ++u) rowp[(pos4 >> (8 * u)) & 0xFFu] = (uint8_t)(vx >> (8 * u));
+        }
         }
       }
       // The packed stage goes back to the TMA thread only now: shared-memory loads are
