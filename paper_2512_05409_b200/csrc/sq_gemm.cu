@@ -72,13 +72,12 @@
 
 #include "sq_host.h"
 
+// How the producers wait for a packed stage to land / a widened stage to be consumed: parked by
+// the hardware (idle producers must not take issue slots from the epilogue warps); the TMA
+// threads (one lane each) poll.
 #define WAIT_PE mbar_wait_park
 #define WAIT_PF mbar_wait_park
-#ifdef PARK_T
-#define WAIT_T mbar_wait_park
-#else
 #define WAIT_T mbar_wait
-#endif
 namespace sq {
 
 namespace {
