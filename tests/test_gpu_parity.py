@@ -315,7 +315,7 @@ def test_split_k_with_workspace(b, k, static, M, K):
 # ----------------------------------------------------------------------------- many rows: pre-widened activations
 
 @pytest.mark.parametrize("b,k,static", [(64, 8, False), (32, 1, False), (128, 64, False), (128, 16, True), (64, 4, True)])
-@pytest.mark.parametrize("M,K", [(200, 384), (513, 1024)])
+@pytest.mark.parametrize("M,K", [(200, 384), (513, 1024), (300, 128)])
 def test_prewidened_activations_with_workspace(b, k, static, M, K):
     """sq_gemm_ws with M*K bytes of workspace (activations expanded once into 8-bit tensor-core
     operands) against the oracle and, bit for bit, against the calls without or with too little
