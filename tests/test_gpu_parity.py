@@ -424,3 +424,30 @@ def test_indep_gemm_rejects_what_it_cannot_run():
     assert e.value.status == sq.SQ_ERR_UNSUPPORTED
     with pytest.raises(ValueError):
         sq.make_format(64, 8, False, independent_scales=True)
+
+
+@pytest.mark.parametrize("static", [False, True])
+@pytest.mark.parametrize("M,N,K", [(128, 8, 2048), (3, 264, 512), (100, 1032, 1024), (16, 2048, 4096)])
+def test_few_rows_without_workspace(static, M, N, K):
+    """Plain sq_gemm at M <= 128: K cut into parts that form one thread-block cluster per column
+    tile (clusters of 2, 4 and 8; one, two, five and eight tiles, with ragged edges)."""
+    b, k = 64, 8
+    fmt = sq.make_format(b, k, static)
+    X = gen.activations(M, K, seed=M + N, outlier_fraction=0.01, outlier_scale=20.0, device="cuda")
+    W = gen.weights(N, K, seed=N + K, device="cuda")
+    pos = pos_ref = None
+    if static:
+        pos = sq.sq_calib_positions(fmt, gen.calibration_batch(64, K, seed=K, device="cuda"), W)
+        pos_ref = _np(pos)
+    w = sq.sq_pack_weights(fmt, W, pos)
+    enc = sq.sq_encode(fmt, X, pos)
+    acc = torch.empty(M, N, dtype=torch.int32, device="cuda")
+    out = sq.sq_gemm(fmt, enc, w, pos, acc_out=acc, use_workspace=False)
+    again = sq.sq_gemm(fmt, enc, w, pos, use_workspace=False).clone()
+    check_status()
+    enc_ref = oracle.encode(b, k, _bits(X), pos_ref)
+    w_ref = oracle.pack_weights(b, k, _bits(W), pos_ref)
+    acc_ref, ref32, out_ref = oracle.gemm(b, k, enc_ref, w_ref, pos_ref)
+    assert np.array_equal(_np(acc), acc_ref)
+    assert_bf16_close(out, ref32)
+    assert np.array_equal(_bits(out), out_ref) and torch.equal(out, again)
