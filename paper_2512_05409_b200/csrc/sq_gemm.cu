@@ -104,7 +104,6 @@ constexpr int kThreads = (kProdWarps + 1 + kEpiWarps + 3) * 32;
 // so four more warps (16..19) join it: two warps per tensor-memory lane quarter.
 constexpr int kEpiWarpsA8 = 8;
 constexpr int kThreadsA8 = kThreads + (kEpiWarpsA8 - kEpiWarps) * 32;
-constexpr int kStageA = 2 * BM * BK;  // 32 KB: two sub-tiles of A
 constexpr int kCtlBytes = 256;            // barriers, tensor-memory slot, abort flag
 constexpr int kEpiConstBytes = 2 * BN * 4;  // per tile: 2048 * colsum[n] and s_w[n] of its columns
 constexpr int kOutBlock = 32 * 32 * 2;        // one staged output block: 32 rows x 32 bf16
@@ -120,11 +119,15 @@ constexpr int kATasks = kRowsPerWarp / 8;  // 16-byte packed chunks of A per pro
 // its shared memory serves a third less operand traffic -- the pipe this kernel is bound by.
 template <int PAIR, int MODE = kModeTma>
 struct Geo {
-  // packed A per stage: 256 rows x 64 bytes; none when TMA delivers 8-bit activations
-  static constexpr int kPackA = MODE == kModeA8 ? 0 : 2 * BM * (BK / 2);
+  // rows of A per stage: two sub-tiles per CTA of a pair; a lone CTA (at most 128 rows in the
+  // whole launch) only ever has one, and the room goes to a third widened stage
+  static constexpr int kRowsA = PAIR == 1 ? BM : 2 * BM;
+  static constexpr int kStageA = kRowsA * BK;  // 16 / 32 KB widened
+  // packed A per stage: 64 bytes per row; none when TMA delivers 8-bit activations
+  static constexpr int kPackA = MODE == kModeA8 ? 0 : kRowsA * (BK / 2);
   // stages of widened (8-bit) operands; 8-bit activation tiles land there directly, so that ring
   // alone hides their latency and gets the room the packed A ring does not need
-  static constexpr int NS = PAIR == 2 ? (MODE == kModeA8 ? 4 : 3) : 2;
+  static constexpr int NS = PAIR == 2 ? (MODE == kModeA8 ? 4 : 3) : 3;
   // stages of packed (4-bit) operands as TMA delivers them (with 8-bit activations only weights
   // pass through them, and the third stage's room goes to the output staging below)
   static constexpr int NP = MODE == kModeA8 ? 2 : 3;
@@ -314,7 +317,7 @@ __global__ void __launch_bounds__(threads_of(MODE), 1)
   constexpr int kEpiAll = A8 ? kEpiWarpsA8 : kEpiHelpers;  // warps that read out a tile
   constexpr int kEpiStep = A8 ? kEpiWarpsA8 / 4 : kEpiStride;  // ... per tensor-memory lane quarter
   constexpr int NS = G::NS, NP = G::NP;
-  constexpr int kStageB = G::kStageB, kPackB = G::kPackB, kBTasks = G::kBTasks, kPackA = G::kPackA;
+  constexpr int kStageA = G::kStageA, kStageB = G::kStageB, kPackB = G::kPackB, kBTasks = G::kBTasks, kPackA = G::kPackA;
   // The kernel has no static shared memory, so the dynamic block starts at the 1024-byte
   // aligned base the swizzled operand layout needs; checked below, never assumed.
   extern __shared__ __align__(1024) uint8_t smem_raw[];
@@ -324,7 +327,7 @@ __global__ void __launch_bounds__(threads_of(MODE), 1)
     if (threadIdx.x == 0) atomicExch(p.status, (int)SQ_ERR_CUDA);
     return;
   }
-  uint8_t* sA = smem;                      // NS x [256][128] widened A
+  uint8_t* sA = smem;                      // NS x [kRowsA][128] widened A
   uint8_t* sB = sA + NS * kStageA;         // NS x [BNL][128] widened B
   uint8_t* sPA = sB + NS * kStageB;        // NP x [256][64]  packed A as loaded
   uint8_t* sPB = sPA + NP * kPackA;        // NP x [BNL][64]  packed B as loaded
@@ -608,7 +611,7 @@ __global__ void __launch_bounds__(threads_of(MODE), 1)
       const uint8_t* pa = sPA + ps * kPackA + prow0;
       const uint8_t* pb = sPB + ps * kPackB + prowb0;
 #pragma unroll
-      for (int i = 0; i < kATasks; ++i) ra[i] = *reinterpret_cast<const uint4*>(pa + i * 512);
+      for (int i = 0; i < kATasks; ++i) ra[i] = has_a ? *reinterpret_cast<const uint4*>(pa + i * 512) : make_uint4(0, 0, 0, 0);
 #pragma unroll
       for (int i = 0; i < kBTasks; ++i) rb[i] = *reinterpret_cast<const uint4*>(pb + i * 512);
       ++pit;
@@ -1399,7 +1402,7 @@ cudaError_t launch_gemm(int b, int k, bool indep, const sq_encoded& A, const sq_
     const cuuint64_t pitch4[1] = {(cuuint64_t)(K / 2)};
     const cuuint64_t dim_a4[2] = {(cuuint64_t)(K / 2), (cuuint64_t)M};
     const cuuint64_t dim_b4[2] = {(cuuint64_t)(K / 2), (cuuint64_t)N};
-    const cuuint32_t box4[2] = {BK / 2, 2 * BM};
+    const cuuint32_t box4[2] = {BK / 2, (cuuint32_t)(pair == 1 ? BM : 2 * BM)};
     const cuuint32_t box4b[2] = {BK / 2, (cuuint32_t)(BN / pair)};
     if (encode(&map_a4, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, A.dq4, dim_a4, pitch4, box4, estr,
                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
@@ -1415,7 +1418,7 @@ cudaError_t launch_gemm(int b, int k, bool indep, const sq_encoded& A, const sq_
     const cuuint64_t pitch[1] = {(cuuint64_t)GK};
     const cuuint64_t dim_a[2] = {(cuuint64_t)GK, (cuuint64_t)M};
     const cuuint64_t dim_b[2] = {(cuuint64_t)GK, (cuuint64_t)N};
-    const cuuint32_t box_a[2] = {BK, 2 * BM};
+    const cuuint32_t box_a[2] = {BK, (cuuint32_t)(pair == 1 ? BM : 2 * BM)};
     const cuuint32_t box_b[2] = {BK, (cuuint32_t)(BN / pair)};
     if (encode(&map_a, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<int8_t*>(A.vals), dim_a, pitch, box_a, estr,
                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
