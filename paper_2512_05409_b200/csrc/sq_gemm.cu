@@ -169,6 +169,8 @@ struct GemmParams {
   // a row unit is 128 rows per CTA of the pair (128 or 256 rows)
   int n_pairs, n_singles, n_split;  // n_split: singles that come from cutting pair tiles in two
   int mp, mu, tiles_n;              // row pairs, row units, column tiles
+  int rows_a;                       // rows the activation TMA boxes fetch (a lone CTA: M rounded up to 8, so
+                                    // that a few tokens do not cost the TMA unit 128 row requests per step)
 };
 
 struct Tile {
@@ -807,7 +809,7 @@ __global__ void __launch_bounds__(threads_of(MODE), 1)
           ok = WAIT_T(bar_pempty + 8 * ps, ((pit / NP) & 1u) ^ 1u, abort_flag);
           if (!ok) break;
           // rows past M / N come back as zeros (code 0)
-          mbar_expect_tx(bar_pfull + 8 * ps, (uint32_t)((A8 ? 0 : kPackA) + kPackB));
+          mbar_expect_tx(bar_pfull + 8 * ps, (uint32_t)((A8 ? 0 : p.rows_a * (BK / 2)) + kPackB));
           if (!A8) tma_load_2d(smem_u32(sPA + ps * kPackA), &map_a4, (t.k0 + ks) * (BK / 2), t.m0, bar_pfull + 8 * ps);
           tma_load_2d(smem_u32(sPB + ps * kPackB), &map_b4, (t.k0 + ks) * (BK / 2), t.nb0, bar_pfull + 8 * ps);
         }
@@ -870,7 +872,7 @@ __global__ void __launch_bounds__(threads_of(MODE), 1)
             if (step < KS) continue;
             const int ss = step - KS;
             // rows past M / N and columns past G*k are filled with zeros by the TMA unit
-            mbar_expect_tx(bar_sfull + 8 * s, (uint32_t)(kStageA + kStageB));
+            mbar_expect_tx(bar_sfull + 8 * s, (uint32_t)(p.rows_a * BK + kStageB));
             tma_load_2d(smem_u32(sA + s * kStageA), &map_a, ss * BK, t.m0, bar_sfull + 8 * s);
             tma_load_2d(smem_u32(sB + s * kStageB), &map_b, ss * BK, t.nb0, bar_sfull + 8 * s);
           }
@@ -1308,6 +1310,7 @@ cudaError_t launch_gemm(int b, int k, bool indep, const sq_encoded& A, const sq_
   // remainder of the row pairs is cut into tiles of one row unit so the last wave spreads over
   // twice as many slots.  (Row unit: 128 rows per CTA of the tile.)
   const int U = BM * pair;
+  p.rows_a = pair == 1 ? (int)((M + 7) / 8 * 8) : 2 * BM;
   p.mu = (int)((M + U - 1) / U);
   p.mp = p.mu / 2;
   p.tiles_n = (int)((N + BN - 1) / BN);
@@ -1402,7 +1405,7 @@ cudaError_t launch_gemm(int b, int k, bool indep, const sq_encoded& A, const sq_
     const cuuint64_t pitch4[1] = {(cuuint64_t)(K / 2)};
     const cuuint64_t dim_a4[2] = {(cuuint64_t)(K / 2), (cuuint64_t)M};
     const cuuint64_t dim_b4[2] = {(cuuint64_t)(K / 2), (cuuint64_t)N};
-    const cuuint32_t box4[2] = {BK / 2, (cuuint32_t)(pair == 1 ? BM : 2 * BM)};
+    const cuuint32_t box4[2] = {BK / 2, (cuuint32_t)p.rows_a};
     const cuuint32_t box4b[2] = {BK / 2, (cuuint32_t)(BN / pair)};
     if (encode(&map_a4, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, A.dq4, dim_a4, pitch4, box4, estr,
                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
@@ -1418,7 +1421,7 @@ cudaError_t launch_gemm(int b, int k, bool indep, const sq_encoded& A, const sq_
     const cuuint64_t pitch[1] = {(cuuint64_t)GK};
     const cuuint64_t dim_a[2] = {(cuuint64_t)GK, (cuuint64_t)M};
     const cuuint64_t dim_b[2] = {(cuuint64_t)GK, (cuuint64_t)N};
-    const cuuint32_t box_a[2] = {BK, (cuuint32_t)(pair == 1 ? BM : 2 * BM)};
+    const cuuint32_t box_a[2] = {BK, (cuuint32_t)p.rows_a};
     const cuuint32_t box_b[2] = {BK, (cuuint32_t)(BN / pair)};
     if (encode(&map_a, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<int8_t*>(A.vals), dim_a, pitch, box_a, estr,
                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
