@@ -37,6 +37,15 @@
  *     out records SQ_ERR_TIMEOUT in a per-device status word (see sq_device_status)
  *     and the kernel returns after releasing its tensor memory.
  *   - No exceptions, no aborts, no printing.  The library needs an sm_100 device.
+ *   - Threads: every call may be made from any host thread, and calls may run concurrently
+ *     (the CUDA current device is the calling thread's, as for the CUDA runtime).  The library
+ *     keeps per-device host state of two kinds only: first-use caches (device attributes, kernel
+ *     attributes, symbol addresses; filled under a lock) and the device status word.  The first
+ *     call per device and kernel variant therefore costs more than later ones.  What the library
+ *     does NOT arbitrate is the GPU memory the caller passes in: calls that share an output, a
+ *     workspace or the static scratch array must be ordered on the GPU by the caller.
+ *   - Size limits beyond the shape rules (SQ_ERR_UNSUPPORTED): K <= SQ_MAX_K everywhere; for the
+ *     GEMM calls M*K/2, N*K/2 and M*(K/b)*k must each stay below 2^32 bytes and M below 2^23.
  *
  * Number formats (layout version 1)
  *   - INT4 codes are symmetric in [-7, 7] and INT8 codes in [-127, 127]: the most
@@ -250,6 +259,12 @@ sq_status sq_decode(const sq_format* fmt, const sq_encoded* A, const uint8_t* po
  * SQ_OK, SQ_ERR_TIMEOUT if a kernel gave up on a bounded wait since the last call
  * (its outputs are then undefined), or SQ_ERR_CUDA if the stream reports an error. */
 sq_status sq_device_status(void* cuda_stream);
+
+/* Device address of the current device's status word (an int: 0, or the sq_status a kernel
+ * recorded), for callers that watch it without synchronising a stream, e.g. with their own
+ * asynchronous copy at the end of a batch.  The word belongs to the library; sq_device_status
+ * remains the call that clears it.  *device_word is a DEVICE pointer. */
+sq_status sq_device_status_word(int** device_word);
 
 #ifdef __cplusplus
 }

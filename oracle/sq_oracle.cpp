@@ -141,10 +141,8 @@ void sqo_calib_positions(int b, int k, const uint16_t* calib, long T, long K,
 //   wq   = clamp(RNE(W[n,j] * c), -7, 7); zero channel -> codes 0, s_w = 0
 //   wq4[n, j/2]: element 2*(j/2) in the low nibble, the next one in the high
 //   nibble, two's complement; colsum[n] = sum_j wq
-//   static only: w_sparse[n, g*k+i] = 16 * wq[n, g*b + positions[g][i]]  (Alg. 2 reorder).
-//   Reading: the paper only says the rows are reordered by the mask; the gathered copy is
-//   kept in sixteenths (the code sits in the high nibble of its byte, |16*code| <= 112),
-//   the fixed-point unit the INT8 tensor-core operand of the GEMM uses for weights.
+//   static only: w_sparse[n, g*k+i] = wq[n, g*b + positions[g][i]]: the codes of the selected
+//   input channels gathered bank by bank, which is all Algorithm 2's "reorder" line states.
 void sqo_pack_weights(int b, int k, const uint16_t* W, long N, long K, const uint8_t* positions,
                       uint8_t* wq4, float* s_w, int32_t* colsum, int8_t* w_sparse /*or NULL*/,
                       int8_t* wq_plain /*[N,K] or NULL*/) {
@@ -173,7 +171,7 @@ void sqo_pack_weights(int b, int k, const uint16_t* W, long N, long K, const uin
     if (positions && w_sparse)
       for (long g = 0; g < G; ++g)
         for (int i = 0; i < k; ++i)
-          w_sparse[n * G * k + g * k + i] = (int8_t)(16 * q[g * b + positions[g * k + i]]);
+          w_sparse[n * G * k + g * k + i] = (int8_t)q[g * b + positions[g * k + i]];
   }
 }
 

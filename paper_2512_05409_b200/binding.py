@@ -73,9 +73,10 @@ def _load() -> ctypes.CDLL:
     lib.sq_gemm_static_scratch.argtypes = [P(sq_format), P(sq_encoded), P(sq_weights), VP, I64, I64, I64, VP, VP, VP]
     lib.sq_decode.argtypes = [P(sq_format), P(sq_encoded), VP, I64, I64, VP, VP]
     lib.sq_device_status.argtypes = [VP]
+    lib.sq_device_status_word.argtypes = [P(VP)]
     for name in ("sq_encoded_sizes", "sq_weights_sizes", "sq_calib_positions", "sq_pack_weights",
                  "sq_encode", "sq_gemm", "sq_gemm_ws", "sq_gemm_workspace_bytes", "sq_gemm_static_scratch", "sq_decode",
-                 "sq_device_status"):
+                 "sq_device_status", "sq_device_status_word"):
         getattr(lib, name).restype = ctypes.c_int
     return lib
 
@@ -314,6 +315,13 @@ def sq_decode(fmt: sq_format, A: Encoded, positions: torch.Tensor | None = None,
 
 def sq_device_status(stream=None) -> int:
     return int(_lib.sq_device_status(_stream(stream)))
+
+
+def sq_device_status_word() -> int:
+    """Device address of the current device's status word."""
+    out = ctypes.c_void_p(0)
+    _check(_lib.sq_device_status_word(ctypes.byref(out)), "sq_device_status_word")
+    return int(out.value)
 
 
 def raw():

@@ -9,13 +9,18 @@ __device__ int g_status_word;
 
 int* status_word() {
   // looked up once per device (the call is not free, and decode-sized launches are host-bound)
-  static int* cached[64] = {nullptr};
+  static std::atomic<int*> cached[64];
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) return nullptr;
-  if (dev >= 0 && dev < 64 && cached[dev] != nullptr) return cached[dev];
+  const bool slot = dev >= 0 && dev < 64;
+  if (slot) {
+    int* hit = cached[dev].load(std::memory_order_acquire);
+    if (hit != nullptr) return hit;
+  }
+  std::lock_guard<std::mutex> lock(setup_mutex());
   int* ptr = nullptr;
   if (cudaGetSymbolAddress(reinterpret_cast<void**>(&ptr), g_status_word) != cudaSuccess) return nullptr;
-  if (dev >= 0 && dev < 64) cached[dev] = ptr;
+  if (slot) cached[dev].store(ptr, std::memory_order_release);
   return ptr;
 }
 
@@ -44,12 +49,15 @@ sq_status check_k(int64_t K) {
 
 // The kernels are built for sm_100a only; refuse anything else before launching.
 sq_status check_device() {
-  static int major_of[64] = {0};  // per device, asked once
+  static std::atomic<int> major_of[64];  // per device, asked once
   int dev = 0, major = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) return SQ_ERR_CUDA;
-  if (dev >= 0 && dev < 64 && major_of[dev] != 0) return major_of[dev] == 10 ? SQ_OK : SQ_ERR_ARCH;
-  if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return SQ_ERR_CUDA;
-  if (dev >= 0 && dev < 64) major_of[dev] = major;
+  const bool slot = dev >= 0 && dev < 64;
+  if (slot) major = major_of[dev].load(std::memory_order_acquire);
+  if (major == 0) {
+    if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return SQ_ERR_CUDA;
+    if (slot) major_of[dev].store(major, std::memory_order_release);
+  }
   return major == 10 ? SQ_OK : SQ_ERR_ARCH;
 }
 
@@ -90,6 +98,13 @@ sq_status check_positions(const sq_format* fmt, const uint8_t* positions) {
 }
 
 sq_status from_cuda(cudaError_t err) { return err == cudaSuccess ? SQ_OK : SQ_ERR_CUDA; }
+
+// The GEMM kernels address the packed tensors with 32-bit byte offsets.
+sq_status check_gemm_extent(const sq_format* fmt, int64_t M, int64_t N, int64_t K) {
+  const int64_t lim = 1ll << 32;
+  if (M * (K / 2) >= lim || N * (K / 2) >= lim || M * ((K / fmt->bank) * fmt->k) >= lim) return SQ_ERR_UNSUPPORTED;
+  return SQ_OK;
+}
 
 }  // namespace
 }  // namespace sq
@@ -214,6 +229,7 @@ sq_status sq_gemm_ws(const sq_format* fmt, const sq_encoded* A, const sq_weights
   if (out_bf16 == nullptr) return SQ_ERR_NULL_POINTER;
   if (!aligned16(out_bf16) || !aligned16(acc_out) || !aligned16(workspace)) return SQ_ERR_ALIGNMENT;
   if ((M + 127) / 128 > 65535) return SQ_ERR_UNSUPPORTED;
+  SQ_TRY(check_gemm_extent(fmt, M, N, K));
   // independent scales: the sparse product runs as TMA-fed K steps of its own, whose row pitch
   // (G*k bytes) must be a multiple of 16
   if (is_indep(fmt) && ((K / fmt->bank) * fmt->k) % 16 != 0) return SQ_ERR_UNSUPPORTED;
@@ -235,6 +251,7 @@ sq_status sq_gemm_static_scratch(const sq_format* fmt, const sq_encoded* A, cons
   // Only the few-row case has a use for scratch, and at least two parts of K must fit.
   if (M > 128 || is_indep(fmt)) return SQ_ERR_UNSUPPORTED;
   if ((uint64_t)2 * (uint64_t)M * (uint64_t)N * 4u > (uint64_t)gemm_static_scratch_bytes()) return SQ_ERR_UNSUPPORTED;
+  SQ_TRY(check_gemm_extent(fmt, M, N, K));
   SQ_TRY(check_positions(fmt, positions));
   SQ_TRY(check_encoded(fmt, A));
   SQ_TRY(check_weights(fmt, W));
@@ -282,6 +299,14 @@ sq_status sq_device_status(void* cuda_stream) {
     return static_cast<sq_status>(word);
   }
   return SQ_OK;
+}
+
+
+sq_status sq_device_status_word(int** device_word) {
+  if (device_word == nullptr) return SQ_ERR_NULL_POINTER;
+  SQ_TRY(check_device());
+  *device_word = status_word();
+  return *device_word != nullptr ? SQ_OK : SQ_ERR_CUDA;
 }
 
 }  // extern "C"

@@ -141,8 +141,10 @@ __device__ __forceinline__ void cluster_sync_all() {
 constexpr uint32_t kSpinLimit = 1u << 24;
 constexpr uint32_t kIdleLimit = 1u << 21;
 
+// (The limits are template parameters so that a test can make a wait run out within microseconds.)
+template <uint32_t LIMIT = kSpinLimit>
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
-  for (uint32_t it = 0; it < kSpinLimit; ++it) {
+  for (uint32_t it = 0; it < LIMIT; ++it) {
     if (mbar_test(bar, parity)) return true;
     if ((it & 1023u) == 1023u && *abort_flag) return false;
   }
@@ -154,9 +156,10 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
 // for waits on data in flight from HBM, where a microsecond of wake-up slack costs nothing but
 // polling would take issue slots from the warps that have work.  Bounded like the others.
 constexpr uint32_t kParkTries = 1u << 17;
+template <uint32_t LIMIT = kParkTries>
 __device__ __forceinline__ bool mbar_wait_park(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
   if (mbar_test(bar, parity)) return true;
-  for (uint32_t it = 0; it < kParkTries; ++it) {
+  for (uint32_t it = 0; it < LIMIT; ++it) {
     if (mbar_try(bar, parity, 2000u)) return true;
     if (*abort_flag) return false;
   }
@@ -164,8 +167,9 @@ __device__ __forceinline__ bool mbar_wait_park(uint32_t bar, uint32_t parity, vo
   return false;
 }
 
+template <uint32_t LIMIT = kSpinLimit>
 __device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
-  for (uint32_t it = 0; it < kSpinLimit; ++it) {
+  for (uint32_t it = 0; it < LIMIT; ++it) {
     if (mbar_test_cluster(bar, parity)) return true;
     if ((it & 1023u) == 1023u && *abort_flag) return false;
   }
@@ -173,8 +177,9 @@ __device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity,
   return false;
 }
 
+template <uint32_t LIMIT = kIdleLimit>
 __device__ __forceinline__ bool mbar_wait_idle(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
-  for (uint32_t it = 0; it < kIdleLimit; ++it) {
+  for (uint32_t it = 0; it < LIMIT; ++it) {
     if (mbar_test(bar, parity)) return true;
     if (*abort_flag) return false;
     __nanosleep(100);

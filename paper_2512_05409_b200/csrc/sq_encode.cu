@@ -924,26 +924,32 @@ namespace {
 // The current device and its SM count (asked once per device: the encode of a few decode tokens
 // is bound by the host's launch path).
 static cudaError_t device_and_sms(int* dev, int* sms) {
-  static int cached[64] = {0};
+  static std::atomic<int> cached[64];
   cudaError_t err = cudaGetDevice(dev);
   if (err != cudaSuccess) return err;
   if (*dev < 0 || *dev >= 64) return cudaErrorInvalidDevice;
-  if (cached[*dev] == 0) {
-    err = cudaDeviceGetAttribute(&cached[*dev], cudaDevAttrMultiProcessorCount, *dev);
+  int n = cached[*dev].load(std::memory_order_acquire);
+  if (n == 0) {
+    err = cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, *dev);
     if (err != cudaSuccess) return err;
+    cached[*dev].store(n, std::memory_order_release);
   }
-  *sms = cached[*dev];
+  *sms = n;
   return cudaSuccess;
 }
-// Raises a kernel's dynamic shared memory limit when a launch needs more than any before it.
-#define SQ_ENSURE_SMEM(KERNEL_, DEV_, BYTES_)                                                        \
-  do {                                                                                               \
-    static size_t limit_[64] = {0};                                                                  \
-    if ((BYTES_) > limit_[DEV_]) {                                                                   \
-      err = cudaFuncSetAttribute(KERNEL_, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(BYTES_)); \
-      if (err != cudaSuccess) return err;                                                            \
-      limit_[DEV_] = (BYTES_);                                                                       \
-    }                                                                                                \
+// Raises a kernel's dynamic shared memory limit when a launch needs more than any before it
+// (the limit only ever grows, so a concurrent launch that needs less is never cut short).
+#define SQ_ENSURE_SMEM(KERNEL_, DEV_, BYTES_)                                                            \
+  do {                                                                                                   \
+    static std::atomic<size_t> limit_[64];                                                               \
+    if ((BYTES_) > limit_[DEV_].load(std::memory_order_acquire)) {                                       \
+      std::lock_guard<std::mutex> lock_(setup_mutex());                                                  \
+      if ((BYTES_) > limit_[DEV_].load(std::memory_order_relaxed)) {                                     \
+        err = cudaFuncSetAttribute(KERNEL_, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(BYTES_)); \
+        if (err != cudaSuccess) return err;                                                              \
+        limit_[DEV_].store((BYTES_), std::memory_order_release);                                         \
+      }                                                                                                  \
+    }                                                                                                    \
   } while (0)
 
 template <int B, int KK>
@@ -973,7 +979,7 @@ cudaError_t launch_rows(const EncodeParams& base, cudaStream_t st) {
     }
   }
   const size_t per_group = (((size_t)nbuf * row + extra) + 127) & ~(size_t)127;
-  if (per_group > 224 * 1024) return cudaErrorInvalidValue;
+  if (per_group > 224 * 1024) return cudaErrorNotSupported;
   int ngroups = kMaxWarps / rw;
   {
     const size_t fit = (208 * 1024 - table) / ((((size_t)nbuf * row + extra) + 127) & ~(size_t)127);
@@ -984,6 +990,7 @@ cudaError_t launch_rows(const EncodeParams& base, cudaStream_t st) {
   p.rw = rw;
   p.group_stride = (int)per_group;
   const size_t smem = table + per_group * ngroups;
+  if (smem > 227 * 1024) return cudaErrorNotSupported;  // long rows with many selected places: the plain kernel
 
   int dev = 0, sms = 0;
   cudaError_t err = device_and_sms(&dev, &sms);
@@ -1077,15 +1084,21 @@ cudaError_t launch_encode(int b, int k, bool is_static, bool indep, const uint16
     return launch_generic<128>(k, true, true, X, M, K, positions, out, st);
   }
   if (is_static) {
-    const cudaError_t err = launch_static_regs<false>(p, st);
+    cudaError_t err = launch_static_regs<false>(p, st);
     if (err != cudaErrorNotSupported) return err;
-    if (b == 32) return launch_rows<32, 0>(p, st);
-    if (b == 64) return launch_rows<64, 0>(p, st);
-    return launch_rows<128, 0>(p, st);
+    err = b == 32 ? launch_rows<32, 0>(p, st) : (b == 64 ? launch_rows<64, 0>(p, st) : launch_rows<128, 0>(p, st));
+    if (err != cudaErrorNotSupported) return err;
+    // a row, its offset table and its stash together exceed shared memory: one block per row
+    if (b == 32) return launch_generic<32>(k, true, false, X, M, K, positions, out, st);
+    if (b == 64) return launch_generic<64>(k, true, false, X, M, K, positions, out, st);
+    return launch_generic<128>(k, true, false, X, M, K, positions, out, st);
   }
   // dynamic fast kernels: k/b in {1/16, 1/8, 1/4, 1/2}
-#define SQ_DYN(BB, KK_) \
-  if (b == BB && k == KK_) return launch_rows<BB, KK_>(p, st);
+#define SQ_DYN(BB, KK_)                                       \
+  if (b == BB && k == KK_) {                                  \
+    const cudaError_t err = launch_rows<BB, KK_>(p, st);      \
+    if (err != cudaErrorNotSupported) return err;             \
+  }
   SQ_DYN(32, 2) SQ_DYN(32, 4) SQ_DYN(32, 8) SQ_DYN(32, 16)
   SQ_DYN(64, 4) SQ_DYN(64, 8) SQ_DYN(64, 16) SQ_DYN(64, 32)
   SQ_DYN(128, 8) SQ_DYN(128, 16) SQ_DYN(128, 32) SQ_DYN(128, 64)

@@ -1255,15 +1255,17 @@ cudaError_t launch_gemm(int b, int k, bool indep, const sq_encoded& A, const sq_
     p.log2k = l;
   }
 
-  static int sm_count[64] = {0};
-  static int pair_slots[64][5] = {{0}};  // CTA pairs that can be resident at once, per kernel variant
+  static std::atomic<int> sm_count_of[64];
+  static std::atomic<int> pair_slots[64][5];  // CTA pairs that can be resident at once, per kernel variant
   int dev = 0;
   cudaError_t err = cudaGetDevice(&dev);
   if (err != cudaSuccess) return err;
   if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
-  if (sm_count[dev] == 0) {
-    err = cudaDeviceGetAttribute(&sm_count[dev], cudaDevAttrMultiProcessorCount, dev);
+  int sms = sm_count_of[dev].load(std::memory_order_acquire);
+  if (sms == 0) {
+    err = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     if (err != cudaSuccess) return err;
+    sm_count_of[dev].store(sms, std::memory_order_release);
   }
   const bool stma = positions != nullptr && GK % 16 == 0;
   // 16 sparse entries per row and K step, fetched with aligned 16-byte loads: the producers merge
@@ -1276,9 +1278,10 @@ cudaError_t launch_gemm(int b, int k, bool indep, const sq_encoded& A, const sq_
   const int mode = indep ? kModeIndep : a8 ? kModeA8 : (stma ? kModeTma : (pmerge ? kModeMergeProd : kModeMergeEpi));
   // One CTA per tile for at most 128 rows (a second CTA would have no rows); CTA pairs otherwise.
   const int pair = M > BM ? 2 : 1;
-  int slots = sm_count[dev];  // tiles in flight at once
+  int slots = sms;  // tiles in flight at once
   if (pair == 2) {
-    if (pair_slots[dev][mode] == 0) {
+    if (pair_slots[dev][mode].load(std::memory_order_acquire) == 0) {
+      std::lock_guard<std::mutex> lock(setup_mutex());
       cudaLaunchConfig_t qc;
       memset(&qc, 0, sizeof(qc));
       cudaLaunchAttribute qa[1];
@@ -1286,7 +1289,7 @@ cudaError_t launch_gemm(int b, int k, bool indep, const sq_encoded& A, const sq_
       qa[0].val.clusterDim.x = 2;
       qa[0].val.clusterDim.y = 1;
       qa[0].val.clusterDim.z = 1;
-      qc.gridDim = dim3((unsigned)(sm_count[dev] & ~1), 1, 1);
+      qc.gridDim = dim3((unsigned)(sms & ~1), 1, 1);
       qc.blockDim = dim3(threads_of(mode), 1, 1);
       qc.dynamicSmemBytes = (mode == kModeA8 ? Geo<2, kModeA8>::kSmemBytes : Geo<2>::kSmemBytes);
       qc.attrs = qa;
@@ -1301,9 +1304,9 @@ cudaError_t launch_gemm(int b, int k, bool indep, const sq_encoded& A, const sq_
       if (err == cudaSuccess) err = cudaOccupancyMaxActiveClusters(&n, fn, &qc);
       if (err != cudaSuccess) return err;
       if (n < 1) return cudaErrorLaunchOutOfResources;
-      pair_slots[dev][mode] = n;
+      pair_slots[dev][mode].store(n, std::memory_order_release);
     }
-    slots = pair_slots[dev][mode];
+    slots = pair_slots[dev][mode].load(std::memory_order_acquire);
   }
 
   // Work list: tiles of two row units per CTA while they fill whole waves of the slots; the
@@ -1333,24 +1336,26 @@ cudaError_t launch_gemm(int b, int k, bool indep, const sq_encoded& A, const sq_
   p.KS = (int)(K / BK);
   int cluster_x = pair;  // CTAs per thread-block cluster
   if (pair == 1 && workspace != nullptr) {
-    const int sp = choose_splits(M, N, K, sm_count[dev], workspace_bytes);
+    const int sp = choose_splits(M, N, K, sms, workspace_bytes);
     if (sp > 1) {
       p.splits = sp;
       p.ws = static_cast<int32_t*>(workspace);
       p.KS = (int)(K / BK / sp);
     }
-  } else if (pair == 1 && !indep) {
+  }
+  if (pair == 1 && !indep && p.ws == nullptr) {  // also: a workspace too small for two parts
     // No workspace: the parts of a column tile run as one thread-block cluster and add their
     // partial sums through distributed shared memory at the end of the kernel (no second kernel).
     // The largest cluster size whose clusters can ALL be resident at once (a cluster needs its
     // SMs inside one GPC, so fewer clusters of 8 fit than SMs / 8; a second wave would cost more
     // than the longer K walk of a smaller cluster).
-    static int resident[64][3][4] = {{{0}}};  // per device, kernel variant, log2(cluster size): 0 = not asked yet
+    static std::atomic<int> resident[64][3][4];  // per device, kernel variant, log2(cluster size): 0 = not asked yet
     const int variant = mode == kModeTma ? 0 : (mode == kModeMergeProd ? 1 : 2);
     const int64_t tiles_n = (N + BN - 1) / BN, ks = K / BK;
     for (int sp = 8, lg = 3; sp >= 2; sp /= 2, --lg) {
-      if (tiles_n * sp > sm_count[dev] || ks % sp != 0 || ks / sp < 2) continue;
-      if (resident[dev][variant][lg] == 0) {
+      if (tiles_n * sp > sms || ks % sp != 0 || ks / sp < 2) continue;
+      if (resident[dev][variant][lg].load(std::memory_order_acquire) == 0) {
+        std::lock_guard<std::mutex> lock(setup_mutex());
         cudaLaunchConfig_t qc;
         memset(&qc, 0, sizeof(qc));
         cudaLaunchAttribute qa[1];
@@ -1358,7 +1363,7 @@ cudaError_t launch_gemm(int b, int k, bool indep, const sq_encoded& A, const sq_
         qa[0].val.clusterDim.x = (unsigned)sp;
         qa[0].val.clusterDim.y = 1;
         qa[0].val.clusterDim.z = 1;
-        qc.gridDim = dim3((unsigned)(sm_count[dev] / sp * sp), 1, 1);
+        qc.gridDim = dim3((unsigned)(sms / sp * sp), 1, 1);
         qc.blockDim = dim3(kThreads, 1, 1);
         qc.dynamicSmemBytes = Geo<1>::kSmemBytes;
         qc.attrs = qa;
@@ -1370,9 +1375,9 @@ cudaError_t launch_gemm(int b, int k, bool indep, const sq_encoded& A, const sq_
         err = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, Geo<1>::kSmemBytes);
         if (err == cudaSuccess) err = cudaOccupancyMaxActiveClusters(&n, fn, &qc);
         if (err != cudaSuccess) return err;
-        resident[dev][variant][lg] = n > 0 ? n : -1;
+        resident[dev][variant][lg].store(n > 0 ? n : -1, std::memory_order_release);
       }
-      if (resident[dev][variant][lg] >= tiles_n) {
+      if (resident[dev][variant][lg].load(std::memory_order_acquire) >= tiles_n) {
         p.splits = sp;
         p.KS = (int)(ks / sp);
         cluster_x = sp;
@@ -1390,7 +1395,8 @@ cudaError_t launch_gemm(int b, int k, bool indep, const sq_encoded& A, const sq_
   CUtensorMap map_a, map_b, map_a4, map_b4;
   memset(&map_a, 0, sizeof(map_a));
   memset(&map_b, 0, sizeof(map_b));
-  static PFN_cuTensorMapEncodeTiled encode = nullptr;
+  static std::atomic<PFN_cuTensorMapEncodeTiled> encode_fn{nullptr};
+  PFN_cuTensorMapEncodeTiled encode = encode_fn.load(std::memory_order_acquire);
   if (encode == nullptr) {
     void* fn = nullptr;
     cudaDriverEntryPointQueryResult qres;
@@ -1398,6 +1404,7 @@ cudaError_t launch_gemm(int b, int k, bool indep, const sq_encoded& A, const sq_
     if (err != cudaSuccess) return err;
     if (fn == nullptr || qres != cudaDriverEntryPointSuccess) return cudaErrorNotSupported;
     encode = reinterpret_cast<PFN_cuTensorMapEncodeTiled>(fn);
+    encode_fn.store(encode, std::memory_order_release);
   }
   const cuuint32_t estr[2] = {1, 1};
   {
@@ -1439,7 +1446,7 @@ cudaError_t launch_gemm(int b, int k, bool indep, const sq_encoded& A, const sq_
     uint8_t* a8buf = static_cast<uint8_t*>(workspace);
     const int64_t units = M * (K / 32);
     int64_t blocks = (units + 255) / 256;
-    if (blocks > 32 * (int64_t)sm_count[dev]) blocks = 32 * (int64_t)sm_count[dev];
+    if (blocks > 32 * (int64_t)sms) blocks = 32 * (int64_t)sms;
     expand_a8_kernel<<<(unsigned)blocks, 256, 0, st>>>(A.dq4, A.vals, positions == nullptr ? A.idx : nullptr, positions,
                                                       A.shift, M, (int)K, b, k, a8buf);
     const cuuint64_t pitch[1] = {(cuuint64_t)K};
@@ -1461,13 +1468,14 @@ cudaError_t launch_gemm(int b, int k, bool indep, const sq_encoded& A, const sq_
 
 #define SQ_LAUNCH_GEMM(PAIR_, MODE_, SPLIT_)                                                                \
   do {                                                                                                      \
-    static bool attr_set_[64] = {false}; /* once per kernel variant and device */                          \
-    if (!attr_set_[dev]) {                                                                                  \
+    static std::atomic<bool> attr_set_[64]; /* once per kernel variant and device */                       \
+    if (!attr_set_[dev].load(std::memory_order_acquire)) {                                                  \
+      std::lock_guard<std::mutex> lock_(setup_mutex());                                                     \
       err = cudaFuncSetAttribute(gemm_kernel<PAIR_, MODE_, SPLIT_>,                                         \
                                  cudaFuncAttributeMaxDynamicSharedMemorySize,                               \
                                  Geo<PAIR_, MODE_>::kSmemBytes);                                            \
       if (err != cudaSuccess) return err;                                                                   \
-      attr_set_[dev] = true;                                                                                \
+      attr_set_[dev].store(true, std::memory_order_release);                                                \
     }                                                                                                       \
     cudaLaunchConfig_t lc;                                                                                  \
     memset(&lc, 0, sizeof(lc));                                                                             \
@@ -1506,7 +1514,7 @@ cudaError_t launch_gemm(int b, int k, bool indep, const sq_encoded& A, const sq_
   if (p.splits > 1 && p.ws != nullptr) {
     const int64_t groups = M * (N / 8);
     int64_t blocks = (groups + 255) / 256;
-    if (blocks > 8 * (int64_t)sm_count[dev]) blocks = 8 * (int64_t)sm_count[dev];
+    if (blocks > 8 * (int64_t)sms) blocks = 8 * (int64_t)sms;
     splitk_finish_kernel<<<(unsigned)blocks, 256, 0, st>>>(p.ws, p.splits, (int)M, (int)N, W.colsum, A.s_hi, W.s_w, out,
                                                          acc_out);
   }
@@ -1527,19 +1535,19 @@ size_t gemm_static_scratch_bytes() { return kStaticScratchBytes; }
 cudaError_t launch_gemm_static_scratch(int b, int k, const sq_encoded& A, const sq_weights& W,
                                        const uint8_t* positions, int64_t M, int64_t N, int64_t K, uint16_t* out,
                                        int32_t* acc_out, int* status, cudaStream_t st) {
-  static void* scratch_addr[64] = {nullptr};
+  static std::atomic<void*> scratch_addr[64];
   int dev = 0;
   cudaError_t err = cudaGetDevice(&dev);
   if (err != cudaSuccess) return err;
   if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
-  if (scratch_addr[dev] == nullptr) {
-    void* ptr = nullptr;
+  void* ptr = scratch_addr[dev].load(std::memory_order_acquire);
+  if (ptr == nullptr) {
     err = cudaGetSymbolAddress(&ptr, g_static_scratch);
     if (err != cudaSuccess) return err;
     if (ptr == nullptr) return cudaErrorInvalidSymbol;
-    scratch_addr[dev] = ptr;
+    scratch_addr[dev].store(ptr, std::memory_order_release);
   }
-  return launch_gemm(b, k, false, A, W, positions, M, N, K, out, acc_out, status, scratch_addr[dev], kStaticScratchBytes, st);
+  return launch_gemm(b, k, false, A, W, positions, M, N, K, out, acc_out, status, ptr, kStaticScratchBytes, st);
 }
 
 }  // namespace sq

@@ -4,9 +4,21 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <atomic>
+#include <mutex>
+
 #include "../../include/sq.h"
 
 namespace sq {
+
+// Host-side state: per-device caches (device attributes, symbol addresses, kernel attributes
+// already raised, occupancy answers) filled on first use.  Readers look at atomics; whoever finds
+// an entry empty fills it under this one lock, so any number of host threads may call into the
+// library at the same time.
+inline std::mutex& setup_mutex() {
+  static std::mutex m;
+  return m;
+}
 
 // Device address of the per-device status word (0 = fine, else an sq_status).
 int* status_word();

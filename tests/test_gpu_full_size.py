@@ -44,7 +44,7 @@ class PackedLinear:
         assert np.array_equal(_np(self.w.colsum)[self.cols], self.w_ref.colsum)
         assert np.array_equal(_np(self.w.s_w)[self.cols].view(np.uint32), self.w_ref.s_w.view(np.uint32))
         if static:
-            assert np.array_equal(_np(self.w.w_sparse)[self.cols], self.w_ref.w_sparse)
+            assert np.array_equal(_np(self.w.w_sparse)[self.cols].astype(np.int16), 16 * self.w_ref.w_sparse.astype(np.int16))
         del self.W
 
 

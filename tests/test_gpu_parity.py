@@ -57,7 +57,9 @@ def compare_weights(w_gpu: sq.Weights, w_ref: oracle.Weights, rows=None):
     assert np.array_equal(_np(w_gpu.colsum)[sl], w_ref.colsum)
     assert np.array_equal(_np(w_gpu.s_w)[sl].view(np.uint32), w_ref.s_w.view(np.uint32))
     if w_ref.w_sparse is not None:
-        assert np.array_equal(_np(w_gpu.w_sparse)[sl], w_ref.w_sparse)
+        # library layout: the gathered codes are stored in sixteenths (the unit of the GEMM's INT8
+        # weight operand); the oracle holds the codes themselves
+        assert np.array_equal(_np(w_gpu.w_sparse)[sl].astype(np.int16), 16 * w_ref.w_sparse.astype(np.int16))
 
 
 def run_pipeline(M, N, K, b, k, static, seed=0, dist="student_t3", frac=0.01, scale=20.0, T=64,
@@ -116,6 +118,10 @@ def run_pipeline(M, N, K, b, k, static, seed=0, dist="student_t3", frac=0.01, sc
 @pytest.mark.parametrize("b,k,static", [
     (64, 8, False), (64, 8, True), (32, 2, False), (32, 8, True), (128, 16, True), (128, 8, False),
     (64, 16, False), (64, 4, True), (128, 32, False), (32, 1, False), (64, 32, True),
+    # k not a power of two: rank-by-counting encode, byte-wise sparse merge in the GEMM, static
+    # positions that TMA cannot fetch ((K/b)*k not a multiple of 16)
+    (64, 12, False), (64, 12, True), (32, 3, False), (32, 3, True), (128, 24, False), (128, 24, True),
+    (64, 5, False), (64, 5, True), (128, 7, False), (32, 15, True),
 ])
 def test_small_ragged_shapes(b, k, static):
     # 2 M-tiles with a ragged tail, 2 N-tiles with a ragged tail, 3 K steps
@@ -182,6 +188,33 @@ def test_maximum_k():
     w_ref = oracle.pack_weights(b, k, _bits(W))
     compare_encoded(enc, enc_ref)
     acc_ref, ref32, _ = oracle.gemm(b, k, enc_ref, w_ref)
+    assert np.array_equal(_np(acc), acc_ref)
+    assert_bf16_close(out, ref32)
+
+
+@pytest.mark.parametrize("b,k", [(128, 64), (32, 16), (64, 5)])
+def test_maximum_k_static(b, k):
+    """K = SQ_MAX_K with static positions, up to half of every bank selected: a row, its offset
+    table and its stash no longer fit the staged kernels' shared memory, so the encoder has to pick
+    a kernel that does; the GEMM walks 512 dense and up to 256 sparse K steps."""
+    K = sq.SQ_MAX_K
+    fmt = sq.make_format(b, k, True)
+    X = gen.activations(5, K, seed=2, device="cuda")
+    W = gen.weights(8, K, seed=2, device="cuda")
+    calib = gen.calibration_batch(16, K, seed=2, device="cuda")
+    pos = sq.sq_calib_positions(fmt, calib, W)
+    pos_ref = oracle.calib_positions(b, k, _bits(calib), _bits(W))
+    assert np.array_equal(_np(pos), pos_ref)
+    enc = sq.sq_encode(fmt, X, pos)
+    w = sq.sq_pack_weights(fmt, W, pos)
+    acc = torch.zeros(5, 8, dtype=torch.int32, device="cuda")
+    out = sq.sq_gemm(fmt, enc, w, pos, acc_out=acc)
+    check_status()
+    enc_ref = oracle.encode(b, k, _bits(X), pos_ref)
+    w_ref = oracle.pack_weights(b, k, _bits(W), pos_ref)
+    compare_encoded(enc, enc_ref)
+    compare_weights(w, w_ref)
+    acc_ref, ref32, _ = oracle.gemm(b, k, enc_ref, w_ref, pos_ref)
     assert np.array_equal(_np(acc), acc_ref)
     assert_bf16_close(out, ref32)
 
@@ -276,6 +309,8 @@ def test_static_encode_row_slices_in_registers(K, b, k):
     (32, 1, False),     # epilogue warps merge, byte path
     (128, 16, True),    # TMA-fed sparse K steps (the first part of K takes them all)
     (64, 4, True),
+    (64, 12, False),    # k not a power of two: byte path
+    (32, 3, True),
 ])
 @pytest.mark.parametrize("M,K", [(1, 1024), (64, 2048), (128, 1536), (17, 4096)])
 def test_split_k_with_workspace(b, k, static, M, K):
@@ -314,7 +349,8 @@ def test_split_k_with_workspace(b, k, static, M, K):
 
 # ----------------------------------------------------------------------------- many rows: pre-widened activations
 
-@pytest.mark.parametrize("b,k,static", [(64, 8, False), (32, 1, False), (128, 64, False), (128, 16, True), (64, 4, True)])
+@pytest.mark.parametrize("b,k,static", [(64, 8, False), (32, 1, False), (128, 64, False), (128, 16, True), (64, 4, True),
+                                        (64, 12, False), (32, 3, True), (128, 24, False), (64, 5, True)])
 @pytest.mark.parametrize("M,K", [(200, 384), (513, 1024), (300, 128)])
 def test_prewidened_activations_with_workspace(b, k, static, M, K):
     """sq_gemm_ws with M*K bytes of workspace (activations expanded once into 8-bit tensor-core

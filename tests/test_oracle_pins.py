@@ -303,7 +303,7 @@ def test_pack_weights_is_per_channel_absmax_int4():
     assert np.array_equal(unpack_nibbles(pw.wq4), pw.wq)
     assert np.array_equal(pw.colsum, pw.wq.astype(np.int64).sum(1).astype(np.int32))
     cols = (np.arange(K // b)[:, None] * b + pos.astype(np.int64)).ravel()
-    assert np.array_equal(pw.w_sparse, 16 * pw.wq[:, cols])      # gathered codes, in sixteenths
+    assert np.array_equal(pw.w_sparse, pw.wq[:, cols])           # the gathered codes themselves
     # textbook torch quantiser agrees
     wt = torch.from_numpy(w)
     wm = wt.abs().amax(1, keepdim=True).clamp_min(1e-30)
@@ -332,7 +332,7 @@ def test_integer_gemm_is_sum_of_component_gemms(b, k, mode):
     assert np.array_equal(acc.astype(np.int64), expect)
     if mode == "static":                      # the sparse product through the reordered weights
         via_sparse = enc.vals.reshape(M, -1).astype(np.int64) @ pw.w_sparse.astype(np.int64).T
-        assert np.array_equal(16 * acc_hi, via_sparse)           # w_sparse holds 16 * code
+        assert np.array_equal(acc_hi, via_sparse)                # w_sparse holds the plain codes
     # epilogue definition and bf16 rounding
     ref = (acc.astype(np.float32) * enc.s_hi[:, None]) * pw.s_w[None, :]
     assert np.array_equal(ref, ref32)
@@ -469,8 +469,8 @@ def test_indep_gemm_is_two_integer_products_and_matches_fp64():
     assert np.array_equal(hi.astype(np.int64), q_hi @ wq.T)
     # the gathered weight rows of Algorithm 2 give the same sparse product
     cols = (np.arange(K // b)[:, None] * b + pos.astype(np.int64)).reshape(-1)
-    assert np.array_equal(hi.astype(np.int64) * 16, enc.vals.reshape(M, -1).astype(np.int64) @ pw.w_sparse.astype(np.int64).T)
-    assert np.array_equal(pw.w_sparse.astype(np.int64), 16 * wq[:, cols])
+    assert np.array_equal(hi.astype(np.int64), enc.vals.reshape(M, -1).astype(np.int64) @ pw.w_sparse.astype(np.int64).T)
+    assert np.array_equal(pw.w_sparse.astype(np.int64), wq[:, cols])
     # fp64 brute force of the dequantised operands
     xhat = np.where(sup, enc.s_hi.astype(np.float64)[:, None] * q_hi, enc.s_lo.astype(np.float64)[:, None] * q_lo)
     what = pw.s_w.astype(np.float64)[:, None] * wq.astype(np.float64)

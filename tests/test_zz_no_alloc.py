@@ -12,17 +12,19 @@ import pytest
 import torch
 
 import gen
+import oracle
 import paper_2512_05409_b200 as sq
 
 pytestmark = pytest.mark.gpu
 
 
-def _setup(M, N, K, b, k, static, seed):
+def _setup(M, N, K, b, k, static, seed, with_inputs=False):
     fmt = sq.make_format(b, k, static)
     X = gen.activations(M, K, seed=seed, outlier_fraction=0.01, outlier_scale=20.0, device="cuda")
     W = gen.weights(N, K, seed=seed, device="cuda")
     pos = sq.sq_calib_positions(fmt, gen.calibration_batch(64, K, seed=seed, device="cuda"), W) if static else None
-    return fmt, sq.sq_encode(fmt, X, pos), sq.sq_pack_weights(fmt, W, pos), pos
+    res = (fmt, sq.sq_encode(fmt, X, pos), sq.sq_pack_weights(fmt, W, pos), pos)
+    return res + (X, W) if with_inputs else res
 
 
 @pytest.mark.parametrize("M,N,K,b,k,static", [
@@ -34,7 +36,7 @@ def test_static_scratch_matches_the_plain_entry_point_twice(M, N, K, b, k, stati
     """Two calls in a row through the C ABI (the second one finds the first one's partial sums still in
     the array) give the plain sq_gemm's result: bit-identical integers, bf16 equal, which is inside
     every tolerance the other tests use."""
-    fmt, enc, w, pos = _setup(M, N, K, b, k, static, seed=M + N)
+    fmt, enc, w, pos, X, W = _setup(M, N, K, b, k, static, seed=M + N, with_inputs=True)
     acc_ref = torch.empty(M, N, dtype=torch.int32, device="cuda")
     out_ref = sq.sq_gemm_ws(fmt, enc, w, pos, acc_out=acc_ref, workspace=None)     # the existing entry point
     outs, accs = [], []
@@ -53,6 +55,13 @@ def test_static_scratch_matches_the_plain_entry_point_twice(M, N, K, b, k, stati
         assert torch.equal(out.view(torch.int16), out_ref.view(torch.int16))
         rel = (out.float() - out_ref.float()).abs() / out_ref.float().abs().clamp_min(1e-30)
         assert float(rel.max()) <= 1e-2
+    # ... and the CPU oracle's: integer sums bit for bit, bf16 bits equal
+    pos_ref = None if pos is None else pos.cpu().numpy()
+    enc_ref = oracle.encode(b, k, gen.bf16_bits(X), pos_ref)
+    w_ref = oracle.pack_weights(b, k, gen.bf16_bits(W), pos_ref)
+    acc_o, _, out_o = oracle.gemm(b, k, enc_ref, w_ref, pos_ref)
+    assert np.array_equal(accs[1].cpu().numpy(), acc_o)
+    assert np.array_equal(gen.bf16_bits(outs[1]), out_o)
 
 
 def test_static_scratch_rejects_what_does_not_fit():
