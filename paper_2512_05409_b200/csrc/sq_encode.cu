@@ -11,11 +11,18 @@
 //   phase 1  (dynamic) each lane owns whole banks.  The k-th largest magnitude of a bank is
 //            found with a sorting network on packed bf16x2 magnitudes (two columns at once;
 //            sorted runs of k merged with truncation), then one compare pass builds the
-//            selection mask and the largest unselected magnitude; equal magnitudes at the
-//            threshold are resolved towards the lower index.
+//            selection mask; equal magnitudes at the threshold are resolved towards the lower
+//            index.  The largest UNSELECTED magnitude of the row, which fixes the shift, is not
+//            tracked element by element: the network yields per bank an upper bound (the k-th
+//            largest) and a lower bound (the largest loser of the last merge) for free, and
+//            only a row whose two bounds give different shifts is swept once more (its
+//            selected places are zero by then) for the exact value.
 //            (static) the given positions are copied out and zeroed in the staged row.
-//   reduce   row maximum and largest unselected magnitude over the group -> inv, s_hi,
-//            shift e, s_lo
+//   reduce   row maximum and the two bounds over the group -> inv, s_hi, shift e, s_lo
+//            The kernel is bound by the integer/logic pipe (16 lanes per cycle and scheduler
+//            for min/max, logic, compares, selects), so whatever integer work can be written
+//            as a multiply-add (magnitudes, picking the k positions out of the mask, nibble
+//            packing) is issued on the multiply-add pipe instead.
 //   phase 2  selected values -> INT8 in ascending position (and their indices), zeroed in
 //            the staged row; then the whole row -> INT4, eight codes per 32-bit word, in a
 //            coalesced sweep (the zeroed places give the zero nibbles the format asks for).
@@ -59,8 +66,27 @@ __device__ __forceinline__ uint32_t ge2_mask(uint32_t a, uint32_t b) {  // 0xFFF
   return d;
 }
 __device__ __forceinline__ uint32_t swap_halves(uint32_t a) { return __byte_perm(a, a, 0x1032); }
+__device__ __forceinline__ uint32_t abs2(uint32_t a) {  // compiles to a packed multiply-add pipe instruction
+  uint32_t d;
+  asm("abs.bf16x2 %0, %1;" : "=r"(d) : "r"(a));
+  return d;
+}
 
-// compare-exchange, larger first
+// The dynamic kernel is bound by the integer/logic pipe (min/max, logic, compares, selects,
+// shifts: 16 lanes per cycle and scheduler) while the multiply-add pipe has room, so integer
+// work that can be written as d = a * m + c is issued as a multiply-add.  The multipliers come
+// from kernel parameters: as immediates the compiler would turn the instruction back into an
+// add or a shift on the busy pipe.
+struct MulK {
+  uint32_t neg1, two, k32, k256, k65536, k16m;
+};
+__device__ __forceinline__ uint32_t imad(uint32_t a, uint32_t m, uint32_t c) {
+  uint32_t d;
+  asm("mad.lo.u32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(m), "r"(c));
+  return d;
+}
+
+// compare-exchange of packed magnitudes, larger first
 __device__ __forceinline__ void ce(uint32_t& a, uint32_t& b) {
   const uint32_t hi = max2(a, b), lo = min2(a, b);
   a = hi;
@@ -144,6 +170,26 @@ __device__ __forceinline__ uint32_t pack_nibbles(const float (&r)[8]) {
   return (ev & 0x0F0F0F0Fu) | ((od << 4) & 0xF0F0F0F0u);
 }
 
+// The same packing for codes that carry an offset of 8 (u = q + 8 in 1..15, produced by adding
+// kMagic + 8 in the rounding FMA): the eight float bit patterns 0x4B400000 + u are summed with
+// weights 16^i by integer multiply-adds (no carries between nibbles since u fits four bits), the
+// constant part is taken off and the offset undone by flipping bit 3 of every nibble.  Seven
+// multiply-adds on the multiply-add pipe instead of nine byte-permute/logic operations on the
+// integer pipe, which is the one this kernel is bound by.
+__device__ __forceinline__ uint32_t mad16(uint32_t hi, uint32_t mul, uint32_t lo) {
+  uint32_t d;
+  asm("mad.lo.u32 %0, %1, %2, %3;" : "=r"(d) : "r"(hi), "r"(mul), "r"(lo));
+  return d;
+}
+__device__ __forceinline__ uint32_t pack_nibbles_off8(const float (&r)[8]) {
+  const uint32_t t01 = mad16(__float_as_uint(r[1]), 16u, __float_as_uint(r[0]));
+  const uint32_t t23 = mad16(__float_as_uint(r[3]), 16u, __float_as_uint(r[2]));
+  const uint32_t t45 = mad16(__float_as_uint(r[5]), 16u, __float_as_uint(r[4]));
+  const uint32_t t67 = mad16(__float_as_uint(r[7]), 16u, __float_as_uint(r[6]));
+  const uint32_t t03 = mad16(t23, 256u, t01), t47 = mad16(t67, 256u, t45);
+  return (mad16(t47, 65536u, t03) - 0x3F400000u) ^ 0x88888888u;  // 0x3F400000 = 0x4B400000 * 0x11111111 mod 2^32
+}
+
 // Row scales from the two maxima (bf16 magnitude bit patterns).
 struct RowScale {
   float inv, inv_lo, s_hi, s_lo;
@@ -216,9 +262,11 @@ __device__ __forceinline__ void bulk_copy_g2s(uint32_t dst, const void* src, uin
 // Eight bf16 (four packed words) times c, rounded half-even to integers held in the low
 // mantissa bits (magic-number rounding); two FMAs per instruction on the packed fp32 pipe,
 // each half rounding like fmaf.
+template <bool OFF8 = false>
 __device__ __forceinline__ void quant8(const uint4& v, float c, float (&r)[8]) {
   const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-  const float2 cc = make_float2(c, c), mm = make_float2(kMagic, kMagic);
+  constexpr float kM = OFF8 ? kMagic + 8.0f : kMagic;
+  const float2 cc = make_float2(c, c), mm = make_float2(kM, kM);
 #pragma unroll
   for (int q = 0; q < 4; ++q) {
     const float2 a = make_float2(__uint_as_float(w[q] << 16), __uint_as_float(w[q] & 0xFFFF0000u));
@@ -240,8 +288,8 @@ __device__ __forceinline__ void dense_sweep(const uint16_t* row, int K, const Ro
 #pragma unroll 2
     for (int i = 0; i < iters; ++i, src += gsize, dst += gsize) {
       float r[8];
-      quant8(*src, c, r);
-      *dst = pack_nibbles(r);
+      quant8<true>(*src, c, r);
+      *dst = pack_nibbles_off8(r);
     }
   } else {
     // Codes beyond +-7 are possible: limit the inputs instead of the codes, two elements per
@@ -257,8 +305,8 @@ __device__ __forceinline__ void dense_sweep(const uint16_t* row, int K, const Ro
       v.z = max2(min2(v.z, hi2), lo2);
       v.w = max2(min2(v.w, hi2), lo2);
       float r[8];
-      quant8(v, c, r);
-      *dst = pack_nibbles(r);
+      quant8<true>(v, c, r);
+      *dst = pack_nibbles_off8(r);
     }
   }
 }
@@ -278,6 +326,7 @@ struct EncodeParams {
   int nbuf;           // row buffers per group (1 or 2)
   int rw;             // warps per row group
   int group_stride;   // bytes of shared memory per group
+  MulK mk;            // -1, 2, 32, 2^8, 2^16, 2^24 (see MulK)
 };
 
 __device__ __forceinline__ void group_sync(int rw, int grp) {
@@ -304,9 +353,10 @@ __global__ void __launch_bounds__(B == 128 ? 256 : 512) encode_rows_kernel(const
   const int K = p.K, G = K / B, k = kStatic ? p.k : KK;
   const int GK = G * k;
   const int nbuf = p.nbuf;
+  const MulK mk = p.mk;
 
   // shared memory: [static only: table of selected element offsets, uint16 [GK]] then per group
-  // [nbuf rows][stash of selected raw values, uint16 [GK]][4 mbarriers][2 x 16 exchange words]
+  // [nbuf rows][stash of selected raw values, uint16 [GK]][4 mbarriers][4 x 16 exchange words]
   const size_t table_bytes = kStatic ? (((size_t)GK * 2 + 127) & ~(size_t)127) : 0;
   uint16_t* jt = reinterpret_cast<uint16_t*>(smem_enc);
   uint8_t* wbase = smem_enc + table_bytes + (size_t)grp * p.group_stride;
@@ -354,25 +404,30 @@ __global__ void __launch_bounds__(B == 128 ? 256 : 512) encode_rows_kernel(const
       if (mn < p.M) bulk_copy_g2s(smem_u32(wbase + (size_t)nb * row_bytes), p.X + mn * K, row_bytes, bar0 + 8 * nb);
     }
     if (!mbar_wait_park(bar0 + 8 * cur, parity, abort_flag)) break;
+    // the row this group takes next is asked into L2 now, so that the copy issued when this row
+    // is done (the buffer is single) finds it there
+    if (nbuf == 1 && lane == 0 && m + wstride < p.M)
+      asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(p.X + (m + wstride) * K), "r"(row_bytes) : "memory");
 
-    uint32_t lane_amax = 0, lane_rmax = 0;
+    // lane_rmax: static positions: the largest unselected magnitude.  Dynamic positions: an UPPER
+    // bound of it (the largest k-th magnitude of any bank), with lane_rlow a LOWER bound (see below).
+    uint32_t lane_amax = 0, lane_rmax = 0, lane_rlow = 0;
     if constexpr (!kStatic) {
       // ------------------------------------------------------------ phase 1: selection
       // conflict-free chunk rotation: consecutive lanes start on different 16-byte bank groups
       const int rot = (B == 32) ? ((lane >> 1) & (NCH - 1)) : (lane & (NCH - 1));
       for (int g = lane; g < G; g += gsize) {
         uint16_t* bank = row + g * B;
-        uint32_t x[NP];
+        // k-th largest magnitude: sorted runs of KK per column, merged with truncation
+        uint32_t x[NP], s[NP];
 #pragma unroll
         for (int c = 0; c < NCH; ++c) {
           const uint4 v = *reinterpret_cast<const uint4*>(bank + ((c + rot) & (NCH - 1)) * 8);
-          x[4 * c] = v.x & 0x7FFF7FFFu;
-          x[4 * c + 1] = v.y & 0x7FFF7FFFu;
-          x[4 * c + 2] = v.z & 0x7FFF7FFFu;
-          x[4 * c + 3] = v.w & 0x7FFF7FFFu;
+          x[4 * c] = abs2(v.x);
+          x[4 * c + 1] = abs2(v.y);
+          x[4 * c + 2] = abs2(v.z);
+          x[4 * c + 3] = abs2(v.w);
         }
-        // k-th largest magnitude: sorted runs of KK per column, merged with truncation
-        uint32_t s[NP];
 #pragma unroll
         for (int i = 0; i < NP; ++i) s[i] = x[i];
 #pragma unroll
@@ -386,36 +441,54 @@ __global__ void __launch_bounds__(B == 128 ? 256 : 512) encode_rows_kernel(const
             bitonic_merge_desc<KK>(s + a);
           }
         }
-        // s[0..KK): per column the KK largest, descending.  Across the two columns:
-        uint32_t d[KK];
+        // s[0..KK): per column the KK largest, descending.  Pairing entry i of one column with
+        // entry KK-1-i of the other splits those 2*KK values into their KK largest (the larger of
+        // each pair) and the rest (the smaller of each pair): T = the smallest of the former is the
+        // bank's k-th largest magnitude (with multiplicity), and the largest of the latter is a
+        // LOWER bound of the bank's (k+1)-th largest, i.e. of its largest unselected magnitude.
+        // (Both halves of a register hold a pair, so half of the entries cover all pairs.)
+        constexpr int HP = KK >= 2 ? KK / 2 : 1;
+        uint32_t dmin, lmax;
+        {
+          uint32_t d[HP], l[HP];
 #pragma unroll
-        for (int i = 0; i < KK; ++i) d[i] = max2(s[i], swap_halves(s[KK - 1 - i]));
+          for (int i = 0; i < HP; ++i) {
+            const uint32_t o = swap_halves(s[KK - 1 - i]);
+            d[i] = max2(s[i], o);
+            l[i] = min2(s[i], o);
+          }
 #pragma unroll
-        for (int w = KK / 2; w >= 1; w /= 2) {
+          for (int w = HP / 2; w >= 1; w /= 2) {
 #pragma unroll
-          for (int i = 0; i < w; ++i) d[i] = min2(d[i], d[i + w]);
+            for (int i = 0; i < w; ++i) {
+              d[i] = min2(d[i], d[i + w]);
+              l[i] = max2(l[i], l[i + w]);
+            }
+          }
+          dmin = min(d[0] & 0xFFFFu, d[0] >> 16);
+          lmax = max(l[0] & 0xFFFFu, l[0] >> 16);
         }
-        const uint32_t T = d[0] & 0xFFFFu;  // k-th largest magnitude of the bank (with multiplicity)
+        const uint32_t T = dmin;  // k-th largest magnitude of the bank (with multiplicity)
         const uint32_t bank_max = max(s[0] & 0xFFFFu, s[0] >> 16);
         lane_amax = max(lane_amax, bank_max);
 
-        // compare pass: selection mask (slot order) and the largest magnitude below T
+        // compare pass: one flag per element reaching T.  Register q of a 16-element group holds
+        // elements 2q and 2q+1; its flags go to bits 2q and 17+2q of the group's word, so that
+        // (word | word >> 16) has the group's 16 flags in element order in its low half.
         const uint32_t T2 = T * 0x10001u;
-        uint32_t acc[NP / 16];
-        uint32_t below = 0;
+        uint32_t acc[NP / 8];
 #pragma unroll
-        for (int w = 0; w < NP / 16; ++w) acc[w] = 0;
+        for (int w = 0; w < NP / 8; ++w) acc[w] = 0;
 #pragma unroll
-        for (int q = 0; q < NP; ++q) {
-          const uint32_t ge = ge2_mask(x[q], T2);
-          acc[q / 16] |= ge & (0x00010001u << (q % 16));
-          below = max2(below, x[q] & ~ge);
-        }
+        for (int q = 0; q < NP; ++q) acc[q / 8] |= ge2_mask(x[q], T2) & (0x00020001u << (2 * (q % 8)));
         uint64_t sel[NM];
 #pragma unroll
         for (int w = 0; w < NM; ++w) sel[w] = 0;
 #pragma unroll
-        for (int w = 0; w < NP / 16; ++w) sel[w / 2] |= (uint64_t)interleave_halves(acc[w]) << (32 * (w & 1));
+        for (int w = 0; w < NP / 16; ++w) {
+          const uint32_t f0 = acc[2 * w] | (acc[2 * w] >> 16), f1 = acc[2 * w + 1] | (acc[2 * w + 1] >> 16);
+          sel[w / 2] |= (uint64_t)__byte_perm(f0, f1, 0x5410) << (32 * (w & 1));
+        }
         // slot order -> element order: slot c holds chunk (c + rot) mod NCH
         if (B == 128) {
           const int sh = 8 * rot;  // 0..120
@@ -443,10 +516,11 @@ __global__ void __launch_bounds__(B == 128 ? 256 : 512) encode_rows_kernel(const
         int cnt = 0;
 #pragma unroll
         for (int w = 0; w < NM; ++w) cnt += __popcll(sel[w]);
-        uint32_t rest = max(below & 0xFFFFu, below >> 16);
+        uint32_t rest_low = lmax;
         if (cnt > KK) {
-          // more than k elements reach T: drop the equal ones with the largest indices
-          rest = T;
+          // more than k elements reach T: drop the equal ones with the largest indices; the
+          // largest unselected magnitude of this bank is then T itself
+          rest_low = T;
           int excess = cnt - KK;
 #pragma unroll
           for (int w = NM - 1; w >= 0; --w) {
@@ -461,7 +535,8 @@ __global__ void __launch_bounds__(B == 128 ? 256 : 512) encode_rows_kernel(const
             }
           }
         }
-        lane_rmax = max(lane_rmax, rest);
+        lane_rmax = max(lane_rmax, T);
+        lane_rlow = max(lane_rlow, rest_low);
 
         // the k selected elements in ascending position: raw values to the stash, zero in the
         // staged row, positions to global memory (they do not depend on the scale)
@@ -474,31 +549,67 @@ __global__ void __launch_bounds__(B == 128 ? 256 : 512) encode_rows_kernel(const
           m3 = (uint32_t)(sel[NM - 1] >> 32);
         }
         uint16_t* sg = stash + g * KK;
+        // positions first (bit arithmetic only), then all loads, then all stores: the loads of
+        // the k raw values are then in flight together instead of each waiting behind the
+        // previous element's stores
+        uint32_t pos[KK];
 #pragma unroll
         for (int i = 0; i < KK; ++i) {
-          // lowest set bit of the (up to 128-bit) mask, then clear it
-          uint32_t word = m0, base = 0;
-          if (B >= 64 && word == 0) {
-            word = m1;
-            base = 32;
+          // lowest set bit of the (up to 128-bit) mask, then clear it.  Which word it sits in is
+          // a 0/1 flag per word (min(word, 1)); selecting the word, adding its base and writing the
+          // remainder back are multiply-adds by those flags, not compares and selects.
+          uint32_t word, rest_bits;
+          if (B == 32) {
+            word = m0;
+            pos[i] = (uint32_t)(__ffs((int)word) - 1);
+            m0 = word & (word - 1u);
+          } else if (B == 64) {
+            const uint32_t n0 = min(m0, 1u), z0 = imad(n0, mk.neg1, 1u);   // m0 != 0, m0 == 0
+            word = imad(z0, m1, m0);                                       // m0 == 0 ? m1 : m0
+            pos[i] = imad(z0, mk.k32, (uint32_t)(__ffs((int)word) - 1));
+            rest_bits = word & (word - 1u);
+            m0 = imad(n0, rest_bits, 0u);                                  // stays 0 once empty
+            m1 = imad(z0, rest_bits, imad(n0, m1, 0u));
+          } else {
+            const bool z0 = m0 == 0;
+            word = z0 ? m1 : m0;
+            uint32_t base = z0 ? 32u : 0u;
+            const bool z1 = (m0 | m1) == 0;
+            const bool z2 = z1 && m2 == 0;
+            word = z1 ? (z2 ? m3 : m2) : word;
+            base = z1 ? (z2 ? 96u : 64u) : base;
+            pos[i] = base + (uint32_t)(__ffs((int)word) - 1);
+            rest_bits = word & (word - 1u);
+            m0 = base == 0 ? rest_bits : m0;
+            m1 = base == 32 ? rest_bits : m1;
+            m2 = base == 64 ? rest_bits : m2;
+            m3 = base == 96 ? rest_bits : m3;
           }
-          if (B == 128 && word == 0) {
-            word = m2;
-            base = 64;
-            if (word == 0) {
-              word = m3;
-              base = 96;
-            }
-          }
-          const uint32_t bit = word & (0u - word);
-          const uint32_t pos = base + (31u - (uint32_t)__clz((int)bit));
-          if (base == 0) m0 ^= bit;
-          else if (base == 32) m1 ^= bit;
-          else if (base == 64) m2 ^= bit;
-          else m3 ^= bit;
-          sg[i] = bank[pos];
-          bank[pos] = 0;
-          iout[i / 4] = __byte_perm(iout[i / 4], pos, 0x3210 ^ (0x4 << (4 * (i % 4))) ^ ((i % 4) << (4 * (i % 4))));
+          // position byte i of the bank's index list
+          iout[i / 4] = (i % 4) == 0 ? pos[i]
+                                     : imad(pos[i], (i % 4) == 1 ? mk.k256 : ((i % 4) == 2 ? mk.k65536 : mk.k16m), iout[i / 4]);
+        }
+        uint32_t raw[KK];
+        const uint32_t bank_s = smem_u32(bank);
+#pragma unroll
+        for (int i = 0; i < KK; ++i) {
+          const uint32_t addr = imad(pos[i], mk.two, bank_s);
+          asm volatile("ld.shared.u16 %0, [%1];" : "=r"(raw[i]) : "r"(addr));
+          pos[i] = addr;
+        }
+#pragma unroll
+        for (int i = 0; i < KK; ++i) asm volatile("st.shared.u16 [%0], %1;" ::"r"(pos[i]), "h"((uint16_t)0) : "memory");
+        if (KK >= 8) {
+#pragma unroll
+          for (int i = 0; i < KK; i += 8)
+            *reinterpret_cast<uint4*>(sg + i) = make_uint4(raw[i] | (raw[i + 1] << 16), raw[i + 2] | (raw[i + 3] << 16),
+                                                           raw[i + 4] | (raw[i + 5] << 16), raw[i + 6] | (raw[i + 7] << 16));
+        } else if (KK == 4) {
+          *reinterpret_cast<uint2*>(sg) = make_uint2(raw[0] | (raw[1] << 16), raw[2] | (raw[3] << 16));
+        } else if (KK == 2) {
+          *reinterpret_cast<uint32_t*>(sg) = raw[0] | (raw[1] << 16);
+        } else {
+          sg[0] = (uint16_t)raw[0];
         }
         uint8_t* idst = p.idx + ((size_t)m * G + g) * KK;
         if (KK >= 16) {
@@ -539,21 +650,50 @@ __global__ void __launch_bounds__(B == 128 ? 256 : 512) encode_rows_kernel(const
 
     uint32_t amax_bits = __reduce_max_sync(0xffffffffu, lane_amax);
     uint32_t rmax_bits = __reduce_max_sync(0xffffffffu, lane_rmax);
+    uint32_t rlow_bits = kStatic ? 0u : __reduce_max_sync(0xffffffffu, lane_rlow);
     if (rw > 1) {
       if ((threadIdx.x & 31) == 0) {
         exch[warp % rw] = amax_bits;
         exch[16 + warp % rw] = rmax_bits;
+        if (!kStatic) exch[32 + warp % rw] = rlow_bits;
       }
       group_sync(rw, grp);  // also: every stash entry of the row is written
-      amax_bits = rmax_bits = 0;
+      amax_bits = rmax_bits = rlow_bits = 0;
       for (int w = 0; w < rw; ++w) {
         amax_bits = max(amax_bits, exch[w]);
         rmax_bits = max(rmax_bits, exch[16 + w]);
+        if (!kStatic) rlow_bits = max(rlow_bits, exch[32 + w]);
       }
     } else {
       __syncwarp();
     }
-    const RowScale rs = row_scale_warp(amax_bits, rmax_bits, threadIdx.x & 31);
+    RowScale rs = row_scale_warp(amax_bits, rmax_bits, threadIdx.x & 31);
+    if constexpr (!kStatic) {
+      // The shift was computed from an upper bound of the largest unselected magnitude.  It is the
+      // true one unless the lower bound would still fit one shift less; only then (the same for
+      // the whole group) the row, whose selected places are zero by now, is swept for the exact
+      // maximum.  (A clamp flag set by the upper bound alone only costs time.)
+      const bool exact =
+          rs.e > 0 && rne_prod(bf16_bits_to_f32(rlow_bits), rs.inv * __int_as_float((127 - (rs.e - 1)) << 23)) <= 7;
+      if (exact) {
+        const uint4* src = reinterpret_cast<const uint4*>(row) + lane;
+        const int iters = (K / 8 - lane + gsize - 1) / gsize;
+        uint32_t mx = 0;
+#pragma unroll 4
+        for (int i = 0; i < iters; ++i, src += gsize) {
+          const uint4 v = *src;
+          mx = max2(mx, max2(max2(v.x & 0x7FFF7FFFu, v.y & 0x7FFF7FFFu), max2(v.z & 0x7FFF7FFFu, v.w & 0x7FFF7FFFu)));
+        }
+        uint32_t rx = __reduce_max_sync(0xffffffffu, max(mx & 0xFFFFu, mx >> 16));
+        if (rw > 1) {
+          if ((threadIdx.x & 31) == 0) exch[48 + warp % rw] = rx;
+          group_sync(rw, grp);
+          rx = 0;
+          for (int w = 0; w < rw; ++w) rx = max(rx, exch[48 + w]);
+        }
+        rs = row_scale_warp(amax_bits, rx, threadIdx.x & 31);
+      }
+    }
     if (lane == 0) {
       p.s_hi[m] = rs.s_hi;
       p.s_lo[m] = rs.s_lo;
@@ -959,9 +1099,9 @@ cudaError_t launch_rows(const EncodeParams& base, cudaStream_t st) {
   constexpr int kMaxWarps = (B == 128) ? 8 : 16;
   const size_t side = (((size_t)G * k * 2) + 15) & ~(size_t)15;            // stash of selected raw values
   const size_t table = (KK == 0) ? ((((size_t)G * k * 2) + 127) & ~(size_t)127) : 0;  // static offset table
-  const size_t budget = 208 * 1024 - table;
+  const size_t budget = 224 * 1024 - table;
   const size_t row = (size_t)K * 2;
-  const size_t extra = side + 32 + 128 + 128;  // side buffer, four mbarriers, exchange words, rounding
+  const size_t extra = side + 32 + 256 + 128;  // side buffer, four mbarriers, exchange words, rounding
   // Rows are single-buffered: with 16 resident warps the rows other groups have in flight
   // hide the copy latency, and a second buffer would only cost warps.  Pick the group size
   // that keeps the most warps resident, preferring smaller groups (less per-row overhead per
@@ -982,7 +1122,7 @@ cudaError_t launch_rows(const EncodeParams& base, cudaStream_t st) {
   if (per_group > 224 * 1024) return cudaErrorNotSupported;
   int ngroups = kMaxWarps / rw;
   {
-    const size_t fit = (208 * 1024 - table) / ((((size_t)nbuf * row + extra) + 127) & ~(size_t)127);
+    const size_t fit = (224 * 1024 - table) / ((((size_t)nbuf * row + extra) + 127) & ~(size_t)127);
     if ((size_t)ngroups > fit) ngroups = (int)fit;
     if (ngroups < 1) ngroups = 1;
   }
@@ -1075,6 +1215,7 @@ cudaError_t launch_encode(int b, int k, bool is_static, bool indep, const uint16
   p.nbuf = 1;
   p.rw = 1;
   p.group_stride = 0;
+  p.mk = MulK{0xFFFFFFFFu, 2u, 32u, 256u, 65536u, 1u << 24};
   if (is_static && indep) {
     // independent scales: the register kernel, or the plain one for row lengths it does not take
     const cudaError_t err = launch_static_regs<true>(p, st);
