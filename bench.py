@@ -164,91 +164,142 @@ class Linear:
             events[2].record()
 
 
+def time_launches(fn, iters, warmup):
+    """Median and best CUDA-event time (ms) of fn(i) over `iters` launches after `warmup`."""
+    for i in range(warmup):
+        fn(i)
+    torch.cuda.synchronize()
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(iters)]
+    for i in range(iters):
+        evs[i][0].record()
+        fn(i)
+        evs[i][1].record()
+    torch.cuda.synchronize()
+    times = [a.elapsed_time(b) for a, b in evs]
+    return statistics.median(times), min(times)
+
+
 def bench_encode_only(sq, dev, peaks, iters=50, warmup=10):
-    """The bandwidth test: 8192 x 8192 bf16, Student-t with 0.5% channels x50, b=64, k in {4,8,16}."""
+    """The bandwidth test: 8192 x 8192 bf16, Student-t with 0.5% channels x50, b=64, k in {4,8,16}.
+    Next to every point: a plain device copy (torch) that moves the same number of bytes, timed the
+    same way in the same run -- what a launch of this size can reach at all on this GPU."""
     M = K = 8192
-    res = []
+    rows = []
     # three input buffers in rotation (384 MB > L2) so no launch finds its input in L2
     Xs = [gen.activations(M, K, seed=s, outlier_fraction=0.005, outlier_scale=50.0, device=dev) for s in range(3)]
     calib = gen.calibration_batch(512, K, seed=0, outlier_fraction=0.005, outlier_scale=50.0, device=dev)
+    copy_dst = torch.empty(M * K, dtype=torch.bfloat16, device=dev)
     for static in (False, True):
         for k in (4, 8, 16):
             fmt = sq.make_format(64, k, static)
             pos = sq.sq_calib_positions(fmt, calib) if static else None
             enc = sq.alloc_encoded(fmt, M, K, dev)
-            for i in range(warmup):
-                sq.sq_encode(fmt, Xs[i % 3], pos, out=enc)
-            torch.cuda.synchronize()
-            evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(iters)]
-            for i in range(iters):
-                evs[i][0].record()
-                sq.sq_encode(fmt, Xs[i % 3], pos, out=enc)
-                evs[i][1].record()
-            torch.cuda.synchronize()
-            times = [a.elapsed_time(b) for a, b in evs]
-            ms = statistics.median(times)
+            ms, best = time_launches(lambda i: sq.sq_encode(fmt, Xs[i % 3], pos, out=enc), iters, warmup)
             nbytes = M * K * (2.0 + 0.5 + (1.0 if static else 2.0) * k / 64) + 9.0 * M
             gbs = nbytes / (ms * 1e-3) / 1e9
-            traffic = ENCODE_TRAFFIC_BYTES_PER_LAUNCH["static" if static else "dynamic"] if k == 8 else None
-            res.append({"mode": "static" if static else "dynamic", "k": k, "ms": round(ms, 4), "best_ms": round(min(times), 4),
-                        "launches": iters,
-                        "algorithmic_bytes": nbytes, "traffic": traffic,
-                        "GBps": round(gbs, 1), "frac_of_measured_hbm": round(gbs / peaks["hbm_gbs"], 4),
-                        "frac_of_8TBps": round(gbs / 8000.0, 4)})
-    return res
+            n_copy = int(nbytes / 4)          # bf16 elements: read + write = nbytes
+            cms, _ = time_launches(lambda i: copy_dst[:n_copy].copy_(Xs[i % 3].view(-1)[:n_copy]), iters, warmup)
+            copy_gbs = nbytes / (cms * 1e-3) / 1e9
+            rows.append(["static" if static else "dynamic", k, round(ms * 1e3, 1), round(best * 1e3, 1), round(gbs),
+                         round(gbs / peaks["hbm_gbs"], 3), round(gbs / 8000.0, 3), round(copy_gbs), round(gbs / copy_gbs, 3)])
+    return {"cols": ["positions", "k", "us_median", "us_best", "GBps", "of_measured_hbm", "of_8TBps",
+                     "same_run_copy_GBps", "of_same_run_copy"],
+            "rows": rows, "launches": iters,
+            "traffic_ncu_bytes_per_launch_k8": ENCODE_TRAFFIC_BYTES_PER_LAUNCH}
+
+
+def graph_replay_us(fn, calls=10, replays=5):
+    """GPU time per call of fn() when `calls` of them are replayed from a CUDA graph (no host cost)."""
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        fn()
+        torch.cuda.synchronize()
+        with torch.cuda.graph(graph, stream=side):
+            for _ in range(calls):
+                fn()
+    torch.cuda.synchronize()
+    graph.replay()
+    torch.cuda.synchronize()
+    g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    g0.record()
+    for _ in range(replays):
+        graph.replay()
+    g1.record()
+    torch.cuda.synchronize()
+    us = g0.elapsed_time(g1) * 1e3 / (calls * replays)
+    del graph
+    return us
 
 
 def bench_8b_dynamic(sq, dev, peaks, iters=20):
-    """sq_encode + sq_gemm on the 8B-decoder-shaped linears with dynamic positions (b=64, k=8):
-    M = 2048 (prefill: TOPS) and M = 16 (decode: bound by the INT4 weight stream N*K/2 bytes)."""
-    res = []
+    """sq_encode + sq_gemm on the 8B-decoder-shaped linears with dynamic positions (b=64, k=8) at
+    M in {1, 16, 128, 2048}, plus the single-GEMM configuration (M=64, K=N=4096, N(0,1) activations).
+    M >= 128: TOPS of the call the binding makes (with its workspace) and of plain sq_gemm (sparse
+    part merged inside the GEMM kernel).  M <= 128: also the GPU time per call replayed from a CUDA
+    graph and the INT4 weight stream N*K/2 bytes over it (those calls are host-bound otherwise)."""
+    rows = []
     int8_peak = peaks["bf16_tflops"] * INT8_OVER_BF16
-    for (K, N) in SHAPES_8B:
-        lin = {M: Linear(sq, M, K, N, 64, 8, False, seed=K + N + M, dev=dev) for M in (2048, 16)}
-        for M, l in lin.items():
-            for _ in range(10):
-                l.step(sq)
-            torch.cuda.synchronize()
-            evs = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(iters)]
-            for e in evs:
-                l.step(sq, e)
-            torch.cuda.synchronize()
-            g_ms = statistics.median(e[1].elapsed_time(e[2]) for e in evs)
-            e_ms = statistics.median(e[0].elapsed_time(e[1]) for e in evs)
-            tops = l.ops / (g_ms * 1e-3) / 1e12
-            graph_us = None
-            if M <= 128:
-                # decode-sized calls are bound by the host's launch path (Python + two launches); the
-                # same ten calls replayed from a CUDA graph give the GPU's own time per call
-                side = torch.cuda.Stream()
-                side.wait_stream(torch.cuda.current_stream())
-                graph = torch.cuda.CUDAGraph()
-                with torch.cuda.stream(side):
-                    sq.sq_gemm(l.fmt, l.enc, l.w, l.pos, out=l.out)
-                    torch.cuda.synchronize()
-                    with torch.cuda.graph(graph, stream=side):
-                        for _ in range(10):
-                            sq.sq_gemm(l.fmt, l.enc, l.w, l.pos, out=l.out)
-                torch.cuda.synchronize()
-                graph.replay()
-                torch.cuda.synchronize()
-                g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                g0.record()
-                for _ in range(5):
-                    graph.replay()
-                g1.record()
-                torch.cuda.synchronize()
-                graph_us = round(g0.elapsed_time(g1) * 1e3 / 50, 1)
-                del graph
-            res.append({"M": M, "K": K, "N": N, "gemm_us": round(g_ms * 1e3, 1), "encode_us": round(e_ms * 1e3, 1),
-                        "gemm_us_graph_replay": graph_us,
-                        "weight_stream_GBps_graph_replay": None if graph_us is None else round(N * K / 2 / (graph_us * 1e-6) / 1e9, 1),
-                        "gemm_TOPS": round(tops, 1), "frac_of_measured_int8": round(tops / int8_peak, 4),
-                        "frac_of_nominal_4500": round(tops / 4500.0, 4),
-                        "weight_stream_GBps": round(N * K / 2 / (g_ms * 1e-3) / 1e9, 1)})
-        del lin
+    shapes = [(K, N, M, "student_t3") for (K, N) in SHAPES_8B for M in (1, 16, 128, 2048)] + [(4096, 4096, 64, "normal")]
+    for (K, N, M, dist) in shapes:
+        l = Linear(sq, M, K, N, 64, 8, False, seed=K + N + M, dev=dev, dist=dist)
+        e_ms, _ = time_launches(lambda i: sq.sq_encode(l.fmt, l.X, l.pos, out=l.enc), iters, 5)
+        g_ms, _ = time_launches(lambda i: sq.sq_gemm(l.fmt, l.enc, l.w, l.pos, out=l.out), iters, 10)
+        f_ms, _ = time_launches(lambda i: sq.sq_gemm(l.fmt, l.enc, l.w, l.pos, out=l.out, use_workspace=False), iters, 5)
+        tops, ftops = l.ops / (g_ms * 1e-3) / 1e12, l.ops / (f_ms * 1e-3) / 1e12
+        graph_us = wgbs = None
+        if M <= 128:
+            graph_us = round(graph_replay_us(lambda: sq.sq_gemm(l.fmt, l.enc, l.w, l.pos, out=l.out)), 1)
+            wgbs = round(N * K / 2 / (graph_us * 1e-6) / 1e9)
+        rows.append([M, K, N, round(e_ms * 1e3, 1), round(g_ms * 1e3, 1), graph_us, wgbs, round(tops, 1),
+                     round(tops / int8_peak, 3), round(tops / 4500.0, 3), round(f_ms * 1e3, 1), round(ftops, 1)])
+        del l
         torch.cuda.empty_cache()
-    return res
+    return {"cols": ["M", "K", "N", "encode_us", "gemm_us", "gemm_us_graph_replay", "weight_stream_GBps_graph_replay",
+                     "TOPS", "of_measured_int8", "of_nominal_4500", "fused_gemm_us", "fused_TOPS"],
+            "rows": rows}
+
+
+def bench_gemm_fused(sq, layers, dev, peaks, iters=10):
+    """Plain sq_gemm (no workspace): the sparse INT8 part runs inside the GEMM kernel -- static
+    positions as TMA-fed gathered K steps, dynamic positions merged into the widened activation
+    tile -- against the call with a workspace (activations expanded once into 8-bit operands by a
+    kernel of their own), on the 70B-shaped linears of the step (static, M = 4096) and, with
+    dynamic positions b=128 k=16, on the same shapes."""
+    int8_peak = peaks["bf16_tflops"] * INT8_OVER_BF16
+    rows = []
+    for l in layers:
+        for ws in (False, True):
+            ms, _ = time_launches(lambda i: sq.sq_gemm(l.fmt, l.enc, l.w, l.pos, out=l.out, use_workspace=ws), iters, 3)
+            tops = l.ops / (ms * 1e-3) / 1e12
+            rows.append([l.K, l.N, l.M, "static", "workspace" if ws else "fused", round(ms * 1e3, 1), round(tops, 1),
+                         round(tops / int8_peak, 3), round(tops / 4500.0, 3)])
+    for (K, N) in SHAPES_70B[:2]:
+        l = Linear(sq, M_70B, K, N, BANK_70B, K_70B, False, seed=K + N, dev=dev)
+        sq.sq_encode(l.fmt, l.X, l.pos, out=l.enc)
+        for ws in (False, True):
+            ms, _ = time_launches(lambda i: sq.sq_gemm(l.fmt, l.enc, l.w, l.pos, out=l.out, use_workspace=ws), iters, 3)
+            tops = l.ops / (ms * 1e-3) / 1e12
+            rows.append([K, N, l.M, "dynamic", "workspace" if ws else "fused", round(ms * 1e3, 1), round(tops, 1),
+                         round(tops / int8_peak, 3), round(tops / 4500.0, 3)])
+        del l
+        torch.cuda.empty_cache()
+    return {"cols": ["K", "N", "M", "positions", "mode", "gemm_us", "TOPS", "of_measured_int8", "of_nominal_4500"],
+            "rows": rows}
+
+
+def bench_same_run_int8(dev, iters=10):
+    """A vendor INT8 GEMM (torch._int_mm, M=4096, N=K=8192) timed in the same run: a yardstick for
+    the tensor pipe's INT8 rate at this run's clocks, never on the product path."""
+    M, K, N = 4096, 8192, 8192
+    try:
+        a = torch.randint(-127, 128, (M, K), dtype=torch.int8, device=dev)
+        b = torch.randint(-7, 8, (N, K), dtype=torch.int8, device=dev).t()
+        ms, _ = time_launches(lambda i: torch._int_mm(a, b), iters, 3)
+        return 2.0 * M * N * K / (ms * 1e-3) / 1e12
+    except Exception:
+        return None
 
 
 def bench_format_sweep(sq, dev, peaks, iters=5):
@@ -290,16 +341,14 @@ def bench_format_sweep(sq, dev, peaks, iters=5):
                     ms = statistics.median(a.elapsed_time(c) for a, c in evs)
                     tops = 2.0 * M * N * K / (ms * 1e-3) / 1e12
                     err = float((out.float() - ref).norm()) / ref_norm
-                    res.append({"b": b, "k": k, "positions": ("static, independent scales" if indep else "static") if static else "dynamic",
-                                "outlier_scale": scale,
-                                "gemm_us": round(ms * 1e3, 1), "gemm_TOPS": round(tops, 1),
-                                "frac_of_measured_int8": round(tops / int8_peak, 4),
-                                "frac_of_nominal_4500": round(tops / 4500.0, 4), "rel_err_vs_fp32": round(err, 5)})
+                    res.append([b, k, ("indep" if indep else "static") if static else "dynamic", int(scale),
+                                round(ms * 1e3, 1), round(tops), round(tops / int8_peak, 3), round(err, 4)])
                     del w, enc
         del X, calib, ref, out
         torch.cuda.empty_cache()
     torch.backends.cuda.matmul.allow_tf32 = tf32
-    return res
+    return {"cols": ["b", "k", "positions", "outlier_scale", "gemm_us", "TOPS", "of_measured_int8", "rel_err_vs_fp32"],
+            "rows": res}
 
 
 def oracle_sample(K, N, bank, k, seed, rows=32, cols=512):
@@ -479,6 +528,7 @@ def run_cuda(args):
         "config": {"workload": (WORKLOAD if not args.linears else WORKLOAD + f" [subset {args.linears}]")
                                + (" [variant: independent scales of the two parts]" if args.independent_scales else ""), "M_per_gpu": M, "bank": BANK_70B, "k": K_70B, "positions": "static",
                    "step": "sq_encode + sq_gemm for each of the four linears",
+                   "gemm_mode": "sq_gemm with a workspace: expand_a8_kernel writes the merged 8-bit activations once (M*K bytes), gemm_kernel consumes them; the gemm_fused block times plain sq_gemm, whose sparse part runs inside the GEMM kernel",
                    "l2": "inputs larger than L2 (packed weights + activations + outputs of a step ~2.5 GB)",
                    "sharding": "tokens (M) per rank, weights replicated, no data-path collective"},
         "clocks": clk,
@@ -495,9 +545,11 @@ def run_cuda(args):
                      "frac_of_nominal_4500": gemm_tops / 4500.0,
                      "avg_launch_ms": gemm_ms / n_gemm, "launches": n_gemm,
                      "algorithmic_bytes_per_launch": sum(l.gemm_bytes for l in layers) / len(layers),
+                     # the timed mode also writes and re-reads the 8-bit copy of the activations
+                     "bytes_per_launch_incl_8bit_copy": sum(l.gemm_bytes + 2.0 * l.M * l.K for l in layers) / len(layers),
                      "traffic": sum(l.gemm_bytes for l in layers) / len(layers)
                      * GEMM_CAPTURE_TRAFFIC_BYTES / GEMM_CAPTURE_ALGO_BYTES,
-                     "traffic_note": "ncu DRAM bytes of a smaller captured launch scaled by algorithmic bytes (see profiles/)"},
+                     "traffic_note": "EXTRAPOLATED: ncu DRAM bytes of a captured M=2048 launch (whose 8-bit copy stayed in L2) scaled by algorithmic bytes; the kernel is tensor-bound, traffic < algorithmic bytes (see profiles/)"},
         "roofline_encode_in_step": {"kernel": "sq_encode", "bound": "hbm", "achieved": enc_gbs,
                                     "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": enc_gbs / peaks["hbm_gbs"],
                                     "peak_source": peaks["source"], "traffic": None},
@@ -505,15 +557,20 @@ def run_cuda(args):
     if rank == 0:
         if not args.no_encode_bench:
             del host_X, host_out
-            line["gemm_8b_dynamic"] = {"workload": "8B-decoder-shaped linears, b=64, k=8, dynamic positions; per-launch CUDA events, median of 20 after 10 warm-ups (small inputs may sit in L2)",
-                                       "results": bench_8b_dynamic(sq, dev, peaks)}
             if not args.no_sweep:
-                line["format_sweep"] = {"workload": "M=4096, K=N=8192; b x k/b x {dynamic, static, static with independent scales} x outlier channels x{10,50}; Student-t nu=3 activations, 1% outlier channels; rel_err = ||out - fp32(X W^T)||_F / ||fp32(X W^T)||_F",
-                                        "results": bench_format_sweep(sq, dev, peaks)}
-            line["encode"] = {"workload": "sq_encode alone: bf16 8192 x 8192, Student-t nu=3, 0.5% channels x50, b=64; 3 inputs in rotation (> L2)",
-                              "observed_bound": {"dynamic": "alu: integer/logic pipe 81% busy (ncu), DRAM 30% of peak; exact top-k by sorting network costs ~9 ALU-pipe lane-instructions per element",
-                                                 "static": "issue/latency: ALU pipe 61%, DRAM 43% of peak; 8192 rows are ~7 rounds of work plus ~8 us of ramp-up and tail"},
-                              "results": bench_encode_only(sq, dev, peaks)}
+                line["format_sweep"] = {"workload": "M=4096, K=N=8192; b x k/b x {dynamic, static, static with independent scales} x outlier channels x{10,50}; Student-t nu=3, 1% outlier channels; rel_err = ||out - fp32(X W^T)||_F / ||fp32(X W^T)||_F",
+                                        **bench_format_sweep(sq, dev, peaks)}
+            line["gemm_8b_dynamic"] = {"workload": "8B-decoder-shaped linears + the single-GEMM configuration (last row), b=64, k=8, dynamic; median of 20 CUDA-event pairs (small inputs may sit in L2); fused = plain sq_gemm without a workspace",
+                                       **bench_8b_dynamic(sq, dev, peaks)}
+            line["encode"] = {"workload": "sq_encode alone: bf16 8192 x 8192, Student-t nu=3, 0.5% channels x50, b=64; 3 inputs in rotation (> L2); median of 50 launches",
+                              "observed_bound": "dynamic: integer/logic pipe (ncu: 72% busy, DRAM 32%); static: launch + ramp of a 40 us kernel (5.2 TB/s on 32768 rows)",
+                              **bench_encode_only(sq, dev, peaks)}
+            line["gemm_fused"] = {"workload": "70B-shaped linears, M=4096, b=128, k=16: plain sq_gemm (sparse part inside the GEMM kernel) vs the workspace call",
+                                  **bench_gemm_fused(sq, layers, dev, peaks)}
+            same = bench_same_run_int8(dev)
+            line["same_run"] = {"int8_gemm_TOPS": None if same is None else round(same, 1),
+                                "what": "torch._int_mm M=4096 N=K=8192 (vendor INT8 GEMM, yardstick only)",
+                                "roofline_frac_of_same_run_int8": None if same is None else round(gemm_tops / same, 3)}
         if not args.no_cpu_baseline and world == 1:
             K, N = SHAPES_70B[1]
             ops = dt = 0.0
@@ -525,7 +582,7 @@ def run_cuda(args):
                 ops, dt, n = ops + o, dt + d, n + 1
             line["cpu_baseline"] = {"value": ops / dt / 1e12, "unit": UNIT, "cores": cores, "kind": "oracle",
                                     "sample": f"{n} x (encode + GEMM of 128 token rows x 1024 output channels of the (K,N)=({K},{N}) linear)"}
-        print(json.dumps(line))
+        print(json.dumps(line, separators=(",", ":")))
     if dist is not None:
         dist.barrier()
         dist.destroy_process_group()
