@@ -212,7 +212,7 @@ sq_status sq_gemm_workspace_bytes(const sq_format* fmt, int64_t M, int64_t N, in
   *bytes = 0;
   if (M == 0 || N == 0) return SQ_OK;
   SQ_TRY(check_device());
-  *bytes = gemm_workspace_bytes(is_static(fmt), is_indep(fmt), M, N, K);
+  *bytes = gemm_workspace_bytes(fmt->bank, fmt->k, is_static(fmt), is_indep(fmt), M, N, K);
   return SQ_OK;
 }
 
@@ -238,7 +238,7 @@ sq_status sq_gemm_ws(const sq_format* fmt, const sq_encoded* A, const sq_weights
   if (status == nullptr) return SQ_ERR_CUDA;
   return from_cuda(launch_gemm(fmt->bank, fmt->k, is_indep(fmt), *A, *W, positions, M, N, K,
                                static_cast<uint16_t*>(out_bf16), acc_out, status, workspace,
-                               workspace == nullptr ? 0 : workspace_bytes, static_cast<cudaStream_t>(cuda_stream)));
+                               workspace == nullptr ? 0 : workspace_bytes, true, static_cast<cudaStream_t>(cuda_stream)));
 }
 
 sq_status sq_gemm_static_scratch(const sq_format* fmt, const sq_encoded* A, const sq_weights* W,

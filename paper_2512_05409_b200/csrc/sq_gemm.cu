@@ -1209,8 +1209,9 @@ static bool use_a8(bool /*is_static*/, int64_t M, int64_t N, int64_t K, size_t w
   return M > BM && (N + BN - 1) / BN >= 4 && (size_t)M * (size_t)K <= ws_bytes;
 }
 
-size_t gemm_workspace_bytes(bool is_static, bool indep, int64_t M, int64_t N, int64_t K) {
+size_t gemm_workspace_bytes(int b, int k, bool is_static, bool indep, int64_t M, int64_t N, int64_t K) {
   if (indep) return 0;  // two accumulators: neither a merged 8-bit operand nor split-K is built for it
+  if (gemm_stream_serves(b, k, is_static, M, K)) return 0;  // the weight-streaming kernel needs none
   int dev = 0, sms = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) return 0;
   if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
@@ -1221,7 +1222,10 @@ size_t gemm_workspace_bytes(bool is_static, bool indep, int64_t M, int64_t N, in
 
 cudaError_t launch_gemm(int b, int k, bool indep, const sq_encoded& A, const sq_weights& W,
                         const uint8_t* positions, int64_t M, int64_t N, int64_t K, uint16_t* out,
-                        int32_t* acc_out, int* status, void* workspace, size_t workspace_bytes, cudaStream_t st) {
+                        int32_t* acc_out, int* status, void* workspace, size_t workspace_bytes, bool allow_stream,
+                        cudaStream_t st) {
+  if (allow_stream && !indep && gemm_stream_serves(b, k, positions != nullptr, M, K))
+    return launch_gemm_stream(b, k, A, W, positions, M, N, K, out, acc_out, status, st);
   GemmParams p;
   p.dq4 = A.dq4;
   p.vals = A.vals;
@@ -1547,7 +1551,7 @@ cudaError_t launch_gemm_static_scratch(int b, int k, const sq_encoded& A, const 
     if (ptr == nullptr) return cudaErrorInvalidSymbol;
     scratch_addr[dev].store(ptr, std::memory_order_release);
   }
-  return launch_gemm(b, k, false, A, W, positions, M, N, K, out, acc_out, status, ptr, kStaticScratchBytes, st);
+  return launch_gemm(b, k, false, A, W, positions, M, N, K, out, acc_out, status, ptr, kStaticScratchBytes, false, st);
 }
 
 }  // namespace sq

@@ -36,11 +36,18 @@ cudaError_t launch_encode(int b, int k, bool is_static, bool indep, const uint16
 cudaError_t launch_decode(int b, int k, const sq_encoded& A, const uint8_t* positions, int64_t M,
                           int64_t K, uint16_t* out, cudaStream_t st);
 
+// allow_stream: few-token calls the weight-streaming kernel serves go to it (it needs no workspace).
 cudaError_t launch_gemm(int b, int k, bool indep, const sq_encoded& A, const sq_weights& W,
                         const uint8_t* positions, int64_t M, int64_t N, int64_t K, uint16_t* out,
-                        int32_t* acc_out, int* status, void* workspace, size_t workspace_bytes, cudaStream_t st);
-// Bytes of workspace launch_gemm can make use of for this shape (0: none).
-size_t gemm_workspace_bytes(bool is_static, bool indep, int64_t M, int64_t N, int64_t K);
+                        int32_t* acc_out, int* status, void* workspace, size_t workspace_bytes, bool allow_stream,
+                        cudaStream_t st);
+// Bytes of workspace launch_gemm can make use of for this shape and format (0: none).
+size_t gemm_workspace_bytes(int b, int k, bool is_static, bool indep, int64_t M, int64_t N, int64_t K);
+// The weight-streaming kernel for at most 32 token rows (sq_gemm_stream.cu).
+bool gemm_stream_serves(int b, int k, bool is_static, int64_t M, int64_t K);
+cudaError_t launch_gemm_stream(int b, int k, const sq_encoded& A, const sq_weights& W, const uint8_t* positions,
+                               int64_t M, int64_t N, int64_t K, uint16_t* out, int32_t* acc_out, int* status,
+                               cudaStream_t st);
 // The same launch with the library's own fixed scratch array as the workspace (no allocation).
 cudaError_t launch_gemm_static_scratch(int b, int k, const sq_encoded& A, const sq_weights& W,
                                        const uint8_t* positions, int64_t M, int64_t N, int64_t K, uint16_t* out,
