@@ -15,16 +15,17 @@ import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "sq_oracle.cpp")
+_SRC_FP = os.path.join(_HERE, "sq_oracle_fp.cpp")
 _LIB = os.path.join(_HERE, "libsq_oracle.so")
 _lib = None
 
 
 def build(force: bool = False) -> str:
     """Compile the oracle with g++ (-O2, no fast-math, OpenMP over rows)."""
-    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < max(os.path.getmtime(_SRC), os.path.getmtime(_SRC_FP)):
         tmp = _LIB + f".tmp{os.getpid()}"
         subprocess.check_call(["g++", "-O2", "-fopenmp", "-ffp-contract=off", "-shared", "-fPIC",
-                               "-o", tmp, _SRC])
+                               "-o", tmp, _SRC, _SRC_FP])
         os.replace(tmp, _LIB)
     return _LIB
 
@@ -187,3 +188,87 @@ def gemm_indep(b: int, k: int, A: Encoded, W: Weights, positions: np.ndarray, ro
     if ov:
         raise OverflowError("an accumulator does not fit in int32")
     return lo, hi, ref, out
+
+
+# ---------------------------------------------------------------------------- floating-point variant (FP8 sparse + FP4 dense)
+
+@dataclass
+class FpEncoded:
+    dq4: np.ndarray      # uint8 [M, K/2] E2M1 codes, two per byte
+    vals: np.ndarray     # uint8 [M, G, k] E4M3 codes
+    idx: np.ndarray | None
+    s_hi: np.ndarray
+    s_lo: np.ndarray
+    shift: np.ndarray
+    a8: np.ndarray       # uint8 [M, K] merged E4M3 operand
+
+
+@dataclass
+class FpWeights:
+    wq4: np.ndarray      # uint8 [N, K/2] E2M1 codes
+    s_w: np.ndarray
+    w8: np.ndarray       # uint8 [N, K] the same values as E4M3 codes
+
+
+def fp_tables():
+    e2 = np.zeros(16, dtype=np.float64)
+    e4 = np.zeros(256, dtype=np.float64)
+    _load().sqo_fp_tables(_p(e2), _p(e4))
+    return e2, e4
+
+
+def fp_round(kind: str, values: np.ndarray) -> np.ndarray:
+    v = np.ascontiguousarray(values, dtype=np.float64).ravel()
+    out = np.zeros(v.size, dtype=np.uint8)
+    _load().sqo_fp_round(ctypes.c_int(0 if kind == "e2m1" else 1), _p(v), _l(v.size), _p(out))
+    return out.reshape(np.shape(values))
+
+
+def fp_pack_weights(W_bits: np.ndarray) -> FpWeights:
+    N, K = W_bits.shape
+    wq4 = np.zeros((N, K // 2), dtype=np.uint8)
+    s_w = np.zeros(N, dtype=np.float32)
+    w8 = np.zeros((N, K), dtype=np.uint8)
+    _load().sqo_fp_pack_weights(_p(W_bits), _l(N), _l(K), _p(wq4), _p(s_w), _p(w8))
+    return FpWeights(wq4, s_w, w8)
+
+
+def fp_encode(b: int, k: int, X_bits: np.ndarray, positions: np.ndarray | None = None) -> FpEncoded:
+    M, K = X_bits.shape
+    G = K // b
+    dq4 = np.zeros((M, K // 2), dtype=np.uint8)
+    vals = np.zeros((M, G, k), dtype=np.uint8)
+    idx = np.zeros((M, G, k), dtype=np.uint8) if positions is None else None
+    s_hi = np.zeros(M, dtype=np.float32)
+    s_lo = np.zeros(M, dtype=np.float32)
+    shift = np.zeros(M, dtype=np.uint8)
+    a8 = np.zeros((M, K), dtype=np.uint8)
+    _load().sqo_fp_encode(ctypes.c_int(b), ctypes.c_int(k), _p(X_bits), _l(M), _l(K), _p(positions), _p(dq4), _p(vals),
+                          _p(idx), _p(s_hi), _p(s_lo), _p(shift), _p(a8))
+    return FpEncoded(dq4, vals, idx, s_hi, s_lo, shift, a8)
+
+
+def fp_gemm(A: FpEncoded, W: FpWeights, rows=None, cols=None):
+    """Returns (acc float32, sum of |products| float32, ref32 float32, out bf16-bits), each [n_rows, n_cols]."""
+    M, K = A.a8.shape
+    N = W.wq4.shape[0]
+    rows_a = None if rows is None else np.ascontiguousarray(rows, dtype=np.int64)
+    cols_a = None if cols is None else np.ascontiguousarray(cols, dtype=np.int64)
+    R = M if rows_a is None else len(rows_a)
+    C = N if cols_a is None else len(cols_a)
+    acc = np.zeros((R, C), dtype=np.float32)
+    sabs = np.zeros((R, C), dtype=np.float32)
+    ref = np.zeros((R, C), dtype=np.float32)
+    out = np.zeros((R, C), dtype=np.uint16)
+    _load().sqo_fp_gemm(_p(A.a8), _p(A.s_hi), _p(W.wq4), _p(W.s_w), _l(M), _l(N), _l(K), _p(rows_a), _l(R), _p(cols_a),
+                        _l(C), _p(acc), _p(sabs), _p(ref), _p(out))
+    return acc, sabs, ref, out
+
+
+def fp_decode(b: int, k: int, A: FpEncoded, positions: np.ndarray | None = None):
+    M, K = A.a8.shape
+    xf = np.zeros((M, K), dtype=np.float32)
+    xb = np.zeros((M, K), dtype=np.uint16)
+    _load().sqo_fp_decode(ctypes.c_int(b), ctypes.c_int(k), _p(A.dq4), _p(A.vals), _p(A.idx), _p(positions), _p(A.s_hi),
+                          _p(A.s_lo), _l(M), _l(K), _p(xf), _p(xb))
+    return xf, xb
