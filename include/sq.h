@@ -249,6 +249,39 @@ sq_status sq_gemm_static_scratch(const sq_format* fmt, const sq_encoded* A, cons
                                  const uint8_t* positions, int64_t M, int64_t N, int64_t K, void* out_bf16,
                                  int32_t* acc_out, void* cuda_stream);
 
+/* ---------------------------------------------------------------------------------------------
+ * Floating-point variant: h_high = FP8 (E4M3), h_low = FP4 (E2M1).  Section 3.1 defines the format
+ * for floating-point precisions as well; the appendix "FP Quantization Results" uses this pair.
+ * The same structs are used with these meanings:
+ *   sq_encoded.dq4   uint8 [M, K/2]   dense E2M1 codes (sign, 2 exponent bits, 1 mantissa bit), element
+ *                                     2i in the low nibble; code 0 at the bank's k selected positions
+ *   sq_encoded.vals  [M, G, k]        sparse E4M3 bytes (OCP FP8: no infinities, largest finite 448)
+ *   sq_encoded.idx, s_hi, s_lo, shift as for the integer format; shift e in 0..6
+ *   a8               uint8 [M, K]     the MERGED operand the GEMM reads: at a dense place the E4M3 byte of
+ *                                     (dense value * 2^e), exact; at a selected place the sparse entry
+ *   wq4              uint8 [N, K/2]   E2M1 weight codes;  s_w float [N];  w8 uint8 [N, K]: the same weight
+ *                                     values as E4M3 bytes (the GEMM's second operand)
+ * Every rounding is to the nearest representable value of the EXACT product, ties to the even
+ * code, saturating; a value that rounds to zero is stored as +0.  Per token row, with a_j = X[m,j]:
+ *   amax = max_j |a_j|;  amax == 0: every code 0, shift 0, scales 0.  Otherwise
+ *   inv = 256.0f / amax, s_hi = amax / 256.0f        (the row maximum maps to 256, not to 448, so
+ *                                                     that every dense value times 2^e is an E4M3 number)
+ *   S as for sq_encode (dynamic: the k largest |a_j| of the bank, ties to the smaller j; static: positions)
+ *   j in S: vals = E4M3(a_j * inv);  rmax = max over j not in S of |a_j|
+ *   e = min{ e in 0..6 : rmax * inv * 2^-e <= 6 };  s_lo = s_hi * 2^e;  j not in S: dq4 = E2M1(a_j * inv * 2^-e)
+ * Weights, per output channel: wmax = max_j |W[n,j]|, s_w = wmax / 6.0f, code = E2M1(W[n,j] * (6.0f / wmax)).
+ * GEMM: acc[m,n] = sum_j value(a8[m,j]) * value(w8[n,j]) on the FP8 tensor-core path with fp32
+ * accumulation (the order of the additions is the hardware's), out = bf16_rne((acc * s_hi[m]) * s_w[n]).
+ * acc_out: device float [M, N] or NULL.  fmt->pos_mode: SQ_POS_DYNAMIC or SQ_POS_STATIC. */
+sq_status sq_fp_pack_weights(const void* W_bf16, int64_t N, int64_t K, uint8_t* wq4, float* s_w, uint8_t* w8,
+                             void* cuda_stream);
+sq_status sq_fp_encode(const sq_format* fmt, const void* X_bf16, int64_t M, int64_t K, const uint8_t* positions,
+                       sq_encoded* out, uint8_t* a8, void* cuda_stream);
+sq_status sq_fp_gemm(const float* s_hi, const uint8_t* a8, const float* s_w, const uint8_t* w8, int64_t M, int64_t N,
+                     int64_t K, void* out_bf16, float* acc_out, void* cuda_stream);
+sq_status sq_fp_decode(const sq_format* fmt, const sq_encoded* A, const uint8_t* positions, int64_t M, int64_t K,
+                       void* out_bf16, void* cuda_stream);
+
 /* Decode (inverse of Eq. 1): out[m,j] = bf16_rne(s_hi[m]*vals) at selected positions,
  * bf16_rne(s_lo[m]*dq4) elsewhere.  out_bf16: device bf16 [M, K], written. */
 sq_status sq_decode(const sq_format* fmt, const sq_encoded* A, const uint8_t* positions,

@@ -73,10 +73,15 @@ def _load() -> ctypes.CDLL:
     lib.sq_gemm_static_scratch.argtypes = [P(sq_format), P(sq_encoded), P(sq_weights), VP, I64, I64, I64, VP, VP, VP]
     lib.sq_decode.argtypes = [P(sq_format), P(sq_encoded), VP, I64, I64, VP, VP]
     lib.sq_device_status.argtypes = [VP]
+    lib.sq_fp_pack_weights.argtypes = [VP, I64, I64, VP, VP, VP, VP]
+    lib.sq_fp_encode.argtypes = [P(sq_format), VP, I64, I64, VP, P(sq_encoded), VP, VP]
+    lib.sq_fp_gemm.argtypes = [VP, VP, VP, VP, I64, I64, I64, VP, VP, VP]
+    lib.sq_fp_decode.argtypes = [P(sq_format), P(sq_encoded), VP, I64, I64, VP, VP]
     lib.sq_device_status_word.argtypes = [P(VP)]
     for name in ("sq_encoded_sizes", "sq_weights_sizes", "sq_calib_positions", "sq_pack_weights",
                  "sq_encode", "sq_gemm", "sq_gemm_ws", "sq_gemm_workspace_bytes", "sq_gemm_static_scratch", "sq_decode",
-                 "sq_device_status", "sq_device_status_word"):
+                 "sq_device_status", "sq_device_status_word", "sq_fp_pack_weights", "sq_fp_encode", "sq_fp_gemm",
+                 "sq_fp_decode"):
         getattr(lib, name).restype = ctypes.c_int
     return lib
 
@@ -315,6 +320,62 @@ def sq_decode(fmt: sq_format, A: Encoded, positions: torch.Tensor | None = None,
 
 def sq_device_status(stream=None) -> int:
     return int(_lib.sq_device_status(_stream(stream)))
+
+
+# ---------------------------------------------------------------------------- floating-point variant
+
+@dataclass
+class FpWeights:
+    """Torch-owned buffers of the floating-point variant's weights."""
+    wq4: torch.Tensor      # uint8 [N, K/2] E2M1 codes
+    s_w: torch.Tensor      # float32 [N]
+    w8: torch.Tensor       # uint8 [N, K] the same values as E4M3 bytes
+
+
+def sq_fp_pack_weights(W: torch.Tensor, stream=None) -> FpWeights:
+    N, K = _bf16_2d(W, "W")
+    out = FpWeights(torch.empty(N, K // 2, dtype=torch.uint8, device=W.device),
+                    torch.empty(max(N, 4), dtype=torch.float32, device=W.device)[:N],
+                    torch.empty(N, K, dtype=torch.uint8, device=W.device))
+    _check(_lib.sq_fp_pack_weights(_ptr(W), N, K, _ptr(out.wq4), _ptr(out.s_w), _ptr(out.w8), _stream(stream)),
+           "sq_fp_pack_weights")
+    return out
+
+
+def sq_fp_encode(fmt: sq_format, X: torch.Tensor, positions: torch.Tensor | None = None, out: Encoded | None = None,
+                 a8: torch.Tensor | None = None, stream=None):
+    """Returns (Encoded, a8): the encoding (vals viewed as int8 holds E4M3 bytes) and the merged E4M3 operand."""
+    M, K = _bf16_2d(X, "X")
+    if out is None:
+        out = alloc_encoded(fmt, M, K, X.device)
+    if a8 is None:
+        a8 = torch.empty(max(M * K, 16), dtype=torch.uint8, device=X.device)[: M * K].view(M, K)
+    cs = out.c_struct()
+    _check(_lib.sq_fp_encode(ctypes.byref(fmt), _ptr(X), M, K, _ptr(positions), ctypes.byref(cs), _ptr(a8),
+                             _stream(stream)), "sq_fp_encode")
+    return out, a8
+
+
+def sq_fp_gemm(A: Encoded, a8: torch.Tensor, W: FpWeights, out: torch.Tensor | None = None,
+               acc_out: torch.Tensor | None = None, stream=None) -> torch.Tensor:
+    M, K = a8.shape
+    N = W.w8.shape[0]
+    if out is None:
+        out = _buf(M * N * 2, torch.bfloat16, a8.device)[: M * N].view(M, N)
+    _check(_lib.sq_fp_gemm(_ptr(A.s_hi), _ptr(a8), _ptr(W.s_w), _ptr(W.w8), M, N, K, _ptr(out), _ptr(acc_out),
+                           _stream(stream)), "sq_fp_gemm")
+    return out
+
+
+def sq_fp_decode(fmt: sq_format, A: Encoded, positions: torch.Tensor | None = None, out: torch.Tensor | None = None,
+                 stream=None) -> torch.Tensor:
+    M, K = A.dq4.shape[0], A.dq4.shape[1] * 2
+    if out is None:
+        out = _buf(M * K * 2, torch.bfloat16, A.dq4.device)[: M * K].view(M, K)
+    ca = A.c_struct()
+    _check(_lib.sq_fp_decode(ctypes.byref(fmt), ctypes.byref(ca), _ptr(positions), M, K, _ptr(out), _stream(stream)),
+           "sq_fp_decode")
+    return out
 
 
 def sq_device_status_word() -> int:

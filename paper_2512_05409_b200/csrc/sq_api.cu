@@ -288,6 +288,68 @@ sq_status sq_decode(const sq_format* fmt, const sq_encoded* A, const uint8_t* po
                                  static_cast<cudaStream_t>(cuda_stream)));
 }
 
+sq_status sq_fp_pack_weights(const void* W_bf16, int64_t N, int64_t K, uint8_t* wq4, float* s_w, uint8_t* w8,
+                             void* cuda_stream) {
+  SQ_TRY(check_k(K));
+  if (N < 0 || N % 8 != 0) return SQ_ERR_INVALID_ARG;
+  if (N == 0) return SQ_OK;
+  if (!W_bf16 || !wq4 || !s_w || !w8) return SQ_ERR_NULL_POINTER;
+  if (!aligned16(W_bf16) || !aligned16(wq4) || !aligned16(s_w) || !aligned16(w8)) return SQ_ERR_ALIGNMENT;
+  SQ_TRY(check_device());
+  return from_cuda(launch_fp_pack_weights(static_cast<const uint16_t*>(W_bf16), N, K, wq4, s_w, w8,
+                                          static_cast<cudaStream_t>(cuda_stream)));
+}
+
+sq_status sq_fp_encode(const sq_format* fmt, const void* X_bf16, int64_t M, int64_t K, const uint8_t* positions,
+                       sq_encoded* out, uint8_t* a8, void* cuda_stream) {
+  SQ_TRY(check_format(fmt));
+  if (is_indep(fmt)) return SQ_ERR_INVALID_ARG;
+  SQ_TRY(check_k(K));
+  if (M < 0) return SQ_ERR_INVALID_ARG;
+  if (M == 0) return SQ_OK;
+  if (X_bf16 == nullptr || a8 == nullptr) return SQ_ERR_NULL_POINTER;
+  if (!aligned16(X_bf16) || !aligned16(a8)) return SQ_ERR_ALIGNMENT;
+  SQ_TRY(check_positions(fmt, positions));
+  SQ_TRY(check_encoded(fmt, out));
+  SQ_TRY(check_device());
+  sq_encoded o = *out;
+  if (is_static(fmt)) o.idx = nullptr;
+  return from_cuda(launch_fp_encode(fmt->bank, fmt->k, static_cast<const uint16_t*>(X_bf16), M, K, positions, o, a8,
+                                    static_cast<cudaStream_t>(cuda_stream)));
+}
+
+sq_status sq_fp_gemm(const float* s_hi, const uint8_t* a8, const float* s_w, const uint8_t* w8, int64_t M, int64_t N,
+                     int64_t K, void* out_bf16, float* acc_out, void* cuda_stream) {
+  SQ_TRY(check_k(K));
+  if (M < 0 || N < 0 || N % 8 != 0 || M > INT32_MAX || N > INT32_MAX) return SQ_ERR_INVALID_ARG;
+  if (M == 0 || N == 0) return SQ_OK;
+  if (!s_hi || !a8 || !s_w || !w8 || !out_bf16) return SQ_ERR_NULL_POINTER;
+  if (!aligned16(a8) || !aligned16(w8) || !aligned16(out_bf16) || !aligned16(acc_out)) return SQ_ERR_ALIGNMENT;
+  SQ_TRY(check_device());
+  int* status = status_word();
+  if (status == nullptr) return SQ_ERR_CUDA;
+  return from_cuda(launch_fp_gemm(s_hi, a8, s_w, w8, M, N, K, static_cast<uint16_t*>(out_bf16), acc_out, status,
+                                  static_cast<cudaStream_t>(cuda_stream)));
+}
+
+sq_status sq_fp_decode(const sq_format* fmt, const sq_encoded* A, const uint8_t* positions, int64_t M, int64_t K,
+                       void* out_bf16, void* cuda_stream) {
+  SQ_TRY(check_format(fmt));
+  if (is_indep(fmt)) return SQ_ERR_INVALID_ARG;
+  SQ_TRY(check_k(K));
+  if (M < 0) return SQ_ERR_INVALID_ARG;
+  if (M == 0) return SQ_OK;
+  SQ_TRY(check_positions(fmt, positions));
+  SQ_TRY(check_encoded(fmt, A));
+  if (out_bf16 == nullptr) return SQ_ERR_NULL_POINTER;
+  if (!aligned16(out_bf16)) return SQ_ERR_ALIGNMENT;
+  SQ_TRY(check_device());
+  sq_encoded a = *A;
+  if (is_static(fmt)) a.idx = nullptr;
+  return from_cuda(launch_fp_decode(fmt->bank, fmt->k, a, positions, M, K, static_cast<uint16_t*>(out_bf16),
+                                    static_cast<cudaStream_t>(cuda_stream)));
+}
+
 sq_status sq_device_status(void* cuda_stream) {
   SQ_TRY(check_device());
   if (cudaStreamSynchronize(static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess) return SQ_ERR_CUDA;
