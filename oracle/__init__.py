@@ -16,16 +16,17 @@ import numpy as np
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "sq_oracle.cpp")
 _SRC_FP = os.path.join(_HERE, "sq_oracle_fp.cpp")
+_SRC_W = os.path.join(_HERE, "sq_oracle_w.cpp")
 _LIB = os.path.join(_HERE, "libsq_oracle.so")
 _lib = None
 
 
 def build(force: bool = False) -> str:
     """Compile the oracle with g++ (-O2, no fast-math, OpenMP over rows)."""
-    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < max(os.path.getmtime(_SRC), os.path.getmtime(_SRC_FP)):
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < max(os.path.getmtime(_SRC), os.path.getmtime(_SRC_FP), os.path.getmtime(_SRC_W)):
         tmp = _LIB + f".tmp{os.getpid()}"
         subprocess.check_call(["g++", "-O2", "-fopenmp", "-ffp-contract=off", "-shared", "-fPIC",
-                               "-o", tmp, _SRC, _SRC_FP])
+                               "-o", tmp, _SRC, _SRC_FP, _SRC_W])
         os.replace(tmp, _LIB)
     return _LIB
 
@@ -272,3 +273,54 @@ def fp_decode(b: int, k: int, A: FpEncoded, positions: np.ndarray | None = None)
     _load().sqo_fp_decode(ctypes.c_int(b), ctypes.c_int(k), _p(A.dq4), _p(A.vals), _p(A.idx), _p(positions), _p(A.s_hi),
                           _p(A.s_lo), _l(M), _l(K), _p(xf), _p(xb))
     return xf, xb
+
+
+# ---------------------------------------------------------------------------- SQ-format on weights (Algorithm 1's format)
+
+@dataclass
+class SqWeights:
+    wq4: np.ndarray      # uint8 [N, K/2]: INT4 codes, the pattern 1000 at high-precision places
+    w_hi: np.ndarray     # int8 [N, G, k]: the high-precision values, in position order
+    s_high: np.ndarray   # float32 [N]
+    s_low: np.ndarray    # float32 [N]
+
+
+def w_encode(b: int, k: int, W_bits: np.ndarray, importance: np.ndarray) -> SqWeights:
+    N, K = W_bits.shape
+    imp = np.ascontiguousarray(importance, dtype=np.float32)
+    wq4 = np.zeros((N, K // 2), dtype=np.uint8)
+    w_hi = np.zeros((N, K // b, k), dtype=np.int8)
+    s_high = np.zeros(N, dtype=np.float32)
+    s_low = np.zeros(N, dtype=np.float32)
+    _load().sqo_w_encode(ctypes.c_int(b), ctypes.c_int(k), _p(W_bits), _p(imp), _l(N), _l(K), _p(wq4), _p(w_hi),
+                         _p(s_high), _p(s_low))
+    return SqWeights(wq4, w_hi, s_high, s_low)
+
+
+def w_decode(b: int, k: int, Wq: SqWeights) -> np.ndarray:
+    N, Kh = Wq.wq4.shape
+    out = np.zeros((N, Kh * 2), dtype=np.float32)
+    _load().sqo_w_decode(ctypes.c_int(b), ctypes.c_int(k), _p(Wq.wq4), _p(Wq.w_hi), _p(Wq.s_high), _p(Wq.s_low), _l(N),
+                         _l(Kh * 2), _p(out))
+    return out
+
+
+def act_quant8(X_bits: np.ndarray):
+    M, K = X_bits.shape
+    xq = np.zeros((M, K), dtype=np.int8)
+    s_x = np.zeros(M, dtype=np.float32)
+    _load().sqo_act_quant8(_p(X_bits), _l(M), _l(K), _p(xq), _p(s_x))
+    return xq, s_x
+
+
+def w_gemm(b: int, k: int, xq: np.ndarray, s_x: np.ndarray, Wq: SqWeights):
+    """Returns (acc_lo int32, acc_hi int32, ref32 float32, out bf16-bits), each [M, N]."""
+    M, K = xq.shape
+    N = Wq.wq4.shape[0]
+    lo = np.zeros((M, N), dtype=np.int32)
+    hi = np.zeros((M, N), dtype=np.int32)
+    ref = np.zeros((M, N), dtype=np.float32)
+    out = np.zeros((M, N), dtype=np.uint16)
+    _load().sqo_w_gemm(ctypes.c_int(b), ctypes.c_int(k), _p(xq), _p(s_x), _p(Wq.wq4), _p(Wq.w_hi), _p(Wq.s_high),
+                       _p(Wq.s_low), _l(M), _l(N), _l(K), _p(lo), _p(hi), _p(ref), _p(out))
+    return lo, hi, ref, out
