@@ -282,6 +282,31 @@ sq_status sq_fp_gemm(const float* s_hi, const uint8_t* a8, const float* s_w, con
 sq_status sq_fp_decode(const sq_format* fmt, const sq_encoded* A, const uint8_t* positions, int64_t M, int64_t K,
                        void* out_bf16, void* cuda_stream);
 
+/* ---------------------------------------------------------------------------------------------
+ * SQ-format on WEIGHTS: the format part of Algorithm 1 ("SQ-format on Weights") with the storage
+ * of Section 3.2.1 and the weight-matrix figure.  Per bank of b input channels of an output
+ * channel the k most important weights (importance[n,j] >= 0 is an INPUT: the paper derives it
+ * from smoothing and a Hessian of calibration data; equal scores: smaller j first) are kept as
+ * INT8 in w_hi [N, K/b, k], compactly and in position order; wq4 [N, K/2] keeps its shape and
+ * holds at those places the code the symmetric INT4 range leaves unused (the bit pattern 1000),
+ * so the mask is implicit.  Separate per-channel scales (Algorithm 1's S_high, S_low):
+ *   s_high[n] = (largest selected |w|) / 127, s_low[n] = (largest other |w|) / 7 (0 for an all-zero part)
+ *   w_hi = clamp(RNE(w * (127.0f / hmax)), -127, 127);  wq4 = clamp(RNE(w * (7.0f / lmax)), -7, 7)
+ * Storage: K/2 + (K/b)*k bytes per channel = ((1-s)*8 + 4)/8 bytes per weight (Section 4.1's W(SQx)).
+ * sq_w_act_quant: per-token symmetric INT8 activations for the product below, s_x = amax / 127,
+ *   xq = clamp(RNE(x * (127.0f / amax)), -127, 127); xq [M, K] is written in the order the product
+ *   kernel reads it (element j of a group of 8 at byte (j & 1) * 4 + (j >> 1) of the group).
+ * sq_w_gemm: the decode-shaped product (weight bytes dominate), M <= 4 tokens, else SQ_ERR_UNSUPPORTED:
+ *   acc_lo[m,n] = sum over unmasked j of xq[m,j] * wq4[n,j];  acc_hi[m,n] = sum over masked j of xq[m,j] * w_hi
+ *   out[m,n] = bf16_rne( fmaf((float)acc_hi, s_high[n], (float)acc_lo * s_low[n]) * s_x[m] )
+ *   acc_out: device int32 [2, M, N] (acc_lo, then acc_hi) or NULL.  Only fmt->bank and fmt->k are used. */
+sq_status sq_w_encode(const sq_format* fmt, const void* W_bf16, const float* importance, int64_t N, int64_t K,
+                      uint8_t* wq4, int8_t* w_hi, float* s_high, float* s_low, void* cuda_stream);
+sq_status sq_w_act_quant(const void* X_bf16, int64_t M, int64_t K, int8_t* xq, float* s_x, void* cuda_stream);
+sq_status sq_w_gemm(const sq_format* fmt, const int8_t* xq, const float* s_x, const uint8_t* wq4, const int8_t* w_hi,
+                    const float* s_high, const float* s_low, int64_t M, int64_t N, int64_t K, void* out_bf16,
+                    int32_t* acc_out, void* cuda_stream);
+
 /* Decode (inverse of Eq. 1): out[m,j] = bf16_rne(s_hi[m]*vals) at selected positions,
  * bf16_rne(s_lo[m]*dq4) elsewhere.  out_bf16: device bf16 [M, K], written. */
 sq_status sq_decode(const sq_format* fmt, const sq_encoded* A, const uint8_t* positions,

@@ -77,11 +77,14 @@ def _load() -> ctypes.CDLL:
     lib.sq_fp_encode.argtypes = [P(sq_format), VP, I64, I64, VP, P(sq_encoded), VP, VP]
     lib.sq_fp_gemm.argtypes = [VP, VP, VP, VP, I64, I64, I64, VP, VP, VP]
     lib.sq_fp_decode.argtypes = [P(sq_format), P(sq_encoded), VP, I64, I64, VP, VP]
+    lib.sq_w_encode.argtypes = [P(sq_format), VP, VP, I64, I64, VP, VP, VP, VP, VP]
+    lib.sq_w_act_quant.argtypes = [VP, I64, I64, VP, VP, VP]
+    lib.sq_w_gemm.argtypes = [P(sq_format), VP, VP, VP, VP, VP, VP, I64, I64, I64, VP, VP, VP]
     lib.sq_device_status_word.argtypes = [P(VP)]
     for name in ("sq_encoded_sizes", "sq_weights_sizes", "sq_calib_positions", "sq_pack_weights",
                  "sq_encode", "sq_gemm", "sq_gemm_ws", "sq_gemm_workspace_bytes", "sq_gemm_static_scratch", "sq_decode",
                  "sq_device_status", "sq_device_status_word", "sq_fp_pack_weights", "sq_fp_encode", "sq_fp_gemm",
-                 "sq_fp_decode"):
+                 "sq_fp_decode", "sq_w_encode", "sq_w_act_quant", "sq_w_gemm"):
         getattr(lib, name).restype = ctypes.c_int
     return lib
 
@@ -375,6 +378,50 @@ def sq_fp_decode(fmt: sq_format, A: Encoded, positions: torch.Tensor | None = No
     ca = A.c_struct()
     _check(_lib.sq_fp_decode(ctypes.byref(fmt), ctypes.byref(ca), _ptr(positions), M, K, _ptr(out), _stream(stream)),
            "sq_fp_decode")
+    return out
+
+
+# ---------------------------------------------------------------------------- SQ-format on weights
+
+@dataclass
+class SqWeights:
+    """Torch-owned buffers of weights in SQ-format (implicit mask: the INT4 pattern 1000)."""
+    wq4: torch.Tensor      # uint8 [N, K/2]
+    w_hi: torch.Tensor     # int8 [N, K/b, k]
+    s_high: torch.Tensor   # float32 [N]
+    s_low: torch.Tensor    # float32 [N]
+
+
+def sq_w_encode(fmt: sq_format, W: torch.Tensor, importance: torch.Tensor, stream=None) -> SqWeights:
+    N, K = _bf16_2d(W, "W")
+    if importance.dtype != torch.float32 or importance.shape != W.shape or not importance.is_contiguous():
+        raise ValueError("importance must be a contiguous float32 tensor of W's shape")
+    out = SqWeights(torch.empty(N, K // 2, dtype=torch.uint8, device=W.device),
+                    torch.empty(N, K // fmt.bank, fmt.k, dtype=torch.int8, device=W.device),
+                    torch.empty(max(N, 4), dtype=torch.float32, device=W.device)[:N],
+                    torch.empty(max(N, 4), dtype=torch.float32, device=W.device)[:N])
+    _check(_lib.sq_w_encode(ctypes.byref(fmt), _ptr(W), _ptr(importance), N, K, _ptr(out.wq4), _ptr(out.w_hi),
+                            _ptr(out.s_high), _ptr(out.s_low), _stream(stream)), "sq_w_encode")
+    return out
+
+
+def sq_w_act_quant(X: torch.Tensor, stream=None):
+    """Returns (xq int8 [M, K] in the product kernel's element order, s_x float32 [M])."""
+    M, K = _bf16_2d(X, "X")
+    xq = torch.empty(max(M * K, 16), dtype=torch.int8, device=X.device)[: M * K].view(M, K)
+    s_x = torch.empty(max(M, 4), dtype=torch.float32, device=X.device)[:M]
+    _check(_lib.sq_w_act_quant(_ptr(X), M, K, _ptr(xq), _ptr(s_x), _stream(stream)), "sq_w_act_quant")
+    return xq, s_x
+
+
+def sq_w_gemm(fmt: sq_format, xq: torch.Tensor, s_x: torch.Tensor, W: SqWeights, out: torch.Tensor | None = None,
+              acc_out: torch.Tensor | None = None, stream=None) -> torch.Tensor:
+    M, K = xq.shape
+    N = W.wq4.shape[0]
+    if out is None:
+        out = _buf(M * N * 2, torch.bfloat16, xq.device)[: M * N].view(M, N)
+    _check(_lib.sq_w_gemm(ctypes.byref(fmt), _ptr(xq), _ptr(s_x), _ptr(W.wq4), _ptr(W.w_hi), _ptr(W.s_high),
+                          _ptr(W.s_low), M, N, K, _ptr(out), _ptr(acc_out), _stream(stream)), "sq_w_gemm")
     return out
 
 

@@ -350,6 +350,46 @@ sq_status sq_fp_decode(const sq_format* fmt, const sq_encoded* A, const uint8_t*
                                     static_cast<cudaStream_t>(cuda_stream)));
 }
 
+sq_status sq_w_encode(const sq_format* fmt, const void* W_bf16, const float* importance, int64_t N, int64_t K,
+                      uint8_t* wq4, int8_t* w_hi, float* s_high, float* s_low, void* cuda_stream) {
+  SQ_TRY(check_format(fmt));
+  SQ_TRY(check_k(K));
+  if (N < 0) return SQ_ERR_INVALID_ARG;
+  if (N == 0) return SQ_OK;
+  if (!W_bf16 || !importance || !wq4 || !w_hi || !s_high || !s_low) return SQ_ERR_NULL_POINTER;
+  if (!aligned16(W_bf16) || !aligned16(importance) || !aligned16(wq4) || !aligned16(w_hi)) return SQ_ERR_ALIGNMENT;
+  SQ_TRY(check_device());
+  return from_cuda(launch_wsq_encode(fmt->bank, fmt->k, static_cast<const uint16_t*>(W_bf16), importance, N, K, wq4,
+                                     w_hi, s_high, s_low, static_cast<cudaStream_t>(cuda_stream)));
+}
+
+sq_status sq_w_act_quant(const void* X_bf16, int64_t M, int64_t K, int8_t* xq, float* s_x, void* cuda_stream) {
+  SQ_TRY(check_k(K));
+  if (M < 0) return SQ_ERR_INVALID_ARG;
+  if (M == 0) return SQ_OK;
+  if (!X_bf16 || !xq || !s_x) return SQ_ERR_NULL_POINTER;
+  if (!aligned16(X_bf16) || !aligned16(xq)) return SQ_ERR_ALIGNMENT;
+  SQ_TRY(check_device());
+  return from_cuda(launch_wsq_act(static_cast<const uint16_t*>(X_bf16), M, K, xq, s_x,
+                                  static_cast<cudaStream_t>(cuda_stream)));
+}
+
+sq_status sq_w_gemm(const sq_format* fmt, const int8_t* xq, const float* s_x, const uint8_t* wq4, const int8_t* w_hi,
+                    const float* s_high, const float* s_low, int64_t M, int64_t N, int64_t K, void* out_bf16,
+                    int32_t* acc_out, void* cuda_stream) {
+  SQ_TRY(check_format(fmt));
+  SQ_TRY(check_k(K));
+  if (M < 0 || N < 0 || N % 8 != 0 || N > INT32_MAX) return SQ_ERR_INVALID_ARG;
+  if (M == 0 || N == 0) return SQ_OK;
+  if (M > 4) return SQ_ERR_UNSUPPORTED;
+  if (!xq || !s_x || !wq4 || !w_hi || !s_high || !s_low || !out_bf16) return SQ_ERR_NULL_POINTER;
+  if (!aligned16(xq) || !aligned16(wq4) || !aligned16(w_hi) || !aligned16(out_bf16)) return SQ_ERR_ALIGNMENT;
+  SQ_TRY(check_device());
+  const cudaError_t err = launch_wsq_gemm(fmt->bank, fmt->k, xq, s_x, wq4, w_hi, s_high, s_low, M, N, K,
+                                          static_cast<uint16_t*>(out_bf16), acc_out, static_cast<cudaStream_t>(cuda_stream));
+  return err == cudaErrorNotSupported ? SQ_ERR_UNSUPPORTED : from_cuda(err);
+}
+
 sq_status sq_device_status(void* cuda_stream) {
   SQ_TRY(check_device());
   if (cudaStreamSynchronize(static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess) return SQ_ERR_CUDA;

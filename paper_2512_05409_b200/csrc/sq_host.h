@@ -64,4 +64,12 @@ cudaError_t launch_fp_decode(int b, int k, const sq_encoded& A, const uint8_t* p
 cudaError_t launch_fp_gemm(const float* s_hi, const uint8_t* a8, const float* s_w, const uint8_t* w8, int64_t M, int64_t N,
                            int64_t K, uint16_t* out, float* acc_out, int* status, cudaStream_t st);
 
+// SQ-format on weights (sq_wsq.cu).
+cudaError_t launch_wsq_encode(int b, int k, const uint16_t* W, const float* I, int64_t N, int64_t K, uint8_t* wq4,
+                              int8_t* w_hi, float* s_high, float* s_low, cudaStream_t st);
+cudaError_t launch_wsq_act(const uint16_t* X, int64_t M, int64_t K, int8_t* xq, float* s_x, cudaStream_t st);
+cudaError_t launch_wsq_gemm(int b, int k, const int8_t* xq, const float* s_x, const uint8_t* wq4, const int8_t* w_hi,
+                            const float* s_high, const float* s_low, int64_t M, int64_t N, int64_t K, uint16_t* out,
+                            int32_t* acc_out, cudaStream_t st);
+
 }  // namespace sq

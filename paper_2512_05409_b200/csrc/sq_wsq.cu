@@ -1,0 +1,302 @@
+// SQ-format on WEIGHTS (format part of Algorithm 1; storage of Section 3.2.1 and the weight-matrix
+// figure): per bank of b input channels of an output channel the k most important weights are
+// kept as INT8, compactly and in position order, and the INT4 array holds the unused code 1000 at
+// their places, so the mask is implicit; each part has its own per-channel scale.  The importance
+// scores are an input (the paper derives them from smoothing and a Hessian of calibration data).
+//
+//   sqw_encode_kernel   one block per output channel: per-bank ranking by importance (ties to the
+//                       smaller index), the two maxima, both codes, compact values by ballot/popc
+//   sqw_act_kernel      per-token symmetric INT8 activations, written in the order the product
+//                       kernel reads them ([4 even | 4 odd] elements per 8)
+//   sqw_gemm_kernel     decode-shaped product for at most 4 tokens: bound by the weight stream.
+//                       The mask differs from channel to channel, so the sparse part is a gather
+//                       per output channel and runs on the general-purpose cores; with this few
+//                       tokens so does the dense part (packed 4-way integer dot products).  A warp
+//                       owns two output channels at a time, a lane whole banks (so the compact
+//                       values of a bank are counted off locally); the activations sit in shared
+//                       memory.  Two int32 sums per output, joined in fp32:
+//                         out = bf16(fmaf(acc_hi, S_high[n], acc_lo * S_low[n]) * s_x[m])
+#include "sq_device.cuh"
+#include "sq_host.h"
+
+namespace sq {
+
+namespace {
+
+__device__ __forceinline__ uint32_t wblock_max(uint32_t v, uint32_t* scratch) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = max(v, __shfl_xor_sync(0xffffffffu, v, o));
+  __syncthreads();
+  if (lane == 0) scratch[warp] = v;
+  __syncthreads();
+  uint32_t r = 0;
+  for (int q = 0; q < (int)(blockDim.x >> 5); ++q) r = max(r, scratch[q]);
+  return r;
+}
+
+}  // namespace
+
+template <int B>
+__global__ void __launch_bounds__(256) sqw_encode_kernel(int k, const uint16_t* __restrict__ W, const float* __restrict__ I,
+                                                         int64_t K, uint8_t* __restrict__ wq4, int8_t* __restrict__ w_hi,
+                                                         float* __restrict__ s_high, float* __restrict__ s_low) {
+  extern __shared__ __align__(16) uint8_t smem_w[];
+  uint16_t* srow = reinterpret_cast<uint16_t*>(smem_w);       // the channel's weights
+  uint8_t* ssel = smem_w + K * 2;                             // 1 at a selected place
+  __shared__ uint32_t scratch[8];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int64_t n = blockIdx.x, G = K / B;
+  constexpr int EPL = B / 32;
+  for (int64_t j = tid; j < K; j += 256) srow[j] = W[n * K + j];
+  // per-bank ranking: an element is selected when fewer than k elements of its bank beat it
+  // (larger score, or equal score and smaller index)
+  for (int64_t g = warp; g < G; g += 8) {
+    float sc[EPL];
+    int rank[EPL];
+#pragma unroll
+    for (int t = 0; t < EPL; ++t) {
+      sc[t] = I[n * K + g * B + lane + 32 * t];
+      rank[t] = 0;
+    }
+#pragma unroll
+    for (int u = 0; u < EPL; ++u)
+      for (int l = 0; l < 32; ++l) {
+        const float other = __shfl_sync(0xffffffffu, sc[u], l);
+        const int oj = l + 32 * u;
+#pragma unroll
+        for (int t = 0; t < EPL; ++t) rank[t] += (other > sc[t] || (other == sc[t] && oj < lane + 32 * t)) ? 1 : 0;
+      }
+#pragma unroll
+    for (int t = 0; t < EPL; ++t) ssel[g * B + lane + 32 * t] = rank[t] < k ? 1 : 0;
+  }
+  __syncthreads();
+  uint32_t hm = 0, lm = 0;
+  for (int64_t j = tid; j < K; j += 256) {
+    const uint32_t mag = srow[j] & 0x7FFFu;
+    if (ssel[j]) hm = max(hm, mag);
+    else lm = max(lm, mag);
+  }
+  const float hmax = bf16_bits_to_f32(wblock_max(hm, scratch)), lmax = bf16_bits_to_f32(wblock_max(lm, scratch));
+  const float inv_hi = hmax > 0.f ? __fdiv_rn(127.0f, hmax) : 0.f, inv_lo = lmax > 0.f ? __fdiv_rn(7.0f, lmax) : 0.f;
+  if (tid == 0) {
+    s_high[n] = hmax > 0.f ? __fdiv_rn(hmax, 127.0f) : 0.f;
+    s_low[n] = lmax > 0.f ? __fdiv_rn(lmax, 7.0f) : 0.f;
+  }
+  // INT4 array (the pattern 1000 at a selected place)
+  for (int64_t j2 = tid; j2 < K / 2; j2 += 256) {
+    uint32_t nb[2];
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      const int64_t j = 2 * j2 + h;
+      nb[h] = ssel[j] ? 8u : ((uint32_t)min(7, max(-7, rne_prod(bf16_bits_to_f32(srow[j]), inv_lo))) & 0xFu);
+    }
+    wq4[n * (K / 2) + j2] = (uint8_t)(nb[0] | (nb[1] << 4));
+  }
+  // compact INT8 values, in position order
+  for (int64_t g = warp; g < G; g += 8) {
+    int before = 0;
+#pragma unroll
+    for (int t = 0; t < EPL; ++t) {
+      const int64_t j = g * B + lane + 32 * t;
+      const bool sel = ssel[j] != 0;
+      const uint32_t mask = __ballot_sync(0xffffffffu, sel);
+      if (sel)
+        w_hi[(n * G + g) * k + before + __popc(mask & ((1u << lane) - 1u))] =
+            (int8_t)min(127, max(-127, rne_prod(bf16_bits_to_f32(srow[j]), inv_hi)));
+      before += __popc(mask);
+    }
+  }
+}
+
+// One block per token: s_x = amax / 127, xq = clamp(RNE(x * 127 / amax)); element j of a group of 8 goes
+// to byte (j & 1) * 4 + (j >> 1) of the group.
+__global__ void __launch_bounds__(256) sqw_act_kernel(const uint16_t* __restrict__ X, int64_t K, int8_t* __restrict__ xq,
+                                                      float* __restrict__ s_x) {
+  __shared__ uint32_t scratch[8];
+  const int tid = threadIdx.x;
+  const int64_t m = blockIdx.x;
+  uint32_t mx = 0;
+  for (int64_t j = tid; j < K; j += 256) mx = max(mx, (uint32_t)(X[m * K + j] & 0x7FFFu));
+  const float amax = bf16_bits_to_f32(wblock_max(mx, scratch));
+  const float inv = amax > 0.f ? __fdiv_rn(127.0f, amax) : 0.f;
+  if (tid == 0) s_x[m] = amax > 0.f ? __fdiv_rn(amax, 127.0f) : 0.f;
+  for (int64_t j = tid; j < K; j += 256) {
+    const int q = min(127, max(-127, rne_prod(bf16_bits_to_f32(X[m * K + j]), inv)));
+    xq[m * K + (j & ~(int64_t)7) + (j & 1) * 4 + ((j & 7) >> 1)] = (int8_t)q;
+  }
+}
+
+namespace {
+constexpr int kWsqWarps = 8;
+constexpr int kWsqCh = 2;  // output channels a warp works on at a time
+}
+
+// MT: tokens (1..4).  Shared memory: the reordered INT8 activations [MT][K].
+template <int B, int MT>
+__global__ void __launch_bounds__(kWsqWarps * 32) sqw_gemm_kernel(int k, const int8_t* __restrict__ xq,
+                                                                  const float* __restrict__ s_x,
+                                                                  const uint8_t* __restrict__ wq4,
+                                                                  const int8_t* __restrict__ w_hi,
+                                                                  const float* __restrict__ s_high,
+                                                                  const float* __restrict__ s_low, int M, int N, int K,
+                                                                  uint16_t* __restrict__ out, int32_t* __restrict__ acc_out) {
+  extern __shared__ __align__(16) int8_t sx[];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int G = K / B;
+  constexpr int WPB = B / 8;  // 32-bit words of nibbles per bank
+  for (int i = tid; i < MT * (K / 16); i += kWsqWarps * 32) {
+    const int m = i / (K / 16), c = i % (K / 16);
+    reinterpret_cast<uint4*>(sx)[i] = m < M ? __ldg(reinterpret_cast<const uint4*>(xq + (size_t)m * K) + c) : make_uint4(0, 0, 0, 0);
+  }
+  __syncthreads();
+  const int pairs = (N + kWsqCh - 1) / kWsqCh;
+  for (int pr = blockIdx.x * kWsqWarps + warp; pr < pairs; pr += gridDim.x * kWsqWarps) {
+    int lo[kWsqCh][MT], hi[kWsqCh][MT];
+#pragma unroll
+    for (int c = 0; c < kWsqCh; ++c)
+#pragma unroll
+      for (int m = 0; m < MT; ++m) lo[c][m] = hi[c][m] = 0;
+    for (int g = lane; g < G; g += 32) {
+      // the bank's activations, reused for both channels
+      const int8_t* xb = sx + g * B;
+#pragma unroll
+      for (int c = 0; c < kWsqCh; ++c) {
+        const int n = min(pr * kWsqCh + c, N - 1);
+        const uint32_t* wp = reinterpret_cast<const uint32_t*>(wq4 + (size_t)n * (K / 2) + g * (B / 2));
+        const int8_t* hp = w_hi + ((size_t)n * G + g) * k;
+        int slot = 0;
+#pragma unroll
+        for (int w = 0; w < WPB; ++w) {
+          const uint32_t word = __ldg(wp + w);
+          // places holding the pattern 1000: bit 3 set and the three low bits clear
+          const uint32_t low3 = word & 0x77777777u;
+          uint32_t flags = word & 0x88888888u & ~((low3 + 0x77777777u) & 0x88888888u);
+          const uint32_t clean = word & ~((flags >> 3) * 15u);
+          const int ev = (int)((clean << 4) & 0xF0F0F0F0u), od = (int)(clean & 0xF0F0F0F0u);  // 16 * code, bytewise
+#pragma unroll
+          for (int m = 0; m < MT; ++m) {
+            const int2 xv = *reinterpret_cast<const int2*>(xb + (size_t)m * K + 8 * w);
+            lo[c][m] = __dp4a(ev, xv.x, __dp4a(od, xv.y, lo[c][m]));
+          }
+          while (flags) {  // the compact values of the bank belong to its masked places in position order
+            const int nibble = (__ffs((int)flags) - 1) >> 2;
+            flags &= flags - 1;
+            const int wv = hp[slot++];
+            const int at = 8 * w + (nibble & 1) * 4 + (nibble >> 1);
+#pragma unroll
+            for (int m = 0; m < MT; ++m) hi[c][m] += wv * (int)xb[(size_t)m * K + at];
+          }
+        }
+      }
+    }
+#pragma unroll
+    for (int c = 0; c < kWsqCh; ++c)
+#pragma unroll
+      for (int m = 0; m < MT; ++m) {
+        lo[c][m] = warp_sum(lo[c][m]);
+        hi[c][m] = warp_sum(hi[c][m]);
+      }
+    if (lane == 0) {
+#pragma unroll
+      for (int c = 0; c < kWsqCh; ++c) {
+        const int n = pr * kWsqCh + c;
+        if (n < N) {
+          const float sh = s_high[n], sl = s_low[n];
+#pragma unroll
+          for (int m = 0; m < MT; ++m)
+            if (m < M) {
+              const int a_lo = lo[c][m] >> 4;  // the dense codes were fed as 16 * code
+              const float f = __fmul_rn(__fmaf_rn((float)hi[c][m], sh, __fmul_rn((float)a_lo, sl)), s_x[m]);
+              out[(size_t)m * N + n] = (uint16_t)f32_to_bf16_bits(f);
+              if (acc_out != nullptr) {
+                acc_out[(size_t)m * N + n] = a_lo;
+                acc_out[(size_t)M * N + (size_t)m * N + n] = hi[c][m];
+              }
+            }
+        }
+      }
+    }
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+
+namespace {
+template <typename KernelT>
+cudaError_t ensure_smem(KernelT kernel, std::atomic<size_t>* limit, size_t smem) {
+  int dev = 0;
+  cudaError_t err = cudaGetDevice(&dev);
+  if (err != cudaSuccess) return err;
+  if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+  if (smem > limit[dev].load(std::memory_order_acquire)) {
+    std::lock_guard<std::mutex> lock(setup_mutex());
+    err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (err != cudaSuccess) return err;
+    limit[dev].store(smem, std::memory_order_release);
+  }
+  return cudaSuccess;
+}
+}  // namespace
+
+cudaError_t launch_wsq_encode(int b, int k, const uint16_t* W, const float* I, int64_t N, int64_t K, uint8_t* wq4,
+                              int8_t* w_hi, float* s_high, float* s_low, cudaStream_t st) {
+  const size_t smem = (size_t)K * 3;
+  cudaError_t err;
+#define SQ_WENC(BB)                                                                        \
+  do {                                                                                     \
+    static std::atomic<size_t> limit[64];                                                  \
+    err = ensure_smem(sqw_encode_kernel<BB>, limit, smem);                                 \
+    if (err != cudaSuccess) return err;                                                    \
+    sqw_encode_kernel<BB><<<(unsigned)N, 256, smem, st>>>(k, W, I, K, wq4, w_hi, s_high, s_low); \
+  } while (0)
+  if (b == 32) SQ_WENC(32);
+  else if (b == 64) SQ_WENC(64);
+  else SQ_WENC(128);
+#undef SQ_WENC
+  return cudaGetLastError();
+}
+
+cudaError_t launch_wsq_act(const uint16_t* X, int64_t M, int64_t K, int8_t* xq, float* s_x, cudaStream_t st) {
+  sqw_act_kernel<<<(unsigned)M, 256, 0, st>>>(X, K, xq, s_x);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_wsq_gemm(int b, int k, const int8_t* xq, const float* s_x, const uint8_t* wq4, const int8_t* w_hi,
+                            const float* s_high, const float* s_low, int64_t M, int64_t N, int64_t K, uint16_t* out,
+                            int32_t* acc_out, cudaStream_t st) {
+  if (M < 1 || M > 4) return cudaErrorNotSupported;
+  const int MT = M <= 1 ? 1 : (M <= 2 ? 2 : 4);
+  const size_t smem = (size_t)MT * K;
+  if (smem > 200 * 1024) return cudaErrorNotSupported;
+  int dev = 0, sms = 0;
+  cudaError_t err = cudaGetDevice(&dev);
+  if (err != cudaSuccess) return err;
+  err = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  if (err != cudaSuccess) return err;
+  const int64_t pairs = (N + kWsqCh - 1) / kWsqCh;
+  int64_t blocks = (pairs + kWsqWarps - 1) / kWsqWarps;
+  if (blocks > 2 * (int64_t)sms) blocks = 2 * (int64_t)sms;
+#define SQ_WGEMM(BB, MM)                                                                                           \
+  do {                                                                                                             \
+    static std::atomic<size_t> limit[64];                                                                          \
+    err = ensure_smem(sqw_gemm_kernel<BB, MM>, limit, smem);                                                       \
+    if (err != cudaSuccess) return err;                                                                            \
+    sqw_gemm_kernel<BB, MM><<<(unsigned)blocks, kWsqWarps * 32, smem, st>>>(k, xq, s_x, wq4, w_hi, s_high, s_low,  \
+                                                                          (int)M, (int)N, (int)K, out, acc_out);  \
+  } while (0)
+#define SQ_WGEMM_B(BB)             \
+  do {                             \
+    if (MT == 1) SQ_WGEMM(BB, 1);  \
+    else if (MT == 2) SQ_WGEMM(BB, 2); \
+    else SQ_WGEMM(BB, 4);          \
+  } while (0)
+  if (b == 32) SQ_WGEMM_B(32);
+  else if (b == 64) SQ_WGEMM_B(64);
+  else SQ_WGEMM_B(128);
+#undef SQ_WGEMM_B
+#undef SQ_WGEMM
+  return cudaGetLastError();
+}
+
+}  // namespace sq
