@@ -166,26 +166,39 @@ __global__ void __launch_bounds__(kWsqWarps * 32) sqw_gemm_kernel(int k, const i
         const uint32_t* wp = reinterpret_cast<const uint32_t*>(wq4 + (size_t)n * (K / 2) + g * (B / 2));
         const int8_t* hp = w_hi + ((size_t)n * G + g) * k;
         int slot = 0;
+        uint32_t words[WPB];
+#pragma unroll
+        for (int w4 = 0; w4 < WPB / 4; ++w4) {
+          const uint4 v = __ldg(reinterpret_cast<const uint4*>(wp) + w4);
+          words[4 * w4] = v.x;
+          words[4 * w4 + 1] = v.y;
+          words[4 * w4 + 2] = v.z;
+          words[4 * w4 + 3] = v.w;
+        }
 #pragma unroll
         for (int w = 0; w < WPB; ++w) {
-          const uint32_t word = __ldg(wp + w);
+          const uint32_t word = words[w];
           // places holding the pattern 1000: bit 3 set and the three low bits clear
           const uint32_t low3 = word & 0x77777777u;
           uint32_t flags = word & 0x88888888u & ~((low3 + 0x77777777u) & 0x88888888u);
           const uint32_t clean = word & ~((flags >> 3) * 15u);
           const int ev = (int)((clean << 4) & 0xF0F0F0F0u), od = (int)(clean & 0xF0F0F0F0u);  // 16 * code, bytewise
+          // the compact values of the bank belong to its masked places in position order: they are
+          // scattered into two words laid out like the dense ones, so that the sparse product is two
+          // more packed dot products against the activations already in registers
+          uint32_t hev = 0, hod = 0;
+          while (flags) {
+            const int nibble = (__ffs((int)flags) - 1) >> 2;
+            flags &= flags - 1;
+            const uint32_t wv = (uint32_t)(uint8_t)hp[slot++] << (8 * (nibble >> 1));
+            if (nibble & 1) hod |= wv;
+            else hev |= wv;
+          }
 #pragma unroll
           for (int m = 0; m < MT; ++m) {
             const int2 xv = *reinterpret_cast<const int2*>(xb + (size_t)m * K + 8 * w);
             lo[c][m] = __dp4a(ev, xv.x, __dp4a(od, xv.y, lo[c][m]));
-          }
-          while (flags) {  // the compact values of the bank belong to its masked places in position order
-            const int nibble = (__ffs((int)flags) - 1) >> 2;
-            flags &= flags - 1;
-            const int wv = hp[slot++];
-            const int at = 8 * w + (nibble & 1) * 4 + (nibble >> 1);
-#pragma unroll
-            for (int m = 0; m < MT; ++m) hi[c][m] += wv * (int)xb[(size_t)m * K + at];
+            hi[c][m] = __dp4a((int)hev, xv.x, __dp4a((int)hod, xv.y, hi[c][m]));
           }
         }
       }
