@@ -289,6 +289,27 @@ def bench_gemm_fused(sq, layers, dev, peaks, iters=10):
             "rows": rows}
 
 
+def bench_weights_sq(sq, dev, peaks):
+    """Weights in SQ-format (Algorithm 1's format, b=64, k=8 INT8 values per bank) against per-token INT8
+    activations on the 8B-decoder shapes at 1 and 4 tokens: GPU time per call replayed from a CUDA graph
+    and the weight stream (0.5 + k/b bytes per weight) over it."""
+    rows = []
+    fmt = sq.make_format(64, 8, True)
+    for (K, N) in SHAPES_8B:
+        W = gen.weights(N, K, seed=K + N, device=dev)
+        enc = sq.sq_w_encode(fmt, W, (W.float() ** 2).contiguous())
+        del W
+        for M in (1, 4):
+            xq, s_x = sq.sq_w_act_quant(gen.activations(M, K, seed=M, outlier_fraction=0.01, outlier_scale=20.0, device=dev))
+            out = torch.empty(M, N, dtype=torch.bfloat16, device=dev)
+            us = graph_replay_us(lambda: sq.sq_w_gemm(fmt, xq, s_x, enc, out=out))
+            gbs = N * K * (0.5 + 8 / 64) / (us * 1e-6) / 1e9
+            rows.append([M, K, N, round(us, 1), round(gbs), round(gbs / peaks["hbm_gbs"], 3)])
+        del enc
+        torch.cuda.empty_cache()
+    return {"cols": ["M", "K", "N", "gemm_us_graph_replay", "weight_stream_GBps", "of_measured_hbm"], "rows": rows}
+
+
 def bench_same_run_int8(dev, iters=10):
     """A vendor INT8 GEMM (torch._int_mm, M=4096, N=K=8192) timed in the same run: a yardstick for
     the tensor pipe's INT8 rate at this run's clocks, never on the product path."""
@@ -344,6 +365,19 @@ def bench_format_sweep(sq, dev, peaks, iters=5):
                     res.append([b, k, ("indep" if indep else "static") if static else "dynamic", int(scale),
                                 round(ms * 1e3, 1), round(tops), round(tops / int8_peak, 3), round(err, 4)])
                     del w, enc
+                # floating-point variant (sparse FP8 E4M3 + dense FP4 E2M1 activations, FP4 weights): the same
+                # shape on the FP8 tensor path (nominal rate = the INT8 one, so the same denominator)
+                for static in (False, True):
+                    fmt = sq.make_format(b, k, static)
+                    pos = sq.sq_calib_positions(fmt, calib, W) if static else None
+                    wf = sq.sq_fp_pack_weights(W)
+                    encf, a8 = sq.sq_fp_encode(fmt, X, pos)
+                    ms, _ = time_launches(lambda i: sq.sq_fp_gemm(encf, a8, wf, out=out), iters, 3)
+                    tops = 2.0 * M * N * K / (ms * 1e-3) / 1e12
+                    err = float((out.float() - ref).norm()) / ref_norm
+                    res.append([b, k, "fp8/fp4 static" if static else "fp8/fp4 dynamic", int(scale), round(ms * 1e3, 1),
+                                round(tops), round(tops / int8_peak, 3), round(err, 4)])
+                    del wf, encf, a8
         del X, calib, ref, out
         torch.cuda.empty_cache()
     torch.backends.cuda.matmul.allow_tf32 = tf32
@@ -558,7 +592,7 @@ def run_cuda(args):
         if not args.no_encode_bench:
             del host_X, host_out
             if not args.no_sweep:
-                line["format_sweep"] = {"workload": "M=4096, K=N=8192; b x k/b x {dynamic, static, static with independent scales} x outlier channels x{10,50}; Student-t nu=3, 1% outlier channels; rel_err = ||out - fp32(X W^T)||_F / ||fp32(X W^T)||_F",
+                line["format_sweep"] = {"workload": "M=4096, K=N=8192; b x k/b x {dynamic, static, static with independent scales, fp8/fp4 dynamic, fp8/fp4 static} x outlier channels x{10,50}; Student-t nu=3, 1% outlier channels; rel_err = ||out - fp32(X W^T)||_F / ||fp32(X W^T)||_F; fp8/fp4 rows: TFLOPS on the FP8 tensor path, same denominator",
                                         **bench_format_sweep(sq, dev, peaks)}
             line["gemm_8b_dynamic"] = {"workload": "8B-decoder-shaped linears + the single-GEMM configuration (last row), b=64, k=8, dynamic; median of 20 CUDA-event pairs (small inputs may sit in L2); fused = plain sq_gemm without a workspace",
                                        **bench_8b_dynamic(sq, dev, peaks)}
@@ -567,6 +601,8 @@ def run_cuda(args):
                               **bench_encode_only(sq, dev, peaks)}
             line["gemm_fused"] = {"workload": "70B-shaped linears, M=4096, b=128, k=16: plain sq_gemm (sparse part inside the GEMM kernel) vs the workspace call",
                                   **bench_gemm_fused(sq, layers, dev, peaks)}
+            line["weights_sq"] = {"workload": "weights in SQ-format (implicit mask, b=64, k=8) x per-token INT8 activations, 8B-decoder shapes, 1 and 4 tokens",
+                                  **bench_weights_sq(sq, dev, peaks)}
             same = bench_same_run_int8(dev)
             line["same_run"] = {"int8_gemm_TOPS": None if same is None else round(same, 1),
                                 "what": "torch._int_mm M=4096 N=K=8192 (vendor INT8 GEMM, yardstick only)",
