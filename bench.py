@@ -132,7 +132,8 @@ def physical_gpu_index(local: int) -> int:
 class Linear:
     """One linear layer of the workload: packed weights, static positions, I/O buffers."""
 
-    def __init__(self, sq, M, K, N, bank, k, static, seed, dev, dist="student_t3", independent_scales=False):
+    def __init__(self, sq, M, K, N, bank, k, static, seed, dev, dist="student_t3", independent_scales=False,
+                 fused_a8=False):
         self.M, self.K, self.N = M, K, N
         self.fmt = sq.make_format(bank, k, static, independent_scales=independent_scales)
         W = gen.weights(N, K, seed=seed, device=dev)
@@ -152,14 +153,28 @@ class Linear:
         payload = 0.5 + (1.0 if static else 2.0) * k / bank
         self.gemm_bytes = M * K * payload + N * K * (0.5 + (k / bank if static else 0.0)) + 2.0 * M * N
         self.encode_bytes = M * K * (2.0 + payload) + 9.0 * M
+        # producer fusion: sq_encode_a8 writes the product's merged 8-bit operand next to the codes
+        # (one more byte per element written by the encode, none of the expansion pass's traffic)
+        self.fused_a8 = fused_a8 and static and not independent_scales and M > 128
+        self.a8 = None
+        if self.fused_a8:
+            self.a8 = torch.empty(M, K, dtype=torch.uint8, device=dev)
+            self.encode_bytes += float(M) * K
+        self.launches = 2 if self.fused_a8 else 2 + (1 if sq.sq_gemm_workspace_bytes(self.fmt, M, N, K) else 0)
 
     def step(self, sq, events=None):
         if events is not None:
             events[0].record()
-        sq.sq_encode(self.fmt, self.X, self.pos, out=self.enc)
+        if self.fused_a8:
+            sq.sq_encode_a8(self.fmt, self.X, self.pos, out=self.enc, a8=self.a8)
+        else:
+            sq.sq_encode(self.fmt, self.X, self.pos, out=self.enc)
         if events is not None:
             events[1].record()
-        sq.sq_gemm(self.fmt, self.enc, self.w, self.pos, out=self.out)
+        if self.fused_a8:
+            sq.sq_gemm_a8(self.fmt, self.enc, self.a8, self.w, self.pos, out=self.out)
+        else:
+            sq.sq_gemm(self.fmt, self.enc, self.w, self.pos, out=self.out)
         if events is not None:
             events[2].record()
 
@@ -447,7 +462,7 @@ def run_cuda(args):
     M = args.m
     chosen = [int(x) for x in args.linears.split(",")] if args.linears else list(range(len(SHAPES_70B)))
     layers = [Linear(sq, M, SHAPES_70B[i][0], SHAPES_70B[i][1], BANK_70B, K_70B, True, seed=rank * 16 + i, dev=dev,
-                     independent_scales=args.independent_scales)
+                     independent_scales=args.independent_scales, fused_a8=not args.separate_expand)
               for i in chosen]
     total_ops = sum(l.ops for l in layers)
 
@@ -561,8 +576,8 @@ def run_cuda(args):
         "scaling": "weak", "vs_baseline": None, "dtype": "int8", "data": "synthetic",
         "config": {"workload": (WORKLOAD if not args.linears else WORKLOAD + f" [subset {args.linears}]")
                                + (" [variant: independent scales of the two parts]" if args.independent_scales else ""), "M_per_gpu": M, "bank": BANK_70B, "k": K_70B, "positions": "static",
-                   "step": "sq_encode + sq_gemm for each of the four linears",
-                   "gemm_mode": "sq_gemm with a workspace: expand_a8_kernel writes the merged 8-bit activations once (M*K bytes), gemm_kernel consumes them; the gemm_fused block times plain sq_gemm, whose sparse part runs inside the GEMM kernel",
+                   "step": ("sq_encode_a8 + sq_gemm_a8" if layers[0].fused_a8 else "sq_encode + sq_gemm") + " for each of the four linears",
+                   "gemm_mode": ("the encode kernel also writes the merged 8-bit activations (M*K bytes), gemm_kernel consumes them: two launches per linear" if layers[0].fused_a8 else "sq_gemm with a workspace: expand_a8_kernel writes the merged 8-bit activations once (M*K bytes), gemm_kernel consumes them") + "; the gemm_fused block times plain sq_gemm, whose sparse part runs inside the GEMM kernel",
                    "l2": "inputs larger than L2 (packed weights + activations + outputs of a step ~2.5 GB)",
                    "sharding": "tokens (M) per rank, weights replicated, no data-path collective"},
         "clocks": clk,
@@ -571,7 +586,7 @@ def run_cuda(args):
                 "note": "pinned host buffers; copies in, kernels and copies out on three streams (PCIe-bound)"},
         # sq_encode + sq_gemm per linear, plus the second kernel a workspace brings with it (activation
         # expansion above 128 rows, split-K finish at or below)
-        "gpu_launches": sum(2 + (1 if sq.sq_gemm_workspace_bytes(l.fmt, l.M, l.N, l.K) else 0) for l in layers) * args.steps,
+        "gpu_launches": sum(l.launches for l in layers) * args.steps,
         "roofline": {"kernel": "sq_gemm", "bound": "tensor", "achieved": gemm_tops, "peak": int8_peak,
                      "unit": "TOPS", "frac": gemm_tops / int8_peak,
                      "peak_source": f"2 x {peaks['source']} bf16 burst ({peaks['bf16_tflops']} TFLOP/s); INT8:bf16 nominal ratio 2",
@@ -579,8 +594,8 @@ def run_cuda(args):
                      "frac_of_nominal_4500": gemm_tops / 4500.0,
                      "avg_launch_ms": gemm_ms / n_gemm, "launches": n_gemm,
                      "algorithmic_bytes_per_launch": sum(l.gemm_bytes for l in layers) / len(layers),
-                     # the timed mode also writes and re-reads the 8-bit copy of the activations
-                     "bytes_per_launch_incl_8bit_copy": sum(l.gemm_bytes + 2.0 * l.M * l.K for l in layers) / len(layers),
+                     # the timed mode reads the 8-bit copy of the activations (and, without the fused encode, writes it too)
+                     "bytes_per_launch_incl_8bit_copy": sum(l.gemm_bytes + (1.0 if l.fused_a8 else 2.0) * l.M * l.K for l in layers) / len(layers),
                      "traffic": sum(l.gemm_bytes for l in layers) / len(layers)
                      * GEMM_CAPTURE_TRAFFIC_BYTES / GEMM_CAPTURE_ALGO_BYTES,
                      "traffic_note": "EXTRAPOLATED: ncu DRAM bytes of a captured M=2048 launch (whose 8-bit copy stayed in L2) scaled by algorithmic bytes; the kernel is tensor-bound, traffic < algorithmic bytes (see profiles/)"},
@@ -636,6 +651,8 @@ def main():
     ap.add_argument("--no-encode-bench", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-sweep", action="store_true", help="skip the format-parameter sweep block")
+    ap.add_argument("--separate-expand", action="store_true",
+                    help="step = sq_encode + sq_gemm with a workspace (a separate kernel expands the merged 8-bit operand) instead of sq_encode_a8 + sq_gemm_a8")
     ap.add_argument("--independent-scales", action="store_true",
                     help="run the step with the independent-scale variant of the static format (not the headline)")
     args = ap.parse_args()

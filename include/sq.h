@@ -196,9 +196,14 @@ sq_status sq_encode(const sq_format* fmt, const void* X_bf16, int64_t M, int64_t
  * out_bf16: device bf16 [M, N], written.  acc_out: device int32 [M, N] or NULL; when
  * given, the raw accumulators are written as well (used by parity tests);
  * SQ_POS_STATIC_INDEP: [2, M, N], acc_lo then acc_hi.
- * Few rows (M <= 128): K is cut into 2-8 parts that run as one thread-block cluster per tile of
- * 256 output channels and add their integer partial sums through distributed shared memory
- * (no scratch memory; the result does not depend on the number of parts). */
+ * Few rows: nothing changes in the result, only in how the work is laid out.
+ *   - M <= 16, dynamic positions, K-step selections of 16..64 entries that are a multiple of 16:
+ *     a weight-streaming kernel.  The packed weights are the 128-row tensor-core operand (every
+ *     SM streams its own slab of output channels), the tokens are the narrow one, K is cut over
+ *     a thread-block cluster whose integer partial sums meet in distributed shared memory.
+ *   - otherwise M <= 128: K is cut into 2-8 parts that run as one thread-block cluster per tile
+ *     of 256 output channels and add their partial sums the same way.
+ * Neither needs scratch memory; the result does not depend on the number of parts. */
 sq_status sq_gemm(const sq_format* fmt, const sq_encoded* A, const sq_weights* W,
                   const uint8_t* positions, int64_t M, int64_t N, int64_t K, void* out_bf16,
                   int32_t* acc_out, void* cuda_stream);
@@ -214,7 +219,8 @@ sq_status sq_gemm(const sq_format* fmt, const sq_encoded* A, const sq_weights* W
  *     ([M][K] bytes in the workspace) instead of being widened and merged again for every
  *     tile of output channels.
  * SQ_POS_STATIC_INDEP has no use for a workspace (two scales cannot share one merged operand).
- * sq_gemm_workspace_bytes: *bytes = the size this shape and format can make use of, 0 if none.
+ * sq_gemm_workspace_bytes: *bytes = the size this shape and format can make use of, 0 if none
+ * (also 0 for the shapes the weight-streaming kernel serves: it needs no scratch).
  * workspace: device memory, 16-byte aligned, or NULL (= sq_gemm); a smaller workspace than
  * asked for is used for fewer parts or not at all, never an error.  Its contents are
  * undefined afterwards; calls that share a workspace must not overlap on the GPU. */
@@ -222,6 +228,28 @@ sq_status sq_gemm_workspace_bytes(const sq_format* fmt, int64_t M, int64_t N, in
 sq_status sq_gemm_ws(const sq_format* fmt, const sq_encoded* A, const sq_weights* W,
                      const uint8_t* positions, int64_t M, int64_t N, int64_t K, void* out_bf16,
                      int32_t* acc_out, void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* Producer fusion (Section 3.3 names fusing the format conversion into the operation that
+ * produces the activations; this is the part of it that lies inside the library's boundary):
+ * sq_encode that ALSO writes the product's merged 8-bit operand, and the product that reads it.
+ *   a8: device uint8 [M, K], 16-byte aligned.  Byte for element j of a row, stored at
+ *       32*(j/32) + 16*(j%2) + (j%32)/2 (the tensor-core K order of one 32-element block:
+ *       16 even elements, then 16 odd):   j in S: vals + 128,   else: (dq4 << shift) + 128.
+ *       It is exactly what sq_gemm_ws writes into an M*K-byte workspace for the same rows.
+ *   sq_encode_a8: out as for sq_encode (bit-identical), a8 written in the same call.  Static
+ *       positions, tied scales, row lengths that are 8/12/14/16 * 256 * {1,2,4,8}: the encode
+ *       kernel writes a8 from the codes it holds in registers; any other format or shape: a
+ *       second kernel expands the codes on the same stream.  SQ_POS_STATIC_INDEP:
+ *       SQ_ERR_UNSUPPORTED (two scales share no merged operand).
+ *   sq_gemm_a8: sq_gemm (bit-identical) reading a8 instead of expanding A again; a8 is never
+ *       written.  Shapes the merged operand does not serve (M <= 128, or fewer than four tiles
+ *       of 256 output channels) run as sq_gemm and ignore a8.  A, positions: those a8 was
+ *       written with. */
+sq_status sq_encode_a8(const sq_format* fmt, const void* X_bf16, int64_t M, int64_t K,
+                       const uint8_t* positions, sq_encoded* out, void* a8, void* cuda_stream);
+sq_status sq_gemm_a8(const sq_format* fmt, const sq_encoded* A, const sq_weights* W,
+                     const uint8_t* positions, int64_t M, int64_t N, int64_t K, void* out_bf16,
+                     int32_t* acc_out, const void* a8, void* cuda_stream);
 
 /* (No counterpart in the paper: a convenience of this library.)
  * sq_gemm_ws for callers that have nowhere to get a workspace from.  Some hosts of this

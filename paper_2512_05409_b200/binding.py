@@ -69,6 +69,8 @@ def _load() -> ctypes.CDLL:
     lib.sq_gemm.argtypes = [P(sq_format), P(sq_encoded), P(sq_weights), VP, I64, I64, I64, VP, VP, VP]
     lib.sq_gemm_ws.argtypes = [P(sq_format), P(sq_encoded), P(sq_weights), VP, I64, I64, I64, VP, VP, VP,
                                ctypes.c_size_t, VP]
+    lib.sq_encode_a8.argtypes = [P(sq_format), VP, I64, I64, VP, P(sq_encoded), VP, VP]
+    lib.sq_gemm_a8.argtypes = [P(sq_format), P(sq_encoded), P(sq_weights), VP, I64, I64, I64, VP, VP, VP, VP]
     lib.sq_gemm_workspace_bytes.argtypes = [P(sq_format), I64, I64, I64, P(ctypes.c_size_t)]
     lib.sq_gemm_static_scratch.argtypes = [P(sq_format), P(sq_encoded), P(sq_weights), VP, I64, I64, I64, VP, VP, VP]
     lib.sq_decode.argtypes = [P(sq_format), P(sq_encoded), VP, I64, I64, VP, VP]
@@ -84,7 +86,7 @@ def _load() -> ctypes.CDLL:
     for name in ("sq_encoded_sizes", "sq_weights_sizes", "sq_calib_positions", "sq_pack_weights",
                  "sq_encode", "sq_gemm", "sq_gemm_ws", "sq_gemm_workspace_bytes", "sq_gemm_static_scratch", "sq_decode",
                  "sq_device_status", "sq_device_status_word", "sq_fp_pack_weights", "sq_fp_encode", "sq_fp_gemm",
-                 "sq_fp_decode", "sq_w_encode", "sq_w_act_quant", "sq_w_gemm"):
+                 "sq_fp_decode", "sq_w_encode", "sq_w_act_quant", "sq_w_gemm", "sq_encode_a8", "sq_gemm_a8"):
         getattr(lib, name).restype = ctypes.c_int
     return lib
 
@@ -243,6 +245,33 @@ def sq_encode(fmt: sq_format, X: torch.Tensor, positions: torch.Tensor | None = 
     cs = out.c_struct()
     _check(_lib.sq_encode(ctypes.byref(fmt), _ptr(X), M, K, _ptr(positions), ctypes.byref(cs),
                           _stream(stream)), "sq_encode")
+    return out
+
+
+def sq_encode_a8(fmt: sq_format, X: torch.Tensor, positions: torch.Tensor | None = None,
+                 out: Encoded | None = None, a8: torch.Tensor | None = None, stream=None):
+    """sq_encode that also writes the product's merged 8-bit operand; returns (Encoded, a8 uint8 [M, K])."""
+    M, K = _bf16_2d(X, "X")
+    if out is None:
+        out = alloc_encoded(fmt, M, K, X.device)
+    if a8 is None:
+        a8 = _buf(M * K, torch.uint8, X.device)[: M * K].view(M, K)
+    cs = out.c_struct()
+    _check(_lib.sq_encode_a8(ctypes.byref(fmt), _ptr(X), M, K, _ptr(positions), ctypes.byref(cs), _ptr(a8),
+                             _stream(stream)), "sq_encode_a8")
+    return out, a8
+
+
+def sq_gemm_a8(fmt: sq_format, A: Encoded, a8: torch.Tensor, W: Weights, positions: torch.Tensor | None = None,
+               out: torch.Tensor | None = None, acc_out: torch.Tensor | None = None, stream=None) -> torch.Tensor:
+    """sq_gemm reading the merged operand sq_encode_a8 wrote for A."""
+    M, K = A.dq4.shape[0], A.dq4.shape[1] * 2
+    N = W.wq4.shape[0]
+    if out is None:
+        out = _buf(M * N * 2, torch.bfloat16, A.dq4.device)[: M * N].view(M, N)
+    ca, cw = A.c_struct(), W.c_struct()
+    _check(_lib.sq_gemm_a8(ctypes.byref(fmt), ctypes.byref(ca), ctypes.byref(cw), _ptr(positions), M, N, K,
+                           _ptr(out), _ptr(acc_out), _ptr(a8), _stream(stream)), "sq_gemm_a8")
     return out
 
 

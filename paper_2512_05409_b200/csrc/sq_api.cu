@@ -204,6 +204,30 @@ sq_status sq_encode(const sq_format* fmt, const void* X_bf16, int64_t M, int64_t
                                  static_cast<cudaStream_t>(cuda_stream)));
 }
 
+sq_status sq_encode_a8(const sq_format* fmt, const void* X_bf16, int64_t M, int64_t K,
+                       const uint8_t* positions, sq_encoded* out, void* a8, void* cuda_stream) {
+  SQ_TRY(check_format(fmt));
+  SQ_TRY(check_k(K));
+  if (is_indep(fmt)) return SQ_ERR_UNSUPPORTED;  // two accumulators: there is no merged operand
+  if (M < 0) return SQ_ERR_INVALID_ARG;
+  if (M == 0) return SQ_OK;
+  if (X_bf16 == nullptr || a8 == nullptr) return SQ_ERR_NULL_POINTER;
+  if (!aligned16(X_bf16) || !aligned16(a8)) return SQ_ERR_ALIGNMENT;
+  SQ_TRY(check_positions(fmt, positions));
+  SQ_TRY(check_encoded(fmt, out));
+  SQ_TRY(check_device());
+  int* status = status_word();
+  if (status == nullptr) return SQ_ERR_CUDA;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  bool written = false;
+  cudaError_t err = launch_encode(fmt->bank, fmt->k, is_static(fmt), false, static_cast<const uint16_t*>(X_bf16), M, K,
+                                  positions, *out, status, st, static_cast<uint8_t*>(a8), &written);
+  if (err == cudaSuccess && !written)
+    err = launch_expand_a8(fmt->bank, fmt->k, *out, is_static(fmt) ? positions : nullptr, M, K,
+                           static_cast<uint8_t*>(a8), st);
+  return from_cuda(err);
+}
+
 sq_status sq_gemm_workspace_bytes(const sq_format* fmt, int64_t M, int64_t N, int64_t K, size_t* bytes) {
   SQ_TRY(check_format(fmt));
   SQ_TRY(check_k(K));
@@ -239,6 +263,29 @@ sq_status sq_gemm_ws(const sq_format* fmt, const sq_encoded* A, const sq_weights
   return from_cuda(launch_gemm(fmt->bank, fmt->k, is_indep(fmt), *A, *W, positions, M, N, K,
                                static_cast<uint16_t*>(out_bf16), acc_out, status, workspace,
                                workspace == nullptr ? 0 : workspace_bytes, true, static_cast<cudaStream_t>(cuda_stream)));
+}
+
+sq_status sq_gemm_a8(const sq_format* fmt, const sq_encoded* A, const sq_weights* W,
+                     const uint8_t* positions, int64_t M, int64_t N, int64_t K, void* out_bf16,
+                     int32_t* acc_out, const void* a8, void* cuda_stream) {
+  SQ_TRY(check_format(fmt));
+  SQ_TRY(check_k(K));
+  if (is_indep(fmt)) return SQ_ERR_UNSUPPORTED;
+  if (M < 0 || N < 0 || N % 8 != 0 || M > INT32_MAX || N > INT32_MAX) return SQ_ERR_INVALID_ARG;
+  if (M == 0 || N == 0) return SQ_OK;
+  SQ_TRY(check_positions(fmt, positions));
+  SQ_TRY(check_encoded(fmt, A));
+  SQ_TRY(check_weights(fmt, W));
+  if (out_bf16 == nullptr || a8 == nullptr) return SQ_ERR_NULL_POINTER;
+  if (!aligned16(out_bf16) || !aligned16(acc_out) || !aligned16(a8)) return SQ_ERR_ALIGNMENT;
+  if ((M + 127) / 128 > 65535) return SQ_ERR_UNSUPPORTED;
+  SQ_TRY(check_gemm_extent(fmt, M, N, K));
+  SQ_TRY(check_device());
+  int* status = status_word();
+  if (status == nullptr) return SQ_ERR_CUDA;
+  return from_cuda(launch_gemm(fmt->bank, fmt->k, false, *A, *W, positions, M, N, K, static_cast<uint16_t*>(out_bf16),
+                               acc_out, status, const_cast<void*>(a8), (size_t)M * (size_t)K, true,
+                               static_cast<cudaStream_t>(cuda_stream), true));
 }
 
 sq_status sq_gemm_static_scratch(const sq_format* fmt, const sq_encoded* A, const sq_weights* W,

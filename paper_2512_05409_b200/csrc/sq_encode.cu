@@ -161,13 +161,18 @@ __device__ __forceinline__ uint32_t interleave_halves(uint32_t x) { return sprea
 
 // Eight fp32 values holding integers in their low mantissa bits (magic-number rounding)
 // -> eight two's-complement nibbles, element i in nibble i.
-__device__ __forceinline__ uint32_t pack_nibbles(const float (&r)[8]) {
+// `ev` / `od` receive the codes of the even / odd elements as four two's-complement bytes each.
+__device__ __forceinline__ uint32_t pack_nibbles(const float (&r)[8], uint32_t& ev, uint32_t& od) {
   const uint32_t u0 = __float_as_uint(r[0]), u1 = __float_as_uint(r[1]), u2 = __float_as_uint(r[2]),
                  u3 = __float_as_uint(r[3]), u4 = __float_as_uint(r[4]), u5 = __float_as_uint(r[5]),
                  u6 = __float_as_uint(r[6]), u7 = __float_as_uint(r[7]);
-  const uint32_t ev = __byte_perm(__byte_perm(u0, u2, 0x0040), __byte_perm(u4, u6, 0x0040), 0x5410);
-  const uint32_t od = __byte_perm(__byte_perm(u1, u3, 0x0040), __byte_perm(u5, u7, 0x0040), 0x5410);
+  ev = __byte_perm(__byte_perm(u0, u2, 0x0040), __byte_perm(u4, u6, 0x0040), 0x5410);
+  od = __byte_perm(__byte_perm(u1, u3, 0x0040), __byte_perm(u5, u7, 0x0040), 0x5410);
   return (ev & 0x0F0F0F0Fu) | ((od << 4) & 0xF0F0F0F0u);
+}
+__device__ __forceinline__ uint32_t pack_nibbles(const float (&r)[8]) {
+  uint32_t ev, od;
+  return pack_nibbles(r, ev, od);
 }
 
 // The same packing for codes that carry an offset of 8 (u = q + 8 in 1..15, produced by adding
@@ -320,6 +325,7 @@ struct EncodeParams {
   float* s_hi;
   float* s_lo;
   uint8_t* shift;
+  uint8_t* a8;        // merged 8-bit operand [M, K] (static register kernel, tied scales), or nullptr
   int* status;
   int64_t M;
   int K, k, b;
@@ -752,6 +758,10 @@ __global__ void __launch_bounds__(B == 128 ? 256 : 512) encode_rows_kernel(const
 //   -> INT8 codes of the selected values, INT4 codes straight from the registers (selected
 //   places were cleared there while taking the maxima).
 // The kernel is bound by instruction issue, which is why the masks are tables.
+// On request (tied scales) the row's merged 8-bit operand for the product is written as well:
+// the dense codes are at hand as bytes while they are packed, so it costs two shifts, two
+// logic operations and two stores per eight elements, plus one byte store per selected place
+// -- instead of a second kernel that reads the codes back and expands them.
 template <int NCL, int NT, bool INDEP>
 __global__ void __launch_bounds__(NT, 1) encode_static_regs_kernel(const EncodeParams p) {
   extern __shared__ __align__(128) uint8_t smem_enc[];
@@ -765,13 +775,17 @@ __global__ void __launch_bounds__(NT, 1) encode_static_regs_kernel(const EncodeP
   constexpr int S8 = NCL * 32;  // 16-byte chunks per warp slice
 
   // shared memory: [magnitude masks, uint16 [K]] [selected offsets, uint16 [GK]] then per group [gathered words, uint32 [GK]] and, after all
-  // of those, 16 exchange words per group
+  // of those, 32 exchange words per group
   const size_t jt_bytes = ((size_t)GK * 2 + 15) & ~(size_t)15;
   const size_t stash_bytes = ((size_t)GK * 4 + 15) & ~(size_t)15;
   uint16_t* hmask = reinterpret_cast<uint16_t*>(smem_enc);
   uint16_t* jt = hmask + K;
   uint32_t* stash = reinterpret_cast<uint32_t*>(reinterpret_cast<uint8_t*>(jt) + jt_bytes + stash_bytes * grp);
-  uint32_t* exch = reinterpret_cast<uint32_t*>(reinterpret_cast<uint8_t*>(jt) + jt_bytes + stash_bytes * ngroups) + grp * 16;
+  uint32_t* exch = reinterpret_cast<uint32_t*>(reinterpret_cast<uint8_t*>(jt) + jt_bytes + stash_bytes * ngroups) + grp * 32;
+  // with the merged operand asked for: the row's INT8 codes once more, per group, after the exchange words
+  const size_t sp8_bytes = ((size_t)GK + 15) & ~(size_t)15;
+  uint8_t* sp8 = reinterpret_cast<uint8_t*>(jt) + jt_bytes + (stash_bytes + 128) * ngroups + sp8_bytes * grp;
+  const bool want_a8 = !INDEP && p.a8 != nullptr;
   const uint32_t stash_s = smem_u32(stash);
 
   for (int i = threadIdx.x; i < K / 2; i += NT) reinterpret_cast<uint32_t*>(hmask)[i] = 0x7FFF7FFFu;
@@ -830,13 +844,13 @@ __global__ void __launch_bounds__(NT, 1) encode_static_regs_kernel(const EncodeP
     if (rw > 1) {
       if (lane == 0) {
         exch[slice] = amax_bits;
-        exch[8 + slice] = rmax_bits;
+        exch[16 + slice] = rmax_bits;
       }
       group_sync(rw, grp);  // also: every gathered word of the row is in the stash
       amax_bits = rmax_bits = 0;
       for (int w = 0; w < rw; ++w) {
         amax_bits = max(amax_bits, exch[w]);
-        rmax_bits = max(rmax_bits, exch[8 + w]);
+        rmax_bits = max(rmax_bits, exch[16 + w]);
       }
     } else {
       __syncwarp();
@@ -864,11 +878,14 @@ __global__ void __launch_bounds__(NT, 1) encode_static_regs_kernel(const EncodeP
             o |= (__float_as_uint(__fmaf_rn(__uint_as_float(a), rs.inv, kMagic)) & 0xFFu) << (8 * q);
           }
           *reinterpret_cast<uint32_t*>(vdst + t4) = o;
+          if (want_a8) *reinterpret_cast<uint32_t*>(sp8 + t4) = o;
         }
       } else {
         for (int t = glane; t < GK; t += gsize) {
           const uint32_t a = (jt[t] & 1u) ? (stash[t] & 0xFFFF0000u) : (stash[t] << 16);
-          vdst[t] = (int8_t)(__float_as_uint(__fmaf_rn(__uint_as_float(a), rs.inv, kMagic)) & 0xFFu);
+          const uint32_t o = __float_as_uint(__fmaf_rn(__uint_as_float(a), rs.inv, kMagic)) & 0xFFu;
+          vdst[t] = (int8_t)o;
+          if (want_a8) sp8[t] = (uint8_t)o;
         }
       }
     }
@@ -889,6 +906,33 @@ __global__ void __launch_bounds__(NT, 1) encode_static_regs_kernel(const EncodeP
         v[c].z = max2(min2(v[c].z, hi2), lo2);
         v[c].w = max2(min2(v[c].w, hi2), lo2);
       }
+    }
+    if (want_a8) {
+      // The merged operand of the same row, in the product's K order ([16 even | 16 odd] bytes per
+      // 32 elements): byte = code * 2^e + 128.  The codes are already at hand as bytes; the
+      // selected places hold code 0 here and receive their INT8 code (+128) below.
+      uint32_t* arow = reinterpret_cast<uint32_t*>(p.a8 + (size_t)m * K);
+      const uint32_t e = (uint32_t)rs.e;
+      const uint32_t keep = 0x01010101u * ((0xFFu << e) & 0xFFu);
+#pragma unroll
+      for (int c = 0; c < NCL; ++c) {
+        float r[8];
+        uint32_t ev, od;
+        quant8(v[c], cq, r);
+        dst[c * 32] = pack_nibbles(r, ev, od);
+        const int wi = slice * S8 + c * 32 + lane;  // this chunk: elements 8 * wi .. 8 * wi + 7
+        uint32_t* aw = arow + (wi >> 2) * 8 + (wi & 3);
+        aw[0] = ((ev << e) & keep) ^ 0x80808080u;
+        aw[4] = ((od << e) & keep) ^ 0x80808080u;
+      }
+      group_sync(rw, grp);  // the stores above are ordered before the byte stores below
+      uint8_t* brow = p.a8 + (size_t)m * K;
+      for (int t = glane; t < GK; t += gsize) {
+        const uint32_t j = jt[t];
+        brow[(j & ~31u) | ((j & 1u) << 4) | ((j & 31u) >> 1)] = sp8[t] ^ 0x80u;
+      }
+      // (sp8 and the stash are next written after the group's barrier in the middle of the next row)
+      continue;
     }
 #pragma unroll
     for (int c = 0; c < NCL; ++c) {
@@ -1150,7 +1194,8 @@ cudaError_t launch_static_regs_as(EncodeParams p, int rw, cudaStream_t st) {
   const int ngroups = (NT / 32) / rw;
   const size_t jt_bytes = ((size_t)GK * 2 + 15) & ~(size_t)15;
   const size_t stash_bytes = ((size_t)GK * 4 + 15) & ~(size_t)15;
-  const size_t smem = (size_t)p.K * 2 + jt_bytes + (stash_bytes + 64) * ngroups;
+  const size_t sp8_bytes = p.a8 != nullptr ? (((size_t)GK + 15) & ~(size_t)15) : 0;
+  const size_t smem = (size_t)p.K * 2 + jt_bytes + (stash_bytes + 128 + sp8_bytes) * ngroups;
   if (smem > 200 * 1024) return cudaErrorNotSupported;
   p.rw = rw;
   int dev = 0, sms = 0;
@@ -1197,8 +1242,11 @@ cudaError_t launch_generic(int k, bool is_static, bool indep, const uint16_t* X,
 }  // namespace
 
 cudaError_t launch_encode(int b, int k, bool is_static, bool indep, const uint16_t* X, int64_t M, int64_t K,
-                          const uint8_t* positions, const sq_encoded& out, int* status, cudaStream_t st) {
+                          const uint8_t* positions, const sq_encoded& out, int* status, cudaStream_t st,
+                          uint8_t* a8, bool* a8_written) {
   EncodeParams p;
+  if (a8_written != nullptr) *a8_written = false;
+  p.a8 = nullptr;
   p.X = X;
   p.positions = positions;
   p.dq4 = out.dq4;
@@ -1225,8 +1273,11 @@ cudaError_t launch_encode(int b, int k, bool is_static, bool indep, const uint16
     return launch_generic<128>(k, true, true, X, M, K, positions, out, st);
   }
   if (is_static) {
+    p.a8 = a8;  // only the register kernel writes the merged operand
     cudaError_t err = launch_static_regs<false>(p, st);
+    if (err == cudaSuccess && a8 != nullptr && a8_written != nullptr) *a8_written = true;
     if (err != cudaErrorNotSupported) return err;
+    p.a8 = nullptr;
     err = b == 32 ? launch_rows<32, 0>(p, st) : (b == 64 ? launch_rows<64, 0>(p, st) : launch_rows<128, 0>(p, st));
     if (err != cudaErrorNotSupported) return err;
     // a row, its offset table and its stash together exceed shared memory: one block per row

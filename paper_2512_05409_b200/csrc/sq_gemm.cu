@@ -1220,10 +1220,25 @@ size_t gemm_workspace_bytes(int b, int k, bool is_static, bool indep, int64_t M,
   return sp > 1 ? (size_t)sp * M * N * 4 : 0;
 }
 
+cudaError_t launch_expand_a8(int b, int k, const sq_encoded& A, const uint8_t* positions, int64_t M, int64_t K,
+                             uint8_t* a8, cudaStream_t st) {
+  int dev = 0, sms = 0;
+  cudaError_t err = cudaGetDevice(&dev);
+  if (err != cudaSuccess) return err;
+  err = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  if (err != cudaSuccess) return err;
+  const int64_t units = M * (K / 32);
+  int64_t blocks = (units + 255) / 256;
+  if (blocks > 32 * (int64_t)sms) blocks = 32 * (int64_t)sms;
+  expand_a8_kernel<<<(unsigned)blocks, 256, 0, st>>>(A.dq4, A.vals, positions == nullptr ? A.idx : nullptr, positions,
+                                                    A.shift, M, (int)K, b, k, a8);
+  return cudaGetLastError();
+}
+
 cudaError_t launch_gemm(int b, int k, bool indep, const sq_encoded& A, const sq_weights& W,
                         const uint8_t* positions, int64_t M, int64_t N, int64_t K, uint16_t* out,
                         int32_t* acc_out, int* status, void* workspace, size_t workspace_bytes, bool allow_stream,
-                        cudaStream_t st) {
+                        cudaStream_t st, bool a8_ready) {
   if (allow_stream && !indep && gemm_stream_serves(b, k, positions != nullptr, M, K))
     return launch_gemm_stream(b, k, A, W, positions, M, N, K, out, acc_out, status, st);
   GemmParams p;
@@ -1279,6 +1294,10 @@ cudaError_t launch_gemm(int b, int k, bool indep, const sq_encoded& A, const sq_
   if (indep && !stma) return cudaErrorNotSupported;
   if (indep) workspace = nullptr;
   const bool a8 = workspace != nullptr && use_a8(positions != nullptr, M, N, K, workspace_bytes);
+  if (a8_ready && !a8) {  // the caller's merged operand is of no use to this shape: leave it untouched
+    workspace = nullptr;
+    workspace_bytes = 0;
+  }
   const int mode = indep ? kModeIndep : a8 ? kModeA8 : (stma ? kModeTma : (pmerge ? kModeMergeProd : kModeMergeEpi));
   // One CTA per tile for at most 128 rows (a second CTA would have no rows); CTA pairs otherwise.
   const int pair = M > BM ? 2 : 1;
@@ -1446,13 +1465,13 @@ cudaError_t launch_gemm(int b, int k, bool indep, const sq_encoded& A, const sq_
   }
 
   if (a8) {
-    // the merged 8-bit activations: written once by expand_a8_kernel, read by TMA as [M, K] bytes
+    // the merged 8-bit activations: written once (by expand_a8_kernel here, or by the caller's
+    // encode already), read by TMA as [M, K] bytes
     uint8_t* a8buf = static_cast<uint8_t*>(workspace);
-    const int64_t units = M * (K / 32);
-    int64_t blocks = (units + 255) / 256;
-    if (blocks > 32 * (int64_t)sms) blocks = 32 * (int64_t)sms;
-    expand_a8_kernel<<<(unsigned)blocks, 256, 0, st>>>(A.dq4, A.vals, positions == nullptr ? A.idx : nullptr, positions,
-                                                      A.shift, M, (int)K, b, k, a8buf);
+    if (!a8_ready) {
+      err = launch_expand_a8(b, k, A, positions, M, K, a8buf, st);
+      if (err != cudaSuccess) return err;
+    }
     const cuuint64_t pitch[1] = {(cuuint64_t)K};
     const cuuint64_t dim_a[2] = {(cuuint64_t)K, (cuuint64_t)M};
     const cuuint32_t box_a[2] = {BK, 2 * BM};

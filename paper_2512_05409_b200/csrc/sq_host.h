@@ -31,7 +31,10 @@ cudaError_t launch_pack_weights(int b, int k, const uint16_t* W, int64_t N, int6
                                 const uint8_t* positions, const sq_weights& out, cudaStream_t st);
 
 cudaError_t launch_encode(int b, int k, bool is_static, bool indep, const uint16_t* X, int64_t M, int64_t K,
-                          const uint8_t* positions, const sq_encoded& out, int* status, cudaStream_t st);
+                          const uint8_t* positions, const sq_encoded& out, int* status, cudaStream_t st,
+                          uint8_t* a8 = nullptr, bool* a8_written = nullptr);
+// a8 != nullptr asks for the product's merged 8-bit operand [M, K] as well; *a8_written tells whether
+// the encode kernel wrote it (static positions, tied scales, row lengths the register kernel takes).
 
 cudaError_t launch_decode(int b, int k, const sq_encoded& A, const uint8_t* positions, int64_t M,
                           int64_t K, uint16_t* out, cudaStream_t st);
@@ -40,7 +43,11 @@ cudaError_t launch_decode(int b, int k, const sq_encoded& A, const uint8_t* posi
 cudaError_t launch_gemm(int b, int k, bool indep, const sq_encoded& A, const sq_weights& W,
                         const uint8_t* positions, int64_t M, int64_t N, int64_t K, uint16_t* out,
                         int32_t* acc_out, int* status, void* workspace, size_t workspace_bytes, bool allow_stream,
-                        cudaStream_t st);
+                        cudaStream_t st, bool a8_ready = false);
+// a8_ready: `workspace` already holds the merged 8-bit operand of A (M*K bytes): it is read, never written.
+// The merged operand alone: what launch_gemm writes into an M*K-byte workspace before its product.
+cudaError_t launch_expand_a8(int b, int k, const sq_encoded& A, const uint8_t* positions, int64_t M, int64_t K,
+                             uint8_t* a8, cudaStream_t st);
 // Bytes of workspace launch_gemm can make use of for this shape and format (0: none).
 size_t gemm_workspace_bytes(int b, int k, bool is_static, bool indep, int64_t M, int64_t N, int64_t K);
 // The weight-streaming kernel for at most 32 token rows (sq_gemm_stream.cu).

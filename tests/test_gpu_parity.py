@@ -527,3 +527,74 @@ def test_few_rows_without_workspace(static, M, N, K):
     assert np.array_equal(_np(acc), acc_ref)
     assert_bf16_close(out, ref32)
     assert np.array_equal(_bits(out), out_ref) and torch.equal(out, again)
+
+
+# ----------------------------------------------------------------------------- producer fusion (Section 3.3)
+
+def merged_operand_from_oracle(b, k, enc_ref, pos_ref):
+    """The product's merged 8-bit operand written out from the oracle's encoding: byte = code * 2^e + 128
+    for a dense element, INT8 code + 128 for a selected one, stored in the tensor-core K order of one
+    32-element block (16 even elements, then 16 odd)."""
+    by = enc_ref.dq4.astype(np.int32)                              # element 2i in the low nibble, 2i+1 in the high one
+    M, K = by.shape[0], by.shape[1] * 2
+    dq = np.empty((M, K), dtype=np.int32)
+    dq[:, 0::2] = ((by & 15) ^ 8) - 8
+    dq[:, 1::2] = ((by >> 4) ^ 8) - 8
+    merged = dq << enc_ref.shift.astype(np.int32)[:, None]
+    G = K // b
+    idx = enc_ref.idx if enc_ref.idx is not None else np.broadcast_to(pos_ref.reshape(1, G, k), (M, G, k))
+    cols = (np.arange(G)[None, :, None] * b + idx.astype(np.int64)).reshape(M, G * k)
+    np.put_along_axis(merged, cols, enc_ref.vals.reshape(M, G * k).astype(np.int32), axis=1)
+    j = np.arange(K)
+    where = 32 * (j // 32) + 16 * (j % 2) + (j % 32) // 2
+    out = np.empty((M, K), dtype=np.uint8)
+    out[:, where] = (merged + 128).astype(np.uint8)
+    return out
+
+
+@pytest.mark.parametrize("M,N,K,b,k,static", [
+    (300, 1024, 2048, 64, 8, True),      # register kernel, one warp per row
+    (257, 1280, 8192, 64, 8, True),      # register kernel, rows split over warps
+    (200, 1024, 4096, 128, 16, True),
+    (130, 1024, 3072, 32, 4, True),
+    (140, 1024, 2048, 64, 6, True),      # k not a multiple of four: byte-wise sparse path
+    (150, 1024, 1024, 64, 8, True),      # row length the register kernel does not take: second kernel
+    (200, 1024, 2048, 64, 8, False),     # dynamic positions: second kernel
+    (40, 512, 2048, 64, 8, True),        # few rows: the product ignores the merged operand
+])
+def test_encode_with_merged_operand(M, N, K, b, k, static):
+    dev = "cuda"
+    fmt = sq.make_format(b, k, static)
+    X = gen.activations(M, K, seed=5, device=dev)
+    W = gen.weights(N, K, seed=5, device=dev)
+    pos = pos_ref = None
+    if static:
+        calib = gen.calibration_batch(64, K, seed=5, device=dev)
+        pos = sq.sq_calib_positions(fmt, calib, W)
+        pos_ref = _np(pos)
+    enc_ref = oracle.encode(b, k, _bits(X), pos_ref)
+    a8 = torch.full((M, K), 0x5A, dtype=torch.uint8, device=dev)
+    enc_gpu, a8 = sq.sq_encode_a8(fmt, X, pos, a8=a8)
+    check_status()
+    compare_encoded(enc_gpu, enc_ref)
+    assert np.array_equal(_np(a8), merged_operand_from_oracle(b, k, enc_ref, pos_ref))
+
+    w_gpu = sq.sq_pack_weights(fmt, W, pos)
+    w_ref = oracle.pack_weights(b, k, _bits(W), pos_ref)
+    keep = a8.clone()
+    acc_gpu = torch.full((M, N), -7, dtype=torch.int32, device=dev)
+    out_gpu = sq.sq_gemm_a8(fmt, enc_gpu, a8, w_gpu, pos, acc_out=acc_gpu)
+    check_status()
+    assert torch.equal(a8, keep)                       # read, never written
+    acc_ref, ref32, out_ref = oracle.gemm(b, k, enc_ref, w_ref, pos_ref)
+    assert np.array_equal(_np(acc_gpu), acc_ref)
+    assert np.array_equal(_bits(out_gpu), out_ref)
+    assert torch.equal(sq.sq_gemm(fmt, enc_gpu, w_gpu, pos), out_gpu)
+
+
+def test_merged_operand_rejects_independent_scales():
+    fmt = sq.make_format(64, 8, True, independent_scales=True)
+    X = gen.activations(8, 1024, seed=1, device="cuda")
+    pos = torch.arange(8, dtype=torch.uint8, device="cuda").repeat(1024 // 64)
+    with pytest.raises(sq.SqError):
+        sq.sq_encode_a8(fmt, X, pos)
