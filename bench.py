@@ -442,6 +442,65 @@ def run_reference(args):
     print(json.dumps(line))
 
 
+PROFILE_CASES = ("encode_dynamic", "encode_static", "encode_static_a8", "gemm_a8", "gemm_stream", "fp_gemm", "wsq_gemm")
+
+
+def run_profile_case(args):
+    """A handful of launches of one kernel on a small case, and nothing else: the command a profiler
+    capture is taken of (inputs larger than L2 where the kernel streams from memory, well under
+    1 GB on the device).  Prints one line naming the case; it is not a benchmark."""
+    import paper_2512_05409_b200 as sq
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(0)
+    case, n = args.profile_case, 6
+    if case.startswith("encode"):
+        M = K = 8192
+        static = case != "encode_dynamic"
+        fmt = sq.make_format(64, 8, static)
+        Xs = [gen.activations(M, K, seed=s, outlier_fraction=0.005, outlier_scale=50.0, device=dev) for s in range(3)]
+        pos = None
+        if static:
+            calib = gen.calibration_batch(512, K, seed=0, outlier_fraction=0.005, outlier_scale=50.0, device=dev)
+            pos = sq.sq_calib_positions(fmt, calib, None)
+        enc = sq.alloc_encoded(fmt, M, K, dev)
+        a8 = torch.empty(M, K, dtype=torch.uint8, device=dev) if case == "encode_static_a8" else None
+        for i in range(n):
+            if a8 is not None:
+                sq.sq_encode_a8(fmt, Xs[i % 3], pos, out=enc, a8=a8)
+            else:
+                sq.sq_encode(fmt, Xs[i % 3], pos, out=enc)
+    elif case == "gemm_a8":
+        l = Linear(sq, 2048, 8192, 8192, BANK_70B, K_70B, True, seed=1, dev=dev, fused_a8=True)
+        for _ in range(n):
+            l.step(sq)
+    elif case == "gemm_stream":
+        K, N = SHAPES_8B[2]
+        l = Linear(sq, 16, K, N, 64, 8, False, seed=2, dev=dev)
+        for _ in range(n):
+            l.step(sq)
+    elif case == "fp_gemm":
+        M, K, N = 2048, 8192, 8192
+        fmt = sq.make_format(64, 8, False)
+        W = gen.weights(N, K, seed=3, device=dev)
+        w = sq.sq_fp_pack_weights(W)
+        enc, a8 = sq.sq_fp_encode(fmt, gen.activations(M, K, seed=3, device=dev))
+        out = torch.empty(M, N, dtype=torch.bfloat16, device=dev)
+        for _ in range(n):
+            sq.sq_fp_gemm(enc, a8, w, out=out)
+    elif case == "wsq_gemm":
+        K, N = SHAPES_8B[2]
+        fmt = sq.make_format(64, 8, True)
+        W = gen.weights(N, K, seed=4, device=dev)
+        enc = sq.sq_w_encode(fmt, W, (W.float() ** 2).contiguous())
+        xq, s_x = sq.sq_w_act_quant(gen.activations(4, K, seed=4, device=dev))
+        out = torch.empty(4, N, dtype=torch.bfloat16, device=dev)
+        for _ in range(n):
+            sq.sq_w_gemm(fmt, xq, s_x, enc, out=out)
+    torch.cuda.synchronize()
+    assert sq.sq_device_status() == sq.SQ_OK
+    print(json.dumps({"profile_case": case, "launches": n}))
+
+
 def run_cuda(args):
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -655,8 +714,12 @@ def main():
                     help="step = sq_encode + sq_gemm with a workspace (a separate kernel expands the merged 8-bit operand) instead of sq_encode_a8 + sq_gemm_a8")
     ap.add_argument("--independent-scales", action="store_true",
                     help="run the step with the independent-scale variant of the static format (not the headline)")
+    ap.add_argument("--profile-case", choices=PROFILE_CASES, default=None,
+                    help="run a few launches of one kernel on a small case and exit (the command profiler captures are taken of)")
     args = ap.parse_args()
-    if args.impl == "reference":
+    if args.profile_case:
+        run_profile_case(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_cuda(args)

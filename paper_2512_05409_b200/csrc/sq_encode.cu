@@ -782,9 +782,11 @@ __global__ void __launch_bounds__(NT, 1) encode_static_regs_kernel(const EncodeP
   uint16_t* jt = hmask + K;
   uint32_t* stash = reinterpret_cast<uint32_t*>(reinterpret_cast<uint8_t*>(jt) + jt_bytes + stash_bytes * grp);
   uint32_t* exch = reinterpret_cast<uint32_t*>(reinterpret_cast<uint8_t*>(jt) + jt_bytes + stash_bytes * ngroups) + grp * 32;
-  // with the merged operand asked for: the row's INT8 codes once more, per group, after the exchange words
-  const size_t sp8_bytes = ((size_t)GK + 15) & ~(size_t)15;
-  uint8_t* sp8 = reinterpret_cast<uint8_t*>(jt) + jt_bytes + (stash_bytes + 128) * ngroups + sp8_bytes * grp;
+  // With the merged operand asked for: per group an image of a row's selected places in the order
+  // the dense loop walks (chunk by chunk, [4 even | 4 odd] bytes): INT8 code ^ 0x80 there, 0x80
+  // everywhere else (written once); and, once per block, where in the image each place lies.
+  uint8_t* img = reinterpret_cast<uint8_t*>(jt) + jt_bytes + (stash_bytes + 128) * ngroups + (size_t)K * grp;
+  uint16_t* jimg = reinterpret_cast<uint16_t*>(reinterpret_cast<uint8_t*>(jt) + jt_bytes + (stash_bytes + 128 + (size_t)K) * ngroups);
   const bool want_a8 = !INDEP && p.a8 != nullptr;
   const uint32_t stash_s = smem_u32(stash);
 
@@ -794,7 +796,11 @@ __global__ void __launch_bounds__(NT, 1) encode_static_regs_kernel(const EncodeP
     const int j = (t / k) * p.b + p.positions[t];
     jt[t] = (uint16_t)j;
     hmask[j] = 0;
+    if (want_a8) jimg[t] = (uint16_t)((j & ~7) | ((j & 1) << 2) | ((j & 7) >> 1));
   }
+  if (want_a8)
+    for (int i = threadIdx.x; i < (K / 4) * ngroups; i += NT)
+      reinterpret_cast<uint32_t*>(reinterpret_cast<uint8_t*>(jt) + jt_bytes + (stash_bytes + 128) * ngroups)[i] = 0x80808080u;
   __syncthreads();
 
   const int64_t gw = (int64_t)blockIdx.x * ngroups + grp;
@@ -878,14 +884,21 @@ __global__ void __launch_bounds__(NT, 1) encode_static_regs_kernel(const EncodeP
             o |= (__float_as_uint(__fmaf_rn(__uint_as_float(a), rs.inv, kMagic)) & 0xFFu) << (8 * q);
           }
           *reinterpret_cast<uint32_t*>(vdst + t4) = o;
-          if (want_a8) *reinterpret_cast<uint32_t*>(sp8 + t4) = o;
+          if (want_a8) {
+            const uint2 ji = *reinterpret_cast<const uint2*>(jimg + t4);
+            const uint32_t ox = o ^ 0x80808080u;
+            img[ji.x & 0xFFFFu] = (uint8_t)ox;
+            img[ji.x >> 16] = (uint8_t)(ox >> 8);
+            img[ji.y & 0xFFFFu] = (uint8_t)(ox >> 16);
+            img[ji.y >> 16] = (uint8_t)(ox >> 24);
+          }
         }
       } else {
         for (int t = glane; t < GK; t += gsize) {
           const uint32_t a = (jt[t] & 1u) ? (stash[t] & 0xFFFF0000u) : (stash[t] << 16);
           const uint32_t o = __float_as_uint(__fmaf_rn(__uint_as_float(a), rs.inv, kMagic)) & 0xFFu;
           vdst[t] = (int8_t)o;
-          if (want_a8) sp8[t] = (uint8_t)o;
+          if (want_a8) img[jimg[t]] = (uint8_t)(o ^ 0x80u);
         }
       }
     }
@@ -909,29 +922,26 @@ __global__ void __launch_bounds__(NT, 1) encode_static_regs_kernel(const EncodeP
     }
     if (want_a8) {
       // The merged operand of the same row, in the product's K order ([16 even | 16 odd] bytes per
-      // 32 elements): byte = code * 2^e + 128.  The codes are already at hand as bytes; the
-      // selected places hold code 0 here and receive their INT8 code (+128) below.
-      uint32_t* arow = reinterpret_cast<uint32_t*>(p.a8 + (size_t)m * K);
+      // 32 elements): byte = code * 2^e + 128 for a dense element -- the codes are at hand as bytes
+      // -- and INT8 code + 128 at a selected place, where the dense code is 0 and the image has it.
+      // chunk c of this lane: elements 8 * wi .. 8 * wi + 7 with wi = slice * S8 + c * 32 + lane, i.e.
+      // block wi / 4 = (slice * S8 + lane) / 4 + 8 * c, quarter lane % 4
+      uint32_t* aw = reinterpret_cast<uint32_t*>(p.a8 + (size_t)m * K) + ((slice * S8 + lane) >> 2) * 8 + (lane & 3);
+      const uint2* iw = reinterpret_cast<const uint2*>(img) + slice * S8 + lane;
       const uint32_t e = (uint32_t)rs.e;
       const uint32_t keep = 0x01010101u * ((0xFFu << e) & 0xFFu);
+      group_sync(rw, grp);  // the image holds this row's codes
 #pragma unroll
       for (int c = 0; c < NCL; ++c) {
         float r[8];
         uint32_t ev, od;
         quant8(v[c], cq, r);
         dst[c * 32] = pack_nibbles(r, ev, od);
-        const int wi = slice * S8 + c * 32 + lane;  // this chunk: elements 8 * wi .. 8 * wi + 7
-        uint32_t* aw = arow + (wi >> 2) * 8 + (wi & 3);
-        aw[0] = ((ev << e) & keep) ^ 0x80808080u;
-        aw[4] = ((od << e) & keep) ^ 0x80808080u;
+        const uint2 im = iw[c * 32];
+        aw[c * 64] = ((ev << e) & keep) ^ im.x;
+        aw[c * 64 + 4] = ((od << e) & keep) ^ im.y;
       }
-      group_sync(rw, grp);  // the stores above are ordered before the byte stores below
-      uint8_t* brow = p.a8 + (size_t)m * K;
-      for (int t = glane; t < GK; t += gsize) {
-        const uint32_t j = jt[t];
-        brow[(j & ~31u) | ((j & 1u) << 4) | ((j & 31u) >> 1)] = sp8[t] ^ 0x80u;
-      }
-      // (sp8 and the stash are next written after the group's barrier in the middle of the next row)
+      group_sync(rw, grp);  // the stash, the image and the exchange words are reused by the next row
       continue;
     }
 #pragma unroll
@@ -1194,8 +1204,8 @@ cudaError_t launch_static_regs_as(EncodeParams p, int rw, cudaStream_t st) {
   const int ngroups = (NT / 32) / rw;
   const size_t jt_bytes = ((size_t)GK * 2 + 15) & ~(size_t)15;
   const size_t stash_bytes = ((size_t)GK * 4 + 15) & ~(size_t)15;
-  const size_t sp8_bytes = p.a8 != nullptr ? (((size_t)GK + 15) & ~(size_t)15) : 0;
-  const size_t smem = (size_t)p.K * 2 + jt_bytes + (stash_bytes + 128 + sp8_bytes) * ngroups;
+  const size_t img_bytes = p.a8 != nullptr ? (size_t)p.K : 0;  // per group: the image of the selected places
+  const size_t smem = (size_t)p.K * 2 + jt_bytes + (stash_bytes + 128 + img_bytes) * ngroups + (p.a8 != nullptr ? jt_bytes : 0);
   if (smem > 200 * 1024) return cudaErrorNotSupported;
   p.rw = rw;
   int dev = 0, sms = 0;
