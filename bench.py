@@ -44,11 +44,11 @@ FALLBACK_HBM_GBS, FALLBACK_BF16_TFLOPS = 6650.0, 1590.0
 # algorithmic bytes; the benchmark's launches are too large to capture with --set full, so their
 # traffic is this ratio times their own algorithmic bytes (the traffic is operand streaming and
 # grows with the operands).  It is below 1 because most of the output is still in L2 at kernel end.
-GEMM_CAPTURE_TRAFFIC_BYTES = 50.58e6 + 4.76e6
+GEMM_CAPTURE_TRAFFIC_BYTES = 50.89e6 + 4.22e6
 GEMM_CAPTURE_ALGO_BYTES = 2048 * 8192 * 0.625 + 8192 * 8192 * 0.625 + 2.0 * 2048 * 8192
 # ncu DRAM traffic of one encode launch of the 8192 x 8192 bandwidth test (dynamic k=8 / static k=8),
 # profiles/encode_kernels_b64_k8_8192x8192.txt
-ENCODE_TRAFFIC_BYTES_PER_LAUNCH = {"dynamic": 134.26e6 + 25.37e6, "static": 134.26e6 + 21.93e6}
+ENCODE_TRAFFIC_BYTES_PER_LAUNCH = {"dynamic": 134.29e6 + 25.98e6, "static": 134.77e6 + 23.95e6}
 
 
 def load_peaks():
