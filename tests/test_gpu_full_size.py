@@ -11,7 +11,7 @@ import torch
 import gen
 import oracle
 import paper_2512_05409_b200 as sq
-from test_gpu_parity import assert_bf16_close, check_status, _np, _bits
+from test_gpu_parity import assert_bf16_close, check_status, merged_operand_from_oracle, _np, _bits
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda"
@@ -74,7 +74,24 @@ def check_linear(lin: PackedLinear, X: torch.Tensor, seed: int, n_rows=24):
     plain = sq.sq_gemm(lin.fmt, enc, lin.w, lin.pos, use_workspace=False)
     check_status()
     assert torch.equal(plain, out)
-    del acc, out, enc, plain
+    del plain
+    # the pair bench.py's step calls: the encode that also writes the product's merged 8-bit operand,
+    # and the product that reads it
+    enc2, a8 = sq.sq_encode_a8(lin.fmt, X, lin.pos)
+    check_status()
+    for got, want in ((enc2.dq4, enc.dq4), (enc2.vals, enc.vals), (enc2.shift, enc.shift)):
+        assert torch.equal(got, want)
+    assert torch.equal(enc2.s_hi.view(torch.int32), enc.s_hi.view(torch.int32))
+    assert torch.equal(enc2.s_lo.view(torch.int32), enc.s_lo.view(torch.int32))
+    if not lin.static:
+        assert torch.equal(enc2.idx, enc.idx)
+    assert np.array_equal(_np(a8[rows_t]), merged_operand_from_oracle(lin.b, lin.k, enc_ref, lin.pos_ref))
+    acc2 = torch.empty(M, lin.N, dtype=torch.int32, device=DEV)
+    out2 = sq.sq_gemm_a8(lin.fmt, enc2, a8, lin.w, lin.pos, acc_out=acc2)
+    check_status()
+    assert np.array_equal(_np(acc2[rows_t][:, cols_t]), acc_ref)
+    assert torch.equal(out2, out)
+    del acc, out, enc, enc2, a8, acc2, out2
 
 
 # ----------------------------------------------------------------------------- config 2: sq_encode alone
