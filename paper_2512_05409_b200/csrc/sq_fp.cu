@@ -225,20 +225,38 @@ __global__ void __launch_bounds__(256) fp_decode_kernel(int b, int k, const uint
 }
 
 // ------------------------------------------------------------------------------------------------
-// GEMM: persistent, one CTA per SM, tiles of 128 rows x 256 output channels, K steps of 128.
-//   warp 0      one thread: TMA loads of the A (a8) and B (w8) tiles of a step into a 4-deep ring
+// GEMM: persistent, one CTA per SM, K steps of 128, everything fed by TMA.
+//   warp 0      one thread: TMA loads of this CTA's A (a8) and B (w8) tiles of a step into a ring
 //               (128-byte swizzle: the layout the tensor core reads), both on one mbarrier
-//   warp 1      one thread: four tcgen05.mma.kind::f8f6f4 (K = 32 each) per step, fp32 accumulation
-//               in tensor memory; two accumulators (all 512 columns), so the epilogue of a tile
-//               overlaps the main loop of the next
+//   warp 1      one thread (of the leader CTA): four tcgen05.mma.kind::f8f6f4 (K = 32 each) per
+//               step, fp32 accumulation in tensor memory; two accumulators (all 512 columns), so
+//               the epilogue of a tile overlaps the main loop of the next
 //   warps 2-5   epilogue: tcgen05.ld, (acc * s_hi[m]) * s_w[n], bf16, 16-byte stores
+// PAIR = 1 (at most 128 rows): tiles of 128 rows x 256 output channels per CTA.  Its shared memory
+// is the bound: per K = 32 instruction 12 KB arrive by TMA and 12 KB are read by the tensor core in
+// the 128 cycles the instruction takes, 192 of the 128 bytes per cycle there are (measured: the
+// tensor pipe 69 % busy).
+// PAIR = 2 (more rows): two CTAs of a cluster share a tile of 256 rows x 256 channels through
+// tcgen05.mma.cta_group::2.  Each holds its own 128 rows of A and HALF of the weight tile, which
+// both tensor cores read from both shared memories: 8 KB in and 8 KB out per instruction and CTA.
+// Only the leader issues; the peer's idle MMA warp reports each of its landed stages to the
+// leader's "full" barrier; completions are multicast to both CTAs' "empty" and "accumulator
+// ready" barriers; both epilogues hand the accumulators back on the leader's barrier.
 // Concurrent CTAs work on neighbouring row tiles of the same 256 channels, so a weight tile is
 // fetched from HBM once and then served by L2.
 namespace {
 
-constexpr int FBM = 128, FBN = 256, FBK = 128, FNS = 4;
-constexpr int kFStageA = FBM * FBK, kFStageB = FBN * FBK;
-constexpr int kFSmem = FNS * (kFStageA + kFStageB) + 256;
+constexpr int FBM = 128, FBN = 256, FBK = 128;
+template <int PAIR>
+struct FGeo {
+  // 128-byte blocks of K per stage.  A pair's stage is 8 instructions: with 4, waiting for the
+  // stage's barrier, issuing and committing take longer than the 0.28 us of tensor work they start.
+  static constexpr int KB = PAIR == 2 ? 2 : 1;
+  static constexpr int NS = PAIR == 2 ? 3 : 4;
+  static constexpr int kStageA = KB * FBM * FBK;             // this CTA's rows
+  static constexpr int kStageB = KB * (FBN / PAIR) * FBK;    // this CTA's share of the output channels
+  static constexpr int kSmem = NS * (kStageA + kStageB) + 256;
+};
 constexpr int kFThreads = 6 * 32;
 
 struct FpGemmParams {
@@ -259,16 +277,28 @@ __device__ __forceinline__ uint64_t fdesc(uint32_t saddr) {
   d |= (uint64_t)2 << 61;
   return d;
 }
-// D = f32 (1 at bit 4); A, B = E4M3 (format 0), K-major; N at bit 17, M at bit 24.
-constexpr uint32_t kFIdesc = (1u << 4) | (0u << 7) | (0u << 10) | ((uint32_t)(FBN >> 3) << 17) | ((uint32_t)(FBM >> 4) << 24);
+// D = f32 (1 at bit 4); A, B = E4M3 (format 0), K-major; N at bit 17, M (of the whole instruction:
+// 128 per participating CTA) at bit 24.
+__device__ __forceinline__ constexpr uint32_t f_idesc(int m) {
+  return (1u << 4) | (0u << 7) | (0u << 10) | ((uint32_t)(FBN >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
+}
 
+template <int CG>
 __device__ __forceinline__ void umma_f8(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
-      "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
-      : "memory");
+  if (CG == 2)
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f8f6f4 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
+        "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+  else
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
+        "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
 }
 __device__ __forceinline__ void f_expect_tx(uint32_t bar, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
@@ -279,49 +309,64 @@ __device__ __forceinline__ void f_tma_2d(uint32_t dst, const CUtensorMap* map, i
       "l"(map), "r"(x), "r"(y), "r"(bar)
       : "memory");
 }
+// A wait of the leader on a barrier the peer also arrives on acquires at cluster scope.
+template <int PAIR>
+__device__ __forceinline__ bool f_wait_leader(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  return PAIR == 2 ? mbar_wait_cluster(bar, parity, abort_flag) : mbar_wait(bar, parity, abort_flag);
+}
 
 }  // namespace
 
+template <int PAIR>
 __global__ void __launch_bounds__(kFThreads, 1)
     fp_gemm_kernel(const FpGemmParams p, const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b) {
+  using G = FGeo<PAIR>;
+  constexpr int NS = G::NS, KB = G::KB, kStageA = G::kStageA, kStageB = G::kStageB;
+  constexpr int TM = FBM * PAIR;  // rows of a tile
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   uint8_t* smem = smem_raw;
-  if ((smem_u32(smem_raw) & 1023u) != 0) {
+  const bool misaligned = (smem_u32(smem_raw) & 1023u) != 0;  // the same in every CTA: nobody is left waiting
+  if (misaligned) {
     if (threadIdx.x == 0) atomicExch(p.status, (int)SQ_ERR_CUDA);
     return;
   }
   uint8_t* sA = smem;
-  uint8_t* sB = sA + FNS * kFStageA;
-  uint8_t* sCtl = sB + FNS * kFStageB;
-  const uint32_t bar_full = smem_u32(sCtl);          // FNS
-  const uint32_t bar_empty = bar_full + 8 * FNS;     // FNS
-  const uint32_t bar_tfull = bar_empty + 8 * FNS;    // 2: accumulator complete
+  uint8_t* sB = sA + NS * kStageA;
+  uint8_t* sCtl = sB + NS * kStageB;
+  const uint32_t bar_full = smem_u32(sCtl);          // NS
+  const uint32_t bar_empty = bar_full + 8 * NS;      // NS
+  const uint32_t bar_tfull = bar_empty + 8 * NS;     // 2: accumulator complete
   const uint32_t bar_tempty = bar_tfull + 16;        // 2: accumulator read out
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(sCtl + 8 * (2 * FNS + 4));
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(sCtl + 8 * (2 * FNS + 4) + 8);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(sCtl + 8 * (2 * NS + 4));
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(sCtl + 8 * (2 * NS + 4) + 8);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int tiles_m = (p.M + FBM - 1) / FBM, tiles_n = (p.N + FBN - 1) / FBN;
-  const int ntiles = tiles_m * tiles_n, KS = p.K / FBK;
+  const int rank = PAIR == 2 ? (int)cluster_ctarank() : 0;
+  const int cl = (int)blockIdx.x / PAIR, ncl = (int)gridDim.x / PAIR;  // this CTA (pair) among the CTAs (pairs)
+  const int tiles_m = (p.M + TM - 1) / TM, tiles_n = (p.N + FBN - 1) / FBN;
+  const int KBT = p.K / FBK;              // 128-byte blocks of K
+  const int ntiles = tiles_m * tiles_n, KS = (KBT + KB - 1) / KB;
 
   if (tid == 0) {
-    for (int s = 0; s < FNS; ++s) {
-      mbar_init(bar_full + 8 * s, 1);
+    for (int s = 0; s < NS; ++s) {
+      // leader of a pair: its own loads' arrival plus the peer's report
+      mbar_init(bar_full + 8 * s, (PAIR == 2 && rank == 0) ? 2 : 1);
       mbar_init(bar_empty + 8 * s, 1);
     }
     for (int a = 0; a < 2; ++a) {
       mbar_init(bar_tfull + 8 * a, 1);
-      mbar_init(bar_tempty + 8 * a, 4 * 32);
+      mbar_init(bar_tempty + 8 * a, PAIR * 4);  // one arrival per epilogue warp (of both CTAs, on the leader's)
     }
     *abort_flag = 0;
     fence_mbar_init();
   }
   if (warp == 1) {
-    tmem_alloc<1>(smem_u32(tmem_slot), 2 * FBN);
-    tmem_relinquish<1>();
+    tmem_alloc<PAIR>(smem_u32(tmem_slot), 2 * FBN);
+    tmem_relinquish<PAIR>();
   }
   tc_fence_before();
   __syncthreads();
+  if (PAIR == 2) cluster_sync_all();  // the peer's barriers exist before anything arrives on them
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
 
@@ -329,50 +374,74 @@ __global__ void __launch_bounds__(kFThreads, 1)
     if (lane == 0) {
       uint32_t it = 0;
       bool ok = true;
-      for (int t = blockIdx.x; t < ntiles && ok; t += gridDim.x) {
-        const int m0 = (t % tiles_m) * FBM, n0 = (t / tiles_m) * FBN;
+      for (int t = cl; t < ntiles && ok; t += ncl) {
+        const int m0 = (t % tiles_m) * TM + rank * FBM, n0 = (t / tiles_m) * FBN + rank * (FBN / PAIR);
         for (int ks = 0; ks < KS && ok; ++ks, ++it) {
-          const int s = it % FNS;
-          ok = mbar_wait(bar_empty + 8 * s, ((it / FNS) & 1u) ^ 1u, abort_flag);
+          const int s = it % NS;
+          ok = mbar_wait(bar_empty + 8 * s, ((it / NS) & 1u) ^ 1u, abort_flag);
           if (!ok) break;
           const uint32_t bar = bar_full + 8 * s;
-          f_expect_tx(bar, (uint32_t)(kFStageA + kFStageB));  // rows past M / N come back as zeros
-          f_tma_2d(smem_u32(sA + s * kFStageA), &map_a, ks * FBK, m0, bar);
-          f_tma_2d(smem_u32(sB + s * kFStageB), &map_b, ks * FBK, n0, bar);
+          const int nkb = min(KB, KBT - ks * KB);
+          f_expect_tx(bar, (uint32_t)(nkb * (kStageA + kStageB) / KB));  // rows past M / N come back as zeros
+          for (int kb = 0; kb < nkb; ++kb) {
+            f_tma_2d(smem_u32(sA + s * kStageA + kb * (FBM * FBK)), &map_a, (ks * KB + kb) * FBK, m0, bar);
+            f_tma_2d(smem_u32(sB + s * kStageB + kb * ((FBN / PAIR) * FBK)), &map_b, (ks * KB + kb) * FBK, n0, bar);
+          }
         }
       }
     }
     __syncwarp();
   } else if (warp == 1) {
-    if (lane == 0) {
+    if (lane == 0 && rank == 0) {
+      constexpr uint32_t idesc = f_idesc(TM);
       uint32_t it = 0, tc = 0;
       bool ok = true;
-      for (int t = blockIdx.x; t < ntiles && ok; t += gridDim.x, ++tc) {
+      for (int t = cl; t < ntiles && ok; t += ncl, ++tc) {
         const uint32_t buf = tc & 1u;
-        ok = mbar_wait(bar_tempty + 8 * buf, ((tc >> 1) & 1u) ^ 1u, abort_flag);  // the accumulator's previous tile was read out
+        // the accumulator's previous tile was read out (by both CTAs)
+        ok = f_wait_leader<PAIR>(bar_tempty + 8 * buf, ((tc >> 1) & 1u) ^ 1u, abort_flag);
         if (!ok) break;
         tc_fence_after();
         for (int ks = 0; ks < KS && ok; ++ks, ++it) {
-          const int s = it % FNS;
-          ok = mbar_wait(bar_full + 8 * s, (it / FNS) & 1u, abort_flag);
+          const int s = it % NS;
+          ok = f_wait_leader<PAIR>(bar_full + 8 * s, (it / NS) & 1u, abort_flag);
           if (!ok) break;
           tc_fence_after();
-          const uint64_t da = fdesc(smem_u32(sA + s * kFStageA)), db = fdesc(smem_u32(sB + s * kFStageB));
 #pragma unroll
-          for (int kk = 0; kk < FBK / 32; ++kk)
-            umma_f8(tmem + buf * FBN, da + 2 * kk, db + 2 * kk, kFIdesc, (ks > 0 || kk > 0) ? 1u : 0u);
-          umma_commit<1>(bar_empty + 8 * s);
+          for (int kb = 0; kb < KB; ++kb) {
+            if (ks * KB + kb < KBT) {  // (the last stage of an odd number of 128-byte blocks is half full)
+              const uint64_t da = fdesc(smem_u32(sA + s * kStageA + kb * (FBM * FBK)));
+              const uint64_t db = fdesc(smem_u32(sB + s * kStageB + kb * ((FBN / PAIR) * FBK)));
+#pragma unroll
+              for (int kk = 0; kk < FBK / 32; ++kk)
+                umma_f8<PAIR>(tmem + buf * FBN, da + 2 * kk, db + 2 * kk, idesc, (ks > 0 || kb > 0 || kk > 0) ? 1u : 0u);
+            }
+          }
+          umma_commit<PAIR>(bar_empty + 8 * s);
         }
-        if (ok) umma_commit<1>(bar_tfull + 8 * buf);
+        if (ok) umma_commit<PAIR>(bar_tfull + 8 * buf);
+      }
+    } else if (lane == 0 && PAIR == 2) {
+      // The leader's MMA thread cannot watch this CTA's barriers: report every landed stage, in
+      // order, on the leader's "full" barrier.  (A stage is re-armed only after the leader has
+      // used it, so no phase can pass unseen.)
+      uint32_t it = 0;
+      bool ok = true;
+      for (int t = cl; t < ntiles && ok; t += ncl) {
+        for (int ks = 0; ks < KS && ok; ++ks, ++it) {
+          const int s = it % NS;
+          ok = mbar_wait(bar_full + 8 * s, (it / NS) & 1u, abort_flag);
+          if (ok) mbar_arrive_cta(bar_full + 8 * s, 0);
+        }
       }
     }
     __syncwarp();
   } else {
     const int q = warp & 3;  // tensor-memory lane quarter this warp may read
     uint32_t tc = 0;
-    for (int t = blockIdx.x; t < ntiles; t += gridDim.x, ++tc) {
+    for (int t = cl; t < ntiles; t += ncl, ++tc) {
       const uint32_t buf = tc & 1u;
-      const int m0 = (t % tiles_m) * FBM, n0 = (t / tiles_m) * FBN;
+      const int m0 = (t % tiles_m) * TM + rank * FBM, n0 = (t / tiles_m) * FBN;
       const int m = m0 + 32 * q + lane;
       const float sh = m < p.M ? __ldg(p.s_hi + m) : 0.f;
       if (!mbar_wait_idle(bar_tfull + 8 * buf, (tc >> 1) & 1u, abort_flag)) break;
@@ -404,13 +473,20 @@ __global__ void __launch_bounds__(kFThreads, 1)
         }
       }
       tc_fence_before();
-      mbar_arrive(bar_tempty + 8 * buf);
+      __syncwarp();
+      if (lane == 0) {
+        if (PAIR == 2) mbar_arrive_cta(bar_tempty + 8 * buf, 0);
+        else mbar_arrive(bar_tempty + 8 * buf);
+      }
     }
   }
   tc_fence_before();
   __syncthreads();
+  // Neither CTA of a pair may leave (or free tensor memory) while the other can still arrive on
+  // its barriers or have instructions reading its shared memory.
+  if (PAIR == 2) cluster_sync_all();
   if (tid == 0 && *abort_flag) atomicExch(p.status, (int)SQ_ERR_TIMEOUT);
-  if (warp == 1) tmem_dealloc<1>(tmem, 2 * FBN);
+  if (warp == 1) tmem_dealloc<PAIR>(tmem, 2 * FBN);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -482,15 +558,19 @@ cudaError_t launch_fp_gemm(const float* s_hi, const uint8_t* a8, const float* s_
   }
   if (!attr_set[dev].load(std::memory_order_acquire)) {
     std::lock_guard<std::mutex> lock(setup_mutex());
-    err = cudaFuncSetAttribute(fp_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kFSmem);
+    err = cudaFuncSetAttribute(fp_gemm_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, FGeo<1>::kSmem);
+    if (err != cudaSuccess) return err;
+    err = cudaFuncSetAttribute(fp_gemm_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, FGeo<2>::kSmem);
     if (err != cudaSuccess) return err;
     attr_set[dev].store(true, std::memory_order_release);
   }
+  // CTA pairs from 129 rows on (a second CTA would have no rows below that)
+  const int pair = M > FBM ? 2 : 1;
   CUtensorMap map_a, map_b;
   const cuuint32_t estr[2] = {1, 1};
   const cuuint64_t pitch[1] = {(cuuint64_t)K};
   const cuuint64_t dim_a[2] = {(cuuint64_t)K, (cuuint64_t)M}, dim_b[2] = {(cuuint64_t)K, (cuuint64_t)N};
-  const cuuint32_t box_a[2] = {FBK, FBM}, box_b[2] = {FBK, FBN};
+  const cuuint32_t box_a[2] = {FBK, FBM}, box_b[2] = {FBK, (cuuint32_t)(FBN / pair)};
   if (encode(&map_a, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<uint8_t*>(a8), dim_a, pitch, box_a, estr,
              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
@@ -508,9 +588,28 @@ cudaError_t launch_fp_gemm(const float* s_hi, const uint8_t* a8, const float* s_
   p.M = (int)M;
   p.N = (int)N;
   p.K = (int)K;
-  const int64_t ntiles = ((M + FBM - 1) / FBM) * ((N + FBN - 1) / FBN);
-  const unsigned grid = (unsigned)(ntiles < sms ? ntiles : sms);
-  fp_gemm_kernel<<<grid, kFThreads, kFSmem, st>>>(p, map_a, map_b);
+  const int64_t ntiles = ((M + FBM * pair - 1) / (FBM * pair)) * ((N + FBN - 1) / FBN);
+  if (pair == 1) {
+    const unsigned grid = (unsigned)(ntiles < sms ? ntiles : sms);
+    fp_gemm_kernel<1><<<grid, kFThreads, FGeo<1>::kSmem, st>>>(p, map_a, map_b);
+  } else {
+    const int64_t slots = sms / 2;
+    cudaLaunchConfig_t lc;
+    memset(&lc, 0, sizeof(lc));
+    cudaLaunchAttribute la[1];
+    la[0].id = cudaLaunchAttributeClusterDimension;
+    la[0].val.clusterDim.x = 2;
+    la[0].val.clusterDim.y = 1;
+    la[0].val.clusterDim.z = 1;
+    lc.gridDim = dim3((unsigned)(2 * (ntiles < slots ? ntiles : slots)), 1, 1);
+    lc.blockDim = dim3(kFThreads, 1, 1);
+    lc.dynamicSmemBytes = FGeo<2>::kSmem;
+    lc.stream = st;
+    lc.attrs = la;
+    lc.numAttrs = 1;
+    err = cudaLaunchKernelEx(&lc, fp_gemm_kernel<2>, p, map_a, map_b);
+    if (err != cudaSuccess) return err;
+  }
   return cudaGetLastError();
 }
 
