@@ -41,10 +41,6 @@ __device__ __forceinline__ uint32_t e2m1_of(double p) {  // sign in bit 3; a val
   const uint32_t c = round_code(fabs(p), 1, 0, 7u);
   return c == 0 ? 0u : (c | (p < 0.0 ? 8u : 0u));
 }
-__device__ __forceinline__ uint32_t e4m3_of(double p) {  // sign in bit 7
-  const uint32_t c = round_code(fabs(p), 3, -6, 0x7Eu);
-  return c == 0 ? 0u : (c | (p < 0.0 ? 0x80u : 0u));
-}
 // E4M3 byte of an E2M1 code's value times 2^e (exact: e <= 6 keeps it at or below 384).
 __device__ __forceinline__ uint32_t e4m3_of_e2m1(uint32_t code, int e) {
   const uint32_t t = code & 7u;
@@ -52,6 +48,31 @@ __device__ __forceinline__ uint32_t e4m3_of_e2m1(uint32_t code, int e) {
   // t = 1 -> 0.5 = 2^-1; t >= 2: exponent (t >> 1) - 1, mantissa bit t & 1
   const uint32_t mag = t == 1 ? (uint32_t)((6 + e) << 3) : ((uint32_t)((t >> 1) + 6 + e) << 3) | ((t & 1u) << 2);
   return mag | ((code & 8u) << 4);
+}
+
+// The same codes without double precision, for the encoder's per-element work: the code of the
+// magnitude |a| * c (a bf16, c fp32 > 0) in a format with `mb` mantissa bits and smallest normal
+// exponent emin.  The spacing of the format's grid at that magnitude is 2^(ex - mb), ex = the
+// (clamped) exponent; one FMA with the constant 1.5 * 2^(ex - mb + 23) rounds the EXACT product to
+// that grid, half-even, and leaves the integer n = round(|a| c / spacing) in its low mantissa
+// bits; code = ((ex - emin) << mb) + n as in round_code.  ex is read off the rounded product: it
+// differs from the exact product's exponent only when that lies within 2^-24 of a power of two from
+// below, where both grids round to the power of two itself.
+template <int MB, int EMIN, uint32_t MAXC>
+__device__ __forceinline__ uint32_t round_code32(float a_abs, float c) {
+  const int ex = max((int)(__float_as_uint(a_abs * c) >> 23) - 127, EMIN);
+  const uint32_t magic = ((uint32_t)(ex - MB + 23 + 127) << 23) | 0x00400000u;
+  const uint32_t n = __float_as_uint(__fmaf_rn(a_abs, c, __uint_as_float(magic))) - magic;
+  return min(((uint32_t)(ex - EMIN) << MB) + n, MAXC);
+}
+// a: bf16 bit pattern (finite); c > 0.
+__device__ __forceinline__ uint32_t e2m1_of32(uint32_t a_bits, float c) {
+  const uint32_t code = round_code32<1, 0, 7u>(__uint_as_float((a_bits & 0x7FFFu) << 16), c);
+  return code == 0 ? 0u : (code | ((a_bits >> 12) & 8u));
+}
+__device__ __forceinline__ uint32_t e4m3_of32(uint32_t a_bits, float c) {
+  const uint32_t code = round_code32<3, -6, 0x7Eu>(__uint_as_float((a_bits & 0x7FFFu) << 16), c);
+  return code == 0 ? 0u : (code | ((a_bits >> 8) & 0x80u));
 }
 
 __device__ __forceinline__ uint32_t block_max(uint32_t v, uint32_t* scratch) {
@@ -91,7 +112,10 @@ __global__ void __launch_bounds__(256) fp_pack_weights_kernel(const uint16_t* __
 }
 
 // One block per token row, the row staged in shared memory (the plain organisation of the integer
-// path's general kernel: this variant is not tuned for bandwidth).
+// path's general kernel).  Dynamic positions: a warp per bank finds the k-th largest magnitude by
+// a bitwise search on warp-wide counts; codes by single-precision magic-number rounding; a
+// selected place is marked in the staged row by a non-finite pattern that carries its byte, so the
+// dense pass writes whole words of nibbles and of the merged operand.
 template <int B>
 __global__ void __launch_bounds__(256) fp_encode_kernel(int k, const uint16_t* __restrict__ X, int64_t K,
                                                         const uint8_t* __restrict__ positions, uint8_t* __restrict__ dq4,
@@ -116,49 +140,58 @@ __global__ void __launch_bounds__(256) fp_encode_kernel(int k, const uint16_t* _
   const float sh = amax > 0.f ? __fdiv_rn(amax, 256.0f) : 0.f;
   uint8_t* arow = a8 + m * K;
 
-  // sparse entries: E4M3 of a * inv, in ascending position; their places are marked in the staged
-  // row (0xFFFF is a NaN pattern, never an input) so that the dense pass skips them
+  // sparse entries: E4M3 of a * inv, in ascending position.  Their places in the staged row are
+  // overwritten with a marker that carries the byte: exponent field all ones (no finite input has
+  // it), the byte's sign in the sign bit, its other seven bits in the mantissa -- the dense pass
+  // recognises the place and finds the merged operand's byte there.
+  auto marker = [](uint32_t q) -> uint16_t { return (uint16_t)(((q & 0x80u) << 8) | 0x7F80u | (q & 0x7Fu)); };
   if (positions != nullptr) {
     for (int64_t t = tid; t < G * k; t += 256) {
       const int64_t j = (t / k) * B + positions[t];
-      const uint32_t q = e4m3_of((double)bf16_bits_to_f32(srow[j]) * (double)inv);
+      const uint32_t q = e4m3_of32(srow[j], inv);
       vals[m * G * k + t] = (uint8_t)q;
-      arow[j] = (uint8_t)q;
-      srow[j] = 0xFFFFu;
+      srow[j] = marker(q);
     }
   } else {
     constexpr int EPL = B / 32;
     for (int64_t g = warp; g < G; g += 8) {
-      uint32_t key[EPL], raw[EPL];
+      uint32_t mag[EPL], raw[EPL];
 #pragma unroll
       for (int t = 0; t < EPL; ++t) {
-        const int j = lane + 32 * t;
-        raw[t] = srow[g * B + j];
-        key[t] = ((raw[t] & 0x7FFFu) << 7) | (uint32_t)(127 - j);  // unique: magnitude, then lower index
+        raw[t] = srow[g * B + lane + 32 * t];
+        mag[t] = raw[t] & 0x7FFFu;
       }
-      int rank[EPL];
+      // T = the k-th largest magnitude of the bank (with multiplicity): the largest T with at least
+      // k magnitudes >= T, built bit by bit from warp-wide counts.  Everything above T is selected;
+      // of the elements equal to T the lowest indices fill what is left.  (Several banks in flight
+      // per warp were measured no faster: the kernel is bound by instruction count, not latency.)
+      uint32_t T = 0;
+      for (int bit = 14; bit >= 0; --bit) {
+        const uint32_t cand = T | (1u << bit);
+        int c = 0;
 #pragma unroll
-      for (int t = 0; t < EPL; ++t) rank[t] = 0;
+        for (int t = 0; t < EPL; ++t) c += mag[t] >= cand ? 1 : 0;
+        if (__reduce_add_sync(0xffffffffu, c) >= k) T = cand;
+      }
+      int above = 0;
 #pragma unroll
-      for (int u = 0; u < EPL; ++u)
-        for (int l = 0; l < 32; ++l) {
-          const uint32_t other = __shfl_sync(0xffffffffu, key[u], l);
+      for (int t = 0; t < EPL; ++t) above += mag[t] > T ? 1 : 0;
+      const int need = k - __reduce_add_sync(0xffffffffu, above);
+      int before_eq = 0, before = 0;
 #pragma unroll
-          for (int t = 0; t < EPL; ++t) rank[t] += (other > key[t]) ? 1 : 0;
-        }
-      int before = 0;
-#pragma unroll
-      for (int t = 0; t < EPL; ++t) {
-        const bool sel = rank[t] < k;
+      for (int t = 0; t < EPL; ++t) {  // index order: t = 0 holds elements 0..31, lanes ascending
+        const bool eq = mag[t] == T;
+        const uint32_t m_eq = __ballot_sync(0xffffffffu, eq);
+        const bool sel = mag[t] > T || (eq && before_eq + __popc(m_eq & ((1u << lane) - 1u)) < need);
+        before_eq += __popc(m_eq);
         const uint32_t mask = __ballot_sync(0xffffffffu, sel);
         if (sel) {
           const int slot = before + __popc(mask & ((1u << lane) - 1u));
           const int j = lane + 32 * t;
-          const uint32_t q = e4m3_of((double)bf16_bits_to_f32(raw[t]) * (double)inv);
+          const uint32_t q = e4m3_of32(raw[t], inv);
           vals[(m * G + g) * k + slot] = (uint8_t)q;
           idx[(m * G + g) * k + slot] = (uint8_t)j;
-          arow[g * B + j] = (uint8_t)q;
-          srow[g * B + j] = 0xFFFFu;
+          srow[g * B + j] = marker(q);
         }
         before += __popc(mask);
       }
@@ -166,9 +199,15 @@ __global__ void __launch_bounds__(256) fp_encode_kernel(int k, const uint16_t* _
   }
   __syncthreads();
   uint32_t rm = 0;
-  for (int64_t i = tid; i < K; i += 256) {
-    const uint32_t v = srow[i];
-    if (v != 0xFFFFu) rm = max(rm, v & 0x7FFFu);
+  for (int64_t i = (int64_t)tid * 8; i < K; i += 256 * 8) {
+    const uint4 v = *reinterpret_cast<const uint4*>(srow + i);
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      const uint32_t lo = w[q] & 0x7FFFu, hi = (w[q] >> 16) & 0x7FFFu;
+      if (lo < 0x7F80u) rm = max(rm, lo);  // (a marker's magnitude bits are at least 0x7F80)
+      if (hi < 0x7F80u) rm = max(rm, hi);
+    }
   }
   const float rmax = bf16_bits_to_f32(block_max(rm, scratch));
   int e = 0;
@@ -182,14 +221,28 @@ __global__ void __launch_bounds__(256) fp_encode_kernel(int k, const uint16_t* _
     s_lo[m] = sh * (float)(1 << e);
     shift[m] = (uint8_t)e;
   }
-  const double inv_lo = (double)(inv * __int_as_float((127 - e) << 23));
-  for (int64_t i = (int64_t)tid * 2; i < K; i += 512) {
-    const uint32_t v0 = srow[i], v1 = srow[i + 1];
-    const uint32_t q0 = v0 == 0xFFFFu ? 0u : e2m1_of((double)bf16_bits_to_f32(v0) * inv_lo);
-    const uint32_t q1 = v1 == 0xFFFFu ? 0u : e2m1_of((double)bf16_bits_to_f32(v1) * inv_lo);
-    dq4[m * (K / 2) + i / 2] = (uint8_t)(q0 | (q1 << 4));
-    if (v0 != 0xFFFFu) arow[i] = (uint8_t)e4m3_of_e2m1(q0, e);
-    if (v1 != 0xFFFFu) arow[i + 1] = (uint8_t)e4m3_of_e2m1(q1, e);
+  // dense codes, eight elements per thread and step: one 32-bit word of nibbles and eight bytes of
+  // the merged operand
+  const float inv_lo = inv * __int_as_float((127 - e) << 23);
+  for (int64_t i = (int64_t)tid * 8; i < K; i += 256 * 8) {
+    const uint4 v = *reinterpret_cast<const uint4*>(srow + i);
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+    uint32_t nib = 0, by[2] = {0, 0};
+#pragma unroll
+    for (int q = 0; q < 8; ++q) {
+      const uint32_t h = (w[q >> 1] >> (16 * (q & 1))) & 0xFFFFu;
+      uint32_t code = 0, byte;
+      if ((h & 0x7F80u) == 0x7F80u) {
+        byte = ((h >> 8) & 0x80u) | (h & 0x7Fu);
+      } else {
+        code = e2m1_of32(h, inv_lo);
+        byte = e4m3_of_e2m1(code, e);
+      }
+      nib |= code << (4 * q);
+      by[q >> 2] |= byte << (8 * (q & 3));
+    }
+    *reinterpret_cast<uint32_t*>(dq4 + m * (K / 2) + i / 2) = nib;
+    *reinterpret_cast<uint2*>(arow + i) = make_uint2(by[0], by[1]);
   }
 }
 
