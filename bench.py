@@ -349,7 +349,7 @@ def bench_format_sweep(sq, dev, peaks, iters=5):
     int8_peak = peaks["bf16_tflops"] * INT8_OVER_BF16
     tf32 = torch.backends.cuda.matmul.allow_tf32
     torch.backends.cuda.matmul.allow_tf32 = False
-    res = []
+    res, fp_enc = [], []
     W = gen.weights(N, K, seed=5, device=dev)
     for scale in (10.0, 50.0):
         X = gen.activations(M, K, seed=5, outlier_fraction=0.01, outlier_scale=scale, device=dev)
@@ -392,12 +392,19 @@ def bench_format_sweep(sq, dev, peaks, iters=5):
                     err = float((out.float() - ref).norm()) / ref_norm
                     res.append([b, k, "fp8/fp4 static" if static else "fp8/fp4 dynamic", int(scale), round(ms * 1e3, 1),
                                 round(tops), round(tops / int8_peak, 3), round(err, 4)])
+                    if b == 64 and k == 8 and scale == 10.0:
+                        ems, _ = time_launches(lambda i: sq.sq_fp_encode(fmt, X, pos, out=encf, a8=a8), iters, 2)
+                        nbytes = M * K * (2.0 + 0.5 + (1.0 if static else 2.0) * k / b + 1.0)
+                        fp_enc.append(["static" if static else "dynamic", round(ems * 1e3, 1),
+                                       round(nbytes / (ems * 1e-3) / 1e9)])
                     del wf, encf, a8
         del X, calib, ref, out
         torch.cuda.empty_cache()
     torch.backends.cuda.matmul.allow_tf32 = tf32
     return {"cols": ["b", "k", "positions", "outlier_scale", "gemm_us", "TOPS", "of_measured_int8", "rel_err_vs_fp32"],
-            "rows": res}
+            "rows": res,
+            # sq_fp_encode at this shape, b=64, k=8 (codes, sparse entries and the merged 8-bit operand written)
+            "fp_encode": {"cols": ["positions", "us", "GBps"], "rows": fp_enc}}
 
 
 def oracle_sample(K, N, bank, k, seed, rows=32, cols=512):

@@ -55,7 +55,7 @@ constexpr int NX = 8;          // widened activation stages
 constexpr int kWGroups = 2, kWGroupThreads = 64, kXWarps = 4;
 constexpr int kTmaWarp = 0, kFirstW = 1, kFirstX = 5, kMmaWarp = 9, kFirstEpi = 10;
 constexpr int kThreadsS = 14 * 32;
-constexpr int kCtlS = 384;
+constexpr int kCtlS = 384 + 2 * SC * 4 + MT * 4;  // barriers, then the slab's constants for the finish
 constexpr int kPitch = SUP * (BK / 2);     // bytes per packed row of a stage
 constexpr int kPackW = SC * kPitch;        // 32 KB
 constexpr int kPackX = MT * kPitch;        // 4 KB
@@ -139,7 +139,10 @@ __global__ void __launch_bounds__(kThreadsS, 2)
   constexpr int kBars = 2 * NPK + 2 * NW + 2 * NX + 1;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(sCtl + 8 * kBars);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(sCtl + 8 * kBars + 8);
-  static_assert(8 * kBars + 16 <= kCtlS, "control block too small");
+  static_assert(8 * kBars + 16 <= 384, "control block too small");
+  int32_t* s_cs = reinterpret_cast<int32_t*>(sCtl + 384);   // colsum of the slab's channels
+  float* s_sw = reinterpret_cast<float*>(s_cs + SC);        // their weight scales
+  float* s_sh = s_sw + SC;                                   // the tokens' scales
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int parts = p.parts;
@@ -168,6 +171,12 @@ __global__ void __launch_bounds__(kThreadsS, 2)
   if (warp == kMmaWarp) {
     tmem_alloc<1>(smem_u32(tmem_slot), kTmemCols);
     tmem_relinquish<1>();
+  }
+  if (warp == kTmaWarp && lane == 0) {  // the descriptors are on their way while the barriers are set up
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&map_w4) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&map_x4) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&map_sv) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&map_si) : "memory");
   }
   tc_fence_before();
   __syncthreads();
@@ -322,6 +331,13 @@ __global__ void __launch_bounds__(kThreadsS, 2)
     // =============================================================== accumulator -> this CTA's partial sums
     // (the rings are idle once the accumulator is complete: every MMA has read its operands)
     const int q = warp & 3;  // a warp reads the tensor-memory lane quarter (warp index mod 4)
+    {
+      // what the finish needs per channel and token, fetched while the K walk runs
+      const int e = tid - kFirstEpi * 32, n = min(n0 + e, p.N - 1);
+      s_cs[e] = __ldg(p.colsum + n);
+      s_sw[e] = __ldg(p.s_w + n);
+      if (e < MT) s_sh[e] = e < p.M ? __ldg(p.s_hi + e) : 0.f;
+    }
     if (mbar_wait_idle(bar_tfull, 0, abort_flag)) {
       tc_fence_after();
       const int ch = 32 * q + lane;
@@ -346,9 +362,9 @@ __global__ void __launch_bounds__(kThreadsS, 2)
   {
     // CTA `part` finishes channels [part * SC / parts, (part + 1) * SC / parts) of the slab for all
     // tokens: adds the parts' sums (integer: order-free) and runs the usual epilogue arithmetic.
-    const int share = SC / parts;
+    const int share = SC / parts, lg = 31 - __clz(share);  // parts is 1, 2, 4 or 8
     for (int i = tid; i < share * p.M; i += kThreadsS) {
-      const int ch = part * share + i % share, m = i / share;
+      const int ch = part * share + (i & (share - 1)), m = i >> lg;
       const int n = n0 + ch;
       if (n >= p.N) continue;
       const uint32_t laddr = smem_u32(smem) + (uint32_t)(ch * MT + m) * 4u;
@@ -356,20 +372,25 @@ __global__ void __launch_bounds__(kThreadsS, 2)
       if (parts == 1) {
         asm volatile("ld.shared.s32 %0, [%1];" : "=r"(v) : "r"(laddr) : "memory");
       } else {
-        for (int sp = 0; sp < parts; ++sp) {
-          int a;
-          asm volatile(
-              "{\n\t.reg .b32 ra;\n\t"
-              "mapa.shared::cluster.u32 ra, %1, %2;\n\t"
-              "ld.shared::cluster.s32 %0, [ra];\n\t}"
-              : "=r"(a)
-              : "r"(laddr), "r"(sp)
-              : "memory");
-          v += a;
+        // all parts' loads first, then the sum: a load followed by its add would wait out one
+        // remote access after the other
+        int a[8];
+#pragma unroll
+        for (int sp = 0; sp < 8; ++sp) {
+          a[sp] = 0;
+          if (sp < parts)
+            asm volatile(
+                "{\n\t.reg .b32 ra;\n\t"
+                "mapa.shared::cluster.u32 ra, %1, %2;\n\t"
+                "ld.shared::cluster.s32 %0, [ra];\n\t}"
+                : "=r"(a[sp])
+                : "r"(laddr), "r"(sp));
         }
+#pragma unroll
+        for (int sp = 0; sp < 8; ++sp) v += a[sp];
       }
-      const int acc = (v - 2048 * p.colsum[n]) >> 4;
-      p.out[(size_t)m * p.N + n] = (uint16_t)f32_to_bf16_bits(((float)acc * p.s_hi[m]) * p.s_w[n]);
+      const int acc = (v - 2048 * s_cs[ch]) >> 4;
+      p.out[(size_t)m * p.N + n] = (uint16_t)f32_to_bf16_bits(((float)acc * s_sh[m]) * s_sw[ch]);
       if (p.acc_out != nullptr) p.acc_out[(size_t)m * p.N + n] = acc;
     }
   }
