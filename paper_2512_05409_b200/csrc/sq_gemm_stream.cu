@@ -53,8 +53,8 @@ constexpr int NPK = 4;         // packed stages in flight
 constexpr int NW = 3;          // widened weight stages
 constexpr int NX = 8;          // widened activation stages
 constexpr int kWGroups = 2, kWGroupThreads = 64, kXWarps = 4;
-constexpr int kTmaWarp = 0, kFirstW = 1, kFirstX = 5, kMmaWarp = 9, kFirstEpi = 10;
-constexpr int kThreadsS = 14 * 32;
+constexpr int kTmaWarp = 0, kFirstW = 1, kFirstX = 5, kMmaWarp = 9, kFirstEpi = 10, kMma2Warp = 14;
+constexpr int kThreadsS = 15 * 32;
 constexpr int kCtlS = 384 + 2 * SC * 4 + MT * 4;  // barriers, then the slab's constants for the finish
 constexpr int kPitch = SUP * (BK / 2);     // bytes per packed row of a stage
 constexpr int kPackW = SC * kPitch;        // 32 KB
@@ -164,7 +164,7 @@ __global__ void __launch_bounds__(kThreadsS, 2)
       mbar_init(bar_xfull + 8 * s, 32);
       mbar_init(bar_xempty + 8 * s, 1);
     }
-    mbar_init(bar_tfull, 1);
+    mbar_init(bar_tfull, KS >= 2 ? 2 : 1);  // one arrival per issuing thread that has steps
     *abort_flag = 0;
     fence_mbar_init();
   }
@@ -307,11 +307,16 @@ __global__ void __launch_bounds__(kThreadsS, 2)
       fence_proxy_async_smem();
       mbar_arrive(bar_xfull + 8 * sx);
     }
-  } else if (warp == kMmaWarp) {
-    // =============================================================== MMA issuer
+  } else if (warp == kMmaWarp || warp == kMma2Warp) {
+    // =============================================================== MMA issuers
+    // A K step is four small instructions, but waiting for its two operands, issuing and
+    // committing take one thread ~0.5 us: that, not the stream, set the pace of the whole kernel.
+    // So TWO threads issue, one the even steps and one the odd ones, each into an accumulator of
+    // its own (the sums are integers: the finish adds the two, in any order the same).
     if (lane == 0) {
+      const int j = warp == kMmaWarp ? 0 : 1;
       bool ok = true;
-      for (int ks = 0; ks < KS && ok; ++ks) {
+      for (int ks = j; ks < KS && ok; ks += 2) {
         const int s = ks % NW, sx = ks % NX;
         ok = mbar_wait(bar_wfull + 8 * s, (ks / NW) & 1u, abort_flag) && mbar_wait(bar_xfull + 8 * sx, (ks / NX) & 1u, abort_flag);
         if (!ok) break;
@@ -320,11 +325,11 @@ __global__ void __launch_bounds__(kThreadsS, 2)
         const uint64_t db = desc_sw128(smem_u32(sX + sx * kStageX));
 #pragma unroll
         for (int kk = 0; kk < BK / 32; ++kk)
-          umma_i8<1>(tmem, da + 2 * kk, db + 2 * kk, kIdescStream, (ks > 0 || kk > 0) ? 1u : 0u);
+          umma_i8<1>(tmem + (uint32_t)(j * MT), da + 2 * kk, db + 2 * kk, kIdescStream, (ks > j || kk > 0) ? 1u : 0u);
         umma_commit<1>(bar_wempty + 8 * s);
         umma_commit<1>(bar_xempty + 8 * sx);
       }
-      if (ok) umma_commit<1>(bar_tfull);
+      if (ok && j < KS) umma_commit<1>(bar_tfull);
     }
     __syncwarp();
   } else if (warp >= kFirstEpi) {
@@ -344,6 +349,13 @@ __global__ void __launch_bounds__(kThreadsS, 2)
       int4* prow = reinterpret_cast<int4*>(smem) + ch * (MT / 4);
       uint32_t v[16];
       tmem_ld16(tmem + ((uint32_t)(32 * q) << 16), v);
+      if (KS >= 2) {  // the odd steps' accumulator
+        uint32_t v2[16];
+        tmem_ld16(tmem + ((uint32_t)(32 * q) << 16) + (uint32_t)MT, v2);
+        tmem_ld_wait();
+#pragma unroll
+        for (int c = 0; c < 16; ++c) v[c] += v2[c];
+      }
       tmem_ld_wait();
       // (a warp's 16-byte stores, one 64-byte row per lane, spread over the banks by themselves)
       prow[0] = make_int4((int)v[0], (int)v[1], (int)v[2], (int)v[3]);
