@@ -29,6 +29,7 @@
 //
 // Formats outside the fast kernels' set (k not a power of two, k/b other than 1/2 .. 1/16 for
 // dynamic positions) take a plain one-block-per-row kernel that ranks every element.
+#include <cstdio>
 #include <cstdlib>
 #include "sq_device.cuh"
 #include "sq_host.h"
@@ -78,7 +79,7 @@ __device__ __forceinline__ uint32_t abs2(uint32_t a) {  // compiles to a packed 
 // from kernel parameters: as immediates the compiler would turn the instruction back into an
 // add or a shift on the busy pipe.
 struct MulK {
-  uint32_t neg1, two, k32, k256, k65536, k16m;
+  uint32_t neg1, two, k32, k256, k65536, k16m, k16, one;
 };
 __device__ __forceinline__ uint32_t imad(uint32_t a, uint32_t m, uint32_t c) {
   uint32_t d;
@@ -955,6 +956,281 @@ __global__ void __launch_bounds__(NT, 1) encode_static_regs_kernel(const EncodeP
 }
 
 // ------------------------------------------------------------------------------------------------
+// Static positions, rows streamed through shared memory.  The register kernel above asks for a
+// row only when its warps are ready for it, so the load's latency is hidden by other groups alone
+// and the selected values have to be fetched a second time from L1/L2.  Here every group of `rw`
+// warps owns a row slot that one bulk asynchronous copy fills (the slot is asked to take its next
+// row the moment its row's selected values have been quantised, about half-way through the
+// row's work, so the copy's latency is covered by the rest of it), and the selected values are
+// plain shared-memory reads of the staged row.  A lane still keeps its NCL 16-byte chunks in
+// registers between the maximum pass and the quantising pass, so the row is read from shared
+// memory once.  The arithmetic that can be written as a multiply-add (magnitudes, the low half's
+// bf16 -> fp32 move, nibble and byte packing) is issued on the multiply-add pipe.  A block owns
+// every gridDim.x-th row and its groups draw the next one from a shared counter.
+// Measured on 8192 x 8192: every row after a group's first takes ~3.7 us, which over the GPU is
+// the memory's full rate; what a launch of this size loses is its start (tables, the first round
+// of rows arriving) and its end (the last row's work with nothing left to fetch).
+//   wait for the slot -> chunks to registers, selected places cleared, maximum of the rest;
+//   maximum of the selected values (read through the offset table) -> group exchange -> scales
+//   -> INT8 codes of the selected values (and, on request, their bytes in the per-group image of
+//   the merged operand) -> slot released and refilled -> INT4 codes (and merged bytes) straight
+//   from the registers.
+// MASK8: the per-element magnitude masks are kept as bytes and widened on the fly (long rows,
+// where a half-word table would not leave room for the slots).
+template <int NCL, int NT, bool INDEP, bool MASK8>
+__global__ void __launch_bounds__(NT, 1) encode_static_ring_kernel(const EncodeParams p) {
+  extern __shared__ __align__(128) uint8_t smem_enc[];
+  const int K = p.K, k = p.k;
+  const int GK = (K / p.b) * k;
+  const int rw = p.rw;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int grp = warp / rw, slice = warp % rw;
+  const int glane = slice * 32 + lane, gsize = rw * 32;
+  const int ngroups = (NT / 32) / rw;
+  constexpr int S8 = NCL * 32;  // 16-byte chunks per warp slice
+  const bool want_a8 = !INDEP && p.a8 != nullptr;
+  const MulK mk = p.mk;
+
+  // shared memory: [magnitude masks: uint16 [K], or uint8 [K]] [selected offsets, uint16 [GK]]
+  // [their places in the image, uint16 [GK] (merged operand only)] then per group
+  // [row slot][image, K bytes (merged operand only)][2 x 32 exchange words][2 next-row words][mbarrier]
+  const size_t mask_bytes = MASK8 ? (size_t)K : (size_t)K * 2;
+  const size_t jt_bytes = ((size_t)GK * 2 + 15) & ~(size_t)15;
+  const size_t row_bytes = (size_t)K * 2;
+  uint8_t* hmask = smem_enc;
+  uint16_t* jt = reinterpret_cast<uint16_t*>(smem_enc + mask_bytes);
+  uint16_t* jimg = reinterpret_cast<uint16_t*>(smem_enc + mask_bytes + jt_bytes);
+  uint8_t* gbase = smem_enc + mask_bytes + jt_bytes * (want_a8 ? 2 : 1) + (size_t)grp * p.group_stride;
+  uint8_t* img = gbase + row_bytes;
+  uint32_t* exch = reinterpret_cast<uint32_t*>(img + (want_a8 ? (size_t)K : 0));
+  volatile int* nexti = reinterpret_cast<volatile int*>(exch + 64);
+  const uint32_t bar0 = smem_u32(exch + 66);
+  __shared__ int abort_flag_s;
+  volatile int* abort_flag = &abort_flag_s;
+
+  // A block owns the rows blockIdx.x + i * gridDim.x; its groups take the next i from a shared
+  // counter whenever they have released their slot, so that no group idles while rows are left.
+  __shared__ int next_row_s;
+  if (threadIdx.x == 0) {
+    abort_flag_s = 0;
+    next_row_s = ngroups;
+  }
+  // The first rows are asked for as early as possible, but after the positions: issued before
+  // them, the grid's first 19 MB of rows would keep the tables waiting.  So every thread first
+  // issues the loads of (up to PQ of) its positions, the block meets, and then the rows go out
+  // while the tables are built.  The rows of the second round are asked into L2 at once: memory
+  // keeps streaming while the first round is being worked on.
+  constexpr int PQ = 4;
+  int pj[PQ];
+#pragma unroll
+  for (int i = 0; i < PQ; ++i) {
+    const int t = threadIdx.x + i * NT;
+    pj[i] = t < GK ? (int)p.positions[t] : 0;
+  }
+  int64_t m = (int64_t)blockIdx.x + (int64_t)grp * gridDim.x;
+  const uint8_t* slot = gbase;
+  const uint16_t* srow = reinterpret_cast<const uint16_t*>(slot);
+  if (glane == 0) {
+    mbar_init(bar0, 1);
+    fence_mbar_init();
+  }
+  __syncthreads();
+  if (glane == 0 && m < p.M) {
+    bulk_copy_g2s(smem_u32(slot), p.X + m * K, (uint32_t)row_bytes, bar0);
+    const int64_t m2 = m + (int64_t)ngroups * gridDim.x;
+    if (m2 < p.M) asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(p.X + m2 * K), "r"((uint32_t)row_bytes) : "memory");
+  }
+  if (MASK8) {
+    for (int i = threadIdx.x; i < K / 4; i += NT) reinterpret_cast<uint32_t*>(hmask)[i] = 0xFFFFFFFFu;
+  } else {
+    for (int i = threadIdx.x; i < K / 2; i += NT) reinterpret_cast<uint32_t*>(hmask)[i] = 0x7FFF7FFFu;
+  }
+  if (want_a8)
+    for (int i = glane; i < K / 4; i += gsize) reinterpret_cast<uint32_t*>(img)[i] = 0u;
+  __syncthreads();
+  for (int t = threadIdx.x, i = 0; t < GK; t += NT, ++i) {
+    int pos = 0;
+    if (i < PQ) {
+#pragma unroll
+      for (int u = 0; u < PQ; ++u)
+        if (u == i) pos = pj[u];
+    } else {
+      pos = p.positions[t];
+    }
+    const int j = (t / k) * p.b + pos;
+    jt[t] = (uint16_t)j;
+    if (MASK8) hmask[j] = 0;
+    else reinterpret_cast<uint16_t*>(hmask)[j] = 0;
+    if (want_a8) jimg[t] = (uint16_t)((j & ~7) | ((j & 1) << 2) | ((j & 7) >> 1));
+  }
+  __syncthreads();
+
+  const int nquads = GK / 4;
+  uint32_t parity = 0, flip = 0;
+  while (m < p.M) {
+    const bool landed = __all_sync(0xffffffffu, mbar_wait_park(bar0, parity, abort_flag));
+    parity ^= 1u;
+
+    uint4 v[NCL];
+    uint32_t r2 = 0, smax = 0;
+    if (landed) {
+      const uint4* src = reinterpret_cast<const uint4*>(slot) + slice * S8 + lane;
+#pragma unroll
+      for (int c = 0; c < NCL; ++c) v[c] = src[c * 32];
+      // selected places become (signed) zeros; the maximum of what is left
+#pragma unroll
+      for (int c = 0; c < NCL; ++c) {
+        uint4 q;
+        if (MASK8) {
+          const uint2 q8 = reinterpret_cast<const uint2*>(hmask)[slice * S8 + c * 32 + lane];
+          q.x = __byte_perm(q8.x, 0, 0x1100) | 0x80008000u;
+          q.y = __byte_perm(q8.x, 0, 0x3322) | 0x80008000u;
+          q.z = __byte_perm(q8.y, 0, 0x1100) | 0x80008000u;
+          q.w = __byte_perm(q8.y, 0, 0x3322) | 0x80008000u;
+          v[c].x &= q.x;
+          v[c].y &= q.y;
+          v[c].z &= q.z;
+          v[c].w &= q.w;
+        } else {
+          q = reinterpret_cast<const uint4*>(hmask)[slice * S8 + c * 32 + lane];
+          v[c].x &= q.x | 0x80008000u;
+          v[c].y &= q.y | 0x80008000u;
+          v[c].z &= q.z | 0x80008000u;
+          v[c].w &= q.w | 0x80008000u;
+        }
+        r2 = max2(r2, max2(max2(abs2(v[c].x), abs2(v[c].y)), max2(abs2(v[c].z), abs2(v[c].w))));
+      }
+      // largest selected magnitude, through the offset table
+      for (int q4 = glane; q4 < nquads; q4 += gsize) {
+        const uint2 jj = *reinterpret_cast<const uint2*>(jt + 4 * q4);
+        const uint32_t a = srow[jj.x & 0xFFFFu], b = srow[jj.x >> 16], c = srow[jj.y & 0xFFFFu], d = srow[jj.y >> 16];
+        smax = max(max(smax, a & 0x7FFFu), max(max(b & 0x7FFFu, c & 0x7FFFu), d & 0x7FFFu));
+      }
+    }
+    uint32_t rmax_bits = __reduce_max_sync(0xffffffffu, max(r2 & 0xFFFFu, r2 >> 16));
+    uint32_t smax_bits = __reduce_max_sync(0xffffffffu, smax);
+    if (!landed) smax_bits = 0xFFFFFFFFu;  // tells the whole group to stop together
+    if (rw > 1) {
+      uint32_t* ex = exch + flip * 32;
+      if (lane == 0) {
+        ex[slice] = smax_bits;
+        ex[16 + slice] = rmax_bits;
+      }
+      group_sync(rw, grp);
+      smax_bits = rmax_bits = 0;
+      for (int w = 0; w < rw; ++w) {
+        smax_bits = max(smax_bits, ex[w]);
+        rmax_bits = max(rmax_bits, ex[16 + w]);
+      }
+    }
+    if (smax_bits == 0xFFFFFFFFu) break;
+    const uint32_t amax_bits = INDEP ? smax_bits : max(smax_bits, rmax_bits);
+    const RowScale rs = INDEP ? row_scale_indep(amax_bits, rmax_bits) : row_scale_warp(amax_bits, rmax_bits, lane);
+    if (glane == 0) {
+      p.s_hi[m] = rs.s_hi;
+      p.s_lo[m] = rs.s_lo;
+      p.shift[m] = (uint8_t)rs.e;
+    }
+
+    // sparse component: INT8 codes of the selected values, four per lane and step
+    {
+      int8_t* vdst = p.vals + (size_t)m * GK;
+#pragma unroll 2
+      for (int q4 = glane; q4 < nquads; q4 += gsize) {
+        const uint2 jj = *reinterpret_cast<const uint2*>(jt + 4 * q4);
+        const uint32_t w[4] = {srow[jj.x & 0xFFFFu], srow[jj.x >> 16], srow[jj.y & 0xFFFFu], srow[jj.y >> 16]};
+        uint32_t o = 0;
+#pragma unroll
+        for (int q = 0; q < 4; ++q)
+          o |= (__float_as_uint(__fmaf_rn(__uint_as_float(w[q] << 16), rs.inv, kMagic)) & 0xFFu) << (8 * q);
+        *reinterpret_cast<uint32_t*>(vdst + 4 * q4) = o;
+        if (want_a8) {
+          const uint2 ji = *reinterpret_cast<const uint2*>(jimg + 4 * q4);
+          img[ji.x & 0xFFFFu] = (uint8_t)o;
+          img[ji.x >> 16] = (uint8_t)(o >> 8);
+          img[ji.y & 0xFFFFu] = (uint8_t)(o >> 16);
+          img[ji.y >> 16] = (uint8_t)(o >> 24);
+        }
+      }
+    }
+    // every lane of the group is done with the slot (and the image holds this row's codes); the
+    // slot is refilled by the async proxy: order this group's generic accesses before it
+    if (glane == 0) nexti[flip] = atomicAdd(&next_row_s, 1);
+    fence_proxy_async_smem();
+    group_sync(rw, grp);
+    const int64_t m_this = m;
+    m = (int64_t)blockIdx.x + (int64_t)nexti[flip] * gridDim.x;
+    flip ^= 1u;
+    if (glane == 0 && m < p.M) bulk_copy_g2s(smem_u32(slot), p.X + m * K, (uint32_t)row_bytes, bar0);
+
+    // dense component: INT4 codes of the registers, one 32-bit word per chunk
+    uint32_t* dst = reinterpret_cast<uint32_t*>(p.dq4 + (size_t)m_this * (K / 2)) + slice * S8 + lane;
+    const float cq = rs.inv_lo;
+    if (rs.clamp) {
+      // Codes beyond +-7 are possible: limit the inputs instead of the codes (see dense_sweep)
+      const uint32_t xl = __float_as_uint(__fdiv_rd(7.0f, cq)) >> 16;
+      const uint32_t hi2 = xl | (xl << 16), lo2 = hi2 | 0x80008000u;
+#pragma unroll
+      for (int c = 0; c < NCL; ++c) {
+        v[c].x = max2(min2(v[c].x, hi2), lo2);
+        v[c].y = max2(min2(v[c].y, hi2), lo2);
+        v[c].z = max2(min2(v[c].z, hi2), lo2);
+        v[c].w = max2(min2(v[c].w, hi2), lo2);
+      }
+    }
+    const float2 cc = make_float2(cq, cq), mm = make_float2(kMagic + 8.0f, kMagic + 8.0f);
+    if (want_a8) {
+      // Codes carry an offset of 8 (u = code + 8 in 1..15 in the low bits of 0x4B400000 + u).
+      // The four even and the four odd ones are summed into bytes by multiply-adds; their
+      // constant parts come off in the last step of each use:
+      //   dq4 word  = (ev + 16 * od - 0x3F400000) ^ 0x88888888
+      //   merged    = ev * 2^e + [0x80808080 - (0x08080808 + 0x8B400000) * 2^e]   (code * 2^e + 128
+      //               per byte, no carries: u * 2^e <= 240), XOR the image's bytes (0 where nothing
+      //               is selected, the INT8 code at a selected place, whose dense byte is 0x80)
+      uint32_t* aw = reinterpret_cast<uint32_t*>(p.a8 + (size_t)m_this * K) + ((slice * S8 + lane) >> 2) * 8 + (lane & 3);
+      const uint2* iw = reinterpret_cast<const uint2*>(img) + slice * S8 + lane;
+      const uint32_t pw = 1u << rs.e;
+      const uint32_t ce = 0x80808080u - (0x08080808u + 0x8B400000u) * pw;
+#pragma unroll
+      for (int c = 0; c < NCL; ++c) {
+        const uint32_t w[4] = {v[c].x, v[c].y, v[c].z, v[c].w};
+        uint32_t u[8];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          const float2 a = make_float2(__uint_as_float(imad(w[q], mk.k65536, 0u)), __uint_as_float(w[q] & 0xFFFF0000u));
+          const float2 d = __ffma2_rn(a, cc, mm);
+          u[2 * q] = __float_as_uint(d.x);
+          u[2 * q + 1] = __float_as_uint(d.y);
+        }
+        const uint32_t ev = imad(imad(u[6], mk.k256, u[4]), mk.k65536, imad(u[2], mk.k256, u[0]));
+        const uint32_t od = imad(imad(u[7], mk.k256, u[5]), mk.k65536, imad(u[3], mk.k256, u[1]));
+        const uint2 im = iw[c * 32];
+        dst[c * 32] = imad(imad(od, mk.k16, ev), mk.one, 0u - 0x3F400000u) ^ 0x88888888u;
+        aw[c * 64] = imad(ev, pw, ce) ^ im.x;
+        aw[c * 64 + 4] = imad(od, pw, ce) ^ im.y;
+      }
+    } else {
+#pragma unroll
+      for (int c = 0; c < NCL; ++c) {
+        const uint32_t w[4] = {v[c].x, v[c].y, v[c].z, v[c].w};
+        uint32_t u[8];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          const float2 a = make_float2(__uint_as_float(imad(w[q], mk.k65536, 0u)), __uint_as_float(w[q] & 0xFFFF0000u));
+          const float2 d = __ffma2_rn(a, cc, mm);
+          u[2 * q] = __float_as_uint(d.x);
+          u[2 * q + 1] = __float_as_uint(d.y);
+        }
+        const uint32_t t03 = imad(imad(u[3], mk.k16, u[2]), mk.k256, imad(u[1], mk.k16, u[0]));
+        const uint32_t t47 = imad(imad(u[7], mk.k16, u[6]), mk.k256, imad(u[5], mk.k16, u[4]));
+        dst[c * 32] = imad(imad(t47, mk.k65536, t03), mk.one, 0u - 0x3F400000u) ^ 0x88888888u;
+      }
+    }
+  }
+  if (*abort_flag && glane == 0) atomicExch(p.status, (int)SQ_ERR_TIMEOUT);
+}
+
+// ------------------------------------------------------------------------------------------------
 // Plain kernel for any (b, k): one block per token row, the row staged in shared memory.
 //   phase 1  load the row, row maximum -> inv = 127/amax, s_hi = amax/127
 //   phase 2  positions: dynamic = rank every element of a bank by (magnitude, then lower
@@ -1218,6 +1494,53 @@ cudaError_t launch_static_regs_as(EncodeParams p, int rw, cudaStream_t st) {
   return cudaGetLastError();
 }
 
+// Ring kernel: `rw` warps per row, 16 / rw groups per block, one slot per group.
+template <int NCL, bool INDEP, bool MASK8>
+cudaError_t launch_static_ring_as(EncodeParams p, int rw, cudaStream_t st) {
+  constexpr int NT = 512;
+  const int GK = (p.K / p.b) * p.k;
+  const int ngroups = (NT / 32) / rw;
+  const bool a8 = !INDEP && p.a8 != nullptr;
+  const size_t mask_bytes = MASK8 ? (size_t)p.K : (size_t)p.K * 2;
+  const size_t jt_bytes = ((size_t)GK * 2 + 15) & ~(size_t)15;
+  const size_t per_group = ((size_t)p.K * 2 + (a8 ? (size_t)p.K : 0) + 256 + 16 + 127) & ~(size_t)127;
+  const size_t smem = mask_bytes + jt_bytes * (a8 ? 2 : 1) + per_group * ngroups;
+  if (smem > 226 * 1024) return cudaErrorNotSupported;
+  p.rw = rw;
+  p.group_stride = (int)per_group;
+  int dev = 0, sms = 0;
+  cudaError_t err = device_and_sms(&dev, &sms);
+  if (err != cudaSuccess) return err;
+  SQ_ENSURE_SMEM((encode_static_ring_kernel<NCL, NT, INDEP, MASK8>), dev, smem);
+  const int64_t blocks = p.M < sms ? p.M : sms;
+  encode_static_ring_kernel<NCL, NT, INDEP, MASK8><<<(unsigned)blocks, NT, smem, st>>>(p);
+  return cudaGetLastError();
+}
+
+// Picks the ring kernel's shape: the fewest warps per row whose slice is an instantiated size
+// (the per-row work that does not shrink with the slice -- scales, barriers -- is then spread over
+// the most elements, and the most rows are in flight); half-word masks if the tables and slots
+// fit, else byte masks.
+template <bool INDEP>
+cudaError_t launch_static_ring(const EncodeParams& p, cudaStream_t st) {
+  if (p.K % 256 != 0 || p.K > 65535 || (reinterpret_cast<uintptr_t>(p.X) & 15) != 0) return cudaErrorNotSupported;
+  for (int mask8 = 0; mask8 < 2; ++mask8) {
+    for (int rw = 1; rw <= 8; rw *= 2) {
+      if ((p.K / 256) % rw != 0) continue;
+      const int ncl = p.K / 256 / rw;
+      cudaError_t err = cudaErrorNotSupported;
+#define SQ_RING(NCL_)                                                                   \
+  if (ncl == NCL_)                                                                      \
+    err = mask8 ? launch_static_ring_as<NCL_, INDEP, true>(p, rw, st)                   \
+                : launch_static_ring_as<NCL_, INDEP, false>(p, rw, st);
+      SQ_RING(8) SQ_RING(12) SQ_RING(14) SQ_RING(16)
+#undef SQ_RING
+      if (err != cudaErrorNotSupported) return err;
+    }
+  }
+  return cudaErrorNotSupported;
+}
+
 // cudaErrorNotSupported = this shape is left to the shared-memory kernel.  Slices of at most
 // 16 chunks per lane keep 16 warps resident (measured faster than fewer warps holding more).
 template <bool INDEP>
@@ -1273,18 +1596,23 @@ cudaError_t launch_encode(int b, int k, bool is_static, bool indep, const uint16
   p.nbuf = 1;
   p.rw = 1;
   p.group_stride = 0;
-  p.mk = MulK{0xFFFFFFFFu, 2u, 32u, 256u, 65536u, 1u << 24};
+  p.mk = MulK{0xFFFFFFFFu, 2u, 32u, 256u, 65536u, 1u << 24, 16u, 1u};
   if (is_static && indep) {
     // independent scales: the register kernel, or the plain one for row lengths it does not take
-    const cudaError_t err = launch_static_regs<true>(p, st);
+    cudaError_t err = launch_static_ring<true>(p, st);
+    if (err != cudaErrorNotSupported) return err;
+    err = launch_static_regs<true>(p, st);
     if (err != cudaErrorNotSupported) return err;
     if (b == 32) return launch_generic<32>(k, true, true, X, M, K, positions, out, st);
     if (b == 64) return launch_generic<64>(k, true, true, X, M, K, positions, out, st);
     return launch_generic<128>(k, true, true, X, M, K, positions, out, st);
   }
   if (is_static) {
-    p.a8 = a8;  // only the register kernel writes the merged operand
-    cudaError_t err = launch_static_regs<false>(p, st);
+    p.a8 = a8;  // only the ring and register kernels write the merged operand
+    cudaError_t err = std::getenv("SQ_ENCODE_RING_OFF") ? cudaErrorNotSupported : launch_static_ring<false>(p, st);
+    if (err == cudaSuccess && a8 != nullptr && a8_written != nullptr) *a8_written = true;
+    if (err != cudaErrorNotSupported) return err;
+    err = launch_static_regs<false>(p, st);
     if (err == cudaSuccess && a8 != nullptr && a8_written != nullptr) *a8_written = true;
     if (err != cudaErrorNotSupported) return err;
     p.a8 = nullptr;

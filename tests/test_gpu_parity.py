@@ -273,15 +273,15 @@ def test_several_tiles_per_sm(M, N, K, b, k, static):
         assert_bf16_close(out[torch.from_numpy(rows).cuda()], ref32)
 
 
-# ----------------------------------------------------------------------------- encode: rows held in registers
+# ----------------------------------------------------------------------------- encode: static positions, staged rows / rows in registers
 
 @pytest.mark.parametrize("K,b,k", [
     (2048, 64, 8), (4096, 32, 4), (4096, 128, 64), (6144, 64, 4), (7168, 128, 16),
     (12288, 64, 8), (14336, 64, 8), (16384, 32, 8), (24576, 128, 16), (32768, 64, 16),
 ])
 def test_static_encode_row_slices_in_registers(K, b, k):
-    """Static positions with rows of 1, 2 or 4 warp slices, a ragged row count, and rows that
-    are all zero, all ties, one-hot, and clamping."""
+    """Static positions with rows of 1, 2, 4 or 8 warp slices (every slice size the kernels are
+    built for), a ragged row count, and rows that are all zero, all ties, one-hot, and clamping."""
     M = 333
     fmt = sq.make_format(b, k, True)
     X = gen.activations(M, K, seed=K + k, outlier_fraction=0.01, outlier_scale=30.0, device="cpu").float()
@@ -553,8 +553,10 @@ def merged_operand_from_oracle(b, k, enc_ref, pos_ref):
 
 
 @pytest.mark.parametrize("M,N,K,b,k,static", [
-    (300, 1024, 2048, 64, 8, True),      # register kernel, one warp per row
-    (257, 1280, 8192, 64, 8, True),      # register kernel, rows split over warps
+    (300, 1024, 2048, 64, 8, True),      # rows staged in shared-memory slots, one warp per row
+    (257, 1280, 8192, 64, 8, True),      # ... rows split over two warps
+    (40, 256, 28672, 128, 16, True),     # ... long rows: eight warps per row, byte masks
+    (20, 256, 32768, 64, 8, True),       # slots, tables and image do not fit: the register kernel
     (200, 1024, 4096, 128, 16, True),
     (130, 1024, 3072, 32, 4, True),
     (140, 1024, 2048, 64, 6, True),      # k not a multiple of four: byte-wise sparse path
