@@ -128,28 +128,60 @@ __global__ void __launch_bounds__(256) sqw_act_kernel(const uint16_t* __restrict
 }
 
 namespace {
+// Byte `sel & 7` of the pair (lo, hi), sign-extended: selector nibbles 1-3 carry bit 3, which makes
+// the permute replicate the chosen byte's sign bit.
+__device__ __forceinline__ int pick_s8(uint32_t lo, uint32_t hi, uint32_t sel) {
+  int d;
+  asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(lo), "r"(hi), "r"(sel));
+  return d;
+}
 constexpr int kWsqWarps = 8;
 constexpr int kWsqCh = 2;  // output channels a warp works on at a time
 }
 
 // MT: tokens (1..4).  Shared memory: the reordered INT8 activations [MT][K].
+//
+// A lane owns whole banks, so it meets exactly k masked places per bank and channel and every lane
+// of a warp runs the same number of steps.  Per bank and channel:
+//   dense part   three operations per word mark the nibbles that hold 1000, one more turns them
+//                into code 0, and the nibbles go as bytes 16 * code into packed 4-way dot products.
+//   mask         five more operations per word squeeze the
+//                eight marks into a byte (two shifts, one logic operation, one multiply whose
+//                partial products do not overlap), and byte permutes string the bytes of four
+//                words together: one bit per weight, in position order.
+//   sparse part  k steps: lowest set bit -> place, the activation of that place from shared
+//                memory, one multiply-add with the compact value (its slot is the step number, so
+//                it is picked out of the registers with constant shifts).
 template <int B, int MT>
-__global__ void __launch_bounds__(kWsqWarps * 32) sqw_gemm_kernel(int k, const int8_t* __restrict__ xq,
-                                                                  const float* __restrict__ s_x,
-                                                                  const uint8_t* __restrict__ wq4,
-                                                                  const int8_t* __restrict__ w_hi,
-                                                                  const float* __restrict__ s_high,
-                                                                  const float* __restrict__ s_low, int M, int N, int K,
-                                                                  uint16_t* __restrict__ out, int32_t* __restrict__ acc_out) {
+__global__ void __launch_bounds__(kWsqWarps * 32, (B == 128 || MT == 4) ? 2 : 3) sqw_gemm_kernel(int k, const int8_t* __restrict__ xq,
+                                                                     const float* __restrict__ s_x,
+                                                                     const uint8_t* __restrict__ wq4,
+                                                                     const int8_t* __restrict__ w_hi,
+                                                                     const float* __restrict__ s_high,
+                                                                     const float* __restrict__ s_low, int M, int N, int K,
+                                                                     uint16_t* __restrict__ out, int32_t* __restrict__ acc_out) {
   extern __shared__ __align__(16) int8_t sx[];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int G = K / B;
-  constexpr int WPB = B / 8;  // 32-bit words of nibbles per bank
+  constexpr int WPB = B / 8;   // 32-bit words of nibbles per bank
+  constexpr int NM = B / 32;   // 32-bit mask registers per bank (one bit per weight)
+  constexpr int KW = B / 8;    // 32-bit words of compact values per bank, at most (k <= B / 2)
+  // Shared-memory image of the activations: bank by bank (the unit a lane owns), inside a bank
+  // word by word (8 elements), inside a word token by token, so that one 16-byte read serves two
+  // tokens; a bank is padded so that the lanes of a warp, which read the same word of 32
+  // consecutive banks, fall on different memory banks.
+  constexpr int kPad = MT == 1 ? 8 : 16;
+  constexpr int kBankStride = B * MT + kPad;
   for (int i = tid; i < MT * (K / 16); i += kWsqWarps * 32) {
     const int m = i / (K / 16), c = i % (K / 16);
-    reinterpret_cast<uint4*>(sx)[i] = m < M ? __ldg(reinterpret_cast<const uint4*>(xq + (size_t)m * K) + c) : make_uint4(0, 0, 0, 0);
+    const uint4 v = m < M ? __ldg(reinterpret_cast<const uint4*>(xq + (size_t)m * K) + c) : make_uint4(0, 0, 0, 0);
+    const int j = 16 * c, g = j / B, w = (j % B) >> 3;  // elements j .. j + 15: words w and w + 1 of bank g
+    int8_t* dst = sx + (size_t)g * kBankStride + w * (8 * MT) + m * 8;
+    *reinterpret_cast<uint2*>(dst) = make_uint2(v.x, v.y);
+    *reinterpret_cast<uint2*>(dst + 8 * MT) = make_uint2(v.z, v.w);
   }
   __syncthreads();
+  const bool words_ok = (k & 3) == 0;  // the compact values of a bank start on a 32-bit boundary
   const int pairs = (N + kWsqCh - 1) / kWsqCh;
   for (int pr = blockIdx.x * kWsqWarps + warp; pr < pairs; pr += gridDim.x * kWsqWarps) {
     int lo[kWsqCh][MT], hi[kWsqCh][MT];
@@ -158,47 +190,100 @@ __global__ void __launch_bounds__(kWsqWarps * 32) sqw_gemm_kernel(int k, const i
 #pragma unroll
       for (int m = 0; m < MT; ++m) lo[c][m] = hi[c][m] = 0;
     for (int g = lane; g < G; g += 32) {
-      // the bank's activations, reused for both channels
-      const int8_t* xb = sx + g * B;
+      const int8_t* xb = sx + (size_t)g * kBankStride;  // the bank's activations, reused for both channels
+      uint32_t words[kWsqCh][WPB], hv[kWsqCh][KW];
 #pragma unroll
       for (int c = 0; c < kWsqCh; ++c) {
         const int n = min(pr * kWsqCh + c, N - 1);
-        const uint32_t* wp = reinterpret_cast<const uint32_t*>(wq4 + (size_t)n * (K / 2) + g * (B / 2));
-        const int8_t* hp = w_hi + ((size_t)n * G + g) * k;
-        int slot = 0;
-        uint32_t words[WPB];
+        const uint4* wp = reinterpret_cast<const uint4*>(wq4 + (size_t)n * (K / 2) + g * (B / 2));
 #pragma unroll
         for (int w4 = 0; w4 < WPB / 4; ++w4) {
-          const uint4 v = __ldg(reinterpret_cast<const uint4*>(wp) + w4);
-          words[4 * w4] = v.x;
-          words[4 * w4 + 1] = v.y;
-          words[4 * w4 + 2] = v.z;
-          words[4 * w4 + 3] = v.w;
+          const uint4 v = __ldg(wp + w4);
+          words[c][4 * w4] = v.x;
+          words[c][4 * w4 + 1] = v.y;
+          words[c][4 * w4 + 2] = v.z;
+          words[c][4 * w4 + 3] = v.w;
         }
+        const int8_t* hp = w_hi + ((size_t)n * G + g) * k;
+        if (words_ok) {
 #pragma unroll
-        for (int w = 0; w < WPB; ++w) {
-          const uint32_t word = words[w];
-          // places holding the pattern 1000: bit 3 set and the three low bits clear
-          const uint32_t low3 = word & 0x77777777u;
-          uint32_t flags = word & 0x88888888u & ~((low3 + 0x77777777u) & 0x88888888u);
-          const uint32_t clean = word & ~((flags >> 3) * 15u);
-          const int ev = (int)((clean << 4) & 0xF0F0F0F0u), od = (int)(clean & 0xF0F0F0F0u);  // 16 * code, bytewise
-          // the compact values of the bank belong to its masked places in position order: they are
-          // scattered into two words laid out like the dense ones, so that the sparse product is two
-          // more packed dot products against the activations already in registers
-          uint32_t hev = 0, hod = 0;
-          while (flags) {
-            const int nibble = (__ffs((int)flags) - 1) >> 2;
-            flags &= flags - 1;
-            const uint32_t wv = (uint32_t)(uint8_t)hp[slot++] << (8 * (nibble >> 1));
-            if (nibble & 1) hod |= wv;
-            else hev |= wv;
+          for (int q = 0; q < KW; ++q) hv[c][q] = 4 * q < k ? __ldg(reinterpret_cast<const uint32_t*>(hp) + q) : 0u;
+        } else {
+#pragma unroll
+          for (int q = 0; q < KW; ++q) {
+            uint32_t v = 0;
+#pragma unroll
+            for (int t = 0; t < 4; ++t)
+              if (4 * q + t < k) v |= (uint32_t)(uint8_t)__ldg(hp + 4 * q + t) << (8 * t);
+            hv[c][q] = v;
           }
+        }
+      }
 #pragma unroll
-          for (int m = 0; m < MT; ++m) {
-            const int2 xv = *reinterpret_cast<const int2*>(xb + (size_t)m * K + 8 * w);
-            lo[c][m] = __dp4a(ev, xv.x, __dp4a(od, xv.y, lo[c][m]));
-            hi[c][m] = __dp4a((int)hev, xv.x, __dp4a((int)hod, xv.y, hi[c][m]));
+      for (int c = 0; c < kWsqCh; ++c) {
+        uint32_t mreg[NM];
+#pragma unroll
+        for (int r = 0; r < NM; ++r) {
+          uint32_t sq[4];
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            const uint32_t word = words[c][4 * r + j];
+            // nibbles holding 1000: bit 3 set and the three low bits clear -> a mark at bit 4i + 3;
+            // flipping the marked bits turns the mask code into code 0
+            const uint32_t t = (word & 0x77777777u) + 0x77777777u;
+            const uint32_t f3 = word & ~t & 0x88888888u;
+            const uint32_t clean = word ^ f3;
+            const int ev = (int)((clean << 4) & 0xF0F0F0F0u), od = (int)(clean & 0xF0F0F0F0u);  // 16 * code, bytewise
+            const int8_t* xw = xb + (4 * r + j) * (8 * MT);
+            if constexpr (MT == 1) {
+              const int2 xv = *reinterpret_cast<const int2*>(xw);
+              lo[c][0] = __dp4a(ev, xv.x, __dp4a(od, xv.y, lo[c][0]));
+            } else {
+#pragma unroll
+              for (int m2 = 0; m2 < MT / 2; ++m2) {
+                const int4 xv = *reinterpret_cast<const int4*>(xw + 16 * m2);
+                lo[c][2 * m2] = __dp4a(ev, xv.x, __dp4a(od, xv.y, lo[c][2 * m2]));
+                lo[c][2 * m2 + 1] = __dp4a(ev, xv.z, __dp4a(od, xv.w, lo[c][2 * m2 + 1]));
+              }
+            }
+            // marks of a byte's two nibbles side by side, then the four pairs into the top byte
+            const uint32_t y = ((f3 >> 3) | (f3 >> 6)) & 0x03030303u;
+            sq[j] = y * 0x01041040u;
+          }
+          mreg[r] = __byte_perm(__byte_perm(sq[0], sq[1], 0x0073), __byte_perm(sq[2], sq[3], 0x0073), 0x5410);
+        }
+        // sparse part: the k masked places in position order
+#pragma unroll
+        for (int s = 0; s < B / 2; ++s) {
+          if ((s & 3) == 0 && s >= k) break;  // (uniform: whole words of compact values are skipped at once)
+          if (s < k) {
+            uint32_t cur = mreg[0];
+            int base = 0;
+#pragma unroll
+            for (int r = 1; r < NM; ++r)
+              if (cur == 0u) {
+                cur = mreg[r];
+                base = 32 * r;
+              }
+            const int pl = base + __ffs((int)cur) - 1;
+#pragma unroll
+            for (int r = 0; r < NM; ++r)
+              if (base == 32 * r) mreg[r] &= mreg[r] - 1u;
+            const int v = (int)(hv[c][s >> 2] << (24 - 8 * (s & 3))) >> 24;
+            const int8_t* xw = xb + (pl >> 3) * (8 * MT);
+            const int rb = ((pl & 1) << 2) | ((pl & 7) >> 1);  // byte of the place inside its word
+            if constexpr (MT == 1) {
+              hi[c][0] += v * (int)xw[rb];
+            } else {
+              // both tokens of a 16-byte read; the byte is picked (and sign-extended) by a byte permute
+              const uint32_t sel = (uint32_t)rb * 0x1111u + 0x8880u;
+#pragma unroll
+              for (int m2 = 0; m2 < MT / 2; ++m2) {
+                const uint4 xv = *reinterpret_cast<const uint4*>(xw + 16 * m2);
+                hi[c][2 * m2] += v * pick_s8(xv.x, xv.y, sel);
+                hi[c][2 * m2 + 1] += v * pick_s8(xv.z, xv.w, sel);
+              }
+            }
           }
         }
       }
@@ -280,7 +365,7 @@ cudaError_t launch_wsq_gemm(int b, int k, const int8_t* xq, const float* s_x, co
                             int32_t* acc_out, cudaStream_t st) {
   if (M < 1 || M > 4) return cudaErrorNotSupported;
   const int MT = M <= 1 ? 1 : (M <= 2 ? 2 : 4);
-  const size_t smem = (size_t)MT * K;
+  const size_t smem = (size_t)MT * K + (size_t)(K / b) * (MT == 1 ? 8 : 16);
   if (smem > 200 * 1024) return cudaErrorNotSupported;
   int dev = 0, sms = 0;
   cudaError_t err = cudaGetDevice(&dev);
@@ -289,7 +374,7 @@ cudaError_t launch_wsq_gemm(int b, int k, const int8_t* xq, const float* s_x, co
   if (err != cudaSuccess) return err;
   const int64_t pairs = (N + kWsqCh - 1) / kWsqCh;
   int64_t blocks = (pairs + kWsqWarps - 1) / kWsqWarps;
-  if (blocks > 2 * (int64_t)sms) blocks = 2 * (int64_t)sms;
+  if (blocks > 3 * (int64_t)sms) blocks = 3 * (int64_t)sms;
 #define SQ_WGEMM(BB, MM)                                                                                           \
   do {                                                                                                             \
     static std::atomic<size_t> limit[64];                                                                          \
