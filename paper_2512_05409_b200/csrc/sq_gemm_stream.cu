@@ -10,20 +10,26 @@
 // packed weights) is a few dozen cycles of tensor work and the kernel streams weights.
 //
 // What a K step costs in this shape is not work but hand-over latency (wait for the tile, read,
-// widen, store, proxy fence, arrive: half a microsecond to a microsecond for one group of
-// threads, whatever the tile's size), so consecutive K steps are handled by DIFFERENT groups:
-//   warp 0      one thread streams the packed tiles of every K step (128 x 64 B of weights,
-//               16 x 64 B of activations, the step's sparse values and bank-local indices,
-//               16 x nb bytes each) into a ring by TMA
-//   warps 1-4   two groups of two warps; group g widens the weights (nibble -> 16 * code, signed)
-//               of steps g, g + 2, ... into a ring of three 8-bit stages in the layout the tensor
-//               core reads (K-major, 128-byte swizzle)
+// widen, store, fence, arrive: a few tenths of a microsecond for one group of threads, whatever
+// the tile's size), so consecutive K steps are handled by DIFFERENT groups; and what two CTAs on
+// one SM ran out of first was shared-memory bandwidth (a step's 8 KB of packed weights were
+// written by TMA, read, written again widened and read by the tensor core: 48 KB), so the widened
+// weights -- the MMA's 128-row operand -- now live in TENSOR memory and never pass through shared
+// memory a second time:
+//   warp 0      one thread streams the packed tiles (boxes of two K steps: 128 x 128 B of weights
+//               with the 128-byte swizzle, 16 x 128 B of activations, the steps' sparse values and
+//               bank-local indices) into a ring by TMA
+//   warps 1-4,  two groups of four warps; group g takes steps g, g + 2, ...  A thread owns one
+//   15-18       output channel (tensor-memory lane = quarter warp % 4, lane): it reads the channel's
+//               64 packed bytes of the step, widens them (nibble -> 16 * code, signed) and stores
+//               them with tcgen05.st into one of six 32-column stages of tensor memory
 //   warps 5-8   warp x widens the activation tile (nibble * 2^e + bias, unsigned, offset 128) of
-//               steps x, x + 4, ... into a ring of eight small stages of its own and merges the
-//               step's sparse INT8 entries into the bytes they belong to
-//   warp 9      one thread issues tcgen05.mma.kind::i8 (M = 128 channels, N = 16 tokens) when
-//               both operands of a step are ready and hands both stages back
-//   warps 10-13 read the accumulator (lane = channel) once the K walk is over
+//               steps x, x + 4, ... into a ring of eight small shared-memory stages of its own and
+//               merges the step's sparse INT8 entries into the bytes they belong to
+//   warps 9, 14 one thread each issues tcgen05.mma.kind::i8 (A from tensor memory, M = 128
+//               channels; B from shared memory, N = 16 tokens) for alternate steps, into an
+//               accumulator of its own, and frees both operands' stages with ONE commit per step
+//   warps 10-13 read the accumulators (lane = channel) once the K walk is over
 //   work item   (slab of 128 output channels, part of K).  The parts of a slab form one
 //               thread-block cluster and add their raw int32 partial sums through distributed
 //               shared memory; CTA r of the cluster finishes a share of the slab's channels
@@ -47,25 +53,28 @@ namespace {
 constexpr int SC = 128;        // output channels per slab = rows of the MMA = tensor-memory lanes
 constexpr int MT = 16;         // token columns of the accumulator
 constexpr int BK = 128;        // K elements per step = bytes per operand row
-constexpr int SUP = 1;         // K steps per packed stage (boxes of 4 steps, 256 bytes per row, with one CTA per SM
-                               // were measured slower than this with two CTAs per SM)
+constexpr int SUP = 2;         // K steps per packed stage: the TMA engine moves a tile row by row, and 128-byte rows cost it
+                               // half of what 64-byte rows do per byte (one step per stage left the weight warps waiting for data)
 constexpr int NPK = 4;         // packed stages in flight
-constexpr int NW = 3;          // widened weight stages
+constexpr int NW = 6;          // widened weight stages (in tensor memory)
 constexpr int NX = 8;          // widened activation stages
-constexpr int kWGroups = 2, kWGroupThreads = 64, kXWarps = 4;
-constexpr int kTmaWarp = 0, kFirstW = 1, kFirstX = 5, kMmaWarp = 9, kFirstEpi = 10, kMma2Warp = 14;
-constexpr int kThreadsS = 15 * 32;
-constexpr int kCtlS = 384 + 2 * SC * 4 + MT * 4;  // barriers, then the slab's constants for the finish
+constexpr int kWGroups = 2, kWGroupThreads = 128, kXWarps = 4;
+constexpr int kTmaWarp = 0, kFirstW = 1, kFirstX = 5, kMmaWarp = 9, kFirstEpi = 10, kMma2Warp = 14, kFirstW2 = 15;
+constexpr int kThreadsS = 19 * 32;
+constexpr int ND = 24;         // "step done" barriers: a common multiple of NW and NX
+constexpr int kCtlBars = 512;
+constexpr int kCtlS = kCtlBars + 2 * SC * 4 + MT * 4;  // barriers, then the slab's constants for the finish
 constexpr int kPitch = SUP * (BK / 2);     // bytes per packed row of a stage
 constexpr int kPackW = SC * kPitch;        // 32 KB
 constexpr int kPackX = MT * kPitch;        // 4 KB
 constexpr int kSide = MT * SUP * 64;       // sparse values / indices of a stage: up to 64 per row and step
 constexpr int kPackStage = kPackW + kPackX + 2 * kSide;
-constexpr int kStageW = SC * BK;           // 16 KB
+constexpr int kColsW = BK / 4;              // tensor-memory columns of a widened weight stage (128 lanes x 128 bytes)
+constexpr int kAccCols = 2 * MT;           // the two accumulators
 constexpr int kStageX = MT * BK;           // 2 KB
-constexpr int kSmemS = NW * kStageW + NX * kStageX + NPK * kPackStage + kCtlS;
-static_assert(kStageX % 1024 == 0 && kPackStage % 128 == 0, "stage alignment");
-static_assert(SC * MT * 4 <= NW * kStageW, "partial sums are parked in the weight ring");
+constexpr int kSmemS = NX * kStageX + NPK * kPackStage + kCtlS;
+static_assert(kStageX % 1024 == 0 && kPackStage % 1024 == 0 && (NX * kStageX) % 1024 == 0 && SUP <= 2, "stage alignment (swizzled weight tiles)");
+static_assert(SC * MT * 4 <= NPK * kPackStage, "partial sums are parked in the packed ring");
 
 struct StreamParams {
   const float* s_hi;
@@ -105,6 +114,24 @@ __device__ __forceinline__ void tma_2d(uint32_t dst, const CUtensorMap* map, int
       "l"(map), "r"(x), "r"(y), "r"(bar)
       : "memory");
 }
+// 32 lanes x 16 consecutive 32-bit columns: thread t of the warp writes lane (base lane + t).
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&v)[16]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};" ::"r"(taddr),
+      "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]), "r"(v[8]), "r"(v[9]),
+      "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15])
+      : "memory");
+}
+// D[tmem] (+)= A[tmem] * B[smem desc]: the 128-row operand is read from tensor memory (lane = row,
+// four 8-bit K elements per 32-bit column), the narrow one from shared memory.
+__device__ __forceinline__ void umma_i8_ta(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::i8 [%0], [%1], %2, %3, p;\n\t}" ::"r"(d_tmem),
+      "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
 __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&v)[16]) {
   asm volatile(
       "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
@@ -125,22 +152,22 @@ __global__ void __launch_bounds__(kThreadsS, 2)
     if (threadIdx.x == 0) atomicExch(p.status, (int)SQ_ERR_CUDA);
     return;  // (uniform over the cluster: every CTA sees the same offset of its dynamic block)
   }
-  uint8_t* sW = smem;                          // NW x [128 x 128] widened weights
-  uint8_t* sX = sW + NW * kStageW;             // NX x [16 x 128] widened (and merged) activations
+  uint8_t* sX = smem;                          // NX x [16 x 128] widened (and merged) activations
   uint8_t* sPack = sX + NX * kStageX;          // NPK x [W 128 x 64 | X 16 x 64 | vals 16 x 64 | idx 16 x 64]
   uint8_t* sCtl = sPack + NPK * kPackStage;
   const uint32_t bar_pfull = smem_u32(sCtl);         // NPK: packed stage landed
   const uint32_t bar_pempty = bar_pfull + 8 * NPK;   // NPK: packed stage read by its weight group and activation warp
   const uint32_t bar_wfull = bar_pempty + 8 * NPK;   // NW: weights widened
-  const uint32_t bar_wempty = bar_wfull + 8 * NW;    // NW: consumed by the MMAs
-  const uint32_t bar_xfull = bar_wempty + 8 * NW;    // NX: activations widened and merged
-  const uint32_t bar_xempty = bar_xfull + 8 * NX;    // NX: consumed by the MMAs
-  const uint32_t bar_tfull = bar_xempty + 8 * NX;    // accumulator complete
-  constexpr int kBars = 2 * NPK + 2 * NW + 2 * NX + 1;
+  const uint32_t bar_xfull = bar_wfull + 8 * NW;     // NX: activations widened and merged
+  const uint32_t bar_done = bar_xfull + 8 * NX;      // ND: the MMAs of step ks (barrier ks % ND) have read their operands:
+                                                     // ONE commit per step frees both the weight and the activation stage
+  const uint32_t bar_tfull = bar_done + 8 * ND;      // accumulator complete
+  constexpr int kBars = 2 * NPK + NW + NX + ND + 1;
+  static_assert(ND % NW == 0 && ND % NX == 0, "a step's barrier must not come round before its stages do");
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(sCtl + 8 * kBars);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(sCtl + 8 * kBars + 8);
-  static_assert(8 * kBars + 16 <= 384, "control block too small");
-  int32_t* s_cs = reinterpret_cast<int32_t*>(sCtl + 384);   // colsum of the slab's channels
+  static_assert(8 * kBars + 16 <= kCtlBars, "control block too small");
+  int32_t* s_cs = reinterpret_cast<int32_t*>(sCtl + kCtlBars);   // colsum of the slab's channels
   float* s_sw = reinterpret_cast<float*>(s_cs + SC);        // their weight scales
   float* s_sh = s_sw + SC;                                   // the tokens' scales
 
@@ -149,7 +176,8 @@ __global__ void __launch_bounds__(kThreadsS, 2)
   const int slab = (int)blockIdx.x / parts, part = (int)blockIdx.x % parts;  // part = rank in the cluster
   const int n0 = slab * SC;
   const int KS = p.KS, k0 = part * KS;
-  constexpr uint32_t kTmemCols = 32;
+  constexpr uint32_t kTmemCols = 256;  // 2 x 16 accumulator columns, then NW x 32 columns of widened weights
+  static_assert(kAccCols + NW * kColsW <= 256, "tensor-memory columns");
 
   if (tid == 0) {
     for (int s = 0; s < NPK; ++s) {
@@ -158,12 +186,11 @@ __global__ void __launch_bounds__(kThreadsS, 2)
     }
     for (int s = 0; s < NW; ++s) {
       mbar_init(bar_wfull + 8 * s, kWGroupThreads);
-      mbar_init(bar_wempty + 8 * s, 1);
     }
     for (int s = 0; s < NX; ++s) {
       mbar_init(bar_xfull + 8 * s, 32);
-      mbar_init(bar_xempty + 8 * s, 1);
     }
+    for (int s = 0; s < ND; ++s) mbar_init(bar_done + 8 * s, 1);
     mbar_init(bar_tfull, KS >= 2 ? 2 : 1);  // one arrival per issuing thread that has steps
     *abort_flag = 0;
     fence_mbar_init();
@@ -192,7 +219,7 @@ __global__ void __launch_bounds__(kThreadsS, 2)
         const int ps = su % NPK;
         // (a last stage that holds fewer than SUP steps of this part never completes its "empty"
         // barrier; nothing is loaded after it, so nothing waits for it)
-        if (!mbar_wait(bar_pempty + 8 * ps, ((su / NPK) & 1u) ^ 1u, abort_flag)) break;
+        if (!mbar_wait_park(bar_pempty + 8 * ps, ((su / NPK) & 1u) ^ 1u, abort_flag)) break;
         const uint32_t dst = smem_u32(sPack + ps * kPackStage), bar = bar_pfull + 8 * ps;
         const int kx = k0 + su * SUP;  // first K step of the stage; columns past K come back as zeros
         expect_tx(bar, bytes);
@@ -203,42 +230,51 @@ __global__ void __launch_bounds__(kThreadsS, 2)
       }
     }
     __syncwarp();
-  } else if (warp >= kFirstW && warp < kFirstX) {
+  } else if ((warp >= kFirstW && warp < kFirstX) || warp >= kFirstW2) {
     // =============================================================== weights: group g takes steps g, g + 2, ...
-    const int wt = tid - kFirstW * 32;            // 0..127
-    const int g = wt / kWGroupThreads, gt = wt % kWGroupThreads;
-    // thread -> (row % 16, packed 16-byte chunk): a quarter warp reads 128 contiguous packed bytes and
-    // its two stores land on eight different 16-byte chunks of the swizzled rows
-    const int r16 = gt >> 2, c = gt & 3;
-    const uint32_t sw_even = (uint32_t)(((2 * c) ^ (r16 & 7)) << 4);
+    // A thread owns one output channel (its tensor-memory lane: quarter warp % 4, lane): it reads the
+    // channel's 64 packed bytes of the step (the tile was laid down with the 64-byte swizzle, so the
+    // 16-byte reads of eight consecutive rows fall on different banks), widens them (nibble ->
+    // 16 * code, signed; [16 even | 16 odd] bytes per 32 elements, the activations' order) and
+    // stores them as the MMA's A operand in TENSOR memory: the 8-bit weights never pass through
+    // shared memory, whose bandwidth two CTAs per SM had used up.
+    const int g = warp >= kFirstW2 ? 1 : 0;
+    const int row = 32 * (warp & 3) + lane;
+    const uint32_t lane_base = (uint32_t)(32 * (warp & 3)) << 16;
     bool ok = true;
     for (int ks = g; ks < KS && ok; ks += kWGroups) {
       const int su = ks / SUP, ps = su % NPK, s = ks % NW;
       ok = mbar_wait_park(bar_pfull + 8 * ps, (su / NPK) & 1u, abort_flag);
       if (!ok) break;
-      const uint8_t* pk = sPack + ps * kPackStage + r16 * kPitch + (ks % SUP) * 64 + c * 16;
-      uint4 rw[8];
+      const uint8_t* pk = sPack + ps * kPackStage + row * kPitch;
+      const uint32_t sz = SUP == 1 ? (uint32_t)((row >> 1) & 3) : (uint32_t)(row & 7);  // 64- / 128-byte swizzle
+      const uint32_t c0 = (uint32_t)(ks % SUP) * 4u;
+      uint4 rw[4];
 #pragma unroll
-      for (int i = 0; i < 8; ++i) rw[i] = *reinterpret_cast<const uint4*>(pk + i * 16 * kPitch);  // rows r16 + 16 * i
-      ok = mbar_wait_park(bar_wempty + 8 * s, ((ks / NW) & 1u) ^ 1u, abort_flag);
+      for (int i = 0; i < 4; ++i) rw[i] = *reinterpret_cast<const uint4*>(pk + (((c0 + (uint32_t)i) ^ sz) << 4));
+      if (ks >= NW) ok = mbar_wait_park(bar_done + 8 * ((ks - NW) % ND), ((ks - NW) / ND) & 1u, abort_flag);
       if (!ok) break;
-      uint8_t* w_st = sW + s * kStageW + r16 * 128;
+      tc_fence_after();
+      const uint32_t tdst = tmem + lane_base + (uint32_t)(kAccCols + s * kColsW);
 #pragma unroll
-      for (int i = 0; i < 8; ++i) {
-        const uint32_t in[4] = {rw[i].x, rw[i].y, rw[i].z, rw[i].w};
-        uint32_t ev[4], od[4];
+      for (int h = 0; h < 2; ++h) {
+        uint32_t o[16];
 #pragma unroll
-        for (int q = 0; q < 4; ++q) {
-          ev[q] = (in[q] << 4) & 0xF0F0F0F0u;
-          od[q] = in[q] & 0xF0F0F0F0u;
+        for (int i = 0; i < 2; ++i) {
+          const uint4 v = rw[2 * h + i];
+          const uint32_t in[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            o[8 * i + q] = (in[q] << 4) & 0xF0F0F0F0u;
+            o[8 * i + 4 + q] = in[q] & 0xF0F0F0F0u;
+          }
         }
-        uint8_t* dst = w_st + i * 16 * 128;
-        *reinterpret_cast<uint4*>(dst + sw_even) = make_uint4(ev[0], ev[1], ev[2], ev[3]);
-        *reinterpret_cast<uint4*>(dst + (sw_even ^ 16u)) = make_uint4(od[0], od[1], od[2], od[3]);
+        tmem_st16(tdst + (uint32_t)(16 * h), o);
       }
       // (only now: every register loaded from the packed stage has been consumed)
       mbar_arrive(bar_pempty + 8 * ps);
-      fence_proxy_async_smem();  // generic-proxy writes -> visible to the tensor core's async reads
+      asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+      tc_fence_before();
       mbar_arrive(bar_wfull + 8 * s);
     }
   } else if (warp >= kFirstX && warp < kMmaWarp) {
@@ -269,7 +305,7 @@ __global__ void __launch_bounds__(kThreadsS, 2)
 #pragma unroll
       for (int i = 0; i < 2; ++i)
         rx[i] = *reinterpret_cast<const uint4*>(pk + ((lane + 32 * i) >> 2) * kPitch + (ks % SUP) * 64 + (lane & 3) * 16);
-      ok = mbar_wait_park(bar_xempty + 8 * sx, ((ks / NX) & 1u) ^ 1u, abort_flag);
+      if (ks >= NX) ok = mbar_wait_park(bar_done + 8 * ((ks - NX) % ND), ((ks - NX) / ND) & 1u, abort_flag);
       if (!ok) break;
       uint8_t* x_st = sX + sx * kStageX;
 #pragma unroll
@@ -295,11 +331,22 @@ __global__ void __launch_bounds__(kThreadsS, 2)
         uint8_t* xrow = x_st + mrow * 128;
         int cnt = c_first;
         uint32_t boff = boff_first;
-        for (int j = 0; j < run; ++j) {
-          xrow[(kpos_byte(si[j]) + boff) ^ swz] = (uint8_t)(sv[j] ^ 0x80u);
-          if (++cnt == p.k) {
-            cnt = 0;
-            boff += (uint32_t)p.b;
+        // eight entries at a time: their indices and values come with one 8-byte read each (a lane's
+        // run starts on an 8-byte boundary: nb is a multiple of 16), and the eight byte stores do
+        // not wait for one another
+        for (int j0 = 0; j0 < run; j0 += 8) {
+          const uint2 iv = *reinterpret_cast<const uint2*>(si + j0);
+          const uint2 vv = *reinterpret_cast<const uint2*>(sv + j0);
+          const uint32_t vx = vv.x ^ 0x80808080u, vy = vv.y ^ 0x80808080u;
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            const uint32_t jj = ((j < 4 ? iv.x : iv.y) >> (8 * (j & 3))) & 0xFFu;
+            const uint32_t val = ((j < 4 ? vx : vy) >> (8 * (j & 3))) & 0xFFu;
+            xrow[(kpos_byte(jj) + boff) ^ swz] = (uint8_t)val;
+            if (++cnt == p.k) {
+              cnt = 0;
+              boff += (uint32_t)p.b;
+            }
           }
         }
       }
@@ -318,16 +365,15 @@ __global__ void __launch_bounds__(kThreadsS, 2)
       bool ok = true;
       for (int ks = j; ks < KS && ok; ks += 2) {
         const int s = ks % NW, sx = ks % NX;
-        ok = mbar_wait(bar_wfull + 8 * s, (ks / NW) & 1u, abort_flag) && mbar_wait(bar_xfull + 8 * sx, (ks / NX) & 1u, abort_flag);
+        ok = mbar_wait_park(bar_wfull + 8 * s, (ks / NW) & 1u, abort_flag) && mbar_wait_park(bar_xfull + 8 * sx, (ks / NX) & 1u, abort_flag);
         if (!ok) break;
         tc_fence_after();
-        const uint64_t da = desc_sw128(smem_u32(sW + s * kStageW));
+        const uint32_t ta = tmem + (uint32_t)(kAccCols + s * kColsW);
         const uint64_t db = desc_sw128(smem_u32(sX + sx * kStageX));
 #pragma unroll
         for (int kk = 0; kk < BK / 32; ++kk)
-          umma_i8<1>(tmem + (uint32_t)(j * MT), da + 2 * kk, db + 2 * kk, kIdescStream, (ks > j || kk > 0) ? 1u : 0u);
-        umma_commit<1>(bar_wempty + 8 * s);
-        umma_commit<1>(bar_xempty + 8 * sx);
+          umma_i8_ta(tmem + (uint32_t)(j * MT), ta + 8 * kk, db + 2 * kk, kIdescStream, (ks > j || kk > 0) ? 1u : 0u);
+        umma_commit<1>(bar_done + 8 * (ks % ND));
       }
       if (ok && j < KS) umma_commit<1>(bar_tfull);
     }
@@ -346,7 +392,7 @@ __global__ void __launch_bounds__(kThreadsS, 2)
     if (mbar_wait_idle(bar_tfull, 0, abort_flag)) {
       tc_fence_after();
       const int ch = 32 * q + lane;
-      int4* prow = reinterpret_cast<int4*>(smem) + ch * (MT / 4);
+      int4* prow = reinterpret_cast<int4*>(sPack) + ch * (MT / 4);
       uint32_t v[16];
       tmem_ld16(tmem + ((uint32_t)(32 * q) << 16), v);
       if (KS >= 2) {  // the odd steps' accumulator
@@ -379,7 +425,7 @@ __global__ void __launch_bounds__(kThreadsS, 2)
       const int ch = part * share + (i & (share - 1)), m = i >> lg;
       const int n = n0 + ch;
       if (n >= p.N) continue;
-      const uint32_t laddr = smem_u32(smem) + (uint32_t)(ch * MT + m) * 4u;
+      const uint32_t laddr = smem_u32(sPack) + (uint32_t)(ch * MT + m) * 4u;
       int v = 0;
       if (parts == 1) {
         asm volatile("ld.shared.s32 %0, [%1];" : "=r"(v) : "r"(laddr) : "memory");
@@ -430,12 +476,12 @@ struct MapKey {
 // the host's launch path, and encoding a tensor map costs about a microsecond, so the last maps are
 // remembered per thread (a map is a pure function of these arguments).
 bool make_map_u8(PFN_cuTensorMapEncodeTiled encode, CUtensorMap* out, const void* ptr, uint64_t d0, uint64_t d1,
-                 uint64_t pitch, uint32_t b0, uint32_t b1, bool swizzle128) {
+                 uint64_t pitch, uint32_t b0, uint32_t b1, int swizzle) {
   constexpr int kSlots = 16;
   thread_local MapKey keys[kSlots];
   thread_local CUtensorMap maps[kSlots];
   thread_local int next = 0;
-  const MapKey key{ptr, d0, d1, pitch, b0, b1, swizzle128 ? 1 : 0};
+  const MapKey key{ptr, d0, d1, pitch, b0, b1, swizzle};
   for (int i = 0; i < kSlots; ++i)
     if (keys[i].ptr != nullptr && keys[i] == key) {
       *out = maps[i];
@@ -446,7 +492,8 @@ bool make_map_u8(PFN_cuTensorMapEncodeTiled encode, CUtensorMap* out, const void
   const cuuint32_t box[2] = {b0, b1};
   const cuuint32_t estr[2] = {1, 1};
   if (encode(out, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(ptr), dims, pitches, box, estr,
-             CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE,
+             CU_TENSOR_MAP_INTERLEAVE_NONE,
+             swizzle == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : (swizzle == 128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE),
              CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
     return false;
   keys[next] = key;
@@ -548,10 +595,10 @@ cudaError_t launch_gemm_stream(int b, int k, const sq_encoded& A, const sq_weigh
   p.KS = (int)(ks / parts);
 
   CUtensorMap mw, mx, msv, msi;
-  if (!make_map_u8(encode, &mw, W.wq4, (uint64_t)(K / 2), (uint64_t)N, (uint64_t)(K / 2), kPitch, SC, false)) return cudaErrorInvalidValue;
-  if (!make_map_u8(encode, &mx, A.dq4, (uint64_t)(K / 2), (uint64_t)M, (uint64_t)(K / 2), kPitch, MT, false)) return cudaErrorInvalidValue;
-  if (!make_map_u8(encode, &msv, A.vals, (uint64_t)GK, (uint64_t)M, (uint64_t)GK, (uint32_t)(SUP * nb), MT, false)) return cudaErrorInvalidValue;
-  if (!make_map_u8(encode, &msi, A.idx, (uint64_t)GK, (uint64_t)M, (uint64_t)GK, (uint32_t)(SUP * nb), MT, false)) return cudaErrorInvalidValue;
+  if (!make_map_u8(encode, &mw, W.wq4, (uint64_t)(K / 2), (uint64_t)N, (uint64_t)(K / 2), kPitch, SC, SUP == 1 ? 64 : 128)) return cudaErrorInvalidValue;
+  if (!make_map_u8(encode, &mx, A.dq4, (uint64_t)(K / 2), (uint64_t)M, (uint64_t)(K / 2), kPitch, MT, 0)) return cudaErrorInvalidValue;
+  if (!make_map_u8(encode, &msv, A.vals, (uint64_t)GK, (uint64_t)M, (uint64_t)GK, (uint32_t)(SUP * nb), MT, 0)) return cudaErrorInvalidValue;
+  if (!make_map_u8(encode, &msi, A.idx, (uint64_t)GK, (uint64_t)M, (uint64_t)GK, (uint32_t)(SUP * nb), MT, 0)) return cudaErrorInvalidValue;
   return launch_stream(p, mw, mx, msv, msi, dev, st);
 }
 
