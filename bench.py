@@ -48,7 +48,7 @@ GEMM_CAPTURE_TRAFFIC_BYTES = 50.89e6 + 4.22e6
 GEMM_CAPTURE_ALGO_BYTES = 2048 * 8192 * 0.625 + 8192 * 8192 * 0.625 + 2.0 * 2048 * 8192
 # ncu DRAM traffic of one encode launch of the 8192 x 8192 bandwidth test (dynamic k=8 / static k=8),
 # profiles/encode_kernels_b64_k8_8192x8192.txt
-ENCODE_TRAFFIC_BYTES_PER_LAUNCH = {"dynamic": 134.29e6 + 25.98e6, "static": 134.77e6 + 23.95e6}
+ENCODE_TRAFFIC_BYTES_PER_LAUNCH = {"dynamic": 134.29e6 + 25.98e6, "static": 134.34e6 + 20.21e6}
 
 
 def load_peaks():
@@ -678,7 +678,7 @@ def run_cuda(args):
             line["gemm_8b_dynamic"] = {"workload": "8B-decoder-shaped linears + the single-GEMM configuration (last row), b=64, k=8, dynamic; median of 20 CUDA-event pairs (small inputs may sit in L2); fused = plain sq_gemm without a workspace",
                                        **bench_8b_dynamic(sq, dev, peaks)}
             line["encode"] = {"workload": "sq_encode alone: bf16 8192 x 8192, Student-t nu=3, 0.5% channels x50, b=64; 3 inputs in rotation (> L2); median of 50 launches",
-                              "observed_bound": "dynamic: integer/logic pipe (ncu: 67% busy at 9.4 of 17.5 lane-instructions per element, DRAM 35%); static: first and last round of a 45 us kernel (steady state 5.6 TB/s)",
+                              "observed_bound": "dynamic: integer/logic pipe (ncu: 67% busy at 9.4 of 17.5 lane-instructions per element, DRAM 35%); static: at the memory's rate between a launch's first and last round of rows (a row group never waits for data after its first row), no pipe above 58%",
                               **bench_encode_only(sq, dev, peaks)}
             line["gemm_fused"] = {"workload": "70B-shaped linears, M=4096, b=128, k=16: plain sq_gemm (sparse part inside the GEMM kernel) vs the workspace call",
                                   **bench_gemm_fused(sq, layers, dev, peaks)}
