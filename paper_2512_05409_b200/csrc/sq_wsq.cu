@@ -153,7 +153,7 @@ constexpr int kWsqCh = 2;  // output channels a warp works on at a time
 //                memory, one multiply-add with the compact value (its slot is the step number, so
 //                it is picked out of the registers with constant shifts).
 template <int B, int MT>
-__global__ void __launch_bounds__(kWsqWarps * 32, (B == 128 || MT == 4) ? 2 : 3) sqw_gemm_kernel(int k, const int8_t* __restrict__ xq,
+__global__ void __launch_bounds__(kWsqWarps * 32, B == 128 ? 2 : 3) sqw_gemm_kernel(int k, const int8_t* __restrict__ xq,
                                                                      const float* __restrict__ s_x,
                                                                      const uint8_t* __restrict__ wq4,
                                                                      const int8_t* __restrict__ w_hi,
@@ -219,14 +219,32 @@ __global__ void __launch_bounds__(kWsqWarps * 32, (B == 128 || MT == 4) ? 2 : 3)
           }
         }
       }
+      // dense part, word by word for both channels (the word's activations are read once), and the
+      // one-bit-per-weight masks
+      uint32_t mreg[kWsqCh][NM];
 #pragma unroll
-      for (int c = 0; c < kWsqCh; ++c) {
-        uint32_t mreg[NM];
+      for (int r = 0; r < NM; ++r) {
+        uint32_t sq[kWsqCh][4];
 #pragma unroll
-        for (int r = 0; r < NM; ++r) {
-          uint32_t sq[4];
+        for (int j = 0; j < 4; ++j) {
+          const int8_t* xw = xb + (4 * r + j) * (8 * MT);
+          int xr[2 * MT];
+          if constexpr (MT == 1) {
+            const int2 xv = *reinterpret_cast<const int2*>(xw);
+            xr[0] = xv.x;
+            xr[1] = xv.y;
+          } else {
 #pragma unroll
-          for (int j = 0; j < 4; ++j) {
+            for (int m2 = 0; m2 < MT / 2; ++m2) {
+              const int4 xv = *reinterpret_cast<const int4*>(xw + 16 * m2);
+              xr[4 * m2] = xv.x;
+              xr[4 * m2 + 1] = xv.y;
+              xr[4 * m2 + 2] = xv.z;
+              xr[4 * m2 + 3] = xv.w;
+            }
+          }
+#pragma unroll
+          for (int c = 0; c < kWsqCh; ++c) {
             const uint32_t word = words[c][4 * r + j];
             // nibbles holding 1000: bit 3 set and the three low bits clear -> a mark at bit 4i + 3;
             // flipping the marked bits turns the mask code into code 0
@@ -234,41 +252,36 @@ __global__ void __launch_bounds__(kWsqWarps * 32, (B == 128 || MT == 4) ? 2 : 3)
             const uint32_t f3 = word & ~t & 0x88888888u;
             const uint32_t clean = word ^ f3;
             const int ev = (int)((clean << 4) & 0xF0F0F0F0u), od = (int)(clean & 0xF0F0F0F0u);  // 16 * code, bytewise
-            const int8_t* xw = xb + (4 * r + j) * (8 * MT);
-            if constexpr (MT == 1) {
-              const int2 xv = *reinterpret_cast<const int2*>(xw);
-              lo[c][0] = __dp4a(ev, xv.x, __dp4a(od, xv.y, lo[c][0]));
-            } else {
 #pragma unroll
-              for (int m2 = 0; m2 < MT / 2; ++m2) {
-                const int4 xv = *reinterpret_cast<const int4*>(xw + 16 * m2);
-                lo[c][2 * m2] = __dp4a(ev, xv.x, __dp4a(od, xv.y, lo[c][2 * m2]));
-                lo[c][2 * m2 + 1] = __dp4a(ev, xv.z, __dp4a(od, xv.w, lo[c][2 * m2 + 1]));
-              }
-            }
+            for (int m = 0; m < MT; ++m) lo[c][m] = __dp4a(ev, xr[2 * m], __dp4a(od, xr[2 * m + 1], lo[c][m]));
             // marks of a byte's two nibbles side by side, then the four pairs into the top byte
             const uint32_t y = ((f3 >> 3) | (f3 >> 6)) & 0x03030303u;
-            sq[j] = y * 0x01041040u;
+            sq[c][j] = y * 0x01041040u;
           }
-          mreg[r] = __byte_perm(__byte_perm(sq[0], sq[1], 0x0073), __byte_perm(sq[2], sq[3], 0x0073), 0x5410);
         }
+#pragma unroll
+        for (int c = 0; c < kWsqCh; ++c)
+          mreg[c][r] = __byte_perm(__byte_perm(sq[c][0], sq[c][1], 0x0073), __byte_perm(sq[c][2], sq[c][3], 0x0073), 0x5410);
+      }
+#pragma unroll
+      for (int c = 0; c < kWsqCh; ++c) {
         // sparse part: the k masked places in position order
 #pragma unroll
         for (int s = 0; s < B / 2; ++s) {
           if ((s & 3) == 0 && s >= k) break;  // (uniform: whole words of compact values are skipped at once)
           if (s < k) {
-            uint32_t cur = mreg[0];
+            uint32_t cur = mreg[c][0];
             int base = 0;
 #pragma unroll
             for (int r = 1; r < NM; ++r)
               if (cur == 0u) {
-                cur = mreg[r];
+                cur = mreg[c][r];
                 base = 32 * r;
               }
             const int pl = base + __ffs((int)cur) - 1;
 #pragma unroll
             for (int r = 0; r < NM; ++r)
-              if (base == 32 * r) mreg[r] &= mreg[r] - 1u;
+              if (base == 32 * r) mreg[c][r] &= mreg[c][r] - 1u;
             const int v = (int)(hv[c][s >> 2] << (24 - 8 * (s & 3))) >> 24;
             const int8_t* xw = xb + (pl >> 3) * (8 * MT);
             const int rb = ((pl & 1) << 2) | ((pl & 7) >> 1);  // byte of the place inside its word
