@@ -421,35 +421,46 @@ __global__ void __launch_bounds__(kThreadsS, 2)
     // CTA `part` finishes channels [part * SC / parts, (part + 1) * SC / parts) of the slab for all
     // tokens: adds the parts' sums (integer: order-free) and runs the usual epilogue arithmetic.
     const int share = SC / parts, lg = 31 - __clz(share);  // parts is 1, 2, 4 or 8
-    for (int i = tid; i < share * p.M; i += kThreadsS) {
-      const int ch = part * share + (i & (share - 1)), m = i >> lg;
+    const int quads = (p.M + 3) >> 2;                        // a thread takes four tokens of one channel:
+    for (int i = tid; i < share * quads; i += kThreadsS) {   // one 16-byte (remote) read per part
+      const int ch = part * share + (i & (share - 1)), m0 = (i >> lg) << 2;
       const int n = n0 + ch;
       if (n >= p.N) continue;
-      const uint32_t laddr = smem_u32(sPack) + (uint32_t)(ch * MT + m) * 4u;
-      int v = 0;
+      const uint32_t laddr = smem_u32(sPack) + (uint32_t)(ch * MT + m0) * 4u;
+      int v[4] = {0, 0, 0, 0};
       if (parts == 1) {
-        asm volatile("ld.shared.s32 %0, [%1];" : "=r"(v) : "r"(laddr) : "memory");
+        asm volatile("ld.shared.v4.s32 {%0, %1, %2, %3}, [%4];" : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]) : "r"(laddr) : "memory");
       } else {
-        // all parts' loads first, then the sum: a load followed by its add would wait out one
+        // all parts' loads first, then the sums: a load followed by its add would wait out one
         // remote access after the other
-        int a[8];
+        int a[8][4];
 #pragma unroll
         for (int sp = 0; sp < 8; ++sp) {
-          a[sp] = 0;
+          a[sp][0] = a[sp][1] = a[sp][2] = a[sp][3] = 0;
           if (sp < parts)
             asm volatile(
                 "{\n\t.reg .b32 ra;\n\t"
-                "mapa.shared::cluster.u32 ra, %1, %2;\n\t"
-                "ld.shared::cluster.s32 %0, [ra];\n\t}"
-                : "=r"(a[sp])
+                "mapa.shared::cluster.u32 ra, %4, %5;\n\t"
+                "ld.shared::cluster.v4.s32 {%0, %1, %2, %3}, [ra];\n\t}"
+                : "=r"(a[sp][0]), "=r"(a[sp][1]), "=r"(a[sp][2]), "=r"(a[sp][3])
                 : "r"(laddr), "r"(sp));
         }
 #pragma unroll
-        for (int sp = 0; sp < 8; ++sp) v += a[sp];
+        for (int sp = 0; sp < 8; ++sp)
+#pragma unroll
+          for (int t = 0; t < 4; ++t) v[t] += a[sp][t];
       }
-      const int acc = (v - 2048 * s_cs[ch]) >> 4;
-      p.out[(size_t)m * p.N + n] = (uint16_t)f32_to_bf16_bits(((float)acc * s_sh[m]) * s_sw[ch]);
-      if (p.acc_out != nullptr) p.acc_out[(size_t)m * p.N + n] = acc;
+      const int cs = 2048 * s_cs[ch];
+      const float sw = s_sw[ch];
+#pragma unroll
+      for (int t = 0; t < 4; ++t) {
+        const int m = m0 + t;
+        if (m < p.M) {
+          const int acc = (v[t] - cs) >> 4;
+          p.out[(size_t)m * p.N + n] = (uint16_t)f32_to_bf16_bits(((float)acc * s_sh[m]) * sw);
+          if (p.acc_out != nullptr) p.acc_out[(size_t)m * p.N + n] = acc;
+        }
+      }
     }
   }
   if (parts > 1) cluster_sync_all();  // nobody leaves while a peer may still read its partial sums
@@ -583,11 +594,13 @@ cudaError_t launch_gemm_stream(int b, int k, const sq_encoded& A, const sq_weigh
   p.b = b;
   p.k = k;
   p.nb = nb;
-  // Parts of K per slab: as many as keep every part at least four K steps long while the launch still
-  // fits the GPU in one wave (two CTAs per SM; a cluster's CTAs are co-scheduled).
+  // Parts of K per slab: up to four, as long as every part is at least four K steps long and the
+  // launch still fits the GPU in one wave (two CTAs per SM; a cluster's CTAs are co-scheduled).
+  // (Eight parts were measured slower on every shape: what a part saves in K steps, 0.3 us each,
+  // the larger cluster's barriers and the finish's remote reads take back.)
   const int64_t slabs = (N + SC - 1) / SC, ks = K / BK;
   int parts = 1;
-  for (int cand = 2; cand <= 8; cand *= 2) {
+  for (int cand = 2; cand <= 4; cand *= 2) {
     if (ks % cand != 0 || ks / cand < 4 || slabs * cand > 2 * (int64_t)sms) break;
     parts = cand;
   }
