@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libsq_b200.so")
 SOURCES = ["sq_api.cu", "sq_setup.cu", "sq_encode.cu", "sq_gemm.cu", "sq_gemm_stream.cu", "sq_fp.cu", "sq_wsq.cu"]
-HEADERS = ["sq_device.cuh", "sq_host.h", os.path.join("..", "..", "include", "sq.h")]
+HEADERS = ["sq_device.cuh", "sq_fp_device.cuh", "sq_host.h", os.path.join("..", "..", "include", "sq.h")]
 
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a",

@@ -361,6 +361,14 @@ sq_status sq_fp_encode(const sq_format* fmt, const void* X_bf16, int64_t M, int6
   SQ_TRY(check_device());
   sq_encoded o = *out;
   if (is_static(fmt)) o.idx = nullptr;
+  if (is_static(fmt)) {
+    // static positions: rows streamed through shared-memory slots (bounded waits, hence the status word)
+    int* status = status_word();
+    if (status == nullptr) return SQ_ERR_CUDA;
+    const cudaError_t err = launch_fp_encode_static_ring(fmt->bank, fmt->k, static_cast<const uint16_t*>(X_bf16), M, K,
+                                                         positions, o, a8, status, static_cast<cudaStream_t>(cuda_stream));
+    if (err != cudaErrorNotSupported) return from_cuda(err);
+  }
   return from_cuda(launch_fp_encode(fmt->bank, fmt->k, static_cast<const uint16_t*>(X_bf16), M, K, positions, o, a8,
                                     static_cast<cudaStream_t>(cuda_stream)));
 }

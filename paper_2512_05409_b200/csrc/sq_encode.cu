@@ -32,6 +32,7 @@
 #include <cstdio>
 #include <cstdlib>
 #include "sq_device.cuh"
+#include "sq_fp_device.cuh"
 #include "sq_host.h"
 
 namespace sq {
@@ -977,7 +978,7 @@ __global__ void __launch_bounds__(NT, 1) encode_static_regs_kernel(const EncodeP
 //   from the registers.
 // MASK8: the per-element magnitude masks are kept as bytes and widened on the fly (long rows,
 // where a half-word table would not leave room for the slots).
-template <int NCL, int NT, bool INDEP, bool MASK8>
+template <int NCL, int NT, bool INDEP, bool MASK8, bool FP = false>
 __global__ void __launch_bounds__(NT, 1) encode_static_ring_kernel(const EncodeParams p) {
   extern __shared__ __align__(128) uint8_t smem_enc[];
   const int K = p.K, k = p.k;
@@ -1061,7 +1062,7 @@ __global__ void __launch_bounds__(NT, 1) encode_static_ring_kernel(const EncodeP
     jt[t] = (uint16_t)j;
     if (MASK8) hmask[j] = 0;
     else reinterpret_cast<uint16_t*>(hmask)[j] = 0;
-    if (want_a8) jimg[t] = (uint16_t)((j & ~7) | ((j & 1) << 2) | ((j & 7) >> 1));
+    if (want_a8) jimg[t] = FP ? (uint16_t)j : (uint16_t)((j & ~7) | ((j & 1) << 2) | ((j & 7) >> 1));
   }
   __syncthreads();
 
@@ -1125,7 +1126,27 @@ __global__ void __launch_bounds__(NT, 1) encode_static_ring_kernel(const EncodeP
     }
     if (smax_bits == 0xFFFFFFFFu) break;
     const uint32_t amax_bits = INDEP ? smax_bits : max(smax_bits, rmax_bits);
-    const RowScale rs = INDEP ? row_scale_indep(amax_bits, rmax_bits) : row_scale_warp(amax_bits, rmax_bits, lane);
+    RowScale rs;
+    if constexpr (FP) {
+      // floating-point variant: the row maximum maps to 256, the dense grid is coarser by the
+      // smallest power of two (up to 2^6) that brings the largest unselected magnitude to at most 6
+      const float amax = bf16_bits_to_f32(amax_bits), rmax = bf16_bits_to_f32(rmax_bits);
+      rs.inv = amax > 0.f ? __fdiv_rn(256.0f, amax) : 0.f;
+      rs.s_hi = amax > 0.f ? __fdiv_rn(amax, 256.0f) : 0.f;
+      int e = 0;
+      if (amax > 0.f) {
+        e = 6;
+#pragma unroll
+        for (int t = 6; t >= 0; --t)
+          if ((double)rmax * (double)(rs.inv * __int_as_float((127 - t) << 23)) <= 6.0) e = t;  // ends on the smallest fitting t
+      }
+      rs.e = e;
+      rs.s_lo = rs.s_hi * (float)(1 << e);
+      rs.inv_lo = rs.inv * __int_as_float((127 - e) << 23);
+      rs.clamp = false;  // the code construction saturates by itself
+    } else {
+      rs = INDEP ? row_scale_indep(amax_bits, rmax_bits) : row_scale_warp(amax_bits, rmax_bits, lane);
+    }
     if (glane == 0) {
       p.s_hi[m] = rs.s_hi;
       p.s_lo[m] = rs.s_lo;
@@ -1141,8 +1162,10 @@ __global__ void __launch_bounds__(NT, 1) encode_static_ring_kernel(const EncodeP
         const uint32_t w[4] = {srow[jj.x & 0xFFFFu], srow[jj.x >> 16], srow[jj.y & 0xFFFFu], srow[jj.y >> 16]};
         uint32_t o = 0;
 #pragma unroll
-        for (int q = 0; q < 4; ++q)
-          o |= (__float_as_uint(__fmaf_rn(__uint_as_float(w[q] << 16), rs.inv, kMagic)) & 0xFFu) << (8 * q);
+        for (int q = 0; q < 4; ++q) {
+          if constexpr (FP) o |= e4m3_of32(w[q], rs.inv) << (8 * q);
+          else o |= (__float_as_uint(__fmaf_rn(__uint_as_float(w[q] << 16), rs.inv, kMagic)) & 0xFFu) << (8 * q);
+        }
         *reinterpret_cast<uint32_t*>(vdst + 4 * q4) = o;
         if (want_a8) {
           const uint2 ji = *reinterpret_cast<const uint2*>(jimg + 4 * q4);
@@ -1179,7 +1202,29 @@ __global__ void __launch_bounds__(NT, 1) encode_static_ring_kernel(const EncodeP
       }
     }
     const float2 cc = make_float2(cq, cq), mm = make_float2(kMagic + 8.0f, kMagic + 8.0f);
-    if (want_a8) {
+    if constexpr (FP) {
+      // E2M1 codes of the registers, eight nibbles per word, and (on request) the merged operand:
+      // the E4M3 byte of code * 2^e in element order, the selected places' bytes from the image
+      uint2* aw = want_a8 ? reinterpret_cast<uint2*>(p.a8 + (size_t)m_this * K) + slice * S8 + lane : nullptr;
+      const uint2* iw = reinterpret_cast<const uint2*>(img) + slice * S8 + lane;
+#pragma unroll
+      for (int c = 0; c < NCL; ++c) {
+        const uint32_t w[4] = {v[c].x, v[c].y, v[c].z, v[c].w};
+        uint32_t nib = 0, by[2] = {0, 0};
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+          const uint32_t h = (w[q >> 1] >> (16 * (q & 1))) & 0xFFFFu;
+          const uint32_t code = e2m1_of32(h, cq);
+          nib |= code << (4 * q);
+          by[q >> 2] |= e4m3_of_e2m1(code, rs.e) << (8 * (q & 3));
+        }
+        dst[c * 32] = nib;
+        if (want_a8) {
+          const uint2 im = iw[c * 32];
+          aw[c * 32] = make_uint2(by[0] | im.x, by[1] | im.y);
+        }
+      }
+    } else if (want_a8) {
       // Codes carry an offset of 8 (u = code + 8 in 1..15 in the low bits of 0x4B400000 + u).
       // The four even and the four odd ones are summed into bytes by multiply-adds; their
       // constant parts come off in the last step of each use:
@@ -1495,7 +1540,7 @@ cudaError_t launch_static_regs_as(EncodeParams p, int rw, cudaStream_t st) {
 }
 
 // Ring kernel: `rw` warps per row, 16 / rw groups per block, one slot per group.
-template <int NCL, bool INDEP, bool MASK8>
+template <int NCL, bool INDEP, bool MASK8, bool FP = false>
 cudaError_t launch_static_ring_as(EncodeParams p, int rw, cudaStream_t st) {
   constexpr int NT = 512;
   const int GK = (p.K / p.b) * p.k;
@@ -1511,9 +1556,9 @@ cudaError_t launch_static_ring_as(EncodeParams p, int rw, cudaStream_t st) {
   int dev = 0, sms = 0;
   cudaError_t err = device_and_sms(&dev, &sms);
   if (err != cudaSuccess) return err;
-  SQ_ENSURE_SMEM((encode_static_ring_kernel<NCL, NT, INDEP, MASK8>), dev, smem);
+  SQ_ENSURE_SMEM((encode_static_ring_kernel<NCL, NT, INDEP, MASK8, FP>), dev, smem);
   const int64_t blocks = p.M < sms ? p.M : sms;
-  encode_static_ring_kernel<NCL, NT, INDEP, MASK8><<<(unsigned)blocks, NT, smem, st>>>(p);
+  encode_static_ring_kernel<NCL, NT, INDEP, MASK8, FP><<<(unsigned)blocks, NT, smem, st>>>(p);
   return cudaGetLastError();
 }
 
@@ -1521,7 +1566,7 @@ cudaError_t launch_static_ring_as(EncodeParams p, int rw, cudaStream_t st) {
 // (the per-row work that does not shrink with the slice -- scales, barriers -- is then spread over
 // the most elements, and the most rows are in flight); half-word masks if the tables and slots
 // fit, else byte masks.
-template <bool INDEP>
+template <bool INDEP, bool FP = false>
 cudaError_t launch_static_ring(const EncodeParams& p, cudaStream_t st) {
   if (p.K % 256 != 0 || p.K > 65535 || (reinterpret_cast<uintptr_t>(p.X) & 15) != 0) return cudaErrorNotSupported;
   for (int mask8 = 0; mask8 < 2; ++mask8) {
@@ -1531,8 +1576,8 @@ cudaError_t launch_static_ring(const EncodeParams& p, cudaStream_t st) {
       cudaError_t err = cudaErrorNotSupported;
 #define SQ_RING(NCL_)                                                                   \
   if (ncl == NCL_)                                                                      \
-    err = mask8 ? launch_static_ring_as<NCL_, INDEP, true>(p, rw, st)                   \
-                : launch_static_ring_as<NCL_, INDEP, false>(p, rw, st);
+    err = mask8 ? launch_static_ring_as<NCL_, INDEP, true, FP>(p, rw, st)               \
+                : launch_static_ring_as<NCL_, INDEP, false, FP>(p, rw, st);
       SQ_RING(8) SQ_RING(12) SQ_RING(14) SQ_RING(16)
 #undef SQ_RING
       if (err != cudaErrorNotSupported) return err;
@@ -1636,6 +1681,33 @@ cudaError_t launch_encode(int b, int k, bool is_static, bool indep, const uint16
   if (b == 32) return launch_generic<32>(k, false, false, X, M, K, positions, out, st);
   if (b == 64) return launch_generic<64>(k, false, false, X, M, K, positions, out, st);
   return launch_generic<128>(k, false, false, X, M, K, positions, out, st);
+}
+
+// Floating-point variant, static positions: the ring kernel with that format's roundings.
+// cudaErrorNotSupported = this shape is left to the variant's own one-block-per-row kernel.
+cudaError_t launch_fp_encode_static_ring(int b, int k, const uint16_t* X, int64_t M, int64_t K, const uint8_t* positions,
+                                         const sq_encoded& out, uint8_t* a8, int* status, cudaStream_t st) {
+  if (positions == nullptr || M < 1) return cudaErrorNotSupported;
+  EncodeParams p;
+  p.a8 = a8;
+  p.X = X;
+  p.positions = positions;
+  p.dq4 = out.dq4;
+  p.vals = out.vals;
+  p.idx = out.idx;
+  p.s_hi = out.s_hi;
+  p.s_lo = out.s_lo;
+  p.shift = out.shift;
+  p.status = status;
+  p.M = M;
+  p.K = (int)K;
+  p.k = k;
+  p.b = b;
+  p.nbuf = 1;
+  p.rw = 1;
+  p.group_stride = 0;
+  p.mk = MulK{0xFFFFFFFFu, 2u, 32u, 256u, 65536u, 1u << 24, 16u, 1u};
+  return launch_static_ring<false, true>(p, st);
 }
 
 cudaError_t launch_decode(int b, int k, const sq_encoded& A, const uint8_t* positions, int64_t M,

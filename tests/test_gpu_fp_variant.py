@@ -87,6 +87,28 @@ def test_fp_degenerate_rows():
     assert sq.sq_device_status() == sq.SQ_OK
 
 
+@pytest.mark.parametrize("K,b,k", [(2048, 64, 8), (3072, 32, 3), (7168, 128, 16), (8192, 64, 32), (28672, 128, 16)])
+def test_fp_static_encode_staged_rows(K, b, k):
+    """Static positions at row lengths the staged-row kernel takes (one, two and eight warps per row,
+    half-word and byte masks), a ragged row count, and rows that are all zero, all equal, one-hot
+    and dominated by an outlier (largest shift, saturating dense codes)."""
+    M = 75
+    fmt = sq.make_format(b, k, True)
+    X = gen.activations(M, K, seed=K + k, outlier_fraction=0.01, outlier_scale=30.0, device="cpu").float()
+    X[0] = 0
+    X[1] = -3.0
+    X[2] = 0
+    X[2, K - 3] = 2.5
+    X[3] = X[3].abs().clamp_min(0.5)
+    X[4, 5] = 3.0e4
+    X[M - 1] = 1.0
+    X = X.to(torch.bfloat16).cuda()
+    pos = sq.sq_calib_positions(fmt, gen.calibration_batch(64, K, seed=K, outlier_fraction=0.01, outlier_scale=30.0, device="cuda"))
+    enc, a8 = sq.sq_fp_encode(fmt, X, pos)
+    assert sq.sq_device_status() == sq.SQ_OK
+    _compare_encoded(enc, a8, oracle.fp_encode(b, k, gen.bf16_bits(X), _np(pos)))
+
+
 @pytest.mark.parametrize("static", [False, True])
 def test_fp_full_size_sweep_shape(static):
     """M = 4096, K = N = 8192 (the format-sweep shape): every row's encoding in full, GEMM on sampled
