@@ -369,6 +369,15 @@ sq_status sq_fp_encode(const sq_format* fmt, const void* X_bf16, int64_t M, int6
                                                          positions, o, a8, status, static_cast<cudaStream_t>(cuda_stream));
     if (err != cudaErrorNotSupported) return from_cuda(err);
   }
+  if (!is_static(fmt)) {
+    // dynamic positions at the integer path's fast ratios: its row-group kernel (selection by
+    // sorting network) with this format's scales and roundings
+    int* status = status_word();
+    if (status == nullptr) return SQ_ERR_CUDA;
+    const cudaError_t err = launch_fp_encode_dynamic_rows(fmt->bank, fmt->k, static_cast<const uint16_t*>(X_bf16), M, K, o, a8,
+                                                          status, static_cast<cudaStream_t>(cuda_stream));
+    if (err != cudaErrorNotSupported) return from_cuda(err);
+  }
   return from_cuda(launch_fp_encode(fmt->bank, fmt->k, static_cast<const uint16_t*>(X_bf16), M, K, positions, o, a8,
                                     static_cast<cudaStream_t>(cuda_stream)));
 }

@@ -318,6 +318,135 @@ __device__ __forceinline__ void dense_sweep(const uint16_t* row, int K, const Ro
   }
 }
 
+// ---- floating-point variant (sparse E4M3 + dense E2M1; the selection is the integer path's)
+// Scales from the row maximum and the largest unselected magnitude (bf16 bit patterns): the row
+// maximum maps to 256; the dense grid is coarser by the smallest power of two (up to 2^6) that
+// brings the largest unselected magnitude to at most 6.
+__device__ __forceinline__ int fp_shift_of(float inv, float rmax, bool nonzero) {
+  int e = 0;
+  if (nonzero) {
+    e = 6;
+#pragma unroll
+    for (int t = 6; t >= 0; --t)
+      if ((double)rmax * (double)(inv * __int_as_float((127 - t) << 23)) <= 6.0) e = t;  // ends on the smallest fitting t
+  }
+  return e;
+}
+__device__ __forceinline__ RowScale row_scale_fp(uint32_t amax_bits, uint32_t rmax_bits) {
+  RowScale rs;
+  const float amax = bf16_bits_to_f32(amax_bits), rmax = bf16_bits_to_f32(rmax_bits);
+  rs.inv = amax > 0.f ? __fdiv_rn(256.0f, amax) : 0.f;
+  rs.s_hi = amax > 0.f ? __fdiv_rn(amax, 256.0f) : 0.f;
+  rs.e = fp_shift_of(rs.inv, rmax, amax > 0.f);
+  rs.s_lo = rs.s_hi * (float)(1 << rs.e);
+  rs.inv_lo = rs.inv * __int_as_float((127 - rs.e) << 23);
+  rs.clamp = false;  // the code construction saturates by itself
+  return rs;
+}
+// A selected place of the staged row carries its E4M3 byte in a non-finite pattern (exponent field
+// all ones, which no finite input has; the byte's sign in the sign bit, its other seven bits in the
+// mantissa), so that the dense pass finds the merged operand's byte there.
+__device__ __forceinline__ uint32_t fp_marker(uint32_t q) { return ((q & 0x80u) << 8) | 0x7F80u | (q & 0x7Fu); }
+// The dense pass over a staged row: E2M1 codes (eight nibbles per word; a selected place has code
+// 0) and the merged operand's E4M3 bytes in element order.
+__device__ __forceinline__ void dense_sweep_fp(const uint16_t* row, int K, const RowScale& rs, uint8_t* dq4_row, uint8_t* a8_row,
+                                               int lane, int gsize) {
+  const float c = rs.inv_lo;
+  const uint4* src = reinterpret_cast<const uint4*>(row) + lane;
+  uint32_t* dst = reinterpret_cast<uint32_t*>(dq4_row) + lane;
+  uint2* adst = reinterpret_cast<uint2*>(a8_row) + lane;
+  const int iters = (K / 8 - lane + gsize - 1) / gsize;
+#pragma unroll 2
+  for (int i = 0; i < iters; ++i, src += gsize, dst += gsize, adst += gsize) {
+    const uint4 v = *src;
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+    uint32_t nib = 0, by[2] = {0, 0};
+#pragma unroll
+    for (int q = 0; q < 8; ++q) {
+      const uint32_t h = (w[q >> 1] >> (16 * (q & 1))) & 0xFFFFu;
+      uint32_t code = 0, byte;
+      if ((h & 0x7F80u) == 0x7F80u) {
+        byte = ((h >> 8) & 0x80u) | (h & 0x7Fu);
+      } else {
+        code = e2m1_of32(h, c);
+        byte = e4m3_of_e2m1(code, rs.e);
+      }
+      nib |= code << (4 * q);
+      by[q >> 2] |= byte << (8 * (q & 3));
+    }
+    *dst = nib;
+    *adst = make_uint2(by[0], by[1]);
+  }
+}
+
+// The dense E2M1 code of a magnitude is a step function of the bf16 input: seven thresholds per
+// row decide it.  Threshold i = the smallest bf16 magnitude a whose exact product a * c reaches the
+// midpoint between the (i-1)-th and the i-th grid value (0, 0.5, 1, 1.5, 2, 3, 4, 6) -- reaches it
+// or passes it, whichever the tie rule (to the even code) asks for.  One fused multiply-add
+// a * c - midpoint has the exact difference's sign, so the candidate from the quotient is checked
+// exactly.  Lane i (0..6) computes threshold i + 1; every lane gets all seven, each in both
+// halves of a register.  With c = 0 no magnitude reaches any threshold (a NaN pattern).
+struct FpSteps {
+  uint32_t t[7];          // thresholds 1..7, duplicated into both halves
+  uint32_t lut_lo, lut_hi;  // E4M3 bytes of the eight magnitudes times 2^e
+};
+__device__ __forceinline__ FpSteps fp_steps(float c, int e, int lane) {
+  const int i = min(lane, 6);
+  const float mid = i == 0 ? 0.25f : i == 1 ? 0.75f : i == 2 ? 1.25f : i == 3 ? 1.75f : i == 4 ? 2.5f : i == 5 ? 3.5f : 5.0f;
+  const bool strict = (i & 1) == 0;  // a tie goes to the even code: codes 0, 2, 4, 6 keep it
+  uint32_t thr = 0x7FFFu;
+  if (c > 0.f) {
+    const uint32_t a0 = __float_as_uint(__fdiv_rn(mid, c)) >> 16;  // the quotient cut to bf16: at or just below the threshold
+    auto reaches = [&](uint32_t a) {
+      const float d = __fmaf_rn(__uint_as_float(a << 16), c, -mid);
+      return strict ? d > 0.f : d >= 0.f;
+    };
+    thr = reaches(a0) ? a0 : (reaches(a0 + 1u) ? a0 + 1u : a0 + 2u);
+    thr = min(thr, 0x7F80u);
+  }
+  FpSteps st;
+#pragma unroll
+  for (int j = 0; j < 7; ++j) st.t[j] = __shfl_sync(0xffffffffu, thr, j) * 0x10001u;
+  uint32_t lo = 0, hi = 0;
+#pragma unroll
+  for (int n = 0; n < 4; ++n) {
+    lo |= e4m3_of_e2m1((uint32_t)n, e) << (8 * n);
+    hi |= e4m3_of_e2m1((uint32_t)(n + 4), e) << (8 * n);
+  }
+  st.lut_lo = lo;
+  st.lut_hi = hi;
+  return st;
+}
+// Two bf16 inputs (one word) -> their E2M1 codes in bits 0-3 and 16-19: three compares walk the
+// thresholds as a binary tree, a fourth tells zero codes (which carry no sign) from the rest.
+__device__ __forceinline__ uint32_t fp_codes2(uint32_t w, const FpSteps& st) {
+  const uint32_t mag = w & 0x7FFF7FFFu;
+  const uint32_t g2 = ge2_mask(mag, st.t[3]);                                   // code >= 4
+  const uint32_t ta = (g2 & st.t[5]) | (~g2 & st.t[1]);
+  const uint32_t g1 = ge2_mask(mag, ta);                                        // next bit
+  const uint32_t hi = (g1 & st.t[6]) | (~g1 & st.t[4]), lo = (g1 & st.t[2]) | (~g1 & st.t[0]);
+  const uint32_t tb = (g2 & hi) | (~g2 & lo);
+  const uint32_t g0 = ge2_mask(mag, tb);                                        // last bit
+  const uint32_t nz = ge2_mask(mag, st.t[0]);
+  return (g2 & 0x00040004u) | (g1 & 0x00020002u) | (g0 & 0x00010001u) | ((w >> 12) & 0x00080008u & nz);
+}
+__device__ __forceinline__ uint32_t prmt_u32(uint32_t a, uint32_t b, uint32_t sel) {
+  uint32_t d;
+  asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(sel));
+  return d;
+}
+// Eight codes (one nibble each, element i in nibble i) -> the eight E4M3 bytes of code * 2^e: the
+// magnitudes through the row's byte table, the signs moved from bit 3 of a nibble to bit 7 of
+// its byte.
+__device__ __forceinline__ uint2 fp_bytes8(uint32_t nib, const FpSteps& st) {
+  const uint32_t mags = nib & 0x77777777u, sg = nib & 0x88888888u;
+  uint2 by;
+  by.x = prmt_u32(st.lut_lo, st.lut_hi, mags) | prmt_u32((sg << 4) & 0x8080u, 0u, 0x4140u) | prmt_u32(sg & 0x8080u, 0u, 0x1404u);
+  const uint32_t sh = sg >> 16;
+  by.y = prmt_u32(st.lut_lo, st.lut_hi, mags >> 16) | prmt_u32((sh << 4) & 0x8080u, 0u, 0x4140u) | prmt_u32(sh & 0x8080u, 0u, 0x1404u);
+  return by;
+}
+
 struct EncodeParams {
   const uint16_t* X;
   const uint8_t* positions;
@@ -346,7 +475,7 @@ __device__ __forceinline__ void group_sync(int rw, int grp) {
 
 // ------------------------------------------------------------------------------------------------
 // Row-group kernel.  B = bank size; KK = k for dynamic positions (a power of two), 0 for static.
-template <int B, int KK>
+template <int B, int KK, bool FP = false>
 __global__ void __launch_bounds__(B == 128 ? 256 : 512) encode_rows_kernel(const EncodeParams p) {
   extern __shared__ __align__(128) uint8_t smem_enc[];
   constexpr bool kStatic = (KK == 0);
@@ -369,7 +498,10 @@ __global__ void __launch_bounds__(B == 128 ? 256 : 512) encode_rows_kernel(const
   uint16_t* jt = reinterpret_cast<uint16_t*>(smem_enc);
   uint8_t* wbase = smem_enc + table_bytes + (size_t)grp * p.group_stride;
   uint16_t* stash = reinterpret_cast<uint16_t*>(wbase + (size_t)nbuf * K * 2);
-  const size_t stash_bytes = ((size_t)GK * 2 + 15) & ~(size_t)15;
+  // (floating-point variant: the stash is followed by the selected places' element offsets)
+  const size_t stash_half = ((size_t)GK * 2 + 15) & ~(size_t)15;
+  const size_t stash_bytes = stash_half * (FP ? 2 : 1);
+  uint16_t* spos = reinterpret_cast<uint16_t*>(reinterpret_cast<uint8_t*>(stash) + stash_half);
   const uint32_t bar0 = smem_u32(reinterpret_cast<uint8_t*>(stash) + stash_bytes);
   uint32_t* exch = reinterpret_cast<uint32_t*>(reinterpret_cast<uint8_t*>(stash) + stash_bytes + 32);
   __shared__ int abort_flag_s;
@@ -597,6 +729,20 @@ __global__ void __launch_bounds__(B == 128 ? 256 : 512) encode_rows_kernel(const
           iout[i / 4] = (i % 4) == 0 ? pos[i]
                                      : imad(pos[i], (i % 4) == 1 ? mk.k256 : ((i % 4) == 2 ? mk.k65536 : mk.k16m), iout[i / 4]);
         }
+        if constexpr (FP) {
+          uint16_t* sp = spos + g * KK;
+          const uint32_t e0 = (uint32_t)(g * B);
+          if (KK >= 8) {
+#pragma unroll
+            for (int i = 0; i < KK; i += 8)
+              *reinterpret_cast<uint4*>(sp + i) =
+                  make_uint4((e0 + pos[i]) | ((e0 + pos[i + 1]) << 16), (e0 + pos[i + 2]) | ((e0 + pos[i + 3]) << 16),
+                             (e0 + pos[i + 4]) | ((e0 + pos[i + 5]) << 16), (e0 + pos[i + 6]) | ((e0 + pos[i + 7]) << 16));
+          } else {
+#pragma unroll
+            for (int i = 0; i < KK; ++i) sp[i] = (uint16_t)(e0 + pos[i]);
+          }
+        }
         uint32_t raw[KK];
         const uint32_t bank_s = smem_u32(bank);
 #pragma unroll
@@ -675,14 +821,15 @@ __global__ void __launch_bounds__(B == 128 ? 256 : 512) encode_rows_kernel(const
     } else {
       __syncwarp();
     }
-    RowScale rs = row_scale_warp(amax_bits, rmax_bits, threadIdx.x & 31);
+    RowScale rs = FP ? row_scale_fp(amax_bits, rmax_bits) : row_scale_warp(amax_bits, rmax_bits, threadIdx.x & 31);
     if constexpr (!kStatic) {
       // The shift was computed from an upper bound of the largest unselected magnitude.  It is the
       // true one unless the lower bound would still fit one shift less; only then (the same for
       // the whole group) the row, whose selected places are zero by now, is swept for the exact
       // maximum.  (A clamp flag set by the upper bound alone only costs time.)
       const bool exact =
-          rs.e > 0 && rne_prod(bf16_bits_to_f32(rlow_bits), rs.inv * __int_as_float((127 - (rs.e - 1)) << 23)) <= 7;
+          FP ? fp_shift_of(rs.inv, bf16_bits_to_f32(rlow_bits), rs.inv > 0.f) < rs.e
+             : rs.e > 0 && rne_prod(bf16_bits_to_f32(rlow_bits), rs.inv * __int_as_float((127 - (rs.e - 1)) << 23)) <= 7;
       if (exact) {
         const uint4* src = reinterpret_cast<const uint4*>(row) + lane;
         const int iters = (K / 8 - lane + gsize - 1) / gsize;
@@ -699,7 +846,7 @@ __global__ void __launch_bounds__(B == 128 ? 256 : 512) encode_rows_kernel(const
           rx = 0;
           for (int w = 0; w < rw; ++w) rx = max(rx, exch[48 + w]);
         }
-        rs = row_scale_warp(amax_bits, rx, threadIdx.x & 31);
+        rs = FP ? row_scale_fp(amax_bits, rx) : row_scale_warp(amax_bits, rx, threadIdx.x & 31);
       }
     }
     if (lane == 0) {
@@ -709,7 +856,18 @@ __global__ void __launch_bounds__(B == 128 ? 256 : 512) encode_rows_kernel(const
     }
 
     // -------------------------------------------------------------- phase 2a: sparse component
-    {
+    if constexpr (FP) {
+      // E4M3 bytes of the selected values; their places in the staged row (zero until now) get
+      // the marker that carries the byte
+      uint8_t* vdst = reinterpret_cast<uint8_t*>(p.vals) + (size_t)m * GK;
+      for (int t = lane; t < GK; t += gsize) {
+        const uint32_t q = e4m3_of32(stash[t], rs.inv);
+        vdst[t] = (uint8_t)q;
+        row[spos[t]] = (uint16_t)fp_marker(q);
+      }
+      group_sync(rw, grp);
+      dense_sweep_fp(row, K, rs, p.dq4 + (size_t)m * (K / 2), p.a8 + (size_t)m * K, lane, gsize);
+    } else {
       int8_t* vdst = p.vals + (size_t)m * GK;
       if ((GK & 3) == 0) {
         for (int t4 = lane * 4; t4 < GK; t4 += gsize * 4) {
@@ -732,7 +890,7 @@ __global__ void __launch_bounds__(B == 128 ? 256 : 512) encode_rows_kernel(const
 
     // -------------------------------------------------------------- phase 2b: dense component
     // (the group barrier above also ordered the zeroing of the selected places before this sweep)
-    dense_sweep(row, K, rs, p.dq4 + (size_t)m * (K / 2), lane, gsize);
+    if constexpr (!FP) dense_sweep(row, K, rs, p.dq4 + (size_t)m * (K / 2), lane, gsize);
 
     // the row buffer is about to be refilled by the async proxy: order this group's generic
     // accesses before it
@@ -1204,24 +1362,20 @@ __global__ void __launch_bounds__(NT, 1) encode_static_ring_kernel(const EncodeP
     const float2 cc = make_float2(cq, cq), mm = make_float2(kMagic + 8.0f, kMagic + 8.0f);
     if constexpr (FP) {
       // E2M1 codes of the registers, eight nibbles per word, and (on request) the merged operand:
-      // the E4M3 byte of code * 2^e in element order, the selected places' bytes from the image
+      // the E4M3 byte of code * 2^e in element order, the selected places' bytes from the image.
+      // Codes by the row's seven thresholds, bytes by the row's table (see fp_steps).
       uint2* aw = want_a8 ? reinterpret_cast<uint2*>(p.a8 + (size_t)m_this * K) + slice * S8 + lane : nullptr;
       const uint2* iw = reinterpret_cast<const uint2*>(img) + slice * S8 + lane;
+      const FpSteps st = fp_steps(cq, rs.e, lane);
 #pragma unroll
       for (int c = 0; c < NCL; ++c) {
-        const uint32_t w[4] = {v[c].x, v[c].y, v[c].z, v[c].w};
-        uint32_t nib = 0, by[2] = {0, 0};
-#pragma unroll
-        for (int q = 0; q < 8; ++q) {
-          const uint32_t h = (w[q >> 1] >> (16 * (q & 1))) & 0xFFFFu;
-          const uint32_t code = e2m1_of32(h, cq);
-          nib |= code << (4 * q);
-          by[q >> 2] |= e4m3_of_e2m1(code, rs.e) << (8 * (q & 3));
-        }
+        const uint32_t c0 = fp_codes2(v[c].x, st), c1 = fp_codes2(v[c].y, st), c2 = fp_codes2(v[c].z, st), c3 = fp_codes2(v[c].w, st);
+        const uint32_t nib = ((c0 | (c0 >> 12)) & 0xFFu) | (((c1 | (c1 >> 12)) & 0xFFu) << 8) | (((c2 | (c2 >> 12)) & 0xFFu) << 16) |
+                             ((c3 | (c3 >> 12)) << 24);
         dst[c * 32] = nib;
         if (want_a8) {
-          const uint2 im = iw[c * 32];
-          aw[c * 32] = make_uint2(by[0] | im.x, by[1] | im.y);
+          const uint2 by = fp_bytes8(nib, st), im = iw[c * 32];
+          aw[c * 32] = make_uint2(by.x | im.x, by.y | im.y);
         }
       }
     } else if (want_a8) {
@@ -1467,12 +1621,12 @@ static cudaError_t device_and_sms(int* dev, int* sms) {
     }                                                                                                    \
   } while (0)
 
-template <int B, int KK>
+template <int B, int KK, bool FP = false>
 cudaError_t launch_rows(const EncodeParams& base, cudaStream_t st) {
   EncodeParams p = base;
   const int K = p.K, G = K / B, k = (KK == 0) ? p.k : KK;
   constexpr int kMaxWarps = (B == 128) ? 8 : 16;
-  const size_t side = (((size_t)G * k * 2) + 15) & ~(size_t)15;            // stash of selected raw values
+  const size_t side = ((((size_t)G * k * 2) + 15) & ~(size_t)15) * (FP ? 2 : 1);  // stash of selected raw values (and their places)
   const size_t table = (KK == 0) ? ((((size_t)G * k * 2) + 127) & ~(size_t)127) : 0;  // static offset table
   const size_t budget = 224 * 1024 - table;
   const size_t row = (size_t)K * 2;
@@ -1510,10 +1664,10 @@ cudaError_t launch_rows(const EncodeParams& base, cudaStream_t st) {
   int dev = 0, sms = 0;
   cudaError_t err = device_and_sms(&dev, &sms);
   if (err != cudaSuccess) return err;
-  SQ_ENSURE_SMEM((encode_rows_kernel<B, KK>), dev, smem);
+  SQ_ENSURE_SMEM((encode_rows_kernel<B, KK, FP>), dev, smem);
   int64_t blocks = (p.M + ngroups - 1) / ngroups;
   if (blocks > sms) blocks = sms;
-  encode_rows_kernel<B, KK><<<(unsigned)blocks, ngroups * rw * 32, smem, st>>>(p);
+  encode_rows_kernel<B, KK, FP><<<(unsigned)blocks, ngroups * rw * 32, smem, st>>>(p);
   return cudaGetLastError();
 }
 
@@ -1708,6 +1862,37 @@ cudaError_t launch_fp_encode_static_ring(int b, int k, const uint16_t* X, int64_
   p.group_stride = 0;
   p.mk = MulK{0xFFFFFFFFu, 2u, 32u, 256u, 65536u, 1u << 24, 16u, 1u};
   return launch_static_ring<false, true>(p, st);
+}
+
+// Floating-point variant, dynamic positions: the row-group kernel's selection with that format's
+// scales and roundings.  cudaErrorNotSupported = left to the variant's own kernel.
+cudaError_t launch_fp_encode_dynamic_rows(int b, int k, const uint16_t* X, int64_t M, int64_t K, const sq_encoded& out,
+                                          uint8_t* a8, int* status, cudaStream_t st) {
+  if (M < 1 || a8 == nullptr) return cudaErrorNotSupported;
+  EncodeParams p;
+  p.a8 = a8;
+  p.X = X;
+  p.positions = nullptr;
+  p.dq4 = out.dq4;
+  p.vals = out.vals;
+  p.idx = out.idx;
+  p.s_hi = out.s_hi;
+  p.s_lo = out.s_lo;
+  p.shift = out.shift;
+  p.status = status;
+  p.M = M;
+  p.K = (int)K;
+  p.k = k;
+  p.b = b;
+  p.nbuf = 1;
+  p.rw = 1;
+  p.group_stride = 0;
+  p.mk = MulK{0xFFFFFFFFu, 2u, 32u, 256u, 65536u, 1u << 24, 16u, 1u};
+#define SQ_DYN_FP(BB, KK_) \
+  if (b == BB && k == KK_) return launch_rows<BB, KK_, true>(p, st);
+  SQ_DYN_FP(32, 4) SQ_DYN_FP(64, 8) SQ_DYN_FP(128, 16) SQ_DYN_FP(64, 4) SQ_DYN_FP(128, 8) SQ_DYN_FP(32, 8) SQ_DYN_FP(64, 16) SQ_DYN_FP(128, 32)
+#undef SQ_DYN_FP
+  return cudaErrorNotSupported;
 }
 
 cudaError_t launch_decode(int b, int k, const sq_encoded& A, const uint8_t* positions, int64_t M,

@@ -68,6 +68,8 @@ cudaError_t launch_fp_encode(int b, int k, const uint16_t* X, int64_t M, int64_t
                              const sq_encoded& out, uint8_t* a8, cudaStream_t st);
 cudaError_t launch_fp_encode_static_ring(int b, int k, const uint16_t* X, int64_t M, int64_t K, const uint8_t* positions,
                                          const sq_encoded& out, uint8_t* a8, int* status, cudaStream_t st);
+cudaError_t launch_fp_encode_dynamic_rows(int b, int k, const uint16_t* X, int64_t M, int64_t K, const sq_encoded& out,
+                                          uint8_t* a8, int* status, cudaStream_t st);
 cudaError_t launch_fp_decode(int b, int k, const sq_encoded& A, const uint8_t* positions, int64_t M, int64_t K,
                              uint16_t* out, cudaStream_t st);
 cudaError_t launch_fp_gemm(const float* s_hi, const uint8_t* a8, const float* s_w, const uint8_t* w8, int64_t M, int64_t N,
