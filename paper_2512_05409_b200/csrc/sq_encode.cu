@@ -343,42 +343,6 @@ __device__ __forceinline__ RowScale row_scale_fp(uint32_t amax_bits, uint32_t rm
   rs.clamp = false;  // the code construction saturates by itself
   return rs;
 }
-// A selected place of the staged row carries its E4M3 byte in a non-finite pattern (exponent field
-// all ones, which no finite input has; the byte's sign in the sign bit, its other seven bits in the
-// mantissa), so that the dense pass finds the merged operand's byte there.
-__device__ __forceinline__ uint32_t fp_marker(uint32_t q) { return ((q & 0x80u) << 8) | 0x7F80u | (q & 0x7Fu); }
-// The dense pass over a staged row: E2M1 codes (eight nibbles per word; a selected place has code
-// 0) and the merged operand's E4M3 bytes in element order.
-__device__ __forceinline__ void dense_sweep_fp(const uint16_t* row, int K, const RowScale& rs, uint8_t* dq4_row, uint8_t* a8_row,
-                                               int lane, int gsize) {
-  const float c = rs.inv_lo;
-  const uint4* src = reinterpret_cast<const uint4*>(row) + lane;
-  uint32_t* dst = reinterpret_cast<uint32_t*>(dq4_row) + lane;
-  uint2* adst = reinterpret_cast<uint2*>(a8_row) + lane;
-  const int iters = (K / 8 - lane + gsize - 1) / gsize;
-#pragma unroll 2
-  for (int i = 0; i < iters; ++i, src += gsize, dst += gsize, adst += gsize) {
-    const uint4 v = *src;
-    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-    uint32_t nib = 0, by[2] = {0, 0};
-#pragma unroll
-    for (int q = 0; q < 8; ++q) {
-      const uint32_t h = (w[q >> 1] >> (16 * (q & 1))) & 0xFFFFu;
-      uint32_t code = 0, byte;
-      if ((h & 0x7F80u) == 0x7F80u) {
-        byte = ((h >> 8) & 0x80u) | (h & 0x7Fu);
-      } else {
-        code = e2m1_of32(h, c);
-        byte = e4m3_of_e2m1(code, rs.e);
-      }
-      nib |= code << (4 * q);
-      by[q >> 2] |= byte << (8 * (q & 3));
-    }
-    *dst = nib;
-    *adst = make_uint2(by[0], by[1]);
-  }
-}
-
 // The dense E2M1 code of a magnitude is a step function of the bf16 input: seven thresholds per
 // row decide it.  Threshold i = the smallest bf16 magnitude a whose exact product a * c reaches the
 // midpoint between the (i-1)-th and the i-th grid value (0, 0.5, 1, 1.5, 2, 3, 4, 6) -- reaches it
@@ -445,6 +409,45 @@ __device__ __forceinline__ uint2 fp_bytes8(uint32_t nib, const FpSteps& st) {
   const uint32_t sh = sg >> 16;
   by.y = prmt_u32(st.lut_lo, st.lut_hi, mags >> 16) | prmt_u32((sh << 4) & 0x8080u, 0u, 0x4140u) | prmt_u32(sh & 0x8080u, 0u, 0x1404u);
   return by;
+}
+
+// A selected place of the staged row carries its E4M3 byte in a NaN pattern (exponent field all
+// ones, which no finite input has; the byte's sign in the sign bit, its other seven bits,
+// complemented, in the mantissa: the byte's low seven bits never reach 0x7F, so the mantissa is
+// never zero and the pattern never an infinity).  Every threshold compare of fp_codes2 is false
+// for a NaN, so such a place gets code 0 by itself, and the dense pass finds the merged operand's
+// byte in the pattern.
+__device__ __forceinline__ uint32_t fp_marker(uint32_t q) { return ((q & 0x80u) << 8) | 0x7F80u | ((q & 0x7Fu) ^ 0x7Fu); }
+__device__ __forceinline__ uint32_t nan2_mask(uint32_t a) {  // 0xFFFF per half that holds a NaN
+  uint32_t d;
+  asm("set.nan.u32.bf16x2 %0, %1, %1;" : "=r"(d) : "r"(a));
+  return d;
+}
+// The bytes carried by the markers among four staged elements (two words), zero elsewhere.
+__device__ __forceinline__ uint32_t fp_marker_bytes4(uint32_t w0, uint32_t w1) {
+  const uint32_t lo4 = prmt_u32(w0, w1, 0x6420u), hi4 = prmt_u32(w0, w1, 0x7531u);  // low / high bytes of the four
+  const uint32_t mk4 = prmt_u32(nan2_mask(w0), nan2_mask(w1), 0x6420u);
+  return (((lo4 ^ 0x7F7F7F7Fu) & 0x7F7F7F7Fu) | (hi4 & 0x80808080u)) & mk4;
+}
+// The dense pass over a staged row: E2M1 codes (eight nibbles per word; a selected place has code
+// 0) and the merged operand's E4M3 bytes in element order.
+__device__ __forceinline__ void dense_sweep_fp(const uint16_t* row, int K, const RowScale& rs, uint8_t* dq4_row, uint8_t* a8_row,
+                                               int lane, int gsize) {
+  const FpSteps st = fp_steps(rs.inv_lo, rs.e, lane & 31);
+  const uint4* src = reinterpret_cast<const uint4*>(row) + lane;
+  uint32_t* dst = reinterpret_cast<uint32_t*>(dq4_row) + lane;
+  uint2* adst = reinterpret_cast<uint2*>(a8_row) + lane;
+  const int iters = (K / 8 - lane + gsize - 1) / gsize;
+#pragma unroll 2
+  for (int i = 0; i < iters; ++i, src += gsize, dst += gsize, adst += gsize) {
+    const uint4 v = *src;
+    const uint32_t c0 = fp_codes2(v.x, st), c1 = fp_codes2(v.y, st), c2 = fp_codes2(v.z, st), c3 = fp_codes2(v.w, st);
+    const uint32_t nib = ((c0 | (c0 >> 12)) & 0xFFu) | (((c1 | (c1 >> 12)) & 0xFFu) << 8) | (((c2 | (c2 >> 12)) & 0xFFu) << 16) |
+                         ((c3 | (c3 >> 12)) << 24);
+    const uint2 by = fp_bytes8(nib, st);
+    *dst = nib;
+    *adst = make_uint2(by.x | fp_marker_bytes4(v.x, v.y), by.y | fp_marker_bytes4(v.z, v.w));
+  }
 }
 
 struct EncodeParams {

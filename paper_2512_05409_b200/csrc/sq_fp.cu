@@ -78,11 +78,12 @@ __global__ void __launch_bounds__(256) fp_pack_weights_kernel(const uint16_t* __
   }
 }
 
-// One block per token row, the row staged in shared memory (the plain organisation of the integer
-// path's general kernel).  Dynamic positions: a warp per bank finds the k-th largest magnitude by
-// a bitwise search on warp-wide counts; codes by single-precision magic-number rounding; a
-// selected place is marked in the staged row by a non-finite pattern that carries its byte, so the
-// dense pass writes whole words of nibbles and of the merged operand.
+// Plain encoder for the formats and row lengths the integer path's fast kernels do not take (those
+// kernels, templated on the format, encode the rest: sq_encode.cu).  One block per token row, the
+// row staged in shared memory.  Dynamic positions: a warp per bank finds the k-th largest
+// magnitude by a bitwise search on warp-wide counts; codes by single-precision magic-number
+// rounding; a selected place is marked in the staged row by a non-finite pattern that carries its
+// byte, so the dense pass writes whole words of nibbles and of the merged operand.
 template <int B>
 __global__ void __launch_bounds__(256) fp_encode_kernel(int k, const uint16_t* __restrict__ X, int64_t K,
                                                         const uint8_t* __restrict__ positions, uint8_t* __restrict__ dq4,
