@@ -110,6 +110,33 @@ def test_fp_static_encode_staged_rows(K, b, k):
 
 
 @pytest.mark.parametrize("static", [False, True])
+def test_fp_dense_codes_at_every_input_near_the_grid(static):
+    """The dense codes come from per-row thresholds on the bf16 input.  Every row here holds EVERY
+    bf16 magnitude of the eleven binades below its maximum (both signs), so for each of 192 row
+    scales every input next to every rounding boundary is present: a threshold off by one input,
+    or a tie sent the wrong way, changes a code."""
+    b, k, K, M = 64, 8, 4096, 192
+    rng = np.random.default_rng(7)
+    rows = np.zeros((M, K), dtype=np.uint16)
+    for r in range(M):
+        top = int(rng.integers(0x3000, 0x4F00))            # the row maximum's bf16 pattern (2^-31 .. 2^31)
+        mags = np.arange(top - 11 * 128, top + 1, dtype=np.int64)   # eleven binades of consecutive patterns
+        vals = np.concatenate([mags, mags | 0x8000]).astype(np.uint16)
+        rng.shuffle(vals)
+        row = np.resize(vals, K)
+        row[int(rng.integers(0, K))] = top
+        rows[r] = row
+    X = torch.from_numpy(rows.view(np.int16)).view(torch.bfloat16).cuda()
+    fmt = sq.make_format(b, k, static)
+    pos = None
+    if static:
+        pos = torch.arange(k, dtype=torch.uint8, device="cuda").mul(7).remainder(b).sort().values.repeat(K // b, 1).contiguous()
+    enc, a8 = sq.sq_fp_encode(fmt, X, pos)
+    assert sq.sq_device_status() == sq.SQ_OK
+    _compare_encoded(enc, a8, oracle.fp_encode(b, k, rows, None if pos is None else _np(pos)))
+
+
+@pytest.mark.parametrize("static", [False, True])
 def test_fp_full_size_sweep_shape(static):
     """M = 4096, K = N = 8192 (the format-sweep shape): every row's encoding in full, GEMM on sampled
     rows x channels."""
