@@ -26,8 +26,8 @@
 //   warps 5-8   warp x widens the activation tile (nibble * 2^e + bias, unsigned, offset 128) of
 //               steps x, x + 4, ... into a ring of eight small shared-memory stages of its own and
 //               merges the step's sparse INT8 entries into the bytes they belong to
-//   warps 9, 14 one thread each issues tcgen05.mma.kind::i8 (A from tensor memory, M = 128
-//               channels; B from shared memory, N = 16 tokens) for alternate steps, into an
+//   warps 9,    one thread each issues tcgen05.mma.kind::i8 (A from tensor memory, M = 128
+//   14, 19      channels; B from shared memory, N = 16 tokens) for every third step, into an
 //               accumulator of its own, and frees both operands' stages with ONE commit per step
 //   warps 10-13 read the accumulators (lane = channel) once the K walk is over
 //   work item   (slab of 128 output channels, part of K).  The parts of a slab form one
@@ -59,8 +59,9 @@ constexpr int NPK = 4;         // packed stages in flight
 constexpr int NW = 6;          // widened weight stages (in tensor memory)
 constexpr int NX = 8;          // widened activation stages
 constexpr int kWGroups = 2, kWGroupThreads = 128, kXWarps = 4;
-constexpr int kTmaWarp = 0, kFirstW = 1, kFirstX = 5, kMmaWarp = 9, kFirstEpi = 10, kMma2Warp = 14, kFirstW2 = 15;
-constexpr int kThreadsS = 19 * 32;
+constexpr int kTmaWarp = 0, kFirstW = 1, kFirstX = 5, kMmaWarp = 9, kFirstEpi = 10, kMma2Warp = 14, kFirstW2 = 15, kMma3Warp = 19;
+constexpr int kIssuers = 3;     // MMA-issuing threads (steps j, j + 3, ... into accumulator j)
+constexpr int kThreadsS = 20 * 32;
 constexpr int ND = 24;         // "step done" barriers: a common multiple of NW and NX
 constexpr int kCtlBars = 512;
 constexpr int kCtlS = kCtlBars + 2 * SC * 4 + MT * 4;  // barriers, then the slab's constants for the finish
@@ -70,7 +71,7 @@ constexpr int kPackX = MT * kPitch;        // 4 KB
 constexpr int kSide = MT * SUP * 64;       // sparse values / indices of a stage: up to 64 per row and step
 constexpr int kPackStage = kPackW + kPackX + 2 * kSide;
 constexpr int kColsW = BK / 4;              // tensor-memory columns of a widened weight stage (128 lanes x 128 bytes)
-constexpr int kAccCols = 2 * MT;           // the two accumulators
+constexpr int kAccCols = kIssuers * MT;    // one accumulator per issuing thread
 constexpr int kStageX = MT * BK;           // 2 KB
 constexpr int kSmemS = NX * kStageX + NPK * kPackStage + kCtlS;
 static_assert(kStageX % 1024 == 0 && kPackStage % 1024 == 0 && (NX * kStageX) % 1024 == 0 && SUP <= 2, "stage alignment (swizzled weight tiles)");
@@ -191,7 +192,7 @@ __global__ void __launch_bounds__(kThreadsS, 2)
       mbar_init(bar_xfull + 8 * s, 32);
     }
     for (int s = 0; s < ND; ++s) mbar_init(bar_done + 8 * s, 1);
-    mbar_init(bar_tfull, KS >= 2 ? 2 : 1);  // one arrival per issuing thread that has steps
+    mbar_init(bar_tfull, KS >= kIssuers ? kIssuers : KS);  // one arrival per issuing thread that has steps
     *abort_flag = 0;
     fence_mbar_init();
   }
@@ -230,7 +231,7 @@ __global__ void __launch_bounds__(kThreadsS, 2)
       }
     }
     __syncwarp();
-  } else if ((warp >= kFirstW && warp < kFirstX) || warp >= kFirstW2) {
+  } else if ((warp >= kFirstW && warp < kFirstX) || (warp >= kFirstW2 && warp < kMma3Warp)) {
     // =============================================================== weights: group g takes steps g, g + 2, ...
     // A thread owns one output channel (its tensor-memory lane: quarter warp % 4, lane): it reads the
     // channel's 64 packed bytes of the step (the tile was laid down with the 64-byte swizzle, so the
@@ -354,16 +355,16 @@ __global__ void __launch_bounds__(kThreadsS, 2)
       fence_proxy_async_smem();
       mbar_arrive(bar_xfull + 8 * sx);
     }
-  } else if (warp == kMmaWarp || warp == kMma2Warp) {
+  } else if (warp == kMmaWarp || warp == kMma2Warp || warp == kMma3Warp) {
     // =============================================================== MMA issuers
     // A K step is four small instructions, but waiting for its two operands, issuing and
     // committing take one thread ~0.5 us: that, not the stream, set the pace of the whole kernel.
-    // So TWO threads issue, one the even steps and one the odd ones, each into an accumulator of
-    // its own (the sums are integers: the finish adds the two, in any order the same).
+    // So THREE threads issue, thread j the steps j, j + 3, ..., each into an accumulator of its own
+    // (the sums are integers: the finish adds them, in any order the same).
     if (lane == 0) {
-      const int j = warp == kMmaWarp ? 0 : 1;
+      const int j = warp == kMmaWarp ? 0 : (warp == kMma2Warp ? 1 : 2);
       bool ok = true;
-      for (int ks = j; ks < KS && ok; ks += 2) {
+      for (int ks = j; ks < KS && ok; ks += kIssuers) {
         const int s = ks % NW, sx = ks % NX;
         ok = mbar_wait_park(bar_wfull + 8 * s, (ks / NW) & 1u, abort_flag) && mbar_wait_park(bar_xfull + 8 * sx, (ks / NX) & 1u, abort_flag);
         if (!ok) break;
@@ -395,13 +396,15 @@ __global__ void __launch_bounds__(kThreadsS, 2)
       int4* prow = reinterpret_cast<int4*>(sPack) + ch * (MT / 4);
       uint32_t v[16];
       tmem_ld16(tmem + ((uint32_t)(32 * q) << 16), v);
-      if (KS >= 2) {  // the odd steps' accumulator
-        uint32_t v2[16];
-        tmem_ld16(tmem + ((uint32_t)(32 * q) << 16) + (uint32_t)MT, v2);
-        tmem_ld_wait();
 #pragma unroll
-        for (int c = 0; c < 16; ++c) v[c] += v2[c];
-      }
+      for (int j = 1; j < kIssuers; ++j)
+        if (KS > j) {  // the other issuing threads' accumulators
+          uint32_t v2[16];
+          tmem_ld16(tmem + ((uint32_t)(32 * q) << 16) + (uint32_t)(j * MT), v2);
+          tmem_ld_wait();
+#pragma unroll
+          for (int c = 0; c < 16; ++c) v[c] += v2[c];
+        }
       tmem_ld_wait();
       // (a warp's 16-byte stores, one 64-byte row per lane, spread over the banks by themselves)
       prow[0] = make_int4((int)v[0], (int)v[1], (int)v[2], (int)v[3]);
