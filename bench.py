@@ -217,10 +217,24 @@ def bench_encode_only(sq, dev, peaks, iters=50, warmup=10):
             copy_gbs = nbytes / (cms * 1e-3) / 1e9
             rows.append(["static" if static else "dynamic", k, round(ms * 1e3, 1), round(best * 1e3, 1), round(gbs),
                          round(gbs / peaks["hbm_gbs"], 3), round(gbs / 8000.0, 3), round(copy_gbs), round(gbs / copy_gbs, 3)])
+    # sq_decode of the same tensor (k = 8): packed codes in, bf16 out; three encodings in rotation
+    dec_rows = []
+    out = torch.empty(M, K, dtype=torch.bfloat16, device=dev)
+    for static in (False, True):
+        fmt = sq.make_format(64, 8, static)
+        pos = sq.sq_calib_positions(fmt, calib) if static else None
+        encs = [sq.sq_encode(fmt, Xs[i], pos) for i in range(3)]
+        ms, best = time_launches(lambda i: sq.sq_decode(fmt, encs[i % 3], pos, out=out), iters, warmup)
+        nbytes = M * K * (2.0 + 0.5 + (1.0 if static else 2.0) * 8 / 64) + 8.0 * M
+        gbs = nbytes / (ms * 1e-3) / 1e9
+        dec_rows.append(["static" if static else "dynamic", 8, round(ms * 1e3, 1), round(best * 1e3, 1), round(gbs),
+                         round(gbs / peaks["hbm_gbs"], 3)])
+        del encs
     return {"cols": ["positions", "k", "us_median", "us_best", "GBps", "of_measured_hbm", "of_8TBps",
                      "same_run_copy_GBps", "of_same_run_copy"],
             "rows": rows, "launches": iters,
-            "traffic_ncu_bytes_per_launch_k8": ENCODE_TRAFFIC_BYTES_PER_LAUNCH}
+            "traffic_ncu_bytes_per_launch_k8": ENCODE_TRAFFIC_BYTES_PER_LAUNCH,
+            "decode": {"cols": ["positions", "k", "us_median", "us_best", "GBps", "of_measured_hbm"], "rows": dec_rows}}
 
 
 def graph_replay_us(fn, calls=10, replays=5):

@@ -1575,14 +1575,28 @@ __global__ void __launch_bounds__(256) decode_kernel(int b, int k, const uint8_t
   __shared__ uint32_t pair_tab[256];  // the two bf16 values of every possible byte of codes, for this row's scale
   const int tid = threadIdx.x;
   const int64_t m = blockIdx.x;
+  const int64_t G = K / b, GK = G * k;
+  const int8_t* vrow = vals + m * GK;
+  const uint8_t* irow = idx != nullptr ? idx + m * GK : positions;
+  const bool words = (GK & 3) == 0 && ((reinterpret_cast<uintptr_t>(vrow) | reinterpret_cast<uintptr_t>(irow)) & 3) == 0;
+  // every global read of this thread's first pass is issued before anything waits for one of them:
+  // a block pays one memory latency, not three in a row
   const float sl = s_lo[m], sh = s_hi[m];
+  const int64_t i0 = (int64_t)tid * 32, t0 = (int64_t)tid * 4;
+  uint4 c0 = make_uint4(0, 0, 0, 0);
+  uint32_t vw0 = 0, iw0 = 0;
+  if (i0 < K) c0 = *reinterpret_cast<const uint4*>(dq4 + m * (K / 2) + i0 / 2);
+  if (words && t0 < GK) {
+    vw0 = *reinterpret_cast<const uint32_t*>(vrow + t0);
+    iw0 = *reinterpret_cast<const uint32_t*>(irow + t0);
+  }
   {
     const int n0 = ((int)((uint32_t)tid << 28)) >> 28, n1 = ((int)((uint32_t)tid << 24)) >> 28;  // sign-extended nibbles
     pair_tab[tid] = f32_to_bf16_bits(sl * (float)n0) | (f32_to_bf16_bits(sl * (float)n1) << 16);
   }
   __syncthreads();
-  for (int64_t i = (int64_t)tid * 32; i < K; i += 256 * 32) {  // 16 bytes of codes -> 32 values
-    const uint4 c = *reinterpret_cast<const uint4*>(dq4 + m * (K / 2) + i / 2);
+  for (int64_t i = i0; i < K; i += 256 * 32) {  // 16 bytes of codes -> 32 values
+    const uint4 c = i == i0 ? c0 : *reinterpret_cast<const uint4*>(dq4 + m * (K / 2) + i / 2);
     const uint32_t w[4] = {c.x, c.y, c.z, c.w};
 #pragma unroll
     for (int q = 0; q < 4; ++q)
@@ -1590,12 +1604,10 @@ __global__ void __launch_bounds__(256) decode_kernel(int b, int k, const uint8_t
                                                              pair_tab[(w[q] >> 16) & 0xFFu], pair_tab[w[q] >> 24]);
   }
   __syncthreads();
-  const int64_t G = K / b, GK = G * k;
-  const int8_t* vrow = vals + m * GK;
-  const uint8_t* irow = idx != nullptr ? idx + m * GK : positions;
-  if ((GK & 3) == 0 && ((reinterpret_cast<uintptr_t>(vrow) | reinterpret_cast<uintptr_t>(irow)) & 3) == 0) {
-    for (int64_t t4 = (int64_t)tid * 4; t4 < GK; t4 += 256 * 4) {  // four entries per pair of 4-byte reads
-      const uint32_t vw = *reinterpret_cast<const uint32_t*>(vrow + t4), iw = *reinterpret_cast<const uint32_t*>(irow + t4);
+  if (words) {
+    for (int64_t t4 = t0; t4 < GK; t4 += 256 * 4) {  // four entries per pair of 4-byte reads
+      const uint32_t vw = t4 == t0 ? vw0 : *reinterpret_cast<const uint32_t*>(vrow + t4);
+      const uint32_t iw = t4 == t0 ? iw0 : *reinterpret_cast<const uint32_t*>(irow + t4);
 #pragma unroll
       for (int q = 0; q < 4; ++q) {
         const int64_t t = t4 + q;
