@@ -180,31 +180,28 @@ __global__ void __launch_bounds__(kThreadsS, 2)
   constexpr uint32_t kTmemCols = 256;  // 2 x 16 accumulator columns, then NW x 32 columns of widened weights
   static_assert(kAccCols + NW * kColsW <= 256, "tensor-memory columns");
 
-  if (tid == 0) {
-    for (int s = 0; s < NPK; ++s) {
-      mbar_init(bar_pfull + 8 * s, 1);
-      mbar_init(bar_pempty + 8 * s, SUP * (kWGroupThreads + 32));
+  if (warp == kTmaWarp) {
+    if (lane == 0) {  // the descriptors are on their way while the barriers are set up
+      asm volatile("prefetch.tensormap [%0];" ::"l"(&map_w4) : "memory");
+      asm volatile("prefetch.tensormap [%0];" ::"l"(&map_x4) : "memory");
+      asm volatile("prefetch.tensormap [%0];" ::"l"(&map_sv) : "memory");
+      asm volatile("prefetch.tensormap [%0];" ::"l"(&map_si) : "memory");
+      *abort_flag = 0;
     }
-    for (int s = 0; s < NW; ++s) {
-      mbar_init(bar_wfull + 8 * s, kWGroupThreads);
+    // the barriers sit one after another in shared memory: the warp's lanes set them up side by side
+    for (int i = lane; i < kBars; i += 32) {
+      uint32_t count = 1;                                             // pfull, step done
+      if (i >= NPK && i < 2 * NPK) count = SUP * (kWGroupThreads + 32);  // pempty
+      else if (i >= 2 * NPK && i < 2 * NPK + NW) count = kWGroupThreads;  // wfull
+      else if (i >= 2 * NPK + NW && i < 2 * NPK + NW + NX) count = 32;    // xfull
+      else if (i == kBars - 1) count = KS >= kIssuers ? kIssuers : KS;    // tfull: one arrival per issuing thread that has steps
+      mbar_init(bar_pfull + 8 * i, count);
     }
-    for (int s = 0; s < NX; ++s) {
-      mbar_init(bar_xfull + 8 * s, 32);
-    }
-    for (int s = 0; s < ND; ++s) mbar_init(bar_done + 8 * s, 1);
-    mbar_init(bar_tfull, KS >= kIssuers ? kIssuers : KS);  // one arrival per issuing thread that has steps
-    *abort_flag = 0;
     fence_mbar_init();
   }
   if (warp == kMmaWarp) {
     tmem_alloc<1>(smem_u32(tmem_slot), kTmemCols);
     tmem_relinquish<1>();
-  }
-  if (warp == kTmaWarp && lane == 0) {  // the descriptors are on their way while the barriers are set up
-    asm volatile("prefetch.tensormap [%0];" ::"l"(&map_w4) : "memory");
-    asm volatile("prefetch.tensormap [%0];" ::"l"(&map_x4) : "memory");
-    asm volatile("prefetch.tensormap [%0];" ::"l"(&map_sv) : "memory");
-    asm volatile("prefetch.tensormap [%0];" ::"l"(&map_si) : "memory");
   }
   tc_fence_before();
   __syncthreads();
