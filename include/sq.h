@@ -268,6 +268,10 @@ sq_status sq_gemm_a8(const sq_format* fmt, const sq_encoded* A, const sq_weights
  *     or 8) as fit the array.
  *   - The first call on each device looks up the array's device address (that device must
  *     be current, as for every call here); make that first call before any stream capture.
+ *     The CUDA runtime loads a library's GPU code lazily, so it is also this first call at
+ *     which the driver sets the array's 16 MiB aside on that device (unless another call
+ *     into the same part of the library has done so before): a host that must know its
+ *     memory budget up front makes one call per device during start-up.
  *   - All calls share the one array.  It keeps whatever the previous call left there, which
  *     is harmless: every element a call reads it has written itself first.  But two calls
  *     that overlap on the GPU (different streams, no ordering between them) race on it:
