@@ -353,6 +353,23 @@ def bench_same_run_int8(dev, iters=10):
         return None
 
 
+def bench_int8_tensor_rate(sq):
+    """The library's tensor-rate probe (tcgen05.mma.kind::i8 on shared-memory-resident operands and
+    nothing else, one CTA per SM) timed in the same run: the INT8 rate the tensor pipe itself
+    sustains -- for ~5 ms (boost clocks) and for a quarter of a second (under the power cap)."""
+    def once(iters):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        ops = sq.sq_probe_int8_tensor_rate(iters)
+        b.record()
+        torch.cuda.synchronize()
+        return ops / (a.elapsed_time(b) * 1e-3) / 1e12
+    once(2000)
+    burst = statistics.median(once(20000) for _ in range(5))
+    sustained = once(1000000)
+    return burst, sustained
+
+
 def bench_format_sweep(sq, dev, peaks, iters=5):
     """The format-parameter sweep at M = 4096, K = N = 8192: bank b in {32, 64, 128} x high-precision
     fraction k/b in {1/16, 1/8, 1/4}, dynamic positions, static positions and static positions with
@@ -700,9 +717,15 @@ def run_cuda(args):
             line["weights_sq"] = {"workload": "weights in SQ-format (implicit mask, b=64, k=8) x per-token INT8 activations, 8B-decoder shapes, 1 and 4 tokens",
                                   **bench_weights_sq(sq, dev, peaks)}
             same = bench_same_run_int8(dev)
+            burst, sustained = bench_int8_tensor_rate(sq)
             line["same_run"] = {"int8_gemm_TOPS": None if same is None else round(same, 1),
                                 "what": "torch._int_mm M=4096 N=K=8192 (vendor INT8 GEMM, yardstick only)",
-                                "roofline_frac_of_same_run_int8": None if same is None else round(gemm_tops / same, 3)}
+                                "roofline_frac_of_same_run_int8": None if same is None else round(gemm_tops / same, 3),
+                                "int8_mma_only_TOPS": round(burst, 1), "int8_mma_only_sustained_TOPS": round(sustained, 1),
+                                "mma_only_what": "sq_probe_int8_tensor_rate: tcgen05.mma.kind::i8 128x256x32 on resident operands, nothing else, one CTA per SM; ~5 ms launches (median of 5) and one ~0.25 s launch",
+                                "roofline_frac_of_mma_only": round(gemm_tops / burst, 3),
+                                "roofline_frac_of_mma_only_sustained": round(gemm_tops / sustained, 3)}
+            line["roofline"]["frac_of_mma_only_same_run"] = round(gemm_tops / burst, 3)
         if not args.no_cpu_baseline and world == 1:
             K, N = SHAPES_70B[1]
             ops = dt = 0.0

@@ -356,6 +356,16 @@ sq_status sq_device_status(void* cuda_stream);
  * remains the call that clears it.  *device_word is a DEVICE pointer. */
 sq_status sq_device_status_word(int** device_word);
 
+/* Measurement aid (the paper has no counterpart): the rate at which this GPU's tensor cores take
+ * the product's own instruction.  One CTA per SM issues `iterations` K steps of
+ * tcgen05.mma.kind::i8 (128 x 256 x 128 per step) on operands resident in shared memory -- no
+ * loads, no widening, no epilogue -- asynchronously on the stream.  *int8_ops (host pointer, may be
+ * NULL) receives the number of INT8 operations the launch issues (2 per multiply-add); divided
+ * by the launch's device time (CUDA events around the call) it is the INT8 tensor rate a
+ * tensor-bound kernel can reach at the clocks of that moment.  1 <= iterations <= 2^24.
+ * Uses all of tensor memory on every SM while it runs: not to be overlapped with other calls. */
+sq_status sq_probe_int8_tensor_rate(int iterations, double* int8_ops, void* cuda_stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -75,6 +75,7 @@ def _load() -> ctypes.CDLL:
     lib.sq_gemm_static_scratch.argtypes = [P(sq_format), P(sq_encoded), P(sq_weights), VP, I64, I64, I64, VP, VP, VP]
     lib.sq_decode.argtypes = [P(sq_format), P(sq_encoded), VP, I64, I64, VP, VP]
     lib.sq_device_status.argtypes = [VP]
+    lib.sq_probe_int8_tensor_rate.argtypes = [ctypes.c_int, P(ctypes.c_double), VP]
     lib.sq_fp_pack_weights.argtypes = [VP, I64, I64, VP, VP, VP, VP]
     lib.sq_fp_encode.argtypes = [P(sq_format), VP, I64, I64, VP, P(sq_encoded), VP, VP]
     lib.sq_fp_gemm.argtypes = [VP, VP, VP, VP, I64, I64, I64, VP, VP, VP]
@@ -452,6 +453,14 @@ def sq_w_gemm(fmt: sq_format, xq: torch.Tensor, s_x: torch.Tensor, W: SqWeights,
     _check(_lib.sq_w_gemm(ctypes.byref(fmt), _ptr(xq), _ptr(s_x), _ptr(W.wq4), _ptr(W.w_hi), _ptr(W.s_high),
                           _ptr(W.s_low), M, N, K, _ptr(out), _ptr(acc_out), _stream(stream)), "sq_w_gemm")
     return out
+
+
+def sq_probe_int8_tensor_rate(iterations: int, stream=None) -> float:
+    """Launches the tensor-rate probe (tcgen05.mma.kind::i8 on resident operands, nothing else);
+    returns the number of INT8 operations the launch issues.  Time it with CUDA events."""
+    ops = ctypes.c_double(0.0)
+    _check(_lib.sq_probe_int8_tensor_rate(int(iterations), ctypes.byref(ops), _stream(stream)), "sq_probe_int8_tensor_rate")
+    return ops.value
 
 
 def sq_device_status_word() -> int:

@@ -1545,6 +1545,79 @@ cudaError_t launch_gemm(int b, int k, bool indep, const sq_encoded& A, const sq_
 }
 
 // ------------------------------------------------------------------------------------------------
+// Measurement aid: the rate at which the tensor core itself takes the product's instruction.  One
+// CTA per SM issues tcgen05.mma.kind::i8 (128 x 256 x 32, the tiled kernel's instruction) on
+// operands that sit in shared memory and are never reloaded, into the two accumulators in turn,
+// and does nothing else: no loads, no widening, no epilogue.  Timed by the caller, it gives the
+// INT8 rate the tensor pipe sustains at the clocks of that moment -- the denominator a
+// tensor-bound kernel can be held against on this GPU.
+__global__ void __launch_bounds__(128, 1) int8_peak_kernel(int iters, int* status) {
+  extern __shared__ __align__(1024) uint8_t smem_pk[];  // A: 128 rows x 128 B | B: 256 rows x 128 B
+  __shared__ uint64_t bar_s;
+  __shared__ uint32_t tmem_slot_s;
+  __shared__ int abort_s;
+  const int tid = threadIdx.x, warp = tid >> 5;
+  if ((smem_u32(smem_pk) & 1023u) != 0) {
+    if (tid == 0) atomicExch(status, (int)SQ_ERR_CUDA);
+    return;
+  }
+  // (operands of mixed bits rather than zeros, so that the datapath toggles as it does in a real product)
+  for (int i = tid; i < (BM + BN) * BK / 16; i += 128) {
+    const uint32_t h = (uint32_t)i * 2654435761u;
+    reinterpret_cast<uint4*>(smem_pk)[i] = make_uint4(h, h * 2246822519u, h ^ 0x9E3779B9u, ~h * 3266489917u);
+  }
+  fence_proxy_async_smem();
+  const uint32_t bar = smem_u32(&bar_s);
+  if (tid == 0) {
+    mbar_init(bar, 1);
+    abort_s = 0;
+    fence_mbar_init();
+  }
+  if (warp == 0) {
+    tmem_alloc<1>(smem_u32(&tmem_slot_s), 2 * BN);
+    tmem_relinquish<1>();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = tmem_slot_s;
+  if (tid == 0) {
+    const uint64_t da = make_desc(smem_u32(smem_pk)), db = make_desc(smem_u32(smem_pk + BM * BK));
+    constexpr uint32_t idesc = make_idesc(false, BM);
+    uint32_t phase = 0;
+    bool ok = true;
+    for (int it = 0; it < iters && ok; ++it) {
+#pragma unroll
+      for (int kk = 0; kk < BK / 32; ++kk) umma_i8<1>(tmem + (uint32_t)((it & 1) * BN), da + 2 * kk, db + 2 * kk, idesc, 1u);
+      if ((it & 63) == 63 || it == iters - 1) {  // a bounded wait every 256 instructions keeps the queue shallow
+        umma_commit<1>(bar);
+        ok = mbar_wait(bar, phase, &abort_s);
+        phase ^= 1u;
+      }
+    }
+    if (!ok) atomicExch(status, (int)SQ_ERR_TIMEOUT);
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 0) tmem_dealloc<1>(tmem, 2 * BN);
+}
+
+// Launches the probe on every SM; *ops = the INT8 operations (2 per multiply-add) the launch issues.
+cudaError_t launch_int8_peak_probe(int iters, double* ops, int* status, cudaStream_t st) {
+  int dev = 0, sms = 0;
+  cudaError_t err = cudaGetDevice(&dev);
+  if (err != cudaSuccess) return err;
+  err = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  if (err != cudaSuccess) return err;
+  const int smem = (BM + BN) * BK;
+  err = cudaFuncSetAttribute(int8_peak_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  if (err != cudaSuccess) return err;
+  if (ops != nullptr) *ops = 2.0 * BM * BN * BK * (double)iters * (double)sms;
+  int8_peak_kernel<<<(unsigned)sms, 128, smem, st>>>(iters, status);
+  return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------------------------------------
 // Split-K scratch that nobody has to allocate: a fixed array in the library's device image.
 // Every GPU that loads the library holds these 16 MiB until the process exits.
 constexpr size_t kStaticScratchBytes = (size_t)16 << 20;
