@@ -600,3 +600,18 @@ def test_merged_operand_rejects_independent_scales():
     pos = torch.arange(8, dtype=torch.uint8, device="cuda").repeat(1024 // 64)
     with pytest.raises(sq.SqError):
         sq.sq_encode_a8(fmt, X, pos)
+
+
+# ----------------------------------------------------------------------------- measurement aid
+
+def test_tensor_rate_probe_runs_and_counts_its_operations():
+    """The probe issues iterations x 128 x 256 x 128 multiply-adds on every SM, leaves the status word
+    alone and hands tensor memory back (a product call right after it works)."""
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    ops = sq.sq_probe_int8_tensor_rate(500)
+    torch.cuda.synchronize()
+    assert ops == 2.0 * 128 * 256 * 128 * 500 * sms
+    check_status()
+    with pytest.raises(sq.SqError):
+        sq.sq_probe_int8_tensor_rate(0)
+    run_pipeline(M=96, N=128, K=256, b=64, k=8, static=False, seed=11)
