@@ -367,7 +367,17 @@ def bench_int8_tensor_rate(sq):
     once(2000)
     burst = statistics.median(once(20000) for _ in range(5))
     sustained = once(1000000)
-    return burst, sustained
+
+    def once_fp8(iters):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        ops = sq.sq_probe_fp8_tensor_rate(iters)
+        b.record()
+        torch.cuda.synchronize()
+        return ops / (a.elapsed_time(b) * 1e-3) / 1e12
+    once_fp8(2000)
+    fp8_burst = statistics.median(once_fp8(20000) for _ in range(5))
+    return burst, sustained, fp8_burst
 
 
 def bench_format_sweep(sq, dev, peaks, iters=5):
@@ -717,15 +727,19 @@ def run_cuda(args):
             line["weights_sq"] = {"workload": "weights in SQ-format (implicit mask, b=64, k=8) x per-token INT8 activations, 8B-decoder shapes, 1 and 4 tokens",
                                   **bench_weights_sq(sq, dev, peaks)}
             same = bench_same_run_int8(dev)
-            burst, sustained = bench_int8_tensor_rate(sq)
+            burst, sustained, fp8_burst = bench_int8_tensor_rate(sq)
             line["same_run"] = {"int8_gemm_TOPS": None if same is None else round(same, 1),
                                 "what": "torch._int_mm M=4096 N=K=8192 (vendor INT8 GEMM, yardstick only)",
                                 "roofline_frac_of_same_run_int8": None if same is None else round(gemm_tops / same, 3),
                                 "int8_mma_only_TOPS": round(burst, 1), "int8_mma_only_sustained_TOPS": round(sustained, 1),
-                                "mma_only_what": "sq_probe_int8_tensor_rate: tcgen05.mma.kind::i8 128x256x32 on resident operands, nothing else, one CTA per SM; ~5 ms launches (median of 5) and one ~0.25 s launch",
+                                "mma_only_what": "sq_probe_int8_tensor_rate (and sq_probe_fp8_tensor_rate for kind::f8f6f4): tcgen05.mma 128x256x32 on resident operands, nothing else, one CTA per SM; ~5 ms launches (median of 5) and one ~0.25 s launch; fp_gemm_frac = [slowest, fastest] fp8/fp4 row of format_sweep over the fp8 rate",
+                                "fp8_mma_only_TFLOPS": round(fp8_burst, 1),
                                 "roofline_frac_of_mma_only": round(gemm_tops / burst, 3),
                                 "roofline_frac_of_mma_only_sustained": round(gemm_tops / sustained, 3)}
             line["roofline"]["frac_of_mma_only_same_run"] = round(gemm_tops / burst, 3)
+            if "format_sweep" in line:
+                fp_tops = [r[5] for r in line["format_sweep"]["rows"] if str(r[2]).startswith("fp8")]
+                line["same_run"]["fp_gemm_frac_of_fp8_mma_only"] = [round(min(fp_tops) / fp8_burst, 3), round(max(fp_tops) / fp8_burst, 3)]
         if not args.no_cpu_baseline and world == 1:
             K, N = SHAPES_70B[1]
             ops = dt = 0.0

@@ -365,6 +365,9 @@ sq_status sq_device_status_word(int** device_word);
  * tensor-bound kernel can reach at the clocks of that moment.  1 <= iterations <= 2^24.
  * Uses all of tensor memory on every SM while it runs: not to be overlapped with other calls. */
 sq_status sq_probe_int8_tensor_rate(int iterations, double* int8_ops, void* cuda_stream);
+/* The same probe for the floating-point variant's instruction (tcgen05.mma.kind::f8f6f4, E4M3 x
+ * E4M3, fp32 accumulation): *fp8_ops receives the floating-point operations of the launch. */
+sq_status sq_probe_fp8_tensor_rate(int iterations, double* fp8_ops, void* cuda_stream);
 
 #ifdef __cplusplus
 }

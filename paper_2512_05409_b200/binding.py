@@ -76,6 +76,7 @@ def _load() -> ctypes.CDLL:
     lib.sq_decode.argtypes = [P(sq_format), P(sq_encoded), VP, I64, I64, VP, VP]
     lib.sq_device_status.argtypes = [VP]
     lib.sq_probe_int8_tensor_rate.argtypes = [ctypes.c_int, P(ctypes.c_double), VP]
+    lib.sq_probe_fp8_tensor_rate.argtypes = [ctypes.c_int, P(ctypes.c_double), VP]
     lib.sq_fp_pack_weights.argtypes = [VP, I64, I64, VP, VP, VP, VP]
     lib.sq_fp_encode.argtypes = [P(sq_format), VP, I64, I64, VP, P(sq_encoded), VP, VP]
     lib.sq_fp_gemm.argtypes = [VP, VP, VP, VP, I64, I64, I64, VP, VP, VP]
@@ -460,6 +461,13 @@ def sq_probe_int8_tensor_rate(iterations: int, stream=None) -> float:
     returns the number of INT8 operations the launch issues.  Time it with CUDA events."""
     ops = ctypes.c_double(0.0)
     _check(_lib.sq_probe_int8_tensor_rate(int(iterations), ctypes.byref(ops), _stream(stream)), "sq_probe_int8_tensor_rate")
+    return ops.value
+
+
+def sq_probe_fp8_tensor_rate(iterations: int, stream=None) -> float:
+    """The same probe for tcgen05.mma.kind::f8f6f4 (E4M3 x E4M3); returns the launch's floating-point operations."""
+    ops = ctypes.c_double(0.0)
+    _check(_lib.sq_probe_fp8_tensor_rate(int(iterations), ctypes.byref(ops), _stream(stream)), "sq_probe_fp8_tensor_rate")
     return ops.value
 
 

@@ -476,6 +476,14 @@ sq_status sq_probe_int8_tensor_rate(int iterations, double* int8_ops, void* cuda
   return from_cuda(launch_int8_peak_probe(iterations, int8_ops, status, static_cast<cudaStream_t>(cuda_stream)));
 }
 
+sq_status sq_probe_fp8_tensor_rate(int iterations, double* fp8_ops, void* cuda_stream) {
+  if (iterations < 1 || iterations > (1 << 24)) return SQ_ERR_INVALID_ARG;
+  SQ_TRY(check_device());
+  int* status = status_word();
+  if (status == nullptr) return SQ_ERR_CUDA;
+  return from_cuda(launch_fp8_peak_probe(iterations, fp8_ops, status, static_cast<cudaStream_t>(cuda_stream)));
+}
+
 sq_status sq_device_status_word(int** device_word) {
   if (device_word == nullptr) return SQ_ERR_NULL_POINTER;
   SQ_TRY(check_device());

@@ -552,6 +552,75 @@ cudaError_t launch_fp_decode(int b, int k, const sq_encoded& A, const uint8_t* p
   return cudaGetLastError();
 }
 
+// Measurement aid, as the integer path's: the rate at which the tensor core takes this variant's
+// instruction (tcgen05.mma.kind::f8f6f4, E4M3 x E4M3, 128 x 256 x 32) on operands that stay in
+// shared memory; no loads, no epilogue.
+__global__ void __launch_bounds__(128, 1) fp8_peak_kernel(int iters, int* status) {
+  extern __shared__ __align__(1024) uint8_t smem_pk[];  // A: 128 rows x 128 B | B: 256 rows x 128 B
+  __shared__ uint64_t bar_s;
+  __shared__ uint32_t tmem_slot_s;
+  __shared__ int abort_s;
+  const int tid = threadIdx.x, warp = tid >> 5;
+  if ((smem_u32(smem_pk) & 1023u) != 0) {
+    if (tid == 0) atomicExch(status, (int)SQ_ERR_CUDA);
+    return;
+  }
+  // operands of mixed bits (small finite E4M3 values: the exponent's top bit stays clear)
+  for (int i = tid; i < (FBM + FBN) * FBK / 16; i += 128) {
+    const uint32_t h = (uint32_t)i * 2654435761u;
+    reinterpret_cast<uint4*>(smem_pk)[i] = make_uint4(h & 0xBFBFBFBFu, (h * 2246822519u) & 0xBFBFBFBFu, (h ^ 0x9E3779B9u) & 0xBFBFBFBFu,
+                                                      (~h * 3266489917u) & 0xBFBFBFBFu);
+  }
+  fence_proxy_async_smem();
+  const uint32_t bar = smem_u32(&bar_s);
+  if (tid == 0) {
+    mbar_init(bar, 1);
+    abort_s = 0;
+    fence_mbar_init();
+  }
+  if (warp == 0) {
+    tmem_alloc<1>(smem_u32(&tmem_slot_s), 2 * FBN);
+    tmem_relinquish<1>();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = tmem_slot_s;
+  if (tid == 0) {
+    const uint64_t da = fdesc(smem_u32(smem_pk)), db = fdesc(smem_u32(smem_pk + FBM * FBK));
+    constexpr uint32_t idesc = f_idesc(FBM);
+    uint32_t phase = 0;
+    bool ok = true;
+    for (int it = 0; it < iters && ok; ++it) {
+#pragma unroll
+      for (int kk = 0; kk < FBK / 32; ++kk) umma_f8<1>(tmem + (uint32_t)((it & 1) * FBN), da + 2 * kk, db + 2 * kk, idesc, 1u);
+      if ((it & 63) == 63 || it == iters - 1) {  // a bounded wait every 256 instructions keeps the queue shallow
+        umma_commit<1>(bar);
+        ok = mbar_wait(bar, phase, &abort_s);
+        phase ^= 1u;
+      }
+    }
+    if (!ok) atomicExch(status, (int)SQ_ERR_TIMEOUT);
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 0) tmem_dealloc<1>(tmem, 2 * FBN);
+}
+
+cudaError_t launch_fp8_peak_probe(int iters, double* ops, int* status, cudaStream_t st) {
+  int dev = 0, sms = 0;
+  cudaError_t err = cudaGetDevice(&dev);
+  if (err != cudaSuccess) return err;
+  err = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  if (err != cudaSuccess) return err;
+  const int smem = (FBM + FBN) * FBK;
+  err = cudaFuncSetAttribute(fp8_peak_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  if (err != cudaSuccess) return err;
+  if (ops != nullptr) *ops = 2.0 * FBM * FBN * FBK * (double)iters * (double)sms;
+  fp8_peak_kernel<<<(unsigned)sms, 128, smem, st>>>(iters, status);
+  return cudaGetLastError();
+}
+
 cudaError_t launch_fp_gemm(const float* s_hi, const uint8_t* a8, const float* s_w, const uint8_t* w8, int64_t M, int64_t N,
                            int64_t K, uint16_t* out, float* acc_out, int* status, cudaStream_t st) {
   static std::atomic<int> sm_count_of[64];

@@ -62,6 +62,7 @@ cudaError_t launch_gemm_static_scratch(int b, int k, const sq_encoded& A, const 
 size_t gemm_static_scratch_bytes();
 // Measurement aid: tcgen05.mma.kind::i8 on shared-memory-resident operands, nothing else (see sq.h).
 cudaError_t launch_int8_peak_probe(int iters, double* ops, int* status, cudaStream_t st);
+cudaError_t launch_fp8_peak_probe(int iters, double* ops, int* status, cudaStream_t st);
 
 // Floating-point variant (sq_fp.cu).
 cudaError_t launch_fp_pack_weights(const uint16_t* W, int64_t N, int64_t K, uint8_t* wq4, float* s_w, uint8_t* w8,

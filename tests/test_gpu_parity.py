@@ -615,3 +615,15 @@ def test_tensor_rate_probe_runs_and_counts_its_operations():
     with pytest.raises(sq.SqError):
         sq.sq_probe_int8_tensor_rate(0)
     run_pipeline(M=96, N=128, K=256, b=64, k=8, static=False, seed=11)
+
+
+def test_fp8_tensor_rate_probe_runs_and_counts_its_operations():
+    """The floating-point variant's probe: the same count, the status word clean, tensor memory handed back."""
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    ops = sq.sq_probe_fp8_tensor_rate(500)
+    torch.cuda.synchronize()
+    assert ops == 2.0 * 128 * 256 * 128 * 500 * sms
+    check_status()
+    with pytest.raises(sq.SqError):
+        sq.sq_probe_fp8_tensor_rate(0)
+    run_pipeline(M=96, N=128, K=256, b=64, k=8, static=False, seed=12)
