@@ -324,3 +324,52 @@ def w_gemm(b: int, k: int, xq: np.ndarray, s_x: np.ndarray, Wq: SqWeights):
     _load().sqo_w_gemm(ctypes.c_int(b), ctypes.c_int(k), _p(xq), _p(s_x), _p(Wq.wq4), _p(Wq.w_hi), _p(Wq.s_high),
                        _p(Wq.s_low), _l(M), _l(N), _l(K), _p(lo), _p(hi), _p(ref), _p(out))
     return lo, hi, ref, out
+
+
+# ---------------------------------------------------------------------------- the producer of an activation
+#
+# The decoder layers whose prefill the appendix "End-to-End Latency Analysis" times feed two of
+# their four quantised linears from a root-mean-square layer normalisation (y = x / rms(x) * gamma).
+# The paper does not spell the normalisation out; this is its usual definition with the roundings
+# of a bf16 decoder made explicit (the reading the CUDA path is held to):
+#   ms = (sum_j x_j^2) / K            in fp64 (every square of a bf16 value is exact there)
+#   r  = fp32(1 / sqrt(ms + eps))     one rounding to fp32
+#   t  = bf16(fp32(x) * r)            fp32 product, round-to-nearest-even to bf16
+#   y  = bf16(fp32(t) * fp32(gamma))  the product of two bf16 values is exact in fp32; one rounding
+# A row is "ambiguous" when 1/sqrt(ms + eps) lies so close to the middle between two fp32 values
+# that the order of the fp64 additions could decide r; callers assert there is none.
+
+def _bf16_rne_bits(f32: np.ndarray) -> np.ndarray:
+    u = np.ascontiguousarray(f32, dtype=np.float32).view(np.uint32).astype(np.uint64)
+    return ((u + 0x7FFF + ((u >> 16) & 1)) >> 16).astype(np.uint16)
+
+
+def rmsnorm(X_bits: np.ndarray, gamma_bits: np.ndarray, eps: float):
+    """(y bits uint16 [M,K], r float32 [M], ambiguous bool [M]) of the definition above."""
+    assert X_bits.dtype == np.uint16 and gamma_bits.dtype == np.uint16 and gamma_bits.shape == (X_bits.shape[1],)
+    M, K = X_bits.shape
+    x32 = (X_bits.astype(np.uint32) << 16).view(np.float32)
+    g32 = (gamma_bits.astype(np.uint32) << 16).view(np.float32)
+    x64 = x32.astype(np.float64)
+    ms = np.array([float(np.sum(x64[m] * x64[m])) for m in range(M)], dtype=np.float64) / float(K)
+    r64 = 1.0 / np.sqrt(ms + float(np.float32(eps)))
+    r = r64.astype(np.float32)
+    # distance of r64 from the nearest rounding boundary of fp32, in units of the fp32 spacing
+    up = np.nextafter(r, np.float32(np.inf)).astype(np.float64)
+    dn = np.nextafter(r, np.float32(-np.inf)).astype(np.float64)
+    r_d = r.astype(np.float64)
+    with np.errstate(invalid="ignore", divide="ignore"):
+        d_up = np.abs(r64 - (r_d + up) / 2) / (up - r_d)
+        d_dn = np.abs(r64 - (r_d + dn) / 2) / (r_d - dn)
+    ambiguous = np.minimum(d_up, d_dn) < 1e-9
+    t = _bf16_rne_bits(x32 * r[:, None])
+    t32 = (t.astype(np.uint32) << 16).view(np.float32)
+    y = _bf16_rne_bits(t32 * g32[None, :])
+    return y, r, ambiguous
+
+
+def rmsnorm_encode(b: int, k: int, X_bits: np.ndarray, gamma_bits: np.ndarray, eps: float, positions: np.ndarray):
+    """The normalisation followed by the static-position encode of its output (Algorithm 2)."""
+    y, _, ambiguous = rmsnorm(X_bits, gamma_bits, eps)
+    assert not ambiguous.any()
+    return encode(b, k, y, positions), y
