@@ -340,6 +340,36 @@ def bench_weights_sq(sq, dev, peaks):
     return {"cols": ["M", "K", "N", "gemm_us_graph_replay", "weight_stream_GBps", "of_measured_hbm"], "rows": rows}
 
 
+def bench_producer_fusion(sq, dev, peaks, iters=30):
+    """sq_rmsnorm_encode (the normalisation that produces two of a decoder layer's four activations, computed
+    inside the static-position encode) next to sq_encode of an already normalised tensor and to a library
+    normalisation (torch rms_norm: read + write of the bf16 tensor, yardstick only): the fused call saves the
+    normalised tensor's trip to memory and back.  Three inputs in rotation (> L2)."""
+    rows = []
+    for M, K, b, k in ((8192, 8192, 64, 8), (4096, 8192, 128, 16), (8192, 4096, 64, 8)):
+        fmt = sq.make_format(b, k, True)
+        Xs = [gen.activations(M, K, seed=s, outlier_fraction=0.005, outlier_scale=50.0, device=dev) for s in range(3)]
+        gamma = (1.0 + 0.1 * gen.weights(1, K, seed=1, std=1.0, device=dev).float()).to(torch.bfloat16).reshape(K).contiguous()
+        pos = sq.sq_calib_positions(fmt, gen.calibration_batch(512, K, seed=0, outlier_fraction=0.005, outlier_scale=50.0, device=dev), None)
+        enc = sq.alloc_encoded(fmt, M, K, dev)
+        a8 = torch.empty(M, K, dtype=torch.uint8, device=dev)
+        t_e, _ = time_launches(lambda i: sq.sq_encode(fmt, Xs[i % 3], pos, out=enc), iters, 5)
+        t_e8, _ = time_launches(lambda i: sq.sq_encode_a8(fmt, Xs[i % 3], pos, out=enc, a8=a8), iters, 5)
+        t_f, _ = time_launches(lambda i: sq.sq_rmsnorm_encode(fmt, Xs[i % 3], gamma, 1e-5, pos, out=enc, want_a8=False), iters, 5)
+        t_f8, _ = time_launches(lambda i: sq.sq_rmsnorm_encode(fmt, Xs[i % 3], gamma, 1e-5, pos, out=enc, a8=a8), iters, 5)
+        try:
+            t_n, _ = time_launches(lambda i: torch.nn.functional.rms_norm(Xs[i % 3], (K,), gamma, 1e-5), 10, 3)
+        except Exception:
+            t_n = None
+        nbytes = M * K * (2.0 + 0.5 + k / b)
+        rows.append([M, K, b, k, round(t_f * 1e3, 1), round(nbytes / (t_f * 1e-3) / 1e9), round(nbytes / (t_f * 1e-3) / 1e9 / peaks["hbm_gbs"], 3),
+                     round(t_f8 * 1e3, 1), round(t_e * 1e3, 1), round(t_e8 * 1e3, 1), None if t_n is None else round(t_n * 1e3, 1)])
+        del Xs, enc, a8
+        torch.cuda.empty_cache()
+    return {"cols": ["M", "K", "b", "k", "rmsnorm_encode_us", "GBps", "of_measured_hbm", "rmsnorm_encode_a8_us", "encode_us",
+                     "encode_a8_us", "library_rms_norm_us"], "rows": rows}
+
+
 def bench_same_run_int8(dev, iters=10):
     """A vendor INT8 GEMM (torch._int_mm, M=4096, N=K=8192) timed in the same run: a yardstick for
     the tensor pipe's INT8 rate at this run's clocks, never on the product path."""
@@ -491,7 +521,8 @@ def run_reference(args):
     print(json.dumps(line))
 
 
-PROFILE_CASES = ("encode_dynamic", "encode_static", "encode_static_a8", "gemm_a8", "gemm_stream", "fp_gemm", "wsq_gemm")
+PROFILE_CASES = ("encode_dynamic", "encode_static", "encode_static_a8", "encode_rmsnorm", "encode_rmsnorm_a8", "gemm_a8", "gemm_stream",
+                 "fp_gemm", "wsq_gemm")
 
 
 def run_profile_case(args):
@@ -512,9 +543,12 @@ def run_profile_case(args):
             calib = gen.calibration_batch(512, K, seed=0, outlier_fraction=0.005, outlier_scale=50.0, device=dev)
             pos = sq.sq_calib_positions(fmt, calib, None)
         enc = sq.alloc_encoded(fmt, M, K, dev)
-        a8 = torch.empty(M, K, dtype=torch.uint8, device=dev) if case == "encode_static_a8" else None
+        a8 = torch.empty(M, K, dtype=torch.uint8, device=dev) if case.endswith("_a8") else None
+        gamma = torch.ones(K, dtype=torch.bfloat16, device=dev)
         for i in range(n):
-            if a8 is not None:
+            if case.startswith("encode_rmsnorm"):
+                sq.sq_rmsnorm_encode(fmt, Xs[i % 3], gamma, 1e-5, pos, out=enc, a8=a8, want_a8=a8 is not None)
+            elif a8 is not None:
                 sq.sq_encode_a8(fmt, Xs[i % 3], pos, out=enc, a8=a8)
             else:
                 sq.sq_encode(fmt, Xs[i % 3], pos, out=enc)
@@ -726,6 +760,8 @@ def run_cuda(args):
                                   **bench_gemm_fused(sq, layers, dev, peaks)}
             line["weights_sq"] = {"workload": "weights in SQ-format (implicit mask, b=64, k=8) x per-token INT8 activations, 8B-decoder shapes, 1 and 4 tokens",
                                   **bench_weights_sq(sq, dev, peaks)}
+            line["producer_fusion"] = {"workload": "sq_rmsnorm_encode: bf16 [M,K] Student-t nu=3, 0.5% channels x50, static positions; GBps = (2 + 0.5 + k/b) bytes per element over the fused call (the unfused pair moves 4 more: the normalised tensor written and read back); median of 30 launches",
+                                       **bench_producer_fusion(sq, dev, peaks)}
             same = bench_same_run_int8(dev)
             burst, sustained, fp8_burst = bench_int8_tensor_rate(sq)
             line["same_run"] = {"int8_gemm_TOPS": None if same is None else round(same, 1),

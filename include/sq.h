@@ -251,6 +251,24 @@ sq_status sq_gemm_a8(const sq_format* fmt, const sq_encoded* A, const sq_weights
                      const uint8_t* positions, int64_t M, int64_t N, int64_t K, void* out_bf16,
                      int32_t* acc_out, const void* a8, void* cuda_stream);
 
+/* Producer fusion, the producer itself: the root-mean-square layer normalisation that feeds two
+ * of the four quantised linears of the decoder layers whose prefill the appendix "End-to-End
+ * Latency Analysis" times, computed inside the encode (static positions, tied scales), so the
+ * normalised activation never travels to memory and back.  Per row of X (bf16 [M, K]):
+ *     ms = (sum_j x_j^2) / K               in fp64 (every square is exact there)
+ *     r  = fp32(1 / sqrt(ms + eps))        one rounding
+ *     t  = bf16(fp32(x_j) * r)             fp32 product, round to nearest even
+ *     y  = bf16(fp32(t) * fp32(gamma_j))   exact product, one rounding
+ * and `out` (and a8, unless NULL) = sq_encode_a8 of y, bit for bit.  gamma_bf16: device bf16
+ * [K], 16-byte aligned; eps >= 0.  Row lengths: those sq_encode_a8's own kernel takes (8/12/14/16
+ * * 256 * {1,2,4,8}) whose row slots, tables and gamma fit shared memory (K = 4096 and 8192 do,
+ * with or without a8); anything else, dynamic positions and SQ_POS_STATIC_INDEP:
+ * SQ_ERR_UNSUPPORTED, nothing launched (normalise separately and call sq_encode).  Inputs
+ * finite; X is not written. */
+sq_status sq_rmsnorm_encode(const sq_format* fmt, const void* X_bf16, const void* gamma_bf16, float eps,
+                            int64_t M, int64_t K, const uint8_t* positions, sq_encoded* out, void* a8,
+                            void* cuda_stream);
+
 /* (No counterpart in the paper: a convenience of this library.)
  * sq_gemm_ws for callers that have nowhere to get a workspace from.  Some hosts of this
  * library hand out all device memory once, at start-up -- a serving process that gives

@@ -70,6 +70,7 @@ def _load() -> ctypes.CDLL:
     lib.sq_gemm_ws.argtypes = [P(sq_format), P(sq_encoded), P(sq_weights), VP, I64, I64, I64, VP, VP, VP,
                                ctypes.c_size_t, VP]
     lib.sq_encode_a8.argtypes = [P(sq_format), VP, I64, I64, VP, P(sq_encoded), VP, VP]
+    lib.sq_rmsnorm_encode.argtypes = [P(sq_format), VP, VP, ctypes.c_float, I64, I64, VP, P(sq_encoded), VP, VP]
     lib.sq_gemm_a8.argtypes = [P(sq_format), P(sq_encoded), P(sq_weights), VP, I64, I64, I64, VP, VP, VP, VP]
     lib.sq_gemm_workspace_bytes.argtypes = [P(sq_format), I64, I64, I64, P(ctypes.c_size_t)]
     lib.sq_gemm_static_scratch.argtypes = [P(sq_format), P(sq_encoded), P(sq_weights), VP, I64, I64, I64, VP, VP, VP]
@@ -88,7 +89,8 @@ def _load() -> ctypes.CDLL:
     for name in ("sq_encoded_sizes", "sq_weights_sizes", "sq_calib_positions", "sq_pack_weights",
                  "sq_encode", "sq_gemm", "sq_gemm_ws", "sq_gemm_workspace_bytes", "sq_gemm_static_scratch", "sq_decode",
                  "sq_device_status", "sq_device_status_word", "sq_fp_pack_weights", "sq_fp_encode", "sq_fp_gemm",
-                 "sq_fp_decode", "sq_w_encode", "sq_w_act_quant", "sq_w_gemm", "sq_encode_a8", "sq_gemm_a8"):
+                 "sq_fp_decode", "sq_w_encode", "sq_w_act_quant", "sq_w_gemm", "sq_encode_a8", "sq_gemm_a8", "sq_rmsnorm_encode",
+                 "sq_probe_int8_tensor_rate", "sq_probe_fp8_tensor_rate"):
         getattr(lib, name).restype = ctypes.c_int
     return lib
 
@@ -261,6 +263,24 @@ def sq_encode_a8(fmt: sq_format, X: torch.Tensor, positions: torch.Tensor | None
     cs = out.c_struct()
     _check(_lib.sq_encode_a8(ctypes.byref(fmt), _ptr(X), M, K, _ptr(positions), ctypes.byref(cs), _ptr(a8),
                              _stream(stream)), "sq_encode_a8")
+    return out, a8
+
+
+
+def sq_rmsnorm_encode(fmt: sq_format, X: torch.Tensor, gamma: torch.Tensor, eps: float,
+                      positions: torch.Tensor, out: Encoded | None = None, a8: torch.Tensor | None = None,
+                      want_a8: bool = True, stream=None):
+    """Root-mean-square normalisation fused into the static-position encode; returns (Encoded, a8 or None)."""
+    M, K = _bf16_2d(X, "X")
+    if gamma.dtype != torch.bfloat16 or gamma.numel() != K or not gamma.is_contiguous():
+        raise ValueError("gamma must be a contiguous bf16 tensor of K elements")
+    if out is None:
+        out = alloc_encoded(fmt, M, K, X.device)
+    if a8 is None and want_a8:
+        a8 = _buf(M * K, torch.uint8, X.device)[: M * K].view(M, K)
+    cs = out.c_struct()
+    _check(_lib.sq_rmsnorm_encode(ctypes.byref(fmt), _ptr(X), _ptr(gamma), ctypes.c_float(eps), M, K, _ptr(positions),
+                                  ctypes.byref(cs), _ptr(a8), _stream(stream)), "sq_rmsnorm_encode")
     return out, a8
 
 

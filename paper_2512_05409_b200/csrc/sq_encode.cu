@@ -467,7 +467,26 @@ struct EncodeParams {
   int rw;             // warps per row group
   int group_stride;   // bytes of shared memory per group
   MulK mk;            // -1, 2, 32, 2^8, 2^16, 2^24 (see MulK)
+  const uint16_t* gamma;  // fused normalisation (ring kernel, NORM): its weights [K], else nullptr
+  float eps;
 };
+
+// A packed pair of the fused normalisation (w and g: two bf16 per word): bf16(bf16(x * r) * gamma),
+// the first product in fp32, the second exact before its rounding; both roundings to nearest even.
+__device__ __forceinline__ uint32_t norm2(uint32_t w, float r, uint32_t g) {
+  const float lo = __fmul_rn(__uint_as_float(w << 16), r), hi = __fmul_rn(__uint_as_float(w & 0xFFFF0000u), r);
+  uint32_t t, y;
+  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(t) : "f"(hi), "f"(lo));
+  asm("mul.rn.bf16x2 %0, %1, %2;" : "=r"(y) : "r"(t), "r"(g));
+  return y;
+}
+// A packed pair normalised as above, their squares added to the fp64 sum `acc` on the way in
+// (the widened values serve both).
+__device__ __forceinline__ void sq2_add(uint32_t w, double& acc) {
+  const double lo = (double)__uint_as_float(w << 16), hi = (double)__uint_as_float(w & 0xFFFF0000u);
+  acc = fma(lo, lo, acc);
+  acc = fma(hi, hi, acc);
+}
 
 __device__ __forceinline__ void group_sync(int rw, int grp) {
   if (rw == 1) __syncwarp();
@@ -1139,7 +1158,7 @@ __global__ void __launch_bounds__(NT, 1) encode_static_regs_kernel(const EncodeP
 //   from the registers.
 // MASK8: the per-element magnitude masks are kept as bytes and widened on the fly (long rows,
 // where a half-word table would not leave room for the slots).
-template <int NCL, int NT, bool INDEP, bool MASK8, bool FP = false>
+template <int NCL, int NT, bool INDEP, bool MASK8, bool FP = false, bool NORM = false>
 __global__ void __launch_bounds__(NT, 1) encode_static_ring_kernel(const EncodeParams p) {
   extern __shared__ __align__(128) uint8_t smem_enc[];
   const int K = p.K, k = p.k;
@@ -1162,7 +1181,11 @@ __global__ void __launch_bounds__(NT, 1) encode_static_ring_kernel(const EncodeP
   uint8_t* hmask = smem_enc;
   uint16_t* jt = reinterpret_cast<uint16_t*>(smem_enc + mask_bytes);
   uint16_t* jimg = reinterpret_cast<uint16_t*>(smem_enc + mask_bytes + jt_bytes);
-  uint8_t* gbase = smem_enc + mask_bytes + jt_bytes * (want_a8 ? 2 : 1) + (size_t)grp * p.group_stride;
+  // (fused normalisation: its weights [K] and the weights at the selected places [GK] follow the tables)
+  uint16_t* gam = reinterpret_cast<uint16_t*>(smem_enc + mask_bytes + jt_bytes * (want_a8 ? 2 : 1));
+  uint16_t* gjt = gam + K;
+  uint8_t* gbase = smem_enc + mask_bytes + jt_bytes * (want_a8 ? 2 : 1) + (NORM ? row_bytes + jt_bytes : 0) +
+                   (size_t)grp * p.group_stride;
   uint8_t* img = gbase + row_bytes;
   uint32_t* exch = reinterpret_cast<uint32_t*>(img + (want_a8 ? (size_t)K : 0));
   volatile int* nexti = reinterpret_cast<volatile int*>(exch + 64);
@@ -1209,6 +1232,8 @@ __global__ void __launch_bounds__(NT, 1) encode_static_ring_kernel(const EncodeP
   }
   if (want_a8)
     for (int i = glane; i < K / 4; i += gsize) reinterpret_cast<uint32_t*>(img)[i] = 0u;
+  if (NORM)
+    for (int i = threadIdx.x; i < K / 8; i += NT) reinterpret_cast<uint4*>(gam)[i] = reinterpret_cast<const uint4*>(p.gamma)[i];
   __syncthreads();
   for (int t = threadIdx.x, i = 0; t < GK; t += NT, ++i) {
     int pos = 0;
@@ -1224,6 +1249,7 @@ __global__ void __launch_bounds__(NT, 1) encode_static_ring_kernel(const EncodeP
     if (MASK8) hmask[j] = 0;
     else reinterpret_cast<uint16_t*>(hmask)[j] = 0;
     if (want_a8) jimg[t] = FP ? (uint16_t)j : (uint16_t)((j & ~7) | ((j & 1) << 2) | ((j & 7) >> 1));
+    if (NORM) gjt[t] = gam[j];
   }
   __syncthreads();
 
@@ -1235,10 +1261,54 @@ __global__ void __launch_bounds__(NT, 1) encode_static_ring_kernel(const EncodeP
 
     uint4 v[NCL];
     uint32_t r2 = 0, smax = 0;
+    float rn = 0.f;  // fused normalisation: 1 / sqrt(mean of squares + eps)
     if (landed) {
       const uint4* src = reinterpret_cast<const uint4*>(slot) + slice * S8 + lane;
 #pragma unroll
       for (int c = 0; c < NCL; ++c) v[c] = src[c * 32];
+    }
+    if constexpr (NORM) {
+      // The row's mean of squares in fp64 (every square exact), across the group; then the chunks in
+      // the registers are replaced by the normalised values (the slot keeps the raw row: the few
+      // selected values read from it below are normalised one by one).
+      double ss = 0.0;
+      if (landed) {
+        double s4[4] = {0.0, 0.0, 0.0, 0.0};  // four chains: a lane's 8 * NCL additions must not wait for one another
+#pragma unroll
+        for (int c = 0; c < NCL; ++c) {
+          sq2_add(v[c].x, s4[0]);
+          sq2_add(v[c].y, s4[1]);
+          sq2_add(v[c].z, s4[2]);
+          sq2_add(v[c].w, s4[3]);
+        }
+        ss = (s4[0] + s4[1]) + (s4[2] + s4[3]);
+      }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+      if (rw > 1) {
+        uint32_t* ex = exch + flip * 32;
+        if (lane == 0) {
+          ex[8 + slice] = (uint32_t)__double2loint(ss);
+          ex[24 + slice] = (uint32_t)__double2hiint(ss);
+        }
+        group_sync(rw, grp);
+        ss = 0.0;
+        for (int w = 0; w < rw; ++w) ss += __hiloint2double((int)ex[24 + w], (int)ex[8 + w]);
+      }
+      rn = (float)(1.0 / sqrt(ss / (double)K + (double)p.eps));
+      if (landed) {
+        const uint4* gsrc = reinterpret_cast<const uint4*>(gam) + slice * S8 + lane;
+#pragma unroll
+        for (int c = 0; c < NCL; ++c) {
+          const uint4 g = gsrc[c * 32];
+          v[c].x = norm2(v[c].x, rn, g.x);
+          v[c].y = norm2(v[c].y, rn, g.y);
+          v[c].z = norm2(v[c].z, rn, g.z);
+          v[c].w = norm2(v[c].w, rn, g.w);
+        }
+      }
+    }
+    if (landed) {
       // selected places become (signed) zeros; the maximum of what is left
 #pragma unroll
       for (int c = 0; c < NCL; ++c) {
@@ -1265,7 +1335,15 @@ __global__ void __launch_bounds__(NT, 1) encode_static_ring_kernel(const EncodeP
       // largest selected magnitude, through the offset table
       for (int q4 = glane; q4 < nquads; q4 += gsize) {
         const uint2 jj = *reinterpret_cast<const uint2*>(jt + 4 * q4);
-        const uint32_t a = srow[jj.x & 0xFFFFu], b = srow[jj.x >> 16], c = srow[jj.y & 0xFFFFu], d = srow[jj.y >> 16];
+        uint32_t a = srow[jj.x & 0xFFFFu], b = srow[jj.x >> 16], c = srow[jj.y & 0xFFFFu], d = srow[jj.y >> 16];
+        if constexpr (NORM) {  // two at a time, as the registers' words
+          const uint2 gg = *reinterpret_cast<const uint2*>(gjt + 4 * q4);
+          const uint32_t y01 = norm2(a | (b << 16), rn, gg.x), y23 = norm2(c | (d << 16), rn, gg.y);
+          a = y01 & 0xFFFFu;
+          b = y01 >> 16;
+          c = y23 & 0xFFFFu;
+          d = y23 >> 16;
+        }
         smax = max(max(smax, a & 0x7FFFu), max(max(b & 0x7FFFu, c & 0x7FFFu), d & 0x7FFFu));
       }
     }
@@ -1320,7 +1398,15 @@ __global__ void __launch_bounds__(NT, 1) encode_static_ring_kernel(const EncodeP
 #pragma unroll 2
       for (int q4 = glane; q4 < nquads; q4 += gsize) {
         const uint2 jj = *reinterpret_cast<const uint2*>(jt + 4 * q4);
-        const uint32_t w[4] = {srow[jj.x & 0xFFFFu], srow[jj.x >> 16], srow[jj.y & 0xFFFFu], srow[jj.y >> 16]};
+        uint32_t w[4] = {srow[jj.x & 0xFFFFu], srow[jj.x >> 16], srow[jj.y & 0xFFFFu], srow[jj.y >> 16]};
+        if constexpr (NORM) {
+          const uint2 gg = *reinterpret_cast<const uint2*>(gjt + 4 * q4);
+          const uint32_t y01 = norm2(w[0] | (w[1] << 16), rn, gg.x), y23 = norm2(w[2] | (w[3] << 16), rn, gg.y);
+          w[0] = y01 & 0xFFFFu;
+          w[1] = y01 >> 16;
+          w[2] = y23 & 0xFFFFu;
+          w[3] = y23 >> 16;
+        }
         uint32_t o = 0;
 #pragma unroll
         for (int q = 0; q < 4; ++q) {
@@ -1730,7 +1816,7 @@ cudaError_t launch_static_regs_as(EncodeParams p, int rw, cudaStream_t st) {
 }
 
 // Ring kernel: `rw` warps per row, 16 / rw groups per block, one slot per group.
-template <int NCL, bool INDEP, bool MASK8, bool FP = false>
+template <int NCL, bool INDEP, bool MASK8, bool FP = false, bool NORM = false>
 cudaError_t launch_static_ring_as(EncodeParams p, int rw, cudaStream_t st) {
   constexpr int NT = 512;
   const int GK = (p.K / p.b) * p.k;
@@ -1739,16 +1825,16 @@ cudaError_t launch_static_ring_as(EncodeParams p, int rw, cudaStream_t st) {
   const size_t mask_bytes = MASK8 ? (size_t)p.K : (size_t)p.K * 2;
   const size_t jt_bytes = ((size_t)GK * 2 + 15) & ~(size_t)15;
   const size_t per_group = ((size_t)p.K * 2 + (a8 ? (size_t)p.K : 0) + 256 + 16 + 127) & ~(size_t)127;
-  const size_t smem = mask_bytes + jt_bytes * (a8 ? 2 : 1) + per_group * ngroups;
+  const size_t smem = mask_bytes + jt_bytes * (a8 ? 2 : 1) + (NORM ? (size_t)p.K * 2 + jt_bytes : 0) + per_group * ngroups;
   if (smem > 226 * 1024) return cudaErrorNotSupported;
   p.rw = rw;
   p.group_stride = (int)per_group;
   int dev = 0, sms = 0;
   cudaError_t err = device_and_sms(&dev, &sms);
   if (err != cudaSuccess) return err;
-  SQ_ENSURE_SMEM((encode_static_ring_kernel<NCL, NT, INDEP, MASK8, FP>), dev, smem);
+  SQ_ENSURE_SMEM((encode_static_ring_kernel<NCL, NT, INDEP, MASK8, FP, NORM>), dev, smem);
   const int64_t blocks = p.M < sms ? p.M : sms;
-  encode_static_ring_kernel<NCL, NT, INDEP, MASK8, FP><<<(unsigned)blocks, NT, smem, st>>>(p);
+  encode_static_ring_kernel<NCL, NT, INDEP, MASK8, FP, NORM><<<(unsigned)blocks, NT, smem, st>>>(p);
   return cudaGetLastError();
 }
 
@@ -1756,7 +1842,7 @@ cudaError_t launch_static_ring_as(EncodeParams p, int rw, cudaStream_t st) {
 // (the per-row work that does not shrink with the slice -- scales, barriers -- is then spread over
 // the most elements, and the most rows are in flight); half-word masks if the tables and slots
 // fit, else byte masks.
-template <bool INDEP, bool FP = false>
+template <bool INDEP, bool FP = false, bool NORM = false>
 cudaError_t launch_static_ring(const EncodeParams& p, cudaStream_t st) {
   if (p.K % 256 != 0 || p.K > 65535 || (reinterpret_cast<uintptr_t>(p.X) & 15) != 0) return cudaErrorNotSupported;
   for (int mask8 = 0; mask8 < 2; ++mask8) {
@@ -1766,8 +1852,8 @@ cudaError_t launch_static_ring(const EncodeParams& p, cudaStream_t st) {
       cudaError_t err = cudaErrorNotSupported;
 #define SQ_RING(NCL_)                                                                   \
   if (ncl == NCL_)                                                                      \
-    err = mask8 ? launch_static_ring_as<NCL_, INDEP, true, FP>(p, rw, st)               \
-                : launch_static_ring_as<NCL_, INDEP, false, FP>(p, rw, st);
+    err = mask8 ? launch_static_ring_as<NCL_, INDEP, true, FP, NORM>(p, rw, st)         \
+                : launch_static_ring_as<NCL_, INDEP, false, FP, NORM>(p, rw, st);
       SQ_RING(8) SQ_RING(12) SQ_RING(14) SQ_RING(16)
 #undef SQ_RING
       if (err != cudaErrorNotSupported) return err;
@@ -1832,6 +1918,8 @@ cudaError_t launch_encode(int b, int k, bool is_static, bool indep, const uint16
   p.rw = 1;
   p.group_stride = 0;
   p.mk = MulK{0xFFFFFFFFu, 2u, 32u, 256u, 65536u, 1u << 24, 16u, 1u};
+  p.gamma = nullptr;
+  p.eps = 0.f;
   if (is_static && indep) {
     // independent scales: the register kernel, or the plain one for row lengths it does not take
     cudaError_t err = launch_static_ring<true>(p, st);
@@ -1897,7 +1985,40 @@ cudaError_t launch_fp_encode_static_ring(int b, int k, const uint16_t* X, int64_
   p.rw = 1;
   p.group_stride = 0;
   p.mk = MulK{0xFFFFFFFFu, 2u, 32u, 256u, 65536u, 1u << 24, 16u, 1u};
+  p.gamma = nullptr;
+  p.eps = 0.f;
   return launch_static_ring<false, true>(p, st);
+}
+
+// Root-mean-square normalisation fused into the static-position encode (tied scales): the ring
+// kernel normalises a row in its registers before it encodes it.  cudaErrorNotSupported = a row
+// length the ring kernel does not take, or one whose slots, tables and weights exceed shared memory.
+cudaError_t launch_rmsnorm_encode(int b, int k, const uint16_t* X, const uint16_t* gamma, float eps, int64_t M, int64_t K,
+                                  const uint8_t* positions, const sq_encoded& out, uint8_t* a8, int* status,
+                                  cudaStream_t st) {
+  if (positions == nullptr || M < 1) return cudaErrorNotSupported;
+  EncodeParams p;
+  p.a8 = a8;
+  p.X = X;
+  p.positions = positions;
+  p.dq4 = out.dq4;
+  p.vals = out.vals;
+  p.idx = out.idx;
+  p.s_hi = out.s_hi;
+  p.s_lo = out.s_lo;
+  p.shift = out.shift;
+  p.status = status;
+  p.M = M;
+  p.K = (int)K;
+  p.k = k;
+  p.b = b;
+  p.nbuf = 1;
+  p.rw = 1;
+  p.group_stride = 0;
+  p.mk = MulK{0xFFFFFFFFu, 2u, 32u, 256u, 65536u, 1u << 24, 16u, 1u};
+  p.gamma = gamma;
+  p.eps = eps;
+  return launch_static_ring<false, false, true>(p, st);
 }
 
 // Floating-point variant, dynamic positions: the row-group kernel's selection with that format's
@@ -1924,6 +2045,8 @@ cudaError_t launch_fp_encode_dynamic_rows(int b, int k, const uint16_t* X, int64
   p.rw = 1;
   p.group_stride = 0;
   p.mk = MulK{0xFFFFFFFFu, 2u, 32u, 256u, 65536u, 1u << 24, 16u, 1u};
+  p.gamma = nullptr;
+  p.eps = 0.f;
 #define SQ_DYN_FP(BB, KK_) \
   if (b == BB && k == KK_) return launch_rows<BB, KK_, true>(p, st);
   SQ_DYN_FP(32, 4) SQ_DYN_FP(64, 8) SQ_DYN_FP(128, 16) SQ_DYN_FP(64, 4) SQ_DYN_FP(128, 8) SQ_DYN_FP(32, 8) SQ_DYN_FP(64, 16) SQ_DYN_FP(128, 32)

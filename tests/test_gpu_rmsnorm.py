@@ -1,0 +1,96 @@
+"""The normalisation fused into the static-position encode (sq_rmsnorm_encode) against the oracle:
+every integer, both scales and the merged 8-bit operand bit for bit; what it does not take is
+refused before anything is launched."""
+import numpy as np
+import pytest
+import torch
+
+import gen
+import oracle
+import paper_2512_05409_b200 as sq
+from test_gpu_parity import _bits, _np, check_status, compare_encoded, merged_operand_from_oracle
+
+pytestmark = pytest.mark.gpu
+
+
+def _gamma(K, seed, device="cuda"):
+    return (1.0 + 0.25 * gen.weights(1, K, seed=seed, std=1.0, device=device).float()).to(torch.bfloat16).reshape(K).contiguous()
+
+
+@pytest.mark.parametrize("want_a8", [False, True])
+@pytest.mark.parametrize("M,K,b,k", [
+    (300, 2048, 64, 8),       # one warp per row
+    (1, 2048, 64, 8),
+    (130, 3072, 32, 4),
+    (1500, 4096, 128, 16),    # more rows than row groups in flight: the slots are refilled
+    (700, 8192, 64, 8),       # two warps per row: the mean of squares crosses warps
+    (257, 8192, 128, 32),
+    (90, 7168, 128, 16),
+])
+def test_rmsnorm_encode_matches_the_oracle(M, K, b, k, want_a8):
+    fmt = sq.make_format(b, k, True)
+    X = gen.activations(M, K, seed=M + K, outlier_fraction=0.01, outlier_scale=30.0, device="cuda")
+    gamma = _gamma(K, seed=K + b)
+    eps = 1e-5
+    pos = sq.sq_calib_positions(fmt, gen.calibration_batch(64, K, seed=K, outlier_fraction=0.01, outlier_scale=30.0, device="cuda"), None)
+    keep = X.clone()
+    a8 = torch.full((M, K), 0x5A, dtype=torch.uint8, device="cuda") if want_a8 else None
+    enc, a8 = sq.sq_rmsnorm_encode(fmt, X, gamma, eps, pos, a8=a8, want_a8=want_a8)
+    check_status()
+    assert torch.equal(X, keep)
+    pos_ref = _np(pos)
+    enc_ref, y = oracle.rmsnorm_encode(b, k, _bits(X), _bits(gamma), eps, pos_ref)
+    compare_encoded(enc, enc_ref)
+    if want_a8:
+        assert np.array_equal(_np(a8), merged_operand_from_oracle(b, k, enc_ref, pos_ref))
+        # ... which is what the unfused pair of calls writes for the normalised rows
+        y_t = torch.from_numpy(y.view(np.int16)).cuda().view(torch.bfloat16)
+        enc2, a8_2 = sq.sq_encode_a8(fmt, y_t, pos)
+        assert torch.equal(a8, a8_2) and torch.equal(enc.dq4, enc2.dq4) and torch.equal(enc.vals, enc2.vals)
+
+
+def test_rmsnorm_encode_degenerate_rows():
+    """Zero rows (r = 1/sqrt(eps), all codes zero), constant rows, one huge value, tiny rows."""
+    M, K, b, k = 8, 4096, 64, 8
+    fmt = sq.make_format(b, k, True)
+    X = gen.activations(M, K, seed=3, device="cuda")
+    X[0] = 0
+    X[1] = 0.75
+    X[2] = 0
+    X[2, 1234] = 3.0e4
+    X[3] *= 2.0 ** -60
+    X[4] *= 2.0 ** 50
+    X[5, ::2] = 0
+    gamma = _gamma(K, seed=9)
+    pos = sq.sq_calib_positions(fmt, gen.calibration_batch(64, K, seed=3, device="cuda"), None)
+    for eps in (1e-6, 0.0):
+        Xe = X.clone()
+        if eps == 0.0:
+            Xe[0] = 1.0      # a zero row without eps has no defined reciprocal root
+        enc, a8 = sq.sq_rmsnorm_encode(fmt, Xe, gamma, eps, pos)
+        check_status()
+        enc_ref, _ = oracle.rmsnorm_encode(b, k, _bits(Xe), _bits(gamma), eps, _np(pos))
+        compare_encoded(enc, enc_ref)
+        assert np.array_equal(_np(a8), merged_operand_from_oracle(b, k, enc_ref, _np(pos)))
+
+
+def test_rmsnorm_encode_refuses_what_it_does_not_take():
+    X = gen.activations(16, 1024, seed=1, device="cuda")
+    gamma = _gamma(1024, seed=2)
+    pos = sq.sq_calib_positions(sq.make_format(64, 8, True), gen.calibration_batch(64, 1024, seed=1, device="cuda"), None)
+    with pytest.raises(sq.SqError) as e:       # a row length its kernel does not take
+        sq.sq_rmsnorm_encode(sq.make_format(64, 8, True), X, gamma, 1e-5, pos)
+    assert e.value.status == sq.SQ_ERR_UNSUPPORTED
+    X2 = gen.activations(16, 2048, seed=1, device="cuda")
+    g2 = _gamma(2048, seed=2)
+    with pytest.raises(sq.SqError) as e:       # dynamic positions
+        sq.sq_rmsnorm_encode(sq.make_format(64, 8, False), X2, g2, 1e-5, None)
+    assert e.value.status == sq.SQ_ERR_UNSUPPORTED
+    pos2 = sq.sq_calib_positions(sq.make_format(64, 8, True), gen.calibration_batch(64, 2048, seed=1, device="cuda"), None)
+    with pytest.raises(sq.SqError) as e:       # independent scales
+        sq.sq_rmsnorm_encode(sq.make_format(64, 8, True, independent_scales=True), X2, g2, 1e-5, pos2)
+    assert e.value.status == sq.SQ_ERR_UNSUPPORTED
+    with pytest.raises(sq.SqError) as e:
+        sq.sq_rmsnorm_encode(sq.make_format(64, 8, True), X2, g2, -1.0, pos2)
+    assert e.value.status == sq.SQ_ERR_INVALID_ARG
+    check_status()
