@@ -370,6 +370,53 @@ def bench_producer_fusion(sq, dev, peaks, iters=30):
                      "encode_a8_us", "library_rms_norm_us"], "rows": rows}
 
 
+def bench_layer_prefill(sq, layers, dev, iters=10):
+    """The benchmark step's four linears as they sit in a decoder layer: the first (fused QKV) and the third
+    (fused gate-up) read the output of a root-mean-square normalisation.  One pass = 4 x (encode + product)
+    with (a) that normalisation inside the encode (sq_rmsnorm_encode), (b) a library normalisation
+    (torch rms_norm, yardstick only) before sq_encode_a8, (c) no normalisation at all (the step `value` is
+    quoted on).  Attention and the gated activation are not part of any of the three."""
+    normed = [l for l in layers[0::2] if l.fused_a8]
+    if len(normed) != 2 or len(layers) != 4:
+        return None
+    gam = {id(l): (1.0 + 0.1 * gen.weights(1, l.K, seed=7, std=1.0, device=dev).float()).to(torch.bfloat16).reshape(l.K).contiguous()
+           for l in normed}
+    try:
+        sq.sq_rmsnorm_encode(normed[0].fmt, normed[0].X, gam[id(normed[0])], 1e-5, normed[0].pos, out=normed[0].enc, a8=normed[0].a8)
+    except sq.SqError:
+        return None
+
+    def one_pass(mode):
+        for l in layers:
+            if id(l) in gam and mode == "fused":
+                sq.sq_rmsnorm_encode(l.fmt, l.X, gam[id(l)], 1e-5, l.pos, out=l.enc, a8=l.a8)
+            elif id(l) in gam and mode == "library":
+                y = torch.nn.functional.rms_norm(l.X, (l.K,), gam[id(l)], 1e-5)
+                sq.sq_encode_a8(l.fmt, y, l.pos, out=l.enc, a8=l.a8)
+            else:
+                sq.sq_encode_a8(l.fmt, l.X, l.pos, out=l.enc, a8=l.a8)
+            sq.sq_gemm_a8(l.fmt, l.enc, l.a8, l.w, l.pos, out=l.out)
+    # the three variants take turns, so that a drift of the clocks under the power cap hits them alike
+    modes = ("fused", "library", "none")
+    try:
+        for mode in modes:
+            one_pass(mode)
+        torch.cuda.synchronize()
+        evs = {mode: [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(iters)] for mode in modes}
+        for i in range(iters):
+            for mode in modes:
+                evs[mode][i][0].record()
+                one_pass(mode)
+                evs[mode][i][1].record()
+        torch.cuda.synchronize()
+        res = {mode: round(statistics.median(a.elapsed_time(b) for a, b in evs[mode]), 4) for mode in modes}
+    except Exception:
+        return None
+    ops = sum(l.ops for l in layers)
+    return {"ms_norm_inside_encode": res["fused"], "ms_library_norm_then_encode": res["library"], "ms_no_norm": res["none"],
+            "TOPS_norm_inside_encode": None if res["fused"] is None else round(ops / (res["fused"] * 1e-3) / 1e12, 1)}
+
+
 def bench_same_run_int8(dev, iters=10):
     """A vendor INT8 GEMM (torch._int_mm, M=4096, N=K=8192) timed in the same run: a yardstick for
     the tensor pipe's INT8 rate at this run's clocks, never on the product path."""
@@ -762,6 +809,9 @@ def run_cuda(args):
                                   **bench_weights_sq(sq, dev, peaks)}
             line["producer_fusion"] = {"workload": "sq_rmsnorm_encode: bf16 [M,K] Student-t nu=3, 0.5% channels x50, static positions; GBps = (2 + 0.5 + k/b) bytes per element over the fused call (the unfused pair moves 4 more: the normalised tensor written and read back); median of 30 launches",
                                        **bench_producer_fusion(sq, dev, peaks)}
+            lp = bench_layer_prefill(sq, layers, dev)
+            if lp is not None:
+                line["layer_prefill"] = {"workload": "the step's four 70B-shaped linears (M=4096, b=128, k=16 static) with the two layer normalisations of a decoder layer (inputs of the QKV and gate-up projections)", **lp}
             same = bench_same_run_int8(dev)
             burst, sustained, fp8_burst = bench_int8_tensor_rate(sq)
             line["same_run"] = {"int8_gemm_TOPS": None if same is None else round(same, 1),
