@@ -94,3 +94,29 @@ def test_rmsnorm_encode_refuses_what_it_does_not_take():
         sq.sq_rmsnorm_encode(sq.make_format(64, 8, True), X2, g2, -1.0, pos2)
     assert e.value.status == sq.SQ_ERR_INVALID_ARG
     check_status()
+
+
+@pytest.mark.parametrize("M,K,b,k", [(4096, 8192, 128, 16), (2048, 4096, 64, 8), (8192, 8192, 64, 8)])
+def test_rmsnorm_encode_at_the_benchmark_sizes(M, K, b, k):
+    """The launch configurations bench.py times (the inputs of the 70B- and 8B-shaped QKV and gate-up
+    projections, and the 8192 x 8192 bandwidth test): sampled rows against the oracle, every row
+    for sane scales."""
+    fmt = sq.make_format(b, k, True)
+    X = gen.activations(M, K, seed=M + K + 1, dist="student_t3", outlier_fraction=0.005, outlier_scale=50.0, device="cuda")
+    gamma = _gamma(K, seed=K + 3)
+    pos = sq.sq_calib_positions(fmt, gen.calibration_batch(512, K, seed=K + 1, dist="student_t3", outlier_fraction=0.005, outlier_scale=50.0, device="cuda"), None)
+    enc, a8 = sq.sq_rmsnorm_encode(fmt, X, gamma, 1e-5, pos)
+    check_status()
+    rng = np.random.default_rng(M + K)
+    rows = np.unique(np.concatenate([[0, 1, 147, 148, 1183, 1184, M - 1], rng.integers(0, M, size=40)]))
+    rows_t = torch.from_numpy(rows).cuda()
+    pos_ref = _np(pos)
+    enc_ref, y = oracle.rmsnorm_encode(b, k, _bits(X[rows_t]), _bits(gamma), 1e-5, pos_ref)
+    assert np.array_equal(_np(enc.dq4[rows_t]), enc_ref.dq4) and np.array_equal(_np(enc.vals[rows_t]), enc_ref.vals)
+    assert np.array_equal(_np(enc.shift[rows_t]), enc_ref.shift)
+    assert np.array_equal(_np(enc.s_hi[rows_t]).view(np.uint32), enc_ref.s_hi.view(np.uint32))
+    assert np.array_equal(_np(enc.s_lo[rows_t]).view(np.uint32), enc_ref.s_lo.view(np.uint32))
+    assert np.array_equal(_np(a8[rows_t]), merged_operand_from_oracle(b, k, enc_ref, pos_ref))
+    # every row: scales are positive and finite, the largest INT8 magnitude of a row is 127
+    assert torch.isfinite(enc.s_hi).all() and (enc.s_hi > 0).all()
+    assert int(enc.vals.view(M, -1).abs().max(dim=1).values.min()) <= 127
