@@ -327,6 +327,13 @@ sq_status sq_fp_pack_weights(const void* W_bf16, int64_t N, int64_t K, uint8_t* 
                              void* cuda_stream);
 sq_status sq_fp_encode(const sq_format* fmt, const void* X_bf16, int64_t M, int64_t K, const uint8_t* positions,
                        sq_encoded* out, uint8_t* a8, void* cuda_stream);
+/* sq_fp_encode of the output of a root-mean-square layer normalisation, the normalisation computed
+ * inside the encode (see sq_rmsnorm_encode: the same definition of y, the same row lengths, static
+ * positions only; anything else: SQ_ERR_UNSUPPORTED, nothing launched).  out and a8 = sq_fp_encode
+ * of y, bit for bit. */
+sq_status sq_fp_rmsnorm_encode(const sq_format* fmt, const void* X_bf16, const void* gamma_bf16, float eps,
+                               int64_t M, int64_t K, const uint8_t* positions, sq_encoded* out, uint8_t* a8,
+                               void* cuda_stream);
 sq_status sq_fp_gemm(const float* s_hi, const uint8_t* a8, const float* s_w, const uint8_t* w8, int64_t M, int64_t N,
                      int64_t K, void* out_bf16, float* acc_out, void* cuda_stream);
 sq_status sq_fp_decode(const sq_format* fmt, const sq_encoded* A, const uint8_t* positions, int64_t M, int64_t K,

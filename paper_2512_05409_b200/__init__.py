@@ -11,6 +11,6 @@ from .binding import (  # noqa: F401
     sq_weights_sizes, sq_calib_positions, sq_pack_weights, sq_encode, sq_gemm, sq_gemm_ws,
     sq_gemm_workspace_bytes, sq_gemm_static_scratch, SQ_STATIC_SCRATCH_BYTES, sq_decode,
     sq_device_status, sq_device_status_word, raw, FpWeights, sq_fp_pack_weights, sq_fp_encode, sq_fp_gemm, sq_fp_decode, SqWeights, sq_w_encode, sq_w_act_quant, sq_w_gemm,
-    sq_encode_a8, sq_gemm_a8, sq_probe_int8_tensor_rate, sq_probe_fp8_tensor_rate, sq_rmsnorm_encode,
+    sq_encode_a8, sq_gemm_a8, sq_probe_int8_tensor_rate, sq_probe_fp8_tensor_rate, sq_rmsnorm_encode, sq_fp_rmsnorm_encode,
 )
 from .sharding import row_shard  # noqa: F401,E402

@@ -80,6 +80,7 @@ def _load() -> ctypes.CDLL:
     lib.sq_probe_fp8_tensor_rate.argtypes = [ctypes.c_int, P(ctypes.c_double), VP]
     lib.sq_fp_pack_weights.argtypes = [VP, I64, I64, VP, VP, VP, VP]
     lib.sq_fp_encode.argtypes = [P(sq_format), VP, I64, I64, VP, P(sq_encoded), VP, VP]
+    lib.sq_fp_rmsnorm_encode.argtypes = [P(sq_format), VP, VP, ctypes.c_float, I64, I64, VP, P(sq_encoded), VP, VP]
     lib.sq_fp_gemm.argtypes = [VP, VP, VP, VP, I64, I64, I64, VP, VP, VP]
     lib.sq_fp_decode.argtypes = [P(sq_format), P(sq_encoded), VP, I64, I64, VP, VP]
     lib.sq_w_encode.argtypes = [P(sq_format), VP, VP, I64, I64, VP, VP, VP, VP, VP]
@@ -89,7 +90,7 @@ def _load() -> ctypes.CDLL:
     for name in ("sq_encoded_sizes", "sq_weights_sizes", "sq_calib_positions", "sq_pack_weights",
                  "sq_encode", "sq_gemm", "sq_gemm_ws", "sq_gemm_workspace_bytes", "sq_gemm_static_scratch", "sq_decode",
                  "sq_device_status", "sq_device_status_word", "sq_fp_pack_weights", "sq_fp_encode", "sq_fp_gemm",
-                 "sq_fp_decode", "sq_w_encode", "sq_w_act_quant", "sq_w_gemm", "sq_encode_a8", "sq_gemm_a8", "sq_rmsnorm_encode",
+                 "sq_fp_decode", "sq_w_encode", "sq_w_act_quant", "sq_w_gemm", "sq_encode_a8", "sq_gemm_a8", "sq_rmsnorm_encode", "sq_fp_rmsnorm_encode",
                  "sq_probe_int8_tensor_rate", "sq_probe_fp8_tensor_rate"):
         getattr(lib, name).restype = ctypes.c_int
     return lib
@@ -407,6 +408,23 @@ def sq_fp_encode(fmt: sq_format, X: torch.Tensor, positions: torch.Tensor | None
     cs = out.c_struct()
     _check(_lib.sq_fp_encode(ctypes.byref(fmt), _ptr(X), M, K, _ptr(positions), ctypes.byref(cs), _ptr(a8),
                              _stream(stream)), "sq_fp_encode")
+    return out, a8
+
+
+
+def sq_fp_rmsnorm_encode(fmt: sq_format, X: torch.Tensor, gamma: torch.Tensor, eps: float, positions: torch.Tensor,
+                         out: Encoded | None = None, a8: torch.Tensor | None = None, stream=None):
+    """sq_fp_encode of rmsnorm(X) * gamma, the normalisation computed inside the encode; returns (Encoded, a8)."""
+    M, K = _bf16_2d(X, "X")
+    if gamma.dtype != torch.bfloat16 or gamma.numel() != K or not gamma.is_contiguous():
+        raise ValueError("gamma must be a contiguous bf16 tensor of K elements")
+    if out is None:
+        out = alloc_encoded(fmt, M, K, X.device)
+    if a8 is None:
+        a8 = torch.empty(max(M * K, 16), dtype=torch.uint8, device=X.device)[: M * K].view(M, K)
+    cs = out.c_struct()
+    _check(_lib.sq_fp_rmsnorm_encode(ctypes.byref(fmt), _ptr(X), _ptr(gamma), ctypes.c_float(eps), M, K, _ptr(positions),
+                                     ctypes.byref(cs), _ptr(a8), _stream(stream)), "sq_fp_rmsnorm_encode")
     return out, a8
 
 

@@ -242,7 +242,7 @@ sq_status sq_rmsnorm_encode(const sq_format* fmt, const void* X_bf16, const void
   SQ_TRY(check_device());
   int* status = status_word();
   if (status == nullptr) return SQ_ERR_CUDA;
-  const cudaError_t err = launch_rmsnorm_encode(fmt->bank, fmt->k, static_cast<const uint16_t*>(X_bf16),
+  const cudaError_t err = launch_rmsnorm_encode(fmt->bank, fmt->k, false, static_cast<const uint16_t*>(X_bf16),
                                                 static_cast<const uint16_t*>(gamma_bf16), eps, M, K, positions, *out,
                                                 static_cast<uint8_t*>(a8), status, static_cast<cudaStream_t>(cuda_stream));
   return err == cudaErrorNotSupported ? SQ_ERR_UNSUPPORTED : from_cuda(err);
@@ -400,6 +400,28 @@ sq_status sq_fp_encode(const sq_format* fmt, const void* X_bf16, int64_t M, int6
   }
   return from_cuda(launch_fp_encode(fmt->bank, fmt->k, static_cast<const uint16_t*>(X_bf16), M, K, positions, o, a8,
                                     static_cast<cudaStream_t>(cuda_stream)));
+}
+
+sq_status sq_fp_rmsnorm_encode(const sq_format* fmt, const void* X_bf16, const void* gamma_bf16, float eps, int64_t M,
+                               int64_t K, const uint8_t* positions, sq_encoded* out, uint8_t* a8, void* cuda_stream) {
+  SQ_TRY(check_format(fmt));
+  SQ_TRY(check_k(K));
+  if (!is_static(fmt) || is_indep(fmt)) return SQ_ERR_UNSUPPORTED;
+  if (M < 0 || !(eps >= 0.f)) return SQ_ERR_INVALID_ARG;
+  if (M == 0) return SQ_OK;
+  if (X_bf16 == nullptr || gamma_bf16 == nullptr || a8 == nullptr) return SQ_ERR_NULL_POINTER;
+  if (!aligned16(X_bf16) || !aligned16(gamma_bf16) || !aligned16(a8)) return SQ_ERR_ALIGNMENT;
+  SQ_TRY(check_positions(fmt, positions));
+  SQ_TRY(check_encoded(fmt, out));
+  SQ_TRY(check_device());
+  int* status = status_word();
+  if (status == nullptr) return SQ_ERR_CUDA;
+  sq_encoded o = *out;
+  o.idx = nullptr;
+  const cudaError_t err = launch_rmsnorm_encode(fmt->bank, fmt->k, true, static_cast<const uint16_t*>(X_bf16),
+                                                static_cast<const uint16_t*>(gamma_bf16), eps, M, K, positions, o, a8,
+                                                status, static_cast<cudaStream_t>(cuda_stream));
+  return err == cudaErrorNotSupported ? SQ_ERR_UNSUPPORTED : from_cuda(err);
 }
 
 sq_status sq_fp_gemm(const float* s_hi, const uint8_t* a8, const float* s_w, const uint8_t* w8, int64_t M, int64_t N,

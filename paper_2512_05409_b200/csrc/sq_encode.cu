@@ -1993,8 +1993,8 @@ cudaError_t launch_fp_encode_static_ring(int b, int k, const uint16_t* X, int64_
 // Root-mean-square normalisation fused into the static-position encode (tied scales): the ring
 // kernel normalises a row in its registers before it encodes it.  cudaErrorNotSupported = a row
 // length the ring kernel does not take, or one whose slots, tables and weights exceed shared memory.
-cudaError_t launch_rmsnorm_encode(int b, int k, const uint16_t* X, const uint16_t* gamma, float eps, int64_t M, int64_t K,
-                                  const uint8_t* positions, const sq_encoded& out, uint8_t* a8, int* status,
+cudaError_t launch_rmsnorm_encode(int b, int k, bool fp, const uint16_t* X, const uint16_t* gamma, float eps, int64_t M,
+                                  int64_t K, const uint8_t* positions, const sq_encoded& out, uint8_t* a8, int* status,
                                   cudaStream_t st) {
   if (positions == nullptr || M < 1) return cudaErrorNotSupported;
   EncodeParams p;
@@ -2018,6 +2018,7 @@ cudaError_t launch_rmsnorm_encode(int b, int k, const uint16_t* X, const uint16_
   p.mk = MulK{0xFFFFFFFFu, 2u, 32u, 256u, 65536u, 1u << 24, 16u, 1u};
   p.gamma = gamma;
   p.eps = eps;
+  if (fp) return launch_static_ring<false, true, true>(p, st);  // the floating-point variant's codes and scales
   return launch_static_ring<false, false, true>(p, st);
 }
 

@@ -69,8 +69,8 @@ cudaError_t launch_fp_pack_weights(const uint16_t* W, int64_t N, int64_t K, uint
                                    cudaStream_t st);
 cudaError_t launch_fp_encode(int b, int k, const uint16_t* X, int64_t M, int64_t K, const uint8_t* positions,
                              const sq_encoded& out, uint8_t* a8, cudaStream_t st);
-cudaError_t launch_rmsnorm_encode(int b, int k, const uint16_t* X, const uint16_t* gamma, float eps, int64_t M, int64_t K,
-                                  const uint8_t* positions, const sq_encoded& out, uint8_t* a8, int* status,
+cudaError_t launch_rmsnorm_encode(int b, int k, bool fp, const uint16_t* X, const uint16_t* gamma, float eps, int64_t M,
+                                  int64_t K, const uint8_t* positions, const sq_encoded& out, uint8_t* a8, int* status,
                                   cudaStream_t st);
 cudaError_t launch_fp_encode_static_ring(int b, int k, const uint16_t* X, int64_t M, int64_t K, const uint8_t* positions,
                                          const sq_encoded& out, uint8_t* a8, int* status, cudaStream_t st);

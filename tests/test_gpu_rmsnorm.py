@@ -120,3 +120,24 @@ def test_rmsnorm_encode_at_the_benchmark_sizes(M, K, b, k):
     # every row: scales are positive and finite, the largest INT8 magnitude of a row is 127
     assert torch.isfinite(enc.s_hi).all() and (enc.s_hi > 0).all()
     assert int(enc.vals.view(M, -1).abs().max(dim=1).values.min()) <= 127
+
+
+@pytest.mark.parametrize("M,K,b,k", [(75, 2048, 64, 8), (300, 4096, 128, 16), (513, 8192, 64, 8), (40, 7168, 128, 32)])
+def test_fp_rmsnorm_encode_matches_the_oracle(M, K, b, k):
+    """The floating-point variant's encode of the normalised rows, the normalisation inside the kernel:
+    codes, scales and the merged E4M3 operand against the oracle's encode of the oracle's normalisation."""
+    from test_gpu_fp_variant import _compare_encoded
+    fmt = sq.make_format(b, k, True)
+    X = gen.activations(M, K, seed=M + K + 2, outlier_fraction=0.01, outlier_scale=30.0, device="cuda")
+    X[0] = 0
+    X[1] = -3.0
+    gamma = _gamma(K, seed=K + 5)
+    pos = sq.sq_calib_positions(fmt, gen.calibration_batch(64, K, seed=K, outlier_fraction=0.01, outlier_scale=30.0, device="cuda"), None)
+    enc, a8 = sq.sq_fp_rmsnorm_encode(fmt, X, gamma, 1e-5, pos)
+    check_status()
+    y, _, ambiguous = oracle.rmsnorm(_bits(X), _bits(gamma), 1e-5)
+    assert not ambiguous.any()
+    _compare_encoded(enc, a8, oracle.fp_encode(b, k, y, _np(pos)))
+    with pytest.raises(sq.SqError) as e:
+        sq.sq_fp_rmsnorm_encode(sq.make_format(b, k, False), X, gamma, 1e-5, None)
+    assert e.value.status == sq.SQ_ERR_UNSUPPORTED
