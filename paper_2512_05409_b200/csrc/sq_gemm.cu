@@ -349,9 +349,12 @@ __global__ void __launch_bounds__(threads_of(MODE), 1)
   const uint32_t bar_eready = bar_wfull + 8 * NS;   // epilogue: column constants staged, every helper present
   const uint32_t bar_edone = bar_eready + 8;        // epilogue: every helper done with the constants
   const uint32_t bar_sfullp = bar_edone + 8;        // NS, leader: sparse K step filled by the peer's TMA
-  static_assert(8 * (5 * NS + 2 * NP + 4) + 16 <= kCtlBytes, "control block too small");
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(sCtl + 8 * (5 * NS + 2 * NP + 4));
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(sCtl + 8 * (5 * NS + 2 * NP + 4) + 8);
+  // leader, two issuing threads: the SECOND sub-tile's accumulator read out (bar_tempty is then the
+  // first one's alone, so its thread starts the next tile while the second is still being drained)
+  const uint32_t bar_tempty1 = bar_sfullp + 8 * NS;
+  static_assert(8 * (5 * NS + 2 * NP + 5) + 16 <= kCtlBytes, "control block too small");
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(sCtl + 8 * (5 * NS + 2 * NP + 5));
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(sCtl + 8 * (5 * NS + 2 * NP + 5) + 8);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   // Rank in the pair (0 = leader; clusters are (PAIR,1,1), so it is blockIdx.x % PAIR), this
@@ -382,6 +385,7 @@ __global__ void __launch_bounds__(threads_of(MODE), 1)
     }
     mbar_init(bar_tfull, A8 ? 2 : 1);
     mbar_init(bar_tempty, PAIR * kEpiAll * 32);
+    mbar_init(bar_tempty1, PAIR * kEpiAll * 32);
     mbar_init(bar_eready, kEpiAll * 32);
     mbar_init(bar_edone, kEpiAll * 32);
     *abort_flag = 0;
@@ -421,8 +425,14 @@ __global__ void __launch_bounds__(threads_of(MODE), 1)
     tc_fence_after();
     mbar_arrive(bar_eready);
     if (!mbar_wait(bar_eready, tile_count & 1u, abort_flag)) return false;
+    bool released0 = false;
     for (int ci = helper; ci < t.nsub * (BN / 32); ci += kEpiStep) {
       const int sub = ci / (BN / 32), c0 = (ci % (BN / 32)) * 32;
+      if (A8 && sub == 1 && !released0) {  // this thread's loads of the first accumulator are complete
+        tc_fence_before();
+        arrive_leader<PAIR>(bar_tempty);
+        released0 = true;
+      }
       const int m = t.m0 + sub * BM + 32 * q + lane;
       const float sh = sub == 0 ? sh2[0] : sh2[1];
       uint32_t v[32];
@@ -538,7 +548,8 @@ __global__ void __launch_bounds__(threads_of(MODE), 1)
       }
     }
     tc_fence_before();
-    arrive_leader<PAIR>(bar_tempty);
+    if (!released0) arrive_leader<PAIR>(bar_tempty);
+    if (A8) arrive_leader<PAIR>(bar_tempty1);
     mbar_arrive(bar_edone);
     return true;
   };
@@ -741,7 +752,8 @@ __global__ void __launch_bounds__(threads_of(MODE), 1)
         const Tile mt = tile_of<PAIR, SPLITK>(p, j, rank);
         const int nsub = mt.nsub;
         const int SS = STMA ? mt.ss : 0;
-        ok = wait_leader<PAIR>(bar_tempty, (tc & 1u) ^ 1u, abort_flag);  // previous tile's accumulators read out (both CTAs)
+        // previous tile's accumulator(s) read out (both CTAs); with two issuing threads each waits for its own
+        ok = wait_leader<PAIR>((A8 && warp == kMma2Warp) ? bar_tempty1 : bar_tempty, (tc & 1u) ^ 1u, abort_flag);
         if (!ok) break;
         tc_fence_after();
         // What a K step waits for: dense = the stage's "full" barrier (the producers or merge
