@@ -201,6 +201,12 @@ sq_status sq_encode(const sq_format* fmt, const void* X_bf16, int64_t M, int64_t
  *     a weight-streaming kernel.  The packed weights are the 128-row tensor-core operand (every
  *     SM streams its own slab of output channels), the tokens are the narrow one, K is cut over
  *     a thread-block cluster whose integer partial sums meet in distributed shared memory.
+ *     This kernel is launched with permission to start before its predecessor on the stream has
+ *     completed (programmatic dependent launch): until the predecessor has, it reads nothing but
+ *     W's packed codes -- its first weight tiles travel while, say, sq_encode of the same tokens
+ *     still runs (sq_encode's few-token kernel and this kernel allow their successor that early
+ *     start).  So W must not be the output of a kernel that is still running when this call is
+ *     made AND that itself releases its successors early; sq_pack_weights does not.
  *   - otherwise M <= 128: K is cut into 2-8 parts that run as one thread-block cluster per tile
  *     of 256 output channels and add their partial sums the same way.
  * Neither needs scratch memory; the result does not depend on the number of parts. */

@@ -516,6 +516,10 @@ __global__ void __launch_bounds__(B == 128 ? 256 : 512) encode_rows_kernel(const
 
   // shared memory: [static only: table of selected element offsets, uint16 [GK]] then per group
   // [nbuf rows][stash of selected raw values, uint16 [GK]][4 mbarriers][4 x 16 exchange words]
+  // A successor that was launched with permission to start early may do so now: what it does before
+  // its own wait for this kernel (the few-token product fetches its first weight tiles) runs beside
+  // the encode.  (This kernel itself starts only when its predecessor has completed.)
+  if (threadIdx.x == 0) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   const size_t table_bytes = kStatic ? (((size_t)GK * 2 + 127) & ~(size_t)127) : 0;
   uint16_t* jt = reinterpret_cast<uint16_t*>(smem_enc);
   uint8_t* wbase = smem_enc + table_bytes + (size_t)grp * p.group_stride;

@@ -142,6 +142,13 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&v)[16]) {
       : "memory");
 }
 
+// Programmatic dependent launch: this kernel may be started while its predecessor on the stream is
+// still running.  Until pdl_wait() returns (the predecessor has completed and its writes are
+// visible) it touches nothing a predecessor may have written -- only the weights, which are set up
+// long before: their first tiles are on their way while the activations are still being encoded.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 }  // namespace
 
 __global__ void __launch_bounds__(kThreadsS, 2)
@@ -213,7 +220,24 @@ __global__ void __launch_bounds__(kThreadsS, 2)
     if (lane == 0) {
       const uint32_t bytes = (uint32_t)(kPackW + kPackX + 2 * MT * SUP * p.nb);
       const int nsup = (KS + SUP - 1) / SUP;
-      for (int su = 0; su < nsup; ++su) {
+      // the ring's first stages: the weight tiles at once, the activation tiles when the predecessor is done
+      const int npre = nsup < NPK ? nsup : NPK;
+      for (int su = 0; su < npre; ++su) {
+        expect_tx(bar_pfull + 8 * su, bytes);
+        tma_2d(smem_u32(sPack + su * kPackStage), &map_w4, (k0 + su * SUP) * (BK / 2), n0, bar_pfull + 8 * su);
+      }
+      pdl_wait();
+      // From here on a successor may be started: whatever it does before its own wait (fetch its first
+      // weight tiles) overlaps this kernel, and its wait still covers this kernel's predecessor too.
+      pdl_launch_dependents();
+      for (int su = 0; su < npre; ++su) {
+        const uint32_t dst = smem_u32(sPack + su * kPackStage), bar = bar_pfull + 8 * su;
+        const int kx = k0 + su * SUP;
+        tma_2d(dst + kPackW, &map_x4, kx * (BK / 2), 0, bar);
+        tma_2d(dst + kPackW + kPackX, &map_sv, kx * p.nb, 0, bar);
+        tma_2d(dst + kPackW + kPackX + kSide, &map_si, kx * p.nb, 0, bar);
+      }
+      for (int su = npre; su < nsup; ++su) {
         const int ps = su % NPK;
         // (a last stage that holds fewer than SUP steps of this part never completes its "empty"
         // barrier; nothing is loaded after it, so nothing waits for it)
@@ -229,6 +253,7 @@ __global__ void __launch_bounds__(kThreadsS, 2)
     }
     __syncwarp();
   } else if ((warp >= kFirstW && warp < kFirstX) || (warp >= kFirstW2 && warp < kMma3Warp)) {
+    // (weights only: nothing here depends on the predecessor)
     // =============================================================== weights: group g takes steps g, g + 2, ...
     // A thread owns one output channel (its tensor-memory lane: quarter warp % 4, lane): it reads the
     // channel's 64 packed bytes of the step (the tile was laid down with the 64-byte swizzle, so the
@@ -278,6 +303,7 @@ __global__ void __launch_bounds__(kThreadsS, 2)
   } else if (warp >= kFirstX && warp < kMmaWarp) {
     // =============================================================== activations: warp x takes steps x, x + 4, ...
     const int xw = warp - kFirstX;
+    pdl_wait();  // the tokens' shifts below are the predecessor's to write
     // widening: 64 packed chunks, two per lane: chunk ci = lane + 32 * i -> row ci >> 2, chunk ci & 3
     uint32_t pmul[2], poff[2];
 #pragma unroll
@@ -380,6 +406,7 @@ __global__ void __launch_bounds__(kThreadsS, 2)
     // =============================================================== accumulator -> this CTA's partial sums
     // (the rings are idle once the accumulator is complete: every MMA has read its operands)
     const int q = warp & 3;  // a warp reads the tensor-memory lane quarter (warp index mod 4)
+    pdl_wait();  // the tokens' scales are the predecessor's to write (and `out` may be its to read)
     {
       // what the finish needs per channel and token, fetched while the K walk runs
       const int e = tid - kFirstEpi * 32, n = min(n0 + e, p.N - 1);
@@ -525,17 +552,20 @@ cudaError_t launch_stream(const StreamParams& p, const CUtensorMap& mw, const CU
   }
   cudaLaunchConfig_t lc;
   memset(&lc, 0, sizeof(lc));
-  cudaLaunchAttribute la[1];
-  la[0].id = cudaLaunchAttributeClusterDimension;
-  la[0].val.clusterDim.x = (unsigned)p.parts;
-  la[0].val.clusterDim.y = 1;
-  la[0].val.clusterDim.z = 1;
+  // attributes: the successor-may-start-early permission always, the cluster shape if K is cut
+  cudaLaunchAttribute la[2];
+  la[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  la[0].val.programmaticStreamSerializationAllowed = 1;
+  la[1].id = cudaLaunchAttributeClusterDimension;
+  la[1].val.clusterDim.x = (unsigned)p.parts;
+  la[1].val.clusterDim.y = 1;
+  la[1].val.clusterDim.z = 1;
   lc.gridDim = dim3((unsigned)(((p.N + SC - 1) / SC) * p.parts), 1, 1);
   lc.blockDim = dim3(kThreadsS, 1, 1);
   lc.dynamicSmemBytes = kSmemS;
   lc.stream = st;
   lc.attrs = la;
-  lc.numAttrs = p.parts > 1 ? 1 : 0;
+  lc.numAttrs = p.parts > 1 ? 2 : 1;
   return cudaLaunchKernelEx(&lc, gemm_stream_kernel, p, mw, mx, msv, msi);
 }
 
