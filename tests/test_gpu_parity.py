@@ -627,3 +627,58 @@ def test_fp8_tensor_rate_probe_runs_and_counts_its_operations():
     with pytest.raises(sq.SqError):
         sq.sq_probe_fp8_tensor_rate(0)
     run_pipeline(M=96, N=128, K=256, b=64, k=8, static=False, seed=12)
+
+
+# ----------------------------------------------------------------------------- few-token product started early
+
+def test_few_token_product_in_a_chain_reads_what_its_predecessor_wrote():
+    """The few-token product may start while the encode before it on the stream still runs (it only
+    fetches weights until that one has completed).  Chains of encode -> product over changing
+    inputs, issued back to back on one stream and replayed from a CUDA graph, must give what the
+    calls give one at a time: the product never sees the previous tokens' codes, scales or shifts,
+    and the next encode never overwrites them under a product that still reads them."""
+    fmt = sq.make_format(64, 8, False)
+    M, K, N = 16, 4096, 1032
+    W = gen.weights(N, K, seed=21, device="cuda")
+    w = sq.sq_pack_weights(fmt, W)
+    Xs = [gen.activations(M, K, seed=100 + i, outlier_fraction=0.01, outlier_scale=float(5 * (i + 1)), device="cuda") for i in range(6)]
+    # one at a time, with a synchronisation after every call
+    want = []
+    for X in Xs:
+        enc = sq.sq_encode(fmt, X)
+        torch.cuda.synchronize()
+        want.append(sq.sq_gemm(fmt, enc, w).clone())
+        torch.cuda.synchronize()
+    # back to back: ONE encoding buffer reused by every link of the chain
+    enc = sq.alloc_encoded(fmt, M, K, "cuda")
+    outs = [torch.empty(M, N, dtype=torch.bfloat16, device="cuda") for _ in Xs]
+
+    def chain():
+        for X, out in zip(Xs, outs):
+            sq.sq_encode(fmt, X, out=enc)
+            sq.sq_gemm(fmt, enc, w, out=out)
+    for _ in range(3):
+        for out in outs:
+            out.zero_()
+        chain()
+        torch.cuda.synchronize()
+        for got, ref in zip(outs, want):
+            assert torch.equal(got, ref)
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            chain()
+    for _ in range(3):
+        for out in outs:
+            out.zero_()
+        graph.replay()
+        torch.cuda.synchronize()
+        for got, ref in zip(outs, want):
+            assert torch.equal(got, ref)
+    check_status()
+    # ... and the first of them against the oracle
+    enc_ref = oracle.encode(64, 8, _bits(Xs[0]))
+    _, _, out_ref = oracle.gemm(64, 8, enc_ref, oracle.pack_weights(64, 8, _bits(W)))
+    assert np.array_equal(_bits(want[0]), out_ref)
