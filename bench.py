@@ -277,7 +277,7 @@ def bench_8b_dynamic(sq, dev, peaks, iters=20):
         g_ms, _ = time_launches(lambda i: sq.sq_gemm(l.fmt, l.enc, l.w, l.pos, out=l.out), iters, 10)
         f_ms, _ = time_launches(lambda i: sq.sq_gemm(l.fmt, l.enc, l.w, l.pos, out=l.out, use_workspace=False), iters, 5)
         tops, ftops = l.ops / (g_ms * 1e-3) / 1e12, l.ops / (f_ms * 1e-3) / 1e12
-        graph_us = wgbs = enc_graph_us = pair_graph_us = None
+        graph_us = wgbs = enc_graph_us = pair_graph_us = norm_pair_graph_us = None
         if M <= 128:
             graph_us = round(graph_replay_us(lambda: sq.sq_gemm(l.fmt, l.enc, l.w, l.pos, out=l.out)), 1)
             wgbs = round(N * K / 2 / (graph_us * 1e-6) / 1e9)
@@ -287,14 +287,23 @@ def bench_8b_dynamic(sq, dev, peaks, iters=20):
                 sq.sq_encode(l.fmt, l.X, l.pos, out=l.enc)
                 sq.sq_gemm(l.fmt, l.enc, l.w, l.pos, out=l.out)
             pair_graph_us = round(graph_replay_us(pair), 1)
+            gamma = torch.ones(K, dtype=torch.bfloat16, device=dev)
+
+            def norm_pair():  # the same chain with the layer normalisation inside the encode
+                sq.sq_rmsnorm_encode(l.fmt, l.X, gamma, 1e-5, None, out=l.enc, want_a8=False)
+                sq.sq_gemm(l.fmt, l.enc, l.w, l.pos, out=l.out)
+            try:
+                norm_pair_graph_us = round(graph_replay_us(norm_pair), 1)
+            except sq.SqError:
+                norm_pair_graph_us = None
         rows.append([M, K, N, round(e_ms * 1e3, 1), round(g_ms * 1e3, 1), graph_us, wgbs, round(tops, 1),
                      round(tops / int8_peak, 3), round(tops / 4500.0, 3), round(f_ms * 1e3, 1), round(ftops, 1), enc_graph_us,
-                     pair_graph_us])
+                     pair_graph_us, norm_pair_graph_us])
         del l
         torch.cuda.empty_cache()
     return {"cols": ["M", "K", "N", "encode_us", "gemm_us", "gemm_us_graph_replay", "weight_stream_GBps_graph_replay",
                      "TOPS", "of_measured_int8", "of_nominal_4500", "fused_gemm_us", "fused_TOPS", "encode_us_graph_replay",
-                     "encode_plus_gemm_us_graph_replay"],
+                     "encode_plus_gemm_us_graph_replay", "rmsnorm_encode_plus_gemm_us_graph_replay"],
             "rows": rows}
 
 

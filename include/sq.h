@@ -266,11 +266,15 @@ sq_status sq_gemm_a8(const sq_format* fmt, const sq_encoded* A, const sq_weights
  *     t  = bf16(fp32(x_j) * r)             fp32 product, round to nearest even
  *     y  = bf16(fp32(t) * fp32(gamma_j))   exact product, one rounding
  * and `out` (and a8, unless NULL) = sq_encode_a8 of y, bit for bit.  gamma_bf16: device bf16
- * [K], 16-byte aligned; eps >= 0.  Row lengths: those sq_encode_a8's own kernel takes (8/12/14/16
- * * 256 * {1,2,4,8}) whose row slots, tables and gamma fit shared memory (K = 4096 and 8192 do,
- * with or without a8); anything else, dynamic positions and SQ_POS_STATIC_INDEP:
- * SQ_ERR_UNSUPPORTED, nothing launched (normalise separately and call sq_encode).  Inputs
- * finite; X is not written. */
+ * [K], 16-byte aligned; eps >= 0.
+ *   SQ_POS_STATIC: row lengths that sq_encode_a8's own kernel takes (8/12/14/16 * 256 *
+ *     {1,2,4,8}) whose row slots, tables and gamma fit shared memory (K = 4096 and 8192 do, with
+ *     or without a8).
+ *   SQ_POS_DYNAMIC: k/b in {1/16, 1/8, 1/4, 1/2} (the ratios of sq_encode's fast kernel; the row
+ *     is normalised in shared memory before the selection, which then ranks the NORMALISED
+ *     magnitudes); a8, if given, is expanded from the codes by a second kernel on the stream.
+ *   Anything else, and SQ_POS_STATIC_INDEP: SQ_ERR_UNSUPPORTED, nothing launched (normalise
+ *   separately and call sq_encode).  Inputs finite; X is not written. */
 sq_status sq_rmsnorm_encode(const sq_format* fmt, const void* X_bf16, const void* gamma_bf16, float eps,
                             int64_t M, int64_t K, const uint8_t* positions, sq_encoded* out, void* a8,
                             void* cuda_stream);

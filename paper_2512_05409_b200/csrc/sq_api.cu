@@ -232,7 +232,7 @@ sq_status sq_rmsnorm_encode(const sq_format* fmt, const void* X_bf16, const void
                             int64_t K, const uint8_t* positions, sq_encoded* out, void* a8, void* cuda_stream) {
   SQ_TRY(check_format(fmt));
   SQ_TRY(check_k(K));
-  if (!is_static(fmt) || is_indep(fmt)) return SQ_ERR_UNSUPPORTED;
+  if (is_indep(fmt)) return SQ_ERR_UNSUPPORTED;
   if (M < 0 || !(eps >= 0.f)) return SQ_ERR_INVALID_ARG;
   if (M == 0) return SQ_OK;
   if (X_bf16 == nullptr || gamma_bf16 == nullptr) return SQ_ERR_NULL_POINTER;
@@ -242,10 +242,15 @@ sq_status sq_rmsnorm_encode(const sq_format* fmt, const void* X_bf16, const void
   SQ_TRY(check_device());
   int* status = status_word();
   if (status == nullptr) return SQ_ERR_CUDA;
-  const cudaError_t err = launch_rmsnorm_encode(fmt->bank, fmt->k, false, static_cast<const uint16_t*>(X_bf16),
-                                                static_cast<const uint16_t*>(gamma_bf16), eps, M, K, positions, *out,
-                                                static_cast<uint8_t*>(a8), status, static_cast<cudaStream_t>(cuda_stream));
-  return err == cudaErrorNotSupported ? SQ_ERR_UNSUPPORTED : from_cuda(err);
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  cudaError_t err = launch_rmsnorm_encode(fmt->bank, fmt->k, false, static_cast<const uint16_t*>(X_bf16),
+                                          static_cast<const uint16_t*>(gamma_bf16), eps, M, K,
+                                          is_static(fmt) ? positions : nullptr, *out, static_cast<uint8_t*>(a8), status, st);
+  if (err == cudaErrorNotSupported) return SQ_ERR_UNSUPPORTED;
+  // dynamic positions: the merged operand, if asked for, is expanded from the codes just written
+  if (err == cudaSuccess && !is_static(fmt) && a8 != nullptr)
+    err = launch_expand_a8(fmt->bank, fmt->k, *out, nullptr, M, K, static_cast<uint8_t*>(a8), st);
+  return from_cuda(err);
 }
 
 sq_status sq_gemm_workspace_bytes(const sq_format* fmt, int64_t M, int64_t N, int64_t K, size_t* bytes) {

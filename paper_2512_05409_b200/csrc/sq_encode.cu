@@ -497,7 +497,7 @@ __device__ __forceinline__ void group_sync(int rw, int grp) {
 
 // ------------------------------------------------------------------------------------------------
 // Row-group kernel.  B = bank size; KK = k for dynamic positions (a power of two), 0 for static.
-template <int B, int KK, bool FP = false>
+template <int B, int KK, bool FP = false, bool NORM = false>
 __global__ void __launch_bounds__(B == 128 ? 256 : 512) encode_rows_kernel(const EncodeParams p) {
   extern __shared__ __align__(128) uint8_t smem_enc[];
   constexpr bool kStatic = (KK == 0);
@@ -574,6 +574,46 @@ __global__ void __launch_bounds__(B == 128 ? 256 : 512) encode_rows_kernel(const
     // is done (the buffer is single) finds it there
     if (nbuf == 1 && lane == 0 && m + wstride < p.M)
       asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(p.X + (m + wstride) * K), "r"(row_bytes) : "memory");
+
+    if constexpr (NORM) {
+      // Fused normalisation: the staged row is replaced by bf16(bf16(x * r) * gamma), r from the
+      // row's mean of squares in fp64 (every square exact; four chains per lane), before anything
+      // else looks at it -- the rest of the kernel then encodes the normalised row.
+      uint4* rc = reinterpret_cast<uint4*>(row);
+      double s4[4] = {0.0, 0.0, 0.0, 0.0};
+      for (int c = lane; c < K / 8; c += gsize) {
+        const uint4 v = rc[c];
+        sq2_add(v.x, s4[0]);
+        sq2_add(v.y, s4[1]);
+        sq2_add(v.z, s4[2]);
+        sq2_add(v.w, s4[3]);
+      }
+      double ss = (s4[0] + s4[1]) + (s4[2] + s4[3]);
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+      if (rw > 1) {
+        uint32_t* exn = exch + 64;  // 2 x 16 words of their own
+        if ((threadIdx.x & 31) == 0) {
+          exn[warp % rw] = (uint32_t)__double2loint(ss);
+          exn[16 + warp % rw] = (uint32_t)__double2hiint(ss);
+        }
+        group_sync(rw, grp);
+        ss = 0.0;
+        for (int w = 0; w < rw; ++w) ss += __hiloint2double((int)exn[16 + w], (int)exn[w]);
+      }
+      const float rn = (float)(1.0 / sqrt(ss / (double)K + (double)p.eps));
+      const uint4* gc = reinterpret_cast<const uint4*>(p.gamma);
+      for (int c = lane; c < K / 8; c += gsize) {
+        uint4 v = rc[c];
+        const uint4 g = __ldg(gc + c);
+        v.x = norm2(v.x, rn, g.x);
+        v.y = norm2(v.y, rn, g.y);
+        v.z = norm2(v.z, rn, g.z);
+        v.w = norm2(v.w, rn, g.w);
+        rc[c] = v;
+      }
+      group_sync(rw, grp);  // the banks a lane reads below were written by other lanes
+    }
 
     // lane_rmax: static positions: the largest unselected magnitude.  Dynamic positions: an UPPER
     // bound of it (the largest k-th magnitude of any bank), with lane_rlow a LOWER bound (see below).
@@ -1747,7 +1787,7 @@ static cudaError_t device_and_sms(int* dev, int* sms) {
     }                                                                                                    \
   } while (0)
 
-template <int B, int KK, bool FP = false>
+template <int B, int KK, bool FP = false, bool NORM = false>
 cudaError_t launch_rows(const EncodeParams& base, cudaStream_t st) {
   EncodeParams p = base;
   const int K = p.K, G = K / B, k = (KK == 0) ? p.k : KK;
@@ -1756,7 +1796,7 @@ cudaError_t launch_rows(const EncodeParams& base, cudaStream_t st) {
   const size_t table = (KK == 0) ? ((((size_t)G * k * 2) + 127) & ~(size_t)127) : 0;  // static offset table
   const size_t budget = 224 * 1024 - table;
   const size_t row = (size_t)K * 2;
-  const size_t extra = side + 32 + 256 + 128;  // side buffer, four mbarriers, exchange words, rounding
+  const size_t extra = side + 32 + 256 + 128 + 128;  // side buffer, four mbarriers, exchange words (+ the normalisation's), rounding
   // Rows are single-buffered: with 16 resident warps the rows other groups have in flight
   // hide the copy latency, and a second buffer would only cost warps.  Pick the group size
   // that keeps the most warps resident, preferring smaller groups (less per-row overhead per
@@ -1773,6 +1813,20 @@ cudaError_t launch_rows(const EncodeParams& base, cudaStream_t st) {
       rw = cand;
     }
   }
+  int dev = 0, sms = 0;
+  cudaError_t err = device_and_sms(&dev, &sms);
+  if (err != cudaSuccess) return err;
+  // Few rows (decode, short prompts): latency, not throughput, is what counts.  As many warps per
+  // row as still give every row a group of its own in ONE wave of blocks, and every lane at least
+  // two 16-byte chunks (K = 4096, 16 tokens: 5.6 instead of 7.2 us; K = 14336: 5.9 instead of 9.8).
+  for (int cand = kMaxWarps; cand > rw; cand /= 2) {
+    if ((size_t)cand * 64 > (size_t)K / 8) continue;
+    const int groups = kMaxWarps / cand;
+    if ((p.M + groups - 1) / groups <= sms) {
+      rw = cand;
+      break;
+    }
+  }
   const size_t per_group = (((size_t)nbuf * row + extra) + 127) & ~(size_t)127;
   if (per_group > 224 * 1024) return cudaErrorNotSupported;
   int ngroups = kMaxWarps / rw;
@@ -1787,13 +1841,10 @@ cudaError_t launch_rows(const EncodeParams& base, cudaStream_t st) {
   const size_t smem = table + per_group * ngroups;
   if (smem > 227 * 1024) return cudaErrorNotSupported;  // long rows with many selected places: the plain kernel
 
-  int dev = 0, sms = 0;
-  cudaError_t err = device_and_sms(&dev, &sms);
-  if (err != cudaSuccess) return err;
-  SQ_ENSURE_SMEM((encode_rows_kernel<B, KK, FP>), dev, smem);
+  SQ_ENSURE_SMEM((encode_rows_kernel<B, KK, FP, NORM>), dev, smem);
   int64_t blocks = (p.M + ngroups - 1) / ngroups;
   if (blocks > sms) blocks = sms;
-  encode_rows_kernel<B, KK, FP><<<(unsigned)blocks, ngroups * rw * 32, smem, st>>>(p);
+  encode_rows_kernel<B, KK, FP, NORM><<<(unsigned)blocks, ngroups * rw * 32, smem, st>>>(p);
   return cudaGetLastError();
 }
 
@@ -2000,7 +2051,7 @@ cudaError_t launch_fp_encode_static_ring(int b, int k, const uint16_t* X, int64_
 cudaError_t launch_rmsnorm_encode(int b, int k, bool fp, const uint16_t* X, const uint16_t* gamma, float eps, int64_t M,
                                   int64_t K, const uint8_t* positions, const sq_encoded& out, uint8_t* a8, int* status,
                                   cudaStream_t st) {
-  if (positions == nullptr || M < 1) return cudaErrorNotSupported;
+  if (M < 1) return cudaErrorNotSupported;
   EncodeParams p;
   p.a8 = a8;
   p.X = X;
@@ -2022,6 +2073,19 @@ cudaError_t launch_rmsnorm_encode(int b, int k, bool fp, const uint16_t* X, cons
   p.mk = MulK{0xFFFFFFFFu, 2u, 32u, 256u, 65536u, 1u << 24, 16u, 1u};
   p.gamma = gamma;
   p.eps = eps;
+  if (positions == nullptr) {
+    // dynamic positions (integer variant, the row-group kernel's ratios): the staged row is
+    // normalised in shared memory before the selection; the merged operand is not this kernel's
+    if (fp) return cudaErrorNotSupported;
+    p.a8 = nullptr;
+#define SQ_DYN_NORM(BB, KK_) \
+  if (b == BB && k == KK_) return launch_rows<BB, KK_, false, true>(p, st);
+    SQ_DYN_NORM(32, 2) SQ_DYN_NORM(32, 4) SQ_DYN_NORM(32, 8) SQ_DYN_NORM(32, 16)
+    SQ_DYN_NORM(64, 4) SQ_DYN_NORM(64, 8) SQ_DYN_NORM(64, 16) SQ_DYN_NORM(64, 32)
+    SQ_DYN_NORM(128, 8) SQ_DYN_NORM(128, 16) SQ_DYN_NORM(128, 32) SQ_DYN_NORM(128, 64)
+#undef SQ_DYN_NORM
+    return cudaErrorNotSupported;
+  }
   if (fp) return launch_static_ring<false, true, true>(p, st);  // the floating-point variant's codes and scales
   return launch_static_ring<false, false, true>(p, st);
 }

@@ -682,3 +682,19 @@ def test_few_token_product_in_a_chain_reads_what_its_predecessor_wrote():
     enc_ref = oracle.encode(64, 8, _bits(Xs[0]))
     _, _, out_ref = oracle.gemm(64, 8, enc_ref, oracle.pack_weights(64, 8, _bits(W)))
     assert np.array_equal(_bits(want[0]), out_ref)
+
+
+@pytest.mark.parametrize("b,k", [(64, 8), (128, 16), (32, 4), (64, 32)])
+@pytest.mark.parametrize("M,K", [(1, 4096), (5, 14336), (16, 4096), (100, 14336), (148, 2048), (149, 4096), (300, 14336),
+                                 (37, 28672), (130, 8192)])
+def test_encode_few_rows_many_warps_per_row(b, k, M, K):
+    """Few rows: the encoder gives a row up to sixteen warps (every row a group of its own, all rows
+    in one wave of blocks) instead of packing many one-warp rows into a block; dynamic positions and
+    the static ones of row lengths the staged-row kernels leave to it."""
+    X = gen.activations(M, K, seed=M + K + b, outlier_fraction=0.01, outlier_scale=25.0, device="cuda")
+    fmt = sq.make_format(b, k, False)
+    enc = sq.sq_encode(fmt, X)
+    check_status()
+    compare_encoded(enc, oracle.encode(b, k, _bits(X)))
+    dec = sq.sq_decode(fmt, enc)
+    assert np.array_equal(_bits(dec), oracle.decode(b, k, oracle.encode(b, k, _bits(X)))[1])

@@ -83,8 +83,8 @@ def test_rmsnorm_encode_refuses_what_it_does_not_take():
     assert e.value.status == sq.SQ_ERR_UNSUPPORTED
     X2 = gen.activations(16, 2048, seed=1, device="cuda")
     g2 = _gamma(2048, seed=2)
-    with pytest.raises(sq.SqError) as e:       # dynamic positions
-        sq.sq_rmsnorm_encode(sq.make_format(64, 8, False), X2, g2, 1e-5, None)
+    with pytest.raises(sq.SqError) as e:       # dynamic positions at a ratio k/b the row-group kernel does not take
+        sq.sq_rmsnorm_encode(sq.make_format(64, 5, False), X2, g2, 1e-5, None)
     assert e.value.status == sq.SQ_ERR_UNSUPPORTED
     pos2 = sq.sq_calib_positions(sq.make_format(64, 8, True), gen.calibration_batch(64, 2048, seed=1, device="cuda"), None)
     with pytest.raises(sq.SqError) as e:       # independent scales
@@ -141,3 +141,58 @@ def test_fp_rmsnorm_encode_matches_the_oracle(M, K, b, k):
     with pytest.raises(sq.SqError) as e:
         sq.sq_fp_rmsnorm_encode(sq.make_format(b, k, False), X, gamma, 1e-5, None)
     assert e.value.status == sq.SQ_ERR_UNSUPPORTED
+
+
+@pytest.mark.parametrize("want_a8", [False, True])
+@pytest.mark.parametrize("M,K,b,k", [
+    (1, 4096, 64, 8),         # decode: one token
+    (16, 4096, 64, 8),
+    (16, 14336, 64, 8),       # the down projection's row length
+    (300, 2048, 32, 4),
+    (200, 4096, 128, 16),
+    (700, 8192, 64, 16),
+    (150, 1024, 64, 32),
+])
+def test_rmsnorm_encode_dynamic_positions(M, K, b, k, want_a8):
+    """Dynamic positions (the k largest magnitudes of every bank of the NORMALISED row): the row is
+    normalised in shared memory before the selection; codes, indices, scales and (expanded from
+    them) the merged operand against the oracle."""
+    fmt = sq.make_format(b, k, False)
+    X = gen.activations(M, K, seed=M + K + 7, outlier_fraction=0.01, outlier_scale=30.0, device="cuda")
+    if M > 2:
+        X[1] = 0
+        X[2] = 0.75
+    gamma = _gamma(K, seed=K + b + 1)
+    eps = 1e-5
+    keep = X.clone()
+    a8 = torch.full((M, K), 0x5A, dtype=torch.uint8, device="cuda") if want_a8 else None
+    enc, a8 = sq.sq_rmsnorm_encode(fmt, X, gamma, eps, None, a8=a8, want_a8=want_a8)
+    check_status()
+    assert torch.equal(X, keep)
+    enc_ref, _ = oracle.rmsnorm_encode(b, k, _bits(X), _bits(gamma), eps, None)
+    compare_encoded(enc, enc_ref)
+    if want_a8:
+        assert np.array_equal(_np(a8), merged_operand_from_oracle(b, k, enc_ref, None))
+
+
+def test_rmsnorm_encode_then_few_token_product_in_a_chain():
+    """The decode chain normalisation+encode -> product, back to back over changing tokens, against
+    the oracle's product of the oracle's encoding."""
+    fmt = sq.make_format(64, 8, False)
+    M, K, N = 16, 4096, 520
+    W = gen.weights(N, K, seed=31, device="cuda")
+    w = sq.sq_pack_weights(fmt, W)
+    w_ref = oracle.pack_weights(64, 8, _bits(W))
+    gamma = _gamma(K, seed=32)
+    Xs = [gen.activations(M, K, seed=200 + i, outlier_fraction=0.01, outlier_scale=20.0, device="cuda") for i in range(4)]
+    enc = sq.alloc_encoded(fmt, M, K, "cuda")
+    outs = [torch.empty(M, N, dtype=torch.bfloat16, device="cuda") for _ in Xs]
+    for X, out in zip(Xs, outs):
+        sq.sq_rmsnorm_encode(fmt, X, gamma, 1e-5, None, out=enc, want_a8=False)
+        sq.sq_gemm(fmt, enc, w, out=out)
+    torch.cuda.synchronize()
+    check_status()
+    for X, out in zip(Xs, outs):
+        enc_ref, _ = oracle.rmsnorm_encode(64, 8, _bits(X), _bits(gamma), 1e-5, None)
+        _, _, out_ref = oracle.gemm(64, 8, enc_ref, w_ref)
+        assert np.array_equal(_bits(out), out_ref)
