@@ -307,6 +307,35 @@ def bench_8b_dynamic(sq, dev, peaks, iters=20):
             "rows": rows}
 
 
+def bench_decode_static(sq, dev, peaks):
+    """Few tokens with STATIC positions (b=64, k=8) on the 8B-decoder shapes: GPU time per call of sq_gemm
+    and of the chain sq_encode -> sq_gemm replayed from a CUDA graph, and the INT4 weight stream over the
+    product's time."""
+    rows = []
+    fmt = sq.make_format(64, 8, True)
+    for (K, N) in SHAPES_8B:
+        W = gen.weights(N, K, seed=K + N, device=dev)
+        pos = sq.sq_calib_positions(fmt, gen.calibration_batch(512, K, seed=K, outlier_fraction=0.01, outlier_scale=20.0, device=dev), W)
+        w = sq.sq_pack_weights(fmt, W, pos)
+        del W
+        for M in (1, 16):
+            X = gen.activations(M, K, seed=M, outlier_fraction=0.01, outlier_scale=20.0, device=dev)
+            enc = sq.sq_encode(fmt, X, pos)
+            out = torch.empty(M, N, dtype=torch.bfloat16, device=dev)
+            g_us = graph_replay_us(lambda: sq.sq_gemm(fmt, enc, w, pos, out=out))
+
+            def pair():
+                sq.sq_encode(fmt, X, pos, out=enc)
+                sq.sq_gemm(fmt, enc, w, pos, out=out)
+            p_us = graph_replay_us(pair)
+            gbs = N * K / 2 / (g_us * 1e-6) / 1e9
+            rows.append([M, K, N, round(g_us, 1), round(gbs), round(gbs / peaks["hbm_gbs"], 3), round(p_us, 1)])
+        del w
+        torch.cuda.empty_cache()
+    return {"cols": ["M", "K", "N", "gemm_us_graph_replay", "weight_stream_GBps", "of_measured_hbm", "encode_plus_gemm_us_graph_replay"],
+            "rows": rows}
+
+
 def bench_gemm_fused(sq, layers, dev, peaks, iters=10):
     """Plain sq_gemm (no workspace): the sparse INT8 part runs inside the GEMM kernel -- static
     positions as TMA-fed gathered K steps, dynamic positions merged into the widened activation
@@ -821,6 +850,8 @@ def run_cuda(args):
                               **bench_encode_only(sq, dev, peaks)}
             line["gemm_fused"] = {"workload": "70B-shaped linears, M=4096, b=128, k=16: plain sq_gemm (sparse part inside the GEMM kernel) vs the workspace call",
                                   **bench_gemm_fused(sq, layers, dev, peaks)}
+            line["decode_static"] = {"workload": "8B-decoder-shaped linears, 1 and 16 tokens, b=64, k=8, STATIC positions (the weight-streaming kernel with one shared row of places)",
+                                     **bench_decode_static(sq, dev, peaks)}
             line["weights_sq"] = {"workload": "weights in SQ-format (implicit mask, b=64, k=8) x per-token INT8 activations, 8B-decoder shapes, 1 and 4 tokens",
                                   **bench_weights_sq(sq, dev, peaks)}
             line["producer_fusion"] = {"workload": "sq_rmsnorm_encode: bf16 [M,K] Student-t nu=3, 0.5% channels x50, static positions; GBps = (2 + 0.5 + k/b) bytes per element over the fused call (the unfused pair moves 4 more: the normalised tensor written and read back); median of 30 launches",

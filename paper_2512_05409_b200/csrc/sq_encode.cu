@@ -1243,6 +1243,9 @@ __global__ void __launch_bounds__(NT, 1) encode_static_ring_kernel(const EncodeP
   if (threadIdx.x == 0) {
     abort_flag_s = 0;
     next_row_s = ngroups;
+    // a successor launched with permission to start early (the few-token product: it fetches only
+    // weight tiles until this kernel has completed) may do so now
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   }
   // The first rows are asked for as early as possible, but after the positions: issued before
   // them, the grid's first 19 MB of rows would keep the tables waiting.  So every thread first

@@ -1251,7 +1251,8 @@ cudaError_t launch_gemm(int b, int k, bool indep, const sq_encoded& A, const sq_
                         const uint8_t* positions, int64_t M, int64_t N, int64_t K, uint16_t* out,
                         int32_t* acc_out, int* status, void* workspace, size_t workspace_bytes, bool allow_stream,
                         cudaStream_t st, bool a8_ready) {
-  if (allow_stream && !indep && gemm_stream_serves(b, k, positions != nullptr, M, K))
+  // (the few-token kernel fetches static positions through TMA: 16-byte aligned ones only)
+  if (allow_stream && !indep && (reinterpret_cast<uintptr_t>(positions) & 15) == 0 && gemm_stream_serves(b, k, positions != nullptr, M, K))
     return launch_gemm_stream(b, k, A, W, positions, M, N, K, out, acc_out, status, st);
   GemmParams p;
   p.dq4 = A.dq4;

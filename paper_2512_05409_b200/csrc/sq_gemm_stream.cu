@@ -87,6 +87,7 @@ struct StreamParams {
   int* status;
   int M, N, K, b, k;
   int nb;        // sparse entries per row and K step
+  int shared_positions;  // static positions: every token's entries sit at the same places (one row of them is loaded)
   int parts;     // parts of K per slab = cluster size
   int KS;        // K steps per part
 };
@@ -351,7 +352,8 @@ __global__ void __launch_bounds__(kThreadsS, 2)
       __syncwarp();  // the tile is written: its sparse entries now overwrite the (zero) places they belong to
       if (mrow < p.M) {
         const uint8_t* sv = pk + kPackX + mrow * (SUP * p.nb) + (ks % SUP) * p.nb + first;
-        const uint8_t* si = sv + kSide;
+        // (static positions: the tile of places has one row, shared by all tokens)
+        const uint8_t* si = p.shared_positions ? pk + kPackX + kSide + (ks % SUP) * p.nb + first : sv + kSide;
         uint8_t* xrow = x_st + mrow * 128;
         int cnt = c_first;
         uint32_t boff = boff_first;
@@ -573,7 +575,8 @@ cudaError_t launch_stream(const StreamParams& p, const CUtensorMap& mw, const CU
 
 // Whether launch_gemm_stream takes this call (else the tiled kernel of sq_gemm.cu does).
 bool gemm_stream_serves(int b, int k, bool is_static, int64_t M, int64_t K) {
-  if (M < 1 || M > MT || is_static) return false;
+  (void)is_static;  // static positions: the merge reads one shared row of places instead of a row per token
+  if (M < 1 || M > MT) return false;
   const int64_t GK = (K / b) * k;
   const int nb = (BK / b) * k;
   if (GK % 16 != 0) return false;                     // TMA row pitch of vals / idx
@@ -624,6 +627,7 @@ cudaError_t launch_gemm_stream(int b, int k, const sq_encoded& A, const sq_weigh
   p.b = b;
   p.k = k;
   p.nb = nb;
+  p.shared_positions = positions != nullptr ? 1 : 0;
   // Parts of K per slab: up to four, as long as every part is at least four K steps long and the
   // launch still fits the GPU in one wave (two CTAs per SM; a cluster's CTAs are co-scheduled).
   // (Eight parts were measured slower on every shape: what a part saves in K steps, 0.3 us each,
@@ -641,7 +645,10 @@ cudaError_t launch_gemm_stream(int b, int k, const sq_encoded& A, const sq_weigh
   if (!make_map_u8(encode, &mw, W.wq4, (uint64_t)(K / 2), (uint64_t)N, (uint64_t)(K / 2), kPitch, SC, SUP == 1 ? 64 : 128)) return cudaErrorInvalidValue;
   if (!make_map_u8(encode, &mx, A.dq4, (uint64_t)(K / 2), (uint64_t)M, (uint64_t)(K / 2), kPitch, MT, 0)) return cudaErrorInvalidValue;
   if (!make_map_u8(encode, &msv, A.vals, (uint64_t)GK, (uint64_t)M, (uint64_t)GK, (uint32_t)(SUP * nb), MT, 0)) return cudaErrorInvalidValue;
-  if (!make_map_u8(encode, &msi, A.idx, (uint64_t)GK, (uint64_t)M, (uint64_t)GK, (uint32_t)(SUP * nb), MT, 0)) return cudaErrorInvalidValue;
+  // places: a row per token (dynamic), or the one row of static positions (rows past it come back as zeros, unread)
+  if (!make_map_u8(encode, &msi, positions != nullptr ? positions : A.idx, (uint64_t)GK, positions != nullptr ? 1u : (uint64_t)M,
+                   (uint64_t)GK, (uint32_t)(SUP * nb), MT, 0))
+    return cudaErrorInvalidValue;
   return launch_stream(p, mw, mx, msv, msi, dev, st);
 }
 

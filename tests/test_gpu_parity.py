@@ -698,3 +698,11 @@ def test_encode_few_rows_many_warps_per_row(b, k, M, K):
     compare_encoded(enc, oracle.encode(b, k, _bits(X)))
     dec = sq.sq_decode(fmt, enc)
     assert np.array_equal(_bits(dec), oracle.decode(b, k, oracle.encode(b, k, _bits(X)))[1])
+
+
+@pytest.mark.parametrize("b,k", [(64, 8), (128, 16), (32, 4), (64, 16)])
+@pytest.mark.parametrize("M,N,K", [(1, 520, 1024), (16, 264, 2048), (5, 1032, 4096), (3, 520, 14336), (16, 8, 512), (9, 4104, 4096)])
+def test_few_tokens_static_positions_on_the_weight_streaming_kernel(b, k, M, N, K):
+    """At most 16 tokens with STATIC positions: the weight-streaming kernel merges the sparse entries
+    at the places of one shared row of positions (a per-token row of them for dynamic positions)."""
+    run_pipeline(M=M, N=N, K=K, b=b, k=k, static=True, seed=M + N + K)
