@@ -197,10 +197,11 @@ sq_status sq_encode(const sq_format* fmt, const void* X_bf16, int64_t M, int64_t
  * given, the raw accumulators are written as well (used by parity tests);
  * SQ_POS_STATIC_INDEP: [2, M, N], acc_lo then acc_hi.
  * Few rows: nothing changes in the result, only in how the work is laid out.
- *   - M <= 16, K-step selections of 16..64 entries that are a multiple of 16 (static positions:
- *     a 16-byte aligned positions array):
+ *   - M <= 32 (and 33 <= M <= 64 while N <= 128 * the number of SMs), K-step selections of 16..64
+ *     entries that are a multiple of 16 (static positions: a 16-byte aligned positions array):
  *     a weight-streaming kernel.  The packed weights are the 128-row tensor-core operand (every
- *     SM streams its own slab of output channels), the tokens are the narrow one, K is cut over
+ *     SM streams its own slab of output channels), the tokens are the narrow one (16, 32 or 64
+ *     accumulator columns), K is cut over
  *     a thread-block cluster whose integer partial sums meet in distributed shared memory.
  *     This kernel is launched with permission to start before its predecessor on the stream has
  *     completed (programmatic dependent launch): until the predecessor has, it reads nothing but

@@ -1223,7 +1223,7 @@ static bool use_a8(bool /*is_static*/, int64_t M, int64_t N, int64_t K, size_t w
 
 size_t gemm_workspace_bytes(int b, int k, bool is_static, bool indep, int64_t M, int64_t N, int64_t K) {
   if (indep) return 0;  // two accumulators: neither a merged 8-bit operand nor split-K is built for it
-  if (gemm_stream_serves(b, k, is_static, M, K)) return 0;  // the weight-streaming kernel needs none
+  if (gemm_stream_serves(b, k, is_static, M, N, K)) return 0;  // the weight-streaming kernel needs none
   int dev = 0, sms = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) return 0;
   if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
@@ -1252,7 +1252,7 @@ cudaError_t launch_gemm(int b, int k, bool indep, const sq_encoded& A, const sq_
                         int32_t* acc_out, int* status, void* workspace, size_t workspace_bytes, bool allow_stream,
                         cudaStream_t st, bool a8_ready) {
   // (the few-token kernel fetches static positions through TMA: 16-byte aligned ones only)
-  if (allow_stream && !indep && (reinterpret_cast<uintptr_t>(positions) & 15) == 0 && gemm_stream_serves(b, k, positions != nullptr, M, K))
+  if (allow_stream && !indep && (reinterpret_cast<uintptr_t>(positions) & 15) == 0 && gemm_stream_serves(b, k, positions != nullptr, M, N, K))
     return launch_gemm_stream(b, k, A, W, positions, M, N, K, out, acc_out, status, st);
   GemmParams p;
   p.dq4 = A.dq4;

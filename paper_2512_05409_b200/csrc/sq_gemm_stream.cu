@@ -51,31 +51,43 @@ namespace sq {
 namespace {
 
 constexpr int SC = 128;        // output channels per slab = rows of the MMA = tensor-memory lanes
-constexpr int MT = 16;         // token columns of the accumulator
+constexpr int kMaxTokens = 64; // token columns of the accumulator: 16, 32 or 64 (see SG)
 constexpr int BK = 128;        // K elements per step = bytes per operand row
 constexpr int SUP = 2;         // K steps per packed stage: the TMA engine moves a tile row by row, and 128-byte rows cost it
                                // half of what 64-byte rows do per byte (one step per stage left the weight warps waiting for data)
 constexpr int NPK = 4;         // packed stages in flight
 constexpr int NW = 6;          // widened weight stages (in tensor memory)
-constexpr int NX = 8;          // widened activation stages
 constexpr int kWGroups = 2, kWGroupThreads = 128, kXWarps = 4;
 constexpr int kTmaWarp = 0, kFirstW = 1, kFirstX = 5, kMmaWarp = 9, kFirstEpi = 10, kMma2Warp = 14, kFirstW2 = 15, kMma3Warp = 19;
-constexpr int kIssuers = 3;     // MMA-issuing threads (steps j, j + 3, ... into accumulator j)
 constexpr int kThreadsS = 20 * 32;
 constexpr int ND = 24;         // "step done" barriers: a common multiple of NW and NX
 constexpr int kCtlBars = 512;
-constexpr int kCtlS = kCtlBars + 2 * SC * 4 + MT * 4;  // barriers, then the slab's constants for the finish
 constexpr int kPitch = SUP * (BK / 2);     // bytes per packed row of a stage
-constexpr int kPackW = SC * kPitch;        // 32 KB
-constexpr int kPackX = MT * kPitch;        // 4 KB
-constexpr int kSide = MT * SUP * 64;       // sparse values / indices of a stage: up to 64 per row and step
-constexpr int kPackStage = kPackW + kPackX + 2 * kSide;
+constexpr int kPackW = SC * kPitch;        // 16 KB
 constexpr int kColsW = BK / 4;              // tensor-memory columns of a widened weight stage (128 lanes x 128 bytes)
-constexpr int kAccCols = kIssuers * MT;    // one accumulator per issuing thread
-constexpr int kStageX = MT * BK;           // 2 KB
-constexpr int kSmemS = NX * kStageX + NPK * kPackStage + kCtlS;
-static_assert(kStageX % 1024 == 0 && kPackStage % 1024 == 0 && (NX * kStageX) % 1024 == 0 && SUP <= 2, "stage alignment (swizzled weight tiles)");
-static_assert(SC * MT * 4 <= NPK * kPackStage, "partial sums are parked in the packed ring");
+// What depends on MT, the token columns of the accumulator (= the N of the MMA).  16 tokens: three
+// issuing threads, two CTAs per SM.  32 and 64 tokens: two issuing threads (tensor-memory columns),
+// fewer activation stages (shared memory), one CTA per SM.
+template <int MT_>
+struct SG {
+  static constexpr int MT = MT_;
+  static constexpr int kIssuers = MT == 16 ? 3 : 2;  // MMA-issuing threads (steps j, j + kIssuers, ... into accumulator j)
+  static constexpr int NX = MT == 16 ? 8 : 4;         // widened activation stages
+  static constexpr int kCtlS = kCtlBars + 2 * SC * 4 + MT * 4;  // barriers, then the slab's constants for the finish
+  static constexpr int kPackX = MT * kPitch;        // packed activations of a stage
+  static constexpr int kSide = MT * SUP * 64;       // sparse values / indices of a stage: up to 64 per row and step
+  static constexpr int kPackStage = kPackW + kPackX + 2 * kSide;
+  static constexpr int kAccCols = kIssuers * MT;    // one accumulator per issuing thread
+  static constexpr int kStageX = MT * BK;
+  static constexpr int kSmemS = NX * kStageX + NPK * kPackStage + kCtlS;
+  static constexpr uint32_t kTmemCols = kAccCols + NW * kColsW <= 256 ? 256u : 512u;
+  static constexpr int kCtasPerSm = MT == 16 ? 2 : 1;
+  // D = s32; A (weights, 16 * code) signed; B (activations) unsigned with offset 128; both K-major; M = 128, N = MT
+  static constexpr uint32_t kIdesc = (2u << 4) | (1u << 7) | (0u << 10) | ((uint32_t)(MT >> 3) << 17) | ((uint32_t)(SC >> 4) << 24);
+  static_assert(kStageX % 1024 == 0 && kPackStage % 1024 == 0 && (NX * kStageX) % 1024 == 0 && SUP <= 2, "stage alignment (swizzled weight tiles)");
+  static_assert(SC * MT * 4 <= NPK * kPackStage, "partial sums are parked in the packed ring");
+  static_assert(ND % NX == 0 && kAccCols + NW * kColsW <= 512 && kSmemS <= 227 * 1024, "rings");
+};
 
 struct StreamParams {
   const float* s_hi;
@@ -101,9 +113,6 @@ __device__ __forceinline__ uint64_t desc_sw128(uint32_t saddr) {
   d |= (uint64_t)2 << 61;
   return d;
 }
-// D = s32; A (weights, 16 * code) signed; B (activations) unsigned with offset 128; both K-major;
-// M = 128, N = 16.
-constexpr uint32_t kIdescStream = (2u << 4) | (1u << 7) | (0u << 10) | ((uint32_t)(MT >> 3) << 17) | ((uint32_t)(SC >> 4) << 24);
 __device__ __forceinline__ uint32_t kpos_byte(uint32_t jj) {  // position of bank-local element jj in the MMA's K order
   return (jj & 0x60u) | ((jj & 1u) << 4) | ((jj & 31u) >> 1);
 }
@@ -152,9 +161,13 @@ __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepc
 
 }  // namespace
 
-__global__ void __launch_bounds__(kThreadsS, 2)
+template <int MT>
+__global__ void __launch_bounds__(kThreadsS, SG<MT>::kCtasPerSm)
     gemm_stream_kernel(const StreamParams p, const __grid_constant__ CUtensorMap map_w4, const __grid_constant__ CUtensorMap map_x4,
                        const __grid_constant__ CUtensorMap map_sv, const __grid_constant__ CUtensorMap map_si) {
+  using G = SG<MT>;
+  constexpr int kIssuers = G::kIssuers, NX = G::NX, kPackX = G::kPackX, kSide = G::kSide, kPackStage = G::kPackStage;
+  constexpr int kAccCols = G::kAccCols, kStageX = G::kStageX;
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   uint8_t* smem = smem_raw;
   if ((smem_u32(smem_raw) & 1023u) != 0) {
@@ -172,7 +185,7 @@ __global__ void __launch_bounds__(kThreadsS, 2)
                                                      // ONE commit per step frees both the weight and the activation stage
   const uint32_t bar_tfull = bar_done + 8 * ND;      // accumulator complete
   constexpr int kBars = 2 * NPK + NW + NX + ND + 1;
-  static_assert(ND % NW == 0 && ND % NX == 0, "a step's barrier must not come round before its stages do");
+  static_assert(ND % NW == 0, "a step's barrier must not come round before its stages do");
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(sCtl + 8 * kBars);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(sCtl + 8 * kBars + 8);
   static_assert(8 * kBars + 16 <= kCtlBars, "control block too small");
@@ -185,8 +198,7 @@ __global__ void __launch_bounds__(kThreadsS, 2)
   const int slab = (int)blockIdx.x / parts, part = (int)blockIdx.x % parts;  // part = rank in the cluster
   const int n0 = slab * SC;
   const int KS = p.KS, k0 = part * KS;
-  constexpr uint32_t kTmemCols = 256;  // 2 x 16 accumulator columns, then NW x 32 columns of widened weights
-  static_assert(kAccCols + NW * kColsW <= 256, "tensor-memory columns");
+  constexpr uint32_t kTmemCols = G::kTmemCols;  // the accumulators' columns, then NW x 32 columns of widened weights
 
   if (warp == kTmaWarp) {
     if (lane == 0) {  // the descriptors are on their way while the barriers are set up
@@ -305,36 +317,38 @@ __global__ void __launch_bounds__(kThreadsS, 2)
     // =============================================================== activations: warp x takes steps x, x + 4, ...
     const int xw = warp - kFirstX;
     pdl_wait();  // the tokens' shifts below are the predecessor's to write
-    // widening: 64 packed chunks, two per lane: chunk ci = lane + 32 * i -> row ci >> 2, chunk ci & 3
-    uint32_t pmul[2], poff[2];
+    // widening: 4 * MT packed chunks, CPL per lane: chunk ci = lane + 32 * i -> row ci >> 2, chunk ci & 3
+    constexpr int CPL = MT / 8;
+    uint32_t pmul[CPL], poff[CPL];
 #pragma unroll
-    for (int i = 0; i < 2; ++i) {
+    for (int i = 0; i < CPL; ++i) {
       const int row = (lane + 32 * i) >> 2;
       const uint32_t e = row < p.M ? p.shift[row] : 0u;
       pmul[i] = 1u << e;
       poff[i] = 0x01010101u * (128u - (8u << e));
     }
-    // merge: two lanes share a row; each takes half of the step's nb entries.  The bank of an entry
-    // (and so its K offset inside the step) follows from its index by counting, no division per entry.
-    const int mrow = lane >> 1, run = p.nb >> 1, first = (lane & 1) * run;
+    // merge: LPR lanes share a row (two for 16 tokens, one otherwise), each takes its share of the
+    // step's nb entries; 32 / LPR rows per pass.  The bank of an entry (and so its K offset inside
+    // the step) follows from its index by counting, no division per entry.
+    constexpr int LPR = MT <= 32 ? 32 / MT : 1, RPP = 32 / LPR;
+    const int run = p.nb / LPR, first = (lane % LPR) * run;
     const int c_first = first % p.k;
     const uint32_t boff_first = (uint32_t)((first / p.k) * p.b);
-    const uint32_t swz = (uint32_t)((mrow & 7) << 4);
     bool ok = true;
     for (int ks = xw; ks < KS && ok; ks += kXWarps) {
       const int su = ks / SUP, ps = su % NPK, sx = ks % NX;
       ok = mbar_wait_park(bar_pfull + 8 * ps, (su / NPK) & 1u, abort_flag);
       if (!ok) break;
       const uint8_t* pk = sPack + ps * kPackStage + kPackW;
-      uint4 rx[2];
+      uint4 rx[CPL];
 #pragma unroll
-      for (int i = 0; i < 2; ++i)
+      for (int i = 0; i < CPL; ++i)
         rx[i] = *reinterpret_cast<const uint4*>(pk + ((lane + 32 * i) >> 2) * kPitch + (ks % SUP) * 64 + (lane & 3) * 16);
       if (ks >= NX) ok = mbar_wait_park(bar_done + 8 * ((ks - NX) % ND), ((ks - NX) / ND) & 1u, abort_flag);
       if (!ok) break;
       uint8_t* x_st = sX + sx * kStageX;
 #pragma unroll
-      for (int i = 0; i < 2; ++i) {
+      for (int i = 0; i < CPL; ++i) {
         const int row = (lane + 32 * i) >> 2, cc = lane & 3;
         const uint32_t in[4] = {rx[i].x, rx[i].y, rx[i].z, rx[i].w};
         uint32_t ev[4], od[4];
@@ -350,7 +364,11 @@ __global__ void __launch_bounds__(kThreadsS, 2)
         *reinterpret_cast<uint4*>(dst + (se ^ 16u)) = make_uint4(od[0], od[1], od[2], od[3]);
       }
       __syncwarp();  // the tile is written: its sparse entries now overwrite the (zero) places they belong to
-      if (mrow < p.M) {
+#pragma unroll
+      for (int pass = 0; pass < MT / RPP; ++pass) {
+        const int mrow = pass * RPP + lane / LPR;
+        if (mrow >= p.M) continue;
+        const uint32_t swz = (uint32_t)((mrow & 7) << 4);
         const uint8_t* sv = pk + kPackX + mrow * (SUP * p.nb) + (ks % SUP) * p.nb + first;
         // (static positions: the tile of places has one row, shared by all tokens)
         const uint8_t* si = p.shared_positions ? pk + kPackX + kSide + (ks % SUP) * p.nb + first : sv + kSide;
@@ -384,10 +402,10 @@ __global__ void __launch_bounds__(kThreadsS, 2)
     // =============================================================== MMA issuers
     // A K step is four small instructions, but waiting for its two operands, issuing and
     // committing take one thread ~0.5 us: that, not the stream, set the pace of the whole kernel.
-    // So THREE threads issue, thread j the steps j, j + 3, ..., each into an accumulator of its own
-    // (the sums are integers: the finish adds them, in any order the same).
-    if (lane == 0) {
-      const int j = warp == kMmaWarp ? 0 : (warp == kMma2Warp ? 1 : 2);
+    // So THREE threads issue (two for more than 16 tokens), thread j the steps j, j + kIssuers, ..., each
+    // into an accumulator of its own (the sums are integers: the finish adds them, in any order the same).
+    const int j = warp == kMmaWarp ? 0 : (warp == kMma2Warp ? 1 : 2);
+    if (lane == 0 && j < kIssuers) {
       bool ok = true;
       for (int ks = j; ks < KS && ok; ks += kIssuers) {
         const int s = ks % NW, sx = ks % NX;
@@ -398,7 +416,7 @@ __global__ void __launch_bounds__(kThreadsS, 2)
         const uint64_t db = desc_sw128(smem_u32(sX + sx * kStageX));
 #pragma unroll
         for (int kk = 0; kk < BK / 32; ++kk)
-          umma_i8_ta(tmem + (uint32_t)(j * MT), ta + 8 * kk, db + 2 * kk, kIdescStream, (ks > j || kk > 0) ? 1u : 0u);
+          umma_i8_ta(tmem + (uint32_t)(j * MT), ta + 8 * kk, db + 2 * kk, G::kIdesc, (ks > j || kk > 0) ? 1u : 0u);
         umma_commit<1>(bar_done + 8 * (ks % ND));
       }
       if (ok && j < KS) umma_commit<1>(bar_tfull);
@@ -420,23 +438,26 @@ __global__ void __launch_bounds__(kThreadsS, 2)
       tc_fence_after();
       const int ch = 32 * q + lane;
       int4* prow = reinterpret_cast<int4*>(sPack) + ch * (MT / 4);
-      uint32_t v[16];
-      tmem_ld16(tmem + ((uint32_t)(32 * q) << 16), v);
 #pragma unroll
-      for (int j = 1; j < kIssuers; ++j)
-        if (KS > j) {  // the other issuing threads' accumulators
-          uint32_t v2[16];
-          tmem_ld16(tmem + ((uint32_t)(32 * q) << 16) + (uint32_t)(j * MT), v2);
-          tmem_ld_wait();
+      for (int c16 = 0; c16 < MT / 16; ++c16) {  // sixteen tokens at a time
+        uint32_t v[16];
+        tmem_ld16(tmem + ((uint32_t)(32 * q) << 16) + (uint32_t)(16 * c16), v);
 #pragma unroll
-          for (int c = 0; c < 16; ++c) v[c] += v2[c];
-        }
-      tmem_ld_wait();
-      // (a warp's 16-byte stores, one 64-byte row per lane, spread over the banks by themselves)
-      prow[0] = make_int4((int)v[0], (int)v[1], (int)v[2], (int)v[3]);
-      prow[1] = make_int4((int)v[4], (int)v[5], (int)v[6], (int)v[7]);
-      prow[2] = make_int4((int)v[8], (int)v[9], (int)v[10], (int)v[11]);
-      prow[3] = make_int4((int)v[12], (int)v[13], (int)v[14], (int)v[15]);
+        for (int j = 1; j < kIssuers; ++j)
+          if (KS > j) {  // the other issuing threads' accumulators
+            uint32_t v2[16];
+            tmem_ld16(tmem + ((uint32_t)(32 * q) << 16) + (uint32_t)(j * MT + 16 * c16), v2);
+            tmem_ld_wait();
+#pragma unroll
+            for (int c = 0; c < 16; ++c) v[c] += v2[c];
+          }
+        tmem_ld_wait();
+        // (a warp's 16-byte stores, one row of MT sums per lane, spread over the banks by themselves)
+        prow[4 * c16] = make_int4((int)v[0], (int)v[1], (int)v[2], (int)v[3]);
+        prow[4 * c16 + 1] = make_int4((int)v[4], (int)v[5], (int)v[6], (int)v[7]);
+        prow[4 * c16 + 2] = make_int4((int)v[8], (int)v[9], (int)v[10], (int)v[11]);
+        prow[4 * c16 + 3] = make_int4((int)v[12], (int)v[13], (int)v[14], (int)v[15]);
+      }
     }
     tc_fence_before();
   }
@@ -542,13 +563,14 @@ bool make_map_u8(PFN_cuTensorMapEncodeTiled encode, CUtensorMap* out, const void
   return true;
 }
 
+template <int MT>
 cudaError_t launch_stream(const StreamParams& p, const CUtensorMap& mw, const CUtensorMap& mx, const CUtensorMap& msv,
                           const CUtensorMap& msi, int dev, cudaStream_t st) {
   static std::atomic<bool> attr_set[64];
   cudaError_t err;
   if (!attr_set[dev].load(std::memory_order_acquire)) {
     std::lock_guard<std::mutex> lock(setup_mutex());
-    err = cudaFuncSetAttribute(gemm_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemS);
+    err = cudaFuncSetAttribute(gemm_stream_kernel<MT>, cudaFuncAttributeMaxDynamicSharedMemorySize, SG<MT>::kSmemS);
     if (err != cudaSuccess) return err;
     attr_set[dev].store(true, std::memory_order_release);
   }
@@ -564,19 +586,26 @@ cudaError_t launch_stream(const StreamParams& p, const CUtensorMap& mw, const CU
   la[1].val.clusterDim.z = 1;
   lc.gridDim = dim3((unsigned)(((p.N + SC - 1) / SC) * p.parts), 1, 1);
   lc.blockDim = dim3(kThreadsS, 1, 1);
-  lc.dynamicSmemBytes = kSmemS;
+  lc.dynamicSmemBytes = SG<MT>::kSmemS;
   lc.stream = st;
   lc.attrs = la;
   lc.numAttrs = p.parts > 1 ? 2 : 1;
-  return cudaLaunchKernelEx(&lc, gemm_stream_kernel, p, mw, mx, msv, msi);
+  return cudaLaunchKernelEx(&lc, gemm_stream_kernel<MT>, p, mw, mx, msv, msi);
 }
 
 }  // namespace
 
 // Whether launch_gemm_stream takes this call (else the tiled kernel of sq_gemm.cu does).
-bool gemm_stream_serves(int b, int k, bool is_static, int64_t M, int64_t K) {
+bool gemm_stream_serves(int b, int k, bool is_static, int64_t M, int64_t N, int64_t K) {
   (void)is_static;  // static positions: the merge reads one shared row of places instead of a row per token
-  if (M < 1 || M > MT) return false;
+  if (M < 1 || M > kMaxTokens) return false;
+  // 33..64 tokens run one CTA per SM: worth it only while every slab of 128 channels has an SM of its
+  // own (measured: 13.0 against 14.2 us at N = K = 4096, but 40 against 37 us at N = 28672)
+  if (M > 32) {
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return false;
+    if ((N + SC - 1) / SC > sms) return false;
+  }
   const int64_t GK = (K / b) * k;
   const int nb = (BK / b) * k;
   if (GK % 16 != 0) return false;                     // TMA row pitch of vals / idx
@@ -586,7 +615,7 @@ bool gemm_stream_serves(int b, int k, bool is_static, int64_t M, int64_t K) {
 
 cudaError_t launch_gemm_stream(int b, int k, const sq_encoded& A, const sq_weights& W, const uint8_t* positions, int64_t M,
                                int64_t N, int64_t K, uint16_t* out, int32_t* acc_out, int* status, cudaStream_t st) {
-  if (!gemm_stream_serves(b, k, positions != nullptr, M, K)) return cudaErrorNotSupported;
+  if (!gemm_stream_serves(b, k, positions != nullptr, M, N, K)) return cudaErrorNotSupported;
   const int64_t GK = (K / b) * k;
   const int nb = (BK / b) * k;
 
@@ -632,10 +661,12 @@ cudaError_t launch_gemm_stream(int b, int k, const sq_encoded& A, const sq_weigh
   // launch still fits the GPU in one wave (two CTAs per SM; a cluster's CTAs are co-scheduled).
   // (Eight parts were measured slower on every shape: what a part saves in K steps, 0.3 us each,
   // the larger cluster's barriers and the finish's remote reads take back.)
+  // Token columns: 16, 32 or 64 (more columns: fewer issuing threads and stages, one CTA per SM).
+  const int mt = M <= 16 ? 16 : (M <= 32 ? 32 : 64);
   const int64_t slabs = (N + SC - 1) / SC, ks = K / BK;
   int parts = 1;
   for (int cand = 2; cand <= 4; cand *= 2) {
-    if (ks % cand != 0 || ks / cand < 4 || slabs * cand > 2 * (int64_t)sms) break;
+    if (ks % cand != 0 || ks / cand < 4 || slabs * cand > (mt == 16 ? 2 : 1) * (int64_t)sms) break;
     parts = cand;
   }
   p.parts = parts;
@@ -643,13 +674,15 @@ cudaError_t launch_gemm_stream(int b, int k, const sq_encoded& A, const sq_weigh
 
   CUtensorMap mw, mx, msv, msi;
   if (!make_map_u8(encode, &mw, W.wq4, (uint64_t)(K / 2), (uint64_t)N, (uint64_t)(K / 2), kPitch, SC, SUP == 1 ? 64 : 128)) return cudaErrorInvalidValue;
-  if (!make_map_u8(encode, &mx, A.dq4, (uint64_t)(K / 2), (uint64_t)M, (uint64_t)(K / 2), kPitch, MT, 0)) return cudaErrorInvalidValue;
-  if (!make_map_u8(encode, &msv, A.vals, (uint64_t)GK, (uint64_t)M, (uint64_t)GK, (uint32_t)(SUP * nb), MT, 0)) return cudaErrorInvalidValue;
+  if (!make_map_u8(encode, &mx, A.dq4, (uint64_t)(K / 2), (uint64_t)M, (uint64_t)(K / 2), kPitch, (uint32_t)mt, 0)) return cudaErrorInvalidValue;
+  if (!make_map_u8(encode, &msv, A.vals, (uint64_t)GK, (uint64_t)M, (uint64_t)GK, (uint32_t)(SUP * nb), (uint32_t)mt, 0)) return cudaErrorInvalidValue;
   // places: a row per token (dynamic), or the one row of static positions (rows past it come back as zeros, unread)
   if (!make_map_u8(encode, &msi, positions != nullptr ? positions : A.idx, (uint64_t)GK, positions != nullptr ? 1u : (uint64_t)M,
-                   (uint64_t)GK, (uint32_t)(SUP * nb), MT, 0))
+                   (uint64_t)GK, (uint32_t)(SUP * nb), (uint32_t)mt, 0))
     return cudaErrorInvalidValue;
-  return launch_stream(p, mw, mx, msv, msi, dev, st);
+  if (mt == 16) return launch_stream<16>(p, mw, mx, msv, msi, dev, st);
+  if (mt == 32) return launch_stream<32>(p, mw, mx, msv, msi, dev, st);
+  return launch_stream<64>(p, mw, mx, msv, msi, dev, st);
 }
 
 }  // namespace sq

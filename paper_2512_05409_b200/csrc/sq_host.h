@@ -51,7 +51,7 @@ cudaError_t launch_expand_a8(int b, int k, const sq_encoded& A, const uint8_t* p
 // Bytes of workspace launch_gemm can make use of for this shape and format (0: none).
 size_t gemm_workspace_bytes(int b, int k, bool is_static, bool indep, int64_t M, int64_t N, int64_t K);
 // The weight-streaming kernel for at most 32 token rows (sq_gemm_stream.cu).
-bool gemm_stream_serves(int b, int k, bool is_static, int64_t M, int64_t K);
+bool gemm_stream_serves(int b, int k, bool is_static, int64_t M, int64_t N, int64_t K);
 cudaError_t launch_gemm_stream(int b, int k, const sq_encoded& A, const sq_weights& W, const uint8_t* positions,
                                int64_t M, int64_t N, int64_t K, uint16_t* out, int32_t* acc_out, int* status,
                                cudaStream_t st);

@@ -330,9 +330,9 @@ def test_split_k_with_workspace(b, k, static, M, K):
     enc = sq.sq_encode(fmt, X, pos)
     need = sq.sq_gemm_workspace_bytes(fmt, M, N, K)
     if need == 0:
-        # at most 32 rows in a format the weight-streaming kernel serves: no workspace is of use
+        # at most 64 rows in a format the weight-streaming kernel serves: no workspace is of use
         # (one that is passed anyway is ignored)
-        assert M <= 16
+        assert M <= 64
         need = 8 * M * N * 4
     else:
         assert need % (M * N * 4) == 0 and need // (M * N * 4) in (2, 4, 8)
@@ -706,3 +706,14 @@ def test_few_tokens_static_positions_on_the_weight_streaming_kernel(b, k, M, N, 
     """At most 16 tokens with STATIC positions: the weight-streaming kernel merges the sparse entries
     at the places of one shared row of positions (a per-token row of them for dynamic positions)."""
     run_pipeline(M=M, N=N, K=K, b=b, k=k, static=True, seed=M + N + K)
+
+
+@pytest.mark.parametrize("static", [False, True])
+@pytest.mark.parametrize("b,k", [(64, 8), (128, 16), (32, 4), (64, 32)])
+@pytest.mark.parametrize("M,N,K", [(17, 264, 1024), (32, 1032, 4096), (25, 520, 14336), (33, 264, 2048), (48, 4104, 4096),
+                                   (64, 136, 1536), (64, 19080, 1024)])
+def test_up_to_64_tokens_on_the_weight_streaming_kernel(b, k, static, M, N, K):
+    """17..32 and 33..64 tokens: the weight-streaming kernel with 32 / 64 accumulator columns (two
+    issuing threads, one CTA per SM); the last shape has more slabs of 128 channels than SMs, which
+    sends 33..64 tokens to the tiled kernel instead."""
+    run_pipeline(M=M, N=N, K=K, b=b, k=k, static=static, seed=M + N + K + b)
