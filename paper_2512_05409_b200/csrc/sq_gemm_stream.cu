@@ -57,7 +57,7 @@ constexpr int SUP = 2;         // K steps per packed stage: the TMA engine moves
                                // half of what 64-byte rows do per byte (one step per stage left the weight warps waiting for data)
 constexpr int NPK = 4;         // packed stages in flight
 constexpr int NW = 6;          // widened weight stages (in tensor memory)
-constexpr int kWGroups = 2, kWGroupThreads = 128, kXWarps = 4;
+constexpr int kWGroups = 2, kWGroupThreads = 128;
 constexpr int kTmaWarp = 0, kFirstW = 1, kFirstX = 5, kMmaWarp = 9, kFirstEpi = 10, kMma2Warp = 14, kFirstW2 = 15, kMma3Warp = 19;
 constexpr int kThreadsS = 20 * 32;
 constexpr int ND = 24;         // "step done" barriers: a common multiple of NW and NX
@@ -72,7 +72,10 @@ template <int MT_>
 struct SG {
   static constexpr int MT = MT_;
   static constexpr int kIssuers = MT == 16 ? 3 : 2;  // MMA-issuing threads (steps j, j + kIssuers, ... into accumulator j)
-  static constexpr int NX = MT == 16 ? 8 : 4;         // widened activation stages
+  static constexpr int NX = 8;                         // widened activation stages
+  // warps that widen and merge activations: four; beyond 16 tokens (their work grows with MT) the four
+  // epilogue warps, idle during the K walk, make it eight
+  static constexpr int kXWarps = MT == 16 ? 4 : 8;
   static constexpr int kCtlS = kCtlBars + 2 * SC * 4 + MT * 4;  // barriers, then the slab's constants for the finish
   static constexpr int kPackX = MT * kPitch;        // packed activations of a stage
   static constexpr int kSide = MT * SUP * 64;       // sparse values / indices of a stage: up to 64 per row and step
@@ -166,7 +169,7 @@ __global__ void __launch_bounds__(kThreadsS, SG<MT>::kCtasPerSm)
     gemm_stream_kernel(const StreamParams p, const __grid_constant__ CUtensorMap map_w4, const __grid_constant__ CUtensorMap map_x4,
                        const __grid_constant__ CUtensorMap map_sv, const __grid_constant__ CUtensorMap map_si) {
   using G = SG<MT>;
-  constexpr int kIssuers = G::kIssuers, NX = G::NX, kPackX = G::kPackX, kSide = G::kSide, kPackStage = G::kPackStage;
+  constexpr int kIssuers = G::kIssuers, NX = G::NX, kXWarps = G::kXWarps, kPackX = G::kPackX, kSide = G::kSide, kPackStage = G::kPackStage;
   constexpr int kAccCols = G::kAccCols, kStageX = G::kStageX;
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   uint8_t* smem = smem_raw;
@@ -228,6 +231,91 @@ __global__ void __launch_bounds__(kThreadsS, SG<MT>::kCtasPerSm)
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
 
+  // =============================================================== activations: warp xw of kXWarps takes steps xw, xw + kXWarps, ...
+  auto x_role = [&](const int xw) {
+    pdl_wait();  // the tokens' shifts below are the predecessor's to write
+    // widening: 4 * MT packed chunks, CPL per lane: chunk ci = lane + 32 * i -> row ci >> 2, chunk ci & 3
+    constexpr int CPL = MT / 8;
+    uint32_t pmul[CPL], poff[CPL];
+#pragma unroll
+    for (int i = 0; i < CPL; ++i) {
+      const int row = (lane + 32 * i) >> 2;
+      const uint32_t e = row < p.M ? p.shift[row] : 0u;
+      pmul[i] = 1u << e;
+      poff[i] = 0x01010101u * (128u - (8u << e));
+    }
+    // merge: LPR lanes share a row (two for 16 tokens, one otherwise), each takes its share of the
+    // step's nb entries; 32 / LPR rows per pass.  The bank of an entry (and so its K offset inside
+    // the step) follows from its index by counting, no division per entry.
+    constexpr int LPR = MT <= 32 ? 32 / MT : 1, RPP = 32 / LPR;
+    const int run = p.nb / LPR, first = (lane % LPR) * run;
+    const int c_first = first % p.k;
+    const uint32_t boff_first = (uint32_t)((first / p.k) * p.b);
+    bool ok = true;
+    for (int ks = xw; ks < KS && ok; ks += kXWarps) {
+      const int su = ks / SUP, ps = su % NPK, sx = ks % NX;
+      ok = mbar_wait_park(bar_pfull + 8 * ps, (su / NPK) & 1u, abort_flag);
+      if (!ok) break;
+      const uint8_t* pk = sPack + ps * kPackStage + kPackW;
+      uint4 rx[CPL];
+#pragma unroll
+      for (int i = 0; i < CPL; ++i)
+        rx[i] = *reinterpret_cast<const uint4*>(pk + ((lane + 32 * i) >> 2) * kPitch + (ks % SUP) * 64 + (lane & 3) * 16);
+      if (ks >= NX) ok = mbar_wait_park(bar_done + 8 * ((ks - NX) % ND), ((ks - NX) / ND) & 1u, abort_flag);
+      if (!ok) break;
+      uint8_t* x_st = sX + sx * kStageX;
+#pragma unroll
+      for (int i = 0; i < CPL; ++i) {
+        const int row = (lane + 32 * i) >> 2, cc = lane & 3;
+        const uint32_t in[4] = {rx[i].x, rx[i].y, rx[i].z, rx[i].w};
+        uint32_t ev[4], od[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          const uint32_t u = in[q] ^ 0x88888888u;
+          ev[q] = (u & 0x0F0F0F0Fu) * pmul[i] + poff[i];
+          od[q] = ((u >> 4) & 0x0F0F0F0Fu) * pmul[i] + poff[i];
+        }
+        const uint32_t se = (uint32_t)(((2 * cc) ^ (row & 7)) << 4);
+        uint8_t* dst = x_st + row * 128;
+        *reinterpret_cast<uint4*>(dst + se) = make_uint4(ev[0], ev[1], ev[2], ev[3]);
+        *reinterpret_cast<uint4*>(dst + (se ^ 16u)) = make_uint4(od[0], od[1], od[2], od[3]);
+      }
+      __syncwarp();  // the tile is written: its sparse entries now overwrite the (zero) places they belong to
+#pragma unroll
+      for (int pass = 0; pass < MT / RPP; ++pass) {
+        const int mrow = pass * RPP + lane / LPR;
+        if (mrow >= p.M) continue;
+        const uint32_t swz = (uint32_t)((mrow & 7) << 4);
+        const uint8_t* sv = pk + kPackX + mrow * (SUP * p.nb) + (ks % SUP) * p.nb + first;
+        // (static positions: the tile of places has one row, shared by all tokens)
+        const uint8_t* si = p.shared_positions ? pk + kPackX + kSide + (ks % SUP) * p.nb + first : sv + kSide;
+        uint8_t* xrow = x_st + mrow * 128;
+        int cnt = c_first;
+        uint32_t boff = boff_first;
+        // eight entries at a time: their indices and values come with one 8-byte read each (a lane's
+        // run starts on an 8-byte boundary: nb is a multiple of 16), and the eight byte stores do
+        // not wait for one another
+        for (int j0 = 0; j0 < run; j0 += 8) {
+          const uint2 iv = *reinterpret_cast<const uint2*>(si + j0);
+          const uint2 vv = *reinterpret_cast<const uint2*>(sv + j0);
+          const uint32_t vx = vv.x ^ 0x80808080u, vy = vv.y ^ 0x80808080u;
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            const uint32_t jj = ((j < 4 ? iv.x : iv.y) >> (8 * (j & 3))) & 0xFFu;
+            const uint32_t val = ((j < 4 ? vx : vy) >> (8 * (j & 3))) & 0xFFu;
+            xrow[(kpos_byte(jj) + boff) ^ swz] = (uint8_t)val;
+            if (++cnt == p.k) {
+              cnt = 0;
+              boff += (uint32_t)p.b;
+            }
+          }
+        }
+      }
+      mbar_arrive(bar_pempty + 8 * ps);
+      fence_proxy_async_smem();
+      mbar_arrive(bar_xfull + 8 * sx);
+    }
+  };
   if (warp == kTmaWarp) {
     // =============================================================== TMA: packed tiles of every K step
     if (lane == 0) {
@@ -314,90 +402,7 @@ __global__ void __launch_bounds__(kThreadsS, SG<MT>::kCtasPerSm)
       mbar_arrive(bar_wfull + 8 * s);
     }
   } else if (warp >= kFirstX && warp < kMmaWarp) {
-    // =============================================================== activations: warp x takes steps x, x + 4, ...
-    const int xw = warp - kFirstX;
-    pdl_wait();  // the tokens' shifts below are the predecessor's to write
-    // widening: 4 * MT packed chunks, CPL per lane: chunk ci = lane + 32 * i -> row ci >> 2, chunk ci & 3
-    constexpr int CPL = MT / 8;
-    uint32_t pmul[CPL], poff[CPL];
-#pragma unroll
-    for (int i = 0; i < CPL; ++i) {
-      const int row = (lane + 32 * i) >> 2;
-      const uint32_t e = row < p.M ? p.shift[row] : 0u;
-      pmul[i] = 1u << e;
-      poff[i] = 0x01010101u * (128u - (8u << e));
-    }
-    // merge: LPR lanes share a row (two for 16 tokens, one otherwise), each takes its share of the
-    // step's nb entries; 32 / LPR rows per pass.  The bank of an entry (and so its K offset inside
-    // the step) follows from its index by counting, no division per entry.
-    constexpr int LPR = MT <= 32 ? 32 / MT : 1, RPP = 32 / LPR;
-    const int run = p.nb / LPR, first = (lane % LPR) * run;
-    const int c_first = first % p.k;
-    const uint32_t boff_first = (uint32_t)((first / p.k) * p.b);
-    bool ok = true;
-    for (int ks = xw; ks < KS && ok; ks += kXWarps) {
-      const int su = ks / SUP, ps = su % NPK, sx = ks % NX;
-      ok = mbar_wait_park(bar_pfull + 8 * ps, (su / NPK) & 1u, abort_flag);
-      if (!ok) break;
-      const uint8_t* pk = sPack + ps * kPackStage + kPackW;
-      uint4 rx[CPL];
-#pragma unroll
-      for (int i = 0; i < CPL; ++i)
-        rx[i] = *reinterpret_cast<const uint4*>(pk + ((lane + 32 * i) >> 2) * kPitch + (ks % SUP) * 64 + (lane & 3) * 16);
-      if (ks >= NX) ok = mbar_wait_park(bar_done + 8 * ((ks - NX) % ND), ((ks - NX) / ND) & 1u, abort_flag);
-      if (!ok) break;
-      uint8_t* x_st = sX + sx * kStageX;
-#pragma unroll
-      for (int i = 0; i < CPL; ++i) {
-        const int row = (lane + 32 * i) >> 2, cc = lane & 3;
-        const uint32_t in[4] = {rx[i].x, rx[i].y, rx[i].z, rx[i].w};
-        uint32_t ev[4], od[4];
-#pragma unroll
-        for (int q = 0; q < 4; ++q) {
-          const uint32_t u = in[q] ^ 0x88888888u;
-          ev[q] = (u & 0x0F0F0F0Fu) * pmul[i] + poff[i];
-          od[q] = ((u >> 4) & 0x0F0F0F0Fu) * pmul[i] + poff[i];
-        }
-        const uint32_t se = (uint32_t)(((2 * cc) ^ (row & 7)) << 4);
-        uint8_t* dst = x_st + row * 128;
-        *reinterpret_cast<uint4*>(dst + se) = make_uint4(ev[0], ev[1], ev[2], ev[3]);
-        *reinterpret_cast<uint4*>(dst + (se ^ 16u)) = make_uint4(od[0], od[1], od[2], od[3]);
-      }
-      __syncwarp();  // the tile is written: its sparse entries now overwrite the (zero) places they belong to
-#pragma unroll
-      for (int pass = 0; pass < MT / RPP; ++pass) {
-        const int mrow = pass * RPP + lane / LPR;
-        if (mrow >= p.M) continue;
-        const uint32_t swz = (uint32_t)((mrow & 7) << 4);
-        const uint8_t* sv = pk + kPackX + mrow * (SUP * p.nb) + (ks % SUP) * p.nb + first;
-        // (static positions: the tile of places has one row, shared by all tokens)
-        const uint8_t* si = p.shared_positions ? pk + kPackX + kSide + (ks % SUP) * p.nb + first : sv + kSide;
-        uint8_t* xrow = x_st + mrow * 128;
-        int cnt = c_first;
-        uint32_t boff = boff_first;
-        // eight entries at a time: their indices and values come with one 8-byte read each (a lane's
-        // run starts on an 8-byte boundary: nb is a multiple of 16), and the eight byte stores do
-        // not wait for one another
-        for (int j0 = 0; j0 < run; j0 += 8) {
-          const uint2 iv = *reinterpret_cast<const uint2*>(si + j0);
-          const uint2 vv = *reinterpret_cast<const uint2*>(sv + j0);
-          const uint32_t vx = vv.x ^ 0x80808080u, vy = vv.y ^ 0x80808080u;
-#pragma unroll
-          for (int j = 0; j < 8; ++j) {
-            const uint32_t jj = ((j < 4 ? iv.x : iv.y) >> (8 * (j & 3))) & 0xFFu;
-            const uint32_t val = ((j < 4 ? vx : vy) >> (8 * (j & 3))) & 0xFFu;
-            xrow[(kpos_byte(jj) + boff) ^ swz] = (uint8_t)val;
-            if (++cnt == p.k) {
-              cnt = 0;
-              boff += (uint32_t)p.b;
-            }
-          }
-        }
-      }
-      mbar_arrive(bar_pempty + 8 * ps);
-      fence_proxy_async_smem();
-      mbar_arrive(bar_xfull + 8 * sx);
-    }
+    x_role(warp - kFirstX);
   } else if (warp == kMmaWarp || warp == kMma2Warp || warp == kMma3Warp) {
     // =============================================================== MMA issuers
     // A K step is four small instructions, but waiting for its two operands, issuing and
@@ -434,6 +439,7 @@ __global__ void __launch_bounds__(kThreadsS, SG<MT>::kCtasPerSm)
       s_sw[e] = __ldg(p.s_w + n);
       if (e < MT) s_sh[e] = e < p.M ? __ldg(p.s_hi + e) : 0.f;
     }
+    if constexpr (kXWarps == 8) x_role(4 + (warp - kFirstEpi));  // idle until the accumulator is complete otherwise
     if (mbar_wait_idle(bar_tfull, 0, abort_flag)) {
       tc_fence_after();
       const int ch = 32 * q + lane;
