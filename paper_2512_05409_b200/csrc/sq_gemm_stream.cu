@@ -443,7 +443,9 @@ __global__ void __launch_bounds__(kThreadsS, SG<MT>::kCtasPerSm)
     if (mbar_wait_idle(bar_tfull, 0, abort_flag)) {
       tc_fence_after();
       const int ch = 32 * q + lane;
-      int4* prow = reinterpret_cast<int4*>(sPack) + ch * (MT / 4);
+      // parked token-major, [MT][SC]: a warp's 32 channels of a token are one 128-byte store, and
+      // the finish reads eight channels of a token with two 16-byte loads
+      int32_t* pcol = reinterpret_cast<int32_t*>(sPack) + ch;
 #pragma unroll
       for (int c16 = 0; c16 < MT / 16; ++c16) {  // sixteen tokens at a time
         uint32_t v[16];
@@ -458,11 +460,8 @@ __global__ void __launch_bounds__(kThreadsS, SG<MT>::kCtasPerSm)
             for (int c = 0; c < 16; ++c) v[c] += v2[c];
           }
         tmem_ld_wait();
-        // (a warp's 16-byte stores, one row of MT sums per lane, spread over the banks by themselves)
-        prow[4 * c16] = make_int4((int)v[0], (int)v[1], (int)v[2], (int)v[3]);
-        prow[4 * c16 + 1] = make_int4((int)v[4], (int)v[5], (int)v[6], (int)v[7]);
-        prow[4 * c16 + 2] = make_int4((int)v[8], (int)v[9], (int)v[10], (int)v[11]);
-        prow[4 * c16 + 3] = make_int4((int)v[12], (int)v[13], (int)v[14], (int)v[15]);
+#pragma unroll
+        for (int c = 0; c < 16; ++c) pcol[(16 * c16 + c) * SC] = (int)v[c];
       }
     }
     tc_fence_before();
@@ -476,46 +475,55 @@ __global__ void __launch_bounds__(kThreadsS, SG<MT>::kCtasPerSm)
   {
     // CTA `part` finishes channels [part * SC / parts, (part + 1) * SC / parts) of the slab for all
     // tokens: adds the parts' sums (integer: order-free) and runs the usual epilogue arithmetic.
-    const int share = SC / parts, lg = 31 - __clz(share);  // parts is 1, 2, 4 or 8
-    const int quads = (p.M + 3) >> 2;                        // a thread takes four tokens of one channel:
-    for (int i = tid; i < share * quads; i += kThreadsS) {   // one 16-byte (remote) read per part
-      const int ch = part * share + (i & (share - 1)), m0 = (i >> lg) << 2;
-      const int n = n0 + ch;
+    // A thread takes eight channels of one token: two 16-byte (remote) reads per part, one 16-byte
+    // store of the bf16 outputs (N is a multiple of 8, so a group is inside N or outside).
+    const int share = SC / parts, g8s = share >> 3, lg = 31 - __clz(g8s);  // parts is 1, 2 or 4
+    for (int i = tid; i < p.M * g8s; i += kThreadsS) {
+      const int ch0 = part * share + ((i & (g8s - 1)) << 3), m = i >> lg;
+      const int n = n0 + ch0;
       if (n >= p.N) continue;
-      const uint32_t laddr = smem_u32(sPack) + (uint32_t)(ch * MT + m0) * 4u;
-      int v[4] = {0, 0, 0, 0};
+      const uint32_t laddr = smem_u32(sPack) + (uint32_t)(m * SC + ch0) * 4u;
+      int v[8] = {0, 0, 0, 0, 0, 0, 0, 0};
       if (parts == 1) {
         asm volatile("ld.shared.v4.s32 {%0, %1, %2, %3}, [%4];" : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]) : "r"(laddr) : "memory");
+        asm volatile("ld.shared.v4.s32 {%0, %1, %2, %3}, [%4];" : "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]) : "r"(laddr + 16u) : "memory");
       } else {
         // all parts' loads first, then the sums: a load followed by its add would wait out one
         // remote access after the other
-        int a[8][4];
+        int a[4][8];
 #pragma unroll
-        for (int sp = 0; sp < 8; ++sp) {
-          a[sp][0] = a[sp][1] = a[sp][2] = a[sp][3] = 0;
+        for (int sp = 0; sp < 4; ++sp) {
+#pragma unroll
+          for (int t = 0; t < 8; ++t) a[sp][t] = 0;
           if (sp < parts)
             asm volatile(
                 "{\n\t.reg .b32 ra;\n\t"
-                "mapa.shared::cluster.u32 ra, %4, %5;\n\t"
-                "ld.shared::cluster.v4.s32 {%0, %1, %2, %3}, [ra];\n\t}"
-                : "=r"(a[sp][0]), "=r"(a[sp][1]), "=r"(a[sp][2]), "=r"(a[sp][3])
+                "mapa.shared::cluster.u32 ra, %8, %9;\n\t"
+                "ld.shared::cluster.v4.s32 {%0, %1, %2, %3}, [ra];\n\t"
+                "ld.shared::cluster.v4.s32 {%4, %5, %6, %7}, [ra+16];\n\t}"
+                : "=r"(a[sp][0]), "=r"(a[sp][1]), "=r"(a[sp][2]), "=r"(a[sp][3]), "=r"(a[sp][4]), "=r"(a[sp][5]), "=r"(a[sp][6]),
+                  "=r"(a[sp][7])
                 : "r"(laddr), "r"(sp));
         }
 #pragma unroll
-        for (int sp = 0; sp < 8; ++sp)
+        for (int sp = 0; sp < 4; ++sp)
 #pragma unroll
-          for (int t = 0; t < 4; ++t) v[t] += a[sp][t];
+          for (int t = 0; t < 8; ++t) v[t] += a[sp][t];
       }
-      const int cs = 2048 * s_cs[ch];
-      const float sw = s_sw[ch];
+      const float sh = s_sh[m];
+      int acc[8];
+      uint32_t o[4];
 #pragma unroll
-      for (int t = 0; t < 4; ++t) {
-        const int m = m0 + t;
-        if (m < p.M) {
-          const int acc = (v[t] - cs) >> 4;
-          p.out[(size_t)m * p.N + n] = (uint16_t)f32_to_bf16_bits(((float)acc * s_sh[m]) * sw);
-          if (p.acc_out != nullptr) p.acc_out[(size_t)m * p.N + n] = acc;
-        }
+      for (int t = 0; t < 8; ++t) acc[t] = (v[t] - 2048 * s_cs[ch0 + t]) >> 4;
+#pragma unroll
+      for (int t = 0; t < 8; t += 2)
+        o[t >> 1] = f32_to_bf16_bits(((float)acc[t] * sh) * s_sw[ch0 + t]) |
+                    (f32_to_bf16_bits(((float)acc[t + 1] * sh) * s_sw[ch0 + t + 1]) << 16);
+      *reinterpret_cast<uint4*>(p.out + (size_t)m * p.N + n) = make_uint4(o[0], o[1], o[2], o[3]);
+      if (p.acc_out != nullptr) {
+        int4* dst = reinterpret_cast<int4*>(p.acc_out + (size_t)m * p.N + n);
+        dst[0] = make_int4(acc[0], acc[1], acc[2], acc[3]);
+        dst[1] = make_int4(acc[4], acc[5], acc[6], acc[7]);
       }
     }
   }
